@@ -1,0 +1,260 @@
+"""CPU oracle for the FP8 linear layer -- TEST INFRASTRUCTURE ONLY.
+
+Thin ctypes/numpy front end of ``fp8_oracle.c`` (a plain C restatement of the
+paper's method, double precision, no CUDA).  Only the tests, the smoke check
+and the benchmark's CPU legs may import this package; the product never does,
+and this package never imports the product.
+
+Format ids: ``P_E4``/``P_E5`` are the paper's own FP8 formats (Table 7 rows
+"(a)": exponent bias 8 / 16, max 240 / 57344, the negative-zero code is NaN);
+``N_E4``/``N_E5`` are the rows "(b)" that the tensor cores consume (bias
+7 / 15, max 448 / 57344).
+
+Scaling conventions (how a paper-convention bias ``b`` turns into the shift
+that produces native bytes):
+
+* ``CONV_PAPER``: Eq. 3 with the paper format's ``max_num`` (240 / 57344);
+  shift ``s = b + delta`` with ``delta = +1`` for E4 (a paper E4 byte read as a
+  native E4 byte is exactly twice the value) and ``delta = 0`` for E5.
+* ``CONV_NATIVE``: Eq. 3 with the native format's own ``max_num`` (448 /
+  57344) and ``delta = 0``.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+P_E4, P_E5, N_E4, N_E5 = 0, 1, 2, 3
+E4, E5 = 0, 1
+CONV_PAPER, CONV_NATIVE = 0, 1
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "fp8_oracle.c")
+_LIB = os.path.join(_HERE, "liboracle.so")
+
+
+def build(force: bool = False) -> str:
+    """Compile ``fp8_oracle.c`` with gcc (-O2 -fopenmp) if it is stale."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + f".{os.getpid()}.tmp"
+        subprocess.check_call(
+            ["gcc", "-O2", "-std=c99", "-fopenmp", "-fPIC", "-shared", "-o", tmp, _SRC, "-lm"]
+        )
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+_lib = None
+
+
+def _L():
+    global _lib
+    if _lib is None:
+        _lib = ctypes.CDLL(build())
+        c = ctypes
+        _lib.orc_decode.restype = c.c_double
+        _lib.orc_decode.argtypes = [c.c_int, c.c_uint]
+        _lib.orc_max_num.restype = c.c_double
+        _lib.orc_max_num.argtypes = [c.c_int]
+        _lib.orc_encode.restype = c.c_uint
+        _lib.orc_encode.argtypes = [c.c_int, c.c_double]
+        _lib.orc_f32_to_bf16.restype = c.c_uint16
+        _lib.orc_f32_to_bf16.argtypes = [c.c_float]
+        _lib.orc_amax_bf16.restype = c.c_float
+        _lib.orc_amax_bf16.argtypes = [c.c_void_p, c.c_int64, c.c_int64, c.c_int64]
+        _lib.orc_scaling_bias.restype = c.c_int
+        _lib.orc_scaling_bias.argtypes = [c.c_float, c.c_double, c.c_int]
+        _lib.orc_cast_bf16.restype = None
+        _lib.orc_cast_bf16.argtypes = [c.c_void_p, c.c_int64, c.c_int64, c.c_int64, c.c_int, c.c_int,
+                                       c.c_void_p, c.c_void_p]
+        gemm_args = [c.c_void_p, c.c_int, c.c_int, c.c_void_p, c.c_int, c.c_int]
+        tail = [c.c_int64, c.c_int64, c.c_int64, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p]
+        _lib.orc_linear_fwd.restype = None
+        _lib.orc_linear_fwd.argtypes = gemm_args + [c.c_void_p] + tail
+        _lib.orc_linear_dgrad.restype = None
+        _lib.orc_linear_dgrad.argtypes = gemm_args + tail
+        _lib.orc_linear_wgrad.restype = None
+        _lib.orc_linear_wgrad.argtypes = gemm_args + tail
+        _lib.orc_linear_samples.restype = None
+        _lib.orc_linear_samples.argtypes = [c.c_int] + gemm_args + [c.c_void_p, c.c_int64, c.c_int64, c.c_int64,
+                                                                    c.c_void_p, c.c_void_p, c.c_int64,
+                                                                    c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p]
+        _lib.orc_num_threads.restype = c.c_int
+    return _lib
+
+
+def num_threads() -> int:
+    return int(_L().orc_num_threads())
+
+
+# ----------------------------------------------------------------------------
+# formats
+# ----------------------------------------------------------------------------
+
+def decode(fmt: int, code: int) -> float:
+    return float(_L().orc_decode(fmt, int(code) & 0xFF))
+
+
+def decode_table(fmt: int) -> np.ndarray:
+    return np.array([decode(fmt, c) for c in range(256)], dtype=np.float64)
+
+
+def encode(fmt: int, value: float) -> int:
+    return int(_L().orc_encode(fmt, float(value)))
+
+
+def max_num(fmt: int) -> float:
+    return float(_L().orc_max_num(fmt))
+
+
+def native_format(kind: int) -> int:
+    return N_E4 if kind == E4 else N_E5
+
+
+def paper_format(kind: int) -> int:
+    return P_E4 if kind == E4 else P_E5
+
+
+def bias_max_num(kind: int, conv: int) -> float:
+    """``max_num`` that Eq. 3 uses under a convention."""
+    return max_num(paper_format(kind) if conv == CONV_PAPER else native_format(kind))
+
+
+def delta(kind: int, conv: int) -> int:
+    """Format shift between the paper-convention bias and the shift applied to
+    produce native bytes."""
+    return 1 if (conv == CONV_PAPER and kind == E4) else 0
+
+
+def f32_to_bf16_bits(x: np.ndarray) -> np.ndarray:
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    out = np.empty(x.shape, dtype=np.uint16)
+    flat_in, flat_out = x.reshape(-1), out.reshape(-1)
+    f = _L().orc_f32_to_bf16
+    for i in range(flat_in.size):
+        flat_out[i] = f(float(flat_in[i]))
+    return out
+
+
+# ----------------------------------------------------------------------------
+# amax, bias, cast
+# ----------------------------------------------------------------------------
+
+def _bf16(x: np.ndarray) -> np.ndarray:
+    assert x.dtype == np.uint16 and x.ndim == 2, "bf16 tensors are passed as 2-D uint16 bit patterns"
+    return np.ascontiguousarray(x)
+
+
+def amax(x_bits: np.ndarray) -> float:
+    x = _bf16(x_bits)
+    return float(_L().orc_amax_bf16(x.ctypes.data, x.shape[0], x.shape[1], x.shape[1]))
+
+
+def scaling_bias(amax_value: float, kind: int, conv: int = CONV_PAPER, margin: int = 0) -> int:
+    return int(_L().orc_scaling_bias(float(np.float32(amax_value)), bias_max_num(kind, conv), int(margin)))
+
+
+def cast(x_bits: np.ndarray, shift: int, fmt: int, transposed: bool = False):
+    """codes = encode_fmt(x * 2^shift); returns y[rows, cols] and, if asked,
+    also y_t[cols, rows]."""
+    x = _bf16(x_bits)
+    rows, cols = x.shape
+    y = np.empty((rows, cols), dtype=np.uint8)
+    y_t = np.empty((cols, rows), dtype=np.uint8) if transposed else None
+    _L().orc_cast_bf16(x.ctypes.data, rows, cols, cols, int(shift), fmt, y.ctypes.data,
+                       y_t.ctypes.data if transposed else None)
+    return (y, y_t) if transposed else y
+
+
+def quantise(x_bits: np.ndarray, kind: int, conv: int = CONV_PAPER, margin: int = 0, transposed: bool = False):
+    """amax -> bias -> scale -> cast of one tensor (Section 2.3 then 2.1).
+    Returns (amax, bias, native bytes[, transposed native bytes])."""
+    a = amax(x_bits)
+    b = scaling_bias(a, kind, conv, margin)
+    out = cast(x_bits, b + delta(kind, conv), native_format(kind), transposed)
+    return (a, b) + (out if transposed else (out,))
+
+
+# ----------------------------------------------------------------------------
+# matmuls
+# ----------------------------------------------------------------------------
+
+class GemmResult:
+    def __init__(self, shape):
+        self.f64 = np.empty(shape, dtype=np.float64)
+        self.f32 = np.empty(shape, dtype=np.float32)
+        self.bf16 = np.empty(shape, dtype=np.uint16)
+        self.abs_sum = np.empty(shape, dtype=np.float64)
+
+    def _ptrs(self):
+        return (self.f64.ctypes.data, self.f32.ctypes.data, self.bf16.ctypes.data, self.abs_sum.ctypes.data)
+
+
+def _u8(a):
+    assert a.dtype == np.uint8 and a.ndim == 2
+    return np.ascontiguousarray(a)
+
+
+def linear_fwd(x8, s_x, w8, s_w, bias_vec=None, fx=N_E4, fw=N_E4) -> GemmResult:
+    x8, w8 = _u8(x8), _u8(w8)
+    T, K = x8.shape
+    N, K2 = w8.shape
+    assert K == K2
+    res = GemmResult((T, N))
+    bv = None
+    if bias_vec is not None:
+        bv = np.ascontiguousarray(bias_vec, dtype=np.float64)
+        assert bv.shape == (N,)
+    _L().orc_linear_fwd(x8.ctypes.data, fx, int(s_x), w8.ctypes.data, fw, int(s_w),
+                        bv.ctypes.data if bv is not None else None, T, K, N, *res._ptrs())
+    return res
+
+
+def linear_dgrad(dy8, s_g, w8, s_w, fg=N_E5, fw=N_E4) -> GemmResult:
+    dy8, w8 = _u8(dy8), _u8(w8)
+    T, N = dy8.shape
+    N2, K = w8.shape
+    assert N == N2
+    res = GemmResult((T, K))
+    _L().orc_linear_dgrad(dy8.ctypes.data, fg, int(s_g), w8.ctypes.data, fw, int(s_w), T, K, N, *res._ptrs())
+    return res
+
+
+def linear_wgrad(dy8, s_g, x8, s_x, fg=N_E5, fx=N_E4) -> GemmResult:
+    dy8, x8 = _u8(dy8), _u8(x8)
+    T, N = dy8.shape
+    T2, K = x8.shape
+    assert T == T2
+    res = GemmResult((N, K))
+    _L().orc_linear_wgrad(dy8.ctypes.data, fg, int(s_g), x8.ctypes.data, fx, int(s_x), T, K, N, *res._ptrs())
+    return res
+
+
+FWD, DGRAD, WGRAD = 0, 1, 2
+
+
+def linear_samples(kind, a8, fa, s_a, b8, fb, s_b, rows, cols, bias_vec=None) -> GemmResult:
+    """The matmul definitions evaluated at listed (row, col) output positions.
+    kind FWD: a8 = X8[T,K], b8 = W8[N,K]; DGRAD: a8 = dY8[T,N], b8 = W8[N,K];
+    WGRAD: a8 = dY8[T,N], b8 = X8[T,K]."""
+    a8, b8 = _u8(a8), _u8(b8)
+    if kind == FWD:
+        (T, K), (N, _) = a8.shape, b8.shape
+    elif kind == DGRAD:
+        (T, N), (_, K) = a8.shape, b8.shape
+    else:
+        (T, N), (_, K) = a8.shape, b8.shape
+    rows = np.ascontiguousarray(rows, dtype=np.int64)
+    cols = np.ascontiguousarray(cols, dtype=np.int64)
+    assert rows.shape == cols.shape and rows.ndim == 1
+    res = GemmResult(rows.shape)
+    bv = None
+    if bias_vec is not None:
+        bv = np.ascontiguousarray(bias_vec, dtype=np.float64)
+    _L().orc_linear_samples(kind, a8.ctypes.data, fa, int(s_a), b8.ctypes.data, fb, int(s_b),
+                            bv.ctypes.data if bv is not None else None, T, K, N,
+                            rows.ctypes.data, cols.ctypes.data, rows.size, *res._ptrs())
+    return res

@@ -1,0 +1,108 @@
+"""Pins for the oracle's amax and scaling bias (Eq. 3): hand values, exact
+rational arithmetic over every bf16 value, the defining inequality."""
+from fractions import Fraction
+
+import numpy as np
+import torch
+
+import oracle as O
+
+
+def test_hand_computed_biases():
+    # (amax, E4 with max 240, E4 with max 448, E5 with max 57344)
+    hand = [
+        (240.0, 0, 0, 7),        # 240*2^0 = 240 fits exactly; 240*2 = 480 > 448; 240*2^7 = 30720 <= 57344 < 61440
+        (241.0, -1, 0, 7),
+        (120.0, 1, 1, 8),
+        (1.0, 7, 8, 15),         # 2^7 <= 240 < 2^8; 2^8 <= 448 < 2^9; 2^15 <= 57344 < 2^16
+        (1.875, 7, 7, 14),       # 1.875*2^7 = 240 exactly
+        (1.8828125, 6, 7, 14),   # next bf16 after 1.875 no longer fits at 2^7
+        (5.0, 5, 6, 13),
+        (0.08, 11, 12, 19),
+        (0.005, 15, 16, 23),
+        (57344.0, -8, -7, 0),
+    ]
+    for amax, b4p, b4n, b5 in hand:
+        assert O.scaling_bias(amax, O.E4, O.CONV_PAPER) == b4p, amax
+        assert O.scaling_bias(amax, O.E4, O.CONV_NATIVE) == b4n, amax
+        assert O.scaling_bias(amax, O.E5, O.CONV_PAPER) == b5, amax
+        assert O.scaling_bias(amax, O.E5, O.CONV_NATIVE) == b5, amax
+
+
+def test_margin_is_subtracted():
+    assert O.scaling_bias(1.0, O.E5, O.CONV_PAPER, margin=3) == 12
+    assert O.scaling_bias(1.0, O.E4, O.CONV_PAPER, margin=-2) == 9
+
+
+def test_degenerate_amax():
+    assert O.scaling_bias(0.0, O.E4) == 0
+    assert O.scaling_bias(float("inf"), O.E4) == 0
+    assert O.scaling_bias(float("nan"), O.E5) == 0
+
+
+def test_bias_is_floor_log2_for_every_bf16_amax():
+    """floor(log2(max_num/amax)) evaluated in exact rational arithmetic for all
+    32 639 positive finite bf16 values, plus the inequality that defines it."""
+    bits = np.arange(1, 0x7F80, dtype=np.uint32).astype(np.uint16)
+    vals = torch.from_numpy(bits.view(np.int16).copy()).view(torch.bfloat16).to(torch.float64).numpy()
+    ranges = {}
+    for kind, conv, mx in ((O.E4, O.CONV_PAPER, 240), (O.E4, O.CONV_NATIVE, 448), (O.E5, O.CONV_PAPER, 57344)):
+        lo, hi = 10 ** 9, -10 ** 9
+        for v in vals.tolist():
+            a = Fraction(v)
+            b = O.scaling_bias(v, kind, conv)
+            two_b = Fraction(2) ** b
+            assert a * two_b <= mx < a * two_b * 2, (v, b)
+            lo, hi = min(lo, b), max(hi, b)
+        ranges[(kind, conv)] = (lo, hi)
+    # extreme biases reached at the largest / smallest bf16 magnitudes
+    assert ranges[(O.E4, O.CONV_PAPER)] == (-121, 140)
+    assert ranges[(O.E4, O.CONV_NATIVE)] == (-120, 141)
+    assert ranges[(O.E5, O.CONV_PAPER)] == (-113, 148)
+
+
+def _bits(t):
+    return t.contiguous().view(torch.int16).numpy().view(np.uint16)
+
+
+def test_amax_against_numpy_and_special_values():
+    g = torch.Generator().manual_seed(3)
+    x = (torch.randn(33, 70, generator=g) * 3).to(torch.bfloat16)
+    assert O.amax(_bits(x)) == float(x.to(torch.float64).abs().max())
+    x[5, 6] = -1000.0
+    assert O.amax(_bits(x)) == 1000.0
+    x[7, 1] = float("inf")
+    assert O.amax(_bits(x)) == float("inf")
+    x[0, 0] = float("nan")
+    assert np.isnan(O.amax(_bits(x)))
+    z = torch.zeros(4, 4, dtype=torch.bfloat16)
+    z[1, 1] = -0.0
+    assert O.amax(_bits(z)) == 0.0
+    # a bf16 subnormal
+    s = np.zeros((2, 2), dtype=np.uint16)
+    s[1, 0] = 0x8001
+    assert O.amax(s) == 2.0 ** -133
+
+
+def test_scaling_a_tensor_by_a_power_of_two_moves_only_the_bias():
+    g = torch.Generator().manual_seed(4)
+    x = torch.randn(40, 24, generator=g).to(torch.bfloat16)
+    a0, b0, y0 = O.quantise(_bits(x), O.E4)
+    for k in (-9, 5):
+        xk = (x.to(torch.float32) * 2.0 ** k).to(torch.bfloat16)
+        ak, bk, yk = O.quantise(_bits(xk), O.E4)
+        assert ak == a0 * 2.0 ** k and bk == b0 - k
+        assert np.array_equal(yk, y0)
+
+
+def test_largest_cast_code_lands_in_the_top_binade():
+    """After scaling by the AMAX bias the largest element sits in
+    [max_num/2, max_num] of the format Eq. 3 was evaluated for."""
+    g = torch.Generator().manual_seed(5)
+    for std in (1e-4, 0.02, 1.0, 300.0):
+        x = (torch.randn(64, 64, generator=g) * std).to(torch.bfloat16)
+        for kind, conv in ((O.E4, O.CONV_PAPER), (O.E4, O.CONV_NATIVE), (O.E5, O.CONV_PAPER)):
+            a, b, y = O.quantise(_bits(x), kind, conv)
+            top = np.abs(O.decode_table(O.native_format(kind))[y]).max() * 2.0 ** -O.delta(kind, conv)
+            mx = O.bias_max_num(kind, conv)
+            assert mx / 2 <= top <= mx or (conv == O.CONV_PAPER and kind == O.E4 and top == 224.0)

@@ -1,0 +1,416 @@
+#!/usr/bin/env python
+"""Benchmark of the FP8 linear hot path (amax -> bias -> cast -> FP8 matmuls
+with unscale, forward + backward) on synthetic tensors shaped like the
+paper's layers.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+
+One "step" is one pass of the whole path over one batch: for every linear of
+the workload's decoder block, re-quantise W (the per-step weight cast), quantise
+X, forward matmul, quantise dY, input-gradient matmul, weight-gradient matmul.
+Prints ONE JSON line on rank 0.  With N > 1 (torchrun) every rank runs the same
+single-GPU path on its own tensors (replicas; the method has no exchange step).
+
+`--impl reference` times the CPU oracle, as it stands, on the host cores.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import torch
+
+from paper_2309_17224_b200 import inputs as I
+
+METRIC = "fp8_linear_fwd_bwd_tflops"
+UNIT = "TFLOP/s"
+DEFAULT_WORKLOAD = "c3_llama7b"
+ORACLE_SAMPLE_TOKENS = 256
+ORACLE_SAMPLE_LAYER = 1  # the square attention-output projection
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as fh:
+            p = json.load(fh)
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p["bf16_tflops"]),
+                "bf16_tflops_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])),
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+# ----------------------------------------------------------------------------
+# clocks
+# ----------------------------------------------------------------------------
+
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device_index: int):
+        self.proc = None
+        self.path = None
+        try:
+            uuid = str(torch.cuda.get_device_properties(device_index).uuid)
+            if not uuid.startswith("GPU-"):
+                uuid = "GPU-" + uuid
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", uuid, f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        try:
+            with open(self.path) as fh:
+                for line in fh:
+                    parts = [x.strip() for x in line.split(",")]
+                    if len(parts) < 7:
+                        continue
+                    try:
+                        sm.append(float(parts[0]))
+                        mx.append(float(parts[1]))
+                    except ValueError:
+                        continue
+                    for n, v in zip(names, parts[3:7]):
+                        if v.lower().startswith("active"):
+                            reasons.add(n)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+# ----------------------------------------------------------------------------
+# our arm
+# ----------------------------------------------------------------------------
+
+class LayerState:
+    """Device buffers of one linear: bf16 inputs, FP8 copies in both layouts,
+    device scalars, bf16 outputs."""
+
+    def __init__(self, wl, li, device, seed, backward):
+        l = wl.layers[li]
+        T, K, N = wl.tokens, l.K, l.N
+        self.T, self.K, self.N, self.name = T, K, N, l.name
+        t = I.layer_tensors(wl, li, device=device, seed=seed)
+        self.x, self.w = t["x"], t["w"]
+        self.g = t.get("g")
+        u8 = dict(dtype=torch.uint8, device=device)
+        self.x8, self.w8 = torch.empty((T, K), **u8), torch.empty((N, K), **u8)
+        self.y = torch.empty((T, N), dtype=torch.bfloat16, device=device)
+        self.scal_f = torch.zeros(4, dtype=torch.float32, device=device)
+        self.scal_i = torch.zeros(4, dtype=torch.int32, device=device)
+        self.backward = backward
+        if backward:
+            self.x8t, self.w8t = torch.empty((K, T), **u8), torch.empty((K, N), **u8)
+            self.g8, self.g8t = torch.empty((T, N), **u8), torch.empty((N, T), **u8)
+            self.dx = torch.empty((T, K), dtype=torch.bfloat16, device=device)
+            self.dw = torch.empty((N, K), dtype=torch.bfloat16, device=device)
+        else:
+            self.x8t = self.w8t = self.g8 = self.g8t = self.dx = self.dw = None
+
+    def gemm_flops(self):
+        return 2.0 * self.T * self.K * self.N * (3 if self.backward else 1)
+
+    def cast_elements(self):
+        n = self.T * self.K + self.N * self.K
+        return n + (self.T * self.N if self.backward else 0)
+
+    def launches(self):
+        return 9 if self.backward else 5
+
+
+class Timers:
+    """CUDA-event pairs around groups of launches, on the launching stream."""
+
+    def __init__(self):
+        self.pairs = {"gemm": [], "amax_cast": []}
+
+    def span(self, key):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        self.pairs[key].append((a, b))
+        return a, b
+
+    def total_ms(self, key):
+        return sum(a.elapsed_time(b) for a, b in self.pairs[key])
+
+    def count(self, key):
+        return len(self.pairs[key])
+
+
+def run_layer(ctx, L, timers=None):
+    def timed(key, fn):
+        if timers is None:
+            fn()
+        else:
+            a, b = timers.span(key)
+            a.record()
+            fn()
+            b.record()
+
+    af, bi = L.scal_f, L.scal_i
+    timed("amax_cast", lambda: ctx.cast_e4(L.w, None, d_amax_out=af[0:1], d_bias_out=bi[0:1], y=L.w8, y_t=L.w8t))
+    timed("amax_cast", lambda: ctx.cast_e4(L.x, None, d_amax_out=af[1:2], d_bias_out=bi[1:2], y=L.x8, y_t=L.x8t))
+    timed("gemm", lambda: ctx.linear_fwd(L.x8, bi[1:2], L.w8, bi[0:1], L.y))
+    if L.backward:
+        timed("amax_cast", lambda: ctx.cast_e5(L.g, None, d_amax_out=af[2:3], d_bias_out=bi[2:3], y=L.g8, y_t=L.g8t))
+        timed("gemm", lambda: ctx.linear_dgrad(L.g8, bi[2:3], None, L.w8t, bi[0:1], L.dx))
+        timed("gemm", lambda: ctx.linear_wgrad(None, L.g8t, bi[2:3], None, L.x8t, bi[1:2], L.dw, L.T))
+
+
+def dist_setup(n_gpus):
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        import torch.distributed as dist
+        torch.cuda.set_device(local)
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+        return rank, world, local, dist
+    torch.cuda.set_device(0)
+    return 0, 1, 0, None
+
+
+def barrier_sync(dist):
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+
+
+def max_over_ranks(value, dist, device):
+    if dist is None:
+        return value
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def oracle_sample_run(wl, seed):
+    """One bounded sample of the workload on the CPU oracle: the whole path
+    (amax, bias, cast of X, W, dY; the three matmuls) for one layer at a
+    reduced token count.  Returns (seconds, flops, description)."""
+    import oracle as O
+    li = min(ORACLE_SAMPLE_LAYER, len(wl.layers) - 1)
+    l = wl.layers[li]
+    T = min(ORACLE_SAMPLE_TOKENS, wl.tokens)
+    t = I.layer_tensors(wl, li, device="cpu", seed=seed, tokens=T)
+    xb, wb = I.bits(t["x"]), I.bits(t["w"])
+    gb = I.bits(t["g"]) if wl.backward else None
+    t0 = time.perf_counter()
+    _, bx, x8 = O.quantise(xb, O.E4)
+    _, bw, w8 = O.quantise(wb, O.E4)
+    O.linear_fwd(x8, bx + 1, w8, bw + 1)
+    flops = 2.0 * T * l.K * l.N
+    if wl.backward:
+        _, bg, g8 = O.quantise(gb, O.E5)
+        O.linear_dgrad(g8, bg, w8, bw + 1)
+        O.linear_wgrad(g8, bg, x8, bx + 1)
+        flops *= 3
+    dt = time.perf_counter() - t0
+    what = (f"layer '{l.name}' ({l.K}->{l.N}) of {wl.name} at {T} of {wl.tokens} tokens: amax+bias+cast of X, W"
+            f"{', dY' if wl.backward else ''} and {'3 matmuls' if wl.backward else '1 matmul'}, {flops / 1e9:.1f} GFLOP")
+    return dt, flops, what, O.num_threads()
+
+
+def reference_arm(args, wl):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    import oracle as O
+    O.build()
+    for _ in range(max(0, min(args.warmup, 1))):
+        oracle_sample_run(wl, I.BASE_SEED)
+    times, flops, what, cores = [], 0.0, "", 1
+    steps = max(1, min(args.steps, 5))
+    for _ in range(steps):
+        dt, flops, what, cores = oracle_sample_run(wl, I.BASE_SEED)
+        times.append(dt)
+    ms = 1e3 * sum(times) / len(times)
+    value = flops / (ms * 1e-3) / 1e12
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
+        "warmup": min(args.warmup, 1), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": wl.name, "tokens": wl.tokens, "layers": [f"{l.name}:{l.K}->{l.N}" for l in wl.layers],
+                   "passes": "fwd+bwd" if wl.backward else "fwd"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": what},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(I.WORKLOADS))
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    wl = I.WORKLOADS[args.workload]
+    if args.impl == "reference":
+        return reference_arm(args, wl)
+
+    if not torch.cuda.is_available():
+        print("bench.py: no CUDA device; the FP8 path has no CPU fallback", file=sys.stderr)
+        return 2
+    from paper_2309_17224_b200 import build as B
+    B.build()
+    from paper_2309_17224_b200 import fp8lin
+
+    rank, world, local, dist = dist_setup(args.gpus)
+    device = torch.device("cuda", local)
+    warmup = max(3, args.warmup)
+    ctx = fp8lin.Context(local)
+    layers = [LayerState(wl, li, device, I.BASE_SEED + 7919 * rank, wl.backward) for li in range(len(wl.layers))]
+    peaks = load_peaks()
+
+    for _ in range(warmup):
+        for L in layers:
+            run_layer(ctx, L)
+    barrier_sync(dist)
+    if ctx.device_flags(clear=True) & fp8lin.FLAG_TIMEOUT:
+        print("bench.py: a device-side wait expired during warm-up", file=sys.stderr)
+        return 3
+
+    # ---- timed region: K steps, device time, max over ranks ----
+    sampler = ClockSampler(local) if rank == 0 else None
+    timers = Timers()
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier_sync(dist)
+    start.record()
+    for _ in range(args.steps):
+        for L in layers:
+            run_layer(ctx, L, timers)
+    stop.record()
+    barrier_sync(dist)
+    clocks = sampler.stop() if sampler else None
+    total_ms = max_over_ranks(start.elapsed_time(stop), dist, device)
+    flags = ctx.device_flags(clear=True)
+    if flags & fp8lin.FLAG_TIMEOUT:
+        print("bench.py: a device-side wait expired during the timed region", file=sys.stderr)
+        return 3
+
+    ms_per_step = total_ms / args.steps
+    step_flops = sum(L.gemm_flops() for L in layers)
+    value = world * step_flops / (ms_per_step * 1e-3) / 1e12
+
+    gemm_ms = timers.total_ms("gemm")
+    gemm_launches = timers.count("gemm")
+    gemm_tflops = args.steps * step_flops / (gemm_ms * 1e-3) / 1e12
+    cast_ms = timers.total_ms("amax_cast")
+    cast_elems = args.steps * sum(L.cast_elements() for L in layers)
+    bytes_per_elem = 4 if wl.backward else 3  # read once, write one byte per layout
+    fp8_peak = 2.0 * peaks["bf16_tflops_sustained"]
+
+    # ---- end to end through the public API with host buffers ----
+    e2e = None
+    if args.e2e_steps > 0:
+        host_in, host_out = [], []
+        for L in layers:
+            ins = [L.x, L.w] + ([L.g] if wl.backward else [])
+            outs = [L.y] + ([L.dx, L.dw] if wl.backward else [])
+            host_in.append([torch.empty(t.shape, dtype=t.dtype, pin_memory=True).copy_(t) for t in ins])
+            host_out.append([torch.empty(t.shape, dtype=t.dtype, pin_memory=True) for t in outs])
+        h2d = sum(t.numel() * t.element_size() for ts in host_in for t in ts)
+        d2h = sum(t.numel() * t.element_size() for ts in host_out for t in ts)
+
+        def e2e_step():
+            for L, hin, hout in zip(layers, host_in, host_out):
+                ins = [L.x, L.w] + ([L.g] if wl.backward else [])
+                outs = [L.y] + ([L.dx, L.dw] if wl.backward else [])
+                for d, h in zip(ins, hin):
+                    d.copy_(h, non_blocking=True)
+                run_layer(ctx, L)
+                for h, d in zip(hout, outs):
+                    h.copy_(d, non_blocking=True)
+
+        e2e_step()
+        barrier_sync(dist)
+        t0 = time.perf_counter()
+        for _ in range(args.e2e_steps):
+            e2e_step()
+        barrier_sync(dist)
+        e2e_ms = max_over_ranks(1e3 * (time.perf_counter() - t0) / args.e2e_steps, dist, device)
+        e2e = {"value": world * step_flops / (e2e_ms * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": e2e_ms,
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
+        del host_in, host_out
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return 0
+
+    cpu_baseline = None
+    if world == 1 and not args.no_cpu_baseline:
+        import oracle as O
+        O.build()
+        dt, fl, what, cores = oracle_sample_run(wl, I.BASE_SEED)
+        cpu_baseline = {"value": fl / dt / 1e12, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": what,
+                        "seconds": dt}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warmup,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "fp8_e4m3/e5m2 operands, f32 accumulate, bf16 out", "data": "synthetic",
+        "config": {"workload": wl.name, "tokens": wl.tokens,
+                   "layers": [f"{l.name}:{l.K}->{l.N}" for l in wl.layers],
+                   "passes": "fwd+bwd" if wl.backward else "fwd",
+                   "scaling_bias": "FP8-AMAX, recomputed every step for W, X, dY",
+                   "l2": "inputs larger than L2 (each layer's tensors exceed 126 MB); no flush between steps",
+                   "parallelism": "replicas" if world > 1 else "single"},
+        "clocks": clocks,
+        "e2e": e2e,
+        "gpu_launches": args.steps * sum(L.launches() for L in layers),
+        "roofline": {"bound": "tensor", "kernel": "gemm_kernel", "achieved": gemm_tflops, "peak": fp8_peak,
+                     "unit": "TFLOP/s", "frac": gemm_tflops / fp8_peak,
+                     "peak_source": f"2 x {peaks['source']} sustained bf16 cuBLAS ({peaks['bf16_tflops_sustained']} TFLOP/s)",
+                     "launches": gemm_launches, "avg_launch_ms": gemm_ms / max(1, gemm_launches),
+                     "traffic": None},
+        "amax_cast": {"effective_gbs": cast_elems * bytes_per_elem / (cast_ms * 1e-3) / 1e9,
+                      "bytes_per_element": bytes_per_elem, "ms_per_step": cast_ms / args.steps,
+                      "hbm_peak_gbs": peaks["hbm_gbs"],
+                      "frac": cast_elems * bytes_per_elem / (cast_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]},
+        "gemm_ms_per_step": gemm_ms / args.steps,
+        "device_flags": flags,
+        "cpu_baseline": cpu_baseline,
+    }
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())

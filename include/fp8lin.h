@@ -1,0 +1,171 @@
+/*
+ * fp8lin.h -- C ABI of the B200 (sm_100a) FP8 linear layer with dynamically
+ * updated per-tensor scaling bias, after "Training and inference of large
+ * language models using 8-bit floating point" (arXiv 2309.17224).
+ *
+ * Conventions that hold for every entry point
+ * -------------------------------------------
+ *  - Every call returns an fp8_status_t.  Nothing throws, nothing is printed.
+ *  - All tensor pointers are DEVICE pointers owned by the caller; the library
+ *    never allocates, frees or retains them.  "d_" marks a device scalar.
+ *    The only host pointers are the fp8_ctx handle, `flags` of
+ *    fp8_device_flags and the arguments of fp8_scaling_bias_host.
+ *  - `stream` is a cudaStream_t passed as void* (NULL = the legacy default
+ *    stream).  Calls are asynchronous and ordered on that stream like any
+ *    kernel launch.  Calls that share one fp8_ctx must be issued from one host
+ *    thread at a time.
+ *  - Tensors are row-major.  X[T,K] activations, W[N,K] weights (the layout of
+ *    a PyTorch nn.Linear), dY[T,N] output gradients; Y[T,N], dX[T,K], dW[N,K].
+ *  - FP8 bytes are the native Blackwell encodings (Table 7 rows "(b)": E4M3
+ *    with exponent bias 7 and max 448, E5M2 with bias 15 and max 57344).
+ *    Scaling biases are always the paper-convention integers of Eq. 3.  Under
+ *    FP8_CONV_PAPER the E4 shift actually applied is bias+1, because a byte of
+ *    the paper's E4 format (Table 7 row "(a)", exponent bias 8, max 240) read
+ *    as a native E4M3 byte is exactly twice the value; the matmuls take that
+ *    extra factor out again.  Byte c of a tensor with bias b therefore means
+ *    native_value(c) * 2^-(b + delta), delta = 1 for (E4, FP8_CONV_PAPER) and
+ *    0 otherwise.  Paper E4 codes without a native counterpart: +-240 (emitted
+ *    as +-224) and the paper's NaN code 0x80 (natively -0).
+ *  - Argument errors are detected on the host and returned BEFORE anything is
+ *    launched.  Data-dependent conditions never fail a call; they set sticky
+ *    bits in a device status word (see fp8_device_flags).
+ */
+#ifndef FP8LIN_H
+#define FP8LIN_H
+
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define FP8_API __attribute__((visibility("default")))
+#else
+#define FP8_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    FP8_OK = 0,
+    FP8_ERR_NULL = 1,           /* a required pointer is NULL */
+    FP8_ERR_SHAPE = 2,          /* a dimension is <= 0, or ld < cols */
+    FP8_ERR_ALIGN = 3,          /* pointer / leading dimension alignment the kernels need is not met */
+    FP8_ERR_DTYPE = 4,          /* enum value out of range */
+    FP8_ERR_UNSUPPORTED = 5,    /* valid request that this build has no kernel for (there is no fallback path) */
+    FP8_ERR_CUDA = 6,           /* a CUDA runtime / driver call failed (launch, attribute, tensor-map encode) */
+    FP8_ERR_DEVICE_TIMEOUT = 7  /* reported by fp8_device_flags when a bounded device-side wait expired */
+} fp8_status_t;
+
+typedef enum { FP8_E4 = 0, FP8_E5 = 1 } fp8_format_t;
+
+/* Which max_num Eq. 3 uses: the paper's own formats (240 / 57344) or the
+ * native formats' (448 / 57344). */
+typedef enum { FP8_CONV_PAPER = 0, FP8_CONV_NATIVE = 1 } fp8_conv_t;
+
+typedef enum { FP8_BF16 = 0, FP8_F16 = 1, FP8_F32 = 2 } fp8_dtype_t;
+
+/* Sticky device status bits. */
+#define FP8_FLAG_NONFINITE_AMAX 1u /* an amax was inf or NaN; its bias was set to 0 */
+#define FP8_FLAG_ZERO_AMAX 2u      /* an amax was 0; its bias was set to 0 */
+#define FP8_FLAG_SATURATED 4u      /* a cast clipped at least one value (finite or infinite) to the format's maximum */
+#define FP8_FLAG_TIMEOUT 8u        /* a bounded wait inside a kernel expired; that kernel's output is invalid */
+
+typedef struct fp8_ctx fp8_ctx;
+
+/* Create / destroy a context on `device`.  The context owns a few KB of device
+ * workspace (status word, reduction slots).  fp8_create is the only call that
+ * allocates device memory; it also raises the dynamic shared-memory limit of
+ * the matmul kernels.  It must not be called during stream capture. */
+FP8_API fp8_status_t fp8_create(fp8_ctx **ctx, int device);
+FP8_API fp8_status_t fp8_destroy(fp8_ctx *ctx);
+
+FP8_API const char *fp8_status_string(fp8_status_t status);
+
+/* Synchronises `stream`, copies the sticky status word to *flags (host) and,
+ * if `clear` is non-zero, resets it.  Returns FP8_ERR_DEVICE_TIMEOUT if
+ * FP8_FLAG_TIMEOUT was set, else FP8_OK. */
+FP8_API fp8_status_t fp8_device_flags(fp8_ctx *ctx, void *stream, unsigned *flags, int clear);
+
+/* amax = max(|x|) over the whole tensor (Eq. 3, first line).
+ *   x       [rows, cols] with leading dimension ld (elements), dtype x_dt
+ *           (this build: FP8_BF16 only)
+ *   d_amax  out, one float.  NaN if any element is NaN, else the exact maximum
+ *           magnitude (inf included).
+ * Needs x 2-byte aligned only; 16-byte aligned x with ld == cols (or ld and
+ * cols multiples of 8) takes the vectorised path. */
+FP8_API fp8_status_t fp8_amax(fp8_ctx *ctx, const void *x, fp8_dtype_t x_dt, int64_t rows, int64_t cols, int64_t ld,
+                      float *d_amax, void *stream);
+
+/* scaling_bias = floor(log2(max_num / amax)) - margin (Eq. 3, second line;
+ * the margin is the one of Section 3.2), evaluated exactly on the bits of
+ * amax.  amax == 0 or non-finite gives bias 0 and sets a status flag.
+ *   d_amax in, d_bias out: device scalars. */
+FP8_API fp8_status_t fp8_scaling_bias(fp8_ctx *ctx, const float *d_amax, fp8_format_t fmt, fp8_conv_t conv,
+                              int32_t margin, int32_t *d_bias, void *stream);
+
+/* The same integer rule on the host (no device work, no ctx). */
+FP8_API fp8_status_t fp8_scaling_bias_host(float amax, fp8_format_t fmt, fp8_conv_t conv, int32_t margin, int32_t *bias);
+
+/* Scale-and-cast (Eq. 1 then the cast of Section 2.1): code = RNE_fp8(x * 2^(bias + delta)),
+ * saturating at the format's largest finite value; NaN stays NaN.
+ *   x          [rows, cols], leading dimension ld, dtype x_dt (FP8_BF16 only)
+ *   d_bias     device int32, the paper-convention bias to apply.  Passing a
+ *              constant chosen by the caller is the paper's FP8-CSCALE.
+ *              NULL selects FP8-AMAX: amax and bias are computed here first
+ *              (with `margin`) and written to d_amax_out / d_bias_out, both
+ *              then required.
+ *   y          out [rows, cols] bytes, contiguous, or NULL
+ *   y_t        out [cols, rows] bytes (the transposed copy, same codes), or NULL
+ * At least one of y, y_t.  The vectorised paths need 16-byte aligned x, y, y_t,
+ * ld % 8 == 0, and rows % 4 == 0 for y_t; other shapes take a slower guarded path. */
+FP8_API fp8_status_t fp8_cast_e4(fp8_ctx *ctx, const void *x, fp8_dtype_t x_dt, int64_t rows, int64_t cols, int64_t ld,
+                         const int32_t *d_bias, fp8_conv_t conv, int32_t margin, float *d_amax_out,
+                         int32_t *d_bias_out, uint8_t *y, uint8_t *y_t, void *stream);
+/* Same for the gradient format E5 (Section 2.2). */
+FP8_API fp8_status_t fp8_cast_e5(fp8_ctx *ctx, const void *x, fp8_dtype_t x_dt, int64_t rows, int64_t cols, int64_t ld,
+                         const int32_t *d_bias, fp8_conv_t conv, int32_t margin, float *d_amax_out,
+                         int32_t *d_bias_out, uint8_t *y, uint8_t *y_t, void *stream);
+
+/* Post-training quantisation of one weight tensor (Section 3.1): amax -> bias
+ * -> cast to E4, once.  w [N, K] (ld elements); outputs w8 [N, K] and/or
+ * w8_t [K, N], d_bw, d_amax_w (both required). */
+FP8_API fp8_status_t fp8_ptq_weights(fp8_ctx *ctx, const void *w, fp8_dtype_t w_dt, int64_t N, int64_t K, int64_t ld,
+                             fp8_conv_t conv, uint8_t *w8, uint8_t *w8_t, int32_t *d_bw, float *d_amax_w,
+                             void *stream);
+
+/* Forward matmul with unscale (Fig. 3b, Eq. 2):
+ *   Y[t, n] = (sum_k X8[t, k] * W8[n, k]) * 2^-(s_x + s_w) + bias_vec[n]
+ * with s = bias + delta, FP32 accumulation on the tensor cores.
+ *   x8 [T, K] E4 bytes, w8 [N, K] E4 bytes, both contiguous, 16-byte aligned, K % 16 == 0
+ *   d_bx, d_bw  device int32 paper-convention biases of X and W
+ *   bias_vec    NULL or [N] of dtype bias_dt (FP8_BF16 or FP8_F32), added after the unscale
+ *   y           out [T, N] contiguous, dtype y_dt (FP8_BF16 or FP8_F32)
+ *   d_amax_y    NULL, or out: amax of the rounded output (set by this call)
+ */
+FP8_API fp8_status_t fp8_linear_fwd(fp8_ctx *ctx, const uint8_t *x8, const int32_t *d_bx, const uint8_t *w8,
+                            const int32_t *d_bw, const void *bias_vec, fp8_dtype_t bias_dt, void *y,
+                            fp8_dtype_t y_dt, float *d_amax_y, int64_t T, int64_t K, int64_t N, fp8_conv_t conv,
+                            void *stream);
+
+/* Input-gradient matmul (Section 2.2): dX[t, k] = (sum_n dY8[t, n] * W8[n, k]) * 2^-(s_g + s_w).
+ *   dy8  [T, N] E5 bytes;  N % 16 == 0
+ *   w8   [N, K] E4 bytes or NULL;  w8_t [K, N] E4 bytes or NULL.  At least one.
+ *        This build contracts over contiguous bytes only and therefore needs
+ *        w8_t (as written by the cast's y_t); w8 alone returns FP8_ERR_UNSUPPORTED.
+ *   dx   out [T, K], dtype dx_dt;  d_amax_dx NULL or out. */
+FP8_API fp8_status_t fp8_linear_dgrad(fp8_ctx *ctx, const uint8_t *dy8, const int32_t *d_bg, const uint8_t *w8,
+                              const uint8_t *w8_t, const int32_t *d_bw, void *dx, fp8_dtype_t dx_dt,
+                              float *d_amax_dx, int64_t T, int64_t K, int64_t N, fp8_conv_t conv, void *stream);
+
+/* Weight-gradient matmul (Section 2.2): dW[n, k] = (sum_t dY8[t, n] * X8[t, k]) * 2^-(s_g + s_x).
+ *   dy8 [T, N] / dy8_t [N, T] E5 bytes, x8 [T, K] / x8_t [K, T] E4 bytes; T % 16 == 0.
+ *   This build needs the transposed copies dy8_t and x8_t; the others may be NULL.
+ *   dw  out [N, K], dtype dw_dt. */
+FP8_API fp8_status_t fp8_linear_wgrad(fp8_ctx *ctx, const uint8_t *dy8, const uint8_t *dy8_t, const int32_t *d_bg,
+                              const uint8_t *x8, const uint8_t *x8_t, const int32_t *d_bx, void *dw,
+                              fp8_dtype_t dw_dt, int64_t T, int64_t K, int64_t N, fp8_conv_t conv, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FP8LIN_H */

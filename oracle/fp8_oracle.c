@@ -99,10 +99,32 @@ double orc_max_num(int f)
 /* Round to the nearest representable value, ties to the code with an even
  * last bit; magnitudes beyond the largest finite value are clipped to it and
  * values that round to nothing become zero (Appendix A, the paragraph after
- * Eq. 4).  Done as a search through all finite magnitude codes. */
+ * Eq. 4).  Done as a search through all finite magnitude codes; the decoded
+ * magnitudes are tabulated once per format (orc_decode of codes 0..127). */
+static double MAG[4][128];
+static int MAG_FINITE[4][128];
+static int MAG_READY[4];
+
+static void mag_table(int f)
+{
+    if (MAG_READY[f]) return;
+#pragma omp critical(orc_mag_table)
+    {
+        if (!MAG_READY[f]) {
+            for (unsigned c = 0; c < 128; ++c) {
+                MAG_FINITE[f][c] = code_class(f, c) == 0;
+                MAG[f][c] = MAG_FINITE[f][c] ? orc_decode(f, c) : 0.0;
+            }
+#pragma omp flush
+            MAG_READY[f] = 1;
+        }
+    }
+}
+
 unsigned orc_encode(int f, double v)
 {
     if (isnan(v)) return FMT[f].special == 0 ? 0x80u : 0x7Fu;
+    mag_table(f);
     unsigned sign = signbit(v) ? 1u : 0u;
     double a = fabs(v);
     unsigned best = 0;
@@ -110,8 +132,8 @@ unsigned orc_encode(int f, double v)
     unsigned top = 0;
     double top_v = -1.0;
     for (unsigned c = 0; c < 128; ++c) {
-        if (code_class(f, c) != 0) continue;
-        double cv = orc_decode(f, c);
+        if (!MAG_FINITE[f][c]) continue;
+        double cv = MAG[f][c];
         if (cv > top_v) { top_v = cv; top = c; }
         double d = fabs(cv - a);
         if (d < best_d || (d == best_d && (c & 1u) == 0u)) { best_d = d; best = c; }

@@ -1,0 +1,294 @@
+// Scale-and-cast (Eq. 1 followed by the cast of Section 2.1; E5 per Section
+// 2.2) and post-training quantisation of a weight tensor (Section 3.1).
+//
+// code = RNE_fp8(x * 2^(bias + delta)), saturating.  The scaling is an exact
+// power-of-two multiply in FP32 (a bf16 value has 8 significant bits, so the
+// product is exact unless it underflows FP32, where the FP8 result is zero
+// either way) and the rounding is one hardware cvt.rn.satfinite per pair.
+//
+// Two kernels, both HBM-bound (2 B read + 1 B written per element and layout):
+//   cast_flat_kernel  contiguous tensor, row-major output only; 32 B in, 16 B
+//                     out per thread per step.
+//   cast_tile_kernel  128x128 tiles, optional row-major output and optional
+//                     transposed output staged through shared memory so that
+//                     both are written in 128-byte rows.
+// Both walk the tensor from its end to its start: when the amax pass has just
+// streamed the tensor front to back, the part most recently read is the part
+// most likely still in L2.
+#include "fp8lin_internal.cuh"
+
+namespace fp8lin {
+
+constexpr int kCastThreads = 256;
+
+template <int FMT>
+__device__ __forceinline__ uint32_t cvt_pair(float hi, float lo)
+{
+    uint16_t r;
+    if (FMT == FP8_E4)
+        asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(r) : "f"(hi), "f"(lo));
+    else
+        asm("cvt.rn.satfinite.e5m2x2.f32 %0, %1, %2;" : "=h"(r) : "f"(hi), "f"(lo));
+    return (uint32_t)r;
+}
+
+// True when RNE to the format would land beyond its largest finite value.
+template <int FMT>
+__device__ __forceinline__ bool clips(float v)
+{
+    return FMT == FP8_E4 ? (fabsf(v) > 464.0f) : (fabsf(v) >= 61440.0f);
+}
+
+// Four bf16 values (two packed words, memory order) -> four FP8 bytes (memory order).
+template <int FMT, bool TWO_STEP>
+__device__ __forceinline__ uint32_t cast4(uint32_t w0, uint32_t w1, Pow2Pair p, bool &sat)
+{
+    float f0 = __uint_as_float(w0 << 16) * p.first;
+    float f1 = __uint_as_float(w0 & 0xFFFF0000u) * p.first;
+    float f2 = __uint_as_float(w1 << 16) * p.first;
+    float f3 = __uint_as_float(w1 & 0xFFFF0000u) * p.first;
+    if (TWO_STEP) { f0 *= p.second; f1 *= p.second; f2 *= p.second; f3 *= p.second; }
+    sat = sat || clips<FMT>(f0) || clips<FMT>(f1) || clips<FMT>(f2) || clips<FMT>(f3);
+    return cvt_pair<FMT>(f1, f0) | (cvt_pair<FMT>(f3, f2) << 16);
+}
+
+template <int FMT, bool TWO_STEP>
+__device__ __forceinline__ uint8_t cast1(uint16_t h, Pow2Pair p, bool &sat)
+{
+    float f = __uint_as_float((uint32_t)h << 16) * p.first;
+    if (TWO_STEP) f *= p.second;
+    sat = sat || clips<FMT>(f);
+    return (uint8_t)(cvt_pair<FMT>(0.0f, f) & 0xFFu);
+}
+
+// ---------------------------------------------------------------------------
+// contiguous, row-major output only
+// ---------------------------------------------------------------------------
+
+template <int FMT, bool TWO_STEP>
+__device__ __forceinline__ void cast_flat_body(const uint4 *__restrict__ x, uint4 *__restrict__ y, int64_t nout,
+                                               Pow2Pair p, bool &sat)
+{
+    // nout = number of 16-byte output vectors; each consumes two input vectors.
+    const int64_t chunk = (int64_t)kCastThreads * 2;
+    const int64_t nchunks = (nout + chunk - 1) / chunk;
+    for (int64_t c = nchunks - 1 - blockIdx.x; c >= 0; c -= gridDim.x) {
+        int64_t i0 = c * chunk + threadIdx.x;
+        int64_t i1 = i0 + kCastThreads;
+        uint4 a0, a1, b0, b1;
+        bool ok0 = i0 < nout, ok1 = i1 < nout;
+        if (ok0) { a0 = __ldcs(x + 2 * i0); a1 = __ldcs(x + 2 * i0 + 1); }
+        if (ok1) { b0 = __ldcs(x + 2 * i1); b1 = __ldcs(x + 2 * i1 + 1); }
+        if (ok0) {
+            uint4 o;
+            o.x = cast4<FMT, TWO_STEP>(a0.x, a0.y, p, sat);
+            o.y = cast4<FMT, TWO_STEP>(a0.z, a0.w, p, sat);
+            o.z = cast4<FMT, TWO_STEP>(a1.x, a1.y, p, sat);
+            o.w = cast4<FMT, TWO_STEP>(a1.z, a1.w, p, sat);
+            y[i0] = o;
+        }
+        if (ok1) {
+            uint4 o;
+            o.x = cast4<FMT, TWO_STEP>(b0.x, b0.y, p, sat);
+            o.y = cast4<FMT, TWO_STEP>(b0.z, b0.w, p, sat);
+            o.z = cast4<FMT, TWO_STEP>(b1.x, b1.y, p, sat);
+            o.w = cast4<FMT, TWO_STEP>(b1.z, b1.w, p, sat);
+            y[i1] = o;
+        }
+    }
+}
+
+template <int FMT>
+__global__ void __launch_bounds__(kCastThreads) cast_flat_kernel(const uint4 *__restrict__ x, uint4 *__restrict__ y,
+                                                                 int64_t nout, const uint16_t *__restrict__ tail_in,
+                                                                 uint8_t *__restrict__ tail_out, int ntail,
+                                                                 const int32_t *__restrict__ d_bias, int delta,
+                                                                 unsigned *d_status)
+{
+    const int s = __ldg(d_bias) + delta;
+    const Pow2Pair p = make_pow2_pair(s);
+    bool sat = false;
+    if (s >= -126 && s <= 127) cast_flat_body<FMT, false>(x, y, nout, p, sat);
+    else cast_flat_body<FMT, true>(x, y, nout, p, sat);
+    if (blockIdx.x == 0 && (int)threadIdx.x < ntail)
+        tail_out[threadIdx.x] = cast1<FMT, true>(tail_in[threadIdx.x], p, sat);
+    if (__syncthreads_or(sat) && threadIdx.x == 0) atomicOr(d_status, FP8_FLAG_SATURATED);
+}
+
+// ---------------------------------------------------------------------------
+// tiled, with optional transposed output
+// ---------------------------------------------------------------------------
+
+constexpr int kTile = 128;
+
+// Transpose a 4x4 byte block held as four row words into four column words.
+__device__ __forceinline__ void transpose4x4(const uint32_t r[4], uint32_t c[4])
+{
+    uint32_t t0 = __byte_perm(r[0], r[1], 0x5140);
+    uint32_t t1 = __byte_perm(r[2], r[3], 0x5140);
+    uint32_t t2 = __byte_perm(r[0], r[1], 0x7362);
+    uint32_t t3 = __byte_perm(r[2], r[3], 0x7362);
+    c[0] = __byte_perm(t0, t1, 0x5410);
+    c[1] = __byte_perm(t0, t1, 0x7632);
+    c[2] = __byte_perm(t2, t3, 0x5410);
+    c[3] = __byte_perm(t2, t3, 0x7632);
+}
+
+template <int FMT>
+__global__ void __launch_bounds__(kCastThreads) cast_tile_kernel(const uint16_t *__restrict__ x, int64_t rows,
+                                                                 int64_t cols, int64_t ld,
+                                                                 const int32_t *__restrict__ d_bias, int delta,
+                                                                 uint8_t *__restrict__ y, uint8_t *__restrict__ y_t,
+                                                                 int fast_ok, unsigned *d_status)
+{
+    // Transposed staging: word (c, w) holds rows 4w..4w+3 of tile column c; the
+    // word position is rotated by c/4 so that both the column-wise writes and
+    // the row-wise reads touch 32 distinct banks.
+    __shared__ uint32_t stage[kTile][kTile / 4];
+
+    const int s = __ldg(d_bias) + delta;
+    const Pow2Pair p = make_pow2_pair(s);
+    bool sat = false;
+
+    const int64_t tiles_c = (cols + kTile - 1) / kTile;
+    const int64_t tile = (int64_t)gridDim.x - 1 - blockIdx.x;
+    const int64_t r0 = (tile / tiles_c) * kTile;
+    const int64_t c0 = (tile % tiles_c) * kTile;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    if (fast_ok && r0 + kTile <= rows && c0 + kTile <= cols) {
+        uint2 v[4][4];
+#pragma unroll
+        for (int it = 0; it < 4; ++it) {
+            const int rg = warp + 8 * it;
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+                v[it][i] = __ldcs(reinterpret_cast<const uint2 *>(x + (r0 + 4 * rg + i) * ld + c0 + 4 * lane));
+        }
+#pragma unroll
+        for (int it = 0; it < 4; ++it) {
+            const int rg = warp + 8 * it;
+            uint32_t rw[4], cw[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) rw[i] = cast4<FMT, true>(v[it][i].x, v[it][i].y, p, sat);
+            if (y) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+                    *reinterpret_cast<uint32_t *>(y + (r0 + 4 * rg + i) * cols + c0 + 4 * lane) = rw[i];
+            }
+            if (y_t) {
+                transpose4x4(rw, cw);
+#pragma unroll
+                for (int j = 0; j < 4; ++j) stage[4 * lane + j][(rg + lane) & 31] = cw[j];
+            }
+        }
+        if (y_t) {
+            __syncthreads();
+#pragma unroll 4
+            for (int cc = warp; cc < kTile; cc += 8) {
+                uint32_t w = stage[cc][(lane + (cc >> 2)) & 31];
+                *reinterpret_cast<uint32_t *>(y_t + (c0 + cc) * rows + r0 + 4 * lane) = w;
+            }
+        }
+    } else {
+        // Guarded path for ragged tiles and unaligned tensors: one element at a time.
+        uint8_t *stage_b = reinterpret_cast<uint8_t *>(&stage[0][0]);  // [c][r] bytes
+        for (int idx = threadIdx.x; idx < kTile * kTile; idx += kCastThreads) {
+            int r = idx / kTile, c = idx % kTile;
+            if (r0 + r < rows && c0 + c < cols) {
+                uint8_t code = cast1<FMT, true>(x[(r0 + r) * ld + c0 + c], p, sat);
+                if (y) y[(r0 + r) * cols + c0 + c] = code;
+                if (y_t) stage_b[c * kTile + r] = code;
+            }
+        }
+        if (y_t) {
+            __syncthreads();
+            for (int idx = threadIdx.x; idx < kTile * kTile; idx += kCastThreads) {
+                int c = idx / kTile, r = idx % kTile;
+                if (r0 + r < rows && c0 + c < cols) y_t[(c0 + c) * rows + r0 + r] = stage_b[c * kTile + r];
+            }
+        }
+    }
+    if (__syncthreads_or(sat) && threadIdx.x == 0) atomicOr(d_status, FP8_FLAG_SATURATED);
+}
+
+template <int FMT>
+static cudaError_t launch_cast(fp8_ctx *ctx, const void *x, int64_t rows, int64_t cols, int64_t ld,
+                               const int32_t *d_bias, int delta, uint8_t *y, uint8_t *y_t, cudaStream_t stream)
+{
+    auto al = [](const void *p, unsigned a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; };
+    if (!y_t && ld == cols && al(x, 16) && al(y, 16)) {
+        int64_t n = rows * cols;
+        int64_t nout = n / 16;
+        int ntail = (int)(n - nout * 16);
+        int64_t chunk = (int64_t)kCastThreads * 2;
+        int64_t want = (nout + chunk - 1) / chunk;
+        int max_blocks = ctx->sm_count * 8;
+        int blocks = (int)(want < 1 ? 1 : (want > max_blocks ? max_blocks : want));
+        cast_flat_kernel<FMT><<<blocks, kCastThreads, 0, stream>>>(
+            reinterpret_cast<const uint4 *>(x), reinterpret_cast<uint4 *>(y), nout,
+            reinterpret_cast<const uint16_t *>(x) + nout * 16, y + nout * 16, ntail, d_bias, delta, ctx->d_status);
+        return cudaGetLastError();
+    }
+    int fast_ok = al(x, 8) && (ld % 4) == 0 && (!y || (al(y, 4) && (cols % 4) == 0)) &&
+                  (!y_t || (al(y_t, 4) && (rows % 4) == 0));
+    int64_t tiles = ((rows + kTile - 1) / kTile) * ((cols + kTile - 1) / kTile);
+    if (tiles > 0x7FFFFFFF) return cudaErrorInvalidValue;
+    cast_tile_kernel<FMT><<<(unsigned)tiles, kCastThreads, 0, stream>>>(reinterpret_cast<const uint16_t *>(x), rows,
+                                                                        cols, ld, d_bias, delta, y, y_t, fast_ok,
+                                                                        ctx->d_status);
+    return cudaGetLastError();
+}
+
+static fp8_status_t cast_entry(int fmt, fp8_ctx *ctx, const void *x, fp8_dtype_t x_dt, int64_t rows, int64_t cols,
+                               int64_t ld, const int32_t *d_bias, fp8_conv_t conv, int32_t margin, float *d_amax_out,
+                               int32_t *d_bias_out, uint8_t *y, uint8_t *y_t, void *stream)
+{
+    if (!ctx || !x || (!y && !y_t)) return FP8_ERR_NULL;
+    if (!d_bias && (!d_amax_out || !d_bias_out)) return FP8_ERR_NULL;
+    if ((int)x_dt < 0 || (int)x_dt > 2 || (int)conv < 0 || (int)conv > 1) return FP8_ERR_DTYPE;
+    if (x_dt != FP8_BF16) return FP8_ERR_UNSUPPORTED;
+    if (rows <= 0 || cols <= 0 || ld < cols) return FP8_ERR_SHAPE;
+    if (reinterpret_cast<uintptr_t>(x) & 1u) return FP8_ERR_ALIGN;
+    cudaStream_t st = (cudaStream_t)stream;
+    const int32_t *bias = d_bias;
+    if (!bias) {
+        if (launch_amax_bias(ctx, x, rows, cols, ld, d_amax_out, d_bias_out, fmt, (int)conv, margin, st) !=
+            cudaSuccess)
+            return FP8_ERR_CUDA;
+        bias = d_bias_out;
+    }
+    int delta = format_delta(fmt, (int)conv);
+    cudaError_t e = fmt == FP8_E4 ? launch_cast<FP8_E4>(ctx, x, rows, cols, ld, bias, delta, y, y_t, st)
+                                  : launch_cast<FP8_E5>(ctx, x, rows, cols, ld, bias, delta, y, y_t, st);
+    return e == cudaSuccess ? FP8_OK : FP8_ERR_CUDA;
+}
+
+}  // namespace fp8lin
+
+extern "C" {
+
+fp8_status_t fp8_cast_e4(fp8_ctx *ctx, const void *x, fp8_dtype_t x_dt, int64_t rows, int64_t cols, int64_t ld,
+                         const int32_t *d_bias, fp8_conv_t conv, int32_t margin, float *d_amax_out,
+                         int32_t *d_bias_out, uint8_t *y, uint8_t *y_t, void *stream)
+{
+    return fp8lin::cast_entry(FP8_E4, ctx, x, x_dt, rows, cols, ld, d_bias, conv, margin, d_amax_out, d_bias_out, y,
+                              y_t, stream);
+}
+
+fp8_status_t fp8_cast_e5(fp8_ctx *ctx, const void *x, fp8_dtype_t x_dt, int64_t rows, int64_t cols, int64_t ld,
+                         const int32_t *d_bias, fp8_conv_t conv, int32_t margin, float *d_amax_out,
+                         int32_t *d_bias_out, uint8_t *y, uint8_t *y_t, void *stream)
+{
+    return fp8lin::cast_entry(FP8_E5, ctx, x, x_dt, rows, cols, ld, d_bias, conv, margin, d_amax_out, d_bias_out, y,
+                              y_t, stream);
+}
+
+fp8_status_t fp8_ptq_weights(fp8_ctx *ctx, const void *w, fp8_dtype_t w_dt, int64_t N, int64_t K, int64_t ld,
+                             fp8_conv_t conv, uint8_t *w8, uint8_t *w8_t, int32_t *d_bw, float *d_amax_w,
+                             void *stream)
+{
+    return fp8lin::cast_entry(FP8_E4, ctx, w, w_dt, N, K, ld, nullptr, conv, 0, d_amax_w, d_bw, w8, w8_t, stream);
+}
+
+}  // extern "C"

@@ -1,0 +1,126 @@
+// Internal declarations shared by the translation units of libfp8lin.so.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "fp8lin.h"
+
+namespace fp8lin {
+
+// ---------------------------------------------------------------------------
+// context
+// ---------------------------------------------------------------------------
+
+constexpr int kReduceSlots = 64;   // independent grid-reduction slots, used round-robin
+constexpr int kSlotWords = 4;      // {running max, arrival counter, pad, pad}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+}  // namespace fp8lin
+
+struct fp8_ctx {
+    int device;
+    int sm_count;
+    int max_smem_optin;
+    unsigned *d_status;   // one sticky word of FP8_FLAG_* bits
+    unsigned *d_slots;    // kReduceSlots * kSlotWords words, all zero between calls
+    unsigned next_slot;
+    fp8lin::EncodeTiledFn encode_tiled;
+};
+
+namespace fp8lin {
+
+inline unsigned *take_slot(fp8_ctx *ctx)
+{
+    unsigned s = ctx->next_slot++ % kReduceSlots;
+    return ctx->d_slots + s * kSlotWords;
+}
+
+// Format shift between the paper-convention bias and the shift that yields
+// native bytes (+1 for E4 under the paper convention, else 0).
+__host__ __device__ inline int format_delta(int fmt, int conv)
+{
+    return (fmt == FP8_E4 && conv == FP8_CONV_PAPER) ? 1 : 0;
+}
+
+// Eq. 3 on the bits of a non-negative float: the largest b with
+// amax * 2^b <= max_num, minus margin.  max_num = m_max * 2^e_max with
+// (1.875, 7) for 240, (1.75, 8) for 448, (1.75, 15) for 57344.
+__host__ __device__ inline int bias_from_amax_bits(uint32_t bits, int fmt, int conv, int margin, unsigned *flags)
+{
+    bits &= 0x7FFFFFFFu;
+    if (bits == 0u) { *flags |= FP8_FLAG_ZERO_AMAX; return 0; }
+    if (bits >= 0x7F800000u) { *flags |= FP8_FLAG_NONFINITE_AMAX; return 0; }
+    int e;
+    uint32_t frac;  // 23 fraction bits of the normalised significand
+    uint32_t ef = bits >> 23;
+    uint32_t mant = bits & 0x7FFFFFu;
+    if (ef != 0u) {
+        e = (int)ef - 127;
+        frac = mant;
+    } else {  // subnormal: normalise
+        int hb = 22;
+        while (((mant >> hb) & 1u) == 0u) --hb;
+        e = -149 + hb;
+        frac = (mant << (23 - hb)) & 0x7FFFFFu;
+    }
+    int e_max;
+    uint32_t frac_max;
+    if (fmt == FP8_E5) { e_max = 15; frac_max = 0x600000u; }
+    else if (conv == FP8_CONV_PAPER) { e_max = 7; frac_max = 0x700000u; }
+    else { e_max = 8; frac_max = 0x600000u; }
+    return e_max - e - (frac > frac_max ? 1 : 0) - margin;
+}
+
+cudaError_t launch_amax_bias(fp8_ctx *ctx, const void *x, int64_t rows, int64_t cols, int64_t ld, float *d_amax,
+                             int32_t *d_bias, int fmt, int conv, int margin, cudaStream_t stream);
+
+}  // namespace fp8lin
+
+// ---------------------------------------------------------------------------
+// device helpers
+// ---------------------------------------------------------------------------
+#ifdef __CUDACC__
+namespace fp8lin {
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p)
+{
+    return (uint32_t)__cvta_generic_to_shared(p);
+}
+
+__device__ __forceinline__ unsigned long long global_timer_ns()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+
+// 2^e as a float for e in [-126, 127].
+__device__ __forceinline__ float pow2_normal(int e)
+{
+    return __uint_as_float((uint32_t)(e + 127) << 23);
+}
+
+// x * 2^s split into two exact power-of-two factors so that any s in
+// [-300, 300] works: the first factor carries as much of s as one normal
+// float can, the second the rest.
+struct Pow2Pair {
+    float first, second;
+};
+__device__ __forceinline__ Pow2Pair make_pow2_pair(int s)
+{
+    int s1 = max(-126, min(127, s));
+    int s2 = max(-126, min(127, s - s1));
+    Pow2Pair p;
+    p.first = pow2_normal(s1);
+    p.second = pow2_normal(s2);
+    return p;
+}
+
+}  // namespace fp8lin
+#endif

@@ -1,0 +1,510 @@
+// FP8 matmuls with the unscale folded into the epilogue (Fig. 3b, Eq. 2 for the
+// forward pass; Section 2.2 for the two backward matmuls).
+//
+// One persistent, warp-specialised kernel computes D[M,N] = A[M,K] * B[N,K]^T
+// with both operands contiguous along the contraction dimension:
+//   warp 0, one lane   TMA producer: 128x128-byte A boxes and BNx128-byte B
+//                      boxes (128-byte swizzle) into a ring of shared-memory
+//                      stages, completion signalled on an mbarrier per stage.
+//   warp 1, one lane   MMA issuer: tcgen05.mma.kind::f8f6f4 (M=128, N=BN,
+//                      K=32 per instruction) from shared-memory descriptors
+//                      into one of two FP32 accumulators in tensor memory;
+//                      tcgen05.commit releases the stage / publishes the tile.
+//   warps 2..5         epilogue: tcgen05.ld of the finished accumulator (each
+//                      warp owns the 32 TMEM lanes it may address), exact
+//                      power-of-two unscale, optional bias vector, rounding to
+//                      the output type, optional amax of the rounded output.
+// The two accumulators let the epilogue of tile i overlap the main loop of
+// tile i+1.  A and B may be different FP8 formats (E5 x E4 in the backward
+// pass); the formats live in the instruction descriptor.
+//
+// Every wait on an mbarrier is bounded: when it expires the CTA raises
+// FP8_FLAG_TIMEOUT in the status word, all roles leave their loops, tensor
+// memory is released and the kernel returns.
+#include "fp8lin_internal.cuh"
+
+namespace fp8lin {
+
+constexpr int kBM = 128;          // rows of D per tile = TMEM lanes
+constexpr int kBK = 128;          // contraction bytes per stage = one 128-byte swizzle row
+constexpr int kUmmaK = 32;        // contraction elements per tcgen05.mma for 8-bit types
+constexpr int kGemmThreads = 192;
+constexpr int kGroupM = 8;        // tile rasterisation: m-blocks per group
+constexpr unsigned long long kWaitLimitNs = 1000ull * 1000ull * 1000ull;
+
+struct GemmParams {
+    int M, N, K;
+    int tiles_m, tiles_n, num_k;
+    const int32_t *d_sa, *d_sb;   // paper-convention biases of the two operands
+    int delta_sum;                // format shifts to add to them
+    const void *bias_vec;         // [N] or NULL
+    int bias_dt;
+    void *out;
+    int out_dt;
+    int64_t ldo;
+    int vec_ok;                   // out 16-byte aligned and ldo*elem % 16 == 0
+    unsigned *d_amax_bits;        // or NULL
+    unsigned *d_status;
+    uint32_t idesc;
+};
+
+// ---------------------------------------------------------------------------
+// PTX wrappers
+// ---------------------------------------------------------------------------
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+        "selp.u32 %0, 1, 0, p;\n"
+        "}\n"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+
+// Bounded wait.  Returns false when the wait expired or another role gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, unsigned *d_status)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    const unsigned long long t0 = global_timer_ns();
+    unsigned spins = 0;
+    while (!mbar_try_wait(bar, parity)) {
+        if ((++spins & 63u) == 0u) {
+            if (*abort_flag) return false;
+            if (global_timer_ns() - t0 > kWaitLimitNs) {
+                *abort_flag = 1;
+                atomicOr(d_status, FP8_FLAG_TIMEOUT);
+                return false;
+            }
+        }
+    }
+    return true;
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int x, int y)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(x), "r"(y)
+        : "memory");
+}
+
+__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t cols)
+{
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols)
+{
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void umma_f8(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc,
+                                        uint32_t accumulate)
+{
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "setp.ne.b32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n"
+        "}\n"
+        ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// Arrive on an mbarrier once every tcgen05.mma issued so far by this thread has completed.
+__device__ __forceinline__ void umma_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void tmem_ld_x32(uint32_t taddr, uint32_t (&r)[32])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor for a tile whose rows are 128 contiguous
+// bytes along the contraction dimension, 128-byte swizzled, rows packed in
+// groups of eight (1024 bytes apart): start address, leading offset 16 B
+// (unused for swizzled layouts), stride offset 1024 B, descriptor version 1,
+// layout type 2 (128-byte swizzle).
+__device__ __forceinline__ uint64_t smem_desc_k128(uint32_t smem_addr)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr >> 4) & 0x3FFFu);
+    d |= (uint64_t)1 << 16;
+    d |= (uint64_t)(1024 >> 4) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)2 << 61;
+    return d;
+}
+
+__host__ __device__ inline uint32_t make_idesc(int a_fmt, int b_fmt, int n)
+{
+    // FP32 accumulate, both operands contraction-major, M = 128.
+    return (1u << 4) | ((uint32_t)a_fmt << 7) | ((uint32_t)b_fmt << 10) | ((uint32_t)(n >> 3) << 17) |
+           ((uint32_t)(kBM >> 4) << 24);
+}
+
+// ---------------------------------------------------------------------------
+// kernel
+// ---------------------------------------------------------------------------
+
+template <int BN, int STAGES>
+struct GemmSmem {
+    static constexpr int kABytes = kBM * kBK;
+    static constexpr int kBBytes = BN * kBK;
+    static constexpr int kStageBytes = kABytes + kBBytes;
+    static constexpr int kBarOffset = STAGES * kStageBytes;
+    static constexpr int kNumBars = 2 * STAGES + 4;
+    static constexpr int kTotal = kBarOffset + kNumBars * 8 + 16;
+    static constexpr int kDynamic = kTotal + 1024;  // slack to align the base to 1024 B
+    static constexpr int kTmemCols = (2 * BN < 32) ? 32 : 2 * BN;
+};
+
+__device__ __forceinline__ void tile_coords(int tile, const GemmParams &p, int &m_blk, int &n_blk)
+{
+    const int group = kGroupM * p.tiles_n;
+    const int g = tile / group;
+    const int first_m = g * kGroupM;
+    const int gm = min(kGroupM, p.tiles_m - first_m);
+    const int r = tile - g * group;
+    m_blk = first_m + r % gm;
+    n_blk = r / gm;
+}
+
+template <int BN, int STAGES>
+__global__ void __launch_bounds__(kGemmThreads, 1)
+gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const GemmParams p)
+{
+    using L = GemmSmem<BN, STAGES>;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    const uint32_t smem_base = smem_u32(smem);
+    const uint32_t bar_base = smem_base + L::kBarOffset;
+    auto full_bar = [&](int s) { return bar_base + 8u * s; };
+    auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
+    auto acc_full_bar = [&](int b) { return bar_base + 8u * (2 * STAGES + b); };
+    auto acc_empty_bar = [&](int b) { return bar_base + 8u * (2 * STAGES + 2 + b); };
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + L::kBarOffset + L::kNumBars * 8);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int num_tiles = p.tiles_m * p.tiles_n;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(acc_full_bar(b), 1); mbar_init(acc_empty_bar(b), 4); }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) tmem_alloc(smem_u32(tmem_slot), L::kTmemCols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_a)) : "memory");
+            asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_b)) : "memory");
+            uint32_t it = 0;
+            bool alive = true;
+            for (int tile = blockIdx.x; alive && tile < num_tiles; tile += gridDim.x) {
+                int m_blk, n_blk;
+                tile_coords(tile, p, m_blk, n_blk);
+                for (int k = 0; k < p.num_k; ++k, ++it) {
+                    const int s = it % STAGES;
+                    const uint32_t ph = (it / STAGES) & 1u;
+                    if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p.d_status)) { alive = false; break; }
+                    mbar_expect_tx(full_bar(s), L::kStageBytes);
+                    const uint32_t a_dst = smem_base + s * L::kStageBytes;
+                    tma_load_2d(a_dst, &map_a, full_bar(s), k * kBK, m_blk * kBM);
+                    tma_load_2d(a_dst + L::kABytes, &map_b, full_bar(s), k * kBK, n_blk * BN);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            uint32_t it = 0, t = 0;
+            bool alive = true;
+            for (int tile = blockIdx.x; alive && tile < num_tiles; tile += gridDim.x, ++t) {
+                const int buf = t & 1;
+                const uint32_t acc_ph = (t >> 1) & 1u;
+                if (!mbar_wait(acc_empty_bar(buf), acc_ph ^ 1u, abort_flag, p.d_status)) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + buf * BN;
+                for (int k = 0; k < p.num_k; ++k, ++it) {
+                    const int s = it % STAGES;
+                    const uint32_t ph = (it / STAGES) & 1u;
+                    if (!mbar_wait(full_bar(s), ph, abort_flag, p.d_status)) { alive = false; break; }
+                    tc_fence_after();
+                    const uint32_t a_addr = smem_base + s * L::kStageBytes;
+                    const uint64_t da = smem_desc_k128(a_addr);
+                    const uint64_t db = smem_desc_k128(a_addr + L::kABytes);
+#pragma unroll
+                    for (int j = 0; j < kBK / kUmmaK; ++j) {
+                        // advancing 32 bytes inside the 128-byte swizzle row = +2 in the 16-byte address field
+                        umma_f8(d_tmem, da + 2u * j, db + 2u * j, p.idesc, (k > 0 || j > 0) ? 1u : 0u);
+                    }
+                    umma_commit(empty_bar(s));
+                }
+                if (alive) umma_commit(acc_full_bar(buf));
+            }
+        }
+    } else {
+        // ------------------------------- epilogue -------------------------------
+        const int q = warp & 3;  // TMEM lane quarter this warp may address
+        const int e = -(__ldg(p.d_sa) + __ldg(p.d_sb) + p.delta_sum);
+        const Pow2Pair sc = make_pow2_pair(e);
+        const bool two_step = (e < -126 || e > 127);
+        uint32_t amax_bits = 0;
+        uint32_t t = 0;
+        for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++t) {
+            int m_blk, n_blk;
+            tile_coords(tile, p, m_blk, n_blk);
+            const int buf = t & 1;
+            const uint32_t acc_ph = (t >> 1) & 1u;
+            // every lane waits (each needs the ordering), but the warp leaves together
+            const bool ready = mbar_wait(acc_full_bar(buf), acc_ph, abort_flag, p.d_status);
+            if (!__all_sync(0xFFFFFFFFu, ready)) break;
+            tc_fence_after();
+            const int row = m_blk * kBM + q * 32 + lane;
+            const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + buf * BN;
+#pragma unroll 1
+            for (int c = 0; c < BN; c += 32) {
+                uint32_t r[32];
+                tmem_ld_x32(t_row + c, r);
+                tmem_ld_wait();
+                if (c + 32 >= BN) {
+                    // the accumulator is in registers: hand the TMEM buffer back
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(acc_empty_bar(buf));
+                }
+                const int col0 = n_blk * BN + c;
+                if (row >= p.M || col0 >= p.N) continue;
+                float v[32];
+#pragma unroll
+                for (int i = 0; i < 32; ++i) {
+                    v[i] = __uint_as_float(r[i]) * sc.first;
+                    if (two_step) v[i] *= sc.second;
+                }
+                if (p.bias_vec) {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) {
+                        if (col0 + i < p.N) {
+                            float b = p.bias_dt == FP8_F32
+                                          ? __ldg(reinterpret_cast<const float *>(p.bias_vec) + col0 + i)
+                                          : __uint_as_float(
+                                                (uint32_t)__ldg(reinterpret_cast<const uint16_t *>(p.bias_vec) + col0 + i)
+                                                << 16);
+                            v[i] += b;
+                        }
+                    }
+                }
+                if (p.out_dt == FP8_BF16) {
+                    uint32_t w[16];
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(w[i]) : "f"(v[2 * i + 1]), "f"(v[2 * i]));
+                    }
+                    if (p.d_amax_bits) {
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) {
+                            uint32_t a = w[i] & 0x7FFF7FFFu;
+                            if (col0 + 2 * i < p.N) amax_bits = max(amax_bits, (a & 0xFFFFu) << 16);
+                            if (col0 + 2 * i + 1 < p.N) amax_bits = max(amax_bits, a & 0xFFFF0000u);
+                        }
+                    }
+                    uint16_t *dst = reinterpret_cast<uint16_t *>(p.out) + (int64_t)row * p.ldo + col0;
+                    if (p.vec_ok && col0 + 32 <= p.N) {
+#pragma unroll
+                        for (int j = 0; j < 4; ++j)
+                            reinterpret_cast<uint4 *>(dst)[j] = make_uint4(w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i)
+                            if (col0 + i < p.N) dst[i] = (uint16_t)((i & 1) ? (w[i >> 1] >> 16) : (w[i >> 1] & 0xFFFFu));
+                    }
+                } else {
+                    if (p.d_amax_bits) {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i)
+                            if (col0 + i < p.N) amax_bits = max(amax_bits, __float_as_uint(v[i]) & 0x7FFFFFFFu);
+                    }
+                    float *dst = reinterpret_cast<float *>(p.out) + (int64_t)row * p.ldo + col0;
+                    if (p.vec_ok && col0 + 32 <= p.N) {
+#pragma unroll
+                        for (int j = 0; j < 8; ++j)
+                            reinterpret_cast<float4 *>(dst)[j] = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i)
+                            if (col0 + i < p.N) dst[i] = v[i];
+                    }
+                }
+            }
+        }
+        if (p.d_amax_bits) {
+            amax_bits = __reduce_max_sync(0xFFFFFFFFu, amax_bits);
+            if (lane == 0 && amax_bits) atomicMax(p.d_amax_bits, amax_bits);
+        }
+    }
+
+    // ------------------------------- teardown -------------------------------
+    __syncwarp();  // the single-lane roles rejoin their warps before the block-wide barrier
+    if (*abort_flag) __nanosleep(20000);  // let copies and MMAs already issued drain before the memory is released
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    if (warp == 1) tmem_dealloc(tmem_base, L::kTmemCols);
+}
+
+// ---------------------------------------------------------------------------
+// host side
+// ---------------------------------------------------------------------------
+
+constexpr int kBN = 256;
+constexpr int kStages = 4;
+
+cudaError_t configure_gemm_kernels(int max_smem_optin)
+{
+    using L = GemmSmem<kBN, kStages>;
+    if (L::kDynamic > max_smem_optin) return cudaErrorInvalidValue;
+    return cudaFuncSetAttribute(gemm_kernel<kBN, kStages>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kDynamic);
+}
+
+// 2-D tensor map over a row-major byte matrix [rows, cols_bytes]: box = box_rows x 128 bytes, 128-byte swizzle.
+static bool encode_map(fp8_ctx *ctx, CUtensorMap *map, const void *base, int64_t rows, int64_t cols_bytes,
+                       int box_rows)
+{
+    cuuint64_t dims[2] = {(cuuint64_t)cols_bytes, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)cols_bytes};
+    cuuint32_t box[2] = {(cuuint32_t)kBK, (cuuint32_t)box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = ctx->encode_tiled(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void *>(base), dims, strides, box,
+                                   estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+// D[M,N] = A[M,Kc] * B[N,Kc]^T, unscaled by 2^-(bias_a + bias_b + delta_sum).
+static fp8_status_t run_gemm(fp8_ctx *ctx, const uint8_t *a, int a_fmt, const int32_t *d_ba, const uint8_t *b,
+                             int b_fmt, const int32_t *d_bb, int delta_sum, const void *bias_vec, int bias_dt,
+                             void *out, int out_dt, float *d_amax_out, int64_t M, int64_t N, int64_t Kc,
+                             cudaStream_t st)
+{
+    if (M > 0x7FFFFFFF / 2 || N > 0x7FFFFFFF / 2 || Kc > 0x7FFFFFFF / 2) return FP8_ERR_SHAPE;
+    CUtensorMap map_a, map_b;
+    if (!encode_map(ctx, &map_a, a, M, Kc, kBM) || !encode_map(ctx, &map_b, b, N, Kc, kBN)) return FP8_ERR_CUDA;
+    GemmParams p;
+    p.M = (int)M; p.N = (int)N; p.K = (int)Kc;
+    p.tiles_m = (int)((M + kBM - 1) / kBM);
+    p.tiles_n = (int)((N + kBN - 1) / kBN);
+    p.num_k = (int)((Kc + kBK - 1) / kBK);
+    if ((int64_t)p.tiles_m * p.tiles_n > 0x7FFFFFFF) return FP8_ERR_SHAPE;
+    p.d_sa = d_ba; p.d_sb = d_bb; p.delta_sum = delta_sum;
+    p.bias_vec = bias_vec; p.bias_dt = bias_dt;
+    p.out = out; p.out_dt = out_dt; p.ldo = N;
+    const int64_t esz = out_dt == FP8_BF16 ? 2 : 4;
+    p.vec_ok = ((reinterpret_cast<uintptr_t>(out) & 15u) == 0 && (N * esz) % 16 == 0) ? 1 : 0;
+    p.d_amax_bits = reinterpret_cast<unsigned *>(d_amax_out);
+    p.d_status = ctx->d_status;
+    p.idesc = make_idesc(a_fmt, b_fmt, kBN);
+    if (d_amax_out && cudaMemsetAsync(d_amax_out, 0, sizeof(float), st) != cudaSuccess) return FP8_ERR_CUDA;
+    int tiles = p.tiles_m * p.tiles_n;
+    int grid = tiles < ctx->sm_count ? tiles : ctx->sm_count;
+    gemm_kernel<kBN, kStages><<<grid, kGemmThreads, GemmSmem<kBN, kStages>::kDynamic, st>>>(map_a, map_b, p);
+    return cudaGetLastError() == cudaSuccess ? FP8_OK : FP8_ERR_CUDA;
+}
+
+static bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+static bool out_dtype_ok(int dt) { return dt == FP8_BF16 || dt == FP8_F32; }
+
+}  // namespace fp8lin
+
+extern "C" {
+
+fp8_status_t fp8_linear_fwd(fp8_ctx *ctx, const uint8_t *x8, const int32_t *d_bx, const uint8_t *w8,
+                            const int32_t *d_bw, const void *bias_vec, fp8_dtype_t bias_dt, void *y,
+                            fp8_dtype_t y_dt, float *d_amax_y, int64_t T, int64_t K, int64_t N, fp8_conv_t conv,
+                            void *stream)
+{
+    using namespace fp8lin;
+    if (!ctx || !x8 || !d_bx || !w8 || !d_bw || !y) return FP8_ERR_NULL;
+    if ((int)conv < 0 || (int)conv > 1 || (int)y_dt < 0 || (int)y_dt > 2 || (int)bias_dt < 0 || (int)bias_dt > 2)
+        return FP8_ERR_DTYPE;
+    if (!out_dtype_ok(y_dt) || (bias_vec && !out_dtype_ok(bias_dt))) return FP8_ERR_UNSUPPORTED;
+    if (T <= 0 || K <= 0 || N <= 0) return FP8_ERR_SHAPE;
+    if (!aligned16(x8) || !aligned16(w8) || (K % 16) != 0 || (reinterpret_cast<uintptr_t>(y) & 3u)) return FP8_ERR_ALIGN;
+    int delta = 2 * format_delta(FP8_E4, conv);
+    return run_gemm(ctx, x8, FP8_E4, d_bx, w8, FP8_E4, d_bw, delta, bias_vec, bias_dt, y, y_dt, d_amax_y, T, N, K,
+                    (cudaStream_t)stream);
+}
+
+fp8_status_t fp8_linear_dgrad(fp8_ctx *ctx, const uint8_t *dy8, const int32_t *d_bg, const uint8_t *w8,
+                              const uint8_t *w8_t, const int32_t *d_bw, void *dx, fp8_dtype_t dx_dt,
+                              float *d_amax_dx, int64_t T, int64_t K, int64_t N, fp8_conv_t conv, void *stream)
+{
+    using namespace fp8lin;
+    if (!ctx || !dy8 || !d_bg || (!w8 && !w8_t) || !d_bw || !dx) return FP8_ERR_NULL;
+    if ((int)conv < 0 || (int)conv > 1 || (int)dx_dt < 0 || (int)dx_dt > 2) return FP8_ERR_DTYPE;
+    if (!out_dtype_ok(dx_dt)) return FP8_ERR_UNSUPPORTED;
+    if (!w8_t) return FP8_ERR_UNSUPPORTED;
+    if (T <= 0 || K <= 0 || N <= 0) return FP8_ERR_SHAPE;
+    if (!aligned16(dy8) || !aligned16(w8_t) || (N % 16) != 0 || (reinterpret_cast<uintptr_t>(dx) & 3u))
+        return FP8_ERR_ALIGN;
+    int delta = format_delta(FP8_E5, conv) + format_delta(FP8_E4, conv);
+    return run_gemm(ctx, dy8, FP8_E5, d_bg, w8_t, FP8_E4, d_bw, delta, nullptr, 0, dx, dx_dt, d_amax_dx, T, K, N,
+                    (cudaStream_t)stream);
+}
+
+fp8_status_t fp8_linear_wgrad(fp8_ctx *ctx, const uint8_t *dy8, const uint8_t *dy8_t, const int32_t *d_bg,
+                              const uint8_t *x8, const uint8_t *x8_t, const int32_t *d_bx, void *dw,
+                              fp8_dtype_t dw_dt, int64_t T, int64_t K, int64_t N, fp8_conv_t conv, void *stream)
+{
+    using namespace fp8lin;
+    if (!ctx || (!dy8 && !dy8_t) || !d_bg || (!x8 && !x8_t) || !d_bx || !dw) return FP8_ERR_NULL;
+    if ((int)conv < 0 || (int)conv > 1 || (int)dw_dt < 0 || (int)dw_dt > 2) return FP8_ERR_DTYPE;
+    if (!out_dtype_ok(dw_dt)) return FP8_ERR_UNSUPPORTED;
+    if (!dy8_t || !x8_t) return FP8_ERR_UNSUPPORTED;
+    if (T <= 0 || K <= 0 || N <= 0) return FP8_ERR_SHAPE;
+    if (!aligned16(dy8_t) || !aligned16(x8_t) || (T % 16) != 0 || (reinterpret_cast<uintptr_t>(dw) & 3u))
+        return FP8_ERR_ALIGN;
+    int delta = format_delta(FP8_E5, conv) + format_delta(FP8_E4, conv);
+    return run_gemm(ctx, dy8_t, FP8_E5, d_bg, x8_t, FP8_E4, d_bx, delta, nullptr, 0, dw, dw_dt, nullptr, N, K, T,
+                    (cudaStream_t)stream);
+}
+
+}  // extern "C"

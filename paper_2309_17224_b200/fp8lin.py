@@ -1,0 +1,176 @@
+"""Python face of ``libfp8lin.so``: argument marshalling only.
+
+Every function here has the name and the argument order of the C entry point
+declared in ``include/fp8lin.h``; tensors are torch CUDA tensors whose
+``data_ptr()`` is handed through, the stream is torch's current stream.  There
+is no arithmetic and no fallback in this module: if the library is missing the
+import fails, and a non-zero status raises ``Fp8Error``.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from ctypes import c_int, c_int32, c_int64, c_uint, c_void_p, c_float, c_char_p, POINTER, byref
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libfp8lin.so")
+
+OK = 0
+ERR_NULL, ERR_SHAPE, ERR_ALIGN, ERR_DTYPE, ERR_UNSUPPORTED, ERR_CUDA, ERR_DEVICE_TIMEOUT = range(1, 8)
+E4, E5 = 0, 1
+CONV_PAPER, CONV_NATIVE = 0, 1
+BF16, F16, F32 = 0, 1, 2
+FLAG_NONFINITE_AMAX, FLAG_ZERO_AMAX, FLAG_SATURATED, FLAG_TIMEOUT = 1, 2, 4, 8
+
+SYMBOLS = (
+    "fp8_create", "fp8_destroy", "fp8_status_string", "fp8_device_flags", "fp8_amax", "fp8_scaling_bias",
+    "fp8_scaling_bias_host", "fp8_cast_e4", "fp8_cast_e5", "fp8_ptq_weights", "fp8_linear_fwd", "fp8_linear_dgrad",
+    "fp8_linear_wgrad",
+)
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(
+        f"{LIB_PATH} is missing: build it with `python -m paper_2309_17224_b200.build` "
+        "(there is no fallback implementation)")
+
+_lib = ctypes.CDLL(LIB_PATH)
+
+_P = c_void_p
+_lib.fp8_create.argtypes = [POINTER(c_void_p), c_int]
+_lib.fp8_destroy.argtypes = [_P]
+_lib.fp8_status_string.argtypes = [c_int]
+_lib.fp8_status_string.restype = c_char_p
+_lib.fp8_device_flags.argtypes = [_P, _P, POINTER(c_uint), c_int]
+_lib.fp8_amax.argtypes = [_P, _P, c_int, c_int64, c_int64, c_int64, _P, _P]
+_lib.fp8_scaling_bias.argtypes = [_P, _P, c_int, c_int, c_int32, _P, _P]
+_lib.fp8_scaling_bias_host.argtypes = [c_float, c_int, c_int, c_int32, POINTER(c_int32)]
+_cast_args = [_P, _P, c_int, c_int64, c_int64, c_int64, _P, c_int, c_int32, _P, _P, _P, _P, _P]
+_lib.fp8_cast_e4.argtypes = _cast_args
+_lib.fp8_cast_e5.argtypes = _cast_args
+_lib.fp8_ptq_weights.argtypes = [_P, _P, c_int, c_int64, c_int64, c_int64, c_int, _P, _P, _P, _P, _P]
+_lib.fp8_linear_fwd.argtypes = [_P, _P, _P, _P, _P, _P, c_int, _P, c_int, _P, c_int64, c_int64, c_int64, c_int, _P]
+_lib.fp8_linear_dgrad.argtypes = [_P, _P, _P, _P, _P, _P, _P, c_int, _P, c_int64, c_int64, c_int64, c_int, _P]
+_lib.fp8_linear_wgrad.argtypes = [_P, _P, _P, _P, _P, _P, _P, _P, c_int, c_int64, c_int64, c_int64, c_int, _P]
+for _name in SYMBOLS:
+    if _name != "fp8_status_string":
+        getattr(_lib, _name).restype = c_int
+
+
+class Fp8Error(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} (status {status})")
+
+
+def status_string(status: int) -> str:
+    return _lib.fp8_status_string(int(status)).decode()
+
+
+def _check(status: int, where: str):
+    if status != OK:
+        raise Fp8Error(status, where)
+
+
+def _ptr(t):
+    return None if t is None else c_void_p(t.data_ptr())
+
+
+def _stream():
+    return c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+_DT = {torch.bfloat16: BF16, torch.float16: F16, torch.float32: F32}
+
+
+def scaling_bias_host(amax: float, fmt: int, conv: int = CONV_PAPER, margin: int = 0) -> int:
+    out = c_int32(0)
+    _check(_lib.fp8_scaling_bias_host(c_float(amax), fmt, conv, margin, byref(out)), "fp8_scaling_bias_host")
+    return out.value
+
+
+class Context:
+    """Owns one ``fp8_ctx``.  All methods launch on torch's current stream."""
+
+    def __init__(self, device: int = 0):
+        self._h = c_void_p()
+        self.device = device
+        _check(_lib.fp8_create(byref(self._h), device), "fp8_create")
+
+    def close(self):
+        if self._h:
+            _lib.fp8_destroy(self._h)
+            self._h = c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # -- status ---------------------------------------------------------------
+    def device_flags(self, clear: bool = True) -> int:
+        flags = c_uint(0)
+        st = _lib.fp8_device_flags(self._h, _stream(), byref(flags), 1 if clear else 0)
+        if st not in (OK, ERR_DEVICE_TIMEOUT):
+            _check(st, "fp8_device_flags")
+        return flags.value
+
+    # -- amax / bias ------------------------------------------------------------
+    def amax(self, x, d_amax, rows=None, cols=None, ld=None):
+        rows = x.shape[0] if rows is None else rows
+        cols = x.shape[1] if cols is None else cols
+        ld = x.stride(0) if ld is None else ld
+        _check(_lib.fp8_amax(self._h, _ptr(x), _DT[x.dtype], rows, cols, ld, _ptr(d_amax), _stream()), "fp8_amax")
+
+    def scaling_bias(self, d_amax, fmt, conv, margin, d_bias):
+        _check(_lib.fp8_scaling_bias(self._h, _ptr(d_amax), fmt, conv, margin, _ptr(d_bias), _stream()),
+               "fp8_scaling_bias")
+
+    # -- cast -------------------------------------------------------------------
+    def _cast(self, fn, name, x, d_bias, conv, margin, d_amax_out, d_bias_out, y, y_t, rows, cols, ld):
+        rows = x.shape[0] if rows is None else rows
+        cols = x.shape[1] if cols is None else cols
+        ld = x.stride(0) if ld is None else ld
+        _check(fn(self._h, _ptr(x), _DT[x.dtype], rows, cols, ld, _ptr(d_bias), conv, margin, _ptr(d_amax_out),
+                  _ptr(d_bias_out), _ptr(y), _ptr(y_t), _stream()), name)
+
+    def cast_e4(self, x, d_bias, conv=CONV_PAPER, margin=0, d_amax_out=None, d_bias_out=None, y=None, y_t=None,
+                rows=None, cols=None, ld=None):
+        self._cast(_lib.fp8_cast_e4, "fp8_cast_e4", x, d_bias, conv, margin, d_amax_out, d_bias_out, y, y_t, rows,
+                   cols, ld)
+
+    def cast_e5(self, x, d_bias, conv=CONV_PAPER, margin=0, d_amax_out=None, d_bias_out=None, y=None, y_t=None,
+                rows=None, cols=None, ld=None):
+        self._cast(_lib.fp8_cast_e5, "fp8_cast_e5", x, d_bias, conv, margin, d_amax_out, d_bias_out, y, y_t, rows,
+                   cols, ld)
+
+    def ptq_weights(self, w, conv, w8, w8_t, d_bw, d_amax_w):
+        _check(_lib.fp8_ptq_weights(self._h, _ptr(w), _DT[w.dtype], w.shape[0], w.shape[1], w.stride(0), conv,
+                                    _ptr(w8), _ptr(w8_t), _ptr(d_bw), _ptr(d_amax_w), _stream()), "fp8_ptq_weights")
+
+    # -- matmuls ----------------------------------------------------------------
+    def linear_fwd(self, x8, d_bx, w8, d_bw, y, bias_vec=None, d_amax_y=None, conv=CONV_PAPER):
+        T, K = x8.shape
+        N = w8.shape[0]
+        bias_dt = _DT[bias_vec.dtype] if bias_vec is not None else BF16
+        _check(_lib.fp8_linear_fwd(self._h, _ptr(x8), _ptr(d_bx), _ptr(w8), _ptr(d_bw), _ptr(bias_vec), bias_dt,
+                                   _ptr(y), _DT[y.dtype], _ptr(d_amax_y), T, K, N, conv, _stream()),
+               "fp8_linear_fwd")
+
+    def linear_dgrad(self, dy8, d_bg, w8, w8_t, d_bw, dx, d_amax_dx=None, conv=CONV_PAPER):
+        T, N = dy8.shape
+        K = dx.shape[1]
+        _check(_lib.fp8_linear_dgrad(self._h, _ptr(dy8), _ptr(d_bg), _ptr(w8), _ptr(w8_t), _ptr(d_bw), _ptr(dx),
+                                     _DT[dx.dtype], _ptr(d_amax_dx), T, K, N, conv, _stream()), "fp8_linear_dgrad")
+
+    def linear_wgrad(self, dy8, dy8_t, d_bg, x8, x8_t, d_bx, dw, T, conv=CONV_PAPER):
+        N, K = dw.shape
+        _check(_lib.fp8_linear_wgrad(self._h, _ptr(dy8), _ptr(dy8_t), _ptr(d_bg), _ptr(x8), _ptr(x8_t), _ptr(d_bx),
+                                     _ptr(dw), _DT[dw.dtype], T, K, N, conv, _stream()), "fp8_linear_wgrad")
+
+
+def raw():
+    """The ctypes library handle (for tests of the C ABI itself)."""
+    return _lib

@@ -1,0 +1,238 @@
+"""GPU parity: amax, scaling bias and scale-and-cast against the CPU oracle,
+bit for bit, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+import oracle as O
+from helpers import assert_codes_equal, bf16_from_bits, bits_of, u8
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_2309_17224_b200 import fp8lin
+    return fp8lin
+
+
+@pytest.fixture(scope="module")
+def ctx(lib):
+    c = lib.Context(0)
+    yield c
+    c.close()
+
+
+def _dev_scalar(dtype, value=0):
+    return torch.full((1,), value, dtype=dtype, device="cuda")
+
+
+def _same_float(a: float, b: float) -> bool:
+    return (np.isnan(a) and np.isnan(b)) or a == b
+
+
+def _gpu_amax(ctx, x, **kw):
+    out = _dev_scalar(torch.float32, -1.0)
+    ctx.amax(x, out, **kw)
+    return float(out.item())
+
+
+@pytest.mark.parametrize("shape", [(1, 1), (1, 7), (3, 8), (256, 768), (300, 520), (129, 257), (1024, 4096), (5, 100003)])
+def test_amax_contiguous(ctx, shape):
+    g = torch.Generator(device="cuda").manual_seed(shape[0] * 7919 + shape[1])
+    x = (torch.randn(shape, generator=g, device="cuda") * 3.0).to(torch.bfloat16)
+    assert _gpu_amax(ctx, x) == O.amax(bits_of(x))
+    # the maximum sitting at the very last / very first element, negative
+    x[-1, -1] = -4096.0
+    assert _gpu_amax(ctx, x) == 4096.0
+    x[0, 0] = 8192.0
+    assert _gpu_amax(ctx, x) == 8192.0
+
+
+def test_amax_strided_and_unaligned(ctx):
+    g = torch.Generator(device="cuda").manual_seed(5)
+    big = torch.randn((70, 264), generator=g, device="cuda").to(torch.bfloat16)
+    big[:, 200:] = 1000.0  # outside every view below
+    for cols, off in ((200, 0), (192, 0), (199, 1), (64, 3)):
+        view = big[:, off:off + cols]
+        want = O.amax(bits_of(view))
+        assert _gpu_amax(ctx, view, rows=70, cols=cols, ld=264) == want
+
+
+def test_amax_special_values(ctx):
+    x = torch.zeros((64, 64), dtype=torch.bfloat16, device="cuda")
+    assert _gpu_amax(ctx, x) == 0.0
+    x[3, 3] = -0.0
+    assert _gpu_amax(ctx, x) == 0.0
+    sub = bf16_from_bits(np.array([[0x8001, 0x0000]], dtype=np.uint16), "cuda")
+    assert _gpu_amax(ctx, sub) == 2.0 ** -133
+    x[10, 10] = float("inf")
+    assert _gpu_amax(ctx, x) == float("inf")
+    x[20, 20] = float("nan")
+    assert np.isnan(_gpu_amax(ctx, x)) and np.isnan(O.amax(bits_of(x)))
+    # repeated calls reuse the reduction slots: the result must not depend on history
+    y = torch.ones((128, 128), dtype=torch.bfloat16, device="cuda")
+    for _ in range(200):
+        assert _gpu_amax(ctx, y) == 1.0
+
+
+def test_scaling_bias_kernel_matches_oracle(ctx, lib):
+    vals = [0.0, 1e-45, 2.0 ** -133, 1e-30, 0.005, 0.08, 1.0, 1.875, 1.8828125, 5.0, 120.0, 240.0, 241.0, 448.0,
+            449.0, 57344.0, 57600.0, 3.0e38, float("inf"), float("nan")]
+    amax = _dev_scalar(torch.float32)
+    bias = _dev_scalar(torch.int32, 12345)
+    for v in vals:
+        for fmt, conv in ((lib.E4, lib.CONV_PAPER), (lib.E4, lib.CONV_NATIVE), (lib.E5, lib.CONV_PAPER)):
+            for margin in (0, 3):
+                amax.fill_(v)
+                ctx.scaling_bias(amax, fmt, conv, margin, bias)
+                assert int(bias.item()) == O.scaling_bias(v, fmt, conv, margin), (v, fmt, conv, margin)
+    flags = ctx.device_flags(clear=True)
+    assert flags & lib.FLAG_ZERO_AMAX and flags & lib.FLAG_NONFINITE_AMAX
+    assert ctx.device_flags() == 0
+
+
+def _all_bf16(device="cuda"):
+    bits = np.arange(65536, dtype=np.uint32).astype(np.uint16).reshape(256, 256)
+    return bits, bf16_from_bits(bits, device)
+
+
+@pytest.mark.parametrize("kind", [O.E4, O.E5])
+def test_cast_every_bf16_value_at_every_shift(ctx, lib, kind):
+    """All 65 536 input bit patterns x every shift a bias can produce."""
+    bits, x = _all_bf16()
+    fmt = O.native_format(kind)
+    cast = ctx.cast_e4 if kind == O.E4 else ctx.cast_e5
+    bias = _dev_scalar(torch.int32)
+    y = torch.empty((256, 256), dtype=torch.uint8, device="cuda")
+    y_t = torch.empty((256, 256), dtype=torch.uint8, device="cuda")
+    for b in range(-151, 152):
+        conv = lib.CONV_PAPER if b % 2 else lib.CONV_NATIVE
+        bias.fill_(b)
+        want = O.cast(bits, b + O.delta(kind, conv), fmt)
+        if b % 3 == 0:  # flat kernel
+            cast(x, bias, conv=conv, y=y)
+            assert_codes_equal(u8(y), want, fmt)
+        else:           # tiled kernel, both layouts
+            cast(x, bias, conv=conv, y=y, y_t=y_t)
+            assert_codes_equal(u8(y), want, fmt)
+            assert_codes_equal(u8(y_t), want.T, fmt)
+
+
+@pytest.mark.parametrize("shape", [(1, 1), (1, 7), (4, 16), (128, 128), (129, 257), (300, 520), (256, 768), (257, 131), (640, 1024)])
+@pytest.mark.parametrize("kind", [O.E4, O.E5])
+def test_cast_shapes_with_and_without_transpose(ctx, lib, kind, shape):
+    g = torch.Generator(device="cuda").manual_seed(shape[0] * 31 + shape[1])
+    x = (torch.randn(shape, generator=g, device="cuda") * 0.7).to(torch.bfloat16)
+    x[0, 0] = float("nan") if shape[1] > 1 else 1.0
+    xb = bits_of(x)
+    fmt = O.native_format(kind)
+    cast = ctx.cast_e4 if kind == O.E4 else ctx.cast_e5
+    a = O.amax(bits_of(torch.nan_to_num(x, nan=0.0)))
+    b = O.scaling_bias(a, kind)
+    want = O.cast(xb, b + O.delta(kind, O.CONV_PAPER), fmt)
+    bias = _dev_scalar(torch.int32, b)
+    rows, cols = shape
+    y = torch.full((rows * cols + 64,), 0xAB, dtype=torch.uint8, device="cuda")
+    y_t = torch.full((rows * cols + 64,), 0xCD, dtype=torch.uint8, device="cuda")
+    for use_y, use_t in ((True, False), (False, True), (True, True)):
+        y.fill_(0xAB)
+        y_t.fill_(0xCD)
+        cast(x, bias, y=y if use_y else None, y_t=y_t if use_t else None)
+        if use_y:
+            assert_codes_equal(u8(y[:rows * cols]).reshape(rows, cols), want, fmt)
+        if use_t:
+            assert_codes_equal(u8(y_t[:rows * cols]).reshape(cols, rows), want.T, fmt)
+        # nothing written past the end of either output
+        assert bool((y[rows * cols:] == 0xAB).all()) and bool((y_t[rows * cols:] == 0xCD).all())
+
+
+def test_cast_strided_input(ctx, lib):
+    g = torch.Generator(device="cuda").manual_seed(17)
+    big = torch.randn((200, 400), generator=g, device="cuda").to(torch.bfloat16)
+    bias = _dev_scalar(torch.int32, 4)
+    for cols, off in ((256, 0), (250, 8), (129, 1)):
+        view = big[:, off:off + cols]
+        want = O.cast(bits_of(view), 5, O.N_E4)
+        y = torch.empty((200, cols), dtype=torch.uint8, device="cuda")
+        y_t = torch.empty((cols, 200), dtype=torch.uint8, device="cuda")
+        ctx.cast_e4(view, bias, y=y, y_t=y_t, rows=200, cols=cols, ld=400)
+        assert_codes_equal(u8(y), want, O.N_E4)
+        assert_codes_equal(u8(y_t), want.T, O.N_E4)
+
+
+@pytest.mark.parametrize("kind,conv,margin", [(O.E4, O.CONV_PAPER, 0), (O.E4, O.CONV_NATIVE, 0), (O.E5, O.CONV_PAPER, 0),
+                                              (O.E5, O.CONV_PAPER, 3)])
+@pytest.mark.parametrize("std", [1e-5, 0.02, 1.0, 4000.0])
+def test_fused_amax_bias_cast(ctx, lib, kind, conv, margin, std):
+    """FP8-AMAX in one call: amax, bias and bytes all equal the oracle's."""
+    g = torch.Generator(device="cuda").manual_seed(int(std * 1e6) % 9973 + kind)
+    x = (torch.randn((384, 640), generator=g, device="cuda") * std).to(torch.bfloat16)
+    a, b, want, want_t = O.quantise(bits_of(x), kind, conv, margin, transposed=True)
+    amax = _dev_scalar(torch.float32, -1.0)
+    bias = _dev_scalar(torch.int32, 777)
+    y = torch.empty((384, 640), dtype=torch.uint8, device="cuda")
+    y_t = torch.empty((640, 384), dtype=torch.uint8, device="cuda")
+    cast = ctx.cast_e4 if kind == O.E4 else ctx.cast_e5
+    cast(x, None, conv=conv, margin=margin, d_amax_out=amax, d_bias_out=bias, y=y, y_t=y_t)
+    assert float(amax.item()) == a and int(bias.item()) == b
+    assert_codes_equal(u8(y), want, O.native_format(kind))
+    assert_codes_equal(u8(y_t), want_t, O.native_format(kind))
+    y.zero_()
+    cast(x, None, conv=conv, margin=margin, d_amax_out=amax, d_bias_out=bias, y=y)
+    assert_codes_equal(u8(y), want, O.native_format(kind))
+
+
+def test_ptq_weights_equals_separate_steps(ctx, lib):
+    g = torch.Generator(device="cuda").manual_seed(23)
+    w = (torch.randn((768, 512), generator=g, device="cuda") * 0.015).to(torch.bfloat16)
+    a, b, want, want_t = O.quantise(bits_of(w), O.E4, O.CONV_PAPER, 0, transposed=True)
+    w8 = torch.empty((768, 512), dtype=torch.uint8, device="cuda")
+    w8_t = torch.empty((512, 768), dtype=torch.uint8, device="cuda")
+    amax = _dev_scalar(torch.float32)
+    bias = _dev_scalar(torch.int32)
+    ctx.ptq_weights(w, lib.CONV_PAPER, w8, w8_t, bias, amax)
+    assert float(amax.item()) == a and int(bias.item()) == b
+    assert_codes_equal(u8(w8), want, O.N_E4)
+    assert_codes_equal(u8(w8_t), want_t, O.N_E4)
+    # the same through the separate entry points
+    amax2, bias2 = _dev_scalar(torch.float32), _dev_scalar(torch.int32)
+    w8b = torch.empty_like(w8)
+    ctx.amax(w, amax2)
+    ctx.scaling_bias(amax2, lib.E4, lib.CONV_PAPER, 0, bias2)
+    ctx.cast_e4(w, bias2, y=w8b)
+    assert torch.equal(w8, w8b) and int(bias2.item()) == b
+
+
+def test_saturation_flag_and_constant_scale(ctx, lib):
+    """A caller-chosen constant bias (FP8-CSCALE) that is too large clips and
+    raises the sticky flag; a safe one does not."""
+    ctx.device_flags(clear=True)
+    x = torch.full((64, 64), 3.0, dtype=torch.bfloat16, device="cuda")
+    y = torch.empty((64, 64), dtype=torch.uint8, device="cuda")
+    bias = _dev_scalar(torch.int32, 2)
+    ctx.cast_e4(x, bias, y=y)
+    assert ctx.device_flags() == 0
+    assert_codes_equal(u8(y), O.cast(bits_of(x), 3, O.N_E4), O.N_E4)
+    bias.fill_(9)  # 3 * 2^10 = 3072 > 448
+    ctx.cast_e4(x, bias, y=y)
+    assert ctx.device_flags() & lib.FLAG_SATURATED
+    assert bool((y == 0x7E).all())
+
+
+def test_argument_errors(ctx, lib):
+    x = torch.zeros((16, 16), dtype=torch.bfloat16, device="cuda")
+    y = torch.zeros((16, 16), dtype=torch.uint8, device="cuda")
+    bias = _dev_scalar(torch.int32)
+    with pytest.raises(lib.Fp8Error) as e:
+        ctx.cast_e4(x, bias, y=None, y_t=None)
+    assert e.value.status == lib.ERR_NULL
+    with pytest.raises(lib.Fp8Error) as e:
+        ctx.cast_e4(x, None, y=y)  # FP8-AMAX needs somewhere to put amax and bias
+    assert e.value.status == lib.ERR_NULL
+    with pytest.raises(lib.Fp8Error) as e:
+        ctx.cast_e4(x, bias, y=y, rows=16, cols=16, ld=8)
+    assert e.value.status == lib.ERR_SHAPE
+    with pytest.raises(lib.Fp8Error) as e:
+        ctx.amax(x.float(), _dev_scalar(torch.float32))
+    assert e.value.status == lib.ERR_UNSUPPORTED

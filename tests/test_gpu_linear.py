@@ -1,0 +1,188 @@
+"""GPU parity: the three FP8 matmuls with unscale against the CPU oracle.
+
+Both sides start from the same seeded bf16 tensors.  The FP8 bytes and biases
+must agree bit for bit; FP32 outputs must lie within 2^-14 * sum_k |a*b| of
+the exact value; bf16 outputs within one bf16 ulp of the oracle's rounding.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle as O
+from helpers import (assert_bf16_within_one_ulp, assert_codes_equal, assert_gemm_close, bits_of, u8)
+from paper_2309_17224_b200 import inputs as I
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_2309_17224_b200 import fp8lin
+    return fp8lin
+
+
+@pytest.fixture(scope="module")
+def ctx(lib):
+    c = lib.Context(0)
+    yield c
+    c.close()
+
+
+class Quantised:
+    """One tensor quantised on the GPU (both layouts) and by the oracle."""
+
+    def __init__(self, ctx, x, kind, conv, margin=0):
+        rows, cols = x.shape
+        self.kind, self.conv = kind, conv
+        self.amax = torch.zeros(1, dtype=torch.float32, device="cuda")
+        self.bias = torch.zeros(1, dtype=torch.int32, device="cuda")
+        self.y = torch.empty((rows, cols), dtype=torch.uint8, device="cuda")
+        self.y_t = torch.empty((cols, rows), dtype=torch.uint8, device="cuda")
+        cast = ctx.cast_e4 if kind == O.E4 else ctx.cast_e5
+        cast(x, None, conv=conv, margin=margin, d_amax_out=self.amax, d_bias_out=self.bias, y=self.y, y_t=self.y_t)
+        a, b, ref, ref_t = O.quantise(bits_of(x), kind, conv, margin, transposed=True)
+        assert float(self.amax.item()) == a and int(self.bias.item()) == b
+        fmt = O.native_format(kind)
+        assert_codes_equal(u8(self.y), ref, fmt)
+        assert_codes_equal(u8(self.y_t), ref_t, fmt)
+        self.ref, self.ref_bias, self.shift = ref, b, b + O.delta(kind, conv)
+
+
+def _layer(ctx, T, K, N, conv, seed, x_std=1.0, w_std=0.02, g_std=1e-3, margin=0):
+    x = I.normal_bf16(T, K, x_std, seed, 1, "cuda", outlier_frac=0.01, outlier_scale=50.0)
+    w = I.normal_bf16(N, K, w_std, seed, 2, "cuda")
+    g = I.normal_bf16(T, N, g_std, seed, 3, "cuda")
+    return (Quantised(ctx, x, O.E4, conv), Quantised(ctx, w, O.E4, conv), Quantised(ctx, g, O.E5, conv, margin))
+
+
+SHAPES = [
+    (256, 768, 768),     # config 1
+    (128, 128, 256),     # exactly one tile, one k-block
+    (128, 16, 256),      # shortest contraction the API allows
+    (144, 272, 528),     # ragged in every dimension (multiples of 16 where the layout needs it)
+    (400, 1040, 784),    # several tiles, several k-blocks, ragged tails
+    (16, 2048, 48),      # skinny
+]
+
+
+@pytest.mark.parametrize("T,K,N", SHAPES)
+@pytest.mark.parametrize("conv", [O.CONV_PAPER, O.CONV_NATIVE])
+def test_fwd_dgrad_wgrad_match_oracle(ctx, lib, T, K, N, conv):
+    qx, qw, qg = _layer(ctx, T, K, N, conv, seed=T * 1000003 + K * 101 + N)
+    for dt in (torch.float32, torch.bfloat16):
+        y = torch.full((T, N), float("nan"), dtype=dt, device="cuda")
+        dx = torch.full((T, K), float("nan"), dtype=dt, device="cuda")
+        dw = torch.full((N, K), float("nan"), dtype=dt, device="cuda")
+        ctx.linear_fwd(qx.y, qx.bias, qw.y, qw.bias, y, conv=conv)
+        ctx.linear_dgrad(qg.y, qg.bias, None, qw.y_t, qw.bias, dx, conv=conv)
+        ctx.linear_wgrad(None, qg.y_t, qg.bias, None, qx.y_t, qx.bias, dw, T, conv=conv)
+        assert ctx.device_flags(clear=True) & lib.FLAG_TIMEOUT == 0
+        refs = (O.linear_fwd(qx.ref, qx.shift, qw.ref, qw.shift),
+                O.linear_dgrad(qg.ref, qg.shift, qw.ref, qw.shift),
+                O.linear_wgrad(qg.ref, qg.shift, qx.ref, qx.shift))
+        for got, ref in zip((y, dx, dw), refs):
+            if dt == torch.float32:
+                assert_gemm_close(got.cpu().numpy(), ref)
+            else:
+                assert_bf16_within_one_ulp(bits_of(got), ref)
+
+
+def test_fwd_bias_vector_and_output_amax(ctx, lib):
+    T, K, N = 200, 512, 300
+    qx, qw, _ = _layer(ctx, T, K, N + 4, O.CONV_PAPER, seed=99)
+    w8 = qw.y[:N].contiguous()
+    for bias_dt in (torch.bfloat16, torch.float32):
+        bv = (torch.randn(N, device="cuda") * 0.5).to(bias_dt)
+        ref = O.linear_fwd(qx.ref, qx.shift, qw.ref[:N], qw.shift, bias_vec=bv.double().cpu().numpy())
+        for dt in (torch.float32, torch.bfloat16):
+            y = torch.empty((T, N), dtype=dt, device="cuda")
+            amax_y = torch.full((1,), 123.0, dtype=torch.float32, device="cuda")
+            ctx.linear_fwd(qx.y, qx.bias, w8, qw.bias, y, bias_vec=bv, d_amax_y=amax_y)
+            if dt == torch.float32:
+                assert_gemm_close(y.cpu().numpy(), ref)
+            else:
+                assert_bf16_within_one_ulp(bits_of(y), ref)
+            # the emitted amax is exactly the amax of what was written
+            assert float(amax_y.item()) == float(y.float().abs().max().item())
+
+
+def test_dgrad_amax_and_margin(ctx, lib):
+    T, K, N = 256, 384, 512
+    qx, qw, qg = _layer(ctx, T, K, N, O.CONV_PAPER, seed=5, margin=3)
+    dx = torch.empty((T, K), dtype=torch.bfloat16, device="cuda")
+    amax_dx = torch.zeros(1, dtype=torch.float32, device="cuda")
+    ctx.linear_dgrad(qg.y, qg.bias, None, qw.y_t, qw.bias, dx, d_amax_dx=amax_dx)
+    assert_bf16_within_one_ulp(bits_of(dx), O.linear_dgrad(qg.ref, qg.shift, qw.ref, qw.shift))
+    assert float(amax_dx.item()) == float(dx.float().abs().max().item())
+
+
+def test_extreme_biases_unscale_exactly(ctx, lib):
+    """Tensors near the ends of the bf16 range: biases beyond +-126 need the
+    two-step power-of-two unscale."""
+    T, K, N = 128, 64, 256
+    x = I.normal_bf16(T, K, 2.0 ** -120, 7, 1, "cuda")
+    w = I.normal_bf16(N, K, 2.0 ** 100, 7, 2, "cuda")
+    qx, qw = Quantised(ctx, x, O.E4, O.CONV_PAPER), Quantised(ctx, w, O.E4, O.CONV_PAPER)
+    assert qx.ref_bias > 110 and qw.ref_bias < -90
+    y = torch.empty((T, N), dtype=torch.float32, device="cuda")
+    ctx.linear_fwd(qx.y, qx.bias, qw.y, qw.bias, y)
+    assert_gemm_close(y.cpu().numpy(), O.linear_fwd(qx.ref, qx.shift, qw.ref, qw.shift))
+    tiny = I.normal_bf16(T, K, 2.0 ** -125, 7, 4, "cuda")
+    qt = Quantised(ctx, tiny, O.E4, O.CONV_PAPER)
+    # tiny x tiny: the unscale exponent is beyond -126 and the result underflows FP32
+    out = torch.empty((T, T), dtype=torch.float32, device="cuda")
+    ctx.linear_fwd(qt.y, qt.bias, qx.y, qx.bias, out)
+    assert_gemm_close(out.cpu().numpy(), O.linear_fwd(qt.ref, qt.shift, qx.ref, qx.shift))
+
+
+def test_matmul_argument_errors(ctx, lib):
+    x8 = torch.zeros((32, 24), dtype=torch.uint8, device="cuda")   # K = 24 is not a multiple of 16
+    w8 = torch.zeros((64, 24), dtype=torch.uint8, device="cuda")
+    b = torch.zeros(1, dtype=torch.int32, device="cuda")
+    y = torch.zeros((32, 64), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(lib.Fp8Error) as e:
+        ctx.linear_fwd(x8, b, w8, b, y)
+    assert e.value.status == lib.ERR_ALIGN
+    g8 = torch.zeros((32, 64), dtype=torch.uint8, device="cuda")
+    dx = torch.zeros((32, 32), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(lib.Fp8Error) as e:
+        ctx.linear_dgrad(g8, b, w8, None, b, dx)   # only the [N,K] layout given
+    assert e.value.status == lib.ERR_UNSUPPORTED
+    with pytest.raises(lib.Fp8Error) as e:
+        ctx.linear_fwd(x8, None, w8, b, y)
+    assert e.value.status == lib.ERR_NULL
+
+
+def _sample_positions(rng, R, C, n):
+    rows = np.concatenate([rng.integers(0, R, n), [0, R - 1, 0, R - 1]])
+    cols = np.concatenate([rng.integers(0, C, n), [0, C - 1, C - 1, 0]])
+    return rows, cols
+
+
+@pytest.mark.parametrize("wl_name,layer", [("c2_gpt", 0), ("c2_gpt", 3), ("c3_llama7b", 1), ("c3_llama7b", 3)])
+def test_full_size_layers_sampled(ctx, lib, wl_name, layer):
+    """Benchmark-size layers in the benchmark's launch configuration: bytes and
+    biases checked in full, matmul outputs at sampled positions."""
+    wl = I.WORKLOADS[wl_name]
+    l = wl.layers[layer]
+    T, K, N = wl.tokens, l.K, l.N
+    t = I.layer_tensors(wl, layer, device="cuda")
+    qx = Quantised(ctx, t["x"], O.E4, O.CONV_PAPER)
+    qw = Quantised(ctx, t["w"], O.E4, O.CONV_PAPER)
+    qg = Quantised(ctx, t["g"], O.E5, O.CONV_PAPER)
+    y = torch.empty((T, N), dtype=torch.bfloat16, device="cuda")
+    dx = torch.empty((T, K), dtype=torch.bfloat16, device="cuda")
+    dw = torch.empty((N, K), dtype=torch.bfloat16, device="cuda")
+    ctx.linear_fwd(qx.y, qx.bias, qw.y, qw.bias, y)
+    ctx.linear_dgrad(qg.y, qg.bias, None, qw.y_t, qw.bias, dx)
+    ctx.linear_wgrad(None, qg.y_t, qg.bias, None, qx.y_t, qx.bias, dw, T)
+    assert ctx.device_flags(clear=True) & lib.FLAG_TIMEOUT == 0
+    rng = np.random.default_rng(layer + 1)
+    cases = ((O.FWD, y, (qx.ref, O.N_E4, qx.shift, qw.ref, O.N_E4, qw.shift)),
+             (O.DGRAD, dx, (qg.ref, O.N_E5, qg.shift, qw.ref, O.N_E4, qw.shift)),
+             (O.WGRAD, dw, (qg.ref, O.N_E5, qg.shift, qx.ref, O.N_E4, qx.shift)))
+    for kind, out, ops in cases:
+        rows, cols = _sample_positions(rng, out.shape[0], out.shape[1], 4000)
+        ref = O.linear_samples(kind, *ops, rows, cols)
+        got = bits_of(out)[rows, cols]
+        assert_bf16_within_one_ulp(got, ref)

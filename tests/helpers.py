@@ -50,11 +50,22 @@ def assert_gemm_close(got_f32: np.ndarray, ref: "O.GemmResult"):
     return float((err / np.maximum(ref.abs_sum, 1e-300)).max())
 
 
+def bf16_bits_to_f64(b: np.ndarray) -> np.ndarray:
+    return (b.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+
+
 def assert_bf16_within_one_ulp(got_bits: np.ndarray, ref: "O.GemmResult"):
+    """bf16 output within one bf16 ulp of the oracle's rounded value.  Where the
+    sum cancels, one bf16 ulp of the result is finer than the FP32 accumulation
+    bar (2^-14 * sum_k |a*b|); there that bar, plus the half ulp of the output
+    rounding itself, is the one that applies."""
     d = np.abs(bf16_ordinal(got_bits) - bf16_ordinal(ref.bf16))
-    bad = d > 1
+    got = bf16_bits_to_f64(got_bits)
+    half_ulp = np.abs(ref.f64) * 2.0 ** -8
+    within_acc = np.abs(got - ref.f64) <= ref.abs_sum * 2.0 ** -14 + half_ulp + 2.0 ** -150
+    bad = (d > 1) & ~within_acc
     if bad.any():
         i = np.argwhere(bad)[0]
         raise AssertionError(f"{bad.sum()} bf16 outputs differ by more than one ulp; first at {i.tolist()}: "
                              f"got {hex(got_bits[tuple(i)])} want {hex(ref.bf16[tuple(i)])}")
-    return float((d > 0).mean())
+    return float((d > 1).mean())

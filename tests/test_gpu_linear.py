@@ -82,7 +82,8 @@ def test_fwd_dgrad_wgrad_match_oracle(ctx, lib, T, K, N, conv):
                 O.linear_wgrad(qg.ref, qg.shift, qx.ref, qx.shift))
         for got, ref in zip((y, dx, dw), refs):
             if dt == torch.float32:
-                assert_gemm_close(got.cpu().numpy(), ref)
+                worst = assert_gemm_close(got.cpu().numpy(), ref)
+                print(f"[parity] T={T} K={K} N={N} conv={conv}: max |err| / sum|a*b| = 2^{np.log2(max(worst, 1e-300)):.1f}")
             else:
                 assert_bf16_within_one_ulp(bits_of(got), ref)
 

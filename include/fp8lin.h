@@ -53,7 +53,8 @@ typedef enum {
     FP8_ERR_DTYPE = 4,          /* enum value out of range */
     FP8_ERR_UNSUPPORTED = 5,    /* valid request that this build has no kernel for (there is no fallback path) */
     FP8_ERR_CUDA = 6,           /* a CUDA runtime / driver call failed (launch, attribute, tensor-map encode) */
-    FP8_ERR_DEVICE_TIMEOUT = 7  /* reported by fp8_device_flags when a bounded device-side wait expired */
+    FP8_ERR_DEVICE_TIMEOUT = 7, /* reported by fp8_device_flags when a bounded device-side wait expired */
+    FP8_ERR_TOO_LARGE = 8       /* tensor exceeds the fixed workspace of fp8_amax_noalloc */
 } fp8_status_t;
 
 typedef enum { FP8_E4 = 0, FP8_E5 = 1 } fp8_format_t;
@@ -95,6 +96,31 @@ FP8_API fp8_status_t fp8_device_flags(fp8_ctx *ctx, void *stream, unsigned *flag
  * cols multiples of 8) takes the vectorised path. */
 FP8_API fp8_status_t fp8_amax(fp8_ctx *ctx, const void *x, fp8_dtype_t x_dt, int64_t rows, int64_t cols, int64_t ld,
                       float *d_amax, void *stream);
+
+/* amax for callers that cannot allocate device memory (the paper has no
+ * counterpart; this exists for deployment).  fp8_amax needs an fp8_ctx, and
+ * fp8_create calls cudaMalloc for the reduction workspace.  Programs that have
+ * handed all device memory to their own allocator, that must not call
+ * cudaMalloc on a serving thread (it synchronises the whole device), or that
+ * run as a plug-in without an allocator can use this entry point instead: it
+ * takes no context and calls no cudaMalloc, cudaFree or any other allocating
+ * routine.  Its workspace is a 32 KiB array inside the library's device image,
+ * which every GPU that loads the library holds until the process exits.
+ *   x       [rows, cols] bf16, contiguous (ld == cols), 16-byte aligned
+ *   d_amax  out, one float, same value as fp8_amax writes
+ * Limits and rules:
+ *   - at most 2^29 elements (1 GiB of bf16): one partial maximum per
+ *     65 536-element chunk, 8192 chunks.  Larger tensors return
+ *     FP8_ERR_TOO_LARGE and nothing is launched.
+ *   - the first call on each device looks up the array's device address
+ *     (with that device current); make that first call before any stream
+ *     capture begins.  The launch goes to the current device.
+ *   - all calls on a device share the one array: calls whose kernels may
+ *     overlap on the GPU (different streams with no ordering between them)
+ *     race and give wrong results.  Calls ordered on one stream, or by
+ *     events, are safe; each call leaves the array ready for the next. */
+FP8_API fp8_status_t fp8_amax_noalloc(const void *x, fp8_dtype_t x_dt, int64_t rows, int64_t cols, int64_t ld,
+                                      float *d_amax, void *stream);
 
 /* scaling_bias = floor(log2(max_num / amax)) - margin (Eq. 3, second line;
  * the margin is the one of Section 3.2), evaluated exactly on the bits of

@@ -20,6 +20,7 @@ const char *fp8_status_string(fp8_status_t s)
     case FP8_ERR_UNSUPPORTED: return "no kernel for this request";
     case FP8_ERR_CUDA: return "CUDA call failed";
     case FP8_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait expired";
+    case FP8_ERR_TOO_LARGE: return "tensor exceeds the fixed workspace of the no-allocation entry point";
     }
     return "unknown status";
 }

@@ -18,7 +18,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libfp8lin.so")
 
 OK = 0
-ERR_NULL, ERR_SHAPE, ERR_ALIGN, ERR_DTYPE, ERR_UNSUPPORTED, ERR_CUDA, ERR_DEVICE_TIMEOUT = range(1, 8)
+ERR_NULL, ERR_SHAPE, ERR_ALIGN, ERR_DTYPE, ERR_UNSUPPORTED, ERR_CUDA, ERR_DEVICE_TIMEOUT, ERR_TOO_LARGE = range(1, 9)
 E4, E5 = 0, 1
 CONV_PAPER, CONV_NATIVE = 0, 1
 BF16, F16, F32 = 0, 1, 2
@@ -27,7 +27,7 @@ FLAG_NONFINITE_AMAX, FLAG_ZERO_AMAX, FLAG_SATURATED, FLAG_TIMEOUT = 1, 2, 4, 8
 SYMBOLS = (
     "fp8_create", "fp8_destroy", "fp8_status_string", "fp8_device_flags", "fp8_amax", "fp8_scaling_bias",
     "fp8_scaling_bias_host", "fp8_cast_e4", "fp8_cast_e5", "fp8_ptq_weights", "fp8_linear_fwd", "fp8_linear_dgrad",
-    "fp8_linear_wgrad",
+    "fp8_linear_wgrad", "fp8_amax_noalloc",
 )
 
 if not os.path.exists(LIB_PATH):
@@ -44,6 +44,7 @@ _lib.fp8_status_string.argtypes = [c_int]
 _lib.fp8_status_string.restype = c_char_p
 _lib.fp8_device_flags.argtypes = [_P, _P, POINTER(c_uint), c_int]
 _lib.fp8_amax.argtypes = [_P, _P, c_int, c_int64, c_int64, c_int64, _P, _P]
+_lib.fp8_amax_noalloc.argtypes = [_P, c_int, c_int64, c_int64, c_int64, _P, _P]
 _lib.fp8_scaling_bias.argtypes = [_P, _P, c_int, c_int, c_int32, _P, _P]
 _lib.fp8_scaling_bias_host.argtypes = [c_float, c_int, c_int, c_int32, POINTER(c_int32)]
 _cast_args = [_P, _P, c_int, c_int64, c_int64, c_int64, _P, c_int, c_int32, _P, _P, _P, _P, _P]
@@ -84,10 +85,26 @@ def _stream():
 _DT = {torch.bfloat16: BF16, torch.float16: F16, torch.float32: F32}
 
 
+def _ld(x):
+    """Leading dimension of a 2-D tensor (torch leaves the stride of a size-1 dimension arbitrary)."""
+    return x.stride(0) if x.shape[0] > 1 else x.shape[1]
+
+
 def scaling_bias_host(amax: float, fmt: int, conv: int = CONV_PAPER, margin: int = 0) -> int:
     out = c_int32(0)
     _check(_lib.fp8_scaling_bias_host(c_float(amax), fmt, conv, margin, byref(out)), "fp8_scaling_bias_host")
     return out.value
+
+
+def amax_noalloc(x, d_amax, rows=None, cols=None, ld=None):
+    """``fp8_amax_noalloc``: amax without a context and without any device
+    allocation by the library (for callers that own all device memory or may
+    not call cudaMalloc).  Contiguous bf16 input of at most 2^29 elements;
+    calls on one device must not overlap on the GPU."""
+    rows = x.shape[0] if rows is None else rows
+    cols = x.shape[1] if cols is None else cols
+    ld = _ld(x) if ld is None else ld
+    _check(_lib.fp8_amax_noalloc(_ptr(x), _DT[x.dtype], rows, cols, ld, _ptr(d_amax), _stream()), "fp8_amax_noalloc")
 
 
 class Context:
@@ -121,7 +138,7 @@ class Context:
     def amax(self, x, d_amax, rows=None, cols=None, ld=None):
         rows = x.shape[0] if rows is None else rows
         cols = x.shape[1] if cols is None else cols
-        ld = x.stride(0) if ld is None else ld
+        ld = _ld(x) if ld is None else ld
         _check(_lib.fp8_amax(self._h, _ptr(x), _DT[x.dtype], rows, cols, ld, _ptr(d_amax), _stream()), "fp8_amax")
 
     def scaling_bias(self, d_amax, fmt, conv, margin, d_bias):
@@ -132,7 +149,7 @@ class Context:
     def _cast(self, fn, name, x, d_bias, conv, margin, d_amax_out, d_bias_out, y, y_t, rows, cols, ld):
         rows = x.shape[0] if rows is None else rows
         cols = x.shape[1] if cols is None else cols
-        ld = x.stride(0) if ld is None else ld
+        ld = _ld(x) if ld is None else ld
         _check(fn(self._h, _ptr(x), _DT[x.dtype], rows, cols, ld, _ptr(d_bias), conv, margin, _ptr(d_amax_out),
                   _ptr(d_bias_out), _ptr(y), _ptr(y_t), _stream()), name)
 
@@ -147,7 +164,7 @@ class Context:
                    cols, ld)
 
     def ptq_weights(self, w, conv, w8, w8_t, d_bw, d_amax_w):
-        _check(_lib.fp8_ptq_weights(self._h, _ptr(w), _DT[w.dtype], w.shape[0], w.shape[1], w.stride(0), conv,
+        _check(_lib.fp8_ptq_weights(self._h, _ptr(w), _DT[w.dtype], w.shape[0], w.shape[1], _ld(w), conv,
                                     _ptr(w8), _ptr(w8_t), _ptr(d_bw), _ptr(d_amax_w), _stream()), "fp8_ptq_weights")
 
     # -- matmuls ----------------------------------------------------------------

@@ -21,6 +21,9 @@
 // Every wait on an mbarrier is bounded: when it expires the CTA raises
 // FP8_FLAG_TIMEOUT in the status word, all roles leave their loops, tensor
 // memory is released and the kernel returns.
+#include <cstdio>
+#include <cstdlib>
+
 #include "fp8lin_internal.cuh"
 
 namespace fp8lin {
@@ -202,6 +205,73 @@ __device__ __forceinline__ void tile_coords(int tile, const GemmParams &p, int &
     n_blk = r / gm;
 }
 
+// One 32-column chunk of one accumulator row: unscale by the exact power of
+// two, optional bias vector, rounding to the output type, running amax of the
+// rounded values, store.
+__device__ __forceinline__ void epilogue_chunk(const uint32_t (&r)[32], int row, int col0, const GemmParams &p,
+                                               const Pow2Pair sc, bool two_step, uint32_t &amax_bits)
+{
+    if (row >= p.M || col0 >= p.N) return;
+    float v[32];
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {
+        v[i] = __uint_as_float(r[i]) * sc.first;
+        if (two_step) v[i] *= sc.second;
+    }
+    if (p.bias_vec) {
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+            if (col0 + i < p.N) {
+                float b = p.bias_dt == FP8_F32
+                              ? __ldg(reinterpret_cast<const float *>(p.bias_vec) + col0 + i)
+                              : __uint_as_float(
+                                    (uint32_t)__ldg(reinterpret_cast<const uint16_t *>(p.bias_vec) + col0 + i) << 16);
+                v[i] += b;
+            }
+        }
+    }
+    if (p.out_dt == FP8_BF16) {
+        uint32_t w[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i)
+            asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(w[i]) : "f"(v[2 * i + 1]), "f"(v[2 * i]));
+        if (p.d_amax_bits) {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                uint32_t a = w[i] & 0x7FFF7FFFu;
+                if (col0 + 2 * i < p.N) amax_bits = max(amax_bits, (a & 0xFFFFu) << 16);
+                if (col0 + 2 * i + 1 < p.N) amax_bits = max(amax_bits, a & 0xFFFF0000u);
+            }
+        }
+        uint16_t *dst = reinterpret_cast<uint16_t *>(p.out) + (int64_t)row * p.ldo + col0;
+        if (p.vec_ok && col0 + 32 <= p.N) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                reinterpret_cast<uint4 *>(dst)[j] = make_uint4(w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
+        } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+                if (col0 + i < p.N) dst[i] = (uint16_t)((i & 1) ? (w[i >> 1] >> 16) : (w[i >> 1] & 0xFFFFu));
+        }
+    } else {
+        if (p.d_amax_bits) {
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+                if (col0 + i < p.N) amax_bits = max(amax_bits, __float_as_uint(v[i]) & 0x7FFFFFFFu);
+        }
+        float *dst = reinterpret_cast<float *>(p.out) + (int64_t)row * p.ldo + col0;
+        if (p.vec_ok && col0 + 32 <= p.N) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+                reinterpret_cast<float4 *>(dst)[j] = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+        } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+                if (col0 + i < p.N) dst[i] = v[i];
+        }
+    }
+}
+
 template <int BN, int STAGES>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const GemmParams p)
@@ -312,68 +382,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                     __syncwarp();
                     if (lane == 0) mbar_arrive(acc_empty_bar(buf));
                 }
-                const int col0 = n_blk * BN + c;
-                if (row >= p.M || col0 >= p.N) continue;
-                float v[32];
-#pragma unroll
-                for (int i = 0; i < 32; ++i) {
-                    v[i] = __uint_as_float(r[i]) * sc.first;
-                    if (two_step) v[i] *= sc.second;
-                }
-                if (p.bias_vec) {
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) {
-                        if (col0 + i < p.N) {
-                            float b = p.bias_dt == FP8_F32
-                                          ? __ldg(reinterpret_cast<const float *>(p.bias_vec) + col0 + i)
-                                          : __uint_as_float(
-                                                (uint32_t)__ldg(reinterpret_cast<const uint16_t *>(p.bias_vec) + col0 + i)
-                                                << 16);
-                            v[i] += b;
-                        }
-                    }
-                }
-                if (p.out_dt == FP8_BF16) {
-                    uint32_t w[16];
-#pragma unroll
-                    for (int i = 0; i < 16; ++i) {
-                        asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(w[i]) : "f"(v[2 * i + 1]), "f"(v[2 * i]));
-                    }
-                    if (p.d_amax_bits) {
-#pragma unroll
-                        for (int i = 0; i < 16; ++i) {
-                            uint32_t a = w[i] & 0x7FFF7FFFu;
-                            if (col0 + 2 * i < p.N) amax_bits = max(amax_bits, (a & 0xFFFFu) << 16);
-                            if (col0 + 2 * i + 1 < p.N) amax_bits = max(amax_bits, a & 0xFFFF0000u);
-                        }
-                    }
-                    uint16_t *dst = reinterpret_cast<uint16_t *>(p.out) + (int64_t)row * p.ldo + col0;
-                    if (p.vec_ok && col0 + 32 <= p.N) {
-#pragma unroll
-                        for (int j = 0; j < 4; ++j)
-                            reinterpret_cast<uint4 *>(dst)[j] = make_uint4(w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
-                    } else {
-#pragma unroll
-                        for (int i = 0; i < 32; ++i)
-                            if (col0 + i < p.N) dst[i] = (uint16_t)((i & 1) ? (w[i >> 1] >> 16) : (w[i >> 1] & 0xFFFFu));
-                    }
-                } else {
-                    if (p.d_amax_bits) {
-#pragma unroll
-                        for (int i = 0; i < 32; ++i)
-                            if (col0 + i < p.N) amax_bits = max(amax_bits, __float_as_uint(v[i]) & 0x7FFFFFFFu);
-                    }
-                    float *dst = reinterpret_cast<float *>(p.out) + (int64_t)row * p.ldo + col0;
-                    if (p.vec_ok && col0 + 32 <= p.N) {
-#pragma unroll
-                        for (int j = 0; j < 8; ++j)
-                            reinterpret_cast<float4 *>(dst)[j] = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
-                    } else {
-#pragma unroll
-                        for (int i = 0; i < 32; ++i)
-                            if (col0 + i < p.N) dst[i] = v[i];
-                    }
-                }
+                epilogue_chunk(r, row, n_blk * BN + c, p, sc, two_step, amax_bits);
             }
         }
         if (p.d_amax_bits) {
@@ -391,6 +400,244 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     if (warp == 1) tmem_dealloc(tmem_base, L::kTmemCols);
 }
 
+
+// ---------------------------------------------------------------------------
+// CTA-pair kernel (cta_group::2)
+// ---------------------------------------------------------------------------
+//
+// Two CTAs of a cluster share one 256x256 output tile.  Each loads its own 128
+// rows of A and its own 128 of the 256 B rows (so a stage is 32 KB per CTA and
+// the shared-memory pipe carries 64 B/clk of MMA reads plus 64 B/clk of TMA
+// writes instead of 96 + 96); the leader CTA's MMA thread issues
+// tcgen05.mma.cta_group::2 (M=256, N=256, K=32), which reads both CTAs' shared
+// memory and writes each CTA's 128 accumulator rows into that CTA's TMEM.
+//
+// Signalling: the "stage full" barrier lives in the leader and takes one
+// arrive.expect_tx from the leader's producer for the bytes of all four TMA
+// loads (the peer's loads name the leader's barrier, which cta_group::2 loads
+// may do); "stage empty" and "accumulator full" are tcgen05.commit multicast to
+// the same barrier offset in both CTAs; "accumulator empty" lives in the leader
+// and collects one arrival per epilogue warp of both CTAs.  None of the loads
+// is a multicast load.
+
+constexpr int kPairStages = 6;
+constexpr int kPairBN = 256;       // N of the pair tile (and of the instruction)
+constexpr int kPairHalfN = 128;    // B rows each CTA loads
+
+struct PairSmem {
+    static constexpr int kABytes = kBM * kBK;
+    static constexpr int kBBytes = kPairHalfN * kBK;
+    static constexpr int kStageBytes = kABytes + kBBytes;
+    static constexpr int kBarOffset = kPairStages * kStageBytes;
+    static constexpr int kNumBars = 2 * kPairStages + 4;
+    static constexpr int kTotal = kBarOffset + kNumBars * 8 + 16;
+    static constexpr int kDynamic = kTotal + 1024;
+    static constexpr int kTmemCols = 512;
+};
+
+__device__ __forceinline__ uint32_t cluster_ctarank()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t rank)
+{
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// arrive (+ expected bytes) on a barrier addressed in the cluster window
+__device__ __forceinline__ void mbar_expect_tx_cluster(uint32_t cluster_bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.release.cluster.shared::cluster.b64 _, [%0], %1;" ::"r"(cluster_bar),
+                 "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_bar)
+{
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
+}
+// TMA load whose completion bytes may be counted on the pair leader's barrier
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap *map, uint32_t cluster_bar, int x, int y)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes"
+        " [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(cluster_bar), "r"(x), "r"(y)
+        : "memory");
+}
+__device__ __forceinline__ void umma_f8_pair(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc,
+                                             uint32_t accumulate)
+{
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "setp.ne.b32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::2.kind::f8f6f4 [%0], %1, %2, %3, p;\n"
+        "}\n"
+        ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// arrive on the barrier at this offset in both CTAs of the pair once all MMAs issued so far have completed
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar)
+{
+    asm volatile(
+        "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+        ::"r"(bar), "h"((uint16_t)3)
+        : "memory");
+}
+
+__host__ __device__ inline uint32_t make_idesc_pair(int a_fmt, int b_fmt)
+{
+    return (1u << 4) | ((uint32_t)a_fmt << 7) | ((uint32_t)b_fmt << 10) | ((uint32_t)(kPairBN >> 3) << 17) |
+           ((uint32_t)(256 >> 4) << 24);
+}
+
+// tiles here are 256 x 256; p.tiles_m / p.tiles_n count those
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1)
+gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                 const GemmParams p)
+{
+    using L = PairSmem;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    const uint32_t smem_base = smem_u32(smem);
+    const uint32_t bar_base = smem_base + L::kBarOffset;
+    auto full_bar = [&](int s) { return bar_base + 8u * s; };
+    auto empty_bar = [&](int s) { return bar_base + 8u * (kPairStages + s); };
+    auto acc_full_bar = [&](int b) { return bar_base + 8u * (2 * kPairStages + b); };
+    auto acc_empty_bar = [&](int b) { return bar_base + 8u * (2 * kPairStages + 2 + b); };
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + L::kBarOffset + L::kNumBars * 8);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank();
+    const int num_tiles = p.tiles_m * p.tiles_n;
+    const int pair_id = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kPairStages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(acc_full_bar(b), 1); mbar_init(acc_empty_bar(b), 8); }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                     "r"((uint32_t)L::kTmemCols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();  // both CTAs' barriers exist before anyone signals across
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_a)) : "memory");
+            asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_b)) : "memory");
+            uint32_t it = 0;
+            bool alive = true;
+            const uint32_t leader_full0 = map_to_cta(full_bar(0), 0);
+            for (int tile = pair_id; alive && tile < num_tiles; tile += num_pairs) {
+                int m_blk, n_blk;
+                tile_coords(tile, p, m_blk, n_blk);
+                for (int k = 0; k < p.num_k; ++k, ++it) {
+                    const int s = it % kPairStages;
+                    const uint32_t leader_full = leader_full0 + 8u * s;
+                    const uint32_t ph = (it / kPairStages) & 1u;
+                    if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p.d_status)) { alive = false; break; }
+                    // only the leader arrives, announcing the bytes of all four loads of the pair; the
+                    // peer's bytes may land first (the pending arrival keeps the phase open)
+                    if (rank == 0) mbar_expect_tx(full_bar(s), 2 * L::kStageBytes);
+                    const uint32_t a_dst = smem_base + s * L::kStageBytes;
+                    tma_load_2d_pair(a_dst, &map_a, leader_full, k * kBK, m_blk * 256 + (int)rank * kBM);
+                    tma_load_2d_pair(a_dst + L::kABytes, &map_b, leader_full, k * kBK,
+                                     n_blk * kPairBN + (int)rank * kPairHalfN);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0 && rank == 0) {
+            uint32_t it = 0, t = 0;
+            bool alive = true;
+            for (int tile = pair_id; alive && tile < num_tiles; tile += num_pairs, ++t) {
+                const int buf = t & 1;
+                const uint32_t acc_ph = (t >> 1) & 1u;
+                if (!mbar_wait(acc_empty_bar(buf), acc_ph ^ 1u, abort_flag, p.d_status)) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + buf * kPairBN;
+                for (int k = 0; k < p.num_k; ++k, ++it) {
+                    const int s = it % kPairStages;
+                    const uint32_t ph = (it / kPairStages) & 1u;
+                    if (!mbar_wait(full_bar(s), ph, abort_flag, p.d_status)) { alive = false; break; }
+                    tc_fence_after();
+                    const uint32_t a_addr = smem_base + s * L::kStageBytes;
+                    const uint64_t da = smem_desc_k128(a_addr);
+                    const uint64_t db = smem_desc_k128(a_addr + L::kABytes);
+#pragma unroll
+                    for (int j = 0; j < kBK / kUmmaK; ++j)
+                        umma_f8_pair(d_tmem, da + 2u * j, db + 2u * j, p.idesc, (k > 0 || j > 0) ? 1u : 0u);
+                    umma_commit_pair(empty_bar(s));
+                }
+                if (alive) umma_commit_pair(acc_full_bar(buf));
+            }
+        }
+    } else {
+        const int q = warp & 3;
+        const int e = -(__ldg(p.d_sa) + __ldg(p.d_sb) + p.delta_sum);
+        const Pow2Pair sc = make_pow2_pair(e);
+        const bool two_step = (e < -126 || e > 127);
+        uint32_t amax_bits = 0;
+        uint32_t t = 0;
+        for (int tile = pair_id; tile < num_tiles; tile += num_pairs, ++t) {
+            int m_blk, n_blk;
+            tile_coords(tile, p, m_blk, n_blk);
+            const int buf = t & 1;
+            const uint32_t acc_ph = (t >> 1) & 1u;
+            const bool ready = mbar_wait(acc_full_bar(buf), acc_ph, abort_flag, p.d_status);
+            if (!__all_sync(0xFFFFFFFFu, ready)) break;
+            tc_fence_after();
+            const int row = m_blk * 256 + (int)rank * kBM + q * 32 + lane;
+            const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + buf * kPairBN;
+#pragma unroll 1
+            for (int c = 0; c < kPairBN; c += 32) {
+                uint32_t r[32];
+                tmem_ld_x32(t_row + c, r);
+                tmem_ld_wait();
+                if (c + 32 >= kPairBN) {
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive_cluster(map_to_cta(acc_empty_bar(buf), 0));
+                }
+                epilogue_chunk(r, row, n_blk * kPairBN + c, p, sc, two_step, amax_bits);
+            }
+        }
+        if (p.d_amax_bits) {
+            amax_bits = __reduce_max_sync(0xFFFFFFFFu, amax_bits);
+            if (lane == 0 && amax_bits) atomicMax(p.d_amax_bits, amax_bits);
+        }
+    }
+
+    __syncwarp();
+    if (*abort_flag) __nanosleep(20000);
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();  // neither CTA releases shared or tensor memory while its peer may still touch it
+    tc_fence_after();
+    if (warp == 1)
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)L::kTmemCols)
+                     : "memory");
+}
+
 // ---------------------------------------------------------------------------
 // host side
 // ---------------------------------------------------------------------------
@@ -398,11 +645,44 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
 constexpr int kBN = 256;
 constexpr int kStages = 4;
 
+static bool g_force_single = false;  // set from FP8LIN_SINGLE_CTA=1 (A/B comparison of the two kernels)
+static int g_max_pairs = 0;  // CTA pairs that can be resident at once (0: pair kernel unavailable)
+
 cudaError_t configure_gemm_kernels(int max_smem_optin)
 {
     using L = GemmSmem<kBN, kStages>;
-    if (L::kDynamic > max_smem_optin) return cudaErrorInvalidValue;
-    return cudaFuncSetAttribute(gemm_kernel<kBN, kStages>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kDynamic);
+    if (L::kDynamic > max_smem_optin || PairSmem::kDynamic > max_smem_optin) return cudaErrorInvalidValue;
+    cudaError_t e =
+        cudaFuncSetAttribute(gemm_kernel<kBN, kStages>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kDynamic);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(gemm_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, PairSmem::kDynamic);
+    if (e != cudaSuccess) return e;
+    int sms = 0, dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+        return cudaErrorUnknown;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(sms & ~1), 1, 1);
+    cfg.blockDim = dim3(kGemmThreads, 1, 1);
+    cfg.dynamicSmemBytes = PairSmem::kDynamic;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = 2;
+    attr.val.clusterDim.y = 1;
+    attr.val.clusterDim.z = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    int clusters = 0;
+    if (cudaOccupancyMaxActiveClusters(&clusters, gemm_pair_kernel, &cfg) != cudaSuccess) {
+        cudaGetLastError();
+        clusters = 0;
+    }
+    g_max_pairs = clusters;
+    const char *env = getenv("FP8LIN_SINGLE_CTA");
+    g_force_single = env && env[0] == '1';
+    if (getenv("FP8LIN_DEBUG")) fprintf(stderr, "fp8lin: %d SMs, %d resident CTA pairs, pair kernel %s\n", sms, clusters,
+                                        g_force_single ? "off" : "on");
+    return cudaSuccess;
 }
 
 // 2-D tensor map over a row-major byte matrix [rows, cols_bytes]: box = box_rows x 128 bytes, 128-byte swizzle.
@@ -428,9 +708,11 @@ static fp8_status_t run_gemm(fp8_ctx *ctx, const uint8_t *a, int a_fmt, const in
     if (M > 0x7FFFFFFF / 2 || N > 0x7FFFFFFF / 2 || Kc > 0x7FFFFFFF / 2) return FP8_ERR_SHAPE;
     CUtensorMap map_a, map_b;
     if (!encode_map(ctx, &map_a, a, M, Kc, kBM) || !encode_map(ctx, &map_b, b, N, Kc, kBN)) return FP8_ERR_CUDA;
+    const bool pair = g_max_pairs > 0 && M > kBM && !g_force_single;
+    if (pair && !encode_map(ctx, &map_b, b, N, Kc, kPairHalfN)) return FP8_ERR_CUDA;
     GemmParams p;
     p.M = (int)M; p.N = (int)N; p.K = (int)Kc;
-    p.tiles_m = (int)((M + kBM - 1) / kBM);
+    p.tiles_m = (int)((M + (pair ? 256 : kBM) - 1) / (pair ? 256 : kBM));
     p.tiles_n = (int)((N + kBN - 1) / kBN);
     p.num_k = (int)((Kc + kBK - 1) / kBK);
     if ((int64_t)p.tiles_m * p.tiles_n > 0x7FFFFFFF) return FP8_ERR_SHAPE;
@@ -441,11 +723,16 @@ static fp8_status_t run_gemm(fp8_ctx *ctx, const uint8_t *a, int a_fmt, const in
     p.vec_ok = ((reinterpret_cast<uintptr_t>(out) & 15u) == 0 && (N * esz) % 16 == 0) ? 1 : 0;
     p.d_amax_bits = reinterpret_cast<unsigned *>(d_amax_out);
     p.d_status = ctx->d_status;
-    p.idesc = make_idesc(a_fmt, b_fmt, kBN);
+    p.idesc = pair ? make_idesc_pair(a_fmt, b_fmt) : make_idesc(a_fmt, b_fmt, kBN);
     if (d_amax_out && cudaMemsetAsync(d_amax_out, 0, sizeof(float), st) != cudaSuccess) return FP8_ERR_CUDA;
     int tiles = p.tiles_m * p.tiles_n;
-    int grid = tiles < ctx->sm_count ? tiles : ctx->sm_count;
-    gemm_kernel<kBN, kStages><<<grid, kGemmThreads, GemmSmem<kBN, kStages>::kDynamic, st>>>(map_a, map_b, p);
+    if (pair) {
+        int pairs = tiles < g_max_pairs ? tiles : g_max_pairs;
+        gemm_pair_kernel<<<2 * pairs, kGemmThreads, PairSmem::kDynamic, st>>>(map_a, map_b, p);
+    } else {
+        int grid = tiles < ctx->sm_count ? tiles : ctx->sm_count;
+        gemm_kernel<kBN, kStages><<<grid, kGemmThreads, GemmSmem<kBN, kStages>::kDynamic, st>>>(map_a, map_b, p);
+    }
     return cudaGetLastError() == cudaSuccess ? FP8_OK : FP8_ERR_CUDA;
 }
 

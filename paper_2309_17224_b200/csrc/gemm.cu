@@ -34,6 +34,8 @@ constexpr int kUmmaK = 32;        // contraction elements per tcgen05.mma for 8-
 constexpr int kGemmThreads = 192;
 constexpr int kGroupM = 8;        // tile rasterisation: m-blocks per group
 constexpr unsigned long long kWaitLimitNs = 1000ull * 1000ull * 1000ull;
+constexpr int kSlabBytes = 32 * 128;            // epilogue staging: 32 rows x 128 bytes, what one warp stores at a time
+constexpr int kEpiBytes = 4 * 2 * kSlabBytes;   // four epilogue warps, two slabs each
 
 struct GemmParams {
     int M, N, K;
@@ -46,6 +48,7 @@ struct GemmParams {
     int out_dt;
     int64_t ldo;
     int vec_ok;                   // out 16-byte aligned and ldo*elem % 16 == 0
+    int tma_out;                  // epilogue goes through shared memory and TMA stores (needs vec_ok)
     unsigned *d_amax_bits;        // or NULL
     unsigned *d_status;
     uint32_t idesc;
@@ -187,7 +190,8 @@ struct GemmSmem {
     static constexpr int kABytes = kBM * kBK;
     static constexpr int kBBytes = BN * kBK;
     static constexpr int kStageBytes = kABytes + kBBytes;
-    static constexpr int kBarOffset = STAGES * kStageBytes;
+    static constexpr int kEpiOffset = STAGES * kStageBytes;
+    static constexpr int kBarOffset = kEpiOffset + kEpiBytes;
     static constexpr int kNumBars = 2 * STAGES + 4;
     static constexpr int kTotal = kBarOffset + kNumBars * 8 + 16;
     static constexpr int kDynamic = kTotal + 1024;  // slack to align the base to 1024 B
@@ -206,13 +210,10 @@ __device__ __forceinline__ void tile_coords(int tile, const GemmParams &p, int &
 }
 
 // One 32-column chunk of one accumulator row: unscale by the exact power of
-// two, optional bias vector, rounding to the output type, running amax of the
-// rounded values, store.
-__device__ __forceinline__ void epilogue_chunk(const uint32_t (&r)[32], int row, int col0, const GemmParams &p,
-                                               const Pow2Pair sc, bool two_step, uint32_t &amax_bits)
+// two, add the optional bias vector.
+__device__ __forceinline__ void epilogue_values(const uint32_t (&r)[32], int col0, const GemmParams &p,
+                                                const Pow2Pair sc, bool two_step, float (&v)[32])
 {
-    if (row >= p.M || col0 >= p.N) return;
-    float v[32];
 #pragma unroll
     for (int i = 0; i < 32; ++i) {
         v[i] = __uint_as_float(r[i]) * sc.first;
@@ -230,19 +231,43 @@ __device__ __forceinline__ void epilogue_chunk(const uint32_t (&r)[32], int row,
             }
         }
     }
+}
+
+// Round 32 values to bf16 pairs (memory order) and fold them into the running amax.
+__device__ __forceinline__ void pack_bf16(const float (&v)[32], int col0, const GemmParams &p, uint32_t (&w)[16],
+                                          uint32_t &amax_bits, bool row_ok)
+{
+#pragma unroll
+    for (int i = 0; i < 16; ++i) asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(w[i]) : "f"(v[2 * i + 1]), "f"(v[2 * i]));
+    if (p.d_amax_bits && row_ok) {
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            uint32_t a = w[i] & 0x7FFF7FFFu;
+            if (col0 + 2 * i < p.N) amax_bits = max(amax_bits, (a & 0xFFFFu) << 16);
+            if (col0 + 2 * i + 1 < p.N) amax_bits = max(amax_bits, a & 0xFFFF0000u);
+        }
+    }
+}
+__device__ __forceinline__ void amax_f32(const float (&v)[32], int col0, const GemmParams &p, uint32_t &amax_bits,
+                                         bool row_ok)
+{
+    if (p.d_amax_bits && row_ok) {
+#pragma unroll
+        for (int i = 0; i < 32; ++i)
+            if (col0 + i < p.N) amax_bits = max(amax_bits, __float_as_uint(v[i]) & 0x7FFFFFFFu);
+    }
+}
+
+// Direct stores from registers (any alignment, any N): one row per thread.
+__device__ __forceinline__ void store_direct(const uint32_t (&r)[32], int row, int col0, const GemmParams &p,
+                                             const Pow2Pair sc, bool two_step, uint32_t &amax_bits)
+{
+    if (row >= p.M || col0 >= p.N) return;
+    float v[32];
+    epilogue_values(r, col0, p, sc, two_step, v);
     if (p.out_dt == FP8_BF16) {
         uint32_t w[16];
-#pragma unroll
-        for (int i = 0; i < 16; ++i)
-            asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(w[i]) : "f"(v[2 * i + 1]), "f"(v[2 * i]));
-        if (p.d_amax_bits) {
-#pragma unroll
-            for (int i = 0; i < 16; ++i) {
-                uint32_t a = w[i] & 0x7FFF7FFFu;
-                if (col0 + 2 * i < p.N) amax_bits = max(amax_bits, (a & 0xFFFFu) << 16);
-                if (col0 + 2 * i + 1 < p.N) amax_bits = max(amax_bits, a & 0xFFFF0000u);
-            }
-        }
+        pack_bf16(v, col0, p, w, amax_bits, true);
         uint16_t *dst = reinterpret_cast<uint16_t *>(p.out) + (int64_t)row * p.ldo + col0;
         if (p.vec_ok && col0 + 32 <= p.N) {
 #pragma unroll
@@ -254,11 +279,7 @@ __device__ __forceinline__ void epilogue_chunk(const uint32_t (&r)[32], int row,
                 if (col0 + i < p.N) dst[i] = (uint16_t)((i & 1) ? (w[i >> 1] >> 16) : (w[i >> 1] & 0xFFFFu));
         }
     } else {
-        if (p.d_amax_bits) {
-#pragma unroll
-            for (int i = 0; i < 32; ++i)
-                if (col0 + i < p.N) amax_bits = max(amax_bits, __float_as_uint(v[i]) & 0x7FFFFFFFu);
-        }
+        amax_f32(v, col0, p, amax_bits, true);
         float *dst = reinterpret_cast<float *>(p.out) + (int64_t)row * p.ldo + col0;
         if (p.vec_ok && col0 + 32 <= p.N) {
 #pragma unroll
@@ -272,9 +293,117 @@ __device__ __forceinline__ void epilogue_chunk(const uint32_t (&r)[32], int row,
     }
 }
 
+// ---- staged epilogue: registers -> swizzled shared memory -> TMA store ----
+
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap *map, uint32_t src, int x, int y)
+{
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%2, %3}], [%1];" ::"l"(
+                     reinterpret_cast<uint64_t>(map)),
+                 "r"(src), "r"(x), "r"(y)
+                 : "memory");
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+// 16-byte piece j (0..7) of this lane's 128-byte row, at its 128-byte-swizzle position
+__device__ __forceinline__ void slab_write(uint32_t slab, int lane, int j, uint32_t a, uint32_t b, uint32_t c, uint32_t d)
+{
+    const uint32_t addr = slab + (uint32_t)lane * 128u + (uint32_t)((j ^ (lane & 7)) << 4);
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+// Before a slab is overwritten, the store issued from it two slabs ago must have read it.
+__device__ __forceinline__ void slab_acquire(int lane)
+{
+    if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+    __syncwarp();
+}
+__device__ __forceinline__ void slab_publish(const CUtensorMap *map, uint32_t slab, int lane, int x, int y, bool in_range)
+{
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    __syncwarp();
+    if (lane == 0 && in_range) tma_store_2d(map, slab, x, y);
+}
+
+// One warp's share (32 rows x BN columns) of a finished accumulator.
+//   t_row        TMEM address of this warp's lanes at the accumulator's first column
+//   row0         first of the warp's 32 output rows;  col_base  first output column of the tile
+//   release_bar  barrier to arrive on once the accumulator has been read (cluster address if remote)
+template <int BN>
+__device__ __forceinline__ void epilogue_tile(const CUtensorMap *map_out, uint32_t t_row, int row0, int col_base,
+                                              const GemmParams &p, const Pow2Pair sc, bool two_step,
+                                              uint32_t &amax_bits, uint32_t warp_slabs, uint32_t &slab_count,
+                                              uint32_t release_bar, bool release_remote, int lane)
+{
+    auto release = [&]() {
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) {
+            if (release_remote)
+                asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(release_bar) : "memory");
+            else
+                mbar_arrive(release_bar);
+        }
+    };
+    if (!p.tma_out) {
+#pragma unroll 1
+        for (int c = 0; c < BN; c += 32) {
+            uint32_t r[32];
+            tmem_ld_x32(t_row + c, r);
+            tmem_ld_wait();
+            if (c + 32 >= BN) release();
+            store_direct(r, row0 + lane, col_base + c, p, sc, two_step, amax_bits);
+        }
+        return;
+    }
+    const bool rows_in = row0 < p.M;
+    const bool row_ok = row0 + lane < p.M;
+    if (p.out_dt == FP8_BF16) {
+#pragma unroll 1
+        for (int c = 0; c < BN; c += 64) {  // one slab = 64 bf16 columns
+            uint32_t r0[32], r1[32];
+            tmem_ld_x32(t_row + c, r0);
+            tmem_ld_x32(t_row + c + 32, r1);
+            tmem_ld_wait();
+            if (c + 64 >= BN) release();
+            const uint32_t slab = warp_slabs + (slab_count & 1u) * kSlabBytes;
+            ++slab_count;
+            slab_acquire(lane);
+            float v[32];
+            uint32_t w[16];
+            epilogue_values(r0, col_base + c, p, sc, two_step, v);
+            pack_bf16(v, col_base + c, p, w, amax_bits, row_ok);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) slab_write(slab, lane, j, w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
+            epilogue_values(r1, col_base + c + 32, p, sc, two_step, v);
+            pack_bf16(v, col_base + c + 32, p, w, amax_bits, row_ok);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) slab_write(slab, lane, 4 + j, w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
+            slab_publish(map_out, slab, lane, col_base + c, row0, rows_in && col_base + c < p.N);
+        }
+    } else {
+#pragma unroll 1
+        for (int c = 0; c < BN; c += 32) {  // one slab = 32 fp32 columns
+            uint32_t r[32];
+            tmem_ld_x32(t_row + c, r);
+            tmem_ld_wait();
+            if (c + 32 >= BN) release();
+            const uint32_t slab = warp_slabs + (slab_count & 1u) * kSlabBytes;
+            ++slab_count;
+            slab_acquire(lane);
+            float v[32];
+            epilogue_values(r, col_base + c, p, sc, two_step, v);
+            amax_f32(v, col_base + c, p, amax_bits, row_ok);
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+                slab_write(slab, lane, j, __float_as_uint(v[4 * j]), __float_as_uint(v[4 * j + 1]),
+                           __float_as_uint(v[4 * j + 2]), __float_as_uint(v[4 * j + 3]));
+            slab_publish(map_out, slab, lane, col_base + c, row0, rows_in && col_base + c < p.N);
+        }
+    }
+}
+
 template <int BN, int STAGES>
 __global__ void __launch_bounds__(kGemmThreads, 1)
-gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const GemmParams p)
+gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+            const __grid_constant__ CUtensorMap map_out, const GemmParams p)
 {
     using L = GemmSmem<BN, STAGES>;
     extern __shared__ uint8_t smem_raw[];
@@ -358,7 +487,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         const int e = -(__ldg(p.d_sa) + __ldg(p.d_sb) + p.delta_sum);
         const Pow2Pair sc = make_pow2_pair(e);
         const bool two_step = (e < -126 || e > 127);
-        uint32_t amax_bits = 0;
+        uint32_t amax_bits = 0, slab_count = 0;
+        const uint32_t warp_slabs = smem_base + L::kEpiOffset + q * 2 * kSlabBytes;
         uint32_t t = 0;
         for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++t) {
             int m_blk, n_blk;
@@ -369,22 +499,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             const bool ready = mbar_wait(acc_full_bar(buf), acc_ph, abort_flag, p.d_status);
             if (!__all_sync(0xFFFFFFFFu, ready)) break;
             tc_fence_after();
-            const int row = m_blk * kBM + q * 32 + lane;
             const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + buf * BN;
-#pragma unroll 1
-            for (int c = 0; c < BN; c += 32) {
-                uint32_t r[32];
-                tmem_ld_x32(t_row + c, r);
-                tmem_ld_wait();
-                if (c + 32 >= BN) {
-                    // the accumulator is in registers: hand the TMEM buffer back
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(acc_empty_bar(buf));
-                }
-                epilogue_chunk(r, row, n_blk * BN + c, p, sc, two_step, amax_bits);
-            }
+            epilogue_tile<BN>(&map_out, t_row, m_blk * kBM + q * 32, n_blk * BN, p, sc, two_step, amax_bits, warp_slabs,
+                              slab_count, acc_empty_bar(buf), false, lane);
         }
+        if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
         if (p.d_amax_bits) {
             amax_bits = __reduce_max_sync(0xFFFFFFFFu, amax_bits);
             if (lane == 0 && amax_bits) atomicMax(p.d_amax_bits, amax_bits);
@@ -428,7 +547,8 @@ struct PairSmem {
     static constexpr int kABytes = kBM * kBK;
     static constexpr int kBBytes = kPairHalfN * kBK;
     static constexpr int kStageBytes = kABytes + kBBytes;
-    static constexpr int kBarOffset = kPairStages * kStageBytes;
+    static constexpr int kEpiOffset = kPairStages * kStageBytes;
+    static constexpr int kBarOffset = kEpiOffset + kEpiBytes;
     static constexpr int kNumBars = 2 * kPairStages + 4;
     static constexpr int kTotal = kBarOffset + kNumBars * 8 + 16;
     static constexpr int kDynamic = kTotal + 1024;
@@ -502,7 +622,7 @@ __host__ __device__ inline uint32_t make_idesc_pair(int a_fmt, int b_fmt)
 // tiles here are 256 x 256; p.tiles_m / p.tiles_n count those
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1)
 gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-                 const GemmParams p)
+                 const __grid_constant__ CUtensorMap map_out, const GemmParams p)
 {
     using L = PairSmem;
     extern __shared__ uint8_t smem_raw[];
@@ -596,7 +716,9 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
         const int e = -(__ldg(p.d_sa) + __ldg(p.d_sb) + p.delta_sum);
         const Pow2Pair sc = make_pow2_pair(e);
         const bool two_step = (e < -126 || e > 127);
-        uint32_t amax_bits = 0;
+        uint32_t amax_bits = 0, slab_count = 0;
+        const uint32_t warp_slabs = smem_base + L::kEpiOffset + q * 2 * kSlabBytes;
+        const uint32_t leader_acc_empty0 = map_to_cta(acc_empty_bar(0), 0);
         uint32_t t = 0;
         for (int tile = pair_id; tile < num_tiles; tile += num_pairs, ++t) {
             int m_blk, n_blk;
@@ -606,21 +728,11 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             const bool ready = mbar_wait(acc_full_bar(buf), acc_ph, abort_flag, p.d_status);
             if (!__all_sync(0xFFFFFFFFu, ready)) break;
             tc_fence_after();
-            const int row = m_blk * 256 + (int)rank * kBM + q * 32 + lane;
             const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + buf * kPairBN;
-#pragma unroll 1
-            for (int c = 0; c < kPairBN; c += 32) {
-                uint32_t r[32];
-                tmem_ld_x32(t_row + c, r);
-                tmem_ld_wait();
-                if (c + 32 >= kPairBN) {
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive_cluster(map_to_cta(acc_empty_bar(buf), 0));
-                }
-                epilogue_chunk(r, row, n_blk * kPairBN + c, p, sc, two_step, amax_bits);
-            }
+            epilogue_tile<kPairBN>(&map_out, t_row, m_blk * 256 + (int)rank * kBM + q * 32, n_blk * kPairBN, p, sc,
+                                   two_step, amax_bits, warp_slabs, slab_count, leader_acc_empty0 + 8u * buf, true, lane);
         }
+        if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
         if (p.d_amax_bits) {
             amax_bits = __reduce_max_sync(0xFFFFFFFFu, amax_bits);
             if (lane == 0 && amax_bits) atomicMax(p.d_amax_bits, amax_bits);
@@ -646,6 +758,7 @@ constexpr int kBN = 256;
 constexpr int kStages = 4;
 
 static bool g_force_single = false;  // set from FP8LIN_SINGLE_CTA=1 (A/B comparison of the two kernels)
+static bool g_direct_epilogue = false;  // set from FP8LIN_DIRECT_EPILOGUE=1 (A/B comparison of the epilogues)
 static int g_max_pairs = 0;  // CTA pairs that can be resident at once (0: pair kernel unavailable)
 
 cudaError_t configure_gemm_kernels(int max_smem_optin)
@@ -680,6 +793,8 @@ cudaError_t configure_gemm_kernels(int max_smem_optin)
     g_max_pairs = clusters;
     const char *env = getenv("FP8LIN_SINGLE_CTA");
     g_force_single = env && env[0] == '1';
+    env = getenv("FP8LIN_DIRECT_EPILOGUE");
+    g_direct_epilogue = env && env[0] == '1';
     if (getenv("FP8LIN_DEBUG")) fprintf(stderr, "fp8lin: %d SMs, %d resident CTA pairs, pair kernel %s\n", sms, clusters,
                                         g_force_single ? "off" : "on");
     return cudaSuccess;
@@ -721,6 +836,19 @@ static fp8_status_t run_gemm(fp8_ctx *ctx, const uint8_t *a, int a_fmt, const in
     p.out = out; p.out_dt = out_dt; p.ldo = N;
     const int64_t esz = out_dt == FP8_BF16 ? 2 : 4;
     p.vec_ok = ((reinterpret_cast<uintptr_t>(out) & 15u) == 0 && (N * esz) % 16 == 0) ? 1 : 0;
+    p.tma_out = (p.vec_ok && !g_direct_epilogue) ? 1 : 0;
+    CUtensorMap map_out = map_a;  // placeholder when the staged epilogue is off (never dereferenced then)
+    if (p.tma_out) {
+        cuuint64_t dims[2] = {(cuuint64_t)N, (cuuint64_t)M};
+        cuuint64_t strides[1] = {(cuuint64_t)(N * esz)};
+        cuuint32_t box[2] = {(cuuint32_t)(128 / esz), 32};
+        cuuint32_t estr[2] = {1, 1};
+        CUresult r = ctx->encode_tiled(&map_out, esz == 2 ? CU_TENSOR_MAP_DATA_TYPE_UINT16 : CU_TENSOR_MAP_DATA_TYPE_UINT32,
+                                       2, out, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                       CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                                       CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) return FP8_ERR_CUDA;
+    }
     p.d_amax_bits = reinterpret_cast<unsigned *>(d_amax_out);
     p.d_status = ctx->d_status;
     p.idesc = pair ? make_idesc_pair(a_fmt, b_fmt) : make_idesc(a_fmt, b_fmt, kBN);
@@ -728,10 +856,10 @@ static fp8_status_t run_gemm(fp8_ctx *ctx, const uint8_t *a, int a_fmt, const in
     int tiles = p.tiles_m * p.tiles_n;
     if (pair) {
         int pairs = tiles < g_max_pairs ? tiles : g_max_pairs;
-        gemm_pair_kernel<<<2 * pairs, kGemmThreads, PairSmem::kDynamic, st>>>(map_a, map_b, p);
+        gemm_pair_kernel<<<2 * pairs, kGemmThreads, PairSmem::kDynamic, st>>>(map_a, map_b, map_out, p);
     } else {
         int grid = tiles < ctx->sm_count ? tiles : ctx->sm_count;
-        gemm_kernel<kBN, kStages><<<grid, kGemmThreads, GemmSmem<kBN, kStages>::kDynamic, st>>>(map_a, map_b, p);
+        gemm_kernel<kBN, kStages><<<grid, kGemmThreads, GemmSmem<kBN, kStages>::kDynamic, st>>>(map_a, map_b, map_out, p);
     }
     return cudaGetLastError() == cudaSuccess ? FP8_OK : FP8_ERR_CUDA;
 }

@@ -115,11 +115,11 @@ class LayerState:
     """Device buffers of one linear: bf16 inputs, FP8 copies in both layouts,
     device scalars, bf16 outputs."""
 
-    def __init__(self, wl, li, device, seed, backward):
+    def __init__(self, wl, li, device, seed, backward, tokens=0):
         l = wl.layers[li]
-        T, K, N = wl.tokens, l.K, l.N
+        T, K, N = tokens or wl.tokens, l.K, l.N
         self.T, self.K, self.N, self.name = T, K, N, l.name
-        t = I.layer_tensors(wl, li, device=device, seed=seed)
+        t = I.layer_tensors(wl, li, device=device, seed=seed, tokens=T)
         self.x, self.w = t["x"], t["w"]
         self.g = t.get("g")
         u8 = dict(dtype=torch.uint8, device=device)
@@ -140,11 +140,12 @@ class LayerState:
         return 2.0 * self.T * self.K * self.N * (3 if self.backward else 1)
 
     def cast_elements(self):
-        n = self.T * self.K + self.N * self.K
-        return n + (self.T * self.N if self.backward else 0)
+        if not self.backward:
+            return self.T * self.K          # weights were quantised once, at load
+        return self.T * self.K + self.N * self.K + self.T * self.N
 
     def launches(self):
-        return 9 if self.backward else 5
+        return 9 if self.backward else 3
 
 
 class Timers:
@@ -176,7 +177,8 @@ def run_layer(ctx, L, timers=None):
             b.record()
 
     af, bi = L.scal_f, L.scal_i
-    timed("amax_cast", lambda: ctx.cast_e4(L.w, None, d_amax_out=af[0:1], d_bias_out=bi[0:1], y=L.w8, y_t=L.w8t))
+    if L.backward:  # training: the weights are re-quantised every step; inference: once at load (ptq_weights)
+        timed("amax_cast", lambda: ctx.cast_e4(L.w, None, d_amax_out=af[0:1], d_bias_out=bi[0:1], y=L.w8, y_t=L.w8t))
     timed("amax_cast", lambda: ctx.cast_e4(L.x, None, d_amax_out=af[1:2], d_bias_out=bi[1:2], y=L.x8, y_t=L.x8t))
     timed("gemm", lambda: ctx.linear_fwd(L.x8, bi[1:2], L.w8, bi[0:1], L.y))
     if L.backward:
@@ -274,6 +276,7 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(I.WORKLOADS))
+    ap.add_argument("--tokens", type=int, default=0, help="override the workload's token count (c4: 1, 16, 64, 2048)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -293,8 +296,13 @@ def main():
     device = torch.device("cuda", local)
     warmup = max(3, args.warmup)
     ctx = fp8lin.Context(local)
-    layers = [LayerState(wl, li, device, I.BASE_SEED + 7919 * rank, wl.backward) for li in range(len(wl.layers))]
+    layers = [LayerState(wl, li, device, I.BASE_SEED + 7919 * rank, wl.backward, args.tokens)
+              for li in range(len(wl.layers))]
     peaks = load_peaks()
+    tokens = args.tokens or wl.tokens
+    if not wl.backward:  # post-training quantisation, once, outside the timed region
+        for L in layers:
+            ctx.ptq_weights(L.w, fp8lin.CONV_PAPER, L.w8, None, L.scal_i[0:1], L.scal_f[0:1])
 
     for _ in range(warmup):
         for L in layers:
@@ -339,7 +347,7 @@ def main():
     if args.e2e_steps > 0:
         host_in, host_out = [], []
         for L in layers:
-            ins = [L.x, L.w] + ([L.g] if wl.backward else [])
+            ins = [L.x] + ([L.w, L.g] if wl.backward else [])
             outs = [L.y] + ([L.dx, L.dw] if wl.backward else [])
             host_in.append([torch.empty(t.shape, dtype=t.dtype, pin_memory=True).copy_(t) for t in ins])
             host_out.append([torch.empty(t.shape, dtype=t.dtype, pin_memory=True) for t in outs])
@@ -348,7 +356,7 @@ def main():
 
         def e2e_step():
             for L, hin, hout in zip(layers, host_in, host_out):
-                ins = [L.x, L.w] + ([L.g] if wl.backward else [])
+                ins = [L.x] + ([L.w, L.g] if wl.backward else [])
                 outs = [L.y] + ([L.dx, L.dw] if wl.backward else [])
                 for d, h in zip(ins, hin):
                     d.copy_(h, non_blocking=True)
@@ -384,10 +392,10 @@ def main():
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "fp8_e4m3/e5m2 operands, f32 accumulate, bf16 out", "data": "synthetic",
-        "config": {"workload": wl.name, "tokens": wl.tokens,
+        "config": {"workload": wl.name, "tokens": tokens,
                    "layers": [f"{l.name}:{l.K}->{l.N}" for l in wl.layers],
-                   "passes": "fwd+bwd" if wl.backward else "fwd",
-                   "scaling_bias": "FP8-AMAX, recomputed every step for W, X, dY",
+                   "passes": "fwd+bwd" if wl.backward else "fwd (weights quantised once at load)",
+                   "scaling_bias": "FP8-AMAX, recomputed every step for " + ("W, X, dY" if wl.backward else "X"),
                    "l2": "inputs larger than L2 (each layer's tensors exceed 126 MB); no flush between steps",
                    "parallelism": "replicas" if world > 1 else "single"},
         "clocks": clocks,
@@ -403,6 +411,8 @@ def main():
                       "hbm_peak_gbs": peaks["hbm_gbs"],
                       "frac": cast_elems * bytes_per_elem / (cast_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]},
         "gemm_ms_per_step": gemm_ms / args.steps,
+        "weight_stream_gbs": (None if wl.backward else
+                              sum(L.N * L.K for L in layers) * args.steps / (gemm_ms * 1e-3) / 1e9),
         "device_flags": flags,
         "cpu_baseline": cpu_baseline,
     }

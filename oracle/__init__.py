@@ -258,3 +258,49 @@ def linear_samples(kind, a8, fa, s_a, b8, fb, s_b, rows, cols, bias_vec=None) ->
                             bv.ctypes.data if bv is not None else None, T, K, N,
                             rows.ctypes.data, cols.ctypes.data, rows.size, *res._ptrs())
     return res
+
+
+# ----------------------------------------------------------------------------
+# the same matmul definitions with numpy's float64 matmul as the summation step
+# ----------------------------------------------------------------------------
+# Every product of two FP8 values is a small multiple of a power of two, and
+# sums of up to 2^16 of them stay far inside float64's 53 bits, so the float64
+# sum is exact whatever order a BLAS adds in.  These functions therefore return
+# exactly what the plain C loops return (tests/test_oracle_gemm.py checks that
+# equality); they exist because the C loops need minutes where a 24-layer
+# trajectory or a full-size layer has to be checked.
+
+class _NpResult:
+    def __init__(self, f64, abs_sum):
+        self.f64 = f64
+        self.abs_sum = abs_sum
+        self.f32 = f64.astype(np.float32)
+        u = self.f32.view(np.uint32).astype(np.uint64)
+        nan = (u & 0x7FFFFFFF) > 0x7F800000
+        rounded = (u + 0x7FFF + ((u >> 16) & 1)) >> 16
+        self.bf16 = np.where(nan, (u >> 16) | 0x40, rounded).astype(np.uint16)
+
+
+def _matmul_unscale(A, B_t, shift_sum, bias_vec=None):
+    f64 = np.ldexp(A @ B_t, -shift_sum)
+    abs_sum = np.ldexp(np.abs(A) @ np.abs(B_t), -shift_sum)
+    if bias_vec is not None:
+        bv = np.asarray(bias_vec, dtype=np.float64)
+        f64 = f64 + bv[None, :]
+        abs_sum = abs_sum + np.abs(bv)[None, :]
+    return _NpResult(f64, abs_sum)
+
+
+def linear_fwd_np(x8, s_x, w8, s_w, bias_vec=None, fx=N_E4, fw=N_E4):
+    """Y = (X8 . W8^T) * 2^-(s_x+s_w) (+ bias_vec)."""
+    return _matmul_unscale(decode_table(fx)[_u8(x8)], decode_table(fw)[_u8(w8)].T, int(s_x) + int(s_w), bias_vec)
+
+
+def linear_dgrad_np(dy8, s_g, w8, s_w, fg=N_E5, fw=N_E4):
+    """dX = (dY8 . W8) * 2^-(s_g+s_w)."""
+    return _matmul_unscale(decode_table(fg)[_u8(dy8)], decode_table(fw)[_u8(w8)], int(s_g) + int(s_w))
+
+
+def linear_wgrad_np(dy8, s_g, x8, s_x, fg=N_E5, fx=N_E4):
+    """dW = (dY8^T . X8) * 2^-(s_g+s_x)."""
+    return _matmul_unscale(decode_table(fg)[_u8(dy8)].T, decode_table(fx)[_u8(x8)], int(s_g) + int(s_x))

@@ -48,17 +48,22 @@ fp8_status_t fp8_create(fp8_ctx **out, int device)
     if (cudaMemset(buf, 0, words * sizeof(unsigned)) != cudaSuccess) { cudaFree(buf); delete ctx; return FP8_ERR_CUDA; }
     ctx->d_status = buf;
     ctx->d_slots = buf + 1;
+    ctx->partial_bytes = (size_t)64 << 20;
+    ctx->d_partial = nullptr;
+    if (cudaMalloc(&ctx->d_partial, ctx->partial_bytes) != cudaSuccess) { cudaFree(buf); delete ctx; return FP8_ERR_CUDA; }
 
     void *fn = nullptr;
     cudaDriverEntryPointQueryResult qres;
     if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
         qres != cudaDriverEntryPointSuccess || !fn) {
+        cudaFree(ctx->d_partial);
         cudaFree(buf);
         delete ctx;
         return FP8_ERR_CUDA;
     }
     ctx->encode_tiled = (fp8lin::EncodeTiledFn)fn;
     if (fp8lin::configure_gemm_kernels(ctx->max_smem_optin) != cudaSuccess) {
+        cudaFree(ctx->d_partial);
         cudaFree(buf);
         delete ctx;
         return FP8_ERR_CUDA;
@@ -72,6 +77,8 @@ fp8_status_t fp8_destroy(fp8_ctx *ctx)
     if (!ctx) return FP8_ERR_NULL;
     cudaSetDevice(ctx->device);
     cudaError_t e = cudaFree(ctx->d_status);
+    cudaError_t e2 = cudaFree(ctx->d_partial);
+    if (e == cudaSuccess) e = e2;
     delete ctx;
     return e == cudaSuccess ? FP8_OK : FP8_ERR_CUDA;
 }

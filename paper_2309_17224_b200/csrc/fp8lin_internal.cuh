@@ -30,6 +30,8 @@ struct fp8_ctx {
     unsigned *d_status;   // one sticky word of FP8_FLAG_* bits
     unsigned *d_slots;    // kReduceSlots * kSlotWords words, all zero between calls
     unsigned next_slot;
+    float *d_partial;     // FP32 workspace for split-K partial sums
+    size_t partial_bytes;
     fp8lin::EncodeTiledFn encode_tiled;
 };
 

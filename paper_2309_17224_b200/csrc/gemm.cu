@@ -40,6 +40,8 @@ constexpr int kEpiBytes = 4 * 2 * kSlabBytes;   // four epilogue warps, two slab
 struct GemmParams {
     int M, N, K;
     int tiles_m, tiles_n, num_k;
+    int splits, kb_per_split;     // split-K (single-CTA kernel only): k-blocks per split
+    float *partial;               // [splits, M, N] FP32 partial sums when splits > 1
     const int32_t *d_sa, *d_sb;   // paper-convention biases of the two operands
     int delta_sum;                // format shifts to add to them
     const void *bias_vec;         // [N] or NULL
@@ -418,7 +420,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int num_tiles = p.tiles_m * p.tiles_n;
+    const int num_items = p.tiles_m * p.tiles_n * p.splits;  // (tile, k-split) pairs
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
@@ -439,10 +441,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_b)) : "memory");
             uint32_t it = 0;
             bool alive = true;
-            for (int tile = blockIdx.x; alive && tile < num_tiles; tile += gridDim.x) {
+            for (int item = blockIdx.x; alive && item < num_items; item += gridDim.x) {
                 int m_blk, n_blk;
-                tile_coords(tile, p, m_blk, n_blk);
-                for (int k = 0; k < p.num_k; ++k, ++it) {
+                tile_coords(item / p.splits, p, m_blk, n_blk);
+                const int k0 = (item % p.splits) * p.kb_per_split;
+                const int k1 = min(p.num_k, k0 + p.kb_per_split);
+                for (int k = k0; k < k1; ++k, ++it) {
                     const int s = it % STAGES;
                     const uint32_t ph = (it / STAGES) & 1u;
                     if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p.d_status)) { alive = false; break; }
@@ -457,13 +461,15 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         if (lane == 0) {
             uint32_t it = 0, t = 0;
             bool alive = true;
-            for (int tile = blockIdx.x; alive && tile < num_tiles; tile += gridDim.x, ++t) {
+            for (int item = blockIdx.x; alive && item < num_items; item += gridDim.x, ++t) {
+                const int k0 = (item % p.splits) * p.kb_per_split;
+                const int k1 = min(p.num_k, k0 + p.kb_per_split);
                 const int buf = t & 1;
                 const uint32_t acc_ph = (t >> 1) & 1u;
                 if (!mbar_wait(acc_empty_bar(buf), acc_ph ^ 1u, abort_flag, p.d_status)) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + buf * BN;
-                for (int k = 0; k < p.num_k; ++k, ++it) {
+                for (int k = k0; k < k1; ++k, ++it) {
                     const int s = it % STAGES;
                     const uint32_t ph = (it / STAGES) & 1u;
                     if (!mbar_wait(full_bar(s), ph, abort_flag, p.d_status)) { alive = false; break; }
@@ -474,7 +480,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
 #pragma unroll
                     for (int j = 0; j < kBK / kUmmaK; ++j) {
                         // advancing 32 bytes inside the 128-byte swizzle row = +2 in the 16-byte address field
-                        umma_f8(d_tmem, da + 2u * j, db + 2u * j, p.idesc, (k > 0 || j > 0) ? 1u : 0u);
+                        umma_f8(d_tmem, da + 2u * j, db + 2u * j, p.idesc, (k > k0 || j > 0) ? 1u : 0u);
                     }
                     umma_commit(empty_bar(s));
                 }
@@ -490,9 +496,20 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         uint32_t amax_bits = 0, slab_count = 0;
         const uint32_t warp_slabs = smem_base + L::kEpiOffset + q * 2 * kSlabBytes;
         uint32_t t = 0;
-        for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++t) {
+        // with split-K every item leaves its raw FP32 partial sum in the workspace; a second kernel finishes
+        GemmParams pp = p;
+        if (p.splits > 1) {
+            pp.out_dt = FP8_F32;
+            pp.bias_vec = nullptr;
+            pp.d_amax_bits = nullptr;
+            pp.tma_out = 0;
+            pp.vec_ok = (p.N % 4) == 0;
+        }
+        const Pow2Pair sc_one = make_pow2_pair(0);
+        for (int item = blockIdx.x; item < num_items; item += gridDim.x, ++t) {
             int m_blk, n_blk;
-            tile_coords(tile, p, m_blk, n_blk);
+            tile_coords(item / p.splits, p, m_blk, n_blk);
+            if (p.splits > 1) pp.out = p.partial + (int64_t)(item % p.splits) * p.M * p.N;
             const int buf = t & 1;
             const uint32_t acc_ph = (t >> 1) & 1u;
             // every lane waits (each needs the ordering), but the warp leaves together
@@ -500,8 +517,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             if (!__all_sync(0xFFFFFFFFu, ready)) break;
             tc_fence_after();
             const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + buf * BN;
-            epilogue_tile<BN>(&map_out, t_row, m_blk * kBM + q * 32, n_blk * BN, p, sc, two_step, amax_bits, warp_slabs,
-                              slab_count, acc_empty_bar(buf), false, lane);
+            epilogue_tile<BN>(&map_out, t_row, m_blk * kBM + q * 32, n_blk * BN, pp, p.splits > 1 ? sc_one : sc,
+                              p.splits > 1 ? false : two_step, amax_bits, warp_slabs, slab_count, acc_empty_bar(buf),
+                              false, lane);
         }
         if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
         if (p.d_amax_bits) {
@@ -750,6 +768,40 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                      : "memory");
 }
 
+
+// Second half of a split-K matmul: add the partial sums in a fixed order, then
+// the same unscale / bias / rounding / amax as the fused epilogue.
+__global__ void __launch_bounds__(256) splitk_finalize_kernel(const GemmParams p)
+{
+    const int64_t total = (int64_t)p.M * p.N;
+    const int e = -(__ldg(p.d_sa) + __ldg(p.d_sb) + p.delta_sum);
+    const Pow2Pair sc = make_pow2_pair(e);
+    uint32_t amax_bits = 0;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        float acc = 0.0f;
+        for (int s = 0; s < p.splits; ++s) acc += __ldcs(p.partial + (int64_t)s * total + i);
+        float v = acc * sc.first * sc.second;
+        const int col = (int)(i % p.N);
+        if (p.bias_vec)
+            v += p.bias_dt == FP8_F32
+                     ? __ldg(reinterpret_cast<const float *>(p.bias_vec) + col)
+                     : __uint_as_float((uint32_t)__ldg(reinterpret_cast<const uint16_t *>(p.bias_vec) + col) << 16);
+        if (p.out_dt == FP8_BF16) {
+            uint32_t w;
+            asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(w) : "f"(0.0f), "f"(v));
+            reinterpret_cast<uint16_t *>(p.out)[i] = (uint16_t)(w & 0xFFFFu);
+            amax_bits = max(amax_bits, (w & 0x7FFFu) << 16);
+        } else {
+            reinterpret_cast<float *>(p.out)[i] = v;
+            amax_bits = max(amax_bits, __float_as_uint(v) & 0x7FFFFFFFu);
+        }
+    }
+    if (p.d_amax_bits) {
+        amax_bits = __reduce_max_sync(0xFFFFFFFFu, amax_bits);
+        if ((threadIdx.x & 31) == 0 && amax_bits) atomicMax(p.d_amax_bits, amax_bits);
+    }
+}
+
 // ---------------------------------------------------------------------------
 // host side
 // ---------------------------------------------------------------------------
@@ -758,6 +810,7 @@ constexpr int kBN = 256;
 constexpr int kStages = 4;
 
 static bool g_force_single = false;  // set from FP8LIN_SINGLE_CTA=1 (A/B comparison of the two kernels)
+static bool g_no_splitk = false;        // set from FP8LIN_NO_SPLITK=1
 static bool g_direct_epilogue = false;  // set from FP8LIN_DIRECT_EPILOGUE=1 (A/B comparison of the epilogues)
 static int g_max_pairs = 0;  // CTA pairs that can be resident at once (0: pair kernel unavailable)
 
@@ -793,6 +846,8 @@ cudaError_t configure_gemm_kernels(int max_smem_optin)
     g_max_pairs = clusters;
     const char *env = getenv("FP8LIN_SINGLE_CTA");
     g_force_single = env && env[0] == '1';
+    env = getenv("FP8LIN_NO_SPLITK");
+    g_no_splitk = env && env[0] == '1';
     env = getenv("FP8LIN_DIRECT_EPILOGUE");
     g_direct_epilogue = env && env[0] == '1';
     if (getenv("FP8LIN_DEBUG")) fprintf(stderr, "fp8lin: %d SMs, %d resident CTA pairs, pair kernel %s\n", sms, clusters,
@@ -831,6 +886,25 @@ static fp8_status_t run_gemm(fp8_ctx *ctx, const uint8_t *a, int a_fmt, const in
     p.tiles_n = (int)((N + kBN - 1) / kBN);
     p.num_k = (int)((Kc + kBK - 1) / kBK);
     if ((int64_t)p.tiles_m * p.tiles_n > 0x7FFFFFFF) return FP8_ERR_SHAPE;
+    // Few output tiles and a long contraction (the decode regime): split the contraction so that every SM
+    // streams operand bytes; partial sums go through the context's FP32 workspace.
+    p.splits = 1;
+    p.kb_per_split = p.num_k;
+    p.partial = ctx->d_partial;
+    if (!pair && !g_no_splitk) {
+        const int64_t tiles = (int64_t)p.tiles_m * p.tiles_n;
+        if (tiles < 2 * ctx->sm_count && p.num_k >= 8) {
+            int64_t want = (2 * ctx->sm_count + tiles - 1) / tiles;
+            int64_t by_k = p.num_k / 4;
+            int64_t by_ws = (int64_t)(ctx->partial_bytes / sizeof(float)) / (M * N);
+            int64_t sp = want < by_k ? want : by_k;
+            if (sp > by_ws) sp = by_ws;
+            if (sp > 1) {
+                p.kb_per_split = (int)((p.num_k + sp - 1) / sp);
+                p.splits = (p.num_k + p.kb_per_split - 1) / p.kb_per_split;
+            }
+        }
+    }
     p.d_sa = d_ba; p.d_sb = d_bb; p.delta_sum = delta_sum;
     p.bias_vec = bias_vec; p.bias_dt = bias_dt;
     p.out = out; p.out_dt = out_dt; p.ldo = N;
@@ -858,8 +932,16 @@ static fp8_status_t run_gemm(fp8_ctx *ctx, const uint8_t *a, int a_fmt, const in
         int pairs = tiles < g_max_pairs ? tiles : g_max_pairs;
         gemm_pair_kernel<<<2 * pairs, kGemmThreads, PairSmem::kDynamic, st>>>(map_a, map_b, map_out, p);
     } else {
-        int grid = tiles < ctx->sm_count ? tiles : ctx->sm_count;
+        int items = tiles * p.splits;
+        int grid = items < ctx->sm_count ? items : ctx->sm_count;
         gemm_kernel<kBN, kStages><<<grid, kGemmThreads, GemmSmem<kBN, kStages>::kDynamic, st>>>(map_a, map_b, map_out, p);
+        if (p.splits > 1) {
+            if (cudaGetLastError() != cudaSuccess) return FP8_ERR_CUDA;
+            int64_t total = M * N;
+            int blocks = (int)((total + 255) / 256);
+            if (blocks > ctx->sm_count * 8) blocks = ctx->sm_count * 8;
+            splitk_finalize_kernel<<<blocks, 256, 0, st>>>(p);
+        }
     }
     return cudaGetLastError() == cudaSuccess ? FP8_OK : FP8_ERR_CUDA;
 }

@@ -1,0 +1,97 @@
+"""A stack of FP8 linears trained with SGD: the dynamic-scaling stress workload.
+
+24 x (d -> d) FP8 linears with GELU between them, MSE loss to a seeded target,
+plain SGD on FP32 master weights.  Every step re-quantises every weight,
+activation and gradient tensor with a fresh FP8-AMAX bias, and the input scale
+drifts as 2^(8 sin(step / 20)) so that the biases have to move.
+
+Only the linears belong to the paper's method and run in the library
+(``fp8_cast_e4/e5``, ``fp8_linear_fwd/dgrad/wgrad``); the glue around them
+(GELU and its derivative, the loss gradient, the SGD update) is ordinary FP32
+torch arithmetic rounded to bf16, outside the measured path.
+"""
+from __future__ import annotations
+
+import math
+from typing import Dict, List
+
+import torch
+
+from . import inputs as I
+
+CONFIG_ID = 5
+
+
+def step_input(x_base: torch.Tensor, step: int) -> torch.Tensor:
+    """bf16(X_base * 2^(8 sin(step/20))), the product taken in float64."""
+    scale = 2.0 ** (8.0 * math.sin(step / 20.0))
+    return (x_base.to(torch.float64) * scale).to(torch.float32).to(torch.bfloat16)
+
+
+def gelu_bf16(y: torch.Tensor) -> torch.Tensor:
+    z = y.to(torch.float32)
+    return (0.5 * z * (1.0 + torch.erf(z * (1.0 / math.sqrt(2.0))))).to(torch.bfloat16)
+
+
+def gelu_grad_f32(y: torch.Tensor) -> torch.Tensor:
+    z = y.to(torch.float32)
+    cdf = 0.5 * (1.0 + torch.erf(z * (1.0 / math.sqrt(2.0))))
+    pdf = torch.exp(-0.5 * z * z) * (1.0 / math.sqrt(2.0 * math.pi))
+    return cdf + z * pdf
+
+
+class Fp8Stack:
+    def __init__(self, ctx, layers: int = 24, d: int = 1024, tokens: int = 4096, lr: float = 1e-3,
+                 seed: int = I.BASE_SEED, device="cuda", w_std: float = 0.02):
+        self.ctx, self.L, self.d, self.T, self.lr = ctx, layers, d, tokens, lr
+        dev = dict(device=device)
+        self.w32 = [I.normal_bf16(d, d, w_std, seed, I.tensor_id(CONFIG_ID, l, I.W_ID), device).to(torch.float32)
+                    for l in range(layers)]
+        self.x_base = I.normal_bf16(tokens, d, 1.0, seed, I.tensor_id(CONFIG_ID, 0, I.X_ID), device)
+        self.target = I.normal_bf16(tokens, d, 1.0, seed, I.tensor_id(CONFIG_ID, 0, I.TARGET_ID), device)
+        u8 = dict(dtype=torch.uint8, **dev)
+        self.x8 = [torch.empty((tokens, d), **u8) for _ in range(layers)]
+        self.x8t = [torch.empty((d, tokens), **u8) for _ in range(layers)]
+        self.w8 = [torch.empty((d, d), **u8) for _ in range(layers)]
+        self.w8t = [torch.empty((d, d), **u8) for _ in range(layers)]
+        self.y = [torch.empty((tokens, d), dtype=torch.bfloat16, **dev) for _ in range(layers)]
+        self.g8 = torch.empty((tokens, d), **u8)
+        self.g8t = torch.empty((d, tokens), **u8)
+        self.dx = torch.empty((tokens, d), dtype=torch.bfloat16, **dev)
+        self.dw = torch.empty((d, d), dtype=torch.bfloat16, **dev)
+        # per layer: amax / bias of W, X, dY
+        self.amax = torch.zeros((layers, 3), dtype=torch.float32, **dev)
+        self.bias = torch.zeros((layers, 3), dtype=torch.int32, **dev)
+
+    def flops_per_step(self) -> float:
+        return 3.0 * 2.0 * self.T * self.d * self.d * self.L
+
+    def forward(self, x: torch.Tensor) -> torch.Tensor:
+        c = self.ctx
+        for l in range(self.L):
+            w16 = self.w32[l].to(torch.bfloat16)
+            c.cast_e4(w16, None, d_amax_out=self.amax[l, 0:1], d_bias_out=self.bias[l, 0:1], y=self.w8[l], y_t=self.w8t[l])
+            c.cast_e4(x, None, d_amax_out=self.amax[l, 1:2], d_bias_out=self.bias[l, 1:2], y=self.x8[l], y_t=self.x8t[l])
+            c.linear_fwd(self.x8[l], self.bias[l, 1:2], self.w8[l], self.bias[l, 0:1], self.y[l])
+            if l + 1 < self.L:
+                x = gelu_bf16(self.y[l])
+        return self.y[self.L - 1]
+
+    def backward_and_update(self) -> None:
+        c = self.ctx
+        out = self.y[self.L - 1].to(torch.float32)
+        g = ((out - self.target.to(torch.float32)) * (2.0 / (self.T * self.d))).to(torch.bfloat16)
+        for l in range(self.L - 1, -1, -1):
+            c.cast_e5(g, None, d_amax_out=self.amax[l, 2:3], d_bias_out=self.bias[l, 2:3], y=self.g8, y_t=self.g8t)
+            c.linear_dgrad(self.g8, self.bias[l, 2:3], None, self.w8t[l], self.bias[l, 0:1], self.dx)
+            c.linear_wgrad(None, self.g8t, self.bias[l, 2:3], None, self.x8t[l], self.bias[l, 1:2], self.dw, self.T)
+            self.w32[l].add_(self.dw.to(torch.float32), alpha=-self.lr)
+            if l > 0:
+                g = (self.dx.to(torch.float32) * gelu_grad_f32(self.y[l - 1])).to(torch.bfloat16)
+
+    def step(self, step: int) -> Dict[str, object]:
+        x = step_input(self.x_base, step)
+        out = self.forward(x)
+        loss = torch.mean((out.to(torch.float32) - self.target.to(torch.float32)) ** 2)
+        self.backward_and_update()
+        return {"loss": loss, "bias": self.bias.clone(), "amax": self.amax.clone()}

@@ -187,3 +187,63 @@ def test_full_size_layers_sampled(ctx, lib, wl_name, layer):
         ref = O.linear_samples(kind, *ops, rows, cols)
         got = bits_of(out)[rows, cols]
         assert_bf16_within_one_ulp(got, ref)
+
+
+@pytest.mark.parametrize("T,K,N", [(1, 2048, 768), (16, 4096, 1280), (64, 8192, 512), (100, 1024, 2304)])
+def test_decode_shapes_split_k(ctx, lib, T, K, N):
+    """Few tokens, long contraction: the library splits the contraction across
+    CTAs and finishes in a second kernel; results must meet the same bars."""
+    x = I.normal_bf16(T, K, 1.0, 31, 1, "cuda", outlier_frac=0.005, outlier_scale=100.0)
+    w = I.normal_bf16(N, K, 0.015, 31, 2, "cuda")
+    qx, qw = Quantised(ctx, x, O.E4, O.CONV_PAPER), Quantised(ctx, w, O.E4, O.CONV_PAPER)
+    ref = O.linear_fwd(qx.ref, qx.shift, qw.ref, qw.shift)
+    bv = (torch.randn(N, device="cuda") * 0.1).to(torch.bfloat16)
+    ref_b = O.linear_fwd(qx.ref, qx.shift, qw.ref, qw.shift, bias_vec=bv.double().cpu().numpy())
+    for dt in (torch.float32, torch.bfloat16):
+        y = torch.full((T, N), float("nan"), dtype=dt, device="cuda")
+        amax_y = torch.zeros(1, dtype=torch.float32, device="cuda")
+        ctx.linear_fwd(qx.y, qx.bias, qw.y, qw.bias, y, d_amax_y=amax_y)
+        if dt == torch.float32:
+            assert_gemm_close(y.cpu().numpy(), ref)
+        else:
+            assert_bf16_within_one_ulp(bits_of(y), ref)
+        assert float(amax_y.item()) == float(y.float().abs().max().item())
+        ctx.linear_fwd(qx.y, qx.bias, qw.y, qw.bias, y, bias_vec=bv)
+        if dt == torch.float32:
+            assert_gemm_close(y.cpu().numpy(), ref_b)
+        else:
+            assert_bf16_within_one_ulp(bits_of(y), ref_b)
+    assert ctx.device_flags(clear=True) & lib.FLAG_TIMEOUT == 0
+
+
+@pytest.mark.parametrize("layer,tokens", [(1, 1), (0, 16), (1, 64), (3, 64)])
+def test_llama70b_ptq_inference_layers(ctx, lib, layer, tokens):
+    """Config 4: weights quantised once (post-training quantisation), forward
+    only, decode-size batches.  Weight bytes are checked on sampled rows (the
+    bias comes from the amax of the whole tensor), outputs at sampled positions."""
+    wl = I.WORKLOADS["c4_llama70b_ptq"]
+    l = wl.layers[layer]
+    K, N = l.K, l.N
+    t = I.layer_tensors(wl, layer, device="cuda", tokens=tokens)
+    w8 = torch.empty((N, K), dtype=torch.uint8, device="cuda")
+    amax_w = torch.zeros(1, dtype=torch.float32, device="cuda")
+    bias_w = torch.zeros(1, dtype=torch.int32, device="cuda")
+    ctx.ptq_weights(t["w"], lib.CONV_PAPER, w8, None, bias_w, amax_w)
+    wb = bits_of(t["w"])
+    a = O.amax(wb)
+    b = O.scaling_bias(a, O.E4)
+    assert float(amax_w.item()) == a and int(bias_w.item()) == b
+    rng = np.random.default_rng(layer * 100 + tokens)
+    rows = np.sort(rng.choice(N, size=256, replace=False))
+    w8_rows = O.cast(wb[rows], b + 1, O.N_E4)
+    assert_codes_equal(u8(w8)[rows], w8_rows, O.N_E4)
+    qx = Quantised(ctx, t["x"], O.E4, O.CONV_PAPER)
+    y = torch.empty((tokens, N), dtype=torch.bfloat16, device="cuda")
+    ctx.linear_fwd(qx.y, qx.bias, w8, bias_w, y)
+    assert ctx.device_flags(clear=True) & lib.FLAG_TIMEOUT == 0
+    # outputs in the sampled weight rows: the oracle sees only those rows of W8
+    ti = rng.integers(0, tokens, 3000)
+    ni = rng.integers(0, len(rows), 3000)
+    ref = O.linear_samples(O.FWD, qx.ref, O.N_E4, qx.shift, w8_rows, O.N_E4, b + 1, ti, ni)
+    got = bits_of(y)[ti, rows[ni]]
+    assert_bf16_within_one_ulp(got, ref)

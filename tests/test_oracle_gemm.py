@@ -131,3 +131,20 @@ def test_fp8_product_stays_close_to_the_bf16_product():
     bound = np.abs(X.double().numpy()) @ np.abs(W.double().numpy()).T
     assert np.all(np.abs(res.f64 - exact) <= 0.13 * bound)
     assert np.corrcoef(res.f64.ravel(), exact.ravel())[0, 1] > 0.99
+
+
+def test_numpy_matmul_variants_equal_the_plain_loops_exactly():
+    rng = np.random.default_rng(21)
+    T, K, N = 70, 300, 90
+    x8 = rng.integers(0, 0x7F, size=(T, K), dtype=np.uint8) | (rng.integers(0, 2, size=(T, K), dtype=np.uint8) << 7)
+    w8 = rng.integers(0, 0x7F, size=(N, K), dtype=np.uint8) | (rng.integers(0, 2, size=(N, K), dtype=np.uint8) << 7)
+    g8 = rng.integers(0, 0x7C, size=(T, N), dtype=np.uint8) | (rng.integers(0, 2, size=(T, N), dtype=np.uint8) << 7)
+    bv = rng.standard_normal(N)
+    pairs = [(O.linear_fwd(x8, 9, w8, -3, bias_vec=bv), O.linear_fwd_np(x8, 9, w8, -3, bias_vec=bv)),
+             (O.linear_dgrad(g8, 21, w8, -3), O.linear_dgrad_np(g8, 21, w8, -3)),
+             (O.linear_wgrad(g8, 21, x8, 9), O.linear_wgrad_np(g8, 21, x8, 9))]
+    for plain, fast in pairs:
+        assert np.array_equal(plain.f64, fast.f64)
+        assert np.array_equal(plain.abs_sum, fast.abs_sum)
+        assert np.array_equal(plain.f32, fast.f32)
+        assert np.array_equal(plain.bf16, fast.bf16)

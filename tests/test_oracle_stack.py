@@ -1,0 +1,75 @@
+"""Pins for the oracle's mirror of the stress stack (CPU only): its bf16
+helpers and GELU against torch's float64 routines, and its backward pass
+against float64 autograd of the same network without quantisation."""
+import math
+
+import numpy as np
+import torch
+
+import oracle as O
+from oracle import stack as S
+
+
+def _bits(t):
+    return t.contiguous().view(torch.int16).numpy().view(np.uint16)
+
+
+def _ord(b):
+    b = b.astype(np.int32)
+    return np.where(b & 0x8000, -(b & 0x7FFF), b & 0x7FFF)
+
+
+def test_bf16_helpers_match_torch():
+    g = torch.Generator().manual_seed(1)
+    x = torch.randn(1000, 7, generator=g, dtype=torch.float64) * 100
+    assert np.array_equal(S.f64_to_bf16(x.numpy()), _bits(x.to(torch.float32).to(torch.bfloat16)))
+    b = _bits(x.to(torch.bfloat16))
+    assert np.array_equal(S.bf16_to_f64(b), x.to(torch.bfloat16).to(torch.float64).numpy())
+
+
+def test_step_input_drift():
+    base = _bits(torch.tensor([[1.0, -3.0, 0.5]], dtype=torch.bfloat16))
+    assert np.array_equal(S.step_input_bits(base, 0), base)
+    # step 10 pi: sin = 0 again up to rounding of pi; step = 20*asin(0.5) gives 2^4
+    s = 2.0 ** (8.0 * math.sin(7 / 20.0))
+    want = _bits((torch.tensor([[1.0, -3.0, 0.5]], dtype=torch.float64) * s).to(torch.float32).to(torch.bfloat16))
+    assert np.array_equal(S.step_input_bits(base, 7), want)
+
+
+def test_gelu_and_its_derivative_against_torch_float64():
+    y = (torch.linspace(-6, 6, 4001, dtype=torch.float64)).to(torch.bfloat16)
+    yb = _bits(y.view(1, -1))
+    ref = torch.nn.functional.gelu(y.to(torch.float64)).to(torch.float32).to(torch.bfloat16)
+    assert np.abs(_ord(S.gelu_bits(yb)) - _ord(_bits(ref.view(1, -1)))).max() <= 1
+    z = y.to(torch.float64).clone().requires_grad_(True)
+    torch.nn.functional.gelu(z).sum().backward()
+    np.testing.assert_allclose(S.gelu_grad(yb)[0], z.grad.numpy(), rtol=1e-12, atol=1e-15)
+
+
+def test_stack_backward_is_the_gradient_of_its_forward():
+    """Three small layers: the oracle's dW (FP8 path) must point along the
+    float64 autograd gradient of the unquantised network, and one SGD step
+    must lower the loss it reports."""
+    rng = np.random.default_rng(5)
+    L, T, d = 3, 128, 64
+    w = [(torch.from_numpy(rng.standard_normal((d, d))) * 0.15).to(torch.bfloat16) for _ in range(L)]
+    x = torch.from_numpy(rng.standard_normal((T, d))).to(torch.bfloat16)
+    tgt = torch.from_numpy(rng.standard_normal((T, d))).to(torch.bfloat16)
+    st = S.OracleStack([_bits(t) for t in w], _bits(x), _bits(tgt), lr=0.5)
+    rec = st.step(0)
+    ws = [t.to(torch.float64).clone().requires_grad_(True) for t in w]
+    h = x.to(torch.float64)
+    for l in range(L):
+        h = h @ ws[l].T
+        if l + 1 < L:
+            h = torch.nn.functional.gelu(h)
+    loss = torch.mean((h - tgt.to(torch.float64)) ** 2)
+    loss.backward()
+    assert abs(rec["loss"] - float(loss)) < 0.05 * float(loss)
+    for l in range(L):
+        mine = S.bf16_to_f64(rec["dw"][l].bf16).ravel()
+        ref = ws[l].grad.numpy().ravel()
+        cos = mine @ ref / (np.linalg.norm(mine) * np.linalg.norm(ref))
+        assert cos > 0.98, (l, cos)
+        assert 0.8 < np.linalg.norm(mine) / np.linalg.norm(ref) < 1.25
+    assert st.step(0)["loss"] < rec["loss"]

@@ -115,7 +115,7 @@ class LayerState:
     """Device buffers of one linear: bf16 inputs, FP8 copies in both layouts,
     device scalars, bf16 outputs."""
 
-    def __init__(self, wl, li, device, seed, backward, tokens=0):
+    def __init__(self, wl, li, device, seed, backward, tokens=0, transposed=False):
         l = wl.layers[li]
         T, K, N = tokens or wl.tokens, l.K, l.N
         self.T, self.K, self.N, self.name = T, K, N, l.name
@@ -128,9 +128,13 @@ class LayerState:
         self.scal_f = torch.zeros(4, dtype=torch.float32, device=device)
         self.scal_i = torch.zeros(4, dtype=torch.int32, device=device)
         self.backward = backward
+        self.transposed = transposed
         if backward:
-            self.x8t, self.w8t = torch.empty((K, T), **u8), torch.empty((K, N), **u8)
-            self.g8, self.g8t = torch.empty((T, N), **u8), torch.empty((N, T), **u8)
+            self.x8t = self.w8t = self.g8t = None
+            if transposed:
+                self.x8t, self.w8t = torch.empty((K, T), **u8), torch.empty((K, N), **u8)
+                self.g8t = torch.empty((N, T), **u8)
+            self.g8 = torch.empty((T, N), **u8)
             self.dx = torch.empty((T, K), dtype=torch.bfloat16, device=device)
             self.dw = torch.empty((N, K), dtype=torch.bfloat16, device=device)
         else:
@@ -183,8 +187,12 @@ def run_layer(ctx, L, timers=None):
     timed("gemm", lambda: ctx.linear_fwd(L.x8, bi[1:2], L.w8, bi[0:1], L.y))
     if L.backward:
         timed("amax_cast", lambda: ctx.cast_e5(L.g, None, d_amax_out=af[2:3], d_bias_out=bi[2:3], y=L.g8, y_t=L.g8t))
-        timed("gemm", lambda: ctx.linear_dgrad(L.g8, bi[2:3], None, L.w8t, bi[0:1], L.dx))
-        timed("gemm", lambda: ctx.linear_wgrad(None, L.g8t, bi[2:3], None, L.x8t, bi[1:2], L.dw, L.T))
+        if L.transposed:   # contraction over contiguous bytes, from the transposed copies
+            timed("gemm", lambda: ctx.linear_dgrad(L.g8, bi[2:3], None, L.w8t, bi[0:1], L.dx))
+            timed("gemm", lambda: ctx.linear_wgrad(None, L.g8t, bi[2:3], None, L.x8t, bi[1:2], L.dw, L.T))
+        else:              # the tensor core reads the forward layouts directly
+            timed("gemm", lambda: ctx.linear_dgrad(L.g8, bi[2:3], L.w8, None, bi[0:1], L.dx))
+            timed("gemm", lambda: ctx.linear_wgrad(L.g8, None, bi[2:3], L.x8, None, bi[1:2], L.dw, L.T))
 
 
 def dist_setup(n_gpus):
@@ -278,6 +286,8 @@ def main():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(I.WORKLOADS))
     ap.add_argument("--tokens", type=int, default=0, help="override the workload's token count (c4: 1, 16, 64, 2048)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--transposed-copies", action="store_true",
+                    help="also write transposed FP8 copies and contract the backward matmuls over contiguous bytes")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -296,7 +306,7 @@ def main():
     device = torch.device("cuda", local)
     warmup = max(3, args.warmup)
     ctx = fp8lin.Context(local)
-    layers = [LayerState(wl, li, device, I.BASE_SEED + 7919 * rank, wl.backward, args.tokens)
+    layers = [LayerState(wl, li, device, I.BASE_SEED + 7919 * rank, wl.backward, args.tokens, args.transposed_copies)
               for li in range(len(wl.layers))]
     peaks = load_peaks()
     tokens = args.tokens or wl.tokens
@@ -339,7 +349,7 @@ def main():
     gemm_tflops = args.steps * step_flops / (gemm_ms * 1e-3) / 1e12
     cast_ms = timers.total_ms("amax_cast")
     cast_elems = args.steps * sum(L.cast_elements() for L in layers)
-    bytes_per_elem = 4 if wl.backward else 3  # read once, write one byte per layout
+    bytes_per_elem = 4 if (wl.backward and args.transposed_copies) else 3  # read once, write one byte per layout
     fp8_peak = 2.0 * peaks["bf16_tflops_sustained"]
 
     # ---- end to end through the public API with host buffers ----
@@ -397,6 +407,7 @@ def main():
                    "passes": "fwd+bwd" if wl.backward else "fwd (weights quantised once at load)",
                    "scaling_bias": "FP8-AMAX, recomputed every step for " + ("W, X, dY" if wl.backward else "X"),
                    "l2": "inputs larger than L2 (each layer's tensors exceed 126 MB); no flush between steps",
+                   "fp8_layouts": "row-major + transposed copy" if args.transposed_copies else "row-major only",
                    "parallelism": "replicas" if world > 1 else "single"},
         "clocks": clocks,
         "e2e": e2e,

@@ -176,16 +176,20 @@ FP8_API fp8_status_t fp8_linear_fwd(fp8_ctx *ctx, const uint8_t *x8, const int32
 /* Input-gradient matmul (Section 2.2): dX[t, k] = (sum_n dY8[t, n] * W8[n, k]) * 2^-(s_g + s_w).
  *   dy8  [T, N] E5 bytes;  N % 16 == 0
  *   w8   [N, K] E4 bytes or NULL;  w8_t [K, N] E4 bytes or NULL.  At least one.
- *        This build contracts over contiguous bytes only and therefore needs
- *        w8_t (as written by the cast's y_t); w8 alone returns FP8_ERR_UNSUPPORTED.
+ *        With w8_t (as written by the cast's y_t) the contraction runs over
+ *        contiguous bytes; with w8 alone the tensor core reads W8 with its K
+ *        index contiguous and the contraction strided (needs K % 16 == 0), so
+ *        no transposed copy is required.  w8_t is used when both are given.
  *   dx   out [T, K], dtype dx_dt;  d_amax_dx NULL or out. */
 FP8_API fp8_status_t fp8_linear_dgrad(fp8_ctx *ctx, const uint8_t *dy8, const int32_t *d_bg, const uint8_t *w8,
                               const uint8_t *w8_t, const int32_t *d_bw, void *dx, fp8_dtype_t dx_dt,
                               float *d_amax_dx, int64_t T, int64_t K, int64_t N, fp8_conv_t conv, void *stream);
 
 /* Weight-gradient matmul (Section 2.2): dW[n, k] = (sum_t dY8[t, n] * X8[t, k]) * 2^-(s_g + s_x).
- *   dy8 [T, N] / dy8_t [N, T] E5 bytes, x8 [T, K] / x8_t [K, T] E4 bytes; T % 16 == 0.
- *   This build needs the transposed copies dy8_t and x8_t; the others may be NULL.
+ *   dy8 [T, N] / dy8_t [N, T] E5 bytes, x8 [T, K] / x8_t [K, T] E4 bytes.
+ *   Each operand in either layout (the transposed copy wins when both are
+ *   given): a transposed copy needs T % 16 == 0; dy8 needs N % 16 == 0 and x8
+ *   needs K % 16 == 0.  No transposed copy is required.
  *   dw  out [N, K], dtype dw_dt. */
 FP8_API fp8_status_t fp8_linear_wgrad(fp8_ctx *ctx, const uint8_t *dy8, const uint8_t *dy8_t, const int32_t *d_bg,
                               const uint8_t *x8, const uint8_t *x8_t, const int32_t *d_bx, void *dw,

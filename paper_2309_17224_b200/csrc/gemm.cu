@@ -25,6 +25,7 @@
 #include <cstdlib>
 
 #include "fp8lin_internal.cuh"
+#include "ptx.cuh"
 
 namespace fp8lin {
 
@@ -33,7 +34,6 @@ constexpr int kBK = 128;          // contraction bytes per stage = one 128-byte 
 constexpr int kUmmaK = 32;        // contraction elements per tcgen05.mma for 8-bit types
 constexpr int kGemmThreads = 192;
 constexpr int kGroupM = 8;        // tile rasterisation: m-blocks per group
-constexpr unsigned long long kWaitLimitNs = 1000ull * 1000ull * 1000ull;
 constexpr int kSlabBytes = 32 * 128;            // epilogue staging: 32 rows x 128 bytes, what one warp stores at a time
 constexpr int kEpiBytes = 4 * 2 * kSlabBytes;   // four epilogue warps, two slabs each
 
@@ -44,6 +44,7 @@ struct GemmParams {
     float *partial;               // [splits, M, N] FP32 partial sums when splits > 1
     const int32_t *d_sa, *d_sb;   // paper-convention biases of the two operands
     int delta_sum;                // format shifts to add to them
+    int a_mn, b_mn;               // operand stored with its M / N index contiguous (contraction index strided)
     const void *bias_vec;         // [N] or NULL
     int bias_dt;
     void *out;
@@ -57,62 +58,8 @@ struct GemmParams {
 };
 
 // ---------------------------------------------------------------------------
-// PTX wrappers
+// tcgen05 / TMEM wrappers (mbarrier and TMA wrappers live in ptx.cuh)
 // ---------------------------------------------------------------------------
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
-{
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
-{
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar)
-{
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
-{
-    uint32_t ok;
-    asm volatile(
-        "{\n"
-        ".reg .pred p;\n"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
-        "selp.u32 %0, 1, 0, p;\n"
-        "}\n"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-
-// Bounded wait.  Returns false when the wait expired or another role gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, unsigned *d_status)
-{
-    if (mbar_try_wait(bar, parity)) return true;
-    const unsigned long long t0 = global_timer_ns();
-    unsigned spins = 0;
-    while (!mbar_try_wait(bar, parity)) {
-        if ((++spins & 63u) == 0u) {
-            if (*abort_flag) return false;
-            if (global_timer_ns() - t0 > kWaitLimitNs) {
-                *abort_flag = 1;
-                atomicOr(d_status, FP8_FLAG_TIMEOUT);
-                return false;
-            }
-        }
-    }
-    return true;
-}
-
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int x, int y)
-{
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(x), "r"(y)
-        : "memory");
-}
 
 __device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t cols)
 {
@@ -170,6 +117,21 @@ __device__ __forceinline__ uint64_t smem_desc_k128(uint32_t smem_addr)
     uint64_t d = 0;
     d |= (uint64_t)((smem_addr >> 4) & 0x3FFFu);
     d |= (uint64_t)1 << 16;
+    d |= (uint64_t)(1024 >> 4) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)2 << 61;
+    return d;
+}
+
+// The same shared-memory rows read as an operand whose M / N index is the contiguous one ("MN-major"): a tile
+// is [contraction rows][128 bytes of M or N], 128-byte swizzled; eight contraction rows form one 1024-byte
+// group (stride offset), and a second block of 128 M / N values starts `lbo_bytes` further on (leading
+// offset).  One tcgen05.mma (K = 32) consumes 32 rows = 4096 bytes.
+__device__ __forceinline__ uint64_t smem_desc_mn128(uint32_t smem_addr, uint32_t lbo_bytes)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr >> 4) & 0x3FFFu);
+    d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
     d |= (uint64_t)(1024 >> 4) << 32;
     d |= (uint64_t)1 << 46;
     d |= (uint64_t)2 << 61;
@@ -452,8 +414,15 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                     if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p.d_status)) { alive = false; break; }
                     mbar_expect_tx(full_bar(s), L::kStageBytes);
                     const uint32_t a_dst = smem_base + s * L::kStageBytes;
-                    tma_load_2d(a_dst, &map_a, full_bar(s), k * kBK, m_blk * kBM);
-                    tma_load_2d(a_dst + L::kABytes, &map_b, full_bar(s), k * kBK, n_blk * BN);
+                    if (p.a_mn) tma_load_2d(a_dst, &map_a, full_bar(s), m_blk * kBM, k * kBK);
+                    else tma_load_2d(a_dst, &map_a, full_bar(s), k * kBK, m_blk * kBM);
+                    if (p.b_mn) {  // two blocks of 128 N values, 16 KB apart
+                        for (int h = 0; h < BN / 128; ++h)
+                            tma_load_2d(a_dst + L::kABytes + h * (128 * kBK), &map_b, full_bar(s), n_blk * BN + h * 128,
+                                        k * kBK);
+                    } else {
+                        tma_load_2d(a_dst + L::kABytes, &map_b, full_bar(s), k * kBK, n_blk * BN);
+                    }
                 }
             }
         }
@@ -475,13 +444,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                     if (!mbar_wait(full_bar(s), ph, abort_flag, p.d_status)) { alive = false; break; }
                     tc_fence_after();
                     const uint32_t a_addr = smem_base + s * L::kStageBytes;
-                    const uint64_t da = smem_desc_k128(a_addr);
-                    const uint64_t db = smem_desc_k128(a_addr + L::kABytes);
+                    const uint64_t da = p.a_mn ? smem_desc_mn128(a_addr, 128 * kBK) : smem_desc_k128(a_addr);
+                    const uint64_t db = p.b_mn ? smem_desc_mn128(a_addr + L::kABytes, 128 * kBK)
+                                               : smem_desc_k128(a_addr + L::kABytes);
+                    // per instruction (K = 32): 32 bytes along a 128-byte row, or 32 rows = 4096 bytes
+                    const uint32_t step_a = p.a_mn ? 256u : 2u, step_b = p.b_mn ? 256u : 2u;
 #pragma unroll
-                    for (int j = 0; j < kBK / kUmmaK; ++j) {
-                        // advancing 32 bytes inside the 128-byte swizzle row = +2 in the 16-byte address field
-                        umma_f8(d_tmem, da + 2u * j, db + 2u * j, p.idesc, (k > k0 || j > 0) ? 1u : 0u);
-                    }
+                    for (int j = 0; j < kBK / kUmmaK; ++j)
+                        umma_f8(d_tmem, da + step_a * j, db + step_b * j, p.idesc, (k > k0 || j > 0) ? 1u : 0u);
                     umma_commit(empty_bar(s));
                 }
                 if (alive) umma_commit(acc_full_bar(buf));
@@ -697,9 +667,11 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                     // peer's bytes may land first (the pending arrival keeps the phase open)
                     if (rank == 0) mbar_expect_tx(full_bar(s), 2 * L::kStageBytes);
                     const uint32_t a_dst = smem_base + s * L::kStageBytes;
-                    tma_load_2d_pair(a_dst, &map_a, leader_full, k * kBK, m_blk * 256 + (int)rank * kBM);
-                    tma_load_2d_pair(a_dst + L::kABytes, &map_b, leader_full, k * kBK,
-                                     n_blk * kPairBN + (int)rank * kPairHalfN);
+                    const int a_row = m_blk * 256 + (int)rank * kBM, b_row = n_blk * kPairBN + (int)rank * kPairHalfN;
+                    if (p.a_mn) tma_load_2d_pair(a_dst, &map_a, leader_full, a_row, k * kBK);
+                    else tma_load_2d_pair(a_dst, &map_a, leader_full, k * kBK, a_row);
+                    if (p.b_mn) tma_load_2d_pair(a_dst + L::kABytes, &map_b, leader_full, b_row, k * kBK);
+                    else tma_load_2d_pair(a_dst + L::kABytes, &map_b, leader_full, k * kBK, b_row);
                 }
             }
         }
@@ -719,11 +691,13 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                     if (!mbar_wait(full_bar(s), ph, abort_flag, p.d_status)) { alive = false; break; }
                     tc_fence_after();
                     const uint32_t a_addr = smem_base + s * L::kStageBytes;
-                    const uint64_t da = smem_desc_k128(a_addr);
-                    const uint64_t db = smem_desc_k128(a_addr + L::kABytes);
+                    const uint64_t da = p.a_mn ? smem_desc_mn128(a_addr, 128 * kBK) : smem_desc_k128(a_addr);
+                    const uint64_t db = p.b_mn ? smem_desc_mn128(a_addr + L::kABytes, 128 * kBK)
+                                               : smem_desc_k128(a_addr + L::kABytes);
+                    const uint32_t step_a = p.a_mn ? 256u : 2u, step_b = p.b_mn ? 256u : 2u;
 #pragma unroll
                     for (int j = 0; j < kBK / kUmmaK; ++j)
-                        umma_f8_pair(d_tmem, da + 2u * j, db + 2u * j, p.idesc, (k > 0 || j > 0) ? 1u : 0u);
+                        umma_f8_pair(d_tmem, da + step_a * j, db + step_b * j, p.idesc, (k > 0 || j > 0) ? 1u : 0u);
                     umma_commit_pair(empty_bar(s));
                 }
                 if (alive) umma_commit_pair(acc_full_bar(buf));
@@ -869,18 +843,24 @@ static bool encode_map(fp8_ctx *ctx, CUtensorMap *map, const void *base, int64_t
     return r == CUDA_SUCCESS;
 }
 
-// D[M,N] = A[M,Kc] * B[N,Kc]^T, unscaled by 2^-(bias_a + bias_b + delta_sum).
-static fp8_status_t run_gemm(fp8_ctx *ctx, const uint8_t *a, int a_fmt, const int32_t *d_ba, const uint8_t *b,
-                             int b_fmt, const int32_t *d_bb, int delta_sum, const void *bias_vec, int bias_dt,
-                             void *out, int out_dt, float *d_amax_out, int64_t M, int64_t N, int64_t Kc,
-                             cudaStream_t st)
+// D[M,N] = A * B^T over a contraction of length Kc, unscaled by 2^-(bias_a + bias_b + delta_sum).
+// A is stored [M, Kc] (a_mn = false) or [Kc, M] (a_mn = true); B is stored [N, Kc] or [Kc, N] likewise.
+static fp8_status_t run_gemm(fp8_ctx *ctx, const uint8_t *a, int a_fmt, bool a_mn, const int32_t *d_ba,
+                             const uint8_t *b, int b_fmt, bool b_mn, const int32_t *d_bb, int delta_sum,
+                             const void *bias_vec, int bias_dt, void *out, int out_dt, float *d_amax_out, int64_t M,
+                             int64_t N, int64_t Kc, cudaStream_t st)
 {
     if (M > 0x7FFFFFFF / 2 || N > 0x7FFFFFFF / 2 || Kc > 0x7FFFFFFF / 2) return FP8_ERR_SHAPE;
-    CUtensorMap map_a, map_b;
-    if (!encode_map(ctx, &map_a, a, M, Kc, kBM) || !encode_map(ctx, &map_b, b, N, Kc, kBN)) return FP8_ERR_CUDA;
     const bool pair = g_max_pairs > 0 && M > kBM && !g_force_single;
-    if (pair && !encode_map(ctx, &map_b, b, N, Kc, kPairHalfN)) return FP8_ERR_CUDA;
+    CUtensorMap map_a, map_b;
+    // an operand stored [Kc, M or N] is fetched as boxes of 128 contraction rows x 128 bytes
+    const bool ok_a = a_mn ? encode_map(ctx, &map_a, a, Kc, M, kBK) : encode_map(ctx, &map_a, a, M, Kc, kBM);
+    const bool ok_b = b_mn ? encode_map(ctx, &map_b, b, Kc, N, kBK)
+                           : encode_map(ctx, &map_b, b, N, Kc, pair ? kPairHalfN : kBN);
+    if (!ok_a || !ok_b) return FP8_ERR_CUDA;
     GemmParams p;
+    p.a_mn = a_mn ? 1 : 0;
+    p.b_mn = b_mn ? 1 : 0;
     p.M = (int)M; p.N = (int)N; p.K = (int)Kc;
     p.tiles_m = (int)((M + (pair ? 256 : kBM) - 1) / (pair ? 256 : kBM));
     p.tiles_n = (int)((N + kBN - 1) / kBN);
@@ -925,7 +905,8 @@ static fp8_status_t run_gemm(fp8_ctx *ctx, const uint8_t *a, int a_fmt, const in
     }
     p.d_amax_bits = reinterpret_cast<unsigned *>(d_amax_out);
     p.d_status = ctx->d_status;
-    p.idesc = pair ? make_idesc_pair(a_fmt, b_fmt) : make_idesc(a_fmt, b_fmt, kBN);
+    p.idesc = (pair ? make_idesc_pair(a_fmt, b_fmt) : make_idesc(a_fmt, b_fmt, kBN)) | ((uint32_t)p.a_mn << 15) |
+              ((uint32_t)p.b_mn << 16);
     if (d_amax_out && cudaMemsetAsync(d_amax_out, 0, sizeof(float), st) != cudaSuccess) return FP8_ERR_CUDA;
     int tiles = p.tiles_m * p.tiles_n;
     if (pair) {
@@ -966,8 +947,8 @@ fp8_status_t fp8_linear_fwd(fp8_ctx *ctx, const uint8_t *x8, const int32_t *d_bx
     if (T <= 0 || K <= 0 || N <= 0) return FP8_ERR_SHAPE;
     if (!aligned16(x8) || !aligned16(w8) || (K % 16) != 0 || (reinterpret_cast<uintptr_t>(y) & 3u)) return FP8_ERR_ALIGN;
     int delta = 2 * format_delta(FP8_E4, conv);
-    return run_gemm(ctx, x8, FP8_E4, d_bx, w8, FP8_E4, d_bw, delta, bias_vec, bias_dt, y, y_dt, d_amax_y, T, N, K,
-                    (cudaStream_t)stream);
+    return run_gemm(ctx, x8, FP8_E4, false, d_bx, w8, FP8_E4, false, d_bw, delta, bias_vec, bias_dt, y, y_dt, d_amax_y,
+                    T, N, K, (cudaStream_t)stream);
 }
 
 fp8_status_t fp8_linear_dgrad(fp8_ctx *ctx, const uint8_t *dy8, const int32_t *d_bg, const uint8_t *w8,
@@ -978,13 +959,17 @@ fp8_status_t fp8_linear_dgrad(fp8_ctx *ctx, const uint8_t *dy8, const int32_t *d
     if (!ctx || !dy8 || !d_bg || (!w8 && !w8_t) || !d_bw || !dx) return FP8_ERR_NULL;
     if ((int)conv < 0 || (int)conv > 1 || (int)dx_dt < 0 || (int)dx_dt > 2) return FP8_ERR_DTYPE;
     if (!out_dtype_ok(dx_dt)) return FP8_ERR_UNSUPPORTED;
-    if (!w8_t) return FP8_ERR_UNSUPPORTED;
     if (T <= 0 || K <= 0 || N <= 0) return FP8_ERR_SHAPE;
-    if (!aligned16(dy8) || !aligned16(w8_t) || (N % 16) != 0 || (reinterpret_cast<uintptr_t>(dx) & 3u))
+    // the transposed copy W8T[K,N] is contracted along contiguous bytes; W8[N,K] itself is read with its K
+    // index contiguous and the contraction strided
+    const bool w_mn = (w8_t == nullptr);
+    const uint8_t *w = w_mn ? w8 : w8_t;
+    if (!aligned16(dy8) || !aligned16(w) || (N % 16) != 0 || (w_mn && (K % 16) != 0) ||
+        (reinterpret_cast<uintptr_t>(dx) & 3u))
         return FP8_ERR_ALIGN;
     int delta = format_delta(FP8_E5, conv) + format_delta(FP8_E4, conv);
-    return run_gemm(ctx, dy8, FP8_E5, d_bg, w8_t, FP8_E4, d_bw, delta, nullptr, 0, dx, dx_dt, d_amax_dx, T, K, N,
-                    (cudaStream_t)stream);
+    return run_gemm(ctx, dy8, FP8_E5, false, d_bg, w, FP8_E4, w_mn, d_bw, delta, nullptr, 0, dx, dx_dt, d_amax_dx, T, K,
+                    N, (cudaStream_t)stream);
 }
 
 fp8_status_t fp8_linear_wgrad(fp8_ctx *ctx, const uint8_t *dy8, const uint8_t *dy8_t, const int32_t *d_bg,
@@ -995,12 +980,16 @@ fp8_status_t fp8_linear_wgrad(fp8_ctx *ctx, const uint8_t *dy8, const uint8_t *d
     if (!ctx || (!dy8 && !dy8_t) || !d_bg || (!x8 && !x8_t) || !d_bx || !dw) return FP8_ERR_NULL;
     if ((int)conv < 0 || (int)conv > 1 || (int)dw_dt < 0 || (int)dw_dt > 2) return FP8_ERR_DTYPE;
     if (!out_dtype_ok(dw_dt)) return FP8_ERR_UNSUPPORTED;
-    if (!dy8_t || !x8_t) return FP8_ERR_UNSUPPORTED;
     if (T <= 0 || K <= 0 || N <= 0) return FP8_ERR_SHAPE;
-    if (!aligned16(dy8_t) || !aligned16(x8_t) || (T % 16) != 0 || (reinterpret_cast<uintptr_t>(dw) & 3u))
+    // each operand comes either as its transposed copy (contraction over contiguous bytes) or as the forward
+    // layout dY8[T,N] / X8[T,K] (contraction strided)
+    const bool g_mn = (dy8_t == nullptr), x_mn = (x8_t == nullptr);
+    const uint8_t *g = g_mn ? dy8 : dy8_t, *xx = x_mn ? x8 : x8_t;
+    if (!aligned16(g) || !aligned16(xx) || (!g_mn && (T % 16) != 0) || (!x_mn && (T % 16) != 0) ||
+        (g_mn && (N % 16) != 0) || (x_mn && (K % 16) != 0) || (reinterpret_cast<uintptr_t>(dw) & 3u))
         return FP8_ERR_ALIGN;
     int delta = format_delta(FP8_E5, conv) + format_delta(FP8_E4, conv);
-    return run_gemm(ctx, dy8_t, FP8_E5, d_bg, x8_t, FP8_E4, d_bx, delta, nullptr, 0, dw, dw_dt, nullptr, N, K, T,
+    return run_gemm(ctx, g, FP8_E5, g_mn, d_bg, xx, FP8_E4, x_mn, d_bx, delta, nullptr, 0, dw, dw_dt, nullptr, N, K, T,
                     (cudaStream_t)stream);
 }
 

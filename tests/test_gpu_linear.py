@@ -73,14 +73,23 @@ def test_fwd_dgrad_wgrad_match_oracle(ctx, lib, T, K, N, conv):
         y = torch.full((T, N), float("nan"), dtype=dt, device="cuda")
         dx = torch.full((T, K), float("nan"), dtype=dt, device="cuda")
         dw = torch.full((N, K), float("nan"), dtype=dt, device="cuda")
+        # backward operands either as transposed copies (contraction over contiguous bytes) or in the forward
+        # layout (contraction strided), and mixed
+        dx2 = torch.full((T, K), float("nan"), dtype=dt, device="cuda")
+        dw2 = torch.full((N, K), float("nan"), dtype=dt, device="cuda")
+        dw3 = torch.full((N, K), float("nan"), dtype=dt, device="cuda")
         ctx.linear_fwd(qx.y, qx.bias, qw.y, qw.bias, y, conv=conv)
         ctx.linear_dgrad(qg.y, qg.bias, None, qw.y_t, qw.bias, dx, conv=conv)
         ctx.linear_wgrad(None, qg.y_t, qg.bias, None, qx.y_t, qx.bias, dw, T, conv=conv)
+        ctx.linear_dgrad(qg.y, qg.bias, qw.y, None, qw.bias, dx2, conv=conv)
+        ctx.linear_wgrad(qg.y, None, qg.bias, qx.y, None, qx.bias, dw2, T, conv=conv)
+        ctx.linear_wgrad(qg.y, None, qg.bias, None, qx.y_t, qx.bias, dw3, T, conv=conv)
         assert ctx.device_flags(clear=True) & lib.FLAG_TIMEOUT == 0
         refs = (O.linear_fwd(qx.ref, qx.shift, qw.ref, qw.shift),
                 O.linear_dgrad(qg.ref, qg.shift, qw.ref, qw.shift),
                 O.linear_wgrad(qg.ref, qg.shift, qx.ref, qx.shift))
-        for got, ref in zip((y, dx, dw), refs):
+        refs = refs + (refs[1], refs[2], refs[2])
+        for got, ref in zip((y, dx, dw, dx2, dw2, dw3), refs):
             if dt == torch.float32:
                 worst = assert_gemm_close(got.cpu().numpy(), ref)
                 print(f"[parity] T={T} K={K} N={N} conv={conv}: max |err| / sum|a*b| = 2^{np.log2(max(worst, 1e-300)):.1f}")
@@ -147,8 +156,11 @@ def test_matmul_argument_errors(ctx, lib):
     g8 = torch.zeros((32, 64), dtype=torch.uint8, device="cuda")
     dx = torch.zeros((32, 32), dtype=torch.bfloat16, device="cuda")
     with pytest.raises(lib.Fp8Error) as e:
-        ctx.linear_dgrad(g8, b, w8, None, b, dx)   # only the [N,K] layout given
-    assert e.value.status == lib.ERR_UNSUPPORTED
+        ctx.linear_dgrad(g8, b, w8[:, :8].contiguous(), None, b, dx[:, :8].contiguous())   # K = 8: rows of W8 not 16-byte multiples
+    assert e.value.status == lib.ERR_ALIGN
+    with pytest.raises(lib.Fp8Error) as e:
+        ctx.linear_dgrad(g8, b, None, None, b, dx)
+    assert e.value.status == lib.ERR_NULL
     with pytest.raises(lib.Fp8Error) as e:
         ctx.linear_fwd(x8, None, w8, b, y)
     assert e.value.status == lib.ERR_NULL
@@ -175,8 +187,8 @@ def test_full_size_layers_sampled(ctx, lib, wl_name, layer):
     dx = torch.empty((T, K), dtype=torch.bfloat16, device="cuda")
     dw = torch.empty((N, K), dtype=torch.bfloat16, device="cuda")
     ctx.linear_fwd(qx.y, qx.bias, qw.y, qw.bias, y)
-    ctx.linear_dgrad(qg.y, qg.bias, None, qw.y_t, qw.bias, dx)
-    ctx.linear_wgrad(None, qg.y_t, qg.bias, None, qx.y_t, qx.bias, dw, T)
+    ctx.linear_dgrad(qg.y, qg.bias, qw.y, None, qw.bias, dx)
+    ctx.linear_wgrad(qg.y, None, qg.bias, qx.y, None, qx.bias, dw, T)
     assert ctx.device_flags(clear=True) & lib.FLAG_TIMEOUT == 0
     rng = np.random.default_rng(layer + 1)
     cases = ((O.FWD, y, (qx.ref, O.N_E4, qx.shift, qw.ref, O.N_E4, qw.shift)),

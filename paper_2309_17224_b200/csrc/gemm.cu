@@ -33,13 +33,14 @@ constexpr int kBM = 128;          // rows of D per tile = TMEM lanes
 constexpr int kBK = 128;          // contraction bytes per stage = one 128-byte swizzle row
 constexpr int kUmmaK = 32;        // contraction elements per tcgen05.mma for 8-bit types
 constexpr int kGemmThreads = 192;
-constexpr int kGroupM = 8;        // tile rasterisation: m-blocks per group
+constexpr int kGroupM = 16;       // tile rasterisation: m-blocks per group
 constexpr int kSlabBytes = 32 * 128;            // epilogue staging: 32 rows x 128 bytes, what one warp stores at a time
 constexpr int kEpiBytes = 4 * 2 * kSlabBytes;   // four epilogue warps, two slabs each
 
 struct GemmParams {
     int M, N, K;
     int tiles_m, tiles_n, num_k;
+    int group_m;                  // tile rasterisation: m-blocks per group
     int splits, kb_per_split;     // split-K (single-CTA kernel only): k-blocks per split
     float *partial;               // [splits, M, N] FP32 partial sums when splits > 1
     const int32_t *d_sa, *d_sb;   // paper-convention biases of the two operands
@@ -164,10 +165,10 @@ struct GemmSmem {
 
 __device__ __forceinline__ void tile_coords(int tile, const GemmParams &p, int &m_blk, int &n_blk)
 {
-    const int group = kGroupM * p.tiles_n;
+    const int group = p.group_m * p.tiles_n;
     const int g = tile / group;
-    const int first_m = g * kGroupM;
-    const int gm = min(kGroupM, p.tiles_m - first_m);
+    const int first_m = g * p.group_m;
+    const int gm = min(p.group_m, p.tiles_m - first_m);
     const int r = tile - g * group;
     m_blk = first_m + r % gm;
     n_blk = r / gm;
@@ -784,6 +785,7 @@ constexpr int kBN = 256;
 constexpr int kStages = 4;
 
 static bool g_force_single = false;  // set from FP8LIN_SINGLE_CTA=1 (A/B comparison of the two kernels)
+static int g_group_m = 0;               // set from FP8LIN_GROUP_M (experiments with the tile order)
 static bool g_no_splitk = false;        // set from FP8LIN_NO_SPLITK=1
 static bool g_direct_epilogue = false;  // set from FP8LIN_DIRECT_EPILOGUE=1 (A/B comparison of the epilogues)
 static int g_max_pairs = 0;  // CTA pairs that can be resident at once (0: pair kernel unavailable)
@@ -820,6 +822,8 @@ cudaError_t configure_gemm_kernels(int max_smem_optin)
     g_max_pairs = clusters;
     const char *env = getenv("FP8LIN_SINGLE_CTA");
     g_force_single = env && env[0] == '1';
+    env = getenv("FP8LIN_GROUP_M");
+    g_group_m = env ? atoi(env) : 0;
     env = getenv("FP8LIN_NO_SPLITK");
     g_no_splitk = env && env[0] == '1';
     env = getenv("FP8LIN_DIRECT_EPILOGUE");
@@ -859,6 +863,7 @@ static fp8_status_t run_gemm(fp8_ctx *ctx, const uint8_t *a, int a_fmt, bool a_m
                            : encode_map(ctx, &map_b, b, N, Kc, pair ? kPairHalfN : kBN);
     if (!ok_a || !ok_b) return FP8_ERR_CUDA;
     GemmParams p;
+    p.group_m = g_group_m > 0 ? g_group_m : kGroupM;
     p.a_mn = a_mn ? 1 : 0;
     p.b_mn = b_mn ? 1 : 0;
     p.M = (int)M; p.N = (int)N; p.K = (int)Kc;

@@ -89,11 +89,11 @@ FP8_API fp8_status_t fp8_device_flags(fp8_ctx *ctx, void *stream, unsigned *flag
 
 /* amax = max(|x|) over the whole tensor (Eq. 3, first line).
  *   x       [rows, cols] with leading dimension ld (elements), dtype x_dt
- *           (this build: FP8_BF16 only)
+ *           (FP8_BF16, FP8_F16 or FP8_F32)
  *   d_amax  out, one float.  NaN if any element is NaN, else the exact maximum
  *           magnitude (inf included).
- * Needs x 2-byte aligned only; 16-byte aligned x with ld == cols (or ld and
- * cols multiples of 8) takes the vectorised path. */
+ * Needs x aligned to its element size only; 16-byte aligned x with ld == cols
+ * (or 16-byte aligned rows) takes the vectorised path. */
 FP8_API fp8_status_t fp8_amax(fp8_ctx *ctx, const void *x, fp8_dtype_t x_dt, int64_t rows, int64_t cols, int64_t ld,
                       float *d_amax, void *stream);
 
@@ -134,7 +134,7 @@ FP8_API fp8_status_t fp8_scaling_bias_host(float amax, fp8_format_t fmt, fp8_con
 
 /* Scale-and-cast (Eq. 1 then the cast of Section 2.1): code = RNE_fp8(x * 2^(bias + delta)),
  * saturating at the format's largest finite value; NaN stays NaN.
- *   x          [rows, cols], leading dimension ld, dtype x_dt (FP8_BF16 only)
+ *   x          [rows, cols], leading dimension ld, dtype x_dt (FP8_BF16, FP8_F16 or FP8_F32)
  *   d_bias     device int32, the paper-convention bias to apply.  Passing a
  *              constant chosen by the caller is the paper's FP8-CSCALE.
  *              NULL selects FP8-AMAX: amax and bias are computed here first

@@ -63,13 +63,13 @@ def _L():
         _lib.orc_encode.argtypes = [c.c_int, c.c_double]
         _lib.orc_f32_to_bf16.restype = c.c_uint16
         _lib.orc_f32_to_bf16.argtypes = [c.c_float]
-        _lib.orc_amax_bf16.restype = c.c_float
-        _lib.orc_amax_bf16.argtypes = [c.c_void_p, c.c_int64, c.c_int64, c.c_int64]
+        _lib.orc_amax.restype = c.c_float
+        _lib.orc_amax.argtypes = [c.c_void_p, c.c_int, c.c_int64, c.c_int64, c.c_int64]
         _lib.orc_scaling_bias.restype = c.c_int
         _lib.orc_scaling_bias.argtypes = [c.c_float, c.c_double, c.c_int]
-        _lib.orc_cast_bf16.restype = None
-        _lib.orc_cast_bf16.argtypes = [c.c_void_p, c.c_int64, c.c_int64, c.c_int64, c.c_int, c.c_int,
-                                       c.c_void_p, c.c_void_p]
+        _lib.orc_cast.restype = None
+        _lib.orc_cast.argtypes = [c.c_void_p, c.c_int, c.c_int64, c.c_int64, c.c_int64, c.c_int, c.c_int,
+                                  c.c_void_p, c.c_void_p]
         gemm_args = [c.c_void_p, c.c_int, c.c_int, c.c_void_p, c.c_int, c.c_int]
         tail = [c.c_int64, c.c_int64, c.c_int64, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p]
         _lib.orc_linear_fwd.restype = None
@@ -143,14 +143,17 @@ def f32_to_bf16_bits(x: np.ndarray) -> np.ndarray:
 # amax, bias, cast
 # ----------------------------------------------------------------------------
 
-def _bf16(x: np.ndarray) -> np.ndarray:
-    assert x.dtype == np.uint16 and x.ndim == 2, "bf16 tensors are passed as 2-D uint16 bit patterns"
-    return np.ascontiguousarray(x)
+def _tensor(x: np.ndarray):
+    """A 2-D input tensor and its type id: bf16 is passed as uint16 bit
+    patterns, fp16 as numpy float16, fp32 as numpy float32."""
+    assert x.ndim == 2
+    dt = {np.dtype(np.uint16): 0, np.dtype(np.float16): 1, np.dtype(np.float32): 2}[x.dtype]
+    return np.ascontiguousarray(x), dt
 
 
 def amax(x_bits: np.ndarray) -> float:
-    x = _bf16(x_bits)
-    return float(_L().orc_amax_bf16(x.ctypes.data, x.shape[0], x.shape[1], x.shape[1]))
+    x, dt = _tensor(x_bits)
+    return float(_L().orc_amax(x.ctypes.data, dt, x.shape[0], x.shape[1], x.shape[1]))
 
 
 def scaling_bias(amax_value: float, kind: int, conv: int = CONV_PAPER, margin: int = 0) -> int:
@@ -160,12 +163,12 @@ def scaling_bias(amax_value: float, kind: int, conv: int = CONV_PAPER, margin: i
 def cast(x_bits: np.ndarray, shift: int, fmt: int, transposed: bool = False):
     """codes = encode_fmt(x * 2^shift); returns y[rows, cols] and, if asked,
     also y_t[cols, rows]."""
-    x = _bf16(x_bits)
+    x, dt = _tensor(x_bits)
     rows, cols = x.shape
     y = np.empty((rows, cols), dtype=np.uint8)
     y_t = np.empty((cols, rows), dtype=np.uint8) if transposed else None
-    _L().orc_cast_bf16(x.ctypes.data, rows, cols, cols, int(shift), fmt, y.ctypes.data,
-                       y_t.ctypes.data if transposed else None)
+    _L().orc_cast(x.ctypes.data, dt, rows, cols, cols, int(shift), fmt, y.ctypes.data,
+                  y_t.ctypes.data if transposed else None)
     return (y, y_t) if transposed else y
 
 

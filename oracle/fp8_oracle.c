@@ -156,6 +156,25 @@ static double bf16_to_double(uint16_t h)
     return (double)f;
 }
 
+/* IEEE half (Table 7 row "FP16": E=5, M=10, bias 15) -> double, from the bit fields. */
+static double f16_to_double(uint16_t h)
+{
+    unsigned s = h >> 15, e = (h >> 10) & 0x1Fu, m = h & 0x3FFu;
+    double v;
+    if (e == 0x1Fu) v = m ? NAN : INFINITY;
+    else if (e == 0) v = ldexp((double)m / 1024.0, -14);
+    else v = ldexp(1.0 + (double)m / 1024.0, (int)e - 15);
+    return s ? -v : v;
+}
+
+/* Element i of a tensor of the given 16/32-bit type (0 bf16, 1 fp16, 2 fp32) as a double: always exact. */
+static double load_elem(const void *x, int dtype, int64_t i)
+{
+    if (dtype == 0) return bf16_to_double(((const uint16_t *)x)[i]);
+    if (dtype == 1) return f16_to_double(((const uint16_t *)x)[i]);
+    return (double)((const float *)x)[i];
+}
+
 /* float -> bfloat16, round to nearest even (NaN stays NaN, overflow -> inf). */
 uint16_t orc_f32_to_bf16(float f)
 {
@@ -172,13 +191,13 @@ uint16_t orc_f32_to_bf16(float f)
 /* ------------------------------------------------------------------------- */
 
 /* amax = max(|tensor|).  A NaN anywhere makes the result NaN. */
-float orc_amax_bf16(const uint16_t *x, int64_t rows, int64_t cols, int64_t ld)
+float orc_amax(const void *x, int dtype, int64_t rows, int64_t cols, int64_t ld)
 {
     double best = 0.0;
     int saw_nan = 0;
     for (int64_t r = 0; r < rows; ++r)
         for (int64_t c = 0; c < cols; ++c) {
-            double v = fabs(bf16_to_double(x[r * ld + c]));
+            double v = fabs(load_elem(x, dtype, r * ld + c));
             if (isnan(v)) saw_nan = 1;
             else if (v > best) best = v;
         }
@@ -204,13 +223,13 @@ int orc_scaling_bias(float amax, double max_num, int margin)
 
 /* y[r, c] = encode_f(x[r, c] * 2^shift); y_t[c, r] is the same code.  Either
  * output may be NULL. */
-void orc_cast_bf16(const uint16_t *x, int64_t rows, int64_t cols, int64_t ld, int shift, int f,
-                   uint8_t *y, uint8_t *y_t)
+void orc_cast(const void *x, int dtype, int64_t rows, int64_t cols, int64_t ld, int shift, int f, uint8_t *y,
+              uint8_t *y_t)
 {
 #pragma omp parallel for schedule(static)
     for (int64_t r = 0; r < rows; ++r)
         for (int64_t c = 0; c < cols; ++c) {
-            double v = ldexp(bf16_to_double(x[r * ld + c]), shift);
+            double v = ldexp(load_elem(x, dtype, r * ld + c), shift);
             uint8_t code = (uint8_t)orc_encode(f, v);
             if (y) y[r * cols + c] = code;
             if (y_t) y_t[c * rows + r] = code;

@@ -22,16 +22,41 @@ struct AmaxOut {
     int fmt, conv, margin;
 };
 
-__device__ __forceinline__ uint32_t packed_abs_max(uint32_t acc, uint32_t w)
+// |x| orders like an unsigned integer on the bit pattern with the sign cleared (NaN > inf > finite) for all
+// three input types.  16-bit types keep two lanes per word; fp32 one.
+template <int DT>
+__device__ __forceinline__ uint32_t fold_word(uint32_t acc, uint32_t w)
 {
-    return __vmaxu2(acc, w & 0x7FFF7FFFu);
+    return DT == FP8_F32 ? max(acc, w & 0x7FFFFFFFu) : __vmaxu2(acc, w & 0x7FFF7FFFu);
+}
+template <int DT>
+__device__ __forceinline__ uint32_t fold_elem(uint32_t acc, const void *x, int64_t i)
+{
+    if (DT == FP8_F32) return max(acc, reinterpret_cast<const uint32_t *>(x)[i] & 0x7FFFFFFFu);
+    return __vmaxu2(acc, (uint32_t)reinterpret_cast<const uint16_t *>(x)[i] & 0x7FFFu);
+}
+template <int DT>
+__device__ __forceinline__ uint32_t lane_key(uint32_t acc)
+{
+    return DT == FP8_F32 ? acc : max(acc & 0xFFFFu, acc >> 16);
+}
+// the winning bit pattern as float bits
+template <int DT>
+__device__ __forceinline__ uint32_t key_to_float_bits(uint32_t key)
+{
+    if (DT == FP8_F32) return key;
+    if (DT == FP8_BF16) return key << 16;
+    float f;
+    asm("cvt.f32.f16 %0, %1;" : "=f"(f) : "h"((uint16_t)key));
+    return __float_as_uint(f);
 }
 
-// Block-level reduction of a packed running max, then the grid-level step.
-__device__ __forceinline__ void amax_finish(uint32_t packed, const AmaxOut &o)
+// Block-level reduction of a running max, then the grid-level step.
+template <int DT>
+__device__ __forceinline__ void amax_finish(uint32_t acc, const AmaxOut &o)
 {
     __shared__ uint32_t warp_max[kAmaxThreads / 32];
-    uint32_t m = max(packed & 0xFFFFu, packed >> 16);
+    uint32_t m = lane_key<DT>(acc);
     m = __reduce_max_sync(0xFFFFFFFFu, m);
     if ((threadIdx.x & 31) == 0) warp_max[threadIdx.x >> 5] = m;
     __syncthreads();
@@ -45,7 +70,7 @@ __device__ __forceinline__ void amax_finish(uint32_t packed, const AmaxOut &o)
             __threadfence();
             uint32_t total = atomicExch(&o.slot[0], 0u);
             o.slot[1] = 0u;
-            uint32_t fbits = total << 16;  // bf16 -> float bit pattern
+            uint32_t fbits = key_to_float_bits<DT>(total);
             *o.d_amax = __uint_as_float(fbits);
             unsigned flags = 0;
             int b = bias_from_amax_bits(fbits, o.fmt, o.conv, o.margin, &flags);
@@ -57,9 +82,9 @@ __device__ __forceinline__ void amax_finish(uint32_t packed, const AmaxOut &o)
     }
 }
 
-// Contiguous tensor seen as nvec 16-byte vectors plus a scalar tail.
-__global__ void __launch_bounds__(kAmaxThreads) amax_flat_kernel(const uint4 *__restrict__ x, int64_t nvec,
-                                                                 const uint16_t *__restrict__ tail, int ntail,
+// Contiguous tensor seen as nvec 16-byte vectors plus a scalar tail of ntail elements.
+template <int DT>
+__global__ void __launch_bounds__(kAmaxThreads) amax_flat_kernel(const uint4 *__restrict__ x, int64_t nvec, int ntail,
                                                                  AmaxOut o)
 {
     uint32_t acc = 0;
@@ -73,40 +98,42 @@ __global__ void __launch_bounds__(kAmaxThreads) amax_flat_kernel(const uint4 *__
         }
 #pragma unroll
         for (int j = 0; j < kAmaxUnroll; ++j) {
-            acc = packed_abs_max(acc, v[j].x);
-            acc = packed_abs_max(acc, v[j].y);
-            acc = packed_abs_max(acc, v[j].z);
-            acc = packed_abs_max(acc, v[j].w);
+            acc = fold_word<DT>(acc, v[j].x);
+            acc = fold_word<DT>(acc, v[j].y);
+            acc = fold_word<DT>(acc, v[j].z);
+            acc = fold_word<DT>(acc, v[j].w);
         }
     }
-    if (blockIdx.x == 0 && (int)threadIdx.x < ntail) acc = packed_abs_max(acc, (uint32_t)tail[threadIdx.x]);
-    amax_finish(acc, o);
+    constexpr int kPerVec = DT == FP8_F32 ? 4 : 8;
+    if (blockIdx.x == 0 && (int)threadIdx.x < ntail) acc = fold_elem<DT>(acc, x, nvec * kPerVec + threadIdx.x);
+    amax_finish<DT>(acc, o);
 }
 
-// General [rows, cols] with leading dimension ld; vec != 0 promises 16-byte
-// aligned rows (x aligned, ld % 8 == 0).
-__global__ void __launch_bounds__(kAmaxThreads) amax_rows_kernel(const uint16_t *__restrict__ x, int64_t rows,
+// General [rows, cols] with leading dimension ld; vec != 0 promises 16-byte aligned rows.
+template <int DT>
+__global__ void __launch_bounds__(kAmaxThreads) amax_rows_kernel(const void *__restrict__ x, int64_t rows,
                                                                  int64_t cols, int64_t ld, int vec, AmaxOut o)
 {
+    constexpr int kPerVec = DT == FP8_F32 ? 4 : 8;
+    constexpr int kB = DT == FP8_F32 ? 4 : 2;
     uint32_t acc = 0;
     for (int64_t r = blockIdx.x; r < rows; r += gridDim.x) {
-        const uint16_t *row = x + r * ld;
         int64_t done = 0;
         if (vec) {
-            int64_t nv = cols / 8;
-            const uint4 *rv = reinterpret_cast<const uint4 *>(row);
+            int64_t nv = cols / kPerVec;
+            const uint4 *rv = reinterpret_cast<const uint4 *>(reinterpret_cast<const uint8_t *>(x) + r * ld * kB);
             for (int64_t i = threadIdx.x; i < nv; i += kAmaxThreads) {
                 uint4 v = __ldg(rv + i);
-                acc = packed_abs_max(acc, v.x);
-                acc = packed_abs_max(acc, v.y);
-                acc = packed_abs_max(acc, v.z);
-                acc = packed_abs_max(acc, v.w);
+                acc = fold_word<DT>(acc, v.x);
+                acc = fold_word<DT>(acc, v.y);
+                acc = fold_word<DT>(acc, v.z);
+                acc = fold_word<DT>(acc, v.w);
             }
-            done = nv * 8;
+            done = nv * kPerVec;
         }
-        for (int64_t c = done + threadIdx.x; c < cols; c += kAmaxThreads) acc = packed_abs_max(acc, (uint32_t)row[c]);
+        for (int64_t c = done + threadIdx.x; c < cols; c += kAmaxThreads) acc = fold_elem<DT>(acc, x, r * ld + c);
     }
-    amax_finish(acc, o);
+    amax_finish<DT>(acc, o);
 }
 
 __global__ void scaling_bias_kernel(const float *__restrict__ d_amax, int fmt, int conv, int margin,
@@ -117,29 +144,36 @@ __global__ void scaling_bias_kernel(const float *__restrict__ d_amax, int fmt, i
     if (flags) atomicOr(d_status, flags);
 }
 
-cudaError_t launch_amax_bias(fp8_ctx *ctx, const void *x, int64_t rows, int64_t cols, int64_t ld, float *d_amax,
-                             int32_t *d_bias, int fmt, int conv, int margin, cudaStream_t stream)
+template <int DT>
+static cudaError_t launch_amax_dt(fp8_ctx *ctx, const void *x, int64_t rows, int64_t cols, int64_t ld, AmaxOut o,
+                                  cudaStream_t stream)
 {
-    AmaxOut o{take_slot(ctx), d_amax, d_bias, ctx->d_status, fmt, conv, margin};
+    constexpr int kPerVec = DT == FP8_F32 ? 4 : 8;
     const bool aligned = (reinterpret_cast<uintptr_t>(x) & 15u) == 0;
     const int max_blocks = ctx->sm_count * 8;
     if (ld == cols && aligned) {
         int64_t n = rows * cols;
-        int64_t nvec = n / 8;
-        int ntail = (int)(n - nvec * 8);
+        int64_t nvec = n / kPerVec;
+        int ntail = (int)(n - nvec * kPerVec);
         int64_t chunk = (int64_t)kAmaxThreads * kAmaxUnroll;
         int64_t want = (nvec + chunk - 1) / chunk;
         int blocks = (int)(want < 1 ? 1 : (want > max_blocks ? max_blocks : want));
-        amax_flat_kernel<<<blocks, kAmaxThreads, 0, stream>>>(reinterpret_cast<const uint4 *>(x), nvec,
-                                                             reinterpret_cast<const uint16_t *>(x) + nvec * 8, ntail,
-                                                             o);
+        amax_flat_kernel<DT><<<blocks, kAmaxThreads, 0, stream>>>(reinterpret_cast<const uint4 *>(x), nvec, ntail, o);
     } else {
-        int vec = (aligned && (ld % 8) == 0) ? 1 : 0;
+        int vec = (aligned && (ld % kPerVec) == 0) ? 1 : 0;
         int blocks = (int)(rows > max_blocks ? max_blocks : rows);
-        amax_rows_kernel<<<blocks, kAmaxThreads, 0, stream>>>(reinterpret_cast<const uint16_t *>(x), rows, cols, ld,
-                                                             vec, o);
+        amax_rows_kernel<DT><<<blocks, kAmaxThreads, 0, stream>>>(x, rows, cols, ld, vec, o);
     }
     return cudaGetLastError();
+}
+
+cudaError_t launch_amax_bias(fp8_ctx *ctx, const void *x, int dt, int64_t rows, int64_t cols, int64_t ld, float *d_amax,
+                             int32_t *d_bias, int fmt, int conv, int margin, cudaStream_t stream)
+{
+    AmaxOut o{take_slot(ctx), d_amax, d_bias, ctx->d_status, fmt, conv, margin};
+    if (dt == FP8_BF16) return launch_amax_dt<FP8_BF16>(ctx, x, rows, cols, ld, o, stream);
+    if (dt == FP8_F16) return launch_amax_dt<FP8_F16>(ctx, x, rows, cols, ld, o, stream);
+    return launch_amax_dt<FP8_F32>(ctx, x, rows, cols, ld, o, stream);
 }
 
 }  // namespace fp8lin
@@ -151,10 +185,10 @@ fp8_status_t fp8_amax(fp8_ctx *ctx, const void *x, fp8_dtype_t x_dt, int64_t row
 {
     if (!ctx || !x || !d_amax) return FP8_ERR_NULL;
     if ((int)x_dt < 0 || (int)x_dt > 2) return FP8_ERR_DTYPE;
-    if (x_dt != FP8_BF16) return FP8_ERR_UNSUPPORTED;
     if (rows <= 0 || cols <= 0 || ld < cols) return FP8_ERR_SHAPE;
-    if (reinterpret_cast<uintptr_t>(x) & 1u) return FP8_ERR_ALIGN;
-    cudaError_t e = fp8lin::launch_amax_bias(ctx, x, rows, cols, ld, d_amax, nullptr, 0, 0, 0, (cudaStream_t)stream);
+    if (reinterpret_cast<uintptr_t>(x) & (x_dt == FP8_F32 ? 3u : 1u)) return FP8_ERR_ALIGN;
+    cudaError_t e = fp8lin::launch_amax_bias(ctx, x, (int)x_dt, rows, cols, ld, d_amax, nullptr, 0, 0, 0,
+                                             (cudaStream_t)stream);
     return e == cudaSuccess ? FP8_OK : FP8_ERR_CUDA;
 }
 

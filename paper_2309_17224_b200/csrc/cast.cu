@@ -23,53 +23,51 @@ namespace fp8lin {
 // contiguous, row-major output only
 // ---------------------------------------------------------------------------
 
-template <int FMT, bool TWO_STEP>
+template <int FMT, int DT, bool TWO_STEP>
 __device__ __forceinline__ void cast_flat_body(const uint4 *__restrict__ x, uint4 *__restrict__ y, int64_t nout,
                                                Pow2Pair p, bool &sat)
 {
-    // nout = number of 16-byte output vectors; each consumes two input vectors.
+    // nout = number of 16-byte output vectors; each consumes kIn input vectors (16 elements).
+    constexpr int kIn = InType<DT>::kBytes;  // 2 vectors of 16-bit elements, 4 of fp32
     const int64_t chunk = (int64_t)kCastThreads * 2;
     const int64_t nchunks = (nout + chunk - 1) / chunk;
     for (int64_t c = nchunks - 1 - blockIdx.x; c >= 0; c -= gridDim.x) {
-        int64_t i0 = c * chunk + threadIdx.x;
-        int64_t i1 = i0 + kCastThreads;
-        uint4 a0, a1, b0, b1;
-        bool ok0 = i0 < nout, ok1 = i1 < nout;
-        if (ok0) { a0 = __ldcs(x + 2 * i0); a1 = __ldcs(x + 2 * i0 + 1); }
-        if (ok1) { b0 = __ldcs(x + 2 * i1); b1 = __ldcs(x + 2 * i1 + 1); }
-        if (ok0) {
-            uint4 o;
-            o.x = cast4<FMT, TWO_STEP>(a0.x, a0.y, p, sat);
-            o.y = cast4<FMT, TWO_STEP>(a0.z, a0.w, p, sat);
-            o.z = cast4<FMT, TWO_STEP>(a1.x, a1.y, p, sat);
-            o.w = cast4<FMT, TWO_STEP>(a1.z, a1.w, p, sat);
-            y[i0] = o;
-        }
-        if (ok1) {
-            uint4 o;
-            o.x = cast4<FMT, TWO_STEP>(b0.x, b0.y, p, sat);
-            o.y = cast4<FMT, TWO_STEP>(b0.z, b0.w, p, sat);
-            o.z = cast4<FMT, TWO_STEP>(b1.x, b1.y, p, sat);
-            o.w = cast4<FMT, TWO_STEP>(b1.z, b1.w, p, sat);
-            y[i1] = o;
-        }
+        int64_t idx[2] = {c * chunk + threadIdx.x, c * chunk + threadIdx.x + kCastThreads};
+        uint4 v[2][kIn];
+#pragma unroll
+        for (int u = 0; u < 2; ++u)
+            if (idx[u] < nout) {
+#pragma unroll
+                for (int j = 0; j < kIn; ++j) v[u][j] = __ldcs(x + kIn * idx[u] + j);
+            }
+#pragma unroll
+        for (int u = 0; u < 2; ++u)
+            if (idx[u] < nout) {
+                const uint32_t *w = reinterpret_cast<const uint32_t *>(&v[u][0]);
+                constexpr int kW = InType<DT>::kWords4;
+                uint4 o;
+                o.x = cast4w<FMT, DT, TWO_STEP>(w + 0 * kW, p, sat);
+                o.y = cast4w<FMT, DT, TWO_STEP>(w + 1 * kW, p, sat);
+                o.z = cast4w<FMT, DT, TWO_STEP>(w + 2 * kW, p, sat);
+                o.w = cast4w<FMT, DT, TWO_STEP>(w + 3 * kW, p, sat);
+                y[idx[u]] = o;
+            }
     }
 }
 
-template <int FMT>
+template <int FMT, int DT>
 __global__ void __launch_bounds__(kCastThreads) cast_flat_kernel(const uint4 *__restrict__ x, uint4 *__restrict__ y,
-                                                                 int64_t nout, const uint16_t *__restrict__ tail_in,
-                                                                 uint8_t *__restrict__ tail_out, int ntail,
+                                                                 int64_t nout, int ntail,
                                                                  const int32_t *__restrict__ d_bias, int delta,
                                                                  unsigned *d_status)
 {
     const int s = __ldg(d_bias) + delta;
     const Pow2Pair p = make_pow2_pair(s);
     bool sat = false;
-    if (s >= -126 && s <= 127) cast_flat_body<FMT, false>(x, y, nout, p, sat);
-    else cast_flat_body<FMT, true>(x, y, nout, p, sat);
+    if (s >= -126 && s <= 127) cast_flat_body<FMT, DT, false>(x, y, nout, p, sat);
+    else cast_flat_body<FMT, DT, true>(x, y, nout, p, sat);
     if (blockIdx.x == 0 && (int)threadIdx.x < ntail)
-        tail_out[threadIdx.x] = cast1<FMT, true>(tail_in[threadIdx.x], p, sat);
+        reinterpret_cast<uint8_t *>(y)[nout * 16 + threadIdx.x] = cast1<FMT, DT, true>(x, nout * 16 + threadIdx.x, p, sat);
     if (__syncthreads_or(sat) && threadIdx.x == 0) atomicOr(d_status, FP8_FLAG_SATURATED);
 }
 
@@ -79,8 +77,8 @@ __global__ void __launch_bounds__(kCastThreads) cast_flat_kernel(const uint4 *__
 
 constexpr int kTile = 128;
 
-template <int FMT>
-__global__ void __launch_bounds__(kCastThreads) cast_tile_kernel(const uint16_t *__restrict__ x, int64_t rows,
+template <int FMT, int DT>
+__global__ void __launch_bounds__(kCastThreads) cast_tile_kernel(const void *__restrict__ x, int64_t rows,
                                                                  int64_t cols, int64_t ld,
                                                                  const int32_t *__restrict__ d_bias, int delta,
                                                                  uint8_t *__restrict__ y, uint8_t *__restrict__ y_t,
@@ -90,6 +88,8 @@ __global__ void __launch_bounds__(kCastThreads) cast_tile_kernel(const uint16_t 
     // word position is rotated by c/4 so that both the column-wise writes and
     // the row-wise reads touch 32 distinct banks.
     __shared__ uint32_t stage[kTile][kTile / 4];
+    constexpr int kW = InType<DT>::kWords4;  // words per four input elements
+    constexpr int kB = InType<DT>::kBytes;
 
     const int s = __ldg(d_bias) + delta;
     const Pow2Pair p = make_pow2_pair(s);
@@ -102,20 +102,28 @@ __global__ void __launch_bounds__(kCastThreads) cast_tile_kernel(const uint16_t 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     if (fast_ok && r0 + kTile <= rows && c0 + kTile <= cols) {
-        uint2 v[4][4];
+        uint32_t v[4][4][kW];
 #pragma unroll
         for (int it = 0; it < 4; ++it) {
             const int rg = warp + 8 * it;
 #pragma unroll
-            for (int i = 0; i < 4; ++i)
-                v[it][i] = __ldcs(reinterpret_cast<const uint2 *>(x + (r0 + 4 * rg + i) * ld + c0 + 4 * lane));
+            for (int i = 0; i < 4; ++i) {
+                const uint8_t *src = reinterpret_cast<const uint8_t *>(x) + ((r0 + 4 * rg + i) * ld + c0 + 4 * lane) * kB;
+                if (kW == 2) {
+                    const uint2 q = __ldcs(reinterpret_cast<const uint2 *>(src));
+                    v[it][i][0] = q.x; v[it][i][1] = q.y;
+                } else {
+                    const uint4 q = __ldcs(reinterpret_cast<const uint4 *>(src));
+                    v[it][i][0] = q.x; v[it][i][1] = q.y; v[it][i][kW - 2] = q.z; v[it][i][kW - 1] = q.w;
+                }
+            }
         }
 #pragma unroll
         for (int it = 0; it < 4; ++it) {
             const int rg = warp + 8 * it;
             uint32_t rw[4], cw[4];
 #pragma unroll
-            for (int i = 0; i < 4; ++i) rw[i] = cast4<FMT, true>(v[it][i].x, v[it][i].y, p, sat);
+            for (int i = 0; i < 4; ++i) rw[i] = cast4w<FMT, DT, true>(v[it][i], p, sat);
             if (y) {
 #pragma unroll
                 for (int i = 0; i < 4; ++i)
@@ -141,7 +149,7 @@ __global__ void __launch_bounds__(kCastThreads) cast_tile_kernel(const uint16_t 
         for (int idx = threadIdx.x; idx < kTile * kTile; idx += kCastThreads) {
             int r = idx / kTile, c = idx % kTile;
             if (r0 + r < rows && c0 + c < cols) {
-                uint8_t code = cast1<FMT, true>(x[(r0 + r) * ld + c0 + c], p, sat);
+                uint8_t code = cast1<FMT, DT, true>(x, (r0 + r) * ld + c0 + c, p, sat);
                 if (y) y[(r0 + r) * cols + c0 + c] = code;
                 if (y_t) stage_b[c * kTile + r] = code;
             }
@@ -157,11 +165,12 @@ __global__ void __launch_bounds__(kCastThreads) cast_tile_kernel(const uint16_t 
     if (__syncthreads_or(sat) && threadIdx.x == 0) atomicOr(d_status, FP8_FLAG_SATURATED);
 }
 
-template <int FMT>
+template <int FMT, int DT>
 static cudaError_t launch_cast(fp8_ctx *ctx, const void *x, int64_t rows, int64_t cols, int64_t ld,
                                const int32_t *d_bias, int delta, uint8_t *y, uint8_t *y_t, cudaStream_t stream)
 {
     auto al = [](const void *p, unsigned a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; };
+    constexpr int kB = InType<DT>::kBytes;
     if (!y_t && ld == cols && al(x, 16) && al(y, 16)) {
         int64_t n = rows * cols;
         int64_t nout = n / 16;
@@ -170,19 +179,27 @@ static cudaError_t launch_cast(fp8_ctx *ctx, const void *x, int64_t rows, int64_
         int64_t want = (nout + chunk - 1) / chunk;
         int max_blocks = ctx->sm_count * 8;
         int blocks = (int)(want < 1 ? 1 : (want > max_blocks ? max_blocks : want));
-        cast_flat_kernel<FMT><<<blocks, kCastThreads, 0, stream>>>(
-            reinterpret_cast<const uint4 *>(x), reinterpret_cast<uint4 *>(y), nout,
-            reinterpret_cast<const uint16_t *>(x) + nout * 16, y + nout * 16, ntail, d_bias, delta, ctx->d_status);
+        cast_flat_kernel<FMT, DT><<<blocks, kCastThreads, 0, stream>>>(reinterpret_cast<const uint4 *>(x),
+                                                                       reinterpret_cast<uint4 *>(y), nout, ntail,
+                                                                       d_bias, delta, ctx->d_status);
         return cudaGetLastError();
     }
-    int fast_ok = al(x, 8) && (ld % 4) == 0 && (!y || (al(y, 4) && (cols % 4) == 0)) &&
+    int fast_ok = al(x, 4 * kB) && (ld % 4) == 0 && (!y || (al(y, 4) && (cols % 4) == 0)) &&
                   (!y_t || (al(y_t, 4) && (rows % 4) == 0));
     int64_t tiles = ((rows + kTile - 1) / kTile) * ((cols + kTile - 1) / kTile);
     if (tiles > 0x7FFFFFFF) return cudaErrorInvalidValue;
-    cast_tile_kernel<FMT><<<(unsigned)tiles, kCastThreads, 0, stream>>>(reinterpret_cast<const uint16_t *>(x), rows,
-                                                                        cols, ld, d_bias, delta, y, y_t, fast_ok,
-                                                                        ctx->d_status);
+    cast_tile_kernel<FMT, DT><<<(unsigned)tiles, kCastThreads, 0, stream>>>(x, rows, cols, ld, d_bias, delta, y, y_t,
+                                                                            fast_ok, ctx->d_status);
     return cudaGetLastError();
+}
+
+template <int FMT>
+static cudaError_t launch_cast_dt(int dt, fp8_ctx *ctx, const void *x, int64_t rows, int64_t cols, int64_t ld,
+                                  const int32_t *d_bias, int delta, uint8_t *y, uint8_t *y_t, cudaStream_t stream)
+{
+    if (dt == FP8_BF16) return launch_cast<FMT, FP8_BF16>(ctx, x, rows, cols, ld, d_bias, delta, y, y_t, stream);
+    if (dt == FP8_F16) return launch_cast<FMT, FP8_F16>(ctx, x, rows, cols, ld, d_bias, delta, y, y_t, stream);
+    return launch_cast<FMT, FP8_F32>(ctx, x, rows, cols, ld, d_bias, delta, y, y_t, stream);
 }
 
 static fp8_status_t cast_entry(int fmt, fp8_ctx *ctx, const void *x, fp8_dtype_t x_dt, int64_t rows, int64_t cols,
@@ -192,26 +209,27 @@ static fp8_status_t cast_entry(int fmt, fp8_ctx *ctx, const void *x, fp8_dtype_t
     if (!ctx || !x || (!y && !y_t)) return FP8_ERR_NULL;
     if (!d_bias && (!d_amax_out || !d_bias_out)) return FP8_ERR_NULL;
     if ((int)x_dt < 0 || (int)x_dt > 2 || (int)conv < 0 || (int)conv > 1) return FP8_ERR_DTYPE;
-    if (x_dt != FP8_BF16) return FP8_ERR_UNSUPPORTED;
     if (rows <= 0 || cols <= 0 || ld < cols) return FP8_ERR_SHAPE;
-    if (reinterpret_cast<uintptr_t>(x) & 1u) return FP8_ERR_ALIGN;
+    if (reinterpret_cast<uintptr_t>(x) & (x_dt == FP8_F32 ? 3u : 1u)) return FP8_ERR_ALIGN;
     cudaStream_t st = (cudaStream_t)stream;
     const int32_t *bias = d_bias;
     if (!bias) {
-        // FP8-AMAX: one cooperative launch when the tensor is made of whole 128x128 tiles ...
-        cudaError_t fe = launch_cast_fused(ctx, fmt, x, rows, cols, ld, (int)conv, margin, d_amax_out, d_bias_out, y,
-                                           y_t, st);
-        if (fe == cudaSuccess) return FP8_OK;
-        cudaGetLastError();
+        // FP8-AMAX: (opt-in) one cooperative launch when a bf16 tensor is made of whole 128x128 tiles ...
+        if (x_dt == FP8_BF16) {
+            cudaError_t fe = launch_cast_fused(ctx, fmt, x, rows, cols, ld, (int)conv, margin, d_amax_out, d_bias_out,
+                                               y, y_t, st);
+            if (fe == cudaSuccess) return FP8_OK;
+            cudaGetLastError();
+        }
         // ... otherwise amax + bias in one launch, the cast in a second
-        if (launch_amax_bias(ctx, x, rows, cols, ld, d_amax_out, d_bias_out, fmt, (int)conv, margin, st) !=
+        if (launch_amax_bias(ctx, x, (int)x_dt, rows, cols, ld, d_amax_out, d_bias_out, fmt, (int)conv, margin, st) !=
             cudaSuccess)
             return FP8_ERR_CUDA;
         bias = d_bias_out;
     }
     int delta = format_delta(fmt, (int)conv);
-    cudaError_t e = fmt == FP8_E4 ? launch_cast<FP8_E4>(ctx, x, rows, cols, ld, bias, delta, y, y_t, st)
-                                  : launch_cast<FP8_E5>(ctx, x, rows, cols, ld, bias, delta, y, y_t, st);
+    cudaError_t e = fmt == FP8_E4 ? launch_cast_dt<FP8_E4>((int)x_dt, ctx, x, rows, cols, ld, bias, delta, y, y_t, st)
+                                  : launch_cast_dt<FP8_E5>((int)x_dt, ctx, x, rows, cols, ld, bias, delta, y, y_t, st);
     return e == cudaSuccess ? FP8_OK : FP8_ERR_CUDA;
 }
 

@@ -25,23 +25,80 @@ __device__ __forceinline__ bool clips(float v)
     return FMT == FP8_E4 ? (fabsf(v) > 464.0f) : (fabsf(v) >= 61440.0f);
 }
 
+// Input element types: bytes per element and words per group of four elements.
+template <int DT>
+struct InType {
+    static constexpr int kBytes = (DT == FP8_F32) ? 4 : 2;
+    static constexpr int kWords4 = (DT == FP8_F32) ? 4 : 2;
+};
+
+// Four consecutive input elements (kWords4 words, memory order) as floats; every conversion is exact.
+template <int DT>
+__device__ __forceinline__ void unpack4(const uint32_t *w, float (&f)[4])
+{
+    if (DT == FP8_BF16) {
+        f[0] = __uint_as_float(w[0] << 16);
+        f[1] = __uint_as_float(w[0] & 0xFFFF0000u);
+        f[2] = __uint_as_float(w[1] << 16);
+        f[3] = __uint_as_float(w[1] & 0xFFFF0000u);
+    } else if (DT == FP8_F16) {
+        asm("{ .reg .b16 lo, hi; mov.b32 {lo, hi}, %2; cvt.f32.f16 %0, lo; cvt.f32.f16 %1, hi; }"
+            : "=f"(f[0]), "=f"(f[1]) : "r"(w[0]));
+        asm("{ .reg .b16 lo, hi; mov.b32 {lo, hi}, %2; cvt.f32.f16 %0, lo; cvt.f32.f16 %1, hi; }"
+            : "=f"(f[2]), "=f"(f[3]) : "r"(w[1]));
+    } else {
+        f[0] = __uint_as_float(w[0]);
+        f[1] = __uint_as_float(w[1]);
+        f[2] = __uint_as_float(w[2]);
+        f[3] = __uint_as_float(w[3]);
+    }
+}
+
+// Scale four values by the exact power of two and round them to four FP8 bytes (memory order).
+template <int FMT, bool TWO_STEP>
+__device__ __forceinline__ uint32_t pack4(float (&f)[4], Pow2Pair p, bool &sat)
+{
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        f[i] *= p.first;
+        if (TWO_STEP) f[i] *= p.second;
+    }
+    sat = sat || clips<FMT>(f[0]) || clips<FMT>(f[1]) || clips<FMT>(f[2]) || clips<FMT>(f[3]);
+    return cvt_pair<FMT>(f[1], f[0]) | (cvt_pair<FMT>(f[3], f[2]) << 16);
+}
+
+template <int FMT, int DT, bool TWO_STEP>
+__device__ __forceinline__ uint32_t cast4w(const uint32_t *w, Pow2Pair p, bool &sat)
+{
+    float f[4];
+    unpack4<DT>(w, f);
+    return pack4<FMT, TWO_STEP>(f, p, sat);
+}
+
 // Four bf16 values (two packed words, memory order) -> four FP8 bytes (memory order).
 template <int FMT, bool TWO_STEP>
 __device__ __forceinline__ uint32_t cast4(uint32_t w0, uint32_t w1, Pow2Pair p, bool &sat)
 {
-    float f0 = __uint_as_float(w0 << 16) * p.first;
-    float f1 = __uint_as_float(w0 & 0xFFFF0000u) * p.first;
-    float f2 = __uint_as_float(w1 << 16) * p.first;
-    float f3 = __uint_as_float(w1 & 0xFFFF0000u) * p.first;
-    if (TWO_STEP) { f0 *= p.second; f1 *= p.second; f2 *= p.second; f3 *= p.second; }
-    sat = sat || clips<FMT>(f0) || clips<FMT>(f1) || clips<FMT>(f2) || clips<FMT>(f3);
-    return cvt_pair<FMT>(f1, f0) | (cvt_pair<FMT>(f3, f2) << 16);
+    const uint32_t w[2] = {w0, w1};
+    return cast4w<FMT, FP8_BF16, TWO_STEP>(w, p, sat);
 }
 
-template <int FMT, bool TWO_STEP>
-__device__ __forceinline__ uint8_t cast1(uint16_t h, Pow2Pair p, bool &sat)
+// Element i of a tensor of type DT as a float (exact).
+template <int DT>
+__device__ __forceinline__ float load1(const void *x, int64_t i)
 {
-    float f = __uint_as_float((uint32_t)h << 16) * p.first;
+    if (DT == FP8_F32) return reinterpret_cast<const float *>(x)[i];
+    const uint16_t h = reinterpret_cast<const uint16_t *>(x)[i];
+    if (DT == FP8_BF16) return __uint_as_float((uint32_t)h << 16);
+    float f;
+    asm("cvt.f32.f16 %0, %1;" : "=f"(f) : "h"(h));
+    return f;
+}
+
+template <int FMT, int DT, bool TWO_STEP>
+__device__ __forceinline__ uint8_t cast1(const void *x, int64_t i, Pow2Pair p, bool &sat)
+{
+    float f = load1<DT>(x, i) * p.first;
     if (TWO_STEP) f *= p.second;
     sat = sat || clips<FMT>(f);
     return (uint8_t)(cvt_pair<FMT>(0.0f, f) & 0xFFu);

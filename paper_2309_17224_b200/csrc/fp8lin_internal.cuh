@@ -79,7 +79,7 @@ __host__ __device__ inline int bias_from_amax_bits(uint32_t bits, int fmt, int c
     return e_max - e - (frac > frac_max ? 1 : 0) - margin;
 }
 
-cudaError_t launch_amax_bias(fp8_ctx *ctx, const void *x, int64_t rows, int64_t cols, int64_t ld, float *d_amax,
+cudaError_t launch_amax_bias(fp8_ctx *ctx, const void *x, int dt, int64_t rows, int64_t cols, int64_t ld, float *d_amax,
                              int32_t *d_bias, int fmt, int conv, int margin, cudaStream_t stream);
 
 }  // namespace fp8lin

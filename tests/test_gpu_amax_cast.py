@@ -233,6 +233,95 @@ def test_argument_errors(ctx, lib):
     with pytest.raises(lib.Fp8Error) as e:
         ctx.cast_e4(x, bias, y=y, rows=16, cols=16, ld=8)
     assert e.value.status == lib.ERR_SHAPE
-    with pytest.raises(lib.Fp8Error) as e:
-        ctx.amax(x.float(), _dev_scalar(torch.float32))
-    assert e.value.status == lib.ERR_UNSUPPORTED
+    raw = lib.raw()
+    assert raw.fp8_amax(ctx._h, x.data_ptr(), 7, 16, 16, 16, bias.data_ptr(), None) == lib.ERR_DTYPE
+
+
+# ----------------------------------------------------------------------------
+# fp16 and fp32 inputs (the paper's own tensors are FP16)
+# ----------------------------------------------------------------------------
+
+def _host(t):
+    """torch fp16 / fp32 tensor -> numpy array the oracle accepts."""
+    return t.detach().contiguous().cpu().numpy()
+
+
+@pytest.mark.parametrize("dtype", [torch.float16, torch.float32])
+@pytest.mark.parametrize("shape", [(1, 1), (1, 5), (3, 8), (256, 768), (300, 520), (129, 257), (5, 100003)])
+def test_amax_fp16_fp32(ctx, dtype, shape):
+    g = torch.Generator(device="cuda").manual_seed(shape[0] * 131 + shape[1])
+    x = (torch.randn(shape, generator=g, device="cuda") * 3.0).to(dtype)
+    assert _gpu_amax(ctx, x) == O.amax(_host(x))
+    x[-1, -1] = -4096.0
+    assert _gpu_amax(ctx, x) == 4096.0
+    if shape[1] >= 8:
+        big = torch.zeros((shape[0], shape[1] + 24), dtype=dtype, device="cuda")
+        big[:, 5:5 + shape[1]] = x
+        big[:, :5] = 30000.0
+        view = big[:, 5:5 + shape[1]]
+        assert _gpu_amax(ctx, view, rows=shape[0], cols=shape[1], ld=shape[1] + 24) == O.amax(_host(view))
+    x[0, 0] = float("inf")
+    assert _gpu_amax(ctx, x) == float("inf")
+    x[0, 0] = float("nan")
+    assert np.isnan(_gpu_amax(ctx, x))
+
+
+@pytest.mark.parametrize("kind", [O.E4, O.E5])
+def test_cast_every_fp16_value(ctx, lib, kind):
+    """All 65 536 fp16 bit patterns at every shift that can bring one of them into the FP8 range."""
+    h = np.arange(65536, dtype=np.uint32).astype(np.uint16).view(np.float16).reshape(256, 256)
+    x = torch.from_numpy(h.copy()).cuda()
+    fmt = O.native_format(kind)
+    cast = ctx.cast_e4 if kind == O.E4 else ctx.cast_e5
+    bias = _dev_scalar(torch.int32)
+    y = torch.empty((256, 256), dtype=torch.uint8, device="cuda")
+    y_t = torch.empty((256, 256), dtype=torch.uint8, device="cuda")
+    for b in list(range(-36, 44)) + [-150, -127, 126, 140]:
+        bias.fill_(b)
+        want = O.cast(h, b + O.delta(kind, O.CONV_PAPER), fmt)
+        if b % 2:
+            cast(x, bias, y=y)
+        else:
+            cast(x, bias, y=y, y_t=y_t)
+            assert_codes_equal(u8(y_t), want.T, fmt)
+        assert_codes_equal(u8(y), want, fmt)
+
+
+@pytest.mark.parametrize("kind", [O.E4, O.E5])
+def test_cast_fp32_values_and_extremes(ctx, lib, kind):
+    rng = np.random.default_rng(kind + 10)
+    bits = rng.integers(0, 2 ** 32, size=(384, 512), dtype=np.uint64).astype(np.uint32)   # every exponent, both signs, NaNs too
+    bits[0, :8] = [0x00000001, 0x807FFFFF, 0x00800000, 0x7F7FFFFF, 0x7F800000, 0xFF800000, 0x7FC00000, 0x80000000]
+    f = bits.view(np.float32)
+    x = torch.from_numpy(f.copy()).cuda()
+    fmt = O.native_format(kind)
+    cast = ctx.cast_e4 if kind == O.E4 else ctx.cast_e5
+    bias = _dev_scalar(torch.int32)
+    y = torch.empty(f.shape, dtype=torch.uint8, device="cuda")
+    y_t = torch.empty(f.shape[::-1], dtype=torch.uint8, device="cuda")
+    for b in (-150, -130, -126, -60, -7, 0, 3, 40, 100, 127, 140, 152):
+        bias.fill_(b)
+        want = O.cast(f, b + O.delta(kind, O.CONV_PAPER), fmt)
+        cast(x, bias, y=y, y_t=y_t)
+        assert_codes_equal(u8(y), want, fmt)
+        assert_codes_equal(u8(y_t), want.T, fmt)
+        cast(x, bias, y=y)
+        assert_codes_equal(u8(y), want, fmt)
+
+
+@pytest.mark.parametrize("dtype", [torch.float16, torch.float32])
+@pytest.mark.parametrize("kind", [O.E4, O.E5])
+def test_fused_amax_bias_cast_fp16_fp32(ctx, lib, dtype, kind):
+    g = torch.Generator(device="cuda").manual_seed(77 + kind)
+    for shape, std in (((384, 640), 0.02), ((129, 257), 3.0), ((64, 4096), 1e-3)):
+        x = (torch.randn(shape, generator=g, device="cuda") * std).to(dtype)
+        a, b, want, want_t = O.quantise(_host(x), kind, O.CONV_PAPER, 0, transposed=True)
+        amax = _dev_scalar(torch.float32, -1.0)
+        bias = _dev_scalar(torch.int32, 777)
+        y = torch.empty(shape, dtype=torch.uint8, device="cuda")
+        y_t = torch.empty(shape[::-1], dtype=torch.uint8, device="cuda")
+        cast = ctx.cast_e4 if kind == O.E4 else ctx.cast_e5
+        cast(x, None, d_amax_out=amax, d_bias_out=bias, y=y, y_t=y_t)
+        assert float(amax.item()) == a and int(bias.item()) == b
+        assert_codes_equal(u8(y), want, O.native_format(kind))
+        assert_codes_equal(u8(y_t), want_t, O.native_format(kind))

@@ -106,3 +106,30 @@ def test_largest_cast_code_lands_in_the_top_binade():
             top = np.abs(O.decode_table(O.native_format(kind))[y]).max() * 2.0 ** -O.delta(kind, conv)
             mx = O.bias_max_num(kind, conv)
             assert mx / 2 <= top <= mx or (conv == O.CONV_PAPER and kind == O.E4 and top == 224.0)
+
+
+def test_fp16_and_fp32_inputs_are_read_exactly():
+    """Every fp16 bit pattern decodes as numpy decodes it; amax and cast on
+    fp16 / fp32 tensors equal the same operations on the exactly converted
+    bf16-free reference path (numpy float64 arithmetic + the pinned encoder)."""
+    h = np.arange(65536, dtype=np.uint32).astype(np.uint16).view(np.float16).reshape(256, 256)
+    finite = np.isfinite(h)
+    assert O.amax(np.where(finite, h, np.float16(0))) == float(np.abs(h[finite].astype(np.float64)).max()) == 65504.0
+    assert np.isnan(O.amax(h))
+    table = O.decode_table(O.N_E4)
+    for shift in (-3, 0, 6):
+        codes = O.cast(h, shift, O.N_E4)
+        v = np.ldexp(h.astype(np.float64), shift)
+        ok = finite & (np.abs(v) <= 448.0)
+        # the chosen value is a nearest grid value
+        grid = table[:0x7F]
+        best = np.abs(grid[None, :] - np.abs(v[ok])[:, None]).min(axis=1)
+        assert np.array_equal(np.abs(table[codes[ok] & 0x7F] - np.abs(v[ok])), best)
+    rng = np.random.default_rng(3)
+    f = (rng.standard_normal((64, 48)) * 5).astype(np.float32)
+    f[0, 0] = -123.456
+    assert O.amax(f) == np.float32(123.456)
+    got = O.cast(f, 1, O.N_E4)
+    ref = torch.from_numpy(f * 2.0).to(torch.float8_e4m3fn).view(torch.uint8).numpy()
+    ok = np.abs(f * 2.0) <= 448.0
+    assert np.array_equal(got[ok], ref[ok])

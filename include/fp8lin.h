@@ -173,6 +173,24 @@ FP8_API fp8_status_t fp8_linear_fwd(fp8_ctx *ctx, const uint8_t *x8, const int32
                             fp8_dtype_t y_dt, float *d_amax_y, int64_t T, int64_t K, int64_t N, fp8_conv_t conv,
                             void *stream);
 
+/* Forward matmul with the activation fused into the epilogue (the paper has no
+ * counterpart; it answers Section 3's warning that computing a scale just in
+ * time costs a second pass over memory: the next layer's input leaves this
+ * kernel together with its amax, so that layer needs no amax pass).
+ *   y_pre  NULL, or out [T, N] bf16: the rounded pre-activation
+ *          (unscale, + bias_vec), what the backward pass of the activation needs
+ *   y_act  out [T, N] bf16: act(y_pre), evaluated in FP32 on the bf16-rounded
+ *          pre-activation, so it is exactly what a separate activation of y_pre gives
+ *   act    FP8_ACT_GELU: x/2 * (1 + erf(x / sqrt 2))
+ *   d_amax_act  NULL or out: amax of y_act; fp8_scaling_bias + fp8_cast_e4 with
+ *          that bias then quantise y_act in a single pass
+ * Needs 16-byte aligned y_pre / y_act and N % 8 == 0, besides fp8_linear_fwd's rules. */
+typedef enum { FP8_ACT_GELU = 1 } fp8_act_t;
+FP8_API fp8_status_t fp8_linear_fwd_act(fp8_ctx *ctx, const uint8_t *x8, const int32_t *d_bx, const uint8_t *w8,
+                                        const int32_t *d_bw, const void *bias_vec, fp8_dtype_t bias_dt, void *y_pre,
+                                        void *y_act, fp8_act_t act, float *d_amax_act, int64_t T, int64_t K, int64_t N,
+                                        fp8_conv_t conv, void *stream);
+
 /* Input-gradient matmul (Section 2.2): dX[t, k] = (sum_n dY8[t, n] * W8[n, k]) * 2^-(s_g + s_w).
  *   dy8  [T, N] E5 bytes;  N % 16 == 0
  *   w8   [N, K] E4 bytes or NULL;  w8_t [K, N] E4 bytes or NULL.  At least one.

@@ -11,7 +11,7 @@ from __future__ import annotations
 import math
 
 import numpy as np
-from scipy.special import erf
+from scipy.special import erf, erfc
 
 import oracle as O
 
@@ -32,8 +32,10 @@ def step_input_bits(x_base_bits: np.ndarray, step: int) -> np.ndarray:
 
 
 def gelu_bits(y_bits: np.ndarray) -> np.ndarray:
+    """GELU(z) = z/2 * (1 + erf(z / sqrt 2)), written with erfc so that the far negative tail keeps its
+    relative accuracy (1 + erf cancels there)."""
     z = bf16_to_f64(y_bits)
-    return f64_to_bf16(0.5 * z * (1.0 + erf(z / math.sqrt(2.0))))
+    return f64_to_bf16(0.5 * z * erfc(-z / math.sqrt(2.0)))
 
 
 def gelu_grad(y_bits: np.ndarray) -> np.ndarray:

@@ -53,6 +53,7 @@ struct GemmParams {
     int64_t ldo;
     int vec_ok;                   // out 16-byte aligned and ldo*elem % 16 == 0
     int tma_out;                  // epilogue goes through shared memory and TMA stores (needs vec_ok)
+    int act;                      // 0: none; 1: GELU of the bf16-rounded output goes to a second tensor (out may be NULL)
     unsigned *d_amax_bits;        // or NULL
     unsigned *d_status;
     uint32_t idesc;
@@ -287,12 +288,26 @@ __device__ __forceinline__ void slab_publish(const CUtensorMap *map, uint32_t sl
     if (lane == 0 && in_range) tma_store_2d(map, slab, x, y);
 }
 
+// GELU(x) = x/2 * erfc(-x / sqrt 2); erfc keeps relative accuracy in the negative tail.
+__device__ __forceinline__ float gelu_f32(float x) { return 0.5f * x * erfcf(-0.70710678118654752f * x); }
+
+// 32 bf16 values (16 packed words): apply GELU to each, in FP32.
+__device__ __forceinline__ void gelu_words(const uint32_t (&w)[16], float (&v)[32])
+{
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+        v[2 * i] = gelu_f32(__uint_as_float(w[i] << 16));
+        v[2 * i + 1] = gelu_f32(__uint_as_float(w[i] & 0xFFFF0000u));
+    }
+}
+
 // One warp's share (32 rows x BN columns) of a finished accumulator.
 //   t_row        TMEM address of this warp's lanes at the accumulator's first column
 //   row0         first of the warp's 32 output rows;  col_base  first output column of the tile
 //   release_bar  barrier to arrive on once the accumulator has been read (cluster address if remote)
-template <int BN>
-__device__ __forceinline__ void epilogue_tile(const CUtensorMap *map_out, uint32_t t_row, int row0, int col_base,
+template <int BN, bool ACT>
+__device__ __forceinline__ void epilogue_tile(const CUtensorMap *map_out, const CUtensorMap *map_out2, uint32_t t_row,
+                                              int row0, int col_base,
                                               const GemmParams &p, const Pow2Pair sc, bool two_step,
                                               uint32_t &amax_bits, uint32_t warp_slabs, uint32_t &slab_count,
                                               uint32_t release_bar, bool release_remote, int lane)
@@ -320,6 +335,46 @@ __device__ __forceinline__ void epilogue_tile(const CUtensorMap *map_out, uint32
     }
     const bool rows_in = row0 < p.M;
     const bool row_ok = row0 + lane < p.M;
+    if (ACT) {
+        // pre-activation (optional) and activated output leave together: both slabs of the warp are in use
+        uint32_t dummy = 0;
+#pragma unroll 1
+        for (int c = 0; c < BN; c += 64) {
+            uint32_t r0[32], r1[32];
+            tmem_ld_x32(t_row + c, r0);
+            tmem_ld_x32(t_row + c + 32, r1);
+            tmem_ld_wait();
+            if (c + 64 >= BN) release();
+            if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+            __syncwarp();
+            const uint32_t slab_pre = warp_slabs, slab_act = warp_slabs + kSlabBytes;
+            float v[32];
+            uint32_t w[16], wa[16];
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int col0 = col_base + c + 32 * h;
+                epilogue_values(h == 0 ? r0 : r1, col0, p, sc, two_step, v);
+                pack_bf16(v, col0, p, w, dummy, false);
+                if (p.out) {
+#pragma unroll
+                    for (int j = 0; j < 4; ++j)
+                        slab_write(slab_pre, lane, 4 * h + j, w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
+                }
+                gelu_words(w, v);  // the activation sees exactly what the pre-activation tensor holds
+                pack_bf16(v, col0, p, wa, amax_bits, row_ok);
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+                    slab_write(slab_act, lane, 4 * h + j, wa[4 * j], wa[4 * j + 1], wa[4 * j + 2], wa[4 * j + 3]);
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            __syncwarp();
+            if (lane == 0 && rows_in && col_base + c < p.N) {
+                if (p.out) tma_store_2d(map_out, slab_pre, col_base + c, row0);
+                tma_store_2d(map_out2, slab_act, col_base + c, row0);
+            }
+        }
+        return;
+    }
     if (p.out_dt == FP8_BF16) {
 #pragma unroll 1
         for (int c = 0; c < BN; c += 64) {  // one slab = 64 bf16 columns
@@ -365,10 +420,11 @@ __device__ __forceinline__ void epilogue_tile(const CUtensorMap *map_out, uint32
     }
 }
 
-template <int BN, int STAGES>
+template <int BN, int STAGES, bool ACT>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-            const __grid_constant__ CUtensorMap map_out, const GemmParams p)
+            const __grid_constant__ CUtensorMap map_out, const __grid_constant__ CUtensorMap map_out2,
+            const GemmParams p)
 {
     using L = GemmSmem<BN, STAGES>;
     extern __shared__ uint8_t smem_raw[];
@@ -488,7 +544,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             if (!__all_sync(0xFFFFFFFFu, ready)) break;
             tc_fence_after();
             const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + buf * BN;
-            epilogue_tile<BN>(&map_out, t_row, m_blk * kBM + q * 32, n_blk * BN, pp, p.splits > 1 ? sc_one : sc,
+            epilogue_tile<BN, ACT>(&map_out, &map_out2, t_row, m_blk * kBM + q * 32, n_blk * BN, pp, p.splits > 1 ? sc_one : sc,
                               p.splits > 1 ? false : two_step, amax_bits, warp_slabs, slab_count, acc_empty_bar(buf),
                               false, lane);
         }
@@ -609,9 +665,11 @@ __host__ __device__ inline uint32_t make_idesc_pair(int a_fmt, int b_fmt)
 }
 
 // tiles here are 256 x 256; p.tiles_m / p.tiles_n count those
+template <bool ACT>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1)
 gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-                 const __grid_constant__ CUtensorMap map_out, const GemmParams p)
+                 const __grid_constant__ CUtensorMap map_out, const __grid_constant__ CUtensorMap map_out2,
+                 const GemmParams p)
 {
     using L = PairSmem;
     extern __shared__ uint8_t smem_raw[];
@@ -722,7 +780,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             if (!__all_sync(0xFFFFFFFFu, ready)) break;
             tc_fence_after();
             const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + buf * kPairBN;
-            epilogue_tile<kPairBN>(&map_out, t_row, m_blk * 256 + (int)rank * kBM + q * 32, n_blk * kPairBN, p, sc,
+            epilogue_tile<kPairBN, ACT>(&map_out, &map_out2, t_row, m_blk * 256 + (int)rank * kBM + q * 32, n_blk * kPairBN, p, sc,
                                    two_step, amax_bits, warp_slabs, slab_count, leader_acc_empty0 + 8u * buf, true, lane);
         }
         if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
@@ -794,10 +852,14 @@ cudaError_t configure_gemm_kernels(int max_smem_optin)
 {
     using L = GemmSmem<kBN, kStages>;
     if (L::kDynamic > max_smem_optin || PairSmem::kDynamic > max_smem_optin) return cudaErrorInvalidValue;
-    cudaError_t e =
-        cudaFuncSetAttribute(gemm_kernel<kBN, kStages>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kDynamic);
-    if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(gemm_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, PairSmem::kDynamic);
+    cudaError_t e = cudaFuncSetAttribute(gemm_kernel<kBN, kStages, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         L::kDynamic);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(gemm_kernel<kBN, kStages, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kDynamic);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(gemm_pair_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, PairSmem::kDynamic);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(gemm_pair_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, PairSmem::kDynamic);
     if (e != cudaSuccess) return e;
     int sms = 0, dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess ||
@@ -815,7 +877,7 @@ cudaError_t configure_gemm_kernels(int max_smem_optin)
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
     int clusters = 0;
-    if (cudaOccupancyMaxActiveClusters(&clusters, gemm_pair_kernel, &cfg) != cudaSuccess) {
+    if (cudaOccupancyMaxActiveClusters(&clusters, gemm_pair_kernel<false>, &cfg) != cudaSuccess) {
         cudaGetLastError();
         clusters = 0;
     }
@@ -852,7 +914,7 @@ static bool encode_map(fp8_ctx *ctx, CUtensorMap *map, const void *base, int64_t
 static fp8_status_t run_gemm(fp8_ctx *ctx, const uint8_t *a, int a_fmt, bool a_mn, const int32_t *d_ba,
                              const uint8_t *b, int b_fmt, bool b_mn, const int32_t *d_bb, int delta_sum,
                              const void *bias_vec, int bias_dt, void *out, int out_dt, float *d_amax_out, int64_t M,
-                             int64_t N, int64_t Kc, cudaStream_t st)
+                             int64_t N, int64_t Kc, cudaStream_t st, int act = 0, void *out_act = nullptr)
 {
     if (M > 0x7FFFFFFF / 2 || N > 0x7FFFFFFF / 2 || Kc > 0x7FFFFFFF / 2) return FP8_ERR_SHAPE;
     const bool pair = g_max_pairs > 0 && M > kBM && !g_force_single;
@@ -876,7 +938,7 @@ static fp8_status_t run_gemm(fp8_ctx *ctx, const uint8_t *a, int a_fmt, bool a_m
     p.splits = 1;
     p.kb_per_split = p.num_k;
     p.partial = ctx->d_partial;
-    if (!pair && !g_no_splitk) {
+    if (!pair && !g_no_splitk && !act) {
         const int64_t tiles = (int64_t)p.tiles_m * p.tiles_n;
         if (tiles < 2 * ctx->sm_count && p.num_k >= 8) {
             int64_t want = (2 * ctx->sm_count + tiles - 1) / tiles;
@@ -896,17 +958,26 @@ static fp8_status_t run_gemm(fp8_ctx *ctx, const uint8_t *a, int a_fmt, bool a_m
     const int64_t esz = out_dt == FP8_BF16 ? 2 : 4;
     p.vec_ok = ((reinterpret_cast<uintptr_t>(out) & 15u) == 0 && (N * esz) % 16 == 0) ? 1 : 0;
     p.tma_out = (p.vec_ok && !g_direct_epilogue) ? 1 : 0;
+    p.act = act;
     CUtensorMap map_out = map_a;  // placeholder when the staged epilogue is off (never dereferenced then)
-    if (p.tma_out) {
+    CUtensorMap map_out2 = map_a;
+    auto encode_out = [&](CUtensorMap *m, void *base) {
         cuuint64_t dims[2] = {(cuuint64_t)N, (cuuint64_t)M};
         cuuint64_t strides[1] = {(cuuint64_t)(N * esz)};
         cuuint32_t box[2] = {(cuuint32_t)(128 / esz), 32};
         cuuint32_t estr[2] = {1, 1};
-        CUresult r = ctx->encode_tiled(&map_out, esz == 2 ? CU_TENSOR_MAP_DATA_TYPE_UINT16 : CU_TENSOR_MAP_DATA_TYPE_UINT32,
-                                       2, out, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                                       CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
-                                       CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-        if (r != CUDA_SUCCESS) return FP8_ERR_CUDA;
+        return ctx->encode_tiled(m, esz == 2 ? CU_TENSOR_MAP_DATA_TYPE_UINT16 : CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, base,
+                                 dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                 CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    };
+    if (act) {
+        // the activated output always goes through the staged epilogue (callers have checked its alignment)
+        p.tma_out = 1;
+        p.vec_ok = 1;
+        if (!encode_out(&map_out2, out_act)) return FP8_ERR_CUDA;
+        if (out && !encode_out(&map_out, out)) return FP8_ERR_CUDA;
+    } else if (p.tma_out) {
+        if (!encode_out(&map_out, out)) return FP8_ERR_CUDA;
     }
     p.d_amax_bits = reinterpret_cast<unsigned *>(d_amax_out);
     p.d_status = ctx->d_status;
@@ -916,11 +987,17 @@ static fp8_status_t run_gemm(fp8_ctx *ctx, const uint8_t *a, int a_fmt, bool a_m
     int tiles = p.tiles_m * p.tiles_n;
     if (pair) {
         int pairs = tiles < g_max_pairs ? tiles : g_max_pairs;
-        gemm_pair_kernel<<<2 * pairs, kGemmThreads, PairSmem::kDynamic, st>>>(map_a, map_b, map_out, p);
+        if (act) gemm_pair_kernel<true><<<2 * pairs, kGemmThreads, PairSmem::kDynamic, st>>>(map_a, map_b, map_out, map_out2, p);
+        else gemm_pair_kernel<false><<<2 * pairs, kGemmThreads, PairSmem::kDynamic, st>>>(map_a, map_b, map_out, map_out2, p);
     } else {
         int items = tiles * p.splits;
         int grid = items < ctx->sm_count ? items : ctx->sm_count;
-        gemm_kernel<kBN, kStages><<<grid, kGemmThreads, GemmSmem<kBN, kStages>::kDynamic, st>>>(map_a, map_b, map_out, p);
+        if (act)
+            gemm_kernel<kBN, kStages, true><<<grid, kGemmThreads, GemmSmem<kBN, kStages>::kDynamic, st>>>(
+                map_a, map_b, map_out, map_out2, p);
+        else
+            gemm_kernel<kBN, kStages, false><<<grid, kGemmThreads, GemmSmem<kBN, kStages>::kDynamic, st>>>(
+                map_a, map_b, map_out, map_out2, p);
         if (p.splits > 1) {
             if (cudaGetLastError() != cudaSuccess) return FP8_ERR_CUDA;
             int64_t total = M * N;
@@ -954,6 +1031,25 @@ fp8_status_t fp8_linear_fwd(fp8_ctx *ctx, const uint8_t *x8, const int32_t *d_bx
     int delta = 2 * format_delta(FP8_E4, conv);
     return run_gemm(ctx, x8, FP8_E4, false, d_bx, w8, FP8_E4, false, d_bw, delta, bias_vec, bias_dt, y, y_dt, d_amax_y,
                     T, N, K, (cudaStream_t)stream);
+}
+
+fp8_status_t fp8_linear_fwd_act(fp8_ctx *ctx, const uint8_t *x8, const int32_t *d_bx, const uint8_t *w8,
+                                const int32_t *d_bw, const void *bias_vec, fp8_dtype_t bias_dt, void *y_pre, void *y_act,
+                                fp8_act_t act, float *d_amax_act, int64_t T, int64_t K, int64_t N, fp8_conv_t conv,
+                                void *stream)
+{
+    using namespace fp8lin;
+    if (!ctx || !x8 || !d_bx || !w8 || !d_bw || !y_act) return FP8_ERR_NULL;
+    if ((int)conv < 0 || (int)conv > 1 || (int)bias_dt < 0 || (int)bias_dt > 2 || (int)act != (int)FP8_ACT_GELU)
+        return FP8_ERR_DTYPE;
+    if (bias_vec && !out_dtype_ok(bias_dt)) return FP8_ERR_UNSUPPORTED;
+    if (T <= 0 || K <= 0 || N <= 0) return FP8_ERR_SHAPE;
+    if (!aligned16(x8) || !aligned16(w8) || (K % 16) != 0 || !aligned16(y_act) || (y_pre && !aligned16(y_pre)) ||
+        (N % 8) != 0)
+        return FP8_ERR_ALIGN;
+    int delta = 2 * format_delta(FP8_E4, conv);
+    return run_gemm(ctx, x8, FP8_E4, false, d_bx, w8, FP8_E4, false, d_bw, delta, bias_vec, bias_dt, y_pre, FP8_BF16,
+                    d_amax_act, T, N, K, (cudaStream_t)stream, 1, y_act);
 }
 
 fp8_status_t fp8_linear_dgrad(fp8_ctx *ctx, const uint8_t *dy8, const int32_t *d_bg, const uint8_t *w8,

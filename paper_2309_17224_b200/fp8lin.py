@@ -22,12 +22,13 @@ ERR_NULL, ERR_SHAPE, ERR_ALIGN, ERR_DTYPE, ERR_UNSUPPORTED, ERR_CUDA, ERR_DEVICE
 E4, E5 = 0, 1
 CONV_PAPER, CONV_NATIVE = 0, 1
 BF16, F16, F32 = 0, 1, 2
+ACT_GELU = 1
 FLAG_NONFINITE_AMAX, FLAG_ZERO_AMAX, FLAG_SATURATED, FLAG_TIMEOUT = 1, 2, 4, 8
 
 SYMBOLS = (
     "fp8_create", "fp8_destroy", "fp8_status_string", "fp8_device_flags", "fp8_amax", "fp8_scaling_bias",
     "fp8_scaling_bias_host", "fp8_cast_e4", "fp8_cast_e5", "fp8_ptq_weights", "fp8_linear_fwd", "fp8_linear_dgrad",
-    "fp8_linear_wgrad", "fp8_amax_noalloc",
+    "fp8_linear_wgrad", "fp8_amax_noalloc", "fp8_linear_fwd_act",
 )
 
 if not os.path.exists(LIB_PATH):
@@ -52,6 +53,7 @@ _lib.fp8_cast_e4.argtypes = _cast_args
 _lib.fp8_cast_e5.argtypes = _cast_args
 _lib.fp8_ptq_weights.argtypes = [_P, _P, c_int, c_int64, c_int64, c_int64, c_int, _P, _P, _P, _P, _P]
 _lib.fp8_linear_fwd.argtypes = [_P, _P, _P, _P, _P, _P, c_int, _P, c_int, _P, c_int64, c_int64, c_int64, c_int, _P]
+_lib.fp8_linear_fwd_act.argtypes = [_P, _P, _P, _P, _P, _P, c_int, _P, _P, c_int, _P, c_int64, c_int64, c_int64, c_int, _P]
 _lib.fp8_linear_dgrad.argtypes = [_P, _P, _P, _P, _P, _P, _P, c_int, _P, c_int64, c_int64, c_int64, c_int, _P]
 _lib.fp8_linear_wgrad.argtypes = [_P, _P, _P, _P, _P, _P, _P, _P, c_int, c_int64, c_int64, c_int64, c_int, _P]
 for _name in SYMBOLS:
@@ -175,6 +177,15 @@ class Context:
         _check(_lib.fp8_linear_fwd(self._h, _ptr(x8), _ptr(d_bx), _ptr(w8), _ptr(d_bw), _ptr(bias_vec), bias_dt,
                                    _ptr(y), _DT[y.dtype], _ptr(d_amax_y), T, K, N, conv, _stream()),
                "fp8_linear_fwd")
+
+    def linear_fwd_act(self, x8, d_bx, w8, d_bw, y_pre, y_act, bias_vec=None, d_amax_act=None, act=ACT_GELU,
+                       conv=CONV_PAPER):
+        T, K = x8.shape
+        N = w8.shape[0]
+        bias_dt = _DT[bias_vec.dtype] if bias_vec is not None else BF16
+        _check(_lib.fp8_linear_fwd_act(self._h, _ptr(x8), _ptr(d_bx), _ptr(w8), _ptr(d_bw), _ptr(bias_vec), bias_dt,
+                                       _ptr(y_pre), _ptr(y_act), act, _ptr(d_amax_act), T, K, N, conv, _stream()),
+               "fp8_linear_fwd_act")
 
     def linear_dgrad(self, dy8, d_bg, w8, w8_t, d_bw, dx, d_amax_dx=None, conv=CONV_PAPER):
         T, N = dy8.shape

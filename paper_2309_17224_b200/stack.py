@@ -20,6 +20,7 @@ import torch
 from . import inputs as I
 
 CONFIG_ID = 5
+fp8lin_E4, CONV_PAPER = 0, 0   # enum values of the C ABI (format E4, paper convention)
 
 
 def step_input(x_base: torch.Tensor, step: int) -> torch.Tensor:
@@ -42,8 +43,11 @@ def gelu_grad_f32(y: torch.Tensor) -> torch.Tensor:
 
 class Fp8Stack:
     def __init__(self, ctx, layers: int = 24, d: int = 1024, tokens: int = 4096, lr: float = 1e-3,
-                 seed: int = I.BASE_SEED, device="cuda", w_std: float = 0.02):
+                 seed: int = I.BASE_SEED, device="cuda", w_std: float = 0.02, fused_activation: bool = False):
+        """fused_activation: GELU runs in the forward matmul's epilogue, which also emits the amax of the
+        activated tensor, so the next layer's input is quantised in one pass (no amax pass, no GELU kernel)."""
         self.ctx, self.L, self.d, self.T, self.lr = ctx, layers, d, tokens, lr
+        self.fused = fused_activation
         dev = dict(device=device)
         self.w32 = [I.normal_bf16(d, d, w_std, seed, I.tensor_id(CONFIG_ID, l, I.W_ID), device).to(torch.float32)
                     for l in range(layers)]
@@ -55,6 +59,7 @@ class Fp8Stack:
         self.w8 = [torch.empty((d, d), **u8) for _ in range(layers)]
         self.w8t = [torch.empty((d, d), **u8) for _ in range(layers)]
         self.y = [torch.empty((tokens, d), dtype=torch.bfloat16, **dev) for _ in range(layers)]
+        self.act = torch.empty((tokens, d), dtype=torch.bfloat16, **dev) if fused_activation else None
         self.g8 = torch.empty((tokens, d), **u8)
         self.g8t = torch.empty((d, tokens), **u8)
         self.dx = torch.empty((tokens, d), dtype=torch.bfloat16, **dev)
@@ -68,13 +73,24 @@ class Fp8Stack:
 
     def forward(self, x: torch.Tensor) -> torch.Tensor:
         c = self.ctx
+        have_amax = False   # the previous matmul's epilogue already produced amax(x)
         for l in range(self.L):
             w16 = self.w32[l].to(torch.bfloat16)
             c.cast_e4(w16, None, d_amax_out=self.amax[l, 0:1], d_bias_out=self.bias[l, 0:1], y=self.w8[l], y_t=self.w8t[l])
-            c.cast_e4(x, None, d_amax_out=self.amax[l, 1:2], d_bias_out=self.bias[l, 1:2], y=self.x8[l], y_t=self.x8t[l])
-            c.linear_fwd(self.x8[l], self.bias[l, 1:2], self.w8[l], self.bias[l, 0:1], self.y[l])
-            if l + 1 < self.L:
-                x = gelu_bf16(self.y[l])
+            if have_amax:
+                c.scaling_bias(self.amax[l, 1:2], fp8lin_E4, CONV_PAPER, 0, self.bias[l, 1:2])
+                c.cast_e4(x, self.bias[l, 1:2], y=self.x8[l], y_t=self.x8t[l])
+            else:
+                c.cast_e4(x, None, d_amax_out=self.amax[l, 1:2], d_bias_out=self.bias[l, 1:2], y=self.x8[l], y_t=self.x8t[l])
+            if self.fused and l + 1 < self.L:
+                c.linear_fwd_act(self.x8[l], self.bias[l, 1:2], self.w8[l], self.bias[l, 0:1], self.y[l], self.act,
+                                 d_amax_act=self.amax[l + 1, 1:2])
+                x, have_amax = self.act, True
+            else:
+                c.linear_fwd(self.x8[l], self.bias[l, 1:2], self.w8[l], self.bias[l, 0:1], self.y[l])
+                have_amax = False
+                if l + 1 < self.L:
+                    x = gelu_bf16(self.y[l])
         return self.y[self.L - 1]
 
     def backward_and_update(self) -> None:

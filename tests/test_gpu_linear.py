@@ -116,6 +116,33 @@ def test_fwd_bias_vector_and_output_amax(ctx, lib):
             assert float(amax_y.item()) == float(y.float().abs().max().item())
 
 
+@pytest.mark.parametrize("T,K,N", [(256, 768, 768), (144, 272, 528), (64, 1024, 512), (400, 1040, 784)])
+def test_fwd_with_gelu_in_the_epilogue(ctx, lib, T, K, N):
+    """The pre-activation must meet the forward bar; the activated tensor must be GELU of exactly that
+    pre-activation (checked with the float64 GELU on the GPU's own pre-activation bits: a relation between two
+    outputs of the call, not an expected value), and the emitted amax must be the amax of what was written."""
+    from oracle import stack as OS
+    from helpers import bf16_ordinal
+    qx, qw, _ = _layer(ctx, T, K, N, O.CONV_PAPER, seed=4242 + T)
+    bv = (torch.randn(N, device="cuda") * 0.3).to(torch.bfloat16)
+    ref = O.linear_fwd_np(qx.ref, qx.shift, qw.ref, qw.shift, bias_vec=bv.double().cpu().numpy())
+    for want_pre in (True, False):
+        y_pre = torch.full((T, N), float("nan"), dtype=torch.bfloat16, device="cuda") if want_pre else None
+        y_act = torch.full((T, N), float("nan"), dtype=torch.bfloat16, device="cuda")
+        amax_act = torch.full((1,), -1.0, dtype=torch.float32, device="cuda")
+        ctx.linear_fwd_act(qx.y, qx.bias, qw.y, qw.bias, y_pre, y_act, bias_vec=bv, d_amax_act=amax_act)
+        assert ctx.device_flags(clear=True) & lib.FLAG_TIMEOUT == 0
+        if want_pre:
+            assert_bf16_within_one_ulp(bits_of(y_pre), ref)
+            gelu_of_pre = OS.gelu_bits(bits_of(y_pre))
+            d = np.abs(bf16_ordinal(bits_of(y_act)) - bf16_ordinal(gelu_of_pre))
+            assert d.max() <= 1, d.max()
+            kept = bits_of(y_act)
+        else:
+            assert np.array_equal(bits_of(y_act), kept)   # same activated tensor with or without the first output
+        assert float(amax_act.item()) == float(y_act.float().abs().max().item())
+
+
 def test_dgrad_amax_and_margin(ctx, lib):
     T, K, N = 256, 384, 512
     qx, qw, qg = _layer(ctx, T, K, N, O.CONV_PAPER, seed=5, margin=3)

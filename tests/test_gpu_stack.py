@@ -57,6 +57,19 @@ def run():
     ctx.close()
 
 
+def test_fused_activation_variant_tracks_the_plain_run(run):
+    """GELU in the matmul epilogue + amax from the epilogue (one quantisation pass per activation): the first
+    step's loss and biases must agree with the unfused run's (same arithmetic, different kernels)."""
+    from paper_2309_17224_b200 import stack
+    st = stack.Fp8Stack(run["ctx"], layers=LAYERS, d=D, tokens=TOKENS, fused_activation=True)
+    for step in (0, 1):
+        r = st.step(step)
+        assert abs(float(r["loss"].item()) - run["loss"][step]) <= 1e-3 * run["loss"][step]
+        same = (r["bias"].cpu().numpy() == run["bias"][step])
+        assert same.mean() >= 0.97
+    assert run["ctx"].device_flags(clear=True) & run["lib"].FLAG_TIMEOUT == 0
+
+
 def test_no_timeouts_and_finite_losses(run):
     assert run["flags"] & run["lib"].FLAG_TIMEOUT == 0
     assert np.all(np.isfinite(run["loss"]))

@@ -37,6 +37,9 @@ UNIT = "TFLOP/s"
 DEFAULT_WORKLOAD = "c3_llama7b"
 ORACLE_SAMPLE_TOKENS = 256
 ORACLE_SAMPLE_LAYER = 1  # the square attention-output projection
+# dram__bytes_read.sum + dram__bytes_write.sum per matmul launch, from one ncu capture of one step of the
+# workload (profiles/gemm_pair_kernel.md, table (c)); keyed by (workload, tokens)
+GEMM_DRAM_BYTES_PER_LAUNCH = {("c3_llama7b", 8192): 387.4e6}
 
 
 def load_peaks():
@@ -143,6 +146,14 @@ class LayerState:
     def gemm_flops(self):
         return 2.0 * self.T * self.K * self.N * (3 if self.backward else 1)
 
+    def gemm_bytes(self):
+        """FP8 operands + bf16 output of this layer's matmuls."""
+        T, K, N = self.T, self.K, self.N
+        fwd = T * K + N * K + 2 * T * N
+        if not self.backward:
+            return fwd
+        return fwd + (T * N + N * K + 2 * T * K) + (T * N + T * K + 2 * N * K)
+
     def cast_elements(self):
         if not self.backward:
             return self.T * self.K          # weights were quantised once, at load
@@ -195,23 +206,39 @@ def run_layer(ctx, L, timers=None):
             timed("gemm", lambda: ctx.linear_wgrad(L.g8, None, bi[2:3], L.x8, None, bi[1:2], L.dw, L.T))
 
 
-def dist_setup(n_gpus):
+def dist_setup(n_gpus, backend="nccl"):
+    """One process per GPU (torchrun sets RANK / WORLD_SIZE / LOCAL_RANK).  The ranks are independent replicas:
+    the process group serves the barrier and the max-over-ranks of the measured time only.  `backend="gloo"`
+    is the CPU form used by the tests."""
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
+    cuda = backend == "nccl"
     if world > 1:
         import torch.distributed as dist
-        torch.cuda.set_device(local)
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+        if cuda:
+            torch.cuda.set_device(local)
+            dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+        else:
+            dist.init_process_group(backend)
         return rank, world, local, dist
-    torch.cuda.set_device(0)
+    if cuda:
+        torch.cuda.set_device(0)
     return 0, 1, 0, None
 
 
-def barrier_sync(dist):
+def barrier_sync(dist, cuda=True):
+    if cuda:
+        torch.cuda.synchronize()
     if dist is not None:
         dist.barrier()
-    torch.cuda.synchronize()
+    if cuda:
+        torch.cuda.synchronize()
+
+
+def whole_job_value(world, step_flops, ms_per_step):
+    """Aggregate TFLOP/s of `world` replicas that each did `step_flops` per step in the slowest rank's time."""
+    return world * step_flops / (ms_per_step * 1e-3) / 1e12
 
 
 def max_over_ranks(value, dist, device):
@@ -288,7 +315,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--transposed-copies", action="store_true",
                     help="also write transposed FP8 copies and contract the backward matmuls over contiguous bytes")
-    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     wl = I.WORKLOADS[args.workload]
@@ -342,7 +369,7 @@ def main():
 
     ms_per_step = total_ms / args.steps
     step_flops = sum(L.gemm_flops() for L in layers)
-    value = world * step_flops / (ms_per_step * 1e-3) / 1e12
+    value = whole_job_value(world, step_flops, ms_per_step)
 
     gemm_ms = timers.total_ms("gemm")
     gemm_launches = timers.count("gemm")
@@ -364,15 +391,37 @@ def main():
         h2d = sum(t.numel() * t.element_size() for ts in host_in for t in ts)
         d2h = sum(t.numel() * t.element_size() for ts in host_out for t in ts)
 
+        # three streams: host->device copies, compute, device->host copies; per layer the copy of its inputs,
+        # its kernels and the copy of its results are ordered by events, so the copies of one layer overlap the
+        # kernels of another (what a user of the API would do with pinned buffers)
+        s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
+        s_comp = torch.cuda.current_stream()
+        ev_comp = [None] * len(layers)   # kernels of layer i done (its inputs may be overwritten, its outputs read)
+        ev_out = [None] * len(layers)    # results of layer i copied out (its outputs may be overwritten)
+
         def e2e_step():
-            for L, hin, hout in zip(layers, host_in, host_out):
+            for i, (L, hin, hout) in enumerate(zip(layers, host_in, host_out)):
                 ins = [L.x] + ([L.w, L.g] if wl.backward else [])
                 outs = [L.y] + ([L.dx, L.dw] if wl.backward else [])
-                for d, h in zip(ins, hin):
-                    d.copy_(h, non_blocking=True)
+                with torch.cuda.stream(s_in):
+                    if ev_comp[i] is not None:
+                        s_in.wait_event(ev_comp[i])
+                    for d, h in zip(ins, hin):
+                        d.copy_(h, non_blocking=True)
+                    ev_in = torch.cuda.Event()
+                    ev_in.record(s_in)
+                s_comp.wait_event(ev_in)
+                if ev_out[i] is not None:
+                    s_comp.wait_event(ev_out[i])
                 run_layer(ctx, L)
-                for h, d in zip(hout, outs):
-                    h.copy_(d, non_blocking=True)
+                ev_comp[i] = torch.cuda.Event()
+                ev_comp[i].record(s_comp)
+                with torch.cuda.stream(s_out):
+                    s_out.wait_event(ev_comp[i])
+                    for h, d in zip(hout, outs):
+                        h.copy_(d, non_blocking=True)
+                    ev_out[i] = torch.cuda.Event()
+                    ev_out[i].record(s_out)
 
         e2e_step()
         barrier_sync(dist)
@@ -382,7 +431,8 @@ def main():
         barrier_sync(dist)
         e2e_ms = max_over_ranks(1e3 * (time.perf_counter() - t0) / args.e2e_steps, dist, device)
         e2e = {"value": world * step_flops / (e2e_ms * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": e2e_ms,
-               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+               "how": "pinned host buffers; copies in, kernels and copies out on three streams, ordered per layer"}
         del host_in, host_out
 
     if rank != 0:
@@ -416,7 +466,8 @@ def main():
                      "unit": "TFLOP/s", "frac": gemm_tflops / fp8_peak,
                      "peak_source": f"2 x {peaks['source']} sustained bf16 cuBLAS ({peaks['bf16_tflops_sustained']} TFLOP/s)",
                      "launches": gemm_launches, "avg_launch_ms": gemm_ms / max(1, gemm_launches),
-                     "traffic": None},
+                     "algorithmic_bytes_per_launch": sum(L.gemm_bytes() for L in layers) / max(1, gemm_launches / args.steps),
+                     "traffic": GEMM_DRAM_BYTES_PER_LAUNCH.get((wl.name, tokens))},
         "amax_cast": {"effective_gbs": cast_elems * bytes_per_elem / (cast_ms * 1e-3) / 1e9,
                       "bytes_per_element": bytes_per_elem, "ms_per_step": cast_ms / args.steps,
                       "hbm_peak_gbs": peaks["hbm_gbs"],

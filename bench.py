@@ -181,7 +181,9 @@ class Timers:
         return len(self.pairs[key])
 
 
-def run_layer(ctx, L, timers=None):
+def run_layer(ctx, L, timers=None, predict=False):
+    """One layer of one step.  predict=True quantises with fp8_cast_predicted: one pass per tensor when the bias
+    left by the previous step still holds (same results either way)."""
     def timed(key, fn):
         if timers is None:
             fn()
@@ -192,12 +194,18 @@ def run_layer(ctx, L, timers=None):
             b.record()
 
     af, bi = L.scal_f, L.scal_i
+    E4, E5 = 0, 1
+    if predict and not L.transposed:
+        quant = lambda fmt, x, j, y, yt: ctx.cast_predicted(fmt, x, af[j:j + 1], bi[j:j + 1], y)
+    else:
+        quant = lambda fmt, x, j, y, yt: (ctx.cast_e4 if fmt == E4 else ctx.cast_e5)(
+            x, None, d_amax_out=af[j:j + 1], d_bias_out=bi[j:j + 1], y=y, y_t=yt)
     if L.backward:  # training: the weights are re-quantised every step; inference: once at load (ptq_weights)
-        timed("amax_cast", lambda: ctx.cast_e4(L.w, None, d_amax_out=af[0:1], d_bias_out=bi[0:1], y=L.w8, y_t=L.w8t))
-    timed("amax_cast", lambda: ctx.cast_e4(L.x, None, d_amax_out=af[1:2], d_bias_out=bi[1:2], y=L.x8, y_t=L.x8t))
+        timed("amax_cast", lambda: quant(E4, L.w, 0, L.w8, L.w8t))
+    timed("amax_cast", lambda: quant(E4, L.x, 1, L.x8, L.x8t))
     timed("gemm", lambda: ctx.linear_fwd(L.x8, bi[1:2], L.w8, bi[0:1], L.y))
     if L.backward:
-        timed("amax_cast", lambda: ctx.cast_e5(L.g, None, d_amax_out=af[2:3], d_bias_out=bi[2:3], y=L.g8, y_t=L.g8t))
+        timed("amax_cast", lambda: quant(E5, L.g, 2, L.g8, L.g8t))
         if L.transposed:   # contraction over contiguous bytes, from the transposed copies
             timed("gemm", lambda: ctx.linear_dgrad(L.g8, bi[2:3], None, L.w8t, bi[0:1], L.dx))
             timed("gemm", lambda: ctx.linear_wgrad(None, L.g8t, bi[2:3], None, L.x8t, bi[1:2], L.dw, L.T))
@@ -315,6 +323,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--transposed-copies", action="store_true",
                     help="also write transposed FP8 copies and contract the backward matmuls over contiguous bytes")
+    ap.add_argument("--no-predicted-leg", action="store_true",
+                    help="skip the extra timed loop that uses fp8_cast_predicted")
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -378,6 +388,32 @@ def main():
     cast_elems = args.steps * sum(L.cast_elements() for L in layers)
     bytes_per_elem = 4 if (wl.backward and args.transposed_copies) else 3  # read once, write one byte per layout
     fp8_peak = 2.0 * peaks["bf16_tflops_sustained"]
+
+    # ---- the same steps with the one-pass quantisation (bias guessed from the previous step, verified) ----
+    predicted = None
+    if wl.backward and not args.transposed_copies and not args.no_predicted_leg:
+        ctx.prediction_stats(clear=True)
+        for _ in range(3):
+            for L in layers:
+                run_layer(ctx, L, predict=True)
+        ctx.prediction_stats(clear=True)
+        p_steps = min(args.steps, 100)
+        p_timers = Timers()
+        p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier_sync(dist)
+        p0.record()
+        for _ in range(p_steps):
+            for L in layers:
+                run_layer(ctx, L, p_timers, predict=True)
+        p1.record()
+        barrier_sync(dist)
+        p_ms = max_over_ranks(p0.elapsed_time(p1), dist, device) / p_steps
+        hits, misses = ctx.prediction_stats(clear=True)
+        predicted = {"value": whole_job_value(world, step_flops, p_ms), "unit": UNIT, "ms_per_step": p_ms, "steps": p_steps,
+                     "amax_cast_ms_per_step": p_timers.total_ms("amax_cast") / p_steps,
+                     "guesses_held": hits, "guesses_missed": misses,
+                     "note": "fp8_cast_predicted; the synthetic tensors repeat every step, so every guess holds "
+                             "(best case); results are bit-identical to the default path"}
 
     # ---- end to end through the public API with host buffers ----
     e2e = None
@@ -472,6 +508,7 @@ def main():
                       "bytes_per_element": bytes_per_elem, "ms_per_step": cast_ms / args.steps,
                       "hbm_peak_gbs": peaks["hbm_gbs"],
                       "frac": cast_elems * bytes_per_elem / (cast_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]},
+        "with_bias_prediction": predicted,
         "gemm_ms_per_step": gemm_ms / args.steps,
         "weight_stream_gbs": (None if wl.backward else
                               sum(L.N * L.K for L in layers) * args.steps / (gemm_ms * 1e-3) / 1e9),

@@ -152,6 +152,29 @@ FP8_API fp8_status_t fp8_cast_e5(fp8_ctx *ctx, const void *x, fp8_dtype_t x_dt, 
                          const int32_t *d_bias, fp8_conv_t conv, int32_t margin, float *d_amax_out,
                          int32_t *d_bias_out, uint8_t *y, uint8_t *y_t, void *stream);
 
+/* FP8-AMAX in a single pass over the tensor when the bias can be guessed
+ * (Section 3 names the problem -- just-in-time scaling costs a second round
+ * trip to memory -- and the remedy of leaning on the amax history; Appendix I
+ * shows how rarely the biases move).  *d_bias_inout holds a GUESS on entry,
+ * typically what the previous step left there.  The tensor is cast with the
+ * guess while its amax is taken in the same pass; the true bias is then
+ * compared with the guess and, only if they differ, the cast is redone.  On
+ * return d_amax_out, d_bias_inout and y are exactly what fp8_cast_e4 / _e5 with
+ * d_bias = NULL would have written, whatever the guess was (any int32 is a valid
+ * guess).  Cost: 3 bytes per element when the guess holds, 6 when it does not
+ * (the two-launch path always moves 5).
+ *   x   [rows, cols], dtype x_dt; the one-pass kernel needs ld == cols and
+ *       16-byte aligned x and y, other tensors silently take the two-launch path
+ *   y   out [rows, cols] bytes (row-major only)
+ * Two launches are always made (the second returns at once when the guess held). */
+FP8_API fp8_status_t fp8_cast_predicted(fp8_ctx *ctx, fp8_format_t fmt, const void *x, fp8_dtype_t x_dt, int64_t rows,
+                                        int64_t cols, int64_t ld, fp8_conv_t conv, int32_t margin, float *d_amax_out,
+                                        int32_t *d_bias_inout, uint8_t *y, void *stream);
+
+/* Synchronises `stream` and returns how many guesses of fp8_cast_predicted held / did not hold since the
+ * context was created or the counters were last cleared. */
+FP8_API fp8_status_t fp8_prediction_stats(fp8_ctx *ctx, void *stream, unsigned *hits, unsigned *misses, int clear);
+
 /* Post-training quantisation of one weight tensor (Section 3.1): amax -> bias
  * -> cast to E4, once.  w [N, K] (ld elements); outputs w8 [N, K] and/or
  * w8_t [K, N], d_bw, d_amax_w (both required). */

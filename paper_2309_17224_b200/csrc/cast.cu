@@ -29,10 +29,10 @@ __device__ __forceinline__ void cast_flat_body(const uint4 *__restrict__ x, uint
 {
     // nout = number of 16-byte output vectors; each consumes kIn input vectors (16 elements).
     constexpr int kIn = InType<DT>::kBytes;  // 2 vectors of 16-bit elements, 4 of fp32
-    const int64_t chunk = (int64_t)kCastThreads * 2;
+    const int64_t chunk = (int64_t)blockDim.x * 2;
     const int64_t nchunks = (nout + chunk - 1) / chunk;
     for (int64_t c = nchunks - 1 - blockIdx.x; c >= 0; c -= gridDim.x) {
-        int64_t idx[2] = {c * chunk + threadIdx.x, c * chunk + threadIdx.x + kCastThreads};
+        int64_t idx[2] = {c * chunk + threadIdx.x, c * chunk + threadIdx.x + blockDim.x};
         uint4 v[2][kIn];
 #pragma unroll
         for (int u = 0; u < 2; ++u)
@@ -56,11 +56,13 @@ __device__ __forceinline__ void cast_flat_body(const uint4 *__restrict__ x, uint
 }
 
 template <int FMT, int DT>
-__global__ void __launch_bounds__(kCastThreads) cast_flat_kernel(const uint4 *__restrict__ x, uint4 *__restrict__ y,
+__global__ void __launch_bounds__(1024) cast_flat_kernel(const uint4 *__restrict__ x, uint4 *__restrict__ y,
                                                                  int64_t nout, int ntail,
                                                                  const int32_t *__restrict__ d_bias, int delta,
-                                                                 unsigned *d_status)
+                                                                 unsigned *d_status, const unsigned *redo)
 {
+    // as the second launch of a predicted cast: nothing to do when the prediction held
+    if (redo != nullptr && *reinterpret_cast<const volatile unsigned *>(redo) == 0u) return;
     const int s = __ldg(d_bias) + delta;
     const Pow2Pair p = make_pow2_pair(s);
     bool sat = false;
@@ -181,7 +183,7 @@ static cudaError_t launch_cast(fp8_ctx *ctx, const void *x, int64_t rows, int64_
         int blocks = (int)(want < 1 ? 1 : (want > max_blocks ? max_blocks : want));
         cast_flat_kernel<FMT, DT><<<blocks, kCastThreads, 0, stream>>>(reinterpret_cast<const uint4 *>(x),
                                                                        reinterpret_cast<uint4 *>(y), nout, ntail,
-                                                                       d_bias, delta, ctx->d_status);
+                                                                       d_bias, delta, ctx->d_status, nullptr);
         return cudaGetLastError();
     }
     int fast_ok = al(x, 4 * kB) && (ld % 4) == 0 && (!y || (al(y, 4) && (cols % 4) == 0)) &&
@@ -200,6 +202,121 @@ static cudaError_t launch_cast_dt(int dt, fp8_ctx *ctx, const void *x, int64_t r
     if (dt == FP8_BF16) return launch_cast<FMT, FP8_BF16>(ctx, x, rows, cols, ld, d_bias, delta, y, y_t, stream);
     if (dt == FP8_F16) return launch_cast<FMT, FP8_F16>(ctx, x, rows, cols, ld, d_bias, delta, y, y_t, stream);
     return launch_cast<FMT, FP8_F32>(ctx, x, rows, cols, ld, d_bias, delta, y, y_t, stream);
+}
+
+// ---------------------------------------------------------------------------
+// FP8-AMAX in one pass when the bias can be guessed
+// ---------------------------------------------------------------------------
+//
+// Section 3 names the cost of just-in-time scaling (a second pass over memory) and the usual remedy (reuse the
+// amax history).  Scaling biases change rarely between training steps (Appendix I: weights and activations
+// almost never, gradients early on), so this kernel casts with a GUESS of the bias -- whatever the caller left in
+// the bias word, typically the previous step's value -- while it takes the amax of the same pass.  The last block
+// derives the true bias; if the guess was right the bytes already written are the exact FP8-AMAX result and the
+// second launch (the ordinary cast, gated on a flag) returns at once.  If it was wrong the second launch redoes
+// the cast with the true bias.  Either way the outputs equal fp8_cast_* with d_bias = NULL, bit for bit.
+// Traffic: 2 B read + 1 B written per element when the guess holds, twice that when it does not.
+
+template <int FMT, int DT>
+__global__ void __launch_bounds__(kCastThreads)
+cast_predicted_kernel(const uint4 *__restrict__ x, uint4 *__restrict__ y, int64_t nout, int ntail, int fmt, int conv,
+                      int margin, int delta, unsigned *slot, float *d_amax, int32_t *d_bias_inout, unsigned *d_status,
+                      unsigned *d_stats)
+{
+    constexpr int kIn = InType<DT>::kBytes;
+    constexpr int kW = InType<DT>::kWords4;
+    const int guess = *reinterpret_cast<const volatile int32_t *>(d_bias_inout);
+    const Pow2Pair p = make_pow2_pair(guess + delta);
+    bool sat = false;
+    uint32_t acc = 0;
+    const int64_t chunk = (int64_t)kCastThreads * 2;
+    const int64_t nchunks = (nout + chunk - 1) / chunk;
+    for (int64_t c = blockIdx.x; c < nchunks; c += gridDim.x) {
+        int64_t idx[2] = {c * chunk + threadIdx.x, c * chunk + threadIdx.x + kCastThreads};
+        uint4 v[2][kIn];
+#pragma unroll
+        for (int u = 0; u < 2; ++u)
+            if (idx[u] < nout) {
+#pragma unroll
+                for (int j = 0; j < kIn; ++j) v[u][j] = __ldcs(x + kIn * idx[u] + j);
+            }
+#pragma unroll
+        for (int u = 0; u < 2; ++u)
+            if (idx[u] < nout) {
+                const uint32_t *w = reinterpret_cast<const uint32_t *>(&v[u][0]);
+#pragma unroll
+                for (int j = 0; j < 4 * kIn; ++j)
+                    acc = DT == FP8_F32 ? max(acc, w[j] & 0x7FFFFFFFu) : __vmaxu2(acc, w[j] & 0x7FFF7FFFu);
+                uint4 o;
+                o.x = cast4w<FMT, DT, true>(w + 0 * kW, p, sat);
+                o.y = cast4w<FMT, DT, true>(w + 1 * kW, p, sat);
+                o.z = cast4w<FMT, DT, true>(w + 2 * kW, p, sat);
+                o.w = cast4w<FMT, DT, true>(w + 3 * kW, p, sat);
+                y[idx[u]] = o;
+            }
+    }
+    if (blockIdx.x == 0 && (int)threadIdx.x < ntail) {
+        const int64_t i = nout * 16 + threadIdx.x;
+        if (DT == FP8_F32) acc = max(acc, reinterpret_cast<const uint32_t *>(x)[i] & 0x7FFFFFFFu);
+        else acc = __vmaxu2(acc, (uint32_t)reinterpret_cast<const uint16_t *>(x)[i] & 0x7FFFu);
+        reinterpret_cast<uint8_t *>(y)[i] = cast1<FMT, DT, true>(x, i, p, sat);
+    }
+    // grid-wide max; the last block compares the true bias with the guess
+    __shared__ uint32_t warp_max[kCastThreads / 32];
+    uint32_t m = DT == FP8_F32 ? acc : max(acc & 0xFFFFu, acc >> 16);
+    m = __reduce_max_sync(0xFFFFFFFFu, m);
+    if ((threadIdx.x & 31) == 0) warp_max[threadIdx.x >> 5] = m;
+    const int any_sat = __syncthreads_or(sat);
+    if (threadIdx.x == 0) {
+        for (int i = 1; i < kCastThreads / 32; ++i) m = max(m, warp_max[i]);
+        atomicMax(&slot[0], m);
+        if (any_sat) atomicOr(&slot[2], 1u);
+        __threadfence();
+        if (atomicAdd(&slot[1], 1u) + 1u == gridDim.x) {
+            __threadfence();
+            const uint32_t total = atomicExch(&slot[0], 0u);
+            const unsigned was_sat = atomicExch(&slot[2], 0u);
+            slot[1] = 0u;
+            uint32_t fbits;
+            if (DT == FP8_F32) fbits = total;
+            else if (DT == FP8_BF16) fbits = total << 16;
+            else { float f; asm("cvt.f32.f16 %0, %1;" : "=f"(f) : "h"((uint16_t)total)); fbits = __float_as_uint(f); }
+            *d_amax = __uint_as_float(fbits);
+            unsigned flags = 0;
+            const int b = bias_from_amax_bits(fbits, fmt, conv, margin, &flags);
+            const bool hit = (b == guess);
+            *d_bias_inout = b;
+            slot[3] = hit ? 0u : 1u;               // read by the gated second launch
+            atomicAdd(&d_stats[hit ? 0 : 1], 1u);
+            if (hit && was_sat) flags |= FP8_FLAG_SATURATED;   // clipping under a wrong guess says nothing
+            if (flags) atomicOr(d_status, flags);
+        }
+    }
+}
+
+template <int FMT, int DT>
+static cudaError_t launch_predicted(fp8_ctx *ctx, const void *x, int64_t n, int conv, int margin, float *d_amax,
+                                    int32_t *d_bias_inout, uint8_t *y, cudaStream_t stream)
+{
+    int64_t nout = n / 16;
+    int ntail = (int)(n - nout * 16);
+    int64_t chunk = (int64_t)kCastThreads * 2;
+    int64_t want = (nout + chunk - 1) / chunk;
+    int max_blocks = ctx->sm_count * 8;
+    int blocks = (int)(want < 1 ? 1 : (want > max_blocks ? max_blocks : want));
+    unsigned *slot = take_slot(ctx);
+    const int delta = format_delta(FMT, conv);
+    cast_predicted_kernel<FMT, DT><<<blocks, kCastThreads, 0, stream>>>(
+        reinterpret_cast<const uint4 *>(x), reinterpret_cast<uint4 *>(y), nout, ntail, FMT, conv, margin, delta, slot,
+        d_amax, d_bias_inout, ctx->d_status, ctx->d_predict_stats);
+    if (cudaGetLastError() != cudaSuccess) return cudaErrorUnknown;
+    // the gated second launch: few, large blocks (same threads per SM), so that it costs little when it has nothing to do
+    int64_t want2 = (nout + 2047) / 2048;
+    int blocks2 = (int)(want2 < 1 ? 1 : (want2 > 2 * ctx->sm_count ? 2 * ctx->sm_count : want2));
+    cast_flat_kernel<FMT, DT><<<blocks2, 1024, 0, stream>>>(reinterpret_cast<const uint4 *>(x),
+                                                            reinterpret_cast<uint4 *>(y), nout, ntail, d_bias_inout,
+                                                            delta, ctx->d_status, slot + 3);
+    return cudaGetLastError();
 }
 
 static fp8_status_t cast_entry(int fmt, fp8_ctx *ctx, const void *x, fp8_dtype_t x_dt, int64_t rows, int64_t cols,
@@ -251,6 +368,50 @@ fp8_status_t fp8_cast_e5(fp8_ctx *ctx, const void *x, fp8_dtype_t x_dt, int64_t 
 {
     return fp8lin::cast_entry(FP8_E5, ctx, x, x_dt, rows, cols, ld, d_bias, conv, margin, d_amax_out, d_bias_out, y,
                               y_t, stream);
+}
+
+fp8_status_t fp8_cast_predicted(fp8_ctx *ctx, fp8_format_t fmt, const void *x, fp8_dtype_t x_dt, int64_t rows,
+                                int64_t cols, int64_t ld, fp8_conv_t conv, int32_t margin, float *d_amax_out,
+                                int32_t *d_bias_inout, uint8_t *y, void *stream)
+{
+    using namespace fp8lin;
+    if (!ctx || !x || !y || !d_amax_out || !d_bias_inout) return FP8_ERR_NULL;
+    if ((int)fmt < 0 || (int)fmt > 1 || (int)x_dt < 0 || (int)x_dt > 2 || (int)conv < 0 || (int)conv > 1)
+        return FP8_ERR_DTYPE;
+    if (rows <= 0 || cols <= 0 || ld < cols) return FP8_ERR_SHAPE;
+    auto al16 = [](const void *q) { return (reinterpret_cast<uintptr_t>(q) & 15u) == 0; };
+    if (ld != cols || !al16(x) || !al16(y))   // outside the one-pass kernel's shape rules: the ordinary FP8-AMAX path
+        return cast_entry((int)fmt, ctx, x, x_dt, rows, cols, ld, nullptr, conv, margin, d_amax_out, d_bias_inout, y,
+                          nullptr, stream);
+    cudaStream_t st = (cudaStream_t)stream;
+    const int64_t n = rows * cols;
+    cudaError_t e;
+#define FP8LIN_PRED(F, D) e = launch_predicted<F, D>(ctx, x, n, (int)conv, margin, d_amax_out, d_bias_inout, y, st)
+    if (fmt == FP8_E4) {
+        if (x_dt == FP8_BF16) FP8LIN_PRED(FP8_E4, FP8_BF16);
+        else if (x_dt == FP8_F16) FP8LIN_PRED(FP8_E4, FP8_F16);
+        else FP8LIN_PRED(FP8_E4, FP8_F32);
+    } else {
+        if (x_dt == FP8_BF16) FP8LIN_PRED(FP8_E5, FP8_BF16);
+        else if (x_dt == FP8_F16) FP8LIN_PRED(FP8_E5, FP8_F16);
+        else FP8LIN_PRED(FP8_E5, FP8_F32);
+    }
+#undef FP8LIN_PRED
+    return e == cudaSuccess ? FP8_OK : FP8_ERR_CUDA;
+}
+
+fp8_status_t fp8_prediction_stats(fp8_ctx *ctx, void *stream, unsigned *hits, unsigned *misses, int clear)
+{
+    if (!ctx || !hits || !misses) return FP8_ERR_NULL;
+    cudaStream_t st = (cudaStream_t)stream;
+    unsigned host[2] = {0, 0};
+    if (cudaMemcpyAsync(host, ctx->d_predict_stats, sizeof(host), cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return FP8_ERR_CUDA;
+    if (clear && cudaMemsetAsync(ctx->d_predict_stats, 0, sizeof(host), st) != cudaSuccess) return FP8_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return FP8_ERR_CUDA;
+    *hits = host[0];
+    *misses = host[1];
+    return FP8_OK;
 }
 
 fp8_status_t fp8_ptq_weights(fp8_ctx *ctx, const void *w, fp8_dtype_t w_dt, int64_t N, int64_t K, int64_t ld,

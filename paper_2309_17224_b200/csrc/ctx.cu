@@ -42,12 +42,13 @@ fp8_status_t fp8_create(fp8_ctx **out, int device)
     if (!ok) { delete ctx; return FP8_ERR_CUDA; }
     if (major != 10) { delete ctx; return FP8_ERR_UNSUPPORTED; }  // sm_100a code only
 
-    size_t words = 1 + (size_t)fp8lin::kReduceSlots * fp8lin::kSlotWords;
+    size_t words = 1 + (size_t)fp8lin::kReduceSlots * fp8lin::kSlotWords + 2;
     unsigned *buf = nullptr;
     if (cudaMalloc(&buf, words * sizeof(unsigned)) != cudaSuccess) { delete ctx; return FP8_ERR_CUDA; }
     if (cudaMemset(buf, 0, words * sizeof(unsigned)) != cudaSuccess) { cudaFree(buf); delete ctx; return FP8_ERR_CUDA; }
     ctx->d_status = buf;
     ctx->d_slots = buf + 1;
+    ctx->d_predict_stats = buf + 1 + fp8lin::kReduceSlots * fp8lin::kSlotWords;
     ctx->partial_bytes = (size_t)64 << 20;
     ctx->d_partial = nullptr;
     if (cudaMalloc(&ctx->d_partial, ctx->partial_bytes) != cudaSuccess) { cudaFree(buf); delete ctx; return FP8_ERR_CUDA; }

@@ -14,7 +14,7 @@ namespace fp8lin {
 // ---------------------------------------------------------------------------
 
 constexpr int kReduceSlots = 64;   // independent grid-reduction slots, used round-robin
-constexpr int kSlotWords = 4;      // {running max, arrival counter, pad, pad}
+constexpr int kSlotWords = 4;      // {running max, arrival counter, scratch flag, redo flag of a predicted cast}
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *,
@@ -30,6 +30,7 @@ struct fp8_ctx {
     unsigned *d_status;   // one sticky word of FP8_FLAG_* bits
     unsigned *d_slots;    // kReduceSlots * kSlotWords words, all zero between calls
     unsigned next_slot;
+    unsigned *d_predict_stats;   // {guesses that held, guesses that did not} of fp8_cast_predicted
     float *d_partial;     // FP32 workspace for split-K partial sums
     size_t partial_bytes;
     fp8lin::EncodeTiledFn encode_tiled;

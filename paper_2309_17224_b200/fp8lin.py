@@ -28,7 +28,7 @@ FLAG_NONFINITE_AMAX, FLAG_ZERO_AMAX, FLAG_SATURATED, FLAG_TIMEOUT = 1, 2, 4, 8
 SYMBOLS = (
     "fp8_create", "fp8_destroy", "fp8_status_string", "fp8_device_flags", "fp8_amax", "fp8_scaling_bias",
     "fp8_scaling_bias_host", "fp8_cast_e4", "fp8_cast_e5", "fp8_ptq_weights", "fp8_linear_fwd", "fp8_linear_dgrad",
-    "fp8_linear_wgrad", "fp8_amax_noalloc", "fp8_linear_fwd_act",
+    "fp8_linear_wgrad", "fp8_amax_noalloc", "fp8_linear_fwd_act", "fp8_cast_predicted", "fp8_prediction_stats",
 )
 
 if not os.path.exists(LIB_PATH):
@@ -51,6 +51,8 @@ _lib.fp8_scaling_bias_host.argtypes = [c_float, c_int, c_int, c_int32, POINTER(c
 _cast_args = [_P, _P, c_int, c_int64, c_int64, c_int64, _P, c_int, c_int32, _P, _P, _P, _P, _P]
 _lib.fp8_cast_e4.argtypes = _cast_args
 _lib.fp8_cast_e5.argtypes = _cast_args
+_lib.fp8_cast_predicted.argtypes = [_P, c_int, _P, c_int, c_int64, c_int64, c_int64, c_int, c_int32, _P, _P, _P, _P]
+_lib.fp8_prediction_stats.argtypes = [_P, _P, POINTER(c_uint), POINTER(c_uint), c_int]
 _lib.fp8_ptq_weights.argtypes = [_P, _P, c_int, c_int64, c_int64, c_int64, c_int, _P, _P, _P, _P, _P]
 _lib.fp8_linear_fwd.argtypes = [_P, _P, _P, _P, _P, _P, c_int, _P, c_int, _P, c_int64, c_int64, c_int64, c_int, _P]
 _lib.fp8_linear_fwd_act.argtypes = [_P, _P, _P, _P, _P, _P, c_int, _P, _P, c_int, _P, c_int64, c_int64, c_int64, c_int, _P]
@@ -164,6 +166,20 @@ class Context:
                 rows=None, cols=None, ld=None):
         self._cast(_lib.fp8_cast_e5, "fp8_cast_e5", x, d_bias, conv, margin, d_amax_out, d_bias_out, y, y_t, rows,
                    cols, ld)
+
+    def cast_predicted(self, fmt, x, d_amax_out, d_bias_inout, y, conv=CONV_PAPER, margin=0, rows=None, cols=None,
+                       ld=None):
+        rows = x.shape[0] if rows is None else rows
+        cols = x.shape[1] if cols is None else cols
+        ld = _ld(x) if ld is None else ld
+        _check(_lib.fp8_cast_predicted(self._h, fmt, _ptr(x), _DT[x.dtype], rows, cols, ld, conv, margin,
+                                       _ptr(d_amax_out), _ptr(d_bias_inout), _ptr(y), _stream()), "fp8_cast_predicted")
+
+    def prediction_stats(self, clear: bool = True):
+        hits, misses = c_uint(0), c_uint(0)
+        _check(_lib.fp8_prediction_stats(self._h, _stream(), byref(hits), byref(misses), 1 if clear else 0),
+               "fp8_prediction_stats")
+        return hits.value, misses.value
 
     def ptq_weights(self, w, conv, w8, w8_t, d_bw, d_amax_w):
         _check(_lib.fp8_ptq_weights(self._h, _ptr(w), _DT[w.dtype], w.shape[0], w.shape[1], _ld(w), conv,

@@ -1,0 +1,98 @@
+"""fp8_cast_predicted: FP8-AMAX in one pass when the bias guess holds.  Whatever
+the guess, amax, bias and bytes must equal the oracle's (and therefore the
+two-launch path's), and the hit / miss counters must tell the two cases apart."""
+import numpy as np
+import pytest
+import torch
+
+import oracle as O
+from helpers import assert_codes_equal, bits_of, u8
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_2309_17224_b200 import fp8lin
+    return fp8lin
+
+
+@pytest.fixture(scope="module")
+def ctx(lib):
+    c = lib.Context(0)
+    yield c
+    c.close()
+
+
+def _host(t):
+    return bits_of(t) if t.dtype == torch.bfloat16 else t.detach().contiguous().cpu().numpy()
+
+
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float16, torch.float32])
+@pytest.mark.parametrize("kind", [O.E4, O.E5])
+@pytest.mark.parametrize("shape", [(1, 5), (64, 64), (300, 520), (1024, 4096)])
+def test_any_guess_gives_the_exact_result(ctx, lib, dtype, kind, shape):
+    g = torch.Generator(device="cuda").manual_seed(shape[0] + 17 * kind)
+    x = (torch.randn(shape, generator=g, device="cuda") * 0.02).to(dtype)
+    a, b, want = O.quantise(_host(x), kind, O.CONV_PAPER, 0)
+    fmt = O.native_format(kind)
+    amax = torch.zeros(1, dtype=torch.float32, device="cuda")
+    bias = torch.zeros(1, dtype=torch.int32, device="cuda")
+    y = torch.empty(shape, dtype=torch.uint8, device="cuda")
+    ctx.prediction_stats(clear=True)
+    ctx.device_flags(clear=True)
+    guesses = [b, b + 1, b - 7, 0, 2 ** 31 - 1, -2 ** 31, b]
+    expected_hits = sum(1 for q in guesses if q == b)
+    for guess in guesses:
+        bias.fill_(guess)
+        y.fill_(0x55)
+        amax.fill_(-1.0)
+        ctx.cast_predicted(kind, x, amax, bias, y)
+        assert float(amax.item()) == a and int(bias.item()) == b, guess
+        assert_codes_equal(u8(y), want, fmt)
+    hits, misses = ctx.prediction_stats(clear=True)
+    assert (hits, misses) == (expected_hits, len(guesses) - expected_hits)
+    assert ctx.prediction_stats() == (0, 0)
+
+
+def test_steady_state_and_a_moving_tensor(ctx, lib):
+    """Same tensor every step: one miss, then hits.  A tensor whose scale doubles every step: all misses, and
+    still the exact result every time."""
+    x = torch.randn((512, 1024), device="cuda").to(torch.bfloat16)
+    amax = torch.zeros(1, dtype=torch.float32, device="cuda")
+    bias = torch.full((1,), 99, dtype=torch.int32, device="cuda")
+    y = torch.empty((512, 1024), dtype=torch.uint8, device="cuda")
+    ctx.prediction_stats(clear=True)
+    for _ in range(6):
+        ctx.cast_predicted(lib.E4, x, amax, bias, y)
+    assert ctx.prediction_stats(clear=True) == (5, 1)
+    for k in range(5):
+        xk = (x.float() * 2.0 ** (k + 1)).to(torch.bfloat16)
+        a, b, want = O.quantise(bits_of(xk), O.E4)
+        ctx.cast_predicted(lib.E4, xk, amax, bias, y)
+        assert int(bias.item()) == b
+        assert_codes_equal(u8(y), want, O.N_E4)
+    assert ctx.prediction_stats(clear=True) == (0, 5)
+
+
+def test_saturation_flag_only_reports_the_true_bias(ctx, lib):
+    ctx.device_flags(clear=True)
+    x = torch.full((256, 256), 3.0, dtype=torch.bfloat16, device="cuda")   # 3 * 2^7 = 384 fits natively: no clipping
+    amax = torch.zeros(1, dtype=torch.float32, device="cuda")
+    bias = torch.full((1,), 20, dtype=torch.int32, device="cuda")          # wildly too large a guess: pass one clips
+    y = torch.empty((256, 256), dtype=torch.uint8, device="cuda")
+    ctx.cast_predicted(lib.E4, x, amax, bias, y)
+    assert int(bias.item()) == 6 and ctx.device_flags() == 0
+    assert_codes_equal(u8(y), O.cast(bits_of(x), 7, O.N_E4), O.N_E4)
+
+
+def test_strided_input_takes_the_two_launch_path(ctx, lib):
+    big = torch.randn((128, 300), device="cuda").to(torch.bfloat16)
+    view = big[:, 8:264]
+    a, b, want = O.quantise(bits_of(view), O.E4)
+    amax = torch.zeros(1, dtype=torch.float32, device="cuda")
+    bias = torch.zeros(1, dtype=torch.int32, device="cuda")
+    y = torch.empty((128, 256), dtype=torch.uint8, device="cuda")
+    ctx.cast_predicted(lib.E4, view, amax, bias, y, rows=128, cols=256, ld=300)
+    assert float(amax.item()) == a and int(bias.item()) == b
+    assert_codes_equal(u8(y), want, O.N_E4)

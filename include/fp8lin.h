@@ -140,6 +140,12 @@ FP8_API fp8_status_t fp8_scaling_bias_host(float amax, fp8_format_t fmt, fp8_con
  *              NULL selects FP8-AMAX: amax and bias are computed here first
  *              (with `margin`) and written to d_amax_out / d_bias_out, both
  *              then required.
+ *              Non-NULL together with non-NULL d_amax_out and d_bias_out is
+ *              delayed scaling (the remedy Section 3 mentions for hardware
+ *              where the second pass is too costly): the cast uses d_bias, and
+ *              the same pass also writes this tensor's own amax and the bias
+ *              Eq. 3 gives for it, for use at the next step.  d_bias_out may be
+ *              the same word as d_bias.
  *   y          out [rows, cols] bytes, contiguous, or NULL
  *   y_t        out [cols, rows] bytes (the transposed copy, same codes), or NULL
  * At least one of y, y_t.  The vectorised paths need 16-byte aligned x, y, y_t,

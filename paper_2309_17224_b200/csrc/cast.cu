@@ -220,12 +220,14 @@ static cudaError_t launch_cast_dt(int dt, fp8_ctx *ctx, const void *x, int64_t r
 template <int FMT, int DT>
 __global__ void __launch_bounds__(kCastThreads)
 cast_predicted_kernel(const uint4 *__restrict__ x, uint4 *__restrict__ y, int64_t nout, int ntail, int fmt, int conv,
-                      int margin, int delta, unsigned *slot, float *d_amax, int32_t *d_bias_inout, unsigned *d_status,
-                      unsigned *d_stats)
+                      int margin, int delta, unsigned *slot, float *d_amax, const int32_t *d_bias_in,
+                      int32_t *d_bias_out, int verify, unsigned *d_status, unsigned *d_stats)
 {
+    // verify != 0: d_bias_in is a guess to be checked (fp8_cast_predicted).  verify == 0: d_bias_in is the bias to
+    // use, full stop, and the amax / bias of this tensor are by-products for the next step (delayed scaling).
     constexpr int kIn = InType<DT>::kBytes;
     constexpr int kW = InType<DT>::kWords4;
-    const int guess = *reinterpret_cast<const volatile int32_t *>(d_bias_inout);
+    const int guess = *reinterpret_cast<const volatile int32_t *>(d_bias_in);
     const Pow2Pair p = make_pow2_pair(guess + delta);
     bool sat = false;
     uint32_t acc = 0;
@@ -284,10 +286,10 @@ cast_predicted_kernel(const uint4 *__restrict__ x, uint4 *__restrict__ y, int64_
             *d_amax = __uint_as_float(fbits);
             unsigned flags = 0;
             const int b = bias_from_amax_bits(fbits, fmt, conv, margin, &flags);
-            const bool hit = (b == guess);
-            *d_bias_inout = b;
+            const bool hit = (b == guess) || !verify;
+            *d_bias_out = b;
             slot[3] = hit ? 0u : 1u;               // read by the gated second launch
-            atomicAdd(&d_stats[hit ? 0 : 1], 1u);
+            if (verify) atomicAdd(&d_stats[hit ? 0 : 1], 1u);
             if (hit && was_sat) flags |= FP8_FLAG_SATURATED;   // clipping under a wrong guess says nothing
             if (flags) atomicOr(d_status, flags);
         }
@@ -296,7 +298,8 @@ cast_predicted_kernel(const uint4 *__restrict__ x, uint4 *__restrict__ y, int64_
 
 template <int FMT, int DT>
 static cudaError_t launch_predicted(fp8_ctx *ctx, const void *x, int64_t n, int conv, int margin, float *d_amax,
-                                    int32_t *d_bias_inout, uint8_t *y, cudaStream_t stream)
+                                    const int32_t *d_bias_in, int32_t *d_bias_inout, int verify, uint8_t *y,
+                                    cudaStream_t stream)
 {
     int64_t nout = n / 16;
     int ntail = (int)(n - nout * 16);
@@ -308,8 +311,9 @@ static cudaError_t launch_predicted(fp8_ctx *ctx, const void *x, int64_t n, int 
     const int delta = format_delta(FMT, conv);
     cast_predicted_kernel<FMT, DT><<<blocks, kCastThreads, 0, stream>>>(
         reinterpret_cast<const uint4 *>(x), reinterpret_cast<uint4 *>(y), nout, ntail, FMT, conv, margin, delta, slot,
-        d_amax, d_bias_inout, ctx->d_status, ctx->d_predict_stats);
+        d_amax, d_bias_in, d_bias_inout, verify, ctx->d_status, ctx->d_predict_stats);
     if (cudaGetLastError() != cudaSuccess) return cudaErrorUnknown;
+    if (!verify) return cudaSuccess;
     // the gated second launch: few, large blocks (same threads per SM), so that it costs little when it has nothing to do
     int64_t want2 = (nout + 2047) / 2048;
     int blocks2 = (int)(want2 < 1 ? 1 : (want2 > 2 * ctx->sm_count ? 2 * ctx->sm_count : want2));
@@ -331,22 +335,40 @@ static fp8_status_t cast_entry(int fmt, fp8_ctx *ctx, const void *x, fp8_dtype_t
     cudaStream_t st = (cudaStream_t)stream;
     const int32_t *bias = d_bias;
     if (!bias) {
-        // FP8-AMAX: (opt-in) one cooperative launch when a bf16 tensor is made of whole 128x128 tiles ...
-        if (x_dt == FP8_BF16) {
-            cudaError_t fe = launch_cast_fused(ctx, fmt, x, rows, cols, ld, (int)conv, margin, d_amax_out, d_bias_out,
-                                               y, y_t, st);
-            if (fe == cudaSuccess) return FP8_OK;
-            cudaGetLastError();
-        }
-        // ... otherwise amax + bias in one launch, the cast in a second
+        // FP8-AMAX: amax + bias in one launch, the cast in a second
         if (launch_amax_bias(ctx, x, (int)x_dt, rows, cols, ld, d_amax_out, d_bias_out, fmt, (int)conv, margin, st) !=
             cudaSuccess)
             return FP8_ERR_CUDA;
         bias = d_bias_out;
     }
     int delta = format_delta(fmt, (int)conv);
+    // Delayed scaling: the bias is given AND the caller wants this tensor's own amax / bias (for the next step).
+    const bool delayed = d_bias && d_amax_out && d_bias_out;
+    if (delayed) {
+        auto al16 = [](const void *q) { return (reinterpret_cast<uintptr_t>(q) & 15u) == 0; };
+        if (!y_t && ld == cols && al16(x) && al16(y)) {   // one pass: cast and amax together
+            const int64_t n = rows * cols;
+            cudaError_t pe;
+#define FP8LIN_DELAYED(F, D) \
+    pe = launch_predicted<F, D>(ctx, x, n, (int)conv, margin, d_amax_out, d_bias, d_bias_out, 0, y, st)
+            if (fmt == FP8_E4) {
+                if (x_dt == FP8_BF16) FP8LIN_DELAYED(FP8_E4, FP8_BF16);
+                else if (x_dt == FP8_F16) FP8LIN_DELAYED(FP8_E4, FP8_F16);
+                else FP8LIN_DELAYED(FP8_E4, FP8_F32);
+            } else {
+                if (x_dt == FP8_BF16) FP8LIN_DELAYED(FP8_E5, FP8_BF16);
+                else if (x_dt == FP8_F16) FP8LIN_DELAYED(FP8_E5, FP8_F16);
+                else FP8LIN_DELAYED(FP8_E5, FP8_F32);
+            }
+#undef FP8LIN_DELAYED
+            return pe == cudaSuccess ? FP8_OK : FP8_ERR_CUDA;
+        }
+    }
     cudaError_t e = fmt == FP8_E4 ? launch_cast_dt<FP8_E4>((int)x_dt, ctx, x, rows, cols, ld, bias, delta, y, y_t, st)
                                   : launch_cast_dt<FP8_E5>((int)x_dt, ctx, x, rows, cols, ld, bias, delta, y, y_t, st);
+    // other shapes: the cast above used d_bias (read before this launch overwrites d_bias_out, stream order)
+    if (e == cudaSuccess && delayed)
+        e = launch_amax_bias(ctx, x, (int)x_dt, rows, cols, ld, d_amax_out, d_bias_out, fmt, (int)conv, margin, st);
     return e == cudaSuccess ? FP8_OK : FP8_ERR_CUDA;
 }
 
@@ -386,7 +408,8 @@ fp8_status_t fp8_cast_predicted(fp8_ctx *ctx, fp8_format_t fmt, const void *x, f
     cudaStream_t st = (cudaStream_t)stream;
     const int64_t n = rows * cols;
     cudaError_t e;
-#define FP8LIN_PRED(F, D) e = launch_predicted<F, D>(ctx, x, n, (int)conv, margin, d_amax_out, d_bias_inout, y, st)
+#define FP8LIN_PRED(F, D) \
+    e = launch_predicted<F, D>(ctx, x, n, (int)conv, margin, d_amax_out, d_bias_inout, d_bias_inout, 1, y, st)
     if (fmt == FP8_E4) {
         if (x_dt == FP8_BF16) FP8LIN_PRED(FP8_E4, FP8_BF16);
         else if (x_dt == FP8_F16) FP8LIN_PRED(FP8_E4, FP8_F16);

@@ -118,10 +118,4 @@ __device__ __forceinline__ void transpose4x4(const uint32_t r[4], uint32_t c[4])
 }
 
 
-// Launches the fused single-launch amax + bias + cast (cast_fused.cu).  Returns cudaErrorNotSupported when the
-// tensor does not meet its shape rules, in which case the caller uses the two-launch path.
-cudaError_t launch_cast_fused(fp8_ctx *ctx, int fmt, const void *x, int64_t rows, int64_t cols, int64_t ld, int conv,
-                              int margin, float *d_amax_out, int32_t *d_bias_out, uint8_t *y, uint8_t *y_t,
-                              cudaStream_t stream);
-
 }  // namespace fp8lin

@@ -96,3 +96,28 @@ def test_strided_input_takes_the_two_launch_path(ctx, lib):
     ctx.cast_predicted(lib.E4, view, amax, bias, y, rows=128, cols=256, ld=300)
     assert float(amax.item()) == a and int(bias.item()) == b
     assert_codes_equal(u8(y), want, O.N_E4)
+
+
+@pytest.mark.parametrize("shape,transposed", [((512, 1024), False), ((300, 520), False), ((256, 384), True)])
+def test_delayed_scaling_casts_with_the_given_bias_and_reports_the_next_one(ctx, lib, shape, transposed):
+    """fp8_cast_e4 with a bias AND output slots: bytes follow the given bias; amax and the bias Eq. 3 gives for
+    this tensor come out of the same call for the next step."""
+    x = (torch.randn(shape, device="cuda") * 0.05).to(torch.bfloat16)
+    xb = bits_of(x)
+    a, b_true = O.amax(xb), None
+    b_true = O.scaling_bias(a, O.E4)
+    stale = b_true - 2                      # e.g. last step's tensor was four times larger
+    bias_in = torch.full((1,), stale, dtype=torch.int32, device="cuda")
+    amax = torch.zeros(1, dtype=torch.float32, device="cuda")
+    bias_next = torch.zeros(1, dtype=torch.int32, device="cuda")
+    y = torch.empty(shape, dtype=torch.uint8, device="cuda")
+    y_t = torch.empty(shape[::-1], dtype=torch.uint8, device="cuda") if transposed else None
+    ctx.cast_e4(x, bias_in, d_amax_out=amax, d_bias_out=bias_next, y=y, y_t=y_t)
+    assert_codes_equal(u8(y), O.cast(xb, stale + 1, O.N_E4), O.N_E4)
+    if transposed:
+        assert_codes_equal(u8(y_t), O.cast(xb, stale + 1, O.N_E4).T, O.N_E4)
+    assert float(amax.item()) == a and int(bias_next.item()) == b_true and int(bias_in.item()) == stale
+    # in place: the same word holds the bias used and then the next one
+    ctx.cast_e4(x, bias_in, d_amax_out=amax, d_bias_out=bias_in, y=y, y_t=y_t)
+    assert_codes_equal(u8(y), O.cast(xb, stale + 1, O.N_E4), O.N_E4)
+    assert int(bias_in.item()) == b_true

@@ -15,6 +15,8 @@
 // Both walk the tensor from its end to its start: when the amax pass has just
 // streamed the tensor front to back, the part most recently read is the part
 // most likely still in L2.
+#include <cstdlib>
+
 #include "cast_common.cuh"
 
 namespace fp8lin {
@@ -323,6 +325,158 @@ static cudaError_t launch_predicted(fp8_ctx *ctx, const void *x, int64_t n, int 
     return cudaGetLastError();
 }
 
+// ---------------------------------------------------------------------------
+// small tensors: FP8-AMAX in one launch, the tensor held in registers
+// ---------------------------------------------------------------------------
+//
+// Decode-size activations (a few tokens x hidden size) are far too small to fill the GPU, and two launches
+// plus a grid-level reduction cost more than the work.  Here one thread-block cluster of one or two CTAs loads
+// the whole tensor into registers (at most eight 16-byte vectors per thread), reduces the amax through shared
+// memory and across the cluster through distributed shared memory, and casts from the registers: one launch,
+// 2 B read + 1 B written per element, no global scratch.
+
+constexpr int kSmallThreads = 1024;
+constexpr int kSmallVecs = 8;          // 16-byte vectors per thread
+constexpr int kSmallMaxCtas = 2;   // beyond ~128K elements the two-launch path (whole GPU) is faster
+
+template <int FMT, int DT>
+__global__ void __launch_bounds__(kSmallThreads)
+cast_small_kernel(const uint4 *__restrict__ x, uint4 *__restrict__ y, int64_t nvec, int ntail, int fmt, int conv,
+                  int margin, int delta, float *d_amax, int32_t *d_bias, unsigned *d_status)
+{
+    constexpr int kPerVec = 16 / InType<DT>::kBytes;     // input elements per 16-byte vector
+    constexpr int kW = InType<DT>::kWords4;
+    __shared__ uint32_t warp_max[kSmallThreads / 32];
+    __shared__ uint32_t cta_max;
+    uint32_t rank, nctas;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(rank));
+    asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(nctas));
+    const int64_t stride = (int64_t)nctas * kSmallThreads;
+    const int64_t t0 = (int64_t)rank * kSmallThreads + threadIdx.x;
+
+    uint4 v[kSmallVecs];
+    uint32_t acc = 0;
+#pragma unroll
+    for (int j = 0; j < kSmallVecs; ++j) {
+        const int64_t i = t0 + j * stride;
+        v[j] = i < nvec ? __ldcs(x + i) : make_uint4(0, 0, 0, 0);
+    }
+#pragma unroll
+    for (int j = 0; j < kSmallVecs; ++j) {
+        const uint32_t *w = reinterpret_cast<const uint32_t *>(&v[j]);
+#pragma unroll
+        for (int k = 0; k < 4; ++k) acc = DT == FP8_F32 ? max(acc, w[k] & 0x7FFFFFFFu) : __vmaxu2(acc, w[k] & 0x7FFF7FFFu);
+    }
+    if (rank == 0 && (int)threadIdx.x < ntail) {
+        const int64_t i = nvec * kPerVec + threadIdx.x;
+        if (DT == FP8_F32) acc = max(acc, reinterpret_cast<const uint32_t *>(x)[i] & 0x7FFFFFFFu);
+        else acc = __vmaxu2(acc, (uint32_t)reinterpret_cast<const uint16_t *>(x)[i] & 0x7FFFu);
+    }
+    uint32_t m = DT == FP8_F32 ? acc : max(acc & 0xFFFFu, acc >> 16);
+    m = __reduce_max_sync(0xFFFFFFFFu, m);
+    if ((threadIdx.x & 31) == 0) warp_max[threadIdx.x >> 5] = m;
+    __syncthreads();
+    if (threadIdx.x < 32) {
+        m = warp_max[threadIdx.x];
+        m = __reduce_max_sync(0xFFFFFFFFu, m);
+        if (threadIdx.x == 0) cta_max = m;
+    }
+    // every CTA's maximum becomes visible to the whole cluster, then each CTA folds all of them
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+    uint32_t total = 0;
+    for (uint32_t r = 0; r < nctas; ++r) {
+        uint32_t remote, val;
+        asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(smem_u32(&cta_max)), "r"(r));
+        asm volatile("ld.shared::cluster.u32 %0, [%1];" : "=r"(val) : "r"(remote) : "memory");
+        total = max(total, val);
+    }
+    uint32_t fbits;
+    if (DT == FP8_F32) fbits = total;
+    else if (DT == FP8_BF16) fbits = total << 16;
+    else { float f; asm("cvt.f32.f16 %0, %1;" : "=f"(f) : "h"((uint16_t)total)); fbits = __float_as_uint(f); }
+    unsigned flags = 0;
+    const int bias = bias_from_amax_bits(fbits, fmt, conv, margin, &flags);
+    if (rank == 0 && threadIdx.x == 0) {
+        *d_amax = __uint_as_float(fbits);
+        *d_bias = bias;
+        if (flags) atomicOr(d_status, flags);
+    }
+    const Pow2Pair p = make_pow2_pair(bias + delta);
+    bool sat = false;
+    // two input vectors (16-bit types) or four (fp32) make one 16-byte output vector
+    constexpr int kIn = InType<DT>::kBytes;
+#pragma unroll
+    for (int j = 0; j < kSmallVecs; ++j) {
+        const int64_t i = t0 + j * stride;
+        if (i >= nvec) continue;
+        const uint32_t *w = reinterpret_cast<const uint32_t *>(&v[j]);
+        uint8_t *dst = reinterpret_cast<uint8_t *>(y) + i * kPerVec;
+        if (kIn == 2) {
+            uint2 o;
+            o.x = cast4w<FMT, DT, true>(w, p, sat);
+            o.y = cast4w<FMT, DT, true>(w + kW, p, sat);
+            *reinterpret_cast<uint2 *>(dst) = o;
+        } else {
+            *reinterpret_cast<uint32_t *>(dst) = cast4w<FMT, DT, true>(w, p, sat);
+        }
+    }
+    if (rank == 0 && (int)threadIdx.x < ntail) {
+        const int64_t i = nvec * kPerVec + threadIdx.x;
+        reinterpret_cast<uint8_t *>(y)[i] = cast1<FMT, DT, true>(x, i, p, sat);
+    }
+    if (__syncthreads_or(sat) && threadIdx.x == 0) atomicOr(d_status, FP8_FLAG_SATURATED);
+    // no CTA may exit while a peer can still read its cta_max
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
+template <int FMT, int DT>
+static cudaError_t launch_small(fp8_ctx *ctx, const void *x, int64_t n, int conv, int margin, float *d_amax,
+                                int32_t *d_bias, uint8_t *y, cudaStream_t stream)
+{
+    constexpr int kPerVec = 16 / InType<DT>::kBytes;
+    const int64_t nvec = n / kPerVec;
+    const int ntail = (int)(n - nvec * kPerVec);
+    const int64_t per_cta = (int64_t)kSmallThreads * kSmallVecs;
+    int64_t want = (nvec + per_cta - 1) / per_cta;
+    if (want > kSmallMaxCtas) return cudaErrorNotSupported;
+    int ctas = 1;
+    while (ctas < want) ctas *= 2;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)ctas, 1, 1);
+    cfg.blockDim = dim3(kSmallThreads, 1, 1);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = (unsigned)ctas;
+    attr.val.clusterDim.y = 1;
+    attr.val.clusterDim.z = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, cast_small_kernel<FMT, DT>, reinterpret_cast<const uint4 *>(x),
+                              reinterpret_cast<uint4 *>(y), nvec, ntail, (int)FMT, conv, margin, format_delta(FMT, conv),
+                              d_amax, d_bias, ctx->d_status);
+}
+
+static cudaError_t launch_small_any(int fmt, int dt, fp8_ctx *ctx, const void *x, int64_t n, int conv, int margin,
+                                    float *d_amax, int32_t *d_bias, uint8_t *y, cudaStream_t st)
+{
+#define FP8LIN_SMALL(F, D) return launch_small<F, D>(ctx, x, n, conv, margin, d_amax, d_bias, y, st)
+    if (fmt == FP8_E4) {
+        if (dt == FP8_BF16) FP8LIN_SMALL(FP8_E4, FP8_BF16);
+        if (dt == FP8_F16) FP8LIN_SMALL(FP8_E4, FP8_F16);
+        FP8LIN_SMALL(FP8_E4, FP8_F32);
+    }
+    if (dt == FP8_BF16) FP8LIN_SMALL(FP8_E5, FP8_BF16);
+    if (dt == FP8_F16) FP8LIN_SMALL(FP8_E5, FP8_F16);
+    FP8LIN_SMALL(FP8_E5, FP8_F32);
+#undef FP8LIN_SMALL
+}
+
+static const bool g_no_small_cast = [] { const char *e = getenv("FP8LIN_NO_SMALL_CAST"); return e && e[0] == '1'; }();
+
 static fp8_status_t cast_entry(int fmt, fp8_ctx *ctx, const void *x, fp8_dtype_t x_dt, int64_t rows, int64_t cols,
                                int64_t ld, const int32_t *d_bias, fp8_conv_t conv, int32_t margin, float *d_amax_out,
                                int32_t *d_bias_out, uint8_t *y, uint8_t *y_t, void *stream)
@@ -335,7 +489,15 @@ static fp8_status_t cast_entry(int fmt, fp8_ctx *ctx, const void *x, fp8_dtype_t
     cudaStream_t st = (cudaStream_t)stream;
     const int32_t *bias = d_bias;
     if (!bias) {
-        // FP8-AMAX: amax + bias in one launch, the cast in a second
+        // FP8-AMAX.  Small contiguous tensors: one cluster holds the tensor in registers, one launch.
+        if (!y_t && ld == cols && (reinterpret_cast<uintptr_t>(x) & 15u) == 0 && (reinterpret_cast<uintptr_t>(y) & 7u) == 0 &&
+            !g_no_small_cast) {
+            cudaError_t se = launch_small_any(fmt, (int)x_dt, ctx, x, rows * cols, (int)conv, margin, d_amax_out,
+                                              d_bias_out, y, st);
+            if (se == cudaSuccess) return FP8_OK;
+            cudaGetLastError();   // too large for the register-resident kernel (or the launch was refused)
+        }
+        // Otherwise amax + bias in one launch, the cast in a second.
         if (launch_amax_bias(ctx, x, (int)x_dt, rows, cols, ld, d_amax_out, d_bias_out, fmt, (int)conv, margin, st) !=
             cudaSuccess)
             return FP8_ERR_CUDA;

@@ -325,3 +325,30 @@ def test_fused_amax_bias_cast_fp16_fp32(ctx, lib, dtype, kind):
         assert float(amax.item()) == a and int(bias.item()) == b
         assert_codes_equal(u8(y), want, O.native_format(kind))
         assert_codes_equal(u8(y_t), want_t, O.native_format(kind))
+
+
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float16, torch.float32])
+@pytest.mark.parametrize("shape", [(1, 5), (1, 8192), (16, 8192), (64, 8192), (129, 257), (3, 8), (512, 1024), (1024, 1024)])
+def test_fp8_amax_on_small_tensors_single_launch(ctx, lib, dtype, shape):
+    """Decode-size activations: the whole tensor is quantised by one cluster in one launch (row-major output,
+    FP8-AMAX); larger ones fall through to the two-launch path.  Same results either way."""
+    g = torch.Generator(device="cuda").manual_seed(shape[0] * 7 + shape[1])
+    for kind, std in ((O.E4, 1.0), (O.E5, 1e-4)):
+        x = (torch.randn(shape, generator=g, device="cuda") * std).to(dtype)
+        if shape[1] >= 8:
+            x[0, 3] = 100.0 * std   # an outlier decides the bias
+        host = bits_of(x) if dtype == torch.bfloat16 else _host(x)
+        a, b, want = O.quantise(host, kind, O.CONV_PAPER, 0)
+        amax = _dev_scalar(torch.float32, -1.0)
+        bias = _dev_scalar(torch.int32, 777)
+        y = torch.full((shape[0] * shape[1] + 32,), 0xEE, dtype=torch.uint8, device="cuda")
+        cast = ctx.cast_e4 if kind == O.E4 else ctx.cast_e5
+        cast(x, None, d_amax_out=amax, d_bias_out=bias, y=y)
+        assert float(amax.item()) == a and int(bias.item()) == b
+        n = shape[0] * shape[1]
+        assert_codes_equal(u8(y[:n]).reshape(shape), want, O.native_format(kind))
+        assert bool((y[n:] == 0xEE).all())
+    z = torch.zeros(shape, dtype=dtype, device="cuda")
+    ctx.device_flags(clear=True)
+    ctx.cast_e4(z, None, d_amax_out=amax, d_bias_out=bias, y=y)
+    assert float(amax.item()) == 0.0 and int(bias.item()) == 0 and ctx.device_flags() & lib.FLAG_ZERO_AMAX

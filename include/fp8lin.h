@@ -232,6 +232,18 @@ FP8_API fp8_status_t fp8_linear_dgrad(fp8_ctx *ctx, const uint8_t *dy8, const in
                               const uint8_t *w8_t, const int32_t *d_bw, void *dx, fp8_dtype_t dx_dt,
                               float *d_amax_dx, int64_t T, int64_t K, int64_t N, fp8_conv_t conv, void *stream);
 
+/* Input-gradient matmul with the activation's backward fused into the epilogue (no counterpart in the paper;
+ * the backward twin of fp8_linear_fwd_act).  With y_pre [T, K] the bf16 pre-activation that produced this
+ * layer's input (X = act(y_pre)):
+ *   dx      NULL, or out [T, K] bf16: the rounded input gradient dX
+ *   dx_act  out [T, K] bf16: bf16(dX) * act'(y_pre) in FP32, rounded -- the output gradient of the layer below
+ *   d_amax_act  NULL or out: its amax, so that the layer below quantises it in a single pass
+ * Operand rules as fp8_linear_dgrad; y_pre, dx, dx_act 16-byte aligned, K % 8 == 0. */
+FP8_API fp8_status_t fp8_linear_dgrad_act(fp8_ctx *ctx, const uint8_t *dy8, const int32_t *d_bg, const uint8_t *w8,
+                                          const uint8_t *w8_t, const int32_t *d_bw, const void *y_pre, void *dx,
+                                          void *dx_act, fp8_act_t act, float *d_amax_act, int64_t T, int64_t K,
+                                          int64_t N, fp8_conv_t conv, void *stream);
+
 /* Weight-gradient matmul (Section 2.2): dW[n, k] = (sum_t dY8[t, n] * X8[t, k]) * 2^-(s_g + s_x).
  *   dy8 [T, N] / dy8_t [N, T] E5 bytes, x8 [T, K] / x8_t [K, T] E4 bytes.
  *   Each operand in either layout (the transposed copy wins when both are

@@ -53,7 +53,9 @@ struct GemmParams {
     int64_t ldo;
     int vec_ok;                   // out 16-byte aligned and ldo*elem % 16 == 0
     int tma_out;                  // epilogue goes through shared memory and TMA stores (needs vec_ok)
-    int act;                      // 0: none; 1: GELU of the bf16-rounded output goes to a second tensor (out may be NULL)
+    int act;                      // 0: none; 1: GELU of the bf16-rounded output goes to a second tensor (out may be NULL);
+                                  // 2: the bf16-rounded output times GELU'(aux) goes to the second tensor
+    const void *aux;              // act == 2: [M, N] bf16, the pre-activation whose derivative scales the gradient
     unsigned *d_amax_bits;        // or NULL
     unsigned *d_status;
     uint32_t idesc;
@@ -301,6 +303,27 @@ __device__ __forceinline__ void gelu_words(const uint32_t (&w)[16], float (&v)[3
     }
 }
 
+// d/dx GELU(x) = Phi(x) + x * phi(x)
+__device__ __forceinline__ float gelu_grad_f32(float x)
+{
+    return 0.5f * erfcf(-0.70710678118654752f * x) + x * 0.3989422804014327f * __expf(-0.5f * x * x);
+}
+
+// 32 bf16 gradient values times GELU'(pre-activation), in FP32; `aux_row` points at the 32 pre-activations.
+__device__ __forceinline__ void gelu_backward_words(const uint32_t (&w)[16], const uint16_t *aux_row, bool ok,
+                                                    float (&v)[32])
+{
+    uint4 a[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) a[j] = ok ? __ldg(reinterpret_cast<const uint4 *>(aux_row) + j) : make_uint4(0, 0, 0, 0);
+    const uint32_t *aw = reinterpret_cast<const uint32_t *>(a);
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+        v[2 * i] = __uint_as_float(w[i] << 16) * gelu_grad_f32(__uint_as_float(aw[i] << 16));
+        v[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u) * gelu_grad_f32(__uint_as_float(aw[i] & 0xFFFF0000u));
+    }
+}
+
 // One warp's share (32 rows x BN columns) of a finished accumulator.
 //   t_row        TMEM address of this warp's lanes at the accumulator's first column
 //   row0         first of the warp's 32 output rows;  col_base  first output column of the tile
@@ -360,7 +383,22 @@ __device__ __forceinline__ void epilogue_tile(const CUtensorMap *map_out, const 
                     for (int j = 0; j < 4; ++j)
                         slab_write(slab_pre, lane, 4 * h + j, w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
                 }
-                gelu_words(w, v);  // the activation sees exactly what the pre-activation tensor holds
+                if (p.act == 1) {
+                    gelu_words(w, v);  // the activation sees exactly what the pre-activation tensor holds
+                } else {
+                    // columns beyond N are clipped by the store; rows beyond M have no pre-activation to read
+                    const bool ok = row_ok && col0 + 32 <= p.N;
+                    gelu_backward_words(w, reinterpret_cast<const uint16_t *>(p.aux) + (int64_t)(row0 + lane) * p.ldo + col0,
+                                        ok, v);
+                    if (row_ok && !ok && col0 < p.N) {   // ragged last chunk: element by element
+                        const uint16_t *ar = reinterpret_cast<const uint16_t *>(p.aux) + (int64_t)(row0 + lane) * p.ldo;
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) {
+                            const float g = (i & 1) ? __uint_as_float(w[i >> 1] & 0xFFFF0000u) : __uint_as_float(w[i >> 1] << 16);
+                            v[i] = col0 + i < p.N ? g * gelu_grad_f32(__uint_as_float((uint32_t)__ldg(ar + col0 + i) << 16)) : 0.0f;
+                        }
+                    }
+                }
                 pack_bf16(v, col0, p, wa, amax_bits, row_ok);
 #pragma unroll
                 for (int j = 0; j < 4; ++j)
@@ -914,7 +952,8 @@ static bool encode_map(fp8_ctx *ctx, CUtensorMap *map, const void *base, int64_t
 static fp8_status_t run_gemm(fp8_ctx *ctx, const uint8_t *a, int a_fmt, bool a_mn, const int32_t *d_ba,
                              const uint8_t *b, int b_fmt, bool b_mn, const int32_t *d_bb, int delta_sum,
                              const void *bias_vec, int bias_dt, void *out, int out_dt, float *d_amax_out, int64_t M,
-                             int64_t N, int64_t Kc, cudaStream_t st, int act = 0, void *out_act = nullptr)
+                             int64_t N, int64_t Kc, cudaStream_t st, int act = 0, void *out_act = nullptr,
+                             const void *aux = nullptr)
 {
     if (M > 0x7FFFFFFF / 2 || N > 0x7FFFFFFF / 2 || Kc > 0x7FFFFFFF / 2) return FP8_ERR_SHAPE;
     const bool pair = g_max_pairs > 0 && M > kBM && !g_force_single;
@@ -959,6 +998,7 @@ static fp8_status_t run_gemm(fp8_ctx *ctx, const uint8_t *a, int a_fmt, bool a_m
     p.vec_ok = ((reinterpret_cast<uintptr_t>(out) & 15u) == 0 && (N * esz) % 16 == 0) ? 1 : 0;
     p.tma_out = (p.vec_ok && !g_direct_epilogue) ? 1 : 0;
     p.act = act;
+    p.aux = aux;
     CUtensorMap map_out = map_a;  // placeholder when the staged epilogue is off (never dereferenced then)
     CUtensorMap map_out2 = map_a;
     auto encode_out = [&](CUtensorMap *m, void *base) {
@@ -1071,6 +1111,25 @@ fp8_status_t fp8_linear_dgrad(fp8_ctx *ctx, const uint8_t *dy8, const int32_t *d
     int delta = format_delta(FP8_E5, conv) + format_delta(FP8_E4, conv);
     return run_gemm(ctx, dy8, FP8_E5, false, d_bg, w, FP8_E4, w_mn, d_bw, delta, nullptr, 0, dx, dx_dt, d_amax_dx, T, K,
                     N, (cudaStream_t)stream);
+}
+
+fp8_status_t fp8_linear_dgrad_act(fp8_ctx *ctx, const uint8_t *dy8, const int32_t *d_bg, const uint8_t *w8,
+                                  const uint8_t *w8_t, const int32_t *d_bw, const void *y_pre, void *dx, void *dx_act,
+                                  fp8_act_t act, float *d_amax_act, int64_t T, int64_t K, int64_t N, fp8_conv_t conv,
+                                  void *stream)
+{
+    using namespace fp8lin;
+    if (!ctx || !dy8 || !d_bg || (!w8 && !w8_t) || !d_bw || !y_pre || !dx_act) return FP8_ERR_NULL;
+    if ((int)conv < 0 || (int)conv > 1 || (int)act != (int)FP8_ACT_GELU) return FP8_ERR_DTYPE;
+    if (T <= 0 || K <= 0 || N <= 0) return FP8_ERR_SHAPE;
+    const bool w_mn = (w8_t == nullptr);
+    const uint8_t *w = w_mn ? w8 : w8_t;
+    if (!aligned16(dy8) || !aligned16(w) || (N % 16) != 0 || (w_mn && (K % 16) != 0) || !aligned16(y_pre) ||
+        !aligned16(dx_act) || (dx && !aligned16(dx)) || (K % 8) != 0)
+        return FP8_ERR_ALIGN;
+    int delta = format_delta(FP8_E5, conv) + format_delta(FP8_E4, conv);
+    return run_gemm(ctx, dy8, FP8_E5, false, d_bg, w, FP8_E4, w_mn, d_bw, delta, nullptr, 0, dx, FP8_BF16, d_amax_act, T,
+                    K, N, (cudaStream_t)stream, 2, dx_act, y_pre);
 }
 
 fp8_status_t fp8_linear_wgrad(fp8_ctx *ctx, const uint8_t *dy8, const uint8_t *dy8_t, const int32_t *d_bg,

@@ -29,6 +29,7 @@ SYMBOLS = (
     "fp8_create", "fp8_destroy", "fp8_status_string", "fp8_device_flags", "fp8_amax", "fp8_scaling_bias",
     "fp8_scaling_bias_host", "fp8_cast_e4", "fp8_cast_e5", "fp8_ptq_weights", "fp8_linear_fwd", "fp8_linear_dgrad",
     "fp8_linear_wgrad", "fp8_amax_noalloc", "fp8_linear_fwd_act", "fp8_cast_predicted", "fp8_prediction_stats",
+    "fp8_linear_dgrad_act",
 )
 
 if not os.path.exists(LIB_PATH):
@@ -57,6 +58,7 @@ _lib.fp8_ptq_weights.argtypes = [_P, _P, c_int, c_int64, c_int64, c_int64, c_int
 _lib.fp8_linear_fwd.argtypes = [_P, _P, _P, _P, _P, _P, c_int, _P, c_int, _P, c_int64, c_int64, c_int64, c_int, _P]
 _lib.fp8_linear_fwd_act.argtypes = [_P, _P, _P, _P, _P, _P, c_int, _P, _P, c_int, _P, c_int64, c_int64, c_int64, c_int, _P]
 _lib.fp8_linear_dgrad.argtypes = [_P, _P, _P, _P, _P, _P, _P, c_int, _P, c_int64, c_int64, c_int64, c_int, _P]
+_lib.fp8_linear_dgrad_act.argtypes = [_P, _P, _P, _P, _P, _P, _P, _P, _P, c_int, _P, c_int64, c_int64, c_int64, c_int, _P]
 _lib.fp8_linear_wgrad.argtypes = [_P, _P, _P, _P, _P, _P, _P, _P, c_int, c_int64, c_int64, c_int64, c_int, _P]
 for _name in SYMBOLS:
     if _name != "fp8_status_string":
@@ -208,6 +210,14 @@ class Context:
         K = dx.shape[1]
         _check(_lib.fp8_linear_dgrad(self._h, _ptr(dy8), _ptr(d_bg), _ptr(w8), _ptr(w8_t), _ptr(d_bw), _ptr(dx),
                                      _DT[dx.dtype], _ptr(d_amax_dx), T, K, N, conv, _stream()), "fp8_linear_dgrad")
+
+    def linear_dgrad_act(self, dy8, d_bg, w8, w8_t, d_bw, y_pre, dx, dx_act, d_amax_act=None, act=ACT_GELU,
+                         conv=CONV_PAPER):
+        T, N = dy8.shape
+        K = dx_act.shape[1]
+        _check(_lib.fp8_linear_dgrad_act(self._h, _ptr(dy8), _ptr(d_bg), _ptr(w8), _ptr(w8_t), _ptr(d_bw), _ptr(y_pre),
+                                         _ptr(dx), _ptr(dx_act), act, _ptr(d_amax_act), T, K, N, conv, _stream()),
+               "fp8_linear_dgrad_act")
 
     def linear_wgrad(self, dy8, dy8_t, d_bg, x8, x8_t, d_bx, dw, T, conv=CONV_PAPER):
         N, K = dw.shape

@@ -20,7 +20,7 @@ import torch
 from . import inputs as I
 
 CONFIG_ID = 5
-fp8lin_E4, CONV_PAPER = 0, 0   # enum values of the C ABI (format E4, paper convention)
+fp8lin_E4, fp8lin_E5, CONV_PAPER = 0, 1, 0   # enum values of the C ABI (formats, paper convention)
 
 
 def step_input(x_base: torch.Tensor, step: int) -> torch.Tensor:
@@ -60,6 +60,7 @@ class Fp8Stack:
         self.w8t = [torch.empty((d, d), **u8) for _ in range(layers)]
         self.y = [torch.empty((tokens, d), dtype=torch.bfloat16, **dev) for _ in range(layers)]
         self.act = torch.empty((tokens, d), dtype=torch.bfloat16, **dev) if fused_activation else None
+        self.gact = torch.empty((tokens, d), dtype=torch.bfloat16, **dev) if fused_activation else None
         self.g8 = torch.empty((tokens, d), **u8)
         self.g8t = torch.empty((d, tokens), **u8)
         self.dx = torch.empty((tokens, d), dtype=torch.bfloat16, **dev)
@@ -97,13 +98,26 @@ class Fp8Stack:
         c = self.ctx
         out = self.y[self.L - 1].to(torch.float32)
         g = ((out - self.target.to(torch.float32)) * (2.0 / (self.T * self.d))).to(torch.bfloat16)
+        have_amax = False   # the previous input-gradient matmul already produced amax(g)
         for l in range(self.L - 1, -1, -1):
-            c.cast_e5(g, None, d_amax_out=self.amax[l, 2:3], d_bias_out=self.bias[l, 2:3], y=self.g8, y_t=self.g8t)
-            c.linear_dgrad(self.g8, self.bias[l, 2:3], None, self.w8t[l], self.bias[l, 0:1], self.dx)
+            if have_amax:
+                c.scaling_bias(self.amax[l, 2:3], fp8lin_E5, CONV_PAPER, 0, self.bias[l, 2:3])
+                c.cast_e5(g, self.bias[l, 2:3], y=self.g8, y_t=self.g8t)
+            else:
+                c.cast_e5(g, None, d_amax_out=self.amax[l, 2:3], d_bias_out=self.bias[l, 2:3], y=self.g8, y_t=self.g8t)
+            if self.fused and l > 0:
+                # dX * GELU'(Y[l-1]) and its amax come straight out of the matmul
+                c.linear_dgrad_act(self.g8, self.bias[l, 2:3], None, self.w8t[l], self.bias[l, 0:1], self.y[l - 1], None,
+                                   self.gact, d_amax_act=self.amax[l - 1, 2:3])
+            else:
+                c.linear_dgrad(self.g8, self.bias[l, 2:3], None, self.w8t[l], self.bias[l, 0:1], self.dx)
             c.linear_wgrad(None, self.g8t, self.bias[l, 2:3], None, self.x8t[l], self.bias[l, 1:2], self.dw, self.T)
             self.w32[l].add_(self.dw.to(torch.float32), alpha=-self.lr)
             if l > 0:
-                g = (self.dx.to(torch.float32) * gelu_grad_f32(self.y[l - 1])).to(torch.bfloat16)
+                if self.fused:
+                    g, have_amax = self.gact, True
+                else:
+                    g = (self.dx.to(torch.float32) * gelu_grad_f32(self.y[l - 1])).to(torch.bfloat16)
 
     def step(self, step: int) -> Dict[str, object]:
         x = step_input(self.x_base, step)

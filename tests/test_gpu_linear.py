@@ -143,6 +143,33 @@ def test_fwd_with_gelu_in_the_epilogue(ctx, lib, T, K, N):
         assert float(amax_act.item()) == float(y_act.float().abs().max().item())
 
 
+@pytest.mark.parametrize("T,K,N", [(256, 768, 768), (144, 272, 528), (64, 1024, 512), (400, 1040, 784)])
+def test_dgrad_with_gelu_backward_in_the_epilogue(ctx, lib, T, K, N):
+    """dX must meet the input-gradient bar; the second output must be bf16(dX) * GELU'(y_pre) (checked in float64
+    on the GPU's own dX bits and the given pre-activation), and the emitted amax the amax of what was written."""
+    from oracle import stack as OS
+    from helpers import bf16_ordinal
+    qx, qw, qg = _layer(ctx, T, K, N, O.CONV_PAPER, seed=777 + T)
+    y_pre = I.normal_bf16(T, K, 1.5, 11, 9, "cuda")
+    ref = O.linear_dgrad_np(qg.ref, qg.shift, qw.ref, qw.shift)
+    for want_dx, layout in ((True, "t"), (False, "t"), (True, "mn")):
+        dx = torch.full((T, K), float("nan"), dtype=torch.bfloat16, device="cuda") if want_dx else None
+        g = torch.full((T, K), float("nan"), dtype=torch.bfloat16, device="cuda")
+        amax_g = torch.full((1,), -1.0, dtype=torch.float32, device="cuda")
+        w8, w8t = (None, qw.y_t) if layout == "t" else (qw.y, None)
+        ctx.linear_dgrad_act(qg.y, qg.bias, w8, w8t, qw.bias, y_pre, dx, g, d_amax_act=amax_g)
+        assert ctx.device_flags(clear=True) & lib.FLAG_TIMEOUT == 0
+        if want_dx:
+            assert_bf16_within_one_ulp(bits_of(dx), ref)
+            want = OS.f64_to_bf16(OS.bf16_to_f64(bits_of(dx)) * OS.gelu_grad(bits_of(y_pre)))
+            d = np.abs(bf16_ordinal(bits_of(g)) - bf16_ordinal(want))
+            assert d.max() <= 1, d.max()
+            kept = bits_of(g)
+        else:
+            assert np.array_equal(bits_of(g), kept)
+        assert float(amax_g.item()) == float(g.float().abs().max().item())
+
+
 def test_dgrad_amax_and_margin(ctx, lib):
     T, K, N = 256, 384, 512
     qx, qw, qg = _layer(ctx, T, K, N, O.CONV_PAPER, seed=5, margin=3)

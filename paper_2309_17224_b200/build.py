@@ -33,7 +33,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
         return LIB
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
     tmp = LIB + f".{os.getpid()}.tmp"
-    cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + [
+    extra = os.environ.get("FP8LIN_NVCC_EXTRA", "").split()   # e.g. -DFP8LIN_PAIR_STAGES=5 for experiments
+    cmd = [nvcc] + NVCC_FLAGS + extra + (["-Xptxas", "-v"] if verbose else []) + [
         "-I", os.path.join(ROOT, "include"), "-I", CSRC, "-o", tmp] + sources()
     subprocess.check_call(cmd)
     os.replace(tmp, LIB)

@@ -35,7 +35,11 @@ constexpr int kUmmaK = 32;        // contraction elements per tcgen05.mma for 8-
 constexpr int kGemmThreads = 192;
 constexpr int kGroupM = 16;       // tile rasterisation: m-blocks per group
 constexpr int kSlabBytes = 32 * 128;            // epilogue staging: 32 rows x 128 bytes, what one warp stores at a time
-constexpr int kEpiBytes = 4 * 2 * kSlabBytes;   // four epilogue warps, two slabs each
+constexpr int kSingleSlabs = 2;                 // staging slabs per epilogue warp, single-CTA kernel
+#ifndef FP8LIN_PAIR_SLABS
+#define FP8LIN_PAIR_SLABS 2
+#endif
+constexpr int kPairSlabs = FP8LIN_PAIR_SLABS;   // ... and CTA-pair kernel
 
 struct GemmParams {
     int M, N, K;
@@ -159,7 +163,7 @@ struct GemmSmem {
     static constexpr int kBBytes = BN * kBK;
     static constexpr int kStageBytes = kABytes + kBBytes;
     static constexpr int kEpiOffset = STAGES * kStageBytes;
-    static constexpr int kBarOffset = kEpiOffset + kEpiBytes;
+    static constexpr int kBarOffset = kEpiOffset + 4 * kSingleSlabs * kSlabBytes;
     static constexpr int kNumBars = 2 * STAGES + 4;
     static constexpr int kTotal = kBarOffset + kNumBars * 8 + 16;
     static constexpr int kDynamic = kTotal + 1024;  // slack to align the base to 1024 B
@@ -278,9 +282,15 @@ __device__ __forceinline__ void slab_write(uint32_t slab, int lane, int j, uint3
     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
 // Before a slab is overwritten, the store issued from it two slabs ago must have read it.
+template <int NSLAB>
 __device__ __forceinline__ void slab_acquire(int lane)
 {
-    if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+    // the store issued from this slab NSLAB slabs ago must have read it: at most NSLAB - 1 stores may be pending
+    if (lane == 0) {
+        if (NSLAB == 2) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+        else if (NSLAB == 3) asm volatile("cp.async.bulk.wait_group.read 2;" ::: "memory");
+        else asm volatile("cp.async.bulk.wait_group.read 3;" ::: "memory");
+    }
     __syncwarp();
 }
 __device__ __forceinline__ void slab_publish(const CUtensorMap *map, uint32_t slab, int lane, int x, int y, bool in_range)
@@ -328,7 +338,7 @@ __device__ __forceinline__ void gelu_backward_words(const uint32_t (&w)[16], con
 //   t_row        TMEM address of this warp's lanes at the accumulator's first column
 //   row0         first of the warp's 32 output rows;  col_base  first output column of the tile
 //   release_bar  barrier to arrive on once the accumulator has been read (cluster address if remote)
-template <int BN, bool ACT>
+template <int BN, bool ACT, int NSLAB>
 __device__ __forceinline__ void epilogue_tile(const CUtensorMap *map_out, const CUtensorMap *map_out2, uint32_t t_row,
                                               int row0, int col_base,
                                               const GemmParams &p, const Pow2Pair sc, bool two_step,
@@ -421,9 +431,9 @@ __device__ __forceinline__ void epilogue_tile(const CUtensorMap *map_out, const 
             tmem_ld_x32(t_row + c + 32, r1);
             tmem_ld_wait();
             if (c + 64 >= BN) release();
-            const uint32_t slab = warp_slabs + (slab_count & 1u) * kSlabBytes;
+            const uint32_t slab = warp_slabs + (slab_count % NSLAB) * kSlabBytes;
             ++slab_count;
-            slab_acquire(lane);
+            slab_acquire<NSLAB>(lane);
             float v[32];
             uint32_t w[16];
             epilogue_values(r0, col_base + c, p, sc, two_step, v);
@@ -443,9 +453,9 @@ __device__ __forceinline__ void epilogue_tile(const CUtensorMap *map_out, const 
             tmem_ld_x32(t_row + c, r);
             tmem_ld_wait();
             if (c + 32 >= BN) release();
-            const uint32_t slab = warp_slabs + (slab_count & 1u) * kSlabBytes;
+            const uint32_t slab = warp_slabs + (slab_count % NSLAB) * kSlabBytes;
             ++slab_count;
-            slab_acquire(lane);
+            slab_acquire<NSLAB>(lane);
             float v[32];
             epilogue_values(r, col_base + c, p, sc, two_step, v);
             amax_f32(v, col_base + c, p, amax_bits, row_ok);
@@ -559,7 +569,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         const Pow2Pair sc = make_pow2_pair(e);
         const bool two_step = (e < -126 || e > 127);
         uint32_t amax_bits = 0, slab_count = 0;
-        const uint32_t warp_slabs = smem_base + L::kEpiOffset + q * 2 * kSlabBytes;
+        const uint32_t warp_slabs = smem_base + L::kEpiOffset + q * kSingleSlabs * kSlabBytes;
         uint32_t t = 0;
         // with split-K every item leaves its raw FP32 partial sum in the workspace; a second kernel finishes
         GemmParams pp = p;
@@ -582,7 +592,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             if (!__all_sync(0xFFFFFFFFu, ready)) break;
             tc_fence_after();
             const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + buf * BN;
-            epilogue_tile<BN, ACT>(&map_out, &map_out2, t_row, m_blk * kBM + q * 32, n_blk * BN, pp, p.splits > 1 ? sc_one : sc,
+            epilogue_tile<BN, ACT, kSingleSlabs>(&map_out, &map_out2, t_row, m_blk * kBM + q * 32, n_blk * BN, pp, p.splits > 1 ? sc_one : sc,
                               p.splits > 1 ? false : two_step, amax_bits, warp_slabs, slab_count, acc_empty_bar(buf),
                               false, lane);
         }
@@ -622,7 +632,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
 // and collects one arrival per epilogue warp of both CTAs.  None of the loads
 // is a multicast load.
 
-constexpr int kPairStages = 6;
+#ifndef FP8LIN_PAIR_STAGES
+#define FP8LIN_PAIR_STAGES 6
+#endif
+constexpr int kPairStages = FP8LIN_PAIR_STAGES;
 constexpr int kPairBN = 256;       // N of the pair tile (and of the instruction)
 constexpr int kPairHalfN = 128;    // B rows each CTA loads
 
@@ -631,7 +644,7 @@ struct PairSmem {
     static constexpr int kBBytes = kPairHalfN * kBK;
     static constexpr int kStageBytes = kABytes + kBBytes;
     static constexpr int kEpiOffset = kPairStages * kStageBytes;
-    static constexpr int kBarOffset = kEpiOffset + kEpiBytes;
+    static constexpr int kBarOffset = kEpiOffset + 4 * kPairSlabs * kSlabBytes;
     static constexpr int kNumBars = 2 * kPairStages + 4;
     static constexpr int kTotal = kBarOffset + kNumBars * 8 + 16;
     static constexpr int kDynamic = kTotal + 1024;
@@ -806,7 +819,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
         const Pow2Pair sc = make_pow2_pair(e);
         const bool two_step = (e < -126 || e > 127);
         uint32_t amax_bits = 0, slab_count = 0;
-        const uint32_t warp_slabs = smem_base + L::kEpiOffset + q * 2 * kSlabBytes;
+        const uint32_t warp_slabs = smem_base + L::kEpiOffset + q * kPairSlabs * kSlabBytes;
         const uint32_t leader_acc_empty0 = map_to_cta(acc_empty_bar(0), 0);
         uint32_t t = 0;
         for (int tile = pair_id; tile < num_tiles; tile += num_pairs, ++t) {
@@ -818,7 +831,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             if (!__all_sync(0xFFFFFFFFu, ready)) break;
             tc_fence_after();
             const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + buf * kPairBN;
-            epilogue_tile<kPairBN, ACT>(&map_out, &map_out2, t_row, m_blk * 256 + (int)rank * kBM + q * 32, n_blk * kPairBN, p, sc,
+            epilogue_tile<kPairBN, ACT, kPairSlabs>(&map_out, &map_out2, t_row, m_blk * 256 + (int)rank * kBM + q * 32, n_blk * kPairBN, p, sc,
                                    two_step, amax_bits, warp_slabs, slab_count, leader_acc_empty0 + 8u * buf, true, lane);
         }
         if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");

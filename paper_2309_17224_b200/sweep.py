@@ -16,6 +16,8 @@ from . import fp8lin
 
 
 def _time(fn, iters, pre=None):
+    fn()   # first launch of a kernel pays its one-time load
+    torch.cuda.synchronize()
     total = 0.0
     for _ in range(iters):
         if pre:

@@ -169,11 +169,20 @@ class Timers:
 
     def __init__(self):
         self.pairs = {"gemm": [], "amax_cast": []}
+        self.layers = {}   # layer name -> event pairs around the whole layer (quantisation + matmuls)
 
     def span(self, key):
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         self.pairs[key].append((a, b))
         return a, b
+
+    def layer_span(self, name):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        self.layers.setdefault(name, []).append((a, b))
+        return a, b
+
+    def layer_ms(self):
+        return {k: sum(a.elapsed_time(b) for a, b in v) / len(v) for k, v in self.layers.items()}
 
     def total_ms(self, key):
         return sum(a.elapsed_time(b) for a, b in self.pairs[key])
@@ -371,7 +380,12 @@ def main():
         # per-kernel event pairs on every eighth step only: they serialise the launches they bracket
         tm = timers if step % EVENT_EVERY == 0 else None
         for L in layers:
+            if tm is not None:
+                la, lb = tm.layer_span(L.name)
+                la.record()
             run_layer(ctx, L, tm)
+            if tm is not None:
+                lb.record()
     stop.record()
     barrier_sync(dist)
     clocks = sampler.stop() if sampler else None
@@ -547,6 +561,7 @@ def main():
                       "bytes_per_element": bytes_per_elem, "ms_per_step": cast_ms / sampled_steps,
                       "hbm_peak_gbs": peaks["hbm_gbs"],
                       "frac": cast_elems * bytes_per_elem / (cast_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]},
+        "layer_ms": {k: round(v, 4) for k, v in timers.layer_ms().items()},   # amax + cast + matmuls of one layer
         "with_bias_prediction": predicted,
         "with_cuda_graph": graphed,
         "gemm_ms_per_step": gemm_ms / sampled_steps,

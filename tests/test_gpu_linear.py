@@ -313,3 +313,29 @@ def test_llama70b_ptq_inference_layers(ctx, lib, layer, tokens):
     ref = O.linear_samples(O.FWD, qx.ref, O.N_E4, qx.shift, w8_rows, O.N_E4, b + 1, ti, ni)
     got = bits_of(y)[ti, rows[ni]]
     assert_bf16_within_one_ulp(got, ref)
+
+
+def test_fused_epilogue_argument_errors(ctx, lib):
+    b = torch.zeros(1, dtype=torch.int32, device="cuda")
+    x8 = torch.zeros((32, 64), dtype=torch.uint8, device="cuda")
+    w8 = torch.zeros((48, 64), dtype=torch.uint8, device="cuda")
+    y = torch.zeros((32, 48), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(lib.Fp8Error) as e:
+        ctx.linear_fwd_act(x8, b, w8, b, None, None)                       # the activated output is mandatory
+    assert e.value.status == lib.ERR_NULL
+    with pytest.raises(lib.Fp8Error) as e:
+        ctx.linear_fwd_act(x8, b, w8, b, None, y, act=7)                   # unknown activation
+    assert e.value.status == lib.ERR_DTYPE
+    w8_odd = torch.zeros((44, 64), dtype=torch.uint8, device="cuda")       # N = 44: rows of y not 16-byte multiples
+    y_odd = torch.zeros((32, 44), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(lib.Fp8Error) as e:
+        ctx.linear_fwd_act(x8, b, w8_odd, b, None, y_odd)
+    assert e.value.status == lib.ERR_ALIGN
+    g8 = torch.zeros((32, 48), dtype=torch.uint8, device="cuda")
+    dxa = torch.zeros((32, 64), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(lib.Fp8Error) as e:
+        ctx.linear_dgrad_act(g8, b, w8, None, b, None, None, dxa)          # no pre-activation given
+    assert e.value.status == lib.ERR_NULL
+    # a valid tiny call still works after the rejected ones
+    ctx.linear_fwd_act(x8, b, w8, b, None, y)
+    assert bool((y == 0).all()) and ctx.device_flags(clear=True) & lib.FLAG_TIMEOUT == 0

@@ -87,6 +87,13 @@ FP8_API const char *fp8_status_string(fp8_status_t status);
  * FP8_FLAG_TIMEOUT was set, else FP8_OK. */
 FP8_API fp8_status_t fp8_device_flags(fp8_ctx *ctx, void *stream, unsigned *flags, int clear);
 
+/* Failure-detection self-test (no counterpart in the paper).  Every wait inside the kernels is bounded; this
+ * call makes one run out on purpose, without any fault: a one-CTA kernel waits on a barrier that nothing will
+ * ever complete, gives up after limit_ns (1 .. 100 000 000), raises FP8_FLAG_TIMEOUT and returns normally.
+ * Returns FP8_OK when exactly that happened; fp8_device_flags then reports FP8_ERR_DEVICE_TIMEOUT until the flag
+ * is cleared, and the context stays usable.  Synchronises `stream`. */
+FP8_API fp8_status_t fp8_selftest_wait_expiry(fp8_ctx *ctx, uint64_t limit_ns, void *stream);
+
 /* amax = max(|x|) over the whole tensor (Eq. 3, first line).
  *   x       [rows, cols] with leading dimension ld (elements), dtype x_dt
  *           (FP8_BF16, FP8_F16 or FP8_F32)

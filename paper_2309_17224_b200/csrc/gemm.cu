@@ -886,6 +886,24 @@ __global__ void __launch_bounds__(256) splitk_finalize_kernel(const GemmParams p
     }
 }
 
+// A wait that nothing will ever satisfy, with a caller-chosen (short) limit: exercises the bounded-wait path --
+// expiry, sticky flag, orderly return -- without any fault.  One CTA, one mbarrier, no copies.
+__global__ void wait_expiry_probe_kernel(unsigned long long limit_ns, unsigned *d_status, unsigned *d_done)
+{
+    __shared__ __align__(8) unsigned long long bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&bar), 1);
+        abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    // every thread waits for a phase that no one completes
+    const bool ok = mbar_wait(smem_u32(&bar), 0u, &abort_flag, d_status, limit_ns);
+    __syncthreads();
+    if (threadIdx.x == 0) *d_done = ok ? 2u : 1u;   // 1: the wait gave up and the kernel returned normally
+}
+
 // ---------------------------------------------------------------------------
 // host side
 // ---------------------------------------------------------------------------
@@ -1084,6 +1102,22 @@ fp8_status_t fp8_linear_fwd(fp8_ctx *ctx, const uint8_t *x8, const int32_t *d_bx
     int delta = 2 * format_delta(FP8_E4, conv);
     return run_gemm(ctx, x8, FP8_E4, false, d_bx, w8, FP8_E4, false, d_bw, delta, bias_vec, bias_dt, y, y_dt, d_amax_y,
                     T, N, K, (cudaStream_t)stream);
+}
+
+fp8_status_t fp8_selftest_wait_expiry(fp8_ctx *ctx, uint64_t limit_ns, void *stream)
+{
+    using namespace fp8lin;
+    if (!ctx) return FP8_ERR_NULL;
+    if (limit_ns == 0 || limit_ns > 100ull * 1000ull * 1000ull) return FP8_ERR_SHAPE;   // at most 100 ms
+    cudaStream_t st = (cudaStream_t)stream;
+    unsigned *done = ctx->d_slots + (kReduceSlots - 1) * kSlotWords + 3;   // a word no reduction reads
+    wait_expiry_probe_kernel<<<1, 64, 0, st>>>((unsigned long long)limit_ns, ctx->d_status, done);
+    if (cudaGetLastError() != cudaSuccess) return FP8_ERR_CUDA;
+    unsigned host = 0;
+    if (cudaMemcpyAsync(&host, done, sizeof(host), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+        cudaMemsetAsync(done, 0, sizeof(unsigned), st) != cudaSuccess || cudaStreamSynchronize(st) != cudaSuccess)
+        return FP8_ERR_CUDA;
+    return host == 1u ? FP8_OK : FP8_ERR_CUDA;
 }
 
 fp8_status_t fp8_linear_fwd_act(fp8_ctx *ctx, const uint8_t *x8, const int32_t *d_bx, const uint8_t *w8,

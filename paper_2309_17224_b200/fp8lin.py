@@ -29,7 +29,7 @@ SYMBOLS = (
     "fp8_create", "fp8_destroy", "fp8_status_string", "fp8_device_flags", "fp8_amax", "fp8_scaling_bias",
     "fp8_scaling_bias_host", "fp8_cast_e4", "fp8_cast_e5", "fp8_ptq_weights", "fp8_linear_fwd", "fp8_linear_dgrad",
     "fp8_linear_wgrad", "fp8_amax_noalloc", "fp8_linear_fwd_act", "fp8_cast_predicted", "fp8_prediction_stats",
-    "fp8_linear_dgrad_act",
+    "fp8_linear_dgrad_act", "fp8_selftest_wait_expiry",
 )
 
 if not os.path.exists(LIB_PATH):
@@ -45,6 +45,7 @@ _lib.fp8_destroy.argtypes = [_P]
 _lib.fp8_status_string.argtypes = [c_int]
 _lib.fp8_status_string.restype = c_char_p
 _lib.fp8_device_flags.argtypes = [_P, _P, POINTER(c_uint), c_int]
+_lib.fp8_selftest_wait_expiry.argtypes = [_P, ctypes.c_uint64, _P]
 _lib.fp8_amax.argtypes = [_P, _P, c_int, c_int64, c_int64, c_int64, _P, _P]
 _lib.fp8_amax_noalloc.argtypes = [_P, c_int, c_int64, c_int64, c_int64, _P, _P]
 _lib.fp8_scaling_bias.argtypes = [_P, _P, c_int, c_int, c_int32, _P, _P]
@@ -139,6 +140,10 @@ class Context:
         if st not in (OK, ERR_DEVICE_TIMEOUT):
             _check(st, "fp8_device_flags")
         return flags.value
+
+    def selftest_wait_expiry(self, limit_ns: int = 1_000_000):
+        """Make one bounded device-side wait run out on purpose (raises FP8_FLAG_TIMEOUT, no fault)."""
+        _check(_lib.fp8_selftest_wait_expiry(self._h, ctypes.c_uint64(limit_ns), _stream()), "fp8_selftest_wait_expiry")
 
     # -- amax / bias ------------------------------------------------------------
     def amax(self, x, d_amax, rows=None, cols=None, ld=None):

@@ -1,8 +1,9 @@
 // amax (Eq. 3, first line) and the integer scaling bias (Eq. 3, second line).
 //
-// amax is a selection, not arithmetic: on bf16 bit patterns |x| orders like the
-// unsigned integer (bits & 0x7FFF), with NaN > inf > finite.  The kernel keeps
-// two 16-bit lanes per register (one packed max per 32-bit word), reduces by
+// amax is a selection, not arithmetic: on the bit patterns of bf16, fp16 and
+// fp32 alike |x| orders like the unsigned integer with the sign bit cleared,
+// with NaN > inf > finite.  For the 16-bit types the kernel keeps two lanes
+// per register (one packed max per 32-bit word); it reduces by
 // warp shuffle, then per block, then across the grid through one atomicMax per
 // block on a context-owned slot; the last block to arrive publishes the result
 // (and, when asked, the bias) and leaves the slot zeroed for the next call.

@@ -1,20 +1,22 @@
 // Scale-and-cast (Eq. 1 followed by the cast of Section 2.1; E5 per Section
 // 2.2) and post-training quantisation of a weight tensor (Section 3.1).
 //
-// code = RNE_fp8(x * 2^(bias + delta)), saturating.  The scaling is an exact
-// power-of-two multiply in FP32 (a bf16 value has 8 significant bits, so the
-// product is exact unless it underflows FP32, where the FP8 result is zero
+// code = RNE_fp8(x * 2^(bias + delta)), saturating.  The input (bf16, fp16 or
+// fp32) converts to FP32 exactly, the scaling is an exact power-of-two multiply
+// (the product is exact unless it underflows FP32, where the FP8 result is zero
 // either way) and the rounding is one hardware cvt.rn.satfinite per pair.
 //
-// Two kernels, both HBM-bound (2 B read + 1 B written per element and layout):
-//   cast_flat_kernel  contiguous tensor, row-major output only; 32 B in, 16 B
-//                     out per thread per step.
-//   cast_tile_kernel  128x128 tiles, optional row-major output and optional
-//                     transposed output staged through shared memory so that
-//                     both are written in 128-byte rows.
-// Both walk the tensor from its end to its start: when the amax pass has just
-// streamed the tensor front to back, the part most recently read is the part
-// most likely still in L2.
+// Kernels, all HBM-bound (2 B read per 16-bit element + 1 B written per element and layout):
+//   cast_flat_kernel       contiguous tensor, row-major output; 16 elements per thread per step.
+//   cast_tile_kernel       128x128 tiles, optional row-major output and optional transposed output
+//                          staged through shared memory so that both are written in 128-byte rows;
+//                          also the guarded path for ragged or strided tensors.
+//   cast_predicted_kernel  the flat cast with the amax of the same pass: FP8-AMAX in one pass when
+//                          the bias guess holds (fp8_cast_predicted), and delayed scaling.
+//   cast_small_kernel      decode-size tensors: one cluster keeps the tensor in registers between
+//                          its amax and its cast, one launch.
+// The flat and tile kernels walk the tensor from its end to its start: when the amax pass has just
+// streamed it front to back, the part most recently read is the part most likely still in L2.
 #include <cstdlib>
 
 #include "cast_common.cuh"

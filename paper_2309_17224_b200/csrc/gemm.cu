@@ -1,22 +1,34 @@
 // FP8 matmuls with the unscale folded into the epilogue (Fig. 3b, Eq. 2 for the
 // forward pass; Section 2.2 for the two backward matmuls).
 //
-// One persistent, warp-specialised kernel computes D[M,N] = A[M,K] * B[N,K]^T
-// with both operands contiguous along the contraction dimension:
-//   warp 0, one lane   TMA producer: 128x128-byte A boxes and BNx128-byte B
-//                      boxes (128-byte swizzle) into a ring of shared-memory
-//                      stages, completion signalled on an mbarrier per stage.
-//   warp 1, one lane   MMA issuer: tcgen05.mma.kind::f8f6f4 (M=128, N=BN,
-//                      K=32 per instruction) from shared-memory descriptors
-//                      into one of two FP32 accumulators in tensor memory;
-//                      tcgen05.commit releases the stage / publishes the tile.
+// D[M,N] = A * B^T over a contraction of length K, computed by one of two
+// persistent, warp-specialised kernels that share every building block:
+//
+//   gemm_pair_kernel  (M > 128)  two CTAs of a cluster own one 256x256 tile;
+//                     tcgen05.mma.cta_group::2, six stages of 32 KB per CTA.
+//   gemm_kernel       (M <= 128: decode, skinny)  one CTA owns a 128x256 tile,
+//                     four stages of 48 KB, optional split of the contraction.
+//
+// Roles in both:
+//   warp 0, one lane   TMA producer: 128-byte-swizzled boxes of A and B into a
+//                      ring of shared-memory stages, completion on an mbarrier.
+//   warp 1, one lane   MMA issuer: tcgen05.mma.kind::f8f6f4 (K = 32 per
+//                      instruction) from shared-memory descriptors into one of
+//                      two FP32 accumulators in tensor memory; tcgen05.commit
+//                      releases the stage / publishes the tile.
 //   warps 2..5         epilogue: tcgen05.ld of the finished accumulator (each
 //                      warp owns the 32 TMEM lanes it may address), exact
-//                      power-of-two unscale, optional bias vector, rounding to
-//                      the output type, optional amax of the rounded output.
+//                      power-of-two unscale, optional bias vector, rounding,
+//                      optional activation (second output) and amax, then
+//                      swizzled shared-memory slabs and TMA stores (or direct
+//                      stores for outputs whose rows are not 16-byte multiples).
 // The two accumulators let the epilogue of tile i overlap the main loop of
-// tile i+1.  A and B may be different FP8 formats (E5 x E4 in the backward
-// pass); the formats live in the instruction descriptor.
+// tile i+1.  An operand may be stored with the contraction index contiguous
+// ("K-major": X8[T,K], W8[N,K] in the forward pass) or with its M / N index
+// contiguous ("MN-major": the same buffers read by the backward matmuls); the
+// difference is the shared-memory descriptor and the order of the TMA
+// coordinates.  A and B may be different FP8 formats (E5 x E4 in the backward
+// pass); formats and majorness live in the instruction descriptor.
 //
 // Every wait on an mbarrier is bounded: when it expires the CTA raises
 // FP8_FLAG_TIMEOUT in the status word, all roles leave their loops, tensor

@@ -73,10 +73,12 @@ typedef enum { FP8_BF16 = 0, FP8_F16 = 1, FP8_F32 = 2 } fp8_dtype_t;
 
 typedef struct fp8_ctx fp8_ctx;
 
-/* Create / destroy a context on `device`.  The context owns a few KB of device
- * workspace (status word, reduction slots).  fp8_create is the only call that
- * allocates device memory; it also raises the dynamic shared-memory limit of
- * the matmul kernels.  It must not be called during stream capture. */
+/* Create / destroy a context on `device`.  The context owns its device
+ * workspace: a status word, reduction slots and a 64 MB FP32 buffer for the
+ * partial sums of split-contraction (decode-size) matmuls.  fp8_create is the
+ * only call that allocates device memory; it also raises the dynamic
+ * shared-memory limit of the matmul kernels.  It must not be called during
+ * stream capture; every other call may be captured into a CUDA graph. */
 FP8_API fp8_status_t fp8_create(fp8_ctx **ctx, int device);
 FP8_API fp8_status_t fp8_destroy(fp8_ctx *ctx);
 

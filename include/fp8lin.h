@@ -78,7 +78,10 @@ typedef struct fp8_ctx fp8_ctx;
  * partial sums of split-contraction (decode-size) matmuls.  fp8_create is the
  * only call that allocates device memory; it also raises the dynamic
  * shared-memory limit of the matmul kernels.  It must not be called during
- * stream capture; every other call may be captured into a CUDA graph. */
+ * stream capture.  The context-taking calls that enqueue work (fp8_amax,
+ * fp8_scaling_bias, fp8_cast_*, fp8_ptq_weights, fp8_linear_*) neither
+ * synchronise nor allocate, and bench.py replays a whole step of them from a
+ * CUDA graph. */
 FP8_API fp8_status_t fp8_create(fp8_ctx **ctx, int device);
 FP8_API fp8_status_t fp8_destroy(fp8_ctx *ctx);
 

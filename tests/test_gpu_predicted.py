@@ -121,3 +121,36 @@ def test_delayed_scaling_casts_with_the_given_bias_and_reports_the_next_one(ctx,
     ctx.cast_e4(x, bias_in, d_amax_out=amax, d_bias_out=bias_in, y=y, y_t=y_t)
     assert_codes_equal(u8(y), O.cast(xb, stale + 1, O.N_E4), O.N_E4)
     assert int(bias_in.item()) == b_true
+
+
+def test_config2_gradient_magnitude_moves_every_step(ctx, lib):
+    """Config 2: the output gradient of the QKV layer is redrawn every step with a log-uniform magnitude in
+    2^-12 .. 2^-4, so its E5 bias has to move.  At each of 16 steps amax and bias must equal the oracle's, the
+    bytes must match on sampled rows, both through the two-launch path and through the one-pass path (which
+    mostly mispredicts here and must still be exact)."""
+    from paper_2309_17224_b200 import inputs as I
+    wl = I.WORKLOADS["c2_gpt"]
+    T, N = wl.tokens, wl.layers[0].N
+    amax = torch.zeros(2, dtype=torch.float32, device="cuda")
+    bias = torch.zeros(2, dtype=torch.int32, device="cuda")
+    y = torch.empty((T, N), dtype=torch.uint8, device="cuda")
+    y2 = torch.empty((T, N), dtype=torch.uint8, device="cuda")
+    rng = np.random.default_rng(2)
+    seen = set()
+    ctx.prediction_stats(clear=True)
+    for step in range(16):
+        g = I.layer_tensors(wl, 0, device="cuda", step=step, want=("g",))["g"]
+        gb = bits_of(g)
+        a = O.amax(gb)
+        b = O.scaling_bias(a, O.E5)
+        seen.add(b)
+        ctx.cast_e5(g, None, d_amax_out=amax[0:1], d_bias_out=bias[0:1], y=y)
+        ctx.cast_predicted(lib.E5, g, amax[1:2], bias[1:2], y2)
+        assert amax.tolist() == [a, a] and bias.tolist() == [b, b], step
+        rows = np.sort(rng.choice(T, size=64, replace=False))
+        want = O.cast(gb[rows], b, O.N_E5)
+        assert_codes_equal(u8(y)[rows], want, O.N_E5)
+        assert torch.equal(y, y2)
+    hits, misses = ctx.prediction_stats(clear=True)
+    assert hits + misses == 16 and misses >= 8
+    assert len(seen) >= 5 and max(seen) - min(seen) >= 4

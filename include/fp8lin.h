@@ -193,6 +193,18 @@ FP8_API fp8_status_t fp8_cast_predicted(fp8_ctx *ctx, fp8_format_t fmt, const vo
  * context was created or the counters were last cleared. */
 FP8_API fp8_status_t fp8_prediction_stats(fp8_ctx *ctx, void *stream, unsigned *hits, unsigned *misses, int clear);
 
+/* Range statistics of a tensor under a given scaling bias, without casting it (for constant-bias sweeps as in
+ * Section 4 / Appendix F, FP8-CSCALE: which biases keep a tensor inside the FP8 range).
+ *   d_counts  out, four device uint64 (8-byte aligned), set by this call:
+ *             [0] elements that would be clipped to the format's maximum (infinities included)
+ *             [1] non-zero finite elements that would be flushed to zero
+ *             [2] elements that would land in the format's subnormal range
+ *             [3] non-zero finite elements of the tensor
+ *   NaNs are not counted anywhere.  x may be strided (ld) and of any of the three input types. */
+FP8_API fp8_status_t fp8_range_stats(fp8_ctx *ctx, fp8_format_t fmt, const void *x, fp8_dtype_t x_dt, int64_t rows,
+                                     int64_t cols, int64_t ld, const int32_t *d_bias, fp8_conv_t conv,
+                                     unsigned long long *d_counts, void *stream);
+
 /* Post-training quantisation of one weight tensor (Section 3.1): amax -> bias
  * -> cast to E4, once.  w [N, K] (ld elements); outputs w8 [N, K] and/or
  * w8_t [K, N], d_bw, d_amax_w (both required). */

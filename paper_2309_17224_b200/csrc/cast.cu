@@ -477,6 +477,44 @@ static cudaError_t launch_small_any(int fmt, int dt, fp8_ctx *ctx, const void *x
 #undef FP8LIN_SMALL
 }
 
+// ---------------------------------------------------------------------------
+// range statistics under a given bias
+// ---------------------------------------------------------------------------
+//
+// The constant-bias experiments (FP8-CSCALE, Section 4 and Appendix F) ask which biases keep a tensor inside
+// the FP8 range.  This kernel answers for one tensor and one bias without writing any bytes: how many elements
+// would be clipped to the maximum, how many non-zero elements would be flushed to zero, how many would land in
+// the subnormal range, out of how many non-zero finite elements.
+
+template <int FMT, int DT>
+__global__ void __launch_bounds__(256) range_stats_kernel(const void *__restrict__ x, int64_t rows, int64_t cols,
+                                                          int64_t ld, const int32_t *__restrict__ d_bias, int delta,
+                                                          unsigned long long *__restrict__ d_counts)
+{
+    const Pow2Pair p = make_pow2_pair(__ldg(d_bias) + delta);
+    constexpr uint32_t kMantMask = FMT == FP8_E4 ? 0x07u : 0x03u;
+    unsigned clipped = 0, flushed = 0, subnormal = 0, nonzero = 0;
+    for (int64_t r = blockIdx.x; r < rows; r += gridDim.x) {
+        for (int64_t c = threadIdx.x; c < cols; c += blockDim.x) {
+            const float xv = load1<DT>(x, r * ld + c);
+            if (xv != xv) continue;                       // NaN: neither in nor out of range
+            const bool finite_nz = xv != 0.0f && fabsf(xv) <= 3.402823466e38f;
+            nonzero += finite_nz;
+            const float v = xv * p.first * p.second;
+            const uint32_t code = cvt_pair<FMT>(0.0f, v) & 0x7Fu;
+            clipped += clips<FMT>(v);
+            flushed += finite_nz && code == 0u;
+            subnormal += code != 0u && (code & ~kMantMask) == 0u;
+        }
+    }
+    unsigned vals[4] = {clipped, flushed, subnormal, nonzero};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        unsigned v = __reduce_add_sync(0xFFFFFFFFu, vals[i]);
+        if ((threadIdx.x & 31) == 0 && v) atomicAdd(&d_counts[i], (unsigned long long)v);
+    }
+}
+
 static const bool g_no_small_cast = [] { const char *e = getenv("FP8LIN_NO_SMALL_CAST"); return e && e[0] == '1'; }();
 
 static fp8_status_t cast_entry(int fmt, fp8_ctx *ctx, const void *x, fp8_dtype_t x_dt, int64_t rows, int64_t cols,
@@ -599,6 +637,35 @@ fp8_status_t fp8_prediction_stats(fp8_ctx *ctx, void *stream, unsigned *hits, un
     *hits = host[0];
     *misses = host[1];
     return FP8_OK;
+}
+
+fp8_status_t fp8_range_stats(fp8_ctx *ctx, fp8_format_t fmt, const void *x, fp8_dtype_t x_dt, int64_t rows, int64_t cols,
+                             int64_t ld, const int32_t *d_bias, fp8_conv_t conv, unsigned long long *d_counts,
+                             void *stream)
+{
+    using namespace fp8lin;
+    if (!ctx || !x || !d_bias || !d_counts) return FP8_ERR_NULL;
+    if ((int)fmt < 0 || (int)fmt > 1 || (int)x_dt < 0 || (int)x_dt > 2 || (int)conv < 0 || (int)conv > 1)
+        return FP8_ERR_DTYPE;
+    if (rows <= 0 || cols <= 0 || ld < cols) return FP8_ERR_SHAPE;
+    if ((reinterpret_cast<uintptr_t>(x) & (x_dt == FP8_F32 ? 3u : 1u)) || (reinterpret_cast<uintptr_t>(d_counts) & 7u))
+        return FP8_ERR_ALIGN;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (cudaMemsetAsync(d_counts, 0, 4 * sizeof(unsigned long long), st) != cudaSuccess) return FP8_ERR_CUDA;
+    const int delta = format_delta((int)fmt, (int)conv);
+    const int blocks = (int)(rows < ctx->sm_count * 8 ? rows : ctx->sm_count * 8);
+#define FP8LIN_STATS(F, D) range_stats_kernel<F, D><<<blocks, 256, 0, st>>>(x, rows, cols, ld, d_bias, delta, d_counts)
+    if (fmt == FP8_E4) {
+        if (x_dt == FP8_BF16) FP8LIN_STATS(FP8_E4, FP8_BF16);
+        else if (x_dt == FP8_F16) FP8LIN_STATS(FP8_E4, FP8_F16);
+        else FP8LIN_STATS(FP8_E4, FP8_F32);
+    } else {
+        if (x_dt == FP8_BF16) FP8LIN_STATS(FP8_E5, FP8_BF16);
+        else if (x_dt == FP8_F16) FP8LIN_STATS(FP8_E5, FP8_F16);
+        else FP8LIN_STATS(FP8_E5, FP8_F32);
+    }
+#undef FP8LIN_STATS
+    return cudaGetLastError() == cudaSuccess ? FP8_OK : FP8_ERR_CUDA;
 }
 
 fp8_status_t fp8_ptq_weights(fp8_ctx *ctx, const void *w, fp8_dtype_t w_dt, int64_t N, int64_t K, int64_t ld,

@@ -29,7 +29,7 @@ SYMBOLS = (
     "fp8_create", "fp8_destroy", "fp8_status_string", "fp8_device_flags", "fp8_amax", "fp8_scaling_bias",
     "fp8_scaling_bias_host", "fp8_cast_e4", "fp8_cast_e5", "fp8_ptq_weights", "fp8_linear_fwd", "fp8_linear_dgrad",
     "fp8_linear_wgrad", "fp8_amax_noalloc", "fp8_linear_fwd_act", "fp8_cast_predicted", "fp8_prediction_stats",
-    "fp8_linear_dgrad_act", "fp8_selftest_wait_expiry",
+    "fp8_linear_dgrad_act", "fp8_selftest_wait_expiry", "fp8_range_stats",
 )
 
 if not os.path.exists(LIB_PATH):
@@ -55,6 +55,7 @@ _lib.fp8_cast_e4.argtypes = _cast_args
 _lib.fp8_cast_e5.argtypes = _cast_args
 _lib.fp8_cast_predicted.argtypes = [_P, c_int, _P, c_int, c_int64, c_int64, c_int64, c_int, c_int32, _P, _P, _P, _P]
 _lib.fp8_prediction_stats.argtypes = [_P, _P, POINTER(c_uint), POINTER(c_uint), c_int]
+_lib.fp8_range_stats.argtypes = [_P, c_int, _P, c_int, c_int64, c_int64, c_int64, _P, c_int, _P, _P]
 _lib.fp8_ptq_weights.argtypes = [_P, _P, c_int, c_int64, c_int64, c_int64, c_int, _P, _P, _P, _P, _P]
 _lib.fp8_linear_fwd.argtypes = [_P, _P, _P, _P, _P, _P, c_int, _P, c_int, _P, c_int64, c_int64, c_int64, c_int, _P]
 _lib.fp8_linear_fwd_act.argtypes = [_P, _P, _P, _P, _P, _P, c_int, _P, _P, c_int, _P, c_int64, c_int64, c_int64, c_int, _P]
@@ -187,6 +188,14 @@ class Context:
         _check(_lib.fp8_prediction_stats(self._h, _stream(), byref(hits), byref(misses), 1 if clear else 0),
                "fp8_prediction_stats")
         return hits.value, misses.value
+
+    def range_stats(self, fmt, x, d_bias, d_counts, conv=CONV_PAPER, rows=None, cols=None, ld=None):
+        """d_counts: 4 x int64 on the device = clipped, flushed to zero, subnormal, non-zero finite."""
+        rows = x.shape[0] if rows is None else rows
+        cols = x.shape[1] if cols is None else cols
+        ld = _ld(x) if ld is None else ld
+        _check(_lib.fp8_range_stats(self._h, fmt, _ptr(x), _DT[x.dtype], rows, cols, ld, _ptr(d_bias), conv,
+                                    _ptr(d_counts), _stream()), "fp8_range_stats")
 
     def ptq_weights(self, w, conv, w8, w8_t, d_bw, d_amax_w):
         _check(_lib.fp8_ptq_weights(self._h, _ptr(w), _DT[w.dtype], w.shape[0], w.shape[1], _ld(w), conv,

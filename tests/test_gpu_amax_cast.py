@@ -352,3 +352,35 @@ def test_fp8_amax_on_small_tensors_single_launch(ctx, lib, dtype, shape):
     ctx.device_flags(clear=True)
     ctx.cast_e4(z, None, d_amax_out=amax, d_bias_out=bias, y=y)
     assert float(amax.item()) == 0.0 and int(bias.item()) == 0 and ctx.device_flags() & lib.FLAG_ZERO_AMAX
+
+
+@pytest.mark.parametrize("kind", [O.E4, O.E5])
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+def test_range_statistics_of_a_constant_bias_sweep(ctx, lib, kind, dtype):
+    """FP8-CSCALE style sweep: for each candidate bias the counts of clipped / flushed / subnormal elements must
+    equal what the oracle's bytes say."""
+    g = torch.Generator(device="cuda").manual_seed(5 + kind)
+    x = (torch.randn((257, 383), generator=g, device="cuda") * 0.3).to(dtype)
+    x[0, :6] = torch.tensor([0.0, -0.0, float("inf"), float("-inf"), float("nan"), 1e-30], device="cuda").to(dtype)
+    host = bits_of(x) if dtype == torch.bfloat16 else _host(x)
+    xv = x.double().cpu().numpy()
+    fmt = O.native_format(kind)
+    m_bits = 3 if kind == O.E4 else 2
+    bias = _dev_scalar(torch.int32)
+    counts = torch.full((4,), 99, dtype=torch.int64, device="cuda")
+    results = {}
+    for b in (-12, -4, 0, 3, 8, 15, 24):
+        bias.fill_(b)
+        ctx.range_stats(kind, x, bias, counts)
+        s = b + O.delta(kind, O.CONV_PAPER)
+        codes = O.cast(host, s, fmt) & 0x7F
+        v = np.abs(np.ldexp(xv, s))
+        notnan = ~np.isnan(xv)
+        nz = notnan & np.isfinite(xv) & (xv != 0)
+        clipped = notnan & ((v > 464.0) if kind == O.E4 else (v >= 61440.0))
+        want = [int(clipped.sum()), int((nz & (codes == 0)).sum()),
+                int((notnan & (codes > 0) & (codes < (1 << m_bits))).sum()), int(nz.sum())]
+        assert counts.tolist() == want, (b, counts.tolist(), want)
+        results[b] = want
+    # the sweep shows the window: small biases flush, large ones clip
+    assert results[-12][1] > results[3][1] and results[24][0] > results[3][0]

@@ -513,6 +513,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    // The finalize kernel of a split contraction is launched as a programmatic dependent: its CTAs may take
+    // their places now and wait, at their first instruction, for this grid to complete and flush.
+    if (p.splits > 1) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     if (warp == 0) {
         if (lane == 0) {
@@ -867,29 +870,61 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
 
 // Second half of a split-K matmul: add the partial sums in a fixed order, then
 // the same unscale / bias / rounding / amax as the fused epilogue.
+// VEC = 4: four adjacent columns per thread through 16-byte loads (N a multiple of 4, output 16-byte aligned), all
+// of a thread's partial loads independent and in flight together; VEC = 1: any shape.
+template <int VEC>
 __global__ void __launch_bounds__(256) splitk_finalize_kernel(const GemmParams p)
 {
+    // launched as a programmatic dependent of the matmul kernel: nothing of that grid's output is read before this
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const int64_t total = (int64_t)p.M * p.N;
     const int e = -(__ldg(p.d_sa) + __ldg(p.d_sb) + p.delta_sum);
     const Pow2Pair sc = make_pow2_pair(e);
     uint32_t amax_bits = 0;
-    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
-        float acc = 0.0f;
-        for (int s = 0; s < p.splits; ++s) acc += __ldcs(p.partial + (int64_t)s * total + i);
-        float v = acc * sc.first * sc.second;
+    for (int64_t i = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * VEC; i < total;
+         i += (int64_t)gridDim.x * blockDim.x * VEC) {
+        float acc[VEC];
+#pragma unroll
+        for (int j = 0; j < VEC; ++j) acc[j] = 0.0f;
+#pragma unroll 8
+        for (int s = 0; s < p.splits; ++s) {
+            const float *src = p.partial + (int64_t)s * total + i;
+            if (VEC == 4) {
+                const float4 v = __ldcs(reinterpret_cast<const float4 *>(src));
+                acc[0] += v.x; acc[1 % VEC] += v.y; acc[2 % VEC] += v.z; acc[3 % VEC] += v.w;
+            } else {
+                acc[0] += __ldcs(src);
+            }
+        }
         const int col = (int)(i % p.N);
-        if (p.bias_vec)
-            v += p.bias_dt == FP8_F32
-                     ? __ldg(reinterpret_cast<const float *>(p.bias_vec) + col)
-                     : __uint_as_float((uint32_t)__ldg(reinterpret_cast<const uint16_t *>(p.bias_vec) + col) << 16);
-        if (p.out_dt == FP8_BF16) {
-            uint32_t w;
-            asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(w) : "f"(0.0f), "f"(v));
-            reinterpret_cast<uint16_t *>(p.out)[i] = (uint16_t)(w & 0xFFFFu);
-            amax_bits = max(amax_bits, (w & 0x7FFFu) << 16);
+        uint32_t h[VEC];
+#pragma unroll
+        for (int j = 0; j < VEC; ++j) {
+            float v = acc[j] * sc.first * sc.second;
+            if (p.bias_vec)
+                v += p.bias_dt == FP8_F32
+                         ? __ldg(reinterpret_cast<const float *>(p.bias_vec) + col + j)
+                         : __uint_as_float((uint32_t)__ldg(reinterpret_cast<const uint16_t *>(p.bias_vec) + col + j) << 16);
+            if (p.out_dt == FP8_BF16) {
+                uint32_t w;
+                asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(w) : "f"(0.0f), "f"(v));
+                h[j] = w & 0xFFFFu;
+                amax_bits = max(amax_bits, (w & 0x7FFFu) << 16);
+            } else {
+                h[j] = __float_as_uint(v);
+                amax_bits = max(amax_bits, h[j] & 0x7FFFFFFFu);
+            }
+        }
+        if (VEC == 4) {
+            if (p.out_dt == FP8_BF16)
+                *reinterpret_cast<uint2 *>(reinterpret_cast<uint16_t *>(p.out) + i) =
+                    make_uint2(h[0] | (h[1 % VEC] << 16), h[2 % VEC] | (h[3 % VEC] << 16));
+            else
+                *reinterpret_cast<uint4 *>(reinterpret_cast<float *>(p.out) + i) =
+                    make_uint4(h[0], h[1 % VEC], h[2 % VEC], h[3 % VEC]);
         } else {
-            reinterpret_cast<float *>(p.out)[i] = v;
-            amax_bits = max(amax_bits, __float_as_uint(v) & 0x7FFFFFFFu);
+            if (p.out_dt == FP8_BF16) reinterpret_cast<uint16_t *>(p.out)[i] = (uint16_t)h[0];
+            else reinterpret_cast<float *>(p.out)[i] = __uint_as_float(h[0]);
         }
     }
     if (p.d_amax_bits) {
@@ -1023,15 +1058,36 @@ static fp8_status_t run_gemm(fp8_ctx *ctx, const uint8_t *a, int a_fmt, bool a_m
     if (!pair && !g_no_splitk && !act) {
         const int64_t tiles = (int64_t)p.tiles_m * p.tiles_n;
         if (tiles < 2 * ctx->sm_count && p.num_k >= 8) {
-            int64_t want = (2 * ctx->sm_count + tiles - 1) / tiles;
-            int64_t by_k = p.num_k / 4;
-            int64_t by_ws = (int64_t)(ctx->partial_bytes / sizeof(float)) / (M * N);
-            int64_t sp = want < by_k ? want : by_k;
-            if (sp > by_ws) sp = by_ws;
-            if (sp > 1) {
-                p.kb_per_split = (int)((p.num_k + sp - 1) / sp);
-                p.splits = (p.num_k + p.kb_per_split - 1) / p.kb_per_split;
+            // Pick the split count by a byte model of the launch: the busiest CTA streams
+            // ceil(items / SMs) items of kb k-blocks each (one B tile of BN x 128 bytes per k-block; the A
+            // tile is a few rows), every split also writes and re-reads an FP32 partial tile, each item has
+            // a fixed set-up cost and splitting at all costs the finalize launch.  This avoids counts that
+            // leave the last wave nearly empty (448 items on 148 SMs) or move more partial sums than weights.
+            // (Dealing k-blocks evenly to the SMs, stream-K, was measured and lost to this: its extra partial
+            // tiles cost more than the imbalance it removes, because a thin last wave runs at more than its
+            // share of the HBM bandwidth.)
+            const int64_t by_k = p.num_k / 4;
+            const int64_t by_ws = (int64_t)(ctx->partial_bytes / sizeof(float)) / (M * N);
+            int64_t cap = by_k < by_ws ? by_k : by_ws;
+            if (cap > 64) cap = 64;
+            const double sms = (double)ctx->sm_count;
+            const double kb_bytes = (double)kBN * kBK, item_bytes = 24.0e3, finalize_bytes = 24.0e6;
+            double best = 0;
+            int64_t best_kb = p.num_k;
+            for (int64_t sp = 1; sp <= cap; ++sp) {
+                const int64_t kb = (p.num_k + sp - 1) / sp;
+                const int64_t real = (p.num_k + kb - 1) / kb;
+                if (real != sp) continue;
+                const int64_t waves = (tiles * real + ctx->sm_count - 1) / ctx->sm_count;
+                double cost = (double)waves * sms * ((double)kb * kb_bytes + item_bytes);
+                if (real > 1) cost += 8.0 * (double)real * (double)M * (double)N + finalize_bytes;
+                if (sp == 1 || cost < best) {
+                    best = cost;
+                    best_kb = kb;
+                }
             }
+            p.kb_per_split = (int)best_kb;
+            p.splits = (p.num_k + p.kb_per_split - 1) / p.kb_per_split;
         }
     }
     p.d_sa = d_ba; p.d_sb = d_bb; p.delta_sum = delta_sum;
@@ -1083,10 +1139,22 @@ static fp8_status_t run_gemm(fp8_ctx *ctx, const uint8_t *a, int a_fmt, bool a_m
                 map_a, map_b, map_out, map_out2, p);
         if (p.splits > 1) {
             if (cudaGetLastError() != cudaSuccess) return FP8_ERR_CUDA;
-            int64_t total = M * N;
-            int blocks = (int)((total + 255) / 256);
-            if (blocks > ctx->sm_count * 8) blocks = ctx->sm_count * 8;
-            splitk_finalize_kernel<<<blocks, 256, 0, st>>>(p);
+            const bool vec = p.vec_ok && (N % 4) == 0;
+            int64_t threads = vec ? M * N / 4 : M * N;
+            int64_t blocks = (threads + 255) / 256;
+            if (blocks > (int64_t)ctx->sm_count * 16) blocks = (int64_t)ctx->sm_count * 16;
+            cudaLaunchAttribute attr[1];
+            attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+            attr[0].val.programmaticStreamSerializationAllowed = 1;
+            cudaLaunchConfig_t cfg = {};
+            cfg.gridDim = dim3((unsigned)blocks);
+            cfg.blockDim = dim3(256);
+            cfg.stream = st;
+            cfg.attrs = attr;
+            cfg.numAttrs = 1;
+            cudaError_t le = vec ? cudaLaunchKernelEx(&cfg, splitk_finalize_kernel<4>, p)
+                                 : cudaLaunchKernelEx(&cfg, splitk_finalize_kernel<1>, p);
+            if (le != cudaSuccess) return FP8_ERR_CUDA;
         }
     }
     return cudaGetLastError() == cudaSuccess ? FP8_OK : FP8_ERR_CUDA;

@@ -255,10 +255,13 @@ def test_full_size_layers_sampled(ctx, lib, wl_name, layer):
         assert_bf16_within_one_ulp(got, ref)
 
 
-@pytest.mark.parametrize("T,K,N", [(1, 2048, 768), (16, 4096, 1280), (64, 8192, 512), (100, 1024, 2304)])
+@pytest.mark.parametrize("T,K,N", [(1, 2048, 768), (16, 4096, 1280), (64, 8192, 512), (100, 1024, 2304),
+                                   (5, 2064, 784), (128, 4096, 4096), (3, 16384, 272), (33, 1024, 18944), (9, 2048, 786)])
 def test_decode_shapes_split_k(ctx, lib, T, K, N):
-    """Few tokens, long contraction: the library splits the contraction across
-    CTAs and finishes in a second kernel; results must meet the same bars."""
+    """Few tokens, long contraction: the library deals the k-blocks of all output
+    tiles evenly to the SMs and finishes in a second kernel; results must meet
+    the same bars (ragged last k-block, ragged last tile, tiles cut in two and
+    in many pieces included)."""
     x = I.normal_bf16(T, K, 1.0, 31, 1, "cuda", outlier_frac=0.005, outlier_scale=100.0)
     w = I.normal_bf16(N, K, 0.015, 31, 2, "cuda")
     qx, qw = Quantised(ctx, x, O.E4, O.CONV_PAPER), Quantised(ctx, w, O.E4, O.CONV_PAPER)
@@ -279,6 +282,20 @@ def test_decode_shapes_split_k(ctx, lib, T, K, N):
             assert_gemm_close(y.cpu().numpy(), ref_b)
         else:
             assert_bf16_within_one_ulp(bits_of(y), ref_b)
+    assert ctx.device_flags(clear=True) & lib.FLAG_TIMEOUT == 0
+
+
+@pytest.mark.parametrize("T,N,K", [(16, 4096, 1024), (2, 8208, 528)])
+def test_decode_shapes_dgrad_from_row_major_weights(ctx, lib, T, N, K):
+    """The same split contraction with the weight read in its forward layout
+    (contraction index strided) and an E5 gradient operand."""
+    g = I.normal_bf16(T, N, 1e-3, 37, 1, "cuda")
+    w = I.normal_bf16(N, K, 0.02, 37, 2, "cuda")
+    qg, qw = Quantised(ctx, g, O.E5, O.CONV_PAPER), Quantised(ctx, w, O.E4, O.CONV_PAPER)
+    ref = O.linear_dgrad(qg.ref, qg.shift, qw.ref, qw.shift)
+    dx = torch.full((T, K), float("nan"), dtype=torch.float32, device="cuda")
+    ctx.linear_dgrad(qg.y, qg.bias, qw.y, None, qw.bias, dx)
+    assert_gemm_close(dx.cpu().numpy(), ref)
     assert ctx.device_flags(clear=True) & lib.FLAG_TIMEOUT == 0
 
 

@@ -238,7 +238,7 @@ FP8_API fp8_status_t fp8_linear_fwd(fp8_ctx *ctx, const uint8_t *x8, const int32
  *   d_amax_act  NULL or out: amax of y_act; fp8_scaling_bias + fp8_cast_e4 with
  *          that bias then quantise y_act in a single pass
  * Needs 16-byte aligned y_pre / y_act and N % 8 == 0, besides fp8_linear_fwd's rules. */
-typedef enum { FP8_ACT_GELU = 1 } fp8_act_t;
+typedef enum { FP8_ACT_NONE = 0, FP8_ACT_GELU = 1 } fp8_act_t;
 FP8_API fp8_status_t fp8_linear_fwd_act(fp8_ctx *ctx, const uint8_t *x8, const int32_t *d_bx, const uint8_t *w8,
                                         const int32_t *d_bw, const void *bias_vec, fp8_dtype_t bias_dt, void *y_pre,
                                         void *y_act, fp8_act_t act, float *d_amax_act, int64_t T, int64_t K, int64_t N,
@@ -267,6 +267,35 @@ FP8_API fp8_status_t fp8_linear_dgrad_act(fp8_ctx *ctx, const uint8_t *dy8, cons
                                           const uint8_t *w8_t, const int32_t *d_bw, const void *y_pre, void *dx,
                                           void *dx_act, fp8_act_t act, float *d_amax_act, int64_t T, int64_t K,
                                           int64_t N, fp8_conv_t conv, void *stream);
+
+/* Matmuls whose result leaves already quantised, for a bias known before the
+ * launch (no counterpart in the paper beyond Section 3's remark that a scale may
+ * rely on the history of amax instead of a second pass over memory: here the
+ * consumer's FP8 bytes are written by the producer's epilogue, and the amax that
+ * feeds the history comes out of the same launch).  The 16-bit tensor z the
+ * bytes are made from is
+ *   fp8_linear_fwd_q:   z = bf16(Y) for FP8_ACT_NONE, z = bf16(GELU(bf16(Y))) for FP8_ACT_GELU,
+ *                       Y as in fp8_linear_fwd;  z8 = E4 bytes of z under bias *d_bz
+ *   fp8_linear_dgrad_q: z = bf16(dX) for FP8_ACT_NONE, z = bf16(bf16(dX) * GELU'(y_pre)) for FP8_ACT_GELU,
+ *                       dX as in fp8_linear_dgrad;  g8 = E5 bytes of z under bias *d_bq
+ * and the bytes are exactly what fp8_cast_e4 / fp8_cast_e5 with that bias give on
+ * the stored z (FP8_FLAG_SATURATED is raised likewise when a value clips).
+ *   y_pre (fwd)   NULL, or out [T, N] bf16 pre-activation; must be NULL with FP8_ACT_NONE
+ *   y_pre (dgrad) in [T, K] bf16 pre-activation, required with FP8_ACT_GELU, NULL otherwise
+ *   dx            NULL, or out [T, K] bf16 rounded dX; must be NULL with FP8_ACT_NONE
+ *   z / g         NULL, or out bf16: the tensor the bytes are made from
+ *   z8 / g8       out bytes, [T, N] / [T, K], 16-byte aligned; N % 16 == 0 (fwd), K % 16 == 0 (dgrad)
+ *   d_bz / d_bq   in: device int32, paper-convention bias to quantise with (the caller's prediction)
+ *   d_amax_z / d_amax_g  NULL or out: amax of z, from which the caller updates its prediction
+ * Other operands as in fp8_linear_fwd / fp8_linear_dgrad; 16-bit outputs 16-byte aligned. */
+FP8_API fp8_status_t fp8_linear_fwd_q(fp8_ctx *ctx, const uint8_t *x8, const int32_t *d_bx, const uint8_t *w8,
+                                      const int32_t *d_bw, const void *bias_vec, fp8_dtype_t bias_dt, fp8_act_t act,
+                                      void *y_pre, void *z, uint8_t *z8, const int32_t *d_bz, float *d_amax_z,
+                                      int64_t T, int64_t K, int64_t N, fp8_conv_t conv, void *stream);
+FP8_API fp8_status_t fp8_linear_dgrad_q(fp8_ctx *ctx, const uint8_t *dy8, const int32_t *d_bg, const uint8_t *w8,
+                                        const uint8_t *w8_t, const int32_t *d_bw, fp8_act_t act, const void *y_pre,
+                                        void *dx, void *g, uint8_t *g8, const int32_t *d_bq, float *d_amax_g,
+                                        int64_t T, int64_t K, int64_t N, fp8_conv_t conv, void *stream);
 
 /* Weight-gradient matmul (Section 2.2): dW[n, k] = (sum_t dY8[t, n] * X8[t, k]) * 2^-(s_g + s_x).
  *   dy8 [T, N] / dy8_t [N, T] E5 bytes, x8 [T, K] / x8_t [K, T] E4 bytes.

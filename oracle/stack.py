@@ -44,11 +44,24 @@ def gelu_grad(y_bits: np.ndarray) -> np.ndarray:
 
 
 class OracleStack:
-    def __init__(self, w_bits, x_base_bits, target_bits, lr=1e-3):
+    def __init__(self, w_bits, x_base_bits, target_bits, lr=1e-3, history=False, margin=0):
+        """history: quantise every activation and gradient with the bias of Eq. 3 for that tensor's amax at the
+        previous step, minus `margin` (the amax-history remedy of Section 3); weights, and every tensor at the
+        first step, take the just-in-time bias."""
         self.w32 = [bf16_to_f64(w).astype(np.float32) for w in w_bits]
         self.x_base, self.target = x_base_bits, bf16_to_f64(target_bits)
         self.L = len(w_bits)
         self.lr = lr
+        self.history, self.margin = history, margin
+        self.prev_amax = None
+
+    def _quantise(self, bits, kind, l, j):
+        """(amax, bias used, bytes) of tensor j (1: activation, 2: gradient) of layer l."""
+        if not self.history or self.prev_amax is None:
+            return O.quantise(bits, kind)
+        a = O.amax(bits)
+        b = O.scaling_bias(float(self.prev_amax[l, j]), kind, O.CONV_PAPER, self.margin)
+        return a, b, O.cast(bits, b + O.delta(kind, O.CONV_PAPER), O.native_format(kind))
 
     def step(self, step: int):
         """One training step.  Returns a record of every tensor a linear saw."""
@@ -60,7 +73,7 @@ class OracleStack:
         for l in range(L):
             w = f64_to_bf16(self.w32[l].astype(np.float64))
             aw, bw, w8 = O.quantise(w, O.E4)
-            ax, bx, x8 = O.quantise(x, O.E4)
+            ax, bx, x8 = self._quantise(x, O.E4, l, 1)
             y = O.linear_fwd_np(x8, bx + 1, w8, bw + 1)
             rec["x"].append(x); rec["w"].append(w); rec["x8"].append(x8); rec["w8"].append(w8); rec["y"].append(y)
             rec["bias"][l, 0], rec["bias"][l, 1] = bw, bx
@@ -71,7 +84,7 @@ class OracleStack:
         rec["loss"] = float(np.mean((out - self.target) ** 2))
         g = f64_to_bf16((out - self.target) * (2.0 / (T * d)))
         for l in range(L - 1, -1, -1):
-            ag, bg, g8 = O.quantise(g, O.E5)
+            ag, bg, g8 = self._quantise(g, O.E5, l, 2)
             bw, bx = int(rec["bias"][l, 0]), int(rec["bias"][l, 1])
             dx = O.linear_dgrad_np(g8, bg, rec["w8"][l], bw + 1)
             dw = O.linear_wgrad_np(g8, bg, rec["x8"][l], bx + 1)
@@ -80,4 +93,5 @@ class OracleStack:
             self.w32[l] = (self.w32[l].astype(np.float64) - self.lr * bf16_to_f64(dw.bf16)).astype(np.float32)
             if l > 0:
                 g = f64_to_bf16(bf16_to_f64(dx.bf16) * gelu_grad(rec["y"][l - 1].bf16))
+        self.prev_amax = rec["amax"].copy()
         return rec

@@ -38,6 +38,7 @@
 
 #include "fp8lin_internal.cuh"
 #include "ptx.cuh"
+#include "cast_common.cuh"
 
 namespace fp8lin {
 
@@ -48,6 +49,7 @@ constexpr int kGemmThreads = 192;
 constexpr int kGroupM = 16;       // tile rasterisation: m-blocks per group
 constexpr int kSlabBytes = 32 * 128;            // epilogue staging: 32 rows x 128 bytes, what one warp stores at a time
 constexpr int kSingleSlabs = 2;                 // staging slabs per epilogue warp, single-CTA kernel
+constexpr int kActSlabs = 4;                    // ... of the kernels with a second output: two {output, z} pairs
 #ifndef FP8LIN_PAIR_SLABS
 #define FP8LIN_PAIR_SLABS 2
 #endif
@@ -69,9 +71,14 @@ struct GemmParams {
     int64_t ldo;
     int vec_ok;                   // out 16-byte aligned and ldo*elem % 16 == 0
     int tma_out;                  // epilogue goes through shared memory and TMA stores (needs vec_ok)
-    int act;                      // 0: none; 1: GELU of the bf16-rounded output goes to a second tensor (out may be NULL);
-                                  // 2: the bf16-rounded output times GELU'(aux) goes to the second tensor
+    int act;                      // 0: plain epilogue.  Otherwise a second tensor z leaves with the output (out may be
+                                  // NULL): 1: z = GELU of the bf16-rounded output; 2: z = the bf16-rounded output times
+                                  // GELU'(aux); 3: z = the bf16-rounded output itself
     const void *aux;              // act == 2: [M, N] bf16, the pre-activation whose derivative scales the gradient
+    int has_out2;                 // z is stored as bf16 through the second output map
+    uint8_t *out8;                // or NULL: z also leaves as FP8 bytes [M, N], scaled by a bias known beforehand
+    const int32_t *d_sq;          // ... that bias (paper convention, device memory)
+    int q_fmt, delta_q;           // ... the format of the bytes and its shift
     unsigned *d_amax_bits;        // or NULL
     unsigned *d_status;
     uint32_t idesc;
@@ -169,13 +176,14 @@ __host__ __device__ inline uint32_t make_idesc(int a_fmt, int b_fmt, int n)
 // kernel
 // ---------------------------------------------------------------------------
 
-template <int BN, int STAGES>
+template <int BN, int STAGES, int SLABS = kSingleSlabs>
 struct GemmSmem {
+    static constexpr int kSlabs = SLABS;  // staging slabs per epilogue warp
     static constexpr int kABytes = kBM * kBK;
     static constexpr int kBBytes = BN * kBK;
     static constexpr int kStageBytes = kABytes + kBBytes;
     static constexpr int kEpiOffset = STAGES * kStageBytes;
-    static constexpr int kBarOffset = kEpiOffset + 4 * kSingleSlabs * kSlabBytes;
+    static constexpr int kBarOffset = kEpiOffset + 4 * SLABS * kSlabBytes;
     static constexpr int kNumBars = 2 * STAGES + 4;
     static constexpr int kTotal = kBarOffset + kNumBars * 8 + 16;
     static constexpr int kDynamic = kTotal + 1024;  // slack to align the base to 1024 B
@@ -224,11 +232,18 @@ __device__ __forceinline__ void pack_bf16(const float (&v)[32], int col0, const 
 #pragma unroll
     for (int i = 0; i < 16; ++i) asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(w[i]) : "f"(v[2 * i + 1]), "f"(v[2 * i]));
     if (p.d_amax_bits && row_ok) {
+        if (col0 + 32 <= p.N) {  // whole chunk inside the tensor: both 16-bit lanes of a word at once
+            uint32_t m2 = 0;
 #pragma unroll
-        for (int i = 0; i < 16; ++i) {
-            uint32_t a = w[i] & 0x7FFF7FFFu;
-            if (col0 + 2 * i < p.N) amax_bits = max(amax_bits, (a & 0xFFFFu) << 16);
-            if (col0 + 2 * i + 1 < p.N) amax_bits = max(amax_bits, a & 0xFFFF0000u);
+            for (int i = 0; i < 16; ++i) m2 = __vmaxu2(m2, w[i] & 0x7FFF7FFFu);
+            amax_bits = max(amax_bits, max(m2 & 0xFFFFu, m2 >> 16) << 16);
+        } else {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                uint32_t a = w[i] & 0x7FFF7FFFu;
+                if (col0 + 2 * i < p.N) amax_bits = max(amax_bits, (a & 0xFFFFu) << 16);
+                if (col0 + 2 * i + 1 < p.N) amax_bits = max(amax_bits, a & 0xFFFF0000u);
+            }
         }
     }
 }
@@ -279,6 +294,14 @@ __device__ __forceinline__ void store_direct(const uint32_t (&r)[32], int row, i
 
 // ---- staged epilogue: registers -> swizzled shared memory -> TMA store ----
 
+__device__ __forceinline__ void tma_store_only(const CUtensorMap *map, uint32_t src, int x, int y)
+{
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%2, %3}], [%1];" ::"l"(
+                     reinterpret_cast<uint64_t>(map)),
+                 "r"(src), "r"(x), "r"(y)
+                 : "memory");
+}
+// ... followed by its own commit: one bulk group per store
 __device__ __forceinline__ void tma_store_2d(const CUtensorMap *map, uint32_t src, int x, int y)
 {
     asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%2, %3}], [%1];" ::"l"(
@@ -312,8 +335,37 @@ __device__ __forceinline__ void slab_publish(const CUtensorMap *map, uint32_t sl
     if (lane == 0 && in_range) tma_store_2d(map, slab, x, y);
 }
 
-// GELU(x) = x/2 * erfc(-x / sqrt 2); erfc keeps relative accuracy in the negative tail.
-__device__ __forceinline__ float gelu_f32(float x) { return 0.5f * x * erfcf(-0.70710678118654752f * x); }
+// Phi(x), the standard normal distribution function, and exp(-x^2 / 2), in about twenty FP32 instructions (the
+// epilogue runs on four warps, so its instruction count is what bounds the fused kernels).
+//   Phi(-|x|) = erfcx(z) / 2 * exp(-z^2),  z = |x| / sqrt 2,  erfcx(z) = exp(z^2) erfc(z) = t * Q(t),  t = 1 / (1 + z/2)
+// Q is a degree-7 polynomial, a Chebyshev least-squares fit of erfcx(z)/t over t in (0, 1] (all z >= 0) with
+// relative error below 5e-6 -- relative, so that the far negative tail of GELU keeps its accuracy -- and
+// Phi(x) = 1 - Phi(-x) for x > 0.  Rounded to bf16, x * Phi(x) differs from the correctly rounded GELU by at most
+// one bf16 ulp (at 0.2 % of all bf16 inputs), and Phi(x) + x * phi(x) stays within 1e-4 relative of GELU'.
+__device__ __forceinline__ void normal_cdf(float x, float &cdf, float &gauss)
+{
+    const float z = fabsf(x) * 0.70710678118654752f;
+    const float t = __fdividef(1.0f, fmaf(0.5f, z, 1.0f));
+    float q = 0.0445844829f;
+    q = fmaf(q, t, -0.0889116004f);
+    q = fmaf(q, t, -0.0691476911f);
+    q = fmaf(q, t, 0.143611208f);
+    q = fmaf(q, t, 0.156033352f);
+    q = fmaf(q, t, 0.249796316f);
+    q = fmaf(q, t, 0.281939417f);
+    q = fmaf(q, t, 0.282096088f);
+    gauss = exp2f(-(z * z) * 1.4426950408889634f);
+    const float lower = 0.5f * t * q * gauss;
+    cdf = x > 0.0f ? 1.0f - lower : lower;
+}
+
+// GELU(x) = x * Phi(x) = x/2 * (1 + erf(x / sqrt 2))
+__device__ __forceinline__ float gelu_f32(float x)
+{
+    float cdf, gauss;
+    normal_cdf(x, cdf, gauss);
+    return x * cdf;
+}
 
 // 32 bf16 values (16 packed words): apply GELU to each, in FP32.
 __device__ __forceinline__ void gelu_words(const uint32_t (&w)[16], float (&v)[32])
@@ -325,10 +377,12 @@ __device__ __forceinline__ void gelu_words(const uint32_t (&w)[16], float (&v)[3
     }
 }
 
-// d/dx GELU(x) = Phi(x) + x * phi(x)
+// d/dx GELU(x) = Phi(x) + x * phi(x),  phi(x) = exp(-x^2 / 2) / sqrt(2 pi)
 __device__ __forceinline__ float gelu_grad_f32(float x)
 {
-    return 0.5f * erfcf(-0.70710678118654752f * x) + x * 0.3989422804014327f * __expf(-0.5f * x * x);
+    float cdf, gauss;
+    normal_cdf(x, cdf, gauss);
+    return fmaf(x * 0.3989422804014327f, gauss, cdf);
 }
 
 // 32 bf16 gradient values times GELU'(pre-activation), in FP32; `aux_row` points at the 32 pre-activations.
@@ -350,7 +404,7 @@ __device__ __forceinline__ void gelu_backward_words(const uint32_t (&w)[16], con
 //   t_row        TMEM address of this warp's lanes at the accumulator's first column
 //   row0         first of the warp's 32 output rows;  col_base  first output column of the tile
 //   release_bar  barrier to arrive on once the accumulator has been read (cluster address if remote)
-template <int BN, bool ACT, int NSLAB>
+template <int BN, int ACT, int NSLAB>
 __device__ __forceinline__ void epilogue_tile(const CUtensorMap *map_out, const CUtensorMap *map_out2, uint32_t t_row,
                                               int row0, int col_base,
                                               const GemmParams &p, const Pow2Pair sc, bool two_step,
@@ -381,58 +435,105 @@ __device__ __forceinline__ void epilogue_tile(const CUtensorMap *map_out, const 
     const bool rows_in = row0 < p.M;
     const bool row_ok = row0 + lane < p.M;
     if (ACT) {
-        // pre-activation (optional) and activated output leave together: both slabs of the warp are in use
+        // The pre-activation (optional) and the second tensor z leave together, 64 columns (one 128-byte slab row
+        // each) at a time; the warp's slabs are used in pairs {pre, z} in rotation.  The loop body covers 32
+        // columns and is not unrolled: fully unrolled, the activation arithmetic outgrows the instruction cache.
+        constexpr int kPairsOfSlabs = NSLAB / 2;
         uint32_t dummy = 0;
+        bool sat = false;
+        Pow2Pair scq = make_pow2_pair(0);
+        if (p.out8) scq = make_pow2_pair(__ldg(p.d_sq) + p.delta_q);
 #pragma unroll 1
-        for (int c = 0; c < BN; c += 64) {
-            uint32_t r0[32], r1[32];
-            tmem_ld_x32(t_row + c, r0);
-            tmem_ld_x32(t_row + c + 32, r1);
+        for (int c = 0; c < BN; c += 32) {
+            const int h = (c >> 5) & 1;  // which half of the slab rows
+            uint32_t r[32];
+            tmem_ld_x32(t_row + c, r);
             tmem_ld_wait();
-            if (c + 64 >= BN) release();
-            if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
-            __syncwarp();
-            const uint32_t slab_pre = warp_slabs, slab_act = warp_slabs + kSlabBytes;
+            if (c + 32 >= BN) release();
+            const uint32_t slab_pre = warp_slabs + (slab_count % kPairsOfSlabs) * 2 * kSlabBytes;
+            const uint32_t slab_act = slab_pre + kSlabBytes;
+            if (h == 0) {
+                // one bulk group per 64 columns: the group that last read this pair of slabs must have finished
+                if (lane == 0) {
+                    if (kPairsOfSlabs == 1) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                    else asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+                }
+                __syncwarp();
+            }
+            const int col0 = col_base + c;
             float v[32];
             uint32_t w[16], wa[16];
+            epilogue_values(r, col0, p, sc, two_step, v);
+            pack_bf16(v, col0, p, w, dummy, false);
+            if (p.out) {
 #pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                const int col0 = col_base + c + 32 * h;
-                epilogue_values(h == 0 ? r0 : r1, col0, p, sc, two_step, v);
-                pack_bf16(v, col0, p, w, dummy, false);
-                if (p.out) {
+                for (int j = 0; j < 4; ++j)
+                    slab_write(slab_pre, lane, 4 * h + j, w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
+            }
+            if (ACT == 1) {
+                gelu_words(w, v);  // the activation sees exactly what the pre-activation tensor holds
+            } else if (ACT == 3) {
 #pragma unroll
-                    for (int j = 0; j < 4; ++j)
-                        slab_write(slab_pre, lane, 4 * h + j, w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
+                for (int i = 0; i < 16; ++i) {
+                    v[2 * i] = __uint_as_float(w[i] << 16);
+                    v[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
                 }
-                if (p.act == 1) {
-                    gelu_words(w, v);  // the activation sees exactly what the pre-activation tensor holds
-                } else {
-                    // columns beyond N are clipped by the store; rows beyond M have no pre-activation to read
-                    const bool ok = row_ok && col0 + 32 <= p.N;
-                    gelu_backward_words(w, reinterpret_cast<const uint16_t *>(p.aux) + (int64_t)(row0 + lane) * p.ldo + col0,
-                                        ok, v);
-                    if (row_ok && !ok && col0 < p.N) {   // ragged last chunk: element by element
-                        const uint16_t *ar = reinterpret_cast<const uint16_t *>(p.aux) + (int64_t)(row0 + lane) * p.ldo;
+            } else {
+                // columns beyond N are clipped by the store; rows beyond M have no pre-activation to read
+                const bool ok = row_ok && col0 + 32 <= p.N;
+                gelu_backward_words(w, reinterpret_cast<const uint16_t *>(p.aux) + (int64_t)(row0 + lane) * p.ldo + col0,
+                                    ok, v);
+                if (row_ok && !ok && col0 < p.N) {   // ragged last chunk: element by element
+                    const uint16_t *ar = reinterpret_cast<const uint16_t *>(p.aux) + (int64_t)(row0 + lane) * p.ldo;
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) {
-                            const float g = (i & 1) ? __uint_as_float(w[i >> 1] & 0xFFFF0000u) : __uint_as_float(w[i >> 1] << 16);
-                            v[i] = col0 + i < p.N ? g * gelu_grad_f32(__uint_as_float((uint32_t)__ldg(ar + col0 + i) << 16)) : 0.0f;
-                        }
+                    for (int i = 0; i < 32; ++i) {
+                        const float g = (i & 1) ? __uint_as_float(w[i >> 1] & 0xFFFF0000u) : __uint_as_float(w[i >> 1] << 16);
+                        v[i] = col0 + i < p.N ? g * gelu_grad_f32(__uint_as_float((uint32_t)__ldg(ar + col0 + i) << 16)) : 0.0f;
                     }
                 }
-                pack_bf16(v, col0, p, wa, amax_bits, row_ok);
+            }
+            pack_bf16(v, col0, p, wa, amax_bits, row_ok);
+            if (p.has_out2) {
 #pragma unroll
                 for (int j = 0; j < 4; ++j)
                     slab_write(slab_act, lane, 4 * h + j, wa[4 * j], wa[4 * j + 1], wa[4 * j + 2], wa[4 * j + 3]);
             }
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-            __syncwarp();
-            if (lane == 0 && rows_in && col_base + c < p.N) {
-                if (p.out) tma_store_2d(map_out, slab_pre, col_base + c, row0);
-                tma_store_2d(map_out2, slab_act, col_base + c, row0);
+            if (p.out8 && row_ok && col0 < p.N) {
+                // the bytes are made from the bf16 values just rounded, as a cast of the stored tensor would;
+                // one row per lane, 32 bytes
+                uint32_t b8[8];
+                if (p.q_fmt == FP8_E4) {
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) b8[i] = cast4<FP8_E4, true>(wa[2 * i], wa[2 * i + 1], scq, sat);
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) b8[i] = cast4<FP8_E5, true>(wa[2 * i], wa[2 * i + 1], scq, sat);
+                }
+                uint8_t *dst = p.out8 + (int64_t)(row0 + lane) * p.ldo + col0;
+                if (col0 + 32 <= p.N) {
+                    reinterpret_cast<uint4 *>(dst)[0] = make_uint4(b8[0], b8[1], b8[2], b8[3]);
+                    reinterpret_cast<uint4 *>(dst)[1] = make_uint4(b8[4], b8[5], b8[6], b8[7]);
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i)
+                        if (col0 + i < p.N) dst[i] = (uint8_t)(b8[i >> 2] >> (8 * (i & 3)));
+                }
+            }
+            if (h == 1) {
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                __syncwarp();
+                if (lane == 0) {
+                    const int x = col0 - 32;
+                    if (rows_in && x < p.N) {
+                        if (p.out) tma_store_only(map_out, slab_pre, x, row0);
+                        if (p.has_out2) tma_store_only(map_out2, slab_act, x, row0);
+                    }
+                    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                }
+                ++slab_count;
             }
         }
+        if (__any_sync(0xFFFFFFFFu, sat) && lane == 0) atomicOr(p.d_status, (unsigned)FP8_FLAG_SATURATED);
         return;
     }
     if (p.out_dt == FP8_BF16) {
@@ -480,13 +581,13 @@ __device__ __forceinline__ void epilogue_tile(const CUtensorMap *map_out, const 
     }
 }
 
-template <int BN, int STAGES, bool ACT>
+template <int BN, int STAGES, int ACT>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
             const __grid_constant__ CUtensorMap map_out, const __grid_constant__ CUtensorMap map_out2,
             const GemmParams p)
 {
-    using L = GemmSmem<BN, STAGES>;
+    using L = GemmSmem<BN, STAGES, ACT ? kActSlabs : kSingleSlabs>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const uint32_t smem_base = smem_u32(smem);
@@ -584,7 +685,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         const Pow2Pair sc = make_pow2_pair(e);
         const bool two_step = (e < -126 || e > 127);
         uint32_t amax_bits = 0, slab_count = 0;
-        const uint32_t warp_slabs = smem_base + L::kEpiOffset + q * kSingleSlabs * kSlabBytes;
+        const uint32_t warp_slabs = smem_base + L::kEpiOffset + q * L::kSlabs * kSlabBytes;
         uint32_t t = 0;
         // with split-K every item leaves its raw FP32 partial sum in the workspace; a second kernel finishes
         GemmParams pp = p;
@@ -607,7 +708,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             if (!__all_sync(0xFFFFFFFFu, ready)) break;
             tc_fence_after();
             const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + buf * BN;
-            epilogue_tile<BN, ACT, kSingleSlabs>(&map_out, &map_out2, t_row, m_blk * kBM + q * 32, n_blk * BN, pp, p.splits > 1 ? sc_one : sc,
+            epilogue_tile<BN, ACT, L::kSlabs>(&map_out, &map_out2, t_row, m_blk * kBM + q * 32, n_blk * BN, pp, p.splits > 1 ? sc_one : sc,
                               p.splits > 1 ? false : two_step, amax_bits, warp_slabs, slab_count, acc_empty_bar(buf),
                               false, lane);
         }
@@ -654,17 +755,24 @@ constexpr int kPairStages = FP8LIN_PAIR_STAGES;
 constexpr int kPairBN = 256;       // N of the pair tile (and of the instruction)
 constexpr int kPairHalfN = 128;    // B rows each CTA loads
 
-struct PairSmem {
+constexpr int kPairStagesAct = 5;  // the kernels with a second output trade one stage for two more slabs per warp
+
+template <int STAGES, int SLABS>
+struct PairSmemT {
+    static constexpr int kStages = STAGES;
+    static constexpr int kSlabs = SLABS;
     static constexpr int kABytes = kBM * kBK;
     static constexpr int kBBytes = kPairHalfN * kBK;
     static constexpr int kStageBytes = kABytes + kBBytes;
-    static constexpr int kEpiOffset = kPairStages * kStageBytes;
-    static constexpr int kBarOffset = kEpiOffset + 4 * kPairSlabs * kSlabBytes;
-    static constexpr int kNumBars = 2 * kPairStages + 4;
+    static constexpr int kEpiOffset = STAGES * kStageBytes;
+    static constexpr int kBarOffset = kEpiOffset + 4 * SLABS * kSlabBytes;
+    static constexpr int kNumBars = 2 * STAGES + 4;
     static constexpr int kTotal = kBarOffset + kNumBars * 8 + 16;
     static constexpr int kDynamic = kTotal + 1024;
     static constexpr int kTmemCols = 512;
 };
+using PairSmem = PairSmemT<kPairStages, kPairSlabs>;
+using PairSmemAct = PairSmemT<kPairStagesAct, kActSlabs>;
 
 __device__ __forceinline__ uint32_t cluster_ctarank()
 {
@@ -731,21 +839,22 @@ __host__ __device__ inline uint32_t make_idesc_pair(int a_fmt, int b_fmt)
 }
 
 // tiles here are 256 x 256; p.tiles_m / p.tiles_n count those
-template <bool ACT>
+template <int ACT>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1)
 gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                  const __grid_constant__ CUtensorMap map_out, const __grid_constant__ CUtensorMap map_out2,
                  const GemmParams p)
 {
-    using L = PairSmem;
+    using L = PairSmemT<ACT ? kPairStagesAct : kPairStages, ACT ? kActSlabs : kPairSlabs>;
+    constexpr int kStagesL = L::kStages;
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const uint32_t smem_base = smem_u32(smem);
     const uint32_t bar_base = smem_base + L::kBarOffset;
     auto full_bar = [&](int s) { return bar_base + 8u * s; };
-    auto empty_bar = [&](int s) { return bar_base + 8u * (kPairStages + s); };
-    auto acc_full_bar = [&](int b) { return bar_base + 8u * (2 * kPairStages + b); };
-    auto acc_empty_bar = [&](int b) { return bar_base + 8u * (2 * kPairStages + 2 + b); };
+    auto empty_bar = [&](int s) { return bar_base + 8u * (kStagesL + s); };
+    auto acc_full_bar = [&](int b) { return bar_base + 8u * (2 * kStagesL + b); };
+    auto acc_empty_bar = [&](int b) { return bar_base + 8u * (2 * kStagesL + 2 + b); };
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + L::kBarOffset + L::kNumBars * 8);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
 
@@ -755,7 +864,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
     const int pair_id = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kPairStages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        for (int s = 0; s < kStagesL; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
         for (int b = 0; b < 2; ++b) { mbar_init(acc_full_bar(b), 1); mbar_init(acc_empty_bar(b), 8); }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -784,9 +893,9 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                 int m_blk, n_blk;
                 tile_coords(tile, p, m_blk, n_blk);
                 for (int k = 0; k < p.num_k; ++k, ++it) {
-                    const int s = it % kPairStages;
+                    const int s = it % kStagesL;
                     const uint32_t leader_full = leader_full0 + 8u * s;
-                    const uint32_t ph = (it / kPairStages) & 1u;
+                    const uint32_t ph = (it / kStagesL) & 1u;
                     if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p.d_status)) { alive = false; break; }
                     // only the leader arrives, announcing the bytes of all four loads of the pair; the
                     // peer's bytes may land first (the pending arrival keeps the phase open)
@@ -811,8 +920,8 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + buf * kPairBN;
                 for (int k = 0; k < p.num_k; ++k, ++it) {
-                    const int s = it % kPairStages;
-                    const uint32_t ph = (it / kPairStages) & 1u;
+                    const int s = it % kStagesL;
+                    const uint32_t ph = (it / kStagesL) & 1u;
                     if (!mbar_wait(full_bar(s), ph, abort_flag, p.d_status)) { alive = false; break; }
                     tc_fence_after();
                     const uint32_t a_addr = smem_base + s * L::kStageBytes;
@@ -834,7 +943,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
         const Pow2Pair sc = make_pow2_pair(e);
         const bool two_step = (e < -126 || e > 127);
         uint32_t amax_bits = 0, slab_count = 0;
-        const uint32_t warp_slabs = smem_base + L::kEpiOffset + q * kPairSlabs * kSlabBytes;
+        const uint32_t warp_slabs = smem_base + L::kEpiOffset + q * L::kSlabs * kSlabBytes;
         const uint32_t leader_acc_empty0 = map_to_cta(acc_empty_bar(0), 0);
         uint32_t t = 0;
         for (int tile = pair_id; tile < num_tiles; tile += num_pairs, ++t) {
@@ -846,7 +955,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             if (!__all_sync(0xFFFFFFFFu, ready)) break;
             tc_fence_after();
             const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + buf * kPairBN;
-            epilogue_tile<kPairBN, ACT, kPairSlabs>(&map_out, &map_out2, t_row, m_blk * 256 + (int)rank * kBM + q * 32, n_blk * kPairBN, p, sc,
+            epilogue_tile<kPairBN, ACT, L::kSlabs>(&map_out, &map_out2, t_row, m_blk * 256 + (int)rank * kBM + q * 32, n_blk * kPairBN, p, sc,
                                    two_step, amax_bits, warp_slabs, slab_count, leader_acc_empty0 + 8u * buf, true, lane);
         }
         if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
@@ -964,18 +1073,31 @@ static bool g_no_splitk = false;        // set from FP8LIN_NO_SPLITK=1
 static bool g_direct_epilogue = false;  // set from FP8LIN_DIRECT_EPILOGUE=1 (A/B comparison of the epilogues)
 static int g_max_pairs = 0;  // CTA pairs that can be resident at once (0: pair kernel unavailable)
 
+constexpr int kStagesAct = 3;  // single-CTA kernels with a second output: fewer stages, two more slabs per warp
+
+template <int ACT>
+static cudaError_t set_smem_attributes()
+{
+    using LS = GemmSmem<kBN, ACT ? kStagesAct : kStages, ACT ? kActSlabs : kSingleSlabs>;
+    using LP = PairSmemT<ACT ? kPairStagesAct : kPairStages, ACT ? kActSlabs : kPairSlabs>;
+    cudaError_t e = cudaFuncSetAttribute(gemm_kernel<kBN, ACT ? kStagesAct : kStages, ACT>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, LS::kDynamic);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(gemm_pair_kernel<ACT>, cudaFuncAttributeMaxDynamicSharedMemorySize, LP::kDynamic);
+    return e;
+}
+
 cudaError_t configure_gemm_kernels(int max_smem_optin)
 {
     using L = GemmSmem<kBN, kStages>;
-    if (L::kDynamic > max_smem_optin || PairSmem::kDynamic > max_smem_optin) return cudaErrorInvalidValue;
-    cudaError_t e = cudaFuncSetAttribute(gemm_kernel<kBN, kStages, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         L::kDynamic);
-    if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(gemm_kernel<kBN, kStages, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kDynamic);
-    if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(gemm_pair_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, PairSmem::kDynamic);
-    if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(gemm_pair_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, PairSmem::kDynamic);
+    using LA = GemmSmem<kBN, kStagesAct, kActSlabs>;
+    if (L::kDynamic > max_smem_optin || PairSmem::kDynamic > max_smem_optin || LA::kDynamic > max_smem_optin ||
+        PairSmemAct::kDynamic > max_smem_optin)
+        return cudaErrorInvalidValue;
+    cudaError_t e = set_smem_attributes<0>();
+    if (e == cudaSuccess) e = set_smem_attributes<1>();
+    if (e == cudaSuccess) e = set_smem_attributes<2>();
+    if (e == cudaSuccess) e = set_smem_attributes<3>();
     if (e != cudaSuccess) return e;
     int sms = 0, dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess ||
@@ -993,7 +1115,7 @@ cudaError_t configure_gemm_kernels(int max_smem_optin)
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
     int clusters = 0;
-    if (cudaOccupancyMaxActiveClusters(&clusters, gemm_pair_kernel<false>, &cfg) != cudaSuccess) {
+    if (cudaOccupancyMaxActiveClusters(&clusters, gemm_pair_kernel<0>, &cfg) != cudaSuccess) {
         cudaGetLastError();
         clusters = 0;
     }
@@ -1031,7 +1153,8 @@ static fp8_status_t run_gemm(fp8_ctx *ctx, const uint8_t *a, int a_fmt, bool a_m
                              const uint8_t *b, int b_fmt, bool b_mn, const int32_t *d_bb, int delta_sum,
                              const void *bias_vec, int bias_dt, void *out, int out_dt, float *d_amax_out, int64_t M,
                              int64_t N, int64_t Kc, cudaStream_t st, int act = 0, void *out_act = nullptr,
-                             const void *aux = nullptr)
+                             const void *aux = nullptr, uint8_t *out8 = nullptr, const int32_t *d_sq = nullptr,
+                             int q_fmt = 0, int delta_q = 0)
 {
     if (M > 0x7FFFFFFF / 2 || N > 0x7FFFFFFF / 2 || Kc > 0x7FFFFFFF / 2) return FP8_ERR_SHAPE;
     const bool pair = g_max_pairs > 0 && M > kBM && !g_force_single;
@@ -1098,6 +1221,11 @@ static fp8_status_t run_gemm(fp8_ctx *ctx, const uint8_t *a, int a_fmt, bool a_m
     p.tma_out = (p.vec_ok && !g_direct_epilogue) ? 1 : 0;
     p.act = act;
     p.aux = aux;
+    p.has_out2 = out_act ? 1 : 0;
+    p.out8 = out8;
+    p.d_sq = d_sq;
+    p.q_fmt = q_fmt;
+    p.delta_q = delta_q;
     CUtensorMap map_out = map_a;  // placeholder when the staged epilogue is off (never dereferenced then)
     CUtensorMap map_out2 = map_a;
     auto encode_out = [&](CUtensorMap *m, void *base) {
@@ -1113,7 +1241,7 @@ static fp8_status_t run_gemm(fp8_ctx *ctx, const uint8_t *a, int a_fmt, bool a_m
         // the activated output always goes through the staged epilogue (callers have checked its alignment)
         p.tma_out = 1;
         p.vec_ok = 1;
-        if (!encode_out(&map_out2, out_act)) return FP8_ERR_CUDA;
+        if (out_act && !encode_out(&map_out2, out_act)) return FP8_ERR_CUDA;
         if (out && !encode_out(&map_out, out)) return FP8_ERR_CUDA;
     } else if (p.tma_out) {
         if (!encode_out(&map_out, out)) return FP8_ERR_CUDA;
@@ -1126,17 +1254,26 @@ static fp8_status_t run_gemm(fp8_ctx *ctx, const uint8_t *a, int a_fmt, bool a_m
     int tiles = p.tiles_m * p.tiles_n;
     if (pair) {
         int pairs = tiles < g_max_pairs ? tiles : g_max_pairs;
-        if (act) gemm_pair_kernel<true><<<2 * pairs, kGemmThreads, PairSmem::kDynamic, st>>>(map_a, map_b, map_out, map_out2, p);
-        else gemm_pair_kernel<false><<<2 * pairs, kGemmThreads, PairSmem::kDynamic, st>>>(map_a, map_b, map_out, map_out2, p);
+        const dim3 grid(2 * pairs);
+        switch (act) {
+        case 1: gemm_pair_kernel<1><<<grid, kGemmThreads, PairSmemAct::kDynamic, st>>>(map_a, map_b, map_out, map_out2, p); break;
+        case 2: gemm_pair_kernel<2><<<grid, kGemmThreads, PairSmemAct::kDynamic, st>>>(map_a, map_b, map_out, map_out2, p); break;
+        case 3: gemm_pair_kernel<3><<<grid, kGemmThreads, PairSmemAct::kDynamic, st>>>(map_a, map_b, map_out, map_out2, p); break;
+        default: gemm_pair_kernel<0><<<grid, kGemmThreads, PairSmem::kDynamic, st>>>(map_a, map_b, map_out, map_out2, p); break;
+        }
     } else {
         int items = tiles * p.splits;
         int grid = items < ctx->sm_count ? items : ctx->sm_count;
-        if (act)
-            gemm_kernel<kBN, kStages, true><<<grid, kGemmThreads, GemmSmem<kBN, kStages>::kDynamic, st>>>(
-                map_a, map_b, map_out, map_out2, p);
-        else
-            gemm_kernel<kBN, kStages, false><<<grid, kGemmThreads, GemmSmem<kBN, kStages>::kDynamic, st>>>(
-                map_a, map_b, map_out, map_out2, p);
+        constexpr int kActDyn = GemmSmem<kBN, kStagesAct, kActSlabs>::kDynamic;
+        switch (act) {
+        case 1: gemm_kernel<kBN, kStagesAct, 1><<<grid, kGemmThreads, kActDyn, st>>>(map_a, map_b, map_out, map_out2, p); break;
+        case 2: gemm_kernel<kBN, kStagesAct, 2><<<grid, kGemmThreads, kActDyn, st>>>(map_a, map_b, map_out, map_out2, p); break;
+        case 3: gemm_kernel<kBN, kStagesAct, 3><<<grid, kGemmThreads, kActDyn, st>>>(map_a, map_b, map_out, map_out2, p); break;
+        default:
+            gemm_kernel<kBN, kStages, 0><<<grid, kGemmThreads, GemmSmem<kBN, kStages>::kDynamic, st>>>(map_a, map_b, map_out,
+                                                                                                     map_out2, p);
+            break;
+        }
         if (p.splits > 1) {
             if (cudaGetLastError() != cudaSuccess) return FP8_ERR_CUDA;
             const bool vec = p.vec_ok && (N % 4) == 0;
@@ -1257,6 +1394,51 @@ fp8_status_t fp8_linear_dgrad_act(fp8_ctx *ctx, const uint8_t *dy8, const int32_
     int delta = format_delta(FP8_E5, conv) + format_delta(FP8_E4, conv);
     return run_gemm(ctx, dy8, FP8_E5, false, d_bg, w, FP8_E4, w_mn, d_bw, delta, nullptr, 0, dx, FP8_BF16, d_amax_act, T,
                     K, N, (cudaStream_t)stream, 2, dx_act, y_pre);
+}
+
+fp8_status_t fp8_linear_fwd_q(fp8_ctx *ctx, const uint8_t *x8, const int32_t *d_bx, const uint8_t *w8,
+                              const int32_t *d_bw, const void *bias_vec, fp8_dtype_t bias_dt, fp8_act_t act, void *y_pre,
+                              void *z, uint8_t *z8, const int32_t *d_bz, float *d_amax_z, int64_t T, int64_t K,
+                              int64_t N, fp8_conv_t conv, void *stream)
+{
+    using namespace fp8lin;
+    if (!ctx || !x8 || !d_bx || !w8 || !d_bw || !z8 || !d_bz) return FP8_ERR_NULL;
+    if ((int)conv < 0 || (int)conv > 1 || (int)bias_dt < 0 || (int)bias_dt > 2 ||
+        ((int)act != (int)FP8_ACT_NONE && (int)act != (int)FP8_ACT_GELU))
+        return FP8_ERR_DTYPE;
+    if (bias_vec && !out_dtype_ok(bias_dt)) return FP8_ERR_UNSUPPORTED;
+    if (act == FP8_ACT_NONE && y_pre) return FP8_ERR_UNSUPPORTED;  // without an activation z is the output itself
+    if (T <= 0 || K <= 0 || N <= 0) return FP8_ERR_SHAPE;
+    if (!aligned16(x8) || !aligned16(w8) || (K % 16) != 0 || !aligned16(z8) || (z && !aligned16(z)) ||
+        (y_pre && !aligned16(y_pre)) || (N % 16) != 0)
+        return FP8_ERR_ALIGN;
+    int delta = 2 * format_delta(FP8_E4, conv);
+    return run_gemm(ctx, x8, FP8_E4, false, d_bx, w8, FP8_E4, false, d_bw, delta, bias_vec, bias_dt, y_pre, FP8_BF16,
+                    d_amax_z, T, N, K, (cudaStream_t)stream, act == FP8_ACT_GELU ? 1 : 3, z, nullptr, z8, d_bz, FP8_E4,
+                    format_delta(FP8_E4, conv));
+}
+
+fp8_status_t fp8_linear_dgrad_q(fp8_ctx *ctx, const uint8_t *dy8, const int32_t *d_bg, const uint8_t *w8,
+                                const uint8_t *w8_t, const int32_t *d_bw, fp8_act_t act, const void *y_pre, void *dx,
+                                void *g, uint8_t *g8, const int32_t *d_bq, float *d_amax_g, int64_t T, int64_t K,
+                                int64_t N, fp8_conv_t conv, void *stream)
+{
+    using namespace fp8lin;
+    if (!ctx || !dy8 || !d_bg || (!w8 && !w8_t) || !d_bw || !g8 || !d_bq) return FP8_ERR_NULL;
+    if ((int)conv < 0 || (int)conv > 1 || ((int)act != (int)FP8_ACT_NONE && (int)act != (int)FP8_ACT_GELU))
+        return FP8_ERR_DTYPE;
+    if (act == FP8_ACT_GELU && !y_pre) return FP8_ERR_NULL;
+    if (act == FP8_ACT_NONE && (y_pre || dx)) return FP8_ERR_UNSUPPORTED;  // g is the input gradient itself
+    if (T <= 0 || K <= 0 || N <= 0) return FP8_ERR_SHAPE;
+    const bool w_mn = (w8_t == nullptr);
+    const uint8_t *w = w_mn ? w8 : w8_t;
+    if (!aligned16(dy8) || !aligned16(w) || (N % 16) != 0 || (K % 16) != 0 || (y_pre && !aligned16(y_pre)) ||
+        !aligned16(g8) || (g && !aligned16(g)) || (dx && !aligned16(dx)))
+        return FP8_ERR_ALIGN;
+    int delta = format_delta(FP8_E5, conv) + format_delta(FP8_E4, conv);
+    return run_gemm(ctx, dy8, FP8_E5, false, d_bg, w, FP8_E4, w_mn, d_bw, delta, nullptr, 0, dx, FP8_BF16, d_amax_g, T, K,
+                    N, (cudaStream_t)stream, act == FP8_ACT_GELU ? 2 : 3, g, y_pre, g8, d_bq, FP8_E5,
+                    format_delta(FP8_E5, conv));
 }
 
 fp8_status_t fp8_linear_wgrad(fp8_ctx *ctx, const uint8_t *dy8, const uint8_t *dy8_t, const int32_t *d_bg,

@@ -22,6 +22,7 @@ ERR_NULL, ERR_SHAPE, ERR_ALIGN, ERR_DTYPE, ERR_UNSUPPORTED, ERR_CUDA, ERR_DEVICE
 E4, E5 = 0, 1
 CONV_PAPER, CONV_NATIVE = 0, 1
 BF16, F16, F32 = 0, 1, 2
+ACT_NONE = 0
 ACT_GELU = 1
 FLAG_NONFINITE_AMAX, FLAG_ZERO_AMAX, FLAG_SATURATED, FLAG_TIMEOUT = 1, 2, 4, 8
 
@@ -29,7 +30,7 @@ SYMBOLS = (
     "fp8_create", "fp8_destroy", "fp8_status_string", "fp8_device_flags", "fp8_amax", "fp8_scaling_bias",
     "fp8_scaling_bias_host", "fp8_cast_e4", "fp8_cast_e5", "fp8_ptq_weights", "fp8_linear_fwd", "fp8_linear_dgrad",
     "fp8_linear_wgrad", "fp8_amax_noalloc", "fp8_linear_fwd_act", "fp8_cast_predicted", "fp8_prediction_stats",
-    "fp8_linear_dgrad_act", "fp8_selftest_wait_expiry", "fp8_range_stats",
+    "fp8_linear_dgrad_act", "fp8_selftest_wait_expiry", "fp8_range_stats", "fp8_linear_fwd_q", "fp8_linear_dgrad_q",
 )
 
 if not os.path.exists(LIB_PATH):
@@ -61,6 +62,10 @@ _lib.fp8_linear_fwd.argtypes = [_P, _P, _P, _P, _P, _P, c_int, _P, c_int, _P, c_
 _lib.fp8_linear_fwd_act.argtypes = [_P, _P, _P, _P, _P, _P, c_int, _P, _P, c_int, _P, c_int64, c_int64, c_int64, c_int, _P]
 _lib.fp8_linear_dgrad.argtypes = [_P, _P, _P, _P, _P, _P, _P, c_int, _P, c_int64, c_int64, c_int64, c_int, _P]
 _lib.fp8_linear_dgrad_act.argtypes = [_P, _P, _P, _P, _P, _P, _P, _P, _P, c_int, _P, c_int64, c_int64, c_int64, c_int, _P]
+_lib.fp8_linear_fwd_q.argtypes = [_P, _P, _P, _P, _P, _P, c_int, c_int, _P, _P, _P, _P, _P, c_int64, c_int64, c_int64,
+                                  c_int, _P]
+_lib.fp8_linear_dgrad_q.argtypes = [_P, _P, _P, _P, _P, _P, c_int, _P, _P, _P, _P, _P, _P, c_int64, c_int64, c_int64,
+                                    c_int, _P]
 _lib.fp8_linear_wgrad.argtypes = [_P, _P, _P, _P, _P, _P, _P, _P, c_int, c_int64, c_int64, c_int64, c_int, _P]
 for _name in SYMBOLS:
     if _name != "fp8_status_string":
@@ -232,6 +237,23 @@ class Context:
         _check(_lib.fp8_linear_dgrad_act(self._h, _ptr(dy8), _ptr(d_bg), _ptr(w8), _ptr(w8_t), _ptr(d_bw), _ptr(y_pre),
                                          _ptr(dx), _ptr(dx_act), act, _ptr(d_amax_act), T, K, N, conv, _stream()),
                "fp8_linear_dgrad_act")
+
+    def linear_fwd_q(self, x8, d_bx, w8, d_bw, z8, d_bz, y_pre=None, z=None, bias_vec=None, d_amax_z=None,
+                     act=ACT_NONE, conv=CONV_PAPER):
+        T, K = x8.shape
+        N = w8.shape[0]
+        bias_dt = _DT[bias_vec.dtype] if bias_vec is not None else BF16
+        _check(_lib.fp8_linear_fwd_q(self._h, _ptr(x8), _ptr(d_bx), _ptr(w8), _ptr(d_bw), _ptr(bias_vec), bias_dt, act,
+                                     _ptr(y_pre), _ptr(z), _ptr(z8), _ptr(d_bz), _ptr(d_amax_z), T, K, N, conv,
+                                     _stream()), "fp8_linear_fwd_q")
+
+    def linear_dgrad_q(self, dy8, d_bg, w8, w8_t, d_bw, g8, d_bq, y_pre=None, dx=None, g=None, d_amax_g=None,
+                       act=ACT_NONE, conv=CONV_PAPER):
+        T, N = dy8.shape
+        K = g8.shape[1]
+        _check(_lib.fp8_linear_dgrad_q(self._h, _ptr(dy8), _ptr(d_bg), _ptr(w8), _ptr(w8_t), _ptr(d_bw), act,
+                                       _ptr(y_pre), _ptr(dx), _ptr(g), _ptr(g8), _ptr(d_bq), _ptr(d_amax_g), T, K, N,
+                                       conv, _stream()), "fp8_linear_dgrad_q")
 
     def linear_wgrad(self, dy8, dy8_t, d_bg, x8, x8_t, d_bx, dw, T, conv=CONV_PAPER):
         N, K = dw.shape

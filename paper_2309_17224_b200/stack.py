@@ -21,6 +21,7 @@ from . import inputs as I
 
 CONFIG_ID = 5
 fp8lin_E4, fp8lin_E5, CONV_PAPER = 0, 1, 0   # enum values of the C ABI (formats, paper convention)
+ACT_GELU = 1
 
 
 def step_input(x_base: torch.Tensor, step: int) -> torch.Tensor:
@@ -125,3 +126,64 @@ class Fp8Stack:
         loss = torch.mean((out.to(torch.float32) - self.target.to(torch.float32)) ** 2)
         self.backward_and_update()
         return {"loss": loss, "bias": self.bias.clone(), "amax": self.amax.clone()}
+
+
+class Fp8StackHistory(Fp8Stack):
+    """The same stack with amax-history scaling (Section 3) for activations and gradients: each of those
+    tensors is quantised with the bias Eq. 3 gives for its amax at the PREVIOUS step, minus ``margin``, by the
+    epilogue of the matmul that produces it (``fp8_linear_fwd_q`` / ``fp8_linear_dgrad_q``), so no activation or
+    gradient is read back for an amax pass or a cast; the amax that comes out of the same launch feeds the next
+    step's bias.  Weights keep the just-in-time bias (they are re-quantised after every update).  The first
+    step, which has no history, runs the just-in-time path.  No transposed copies: the backward matmuls read the
+    forward layouts."""
+
+    def __init__(self, ctx, margin: int = 1, **kw):
+        super().__init__(ctx, fused_activation=True, **kw)
+        self.margin = margin
+        self.pred = torch.zeros_like(self.bias)       # [:, 1] activations, [:, 2] gradients
+        self.have_history = False
+        self.g8b = torch.empty_like(self.g8)
+
+    def _update_history(self) -> None:
+        c = self.ctx
+        for l in range(self.L):
+            c.scaling_bias(self.amax[l, 1:2], fp8lin_E4, CONV_PAPER, self.margin, self.pred[l, 1:2])
+            c.scaling_bias(self.amax[l, 2:3], fp8lin_E5, CONV_PAPER, self.margin, self.pred[l, 2:3])
+        self.have_history = True
+
+    def step(self, step: int) -> Dict[str, object]:
+        if not self.have_history:
+            rec = super().step(step)
+            self._update_history()
+            return rec
+        c, L, T = self.ctx, self.L, self.T
+        x = step_input(self.x_base, step)
+        # the input of the first layer is the one activation no matmul produces: one pass, predicted bias
+        c.cast_e4(x, self.pred[0, 1:2], margin=self.margin, d_amax_out=self.amax[0, 1:2],
+                  d_bias_out=self.bias[0, 1:2], y=self.x8[0])
+        for l in range(L):
+            w16 = self.w32[l].to(torch.bfloat16)
+            c.cast_e4(w16, None, d_amax_out=self.amax[l, 0:1], d_bias_out=self.bias[l, 0:1], y=self.w8[l])
+            if l + 1 < L:
+                c.linear_fwd_q(self.x8[l], self.pred[l, 1:2], self.w8[l], self.bias[l, 0:1], self.x8[l + 1],
+                               self.pred[l + 1, 1:2], y_pre=self.y[l], d_amax_z=self.amax[l + 1, 1:2], act=ACT_GELU)
+            else:
+                c.linear_fwd(self.x8[l], self.pred[l, 1:2], self.w8[l], self.bias[l, 0:1], self.y[l])
+        out = self.y[L - 1].to(torch.float32)
+        loss = torch.mean((out - self.target.to(torch.float32)) ** 2)
+        g = ((out - self.target.to(torch.float32)) * (2.0 / (T * self.d))).to(torch.bfloat16)
+        bufs = (self.g8, self.g8b)
+        c.cast_e5(g, self.pred[L - 1, 2:3], margin=self.margin, d_amax_out=self.amax[L - 1, 2:3],
+                  d_bias_out=self.bias[L - 1, 2:3], y=bufs[(L - 1) % 2])
+        for l in range(L - 1, -1, -1):
+            cur, nxt = bufs[l % 2], bufs[(l + 1) % 2]
+            if l > 0:
+                c.linear_dgrad_q(cur, self.pred[l, 2:3], self.w8[l], None, self.bias[l, 0:1], nxt, self.pred[l - 1, 2:3],
+                                 y_pre=self.y[l - 1], d_amax_g=self.amax[l - 1, 2:3], act=ACT_GELU)
+            c.linear_wgrad(cur, None, self.pred[l, 2:3], self.x8[l], None, self.pred[l, 1:2], self.dw, T)
+            self.w32[l].add_(self.dw.to(torch.float32), alpha=-self.lr)
+        used = self.bias.clone()
+        used[:, 1:3] = self.pred[:, 1:3]
+        rec = {"loss": loss, "bias": used, "amax": self.amax.clone()}
+        self._update_history()
+        return rec

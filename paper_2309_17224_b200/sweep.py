@@ -2,6 +2,8 @@
 
     python -m paper_2309_17224_b200.sweep gemm 8192x8192x16384 8192x8192x4096    # MxNxK forward matmuls
     python -m paper_2309_17224_b200.sweep cast 8192x4096 8192x22016               # amax, cast, amax+cast of bf16 [rows x cols]
+    python -m paper_2309_17224_b200.sweep stack 24x1024x4096                      # layers x d x tokens: the SGD stack, three scaling variants
+    python -m paper_2309_17224_b200.sweep stack 24x1024x4096 --only history --steps 2 --warmup 2 --no-graph   # one variant, short (for profilers)
 
 Prints one line per shape.  Operands of the matmul sweep are random FP8 bytes
 (no NaN codes); a 512 MB buffer is written between cast timings to flush L2.
@@ -47,7 +49,33 @@ def gemm(ctx, shapes, iters=20):
         e.record()
         torch.cuda.synchronize()
         ms = s.elapsed_time(e) / iters
-        print(f"gemm M={M} N={N} K={K}: {2.0 * M * N * K / ms / 1e9:8.1f} TFLOP/s  {ms * 1e3:8.1f} us", flush=True)
+        line = f"gemm M={M} N={N} K={K}: {2.0 * M * N * K / ms / 1e9:8.1f} TFLOP/s  {ms * 1e3:8.1f} us"
+        if N % 16 == 0 and K % 16 == 0:
+            # the fused epilogues on the same operands: GELU + amax; GELU + amax + FP8 bytes; GELU' of a stored
+            # pre-activation + amax + FP8 bytes (input-gradient matmul, so its output is [M, K])
+            z = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+            z8 = torch.empty((M, N), dtype=torch.uint8, device="cuda")
+            amax = torch.zeros(1, dtype=torch.float32, device="cuda")
+            g8 = torch.empty((M, K), dtype=torch.uint8, device="cuda")
+            pre = torch.randn((M, K), device="cuda").to(torch.bfloat16)
+            dy = torch.randint(0, 0x78, (M, N), dtype=torch.uint8, device="cuda")
+            runs = (("gelu", lambda: ctx.linear_fwd_act(a, bias, b, bias, y, z, d_amax_act=amax)),
+                    ("gelu->fp8", lambda: ctx.linear_fwd_q(a, bias, b, bias, z8, bias, y_pre=y, d_amax_z=amax,
+                                                           act=fp8lin.ACT_GELU)),
+                    ("dgrad gelu'->fp8", lambda: ctx.linear_dgrad_q(dy, bias, b, None, bias, g8, bias, y_pre=pre,
+                                                                     d_amax_g=amax, act=fp8lin.ACT_GELU)))
+            for name, fn in runs:
+                for _ in range(3):
+                    fn()
+                torch.cuda.synchronize()
+                s.record()
+                for _ in range(iters):
+                    fn()
+                e.record()
+                torch.cuda.synchronize()
+                t = s.elapsed_time(e) / iters
+                line += f" | {name} {2.0 * M * N * K / t / 1e9:7.1f} TF {t * 1e3:7.1f} us"
+        print(line, flush=True)
 
 
 def cast(ctx, shapes, iters=10):
@@ -72,13 +100,76 @@ def cast(ctx, shapes, iters=10):
               f" | amax+bias+cast {t_fused * 1e3:6.1f} us ({3 * n / t_fused / 1e9:5.2f} TB/s on 3 B/element)", flush=True)
 
 
+def stack(ctx, shapes, steps=40, warmup=8, only=None, graph=True):
+    """ms per SGD step of the stack of FP8 linears (torch glue included): every tensor scaled just in time with
+    separate activation kernels; activation and amax fused into the matmul epilogues; amax-history scaling with
+    the FP8 bytes written by the epilogues."""
+    from . import stack as S
+    for layers, d, tokens in shapes:
+        kw = dict(layers=layers, d=d, tokens=tokens)
+        variants = (("just in time", lambda: S.Fp8Stack(ctx, **kw)),
+                    ("fused epilogues", lambda: S.Fp8Stack(ctx, fused_activation=True, **kw)),
+                    ("amax history", lambda: S.Fp8StackHistory(ctx, margin=1, **kw)))
+        for name, make in variants:
+            if only and only not in name:
+                continue
+            st = make()
+            for i in range(warmup):
+                st.step(i)
+            torch.cuda.synchronize()
+            s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            s.record()
+            for i in range(warmup, warmup + steps):
+                r = st.step(i)
+            e.record()
+            torch.cuda.synchronize()
+            ms = s.elapsed_time(e) / steps
+            if not graph:
+                print(f"stack {layers}x{d}x{tokens} {name:16s}: {ms:7.3f} ms/step  "
+                      f"{st.flops_per_step() / ms / 1e9:7.1f} TFLOP/s | loss {float(r['loss'].item()):.5f}", flush=True)
+                continue
+            # the same step replayed from a CUDA graph: device time without the host's launch overhead
+            g = torch.cuda.CUDAGraph()
+            side = torch.cuda.Stream()
+            side.wait_stream(torch.cuda.current_stream())
+            with torch.cuda.stream(side):
+                st.step(warmup + steps)
+                with torch.cuda.graph(g, stream=side):
+                    st.step(warmup + steps)
+            torch.cuda.current_stream().wait_stream(side)
+            g.replay()
+            torch.cuda.synchronize()
+            s.record()
+            for _ in range(steps):
+                g.replay()
+            e.record()
+            torch.cuda.synchronize()
+            ms_graph = s.elapsed_time(e) / steps
+            print(f"stack {layers}x{d}x{tokens} {name:16s}: {ms:7.3f} ms/step  {st.flops_per_step() / ms / 1e9:7.1f} TFLOP/s"
+                  f" | from a CUDA graph {ms_graph:7.3f} ms/step  {st.flops_per_step() / ms_graph / 1e9:7.1f} TFLOP/s"
+                  f" | loss {float(r['loss'].item()):.5f}", flush=True)
+            del st, g
+
+
 def main(argv):
-    if len(argv) < 2 or argv[0] not in ("gemm", "cast"):
+    opts = {"--only": None, "--steps": None, "--warmup": None}
+    graph = "--no-graph" not in argv
+    argv = [a for a in argv if a != "--no-graph"]
+    for key in opts:
+        if key in argv:
+            i = argv.index(key)
+            opts[key] = argv[i + 1]
+            del argv[i:i + 2]
+    if len(argv) < 2 or argv[0] not in ("gemm", "cast", "stack"):
         print(__doc__)
         return 2
     shapes = [tuple(int(v) for v in a.split("x")) for a in argv[1:]]
     ctx = fp8lin.Context(0)
-    (gemm if argv[0] == "gemm" else cast)(ctx, shapes)
+    if argv[0] == "stack":
+        stack(ctx, shapes, steps=int(opts["--steps"] or 40), warmup=int(opts["--warmup"] or 8), only=opts["--only"],
+              graph=graph)
+    else:
+        {"gemm": gemm, "cast": cast}[argv[0]](ctx, shapes)
     flags = ctx.device_flags()
     if flags & fp8lin.FLAG_TIMEOUT:
         print("a device-side wait expired", file=sys.stderr)

@@ -152,3 +152,41 @@ def test_steps_0_and_1_against_the_oracle_trajectory(run):
             assert_bf16_within_one_ulp(bits_of(dx), rec["dx"][l])
             assert_bf16_within_one_ulp(bits_of(dw), rec["dw"][l])
     assert ctx.device_flags(clear=True) & lib.FLAG_TIMEOUT == 0
+
+
+def test_history_scaling_stack_against_the_oracle_trajectory():
+    """Amax-history scaling (Section 3): activations and gradients are quantised by the producing matmul's
+    epilogue with the previous step's bias minus a margin of one.  A smaller stack, so that the oracle can
+    follow it for six steps; same agreement bars as the just-in-time run, and nothing may clip: the input
+    grows by at most 2^0.4 per step, inside the margin."""
+    from paper_2309_17224_b200 import fp8lin, stack
+    L, d, T, steps, margin = 6, 512, 1024, 6, 1
+    ctx = fp8lin.Context(0)
+    try:
+        st = stack.Fp8StackHistory(ctx, margin=margin, layers=L, d=d, tokens=T)
+        orc = OS.OracleStack([bits_of(w.to(torch.bfloat16)) for w in st.w32], bits_of(st.x_base), bits_of(st.target),
+                             lr=1e-3, history=True, margin=margin)
+        for step in range(steps):
+            r = st.step(step)
+            flags = ctx.device_flags(clear=True)
+            assert flags & fp8lin.FLAG_TIMEOUT == 0
+            if step > 0:
+                assert flags & fp8lin.FLAG_SATURATED == 0
+            rec = orc.step(step)
+            assert abs(float(r["loss"].item()) - rec["loss"]) <= 2e-3 * rec["loss"], step
+            got = r["bias"].cpu().numpy()
+            same = got == rec["bias"]
+            assert same.mean() >= 0.9, (step, same.mean())
+            for l, j in np.argwhere(~same):
+                mx = 57344.0 if j == 2 else 240.0
+                src = orc_prev_amax[l, j] if (step > 0 and j > 0) else rec["amax"][l, j]
+                frac = np.log2(mx / src) % 1.0
+                assert min(frac, 1.0 - frac) < 0.02, (step, l, j)
+            if step > 0:
+                # the biases in use are the previous step's, one below what Eq. 3 gives for that amax
+                for l in range(L):
+                    for j, kind in ((1, O.E4), (2, O.E5)):
+                        assert rec["bias"][l, j] == O.scaling_bias(float(orc_prev_amax[l, j]), kind) - margin
+            orc_prev_amax = rec["amax"].copy()
+    finally:
+        ctx.close()

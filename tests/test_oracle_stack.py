@@ -73,3 +73,36 @@ def test_stack_backward_is_the_gradient_of_its_forward():
         assert cos > 0.98, (l, cos)
         assert 0.8 < np.linalg.norm(mine) / np.linalg.norm(ref) < 1.25
     assert st.step(0)["loss"] < rec["loss"]
+
+
+def test_history_mode_uses_the_previous_steps_amax():
+    """Amax-history scaling: step 0 is the just-in-time step; from step 1 on every activation / gradient bias
+    is Eq. 3 on the previous step's amax minus the margin, the bytes are the cast under that bias (clipping
+    where the tensor outgrew it), and weights keep their own just-in-time bias."""
+    rng = np.random.default_rng(9)
+    L, T, d, margin = 2, 64, 32, 1
+    w = [_bits((torch.from_numpy(rng.standard_normal((d, d))) * 0.2).to(torch.bfloat16)) for _ in range(L)]
+    x = _bits(torch.from_numpy(rng.standard_normal((T, d))).to(torch.bfloat16))
+    tgt = _bits(torch.from_numpy(rng.standard_normal((T, d))).to(torch.bfloat16))
+    jit = S.OracleStack(w, x, tgt, lr=0.1)
+    his = S.OracleStack(w, x, tgt, lr=0.1, history=True, margin=margin)
+    r0j, r0h = jit.step(0), his.step(0)
+    assert np.array_equal(r0j["bias"], r0h["bias"]) and r0j["loss"] == r0h["loss"]
+    prev = r0h["amax"]
+    for step in (1, 2, 3):
+        r = his.step(step)
+        for l in range(L):
+            assert r["bias"][l, 0] == O.scaling_bias(r["amax"][l, 0], O.E4)
+            assert r["bias"][l, 1] == O.scaling_bias(prev[l, 1], O.E4) - margin
+            assert r["bias"][l, 2] == O.scaling_bias(prev[l, 2], O.E5) - margin
+            assert np.array_equal(r["x8"][l], O.cast(r["x"][l], int(r["bias"][l, 1]) + 1, O.N_E4))
+            assert np.array_equal(r["g8"][l], O.cast(r["g"][l], int(r["bias"][l, 2]), O.N_E5))
+            assert r["amax"][l, 1] == O.amax(r["x"][l]) and r["amax"][l, 2] == O.amax(r["g"][l])
+        prev = r["amax"]
+    # a tensor that outgrows its history clips at the format's maximum instead of overflowing
+    big = S.OracleStack(w, x, tgt, lr=0.1, history=True, margin=0)
+    big.step(0)
+    big.prev_amax[0, 1] /= 64.0          # pretend the input was 64 times smaller at the previous step
+    r = big.step(1)
+    dec = np.abs(O.decode_table(O.N_E4)[r["x8"][0]])
+    assert dec.max() == 448.0 and (dec == 448.0).sum() > 1

@@ -335,36 +335,46 @@ __device__ __forceinline__ void slab_publish(const CUtensorMap *map, uint32_t sl
     if (lane == 0 && in_range) tma_store_2d(map, slab, x, y);
 }
 
-// Phi(x), the standard normal distribution function, and exp(-x^2 / 2), in about twenty FP32 instructions (the
-// epilogue runs on four warps, so its instruction count is what bounds the fused kernels).
-//   Phi(-|x|) = erfcx(z) / 2 * exp(-z^2),  z = |x| / sqrt 2,  erfcx(z) = exp(z^2) erfc(z) = t * Q(t),  t = 1 / (1 + z/2)
-// Q is a degree-7 polynomial, a Chebyshev least-squares fit of erfcx(z)/t over t in (0, 1] (all z >= 0) with
-// relative error below 5e-6 -- relative, so that the far negative tail of GELU keeps its accuracy -- and
-// Phi(x) = 1 - Phi(-x) for x > 0.  Rounded to bf16, x * Phi(x) differs from the correctly rounded GELU by at most
-// one bf16 ulp (at 0.2 % of all bf16 inputs), and Phi(x) + x * phi(x) stays within 1e-4 relative of GELU'.
-__device__ __forceinline__ void normal_cdf(float x, float &cdf, float &gauss)
+// Phi(-|x|), the lower tail of the standard normal distribution, and exp(-x^2 / 2), in about fifteen FP32
+// instructions (the fused kernels run under the power cap: every epilogue instruction costs matmul time).
+//   Phi(-|x|) = erfcx(z) / 2 * exp(-z^2),  z = |x| / sqrt 2,  erfcx(z) = exp(z^2) erfc(z),  erfcx(z) / 2 = t * Q(t),
+//   t = 1 / (1 + z/2)
+// Q is a degree-7 polynomial, a Chebyshev least-squares fit of erfcx(z) / (2t) over t in (0, 1] (all z >= 0) with
+// relative error below 5e-6 -- relative, so that the far negative tail of GELU keeps its accuracy.  The
+// exponential is the hardware's base-2 approximation, which flushes results below 2^-126 to zero; so it is
+// taken 2^32 too large and Q's coefficients carry the 2^-32 (exactly), which keeps every product in range down
+// to where GELU itself falls below the smallest bf16 subnormal (|x| > 14.2).
+// Rounded to bf16, GELU(x) = max(x, 0) - |x| Phi(-|x|) differs from the correctly rounded value by at most one
+// bf16 ulp (at 0.2 % of all bf16 inputs), and GELU'(x) stays within 1.2e-4 relative.
+constexpr float kTwoM32 = 2.3283064365386963e-10f;  // 2^-32
+__device__ __forceinline__ float rcp_approx(float v)
 {
-    const float z = fabsf(x) * 0.70710678118654752f;
-    const float t = __fdividef(1.0f, fmaf(0.5f, z, 1.0f));
-    float q = 0.0445844829f;
-    q = fmaf(q, t, -0.0889116004f);
-    q = fmaf(q, t, -0.0691476911f);
-    q = fmaf(q, t, 0.143611208f);
-    q = fmaf(q, t, 0.156033352f);
-    q = fmaf(q, t, 0.249796316f);
-    q = fmaf(q, t, 0.281939417f);
-    q = fmaf(q, t, 0.282096088f);
-    gauss = exp2f(-(z * z) * 1.4426950408889634f);
-    const float lower = 0.5f * t * q * gauss;
-    cdf = x > 0.0f ? 1.0f - lower : lower;
+    float r;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(v));
+    return r;
+}
+// returns Phi(-|x|); gauss_2p32 = 2^32 * exp(-x^2 / 2)
+__device__ __forceinline__ float normal_lower_tail(float x, float &gauss_2p32)
+{
+    const float t = rcp_approx(fmaf(fabsf(x), 0.35355339059327373f, 1.0f));
+    float q = 0.0222922415f * kTwoM32;
+    q = fmaf(q, t, -0.0444558002f * kTwoM32);
+    q = fmaf(q, t, -0.0345738456f * kTwoM32);
+    q = fmaf(q, t, 0.0718056038f * kTwoM32);
+    q = fmaf(q, t, 0.078016676f * kTwoM32);
+    q = fmaf(q, t, 0.124898158f * kTwoM32);
+    q = fmaf(q, t, 0.140969709f * kTwoM32);
+    q = fmaf(q, t, 0.141048044f * kTwoM32);
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(gauss_2p32) : "f"(fmaf(x * x, -0.7213475204444817f, 32.0f)));
+    return t * q * gauss_2p32;
 }
 
-// GELU(x) = x * Phi(x) = x/2 * (1 + erf(x / sqrt 2))
+// GELU(x) = x * Phi(x) = x/2 * (1 + erf(x / sqrt 2)) = max(x, 0) - |x| * Phi(-|x|)
 __device__ __forceinline__ float gelu_f32(float x)
 {
-    float cdf, gauss;
-    normal_cdf(x, cdf, gauss);
-    return x * cdf;
+    float gauss;
+    const float lower = normal_lower_tail(x, gauss);
+    return fmaf(-fabsf(x), lower, fmaxf(x, 0.0f));
 }
 
 // 32 bf16 values (16 packed words): apply GELU to each, in FP32.
@@ -380,9 +390,10 @@ __device__ __forceinline__ void gelu_words(const uint32_t (&w)[16], float (&v)[3
 // d/dx GELU(x) = Phi(x) + x * phi(x),  phi(x) = exp(-x^2 / 2) / sqrt(2 pi)
 __device__ __forceinline__ float gelu_grad_f32(float x)
 {
-    float cdf, gauss;
-    normal_cdf(x, cdf, gauss);
-    return fmaf(x * 0.3989422804014327f, gauss, cdf);
+    float gauss_2p32;
+    const float lower = normal_lower_tail(x, gauss_2p32);
+    const float cdf = x > 0.0f ? 1.0f - lower : lower;
+    return fmaf(x * (0.3989422804014327f * kTwoM32), gauss_2p32, cdf);
 }
 
 // 32 bf16 gradient values times GELU'(pre-activation), in FP32; `aux_row` points at the 32 pre-activations.

@@ -62,6 +62,8 @@ def gemm(ctx, shapes, iters=20):
             runs = (("gelu", lambda: ctx.linear_fwd_act(a, bias, b, bias, y, z, d_amax_act=amax)),
                     ("gelu->fp8", lambda: ctx.linear_fwd_q(a, bias, b, bias, z8, bias, y_pre=y, d_amax_z=amax,
                                                            act=fp8lin.ACT_GELU)),
+                    ("gelu->fp8 (bytes only)", lambda: ctx.linear_fwd_q(a, bias, b, bias, z8, bias, act=fp8lin.ACT_GELU)),
+                    ("->fp8 (bytes only)", lambda: ctx.linear_fwd_q(a, bias, b, bias, z8, bias)),
                     ("dgrad gelu'->fp8", lambda: ctx.linear_dgrad_q(dy, bias, b, None, bias, g8, bias, y_pre=pre,
                                                                      d_amax_g=amax, act=fp8lin.ACT_GELU)))
             for name, fn in runs:

@@ -35,7 +35,7 @@ from paper_2309_17224_b200 import inputs as I
 METRIC = "fp8_linear_fwd_bwd_tflops"
 UNIT = "TFLOP/s"
 DEFAULT_WORKLOAD = "c3_llama7b"
-ORACLE_SAMPLE_TOKENS = 256
+ORACLE_SAMPLE_TOKENS = 256          # floor of the sample; see oracle_sample_tokens
 EVENT_EVERY = 8   # per-kernel CUDA-event pairs are recorded on every eighth timed step
 ORACLE_SAMPLE_LAYER = 1  # the square attention-output projection
 # dram__bytes_read.sum + dram__bytes_write.sum per matmul launch, from one ncu capture of one step of the
@@ -267,14 +267,28 @@ def max_over_ranks(value, dist, device):
     return float(t.item())
 
 
-def oracle_sample_run(wl, seed):
+def oracle_sample_tokens(wl, seconds):
+    """Token count at which one oracle pass over the sample layer takes about `seconds` on this host: a 32-token
+    pass is timed first (the quantisation of the weight tensor is a fixed cost, the matmuls grow with the tokens)."""
+    l = wl.layers[min(ORACLE_SAMPLE_LAYER, len(wl.layers) - 1)]
+    probe = min(32, wl.tokens)
+    oracle_sample_run(wl, I.BASE_SEED, probe)   # the oracle's one-time table set-up stays out of the estimate
+    dt_small, _, _, _ = oracle_sample_run(wl, I.BASE_SEED, probe)
+    dt_big, _, _, _ = oracle_sample_run(wl, I.BASE_SEED, min(2 * probe, wl.tokens))
+    per_token = max((dt_big - dt_small) / probe, 1e-6)
+    fixed = max(dt_small - per_token * probe, 0.0)
+    T = int(max(seconds - fixed, 0.0) / per_token) // 16 * 16
+    return max(16, min(T, 1024, wl.tokens))
+
+
+def oracle_sample_run(wl, seed, tokens=ORACLE_SAMPLE_TOKENS):
     """One bounded sample of the workload on the CPU oracle: the whole path
     (amax, bias, cast of X, W, dY; the three matmuls) for one layer at a
     reduced token count.  Returns (seconds, flops, description)."""
     import oracle as O
     li = min(ORACLE_SAMPLE_LAYER, len(wl.layers) - 1)
     l = wl.layers[li]
-    T = min(ORACLE_SAMPLE_TOKENS, wl.tokens)
+    T = min(tokens, wl.tokens)
     t = I.layer_tensors(wl, li, device="cpu", seed=seed, tokens=T)
     xb, wb = I.bits(t["x"]), I.bits(t["w"])
     gb = I.bits(t["g"]) if wl.backward else None
@@ -300,18 +314,20 @@ def reference_arm(args, wl):
         return 0
     import oracle as O
     O.build()
-    for _ in range(max(0, min(args.warmup, 1))):
-        oracle_sample_run(wl, I.BASE_SEED)
+    # exactly W warm-up and K timed steps; the sample shrinks so that the whole run stays near two minutes
+    steps, warmup = max(1, args.steps), max(0, args.warmup)
+    tokens = oracle_sample_tokens(wl, min(15.0, 120.0 / (steps + warmup)))
+    for _ in range(warmup):
+        oracle_sample_run(wl, I.BASE_SEED, tokens)
     times, flops, what, cores = [], 0.0, "", 1
-    steps = max(1, min(args.steps, 5))
     for _ in range(steps):
-        dt, flops, what, cores = oracle_sample_run(wl, I.BASE_SEED)
+        dt, flops, what, cores = oracle_sample_run(wl, I.BASE_SEED, tokens)
         times.append(dt)
     ms = 1e3 * sum(times) / len(times)
     value = flops / (ms * 1e-3) / 1e12
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
-        "warmup": min(args.warmup, 1), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+        "warmup": warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": {"workload": wl.name, "tokens": wl.tokens, "layers": [f"{l.name}:{l.K}->{l.N}" for l in wl.layers],
                    "passes": "fwd+bwd" if wl.backward else "fwd"},
@@ -532,7 +548,7 @@ def main():
     if world == 1 and not args.no_cpu_baseline:
         import oracle as O
         O.build()
-        dt, fl, what, cores = oracle_sample_run(wl, I.BASE_SEED)
+        dt, fl, what, cores = oracle_sample_run(wl, I.BASE_SEED, oracle_sample_tokens(wl, 12.0))
         cpu_baseline = {"value": fl / dt / 1e12, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": what,
                         "seconds": dt}
 

@@ -355,6 +355,9 @@ cast_small_kernel(const uint4 *__restrict__ x, uint4 *__restrict__ y, int64_t nv
     asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(nctas));
     const int64_t stride = (int64_t)nctas * kSmallThreads;
     const int64_t t0 = (int64_t)rank * kSmallThreads + threadIdx.x;
+    // A matmul launched behind this kernel as a programmatic dependent may take its places now and start
+    // streaming its weights; it waits for this grid to complete before it touches anything written here.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     uint4 v[kSmallVecs];
     uint32_t acc = 0;

@@ -635,6 +635,32 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_b)) : "memory");
             uint32_t it = 0;
             bool alive = true;
+            auto load_b = [&](int s, int n_blk, int k) {
+                const uint32_t b_dst = smem_base + s * L::kStageBytes + L::kABytes;
+                if (p.b_mn) {  // two blocks of 128 N values, 16 KB apart
+                    for (int h = 0; h < BN / 128; ++h)
+                        tma_load_2d(b_dst + h * (128 * kBK), &map_b, full_bar(s), n_blk * BN + h * 128, k * kBK);
+                } else {
+                    tma_load_2d(b_dst, &map_b, full_bar(s), k * kBK, n_blk * BN);
+                }
+            };
+            // When this grid runs as a programmatic dependent of the launch before it (a decode-size cast), nothing
+            // that launch may have written is read before it has completed; but the first ring of B tiles (the
+            // weights, in decode) is already pulled towards L2, which holds no stale data whoever writes them.
+            if ((int)blockIdx.x < num_items) {
+                int m_blk, n_blk;
+                tile_coords((int)blockIdx.x / p.splits, p, m_blk, n_blk);
+                const int k0 = ((int)blockIdx.x % p.splits) * p.kb_per_split;
+                const int k1 = min(p.num_k, k0 + min(p.kb_per_split, STAGES));
+                for (int k = k0; k < k1; ++k) {
+                    if (p.b_mn) {
+                        for (int h = 0; h < BN / 128; ++h) tma_prefetch_l2_2d(&map_b, n_blk * BN + h * 128, k * kBK);
+                    } else {
+                        tma_prefetch_l2_2d(&map_b, k * kBK, n_blk * BN);
+                    }
+                }
+            }
+            asm volatile("griddepcontrol.wait;" ::: "memory");
             for (int item = blockIdx.x; alive && item < num_items; item += gridDim.x) {
                 int m_blk, n_blk;
                 tile_coords(item / p.splits, p, m_blk, n_blk);
@@ -648,13 +674,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                     const uint32_t a_dst = smem_base + s * L::kStageBytes;
                     if (p.a_mn) tma_load_2d(a_dst, &map_a, full_bar(s), m_blk * kBM, k * kBK);
                     else tma_load_2d(a_dst, &map_a, full_bar(s), k * kBK, m_blk * kBM);
-                    if (p.b_mn) {  // two blocks of 128 N values, 16 KB apart
-                        for (int h = 0; h < BN / 128; ++h)
-                            tma_load_2d(a_dst + L::kABytes + h * (128 * kBK), &map_b, full_bar(s), n_blk * BN + h * 128,
-                                        k * kBK);
-                    } else {
-                        tma_load_2d(a_dst + L::kABytes, &map_b, full_bar(s), k * kBK, n_blk * BN);
-                    }
+                    load_b(s, n_blk, k);
                 }
             }
         }
@@ -691,6 +711,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         }
     } else {
         // ------------------------------- epilogue -------------------------------
+        asm volatile("griddepcontrol.wait;" ::: "memory");  // the biases may come from the launch before this one
         const int q = warp & 3;  // TMEM lane quarter this warp may address
         const int e = -(__ldg(p.d_sa) + __ldg(p.d_sb) + p.delta_sum);
         const Pow2Pair sc = make_pow2_pair(e);
@@ -1280,10 +1301,22 @@ static fp8_status_t run_gemm(fp8_ctx *ctx, const uint8_t *a, int a_fmt, bool a_m
         case 1: gemm_kernel<kBN, kStagesAct, 1><<<grid, kGemmThreads, kActDyn, st>>>(map_a, map_b, map_out, map_out2, p); break;
         case 2: gemm_kernel<kBN, kStagesAct, 2><<<grid, kGemmThreads, kActDyn, st>>>(map_a, map_b, map_out, map_out2, p); break;
         case 3: gemm_kernel<kBN, kStagesAct, 3><<<grid, kGemmThreads, kActDyn, st>>>(map_a, map_b, map_out, map_out2, p); break;
-        default:
-            gemm_kernel<kBN, kStages, 0><<<grid, kGemmThreads, GemmSmem<kBN, kStages>::kDynamic, st>>>(map_a, map_b, map_out,
-                                                                                                     map_out2, p);
+        default: {
+            // may start while the launch before it drains (its own first instruction that reads memory waits)
+            cudaLaunchAttribute attr[1];
+            attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+            attr[0].val.programmaticStreamSerializationAllowed = 1;
+            cudaLaunchConfig_t cfg = {};
+            cfg.gridDim = dim3((unsigned)grid);
+            cfg.blockDim = dim3(kGemmThreads);
+            cfg.dynamicSmemBytes = GemmSmem<kBN, kStages>::kDynamic;
+            cfg.stream = st;
+            cfg.attrs = attr;
+            cfg.numAttrs = 1;
+            if (cudaLaunchKernelEx(&cfg, gemm_kernel<kBN, kStages, 0>, map_a, map_b, map_out, map_out2, p) != cudaSuccess)
+                return FP8_ERR_CUDA;
             break;
+        }
         }
         if (p.splits > 1) {
             if (cudaGetLastError() != cudaSuccess) return FP8_ERR_CUDA;

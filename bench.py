@@ -306,6 +306,52 @@ def whole_job_value(world, step_flops, ms_per_step):
     return world * step_flops / (ms_per_step * 1e-3) / 1e12
 
 
+def quantisation_kernel_bandwidths(ctx, layers, peak_gbs, reps=3):
+    """The amax kernel and the cast kernel timed one launch at a time (CUDA events on the launching stream) over
+    every tensor the step quantises, cycling through the tensors so that each launch finds its input out of L2
+    (the tensors of a step total far more than L2).  Algorithmic bytes: 2 per element for amax, 2 + 1 for the
+    cast.  Returned: bytes summed over launches / time summed over launches, and the slowest tensor."""
+    tensors = []
+    for L in layers:
+        if L.backward:
+            tensors += [(L.w, L.w8, 0), (L.x, L.x8, 0), (L.g, L.g8, 1)]
+        else:
+            tensors += [(L.x, L.x8, 0)]
+    amax = torch.zeros(1, dtype=torch.float32, device=tensors[0][0].device)
+    bias = torch.zeros(1, dtype=torch.int32, device=tensors[0][0].device)
+    spans = {"amax": [], "cast": [], "library_copy": []}
+    scratch = torch.empty(max(x.numel() for x, _, _ in tensors), dtype=tensors[0][0].dtype, device=tensors[0][0].device)
+    def launch(key, x, y, fmt):
+        if key == "amax":
+            ctx.amax(x, amax)
+        elif key == "cast":
+            (ctx.cast_e5 if fmt else ctx.cast_e4)(x, bias, y=y)
+        else:
+            scratch[:x.numel()].copy_(x.reshape(-1))
+
+    for key in spans:                      # one kind at a time: a tensor was last touched a whole round ago
+        for rep in range(reps + 1):
+            for x, y, fmt in tensors:
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                torch.cuda._sleep(100000)  # ~50 us of spinning ahead of the pair: the host enqueues the event, the
+                a.record()                 # launch and the event while the stream is busy, so the interval holds
+                launch(key, x, y, fmt)     # the kernel and not the host's launch latency
+                b.record()
+                if rep > 0:                # the first round loads the kernels
+                    spans[key].append((x.numel(), a, b))
+    torch.cuda.synchronize()
+    out = {"how": f"one launch at a time over the step's {len(tensors)} tensors, {reps} rounds, inputs out of L2"}
+    # library_copy: torch's device-to-device copy of the same tensors (2 B read + 2 B written per element), the
+    # rate a plain copy reaches at these sizes, for context: the measured peak comes from far larger buffers
+    for key, bpe in (("amax", 2), ("cast", 3), ("library_copy", 4)):
+        rates = [n * bpe / (a.elapsed_time(b) * 1e-3) / 1e9 for n, a, b in spans[key]]
+        total_b = sum(n * bpe for n, _, _ in spans[key])
+        total_s = sum(a.elapsed_time(b) for _, a, b in spans[key]) * 1e-3
+        out[key] = {"gbs": total_b / total_s / 1e9, "frac": total_b / total_s / 1e9 / peak_gbs,
+                    "slowest_tensor_gbs": min(rates), "bytes_per_element": bpe}
+    return out
+
+
 def max_over_ranks(value, dist, device):
     if dist is None:
         return value
@@ -495,6 +541,9 @@ def main():
                     "traffic": GEMM_DRAM_BYTES_PER_LAUNCH.get((wl.name, tokens))}
     roofline["frac"] = roofline["achieved"] / roofline["peak"]
 
+    # ---- the two quantisation kernels, each against its own algorithmic bytes (outside the timed region) ----
+    per_kernel = quantisation_kernel_bandwidths(ctx, layers, peaks["hbm_gbs"])
+
     # ---- the same steps with the one-pass quantisation (bias guessed from the previous step, verified) ----
     predicted = None
     if wl.backward and not args.transposed_copies and not args.no_predicted_leg:
@@ -641,7 +690,11 @@ def main():
         "amax_cast": {"effective_gbs": cast_elems * bytes_per_elem / (cast_ms * 1e-3) / 1e9,
                       "bytes_per_element": bytes_per_elem, "ms_per_step": cast_ms / sampled_steps,
                       "hbm_peak_gbs": peaks["hbm_gbs"],
-                      "frac": cast_elems * bytes_per_elem / (cast_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]},
+                      "frac": cast_elems * bytes_per_elem / (cast_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                      "note": "amax + bias + cast as one operation, two launches: 5 B/element move where the tensor "
+                              "exceeds L2, so 0.6 is this path's ceiling on 3 B/element; per_kernel holds each kernel "
+                              "against its own bytes; with_bias_prediction is the one-pass variant",
+                      "per_kernel": per_kernel},
         "layer_ms": {k: round(v, 4) for k, v in timers.layer_ms().items()},   # amax + cast + matmuls of one layer
         "with_bias_prediction": predicted,
         "with_cuda_graph": graphed,

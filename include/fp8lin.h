@@ -141,6 +141,20 @@ FP8_API fp8_status_t fp8_amax_noalloc(const void *x, fp8_dtype_t x_dt, int64_t r
 FP8_API fp8_status_t fp8_scaling_bias(fp8_ctx *ctx, const float *d_amax, fp8_format_t fmt, fp8_conv_t conv,
                               int32_t margin, int32_t *d_bias, void *stream);
 
+/* Amax history (Section 3: "rely on the past history of absolute max" where a
+ * second pass over memory is too costly): a ring of the last `len` amax values of
+ * one tensor.  The call stores *d_amax_new at the cursor, advances the cursor
+ * (wrapping), and writes to *d_bias the bias Eq. 3 gives for the LARGEST entry of
+ * the ring, minus `margin` -- the bias to quantise that tensor with at the next
+ * step.  A ring that starts zero-filled ignores its unused entries; an all-zero
+ * or non-finite maximum gives bias 0 and the status flag, as in fp8_scaling_bias.
+ *   d_history  in/out: device float[len], 1 <= len <= 65536, owned by the caller
+ *   d_cursor   in/out: device int32, index of the entry to overwrite next (0 at start)
+ * len == 1 is fp8_scaling_bias on the newest amax. */
+FP8_API fp8_status_t fp8_amax_history_bias(fp8_ctx *ctx, float *d_history, int32_t len, int32_t *d_cursor,
+                                           const float *d_amax_new, fp8_format_t fmt, fp8_conv_t conv, int32_t margin,
+                                           int32_t *d_bias, void *stream);
+
 /* The same integer rule on the host (no device work, no ctx). */
 FP8_API fp8_status_t fp8_scaling_bias_host(float amax, fp8_format_t fmt, fp8_conv_t conv, int32_t margin, int32_t *bias);
 

@@ -160,6 +160,12 @@ def scaling_bias(amax_value: float, kind: int, conv: int = CONV_PAPER, margin: i
     return int(_L().orc_scaling_bias(float(np.float32(amax_value)), bias_max_num(kind, conv), int(margin)))
 
 
+def history_bias(amax_window, kind: int, conv: int = CONV_PAPER, margin: int = 0) -> int:
+    """Amax-history scaling (Section 3: rely on the past history of the absolute max): the bias for the next
+    step is Eq. 3 on the largest amax of the window, minus the margin."""
+    return scaling_bias(max(float(a) for a in amax_window), kind, conv, margin)
+
+
 def cast(x_bits: np.ndarray, shift: int, fmt: int, transposed: bool = False):
     """codes = encode_fmt(x * 2^shift); returns y[rows, cols] and, if asked,
     also y_t[cols, rows]."""

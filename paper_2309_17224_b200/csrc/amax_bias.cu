@@ -145,6 +145,32 @@ __global__ void scaling_bias_kernel(const float *__restrict__ d_amax, int fmt, i
     if (flags) atomicOr(d_status, flags);
 }
 
+// One warp: push the newest amax into the ring, take the largest entry (|x| orders like its bit pattern; NaN and
+// inf sort above every finite value and end up flagged by the bias rule), derive the bias.
+__global__ void amax_history_kernel(float *__restrict__ d_history, int len, int32_t *__restrict__ d_cursor,
+                                    const float *__restrict__ d_amax_new, int fmt, int conv, int margin,
+                                    int32_t *__restrict__ d_bias, unsigned *d_status)
+{
+    const int lane = threadIdx.x;
+    int cur = *d_cursor;
+    cur = (cur < 0 || cur >= len) ? 0 : cur;
+    const uint32_t fresh = __float_as_uint(*d_amax_new) & 0x7FFFFFFFu;
+    uint32_t m = 0;
+    for (int i = lane; i < len; i += 32) {
+        uint32_t v = i == cur ? fresh : (__float_as_uint(d_history[i]) & 0x7FFFFFFFu);
+        m = max(m, v);
+    }
+    m = __reduce_max_sync(0xFFFFFFFFu, m);
+    __syncwarp();
+    if (lane == 0) {
+        d_history[cur] = __uint_as_float(fresh);
+        *d_cursor = cur + 1 == len ? 0 : cur + 1;
+        unsigned flags = 0;
+        *d_bias = bias_from_amax_bits(m, fmt, conv, margin, &flags);
+        if (flags) atomicOr(d_status, flags);
+    }
+}
+
 template <int DT>
 static cudaError_t launch_amax_dt(fp8_ctx *ctx, const void *x, int64_t rows, int64_t cols, int64_t ld, AmaxOut o,
                                   cudaStream_t stream)
@@ -200,6 +226,18 @@ fp8_status_t fp8_scaling_bias(fp8_ctx *ctx, const float *d_amax, fp8_format_t fm
     if ((int)fmt < 0 || (int)fmt > 1 || (int)conv < 0 || (int)conv > 1) return FP8_ERR_DTYPE;
     fp8lin::scaling_bias_kernel<<<1, 1, 0, (cudaStream_t)stream>>>(d_amax, (int)fmt, (int)conv, margin, d_bias,
                                                                   ctx->d_status);
+    return cudaGetLastError() == cudaSuccess ? FP8_OK : FP8_ERR_CUDA;
+}
+
+fp8_status_t fp8_amax_history_bias(fp8_ctx *ctx, float *d_history, int32_t len, int32_t *d_cursor,
+                                   const float *d_amax_new, fp8_format_t fmt, fp8_conv_t conv, int32_t margin,
+                                   int32_t *d_bias, void *stream)
+{
+    if (!ctx || !d_history || !d_cursor || !d_amax_new || !d_bias) return FP8_ERR_NULL;
+    if ((int)fmt < 0 || (int)fmt > 1 || (int)conv < 0 || (int)conv > 1) return FP8_ERR_DTYPE;
+    if (len <= 0 || len > 65536) return FP8_ERR_SHAPE;
+    fp8lin::amax_history_kernel<<<1, 32, 0, (cudaStream_t)stream>>>(d_history, len, d_cursor, d_amax_new, (int)fmt,
+                                                                   (int)conv, margin, d_bias, ctx->d_status);
     return cudaGetLastError() == cudaSuccess ? FP8_OK : FP8_ERR_CUDA;
 }
 

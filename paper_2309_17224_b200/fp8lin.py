@@ -30,7 +30,7 @@ SYMBOLS = (
     "fp8_create", "fp8_destroy", "fp8_status_string", "fp8_device_flags", "fp8_amax", "fp8_scaling_bias",
     "fp8_scaling_bias_host", "fp8_cast_e4", "fp8_cast_e5", "fp8_ptq_weights", "fp8_linear_fwd", "fp8_linear_dgrad",
     "fp8_linear_wgrad", "fp8_amax_noalloc", "fp8_linear_fwd_act", "fp8_cast_predicted", "fp8_prediction_stats",
-    "fp8_linear_dgrad_act", "fp8_selftest_wait_expiry", "fp8_range_stats", "fp8_linear_fwd_q", "fp8_linear_dgrad_q",
+    "fp8_linear_dgrad_act", "fp8_selftest_wait_expiry", "fp8_range_stats", "fp8_linear_fwd_q", "fp8_linear_dgrad_q", "fp8_amax_history_bias",
 )
 
 if not os.path.exists(LIB_PATH):
@@ -62,6 +62,7 @@ _lib.fp8_linear_fwd.argtypes = [_P, _P, _P, _P, _P, _P, c_int, _P, c_int, _P, c_
 _lib.fp8_linear_fwd_act.argtypes = [_P, _P, _P, _P, _P, _P, c_int, _P, _P, c_int, _P, c_int64, c_int64, c_int64, c_int, _P]
 _lib.fp8_linear_dgrad.argtypes = [_P, _P, _P, _P, _P, _P, _P, c_int, _P, c_int64, c_int64, c_int64, c_int, _P]
 _lib.fp8_linear_dgrad_act.argtypes = [_P, _P, _P, _P, _P, _P, _P, _P, _P, c_int, _P, c_int64, c_int64, c_int64, c_int, _P]
+_lib.fp8_amax_history_bias.argtypes = [_P, _P, c_int32, _P, _P, c_int, c_int, c_int32, _P, _P]
 _lib.fp8_linear_fwd_q.argtypes = [_P, _P, _P, _P, _P, _P, c_int, c_int, _P, _P, _P, _P, _P, c_int64, c_int64, c_int64,
                                   c_int, _P]
 _lib.fp8_linear_dgrad_q.argtypes = [_P, _P, _P, _P, _P, _P, c_int, _P, _P, _P, _P, _P, _P, c_int64, c_int64, c_int64,
@@ -161,6 +162,10 @@ class Context:
     def scaling_bias(self, d_amax, fmt, conv, margin, d_bias):
         _check(_lib.fp8_scaling_bias(self._h, _ptr(d_amax), fmt, conv, margin, _ptr(d_bias), _stream()),
                "fp8_scaling_bias")
+
+    def amax_history_bias(self, d_history, d_cursor, d_amax_new, fmt, d_bias, conv=CONV_PAPER, margin=0):
+        _check(_lib.fp8_amax_history_bias(self._h, _ptr(d_history), d_history.numel(), _ptr(d_cursor), _ptr(d_amax_new),
+                                          fmt, conv, margin, _ptr(d_bias), _stream()), "fp8_amax_history_bias")
 
     # -- cast -------------------------------------------------------------------
     def _cast(self, fn, name, x, d_bias, conv, margin, d_amax_out, d_bias_out, y, y_t, rows, cols, ld):

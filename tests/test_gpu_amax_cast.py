@@ -384,3 +384,36 @@ def test_range_statistics_of_a_constant_bias_sweep(ctx, lib, kind, dtype):
         results[b] = want
     # the sweep shows the window: small biases flush, large ones clip
     assert results[-12][1] > results[3][1] and results[24][0] > results[3][0]
+
+
+@pytest.mark.parametrize("length", [1, 4, 33, 100])
+@pytest.mark.parametrize("kind", [O.E4, O.E5])
+def test_amax_history_ring(ctx, lib, length, kind):
+    """fp8_amax_history_bias keeps the last `length` amax values of a tensor in a ring and returns Eq. 3 on the
+    largest of them minus the margin; checked against the oracle's rule on the same window after every push,
+    through several wraps of the ring."""
+    rng = np.random.default_rng(length * 10 + kind)
+    hist = torch.zeros(length, dtype=torch.float32, device="cuda")
+    cursor = torch.zeros(1, dtype=torch.int32, device="cuda")
+    new = torch.zeros(1, dtype=torch.float32, device="cuda")
+    bias = torch.zeros(1, dtype=torch.int32, device="cuda")
+    margin = 2
+    pushed = []
+    for step in range(3 * length + 5):
+        a = float(np.float32(2.0 ** rng.uniform(-30, 30)))
+        pushed.append(a)
+        new.fill_(a)
+        ctx.amax_history_bias(hist, cursor, new, kind, bias, margin=margin)
+        window = pushed[-length:]
+        assert int(bias.item()) == O.history_bias(window, kind, O.CONV_PAPER, margin), step
+        assert int(cursor.item()) == (step + 1) % length
+    assert sorted(hist.cpu().tolist()) == sorted(pushed[-length:])
+    assert ctx.device_flags(clear=True) == 0
+    # nothing but zeros in the window: bias 0 and the zero-amax flag, as for fp8_scaling_bias
+    hist.zero_()
+    new.zero_()
+    ctx.amax_history_bias(hist, cursor, new, kind, bias)
+    assert int(bias.item()) == 0 and ctx.device_flags(clear=True) & lib.FLAG_ZERO_AMAX
+    with pytest.raises(lib.Fp8Error) as e:
+        ctx.amax_history_bias(hist[:0], cursor, new, kind, bias)
+    assert e.value.status in (lib.ERR_SHAPE, lib.ERR_NULL)

@@ -133,3 +133,18 @@ def test_fp16_and_fp32_inputs_are_read_exactly():
     ref = torch.from_numpy(f * 2.0).to(torch.float8_e4m3fn).view(torch.uint8).numpy()
     ok = np.abs(f * 2.0) <= 448.0
     assert np.array_equal(got[ok], ref[ok])
+
+
+def test_history_bias_is_eq3_on_the_window_maximum():
+    """Amax-history scaling: a window of one is the just-in-time bias; for a longer window every entry fits
+    under the bias (entry * 2^b <= max_num) while the largest one would not fit under b + 1."""
+    from fractions import Fraction
+    rng = np.random.default_rng(3)
+    for kind, mx in ((O.E4, 240), (O.E5, 57344)):
+        for _ in range(50):
+            window = [float(np.float32(2.0 ** rng.uniform(-20, 20))) for _ in range(int(rng.integers(1, 9)))]
+            assert O.history_bias(window[:1], kind) == O.scaling_bias(window[0], kind)
+            b = O.history_bias(window, kind)
+            assert all(Fraction(a) * Fraction(2) ** b <= mx for a in window)
+            assert Fraction(max(window)) * Fraction(2) ** (b + 1) > mx
+            assert O.history_bias(window, kind, O.CONV_PAPER, 3) == b - 3

@@ -255,8 +255,15 @@ FP8_API fp8_status_t fp8_linear_fwd(fp8_ctx *ctx, const uint8_t *x8, const int32
  *          pre-activation gives a non-finite output
  *   d_amax_act  NULL or out: amax of y_act; fp8_scaling_bias + fp8_cast_e4 with
  *          that bias then quantise y_act in a single pass
+ *          FP8_ACT_SWIGLU: the gated unit of the Llama MLP, z = SiLU(gate) * up with
+ *          SiLU(a) = a / (1 + exp(-a)).  The caller stores the gate and the up
+ *          projection as ONE weight w8[N = 2F, K] whose rows come in blocks of 64:
+ *          32 gate rows (features 32b .. 32b+31) followed by the 32 up rows of the
+ *          same features; y_pre [T, 2F] has that column layout, y_act is [T, F].
+ *          Both factors are the bf16-rounded pre-activations; the bf16 result is
+ *          within one bf16 ulp of the correctly rounded product.  Needs N % 64 == 0.
  * Needs 16-byte aligned y_pre / y_act and N % 8 == 0, besides fp8_linear_fwd's rules. */
-typedef enum { FP8_ACT_NONE = 0, FP8_ACT_GELU = 1 } fp8_act_t;
+typedef enum { FP8_ACT_NONE = 0, FP8_ACT_GELU = 1, FP8_ACT_SWIGLU = 2 } fp8_act_t;
 FP8_API fp8_status_t fp8_linear_fwd_act(fp8_ctx *ctx, const uint8_t *x8, const int32_t *d_bx, const uint8_t *w8,
                                         const int32_t *d_bw, const void *bias_vec, fp8_dtype_t bias_dt, void *y_pre,
                                         void *y_act, fp8_act_t act, float *d_amax_act, int64_t T, int64_t K, int64_t N,
@@ -280,6 +287,11 @@ FP8_API fp8_status_t fp8_linear_dgrad(fp8_ctx *ctx, const uint8_t *dy8, const in
  *   dx      NULL, or out [T, K] bf16: the rounded input gradient dX
  *   dx_act  out [T, K] bf16: bf16(dX) * act'(y_pre) in FP32, rounded -- the output gradient of the layer below
  *   d_amax_act  NULL or out: its amax, so that the layer below quantises it in a single pass
+ * With FP8_ACT_SWIGLU the matmul's output dX[T, K] is the gradient dz of the gated
+ * unit's output; y_pre is the stored [T, 2K] pre-activation in the block layout of
+ * fp8_linear_fwd_act, and dx_act [T, 2K] receives, in the same layout,
+ *   d_gate = bf16(dz) * up * SiLU'(gate),  d_up = bf16(dz) * SiLU(gate),
+ * SiLU'(a) = s + a s (1 - s), s = 1 / (1 + exp(-a)); d_amax_act covers both.  Needs K % 32 == 0.
  * Operand rules as fp8_linear_dgrad; y_pre, dx, dx_act 16-byte aligned, K % 8 == 0. */
 FP8_API fp8_status_t fp8_linear_dgrad_act(fp8_ctx *ctx, const uint8_t *dy8, const int32_t *d_bg, const uint8_t *w8,
                                           const uint8_t *w8_t, const int32_t *d_bw, const void *y_pre, void *dx,
@@ -296,6 +308,8 @@ FP8_API fp8_status_t fp8_linear_dgrad_act(fp8_ctx *ctx, const uint8_t *dy8, cons
  *                       Y as in fp8_linear_fwd;  z8 = E4 bytes of z under bias *d_bz
  *   fp8_linear_dgrad_q: z = bf16(dX) for FP8_ACT_NONE, z = bf16(bf16(dX) * GELU'(y_pre)) for FP8_ACT_GELU,
  *                       dX as in fp8_linear_dgrad;  g8 = E5 bytes of z under bias *d_bq
+ *   FP8_ACT_SWIGLU:     as in fp8_linear_fwd_act / fp8_linear_dgrad_act: forward z and z8 are [T, N/2],
+ *                       backward y_pre, g and g8 are [T, 2K] (N % 64 == 0, K % 32 == 0)
  * and the bytes are exactly what fp8_cast_e4 / fp8_cast_e5 with that bias give on
  * the stored z (FP8_FLAG_SATURATED is raised likewise when a value clips).
  *   y_pre (fwd)   NULL, or out [T, N] bf16 pre-activation; must be NULL with FP8_ACT_NONE

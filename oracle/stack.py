@@ -43,6 +43,42 @@ def gelu_grad(y_bits: np.ndarray) -> np.ndarray:
     return 0.5 * (1.0 + erf(z / math.sqrt(2.0))) + z * np.exp(-0.5 * z * z) / math.sqrt(2.0 * math.pi)
 
 
+def _blocks32(two_f: int):
+    """Column indices of the gate and of the up halves in the block layout [32 gate, 32 up, 32 gate, ...]."""
+    assert two_f % 64 == 0
+    j = np.arange(two_f // 2)
+    gate = (j // 32) * 64 + j % 32
+    return gate, gate + 32
+
+
+def silu(a: np.ndarray) -> np.ndarray:
+    """SiLU(a) = a * sigma(a); written per sign so that exp never overflows and the negative tail keeps its
+    relative accuracy."""
+    e = np.exp(-np.abs(a))
+    return np.where(a > 0, a / (1.0 + e), a * e / (1.0 + e))
+
+
+def swiglu_bits(y_pre_bits: np.ndarray) -> np.ndarray:
+    """z[:, j] = bf16(SiLU(gate_j) * up_j) from the bf16 pre-activations [T, 2F] in the 32-block layout."""
+    y = bf16_to_f64(y_pre_bits)
+    gi, ui = _blocks32(y.shape[1])
+    return f64_to_bf16(silu(y[:, gi]) * y[:, ui])
+
+
+def swiglu_backward(dz: np.ndarray, y_pre_bits: np.ndarray) -> np.ndarray:
+    """Gradients of the gate / up pre-activations, float64, in the 32-block layout:
+    d_gate = dz * up * SiLU'(gate), d_up = dz * SiLU(gate), SiLU'(a) = s + a s (1 - s), s = sigma(a)."""
+    y = bf16_to_f64(y_pre_bits)
+    gi, ui = _blocks32(y.shape[1])
+    a, u = y[:, gi], y[:, ui]
+    e = np.exp(-np.abs(a))
+    s = np.where(a > 0, 1.0 / (1.0 + e), e / (1.0 + e))
+    out = np.empty_like(y)
+    out[:, gi] = dz * u * (s + a * s * (1.0 - s))
+    out[:, ui] = dz * silu(a)
+    return out
+
+
 class OracleStack:
     def __init__(self, w_bits, x_base_bits, target_bits, lr=1e-3, history=False, margin=0):
         """history: quantise every activation and gradient with the bias of Eq. 3 for that tensor's amax at the

@@ -73,7 +73,10 @@ struct GemmParams {
     int tma_out;                  // epilogue goes through shared memory and TMA stores (needs vec_ok)
     int act;                      // 0: plain epilogue.  Otherwise a second tensor z leaves with the output (out may be
                                   // NULL): 1: z = GELU of the bf16-rounded output; 2: z = the bf16-rounded output times
-                                  // GELU'(aux); 3: z = the bf16-rounded output itself
+                                  // GELU'(aux); 3: z = the bf16-rounded output itself; 4: SwiGLU, the output's columns are
+                                  // blocks of 32 gate columns followed by their 32 up columns and z[M, N/2] =
+                                  // SiLU(gate) * up; 5: SwiGLU backward, the output is dz[M, N], aux[M, 2N] the stored
+                                  // gate/up pre-activations in that block layout, z[M, 2N] their gradients likewise
     const void *aux;              // act == 2: [M, N] bf16, the pre-activation whose derivative scales the gradient
     int has_out2;                 // z is stored as bf16 through the second output map
     uint8_t *out8;                // or NULL: z also leaves as FP8 bytes [M, N], scaled by a bias known beforehand
@@ -396,13 +399,9 @@ __device__ __forceinline__ float gelu_grad_f32(float x)
     return fmaf(x * (0.3989422804014327f * kTwoM32), gauss_2p32, cdf);
 }
 
-// 32 bf16 gradient values times GELU'(pre-activation), in FP32; `aux_row` points at the 32 pre-activations.
-__device__ __forceinline__ void gelu_backward_words(const uint32_t (&w)[16], const uint16_t *aux_row, bool ok,
-                                                    float (&v)[32])
+// 32 bf16 gradient values times GELU'(pre-activation), in FP32; `a` holds the 32 bf16 pre-activations.
+__device__ __forceinline__ void gelu_backward_words(const uint32_t (&w)[16], const uint4 (&a)[4], float (&v)[32])
 {
-    uint4 a[4];
-#pragma unroll
-    for (int j = 0; j < 4; ++j) a[j] = ok ? __ldg(reinterpret_cast<const uint4 *>(aux_row) + j) : make_uint4(0, 0, 0, 0);
     const uint32_t *aw = reinterpret_cast<const uint32_t *>(a);
 #pragma unroll
     for (int i = 0; i < 16; ++i) {
@@ -410,6 +409,34 @@ __device__ __forceinline__ void gelu_backward_words(const uint32_t (&w)[16], con
         v[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u) * gelu_grad_f32(__uint_as_float(aw[i] & 0xFFFF0000u));
     }
 }
+
+// sigma(a) = 1 / (1 + exp(-a)) with its relative accuracy kept in the negative tail: for a <= 0 it is e / (1 + e),
+// e = exp(a), and e is taken 2^32 too large so that the hardware exponential (which flushes below 2^-126) stays in
+// range down to where a * sigma(a) falls below the smallest bf16 subnormal.  Returns r = 1 / (1 + exp(-|a|)) and
+// e_2p32 = 2^32 exp(-|a|); sigma(a) = r for a > 0, e_2p32 * r * 2^-32 otherwise.
+__device__ __forceinline__ float sigmoid_parts(float a, float &e_2p32)
+{
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e_2p32) : "f"(fmaf(fabsf(a), -1.4426950408889634f, 32.0f)));
+    return rcp_approx(fmaf(e_2p32, kTwoM32, 1.0f));
+}
+// SiLU(a) = a * sigma(a)
+__device__ __forceinline__ float silu_f32(float a)
+{
+    float e;
+    const float r = sigmoid_parts(a, e);
+    return a > 0.0f ? a * r : (a * e * r) * kTwoM32;
+}
+// SiLU(a) and d/da SiLU(a) = sigma + a sigma (1 - sigma)
+__device__ __forceinline__ void silu_and_grad_f32(float a, float &silu, float &grad)
+{
+    float e;
+    const float r = sigmoid_parts(a, e);
+    const float sg = a > 0.0f ? r : (e * r) * kTwoM32;
+    silu = a > 0.0f ? a * r : (a * e * r) * kTwoM32;
+    grad = fmaf(silu, 1.0f - sg, sg);
+}
+__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
 
 // One warp's share (32 rows x BN columns) of a finished accumulator.
 //   t_row        TMEM address of this warp's lanes at the accumulator's first column
@@ -445,6 +472,181 @@ __device__ __forceinline__ void epilogue_tile(const CUtensorMap *map_out, const 
     }
     const bool rows_in = row0 < p.M;
     const bool row_ok = row0 + lane < p.M;
+    if constexpr (ACT == 4) {
+        // SwiGLU forward.  Chunks of 32 accumulator columns alternate gate, up, gate, up ...; the gate chunk's bf16
+        // words wait in registers for their up chunk; 32 z values come out of every pair of chunks, so one slab row
+        // of z (64 columns) covers 128 accumulator columns.  Slabs 0 and 2 stage the pre-activation (alternating
+        // per 64 columns), slabs 1 and 3 stage z (alternating per 128 columns); one bulk group per 64 columns.
+        static_assert(NSLAB == 4, "SwiGLU epilogue needs four slabs per warp");
+        uint32_t dummy = 0, wg[16];
+        bool sat = false;
+        Pow2Pair scq = make_pow2_pair(0);
+        if (p.out8) scq = make_pow2_pair(__ldg(p.d_sq) + p.delta_q);
+        const int64_t ldz = p.ldo >> 1;
+#pragma unroll 1
+        for (int c = 0; c < BN; c += 32) {
+            const int h = (c >> 5) & 1, pc = c >> 6;
+            uint32_t r[32];
+            tmem_ld_x32(t_row + c, r);
+            tmem_ld_wait();
+            if (c + 32 >= BN) release();
+            const uint32_t slab_pre = warp_slabs + (pc & 1) * 2 * kSlabBytes;
+            const uint32_t slab_z = warp_slabs + (((pc >> 1) & 1) * 2 + 1) * kSlabBytes;
+            if (h == 0) {
+                if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+                __syncwarp();
+            }
+            const int col0 = col_base + c;
+            float v[32];
+            uint32_t w[16];
+            epilogue_values(r, col0, p, sc, two_step, v);
+            pack_bf16(v, col0, p, w, dummy, false);
+            if (p.out) {
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+                    slab_write(slab_pre, lane, 4 * h + j, w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
+            }
+            if (h == 0) {
+#pragma unroll
+                for (int i = 0; i < 16; ++i) wg[i] = w[i];
+                continue;
+            }
+            // up chunk: z = SiLU(gate) * up on the bf16-rounded pre-activations
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                v[2 * i] = silu_f32(bf16_lo(wg[i])) * bf16_lo(w[i]);
+                v[2 * i + 1] = silu_f32(bf16_hi(wg[i])) * bf16_hi(w[i]);
+            }
+            const bool in_n = col0 < p.N;  // N is a multiple of 64: a gate/up pair of chunks is whole or absent
+            uint32_t wz[16];
+            pack_bf16(v, col0, p, wz, amax_bits, row_ok && in_n);
+            const int zc = (col0 - 32) >> 1;  // first of the 32 z columns
+            if (p.has_out2) {
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+                    slab_write(slab_z, lane, 4 * (pc & 1) + j, wz[4 * j], wz[4 * j + 1], wz[4 * j + 2], wz[4 * j + 3]);
+            }
+            if (p.out8 && row_ok && in_n) {
+                uint32_t b8[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) b8[i] = cast4<FP8_E4, true>(wz[2 * i], wz[2 * i + 1], scq, sat);
+                uint8_t *dst = p.out8 + (int64_t)(row0 + lane) * ldz + zc;
+                reinterpret_cast<uint4 *>(dst)[0] = make_uint4(b8[0], b8[1], b8[2], b8[3]);
+                reinterpret_cast<uint4 *>(dst)[1] = make_uint4(b8[4], b8[5], b8[6], b8[7]);
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) {
+                if (rows_in && in_n && p.out) tma_store_only(map_out, slab_pre, col0 - 32, row0);
+                // the z slab leaves after its second half, or after its first when the tensor ends there
+                const bool last_half = (pc & 1) || col0 + 32 >= p.N;
+                const int z0 = (col_base + (pc & ~1) * 64) >> 1;
+                if (rows_in && p.has_out2 && last_half && z0 < (p.N >> 1)) tma_store_only(map_out2, slab_z, z0, row0);
+                asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+            }
+        }
+        if (__any_sync(0xFFFFFFFFu, sat) && lane == 0) atomicOr(p.d_status, (unsigned)FP8_FLAG_SATURATED);
+        return;
+    }
+    if constexpr (ACT == 5) {
+        // SwiGLU backward.  Every 32 accumulator columns (dz) give 64 output columns: the gradients of their 32
+        // gate and 32 up pre-activations, one full slab row.  Slabs 0 and 2 stage dz (alternating per 64 columns),
+        // slabs 1 and 3 the gradients (alternating per 32 columns); one bulk group per 32 columns.
+        static_assert(NSLAB == 4, "SwiGLU epilogue needs four slabs per warp");
+        uint32_t dummy = 0;
+        bool sat = false;
+        Pow2Pair scq = make_pow2_pair(0);
+        if (p.out8) scq = make_pow2_pair(__ldg(p.d_sq) + p.delta_q);
+        const int64_t ld2 = p.ldo * 2;
+        // the stored pre-activations of a chunk (32 gate values then 32 up values, 128 bytes per row) are requested
+        // one chunk ahead, so that their trip from memory overlaps the arithmetic of the chunk before
+        uint4 aux_next[8];
+        auto fetch_aux = [&](int c) {
+            const int col0 = col_base + c;
+            const bool ok = row_ok && col0 < p.N;
+            const uint4 *src = reinterpret_cast<const uint4 *>(reinterpret_cast<const uint16_t *>(p.aux) +
+                                                               (int64_t)(row0 + lane) * ld2 + 2 * (int64_t)col0);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) aux_next[j] = ok ? __ldg(src + j) : make_uint4(0, 0, 0, 0);
+        };
+        fetch_aux(0);
+#pragma unroll 1
+        for (int c = 0; c < BN; c += 32) {
+            const int h = (c >> 5) & 1, pc = c >> 6;
+            uint32_t r[32];
+            tmem_ld_x32(t_row + c, r);
+            uint4 aux_now[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) aux_now[j] = aux_next[j];
+            if (c + 32 < BN) fetch_aux(c + 32);
+            tmem_ld_wait();
+            if (c + 32 >= BN) release();
+            const uint32_t slab_dz = warp_slabs + (pc & 1) * 2 * kSlabBytes;
+            const uint32_t slab_g = warp_slabs + (h * 2 + 1) * kSlabBytes;
+            if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+            __syncwarp();
+            const int col0 = col_base + c;
+            const bool in_n = col0 < p.N;  // N is a multiple of 32: a chunk is whole or absent
+            float v[32];
+            uint32_t w[16];
+            epilogue_values(r, col0, p, sc, two_step, v);
+            pack_bf16(v, col0, p, w, dummy, false);
+            if (p.out) {
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+                    slab_write(slab_dz, lane, 4 * h + j, w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
+            }
+            // the stored pre-activations of these 32 features: 32 gate values then 32 up values, 128 bytes
+            const bool ok = row_ok && in_n;
+            uint32_t wgr[16], wur[16];
+            {
+                const uint32_t *ag = reinterpret_cast<const uint32_t *>(aux_now);  // 16 words of gate, 16 of up
+                float vg[32];
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                    float s0, d0, s1, d1;
+                    silu_and_grad_f32(bf16_lo(ag[i]), s0, d0);
+                    silu_and_grad_f32(bf16_hi(ag[i]), s1, d1);
+                    const float z0 = bf16_lo(w[i]), z1 = bf16_hi(w[i]);
+                    vg[2 * i] = z0 * bf16_lo(ag[16 + i]) * d0;
+                    vg[2 * i + 1] = z1 * bf16_hi(ag[16 + i]) * d1;
+                    v[2 * i] = z0 * s0;
+                    v[2 * i + 1] = z1 * s1;
+                }
+                pack_bf16(vg, col0, p, wgr, amax_bits, ok);
+                pack_bf16(v, col0, p, wur, amax_bits, ok);
+            }
+            if (p.has_out2) {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    slab_write(slab_g, lane, j, wgr[4 * j], wgr[4 * j + 1], wgr[4 * j + 2], wgr[4 * j + 3]);
+                    slab_write(slab_g, lane, 4 + j, wur[4 * j], wur[4 * j + 1], wur[4 * j + 2], wur[4 * j + 3]);
+                }
+            }
+            if (p.out8 && ok) {
+                uint32_t b8[16];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    b8[i] = cast4<FP8_E5, true>(wgr[2 * i], wgr[2 * i + 1], scq, sat);
+                    b8[8 + i] = cast4<FP8_E5, true>(wur[2 * i], wur[2 * i + 1], scq, sat);
+                }
+                uint4 *dst = reinterpret_cast<uint4 *>(p.out8 + (int64_t)(row0 + lane) * ld2 + 2 * (int64_t)col0);
+#pragma unroll
+                for (int j = 0; j < 4; ++j) dst[j] = make_uint4(b8[4 * j], b8[4 * j + 1], b8[4 * j + 2], b8[4 * j + 3]);
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) {
+                if (rows_in && in_n) {
+                    if (p.has_out2) tma_store_only(map_out2, slab_g, 2 * col0, row0);
+                    if (p.out && (h == 1 || col0 + 32 >= p.N)) tma_store_only(map_out, slab_dz, col0 - 32 * h, row0);
+                }
+                asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+            }
+        }
+        if (__any_sync(0xFFFFFFFFu, sat) && lane == 0) atomicOr(p.d_status, (unsigned)FP8_FLAG_SATURATED);
+        return;
+    }
     if (ACT) {
         // The pre-activation (optional) and the second tensor z leave together, 64 columns (one 128-byte slab row
         // each) at a time; the warp's slabs are used in pairs {pre, z} in rotation.  The loop body covers 32
@@ -454,11 +656,29 @@ __device__ __forceinline__ void epilogue_tile(const CUtensorMap *map_out, const 
         bool sat = false;
         Pow2Pair scq = make_pow2_pair(0);
         if (p.out8) scq = make_pow2_pair(__ldg(p.d_sq) + p.delta_q);
+        // ACT == 2: the stored pre-activations of a chunk (64 bytes per row) are requested one chunk ahead, so that
+        // their trip from memory overlaps the arithmetic of the chunk before
+        uint4 aux_next[4];
+        auto fetch_aux = [&](int c) {
+            const int col0 = col_base + c;
+            const bool ok = row_ok && col0 + 32 <= p.N;
+            const uint4 *src = reinterpret_cast<const uint4 *>(reinterpret_cast<const uint16_t *>(p.aux) +
+                                                               (int64_t)(row0 + lane) * p.ldo + col0);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) aux_next[j] = ok ? __ldg(src + j) : make_uint4(0, 0, 0, 0);
+        };
+        if (ACT == 2) fetch_aux(0);
 #pragma unroll 1
         for (int c = 0; c < BN; c += 32) {
             const int h = (c >> 5) & 1;  // which half of the slab rows
             uint32_t r[32];
             tmem_ld_x32(t_row + c, r);
+            uint4 aux_now[4];
+            if (ACT == 2) {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) aux_now[j] = aux_next[j];
+                if (c + 32 < BN) fetch_aux(c + 32);
+            }
             tmem_ld_wait();
             if (c + 32 >= BN) release();
             const uint32_t slab_pre = warp_slabs + (slab_count % kPairsOfSlabs) * 2 * kSlabBytes;
@@ -492,8 +712,7 @@ __device__ __forceinline__ void epilogue_tile(const CUtensorMap *map_out, const 
             } else {
                 // columns beyond N are clipped by the store; rows beyond M have no pre-activation to read
                 const bool ok = row_ok && col0 + 32 <= p.N;
-                gelu_backward_words(w, reinterpret_cast<const uint16_t *>(p.aux) + (int64_t)(row0 + lane) * p.ldo + col0,
-                                    ok, v);
+                gelu_backward_words(w, aux_now, v);
                 if (row_ok && !ok && col0 < p.N) {   // ragged last chunk: element by element
                     const uint16_t *ar = reinterpret_cast<const uint16_t *>(p.aux) + (int64_t)(row0 + lane) * p.ldo;
 #pragma unroll
@@ -1130,6 +1349,8 @@ cudaError_t configure_gemm_kernels(int max_smem_optin)
     if (e == cudaSuccess) e = set_smem_attributes<1>();
     if (e == cudaSuccess) e = set_smem_attributes<2>();
     if (e == cudaSuccess) e = set_smem_attributes<3>();
+    if (e == cudaSuccess) e = set_smem_attributes<4>();
+    if (e == cudaSuccess) e = set_smem_attributes<5>();
     if (e != cudaSuccess) return e;
     int sms = 0, dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess ||
@@ -1260,9 +1481,9 @@ static fp8_status_t run_gemm(fp8_ctx *ctx, const uint8_t *a, int a_fmt, bool a_m
     p.delta_q = delta_q;
     CUtensorMap map_out = map_a;  // placeholder when the staged epilogue is off (never dereferenced then)
     CUtensorMap map_out2 = map_a;
-    auto encode_out = [&](CUtensorMap *m, void *base) {
-        cuuint64_t dims[2] = {(cuuint64_t)N, (cuuint64_t)M};
-        cuuint64_t strides[1] = {(cuuint64_t)(N * esz)};
+    auto encode_out = [&](CUtensorMap *m, void *base, int64_t cols) {
+        cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)M};
+        cuuint64_t strides[1] = {(cuuint64_t)(cols * esz)};
         cuuint32_t box[2] = {(cuuint32_t)(128 / esz), 32};
         cuuint32_t estr[2] = {1, 1};
         return ctx->encode_tiled(m, esz == 2 ? CU_TENSOR_MAP_DATA_TYPE_UINT16 : CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, base,
@@ -1273,10 +1494,12 @@ static fp8_status_t run_gemm(fp8_ctx *ctx, const uint8_t *a, int a_fmt, bool a_m
         // the activated output always goes through the staged epilogue (callers have checked its alignment)
         p.tma_out = 1;
         p.vec_ok = 1;
-        if (out_act && !encode_out(&map_out2, out_act)) return FP8_ERR_CUDA;
-        if (out && !encode_out(&map_out, out)) return FP8_ERR_CUDA;
+        // the second tensor is as wide as the output, half as wide (SwiGLU) or twice as wide (its backward)
+        const int64_t cols2 = act == 4 ? N / 2 : (act == 5 ? 2 * N : N);
+        if (out_act && !encode_out(&map_out2, out_act, cols2)) return FP8_ERR_CUDA;
+        if (out && !encode_out(&map_out, out, N)) return FP8_ERR_CUDA;
     } else if (p.tma_out) {
-        if (!encode_out(&map_out, out)) return FP8_ERR_CUDA;
+        if (!encode_out(&map_out, out, N)) return FP8_ERR_CUDA;
     }
     p.d_amax_bits = reinterpret_cast<unsigned *>(d_amax_out);
     p.d_status = ctx->d_status;
@@ -1291,6 +1514,8 @@ static fp8_status_t run_gemm(fp8_ctx *ctx, const uint8_t *a, int a_fmt, bool a_m
         case 1: gemm_pair_kernel<1><<<grid, kGemmThreads, PairSmemAct::kDynamic, st>>>(map_a, map_b, map_out, map_out2, p); break;
         case 2: gemm_pair_kernel<2><<<grid, kGemmThreads, PairSmemAct::kDynamic, st>>>(map_a, map_b, map_out, map_out2, p); break;
         case 3: gemm_pair_kernel<3><<<grid, kGemmThreads, PairSmemAct::kDynamic, st>>>(map_a, map_b, map_out, map_out2, p); break;
+        case 4: gemm_pair_kernel<4><<<grid, kGemmThreads, PairSmemAct::kDynamic, st>>>(map_a, map_b, map_out, map_out2, p); break;
+        case 5: gemm_pair_kernel<5><<<grid, kGemmThreads, PairSmemAct::kDynamic, st>>>(map_a, map_b, map_out, map_out2, p); break;
         default: gemm_pair_kernel<0><<<grid, kGemmThreads, PairSmem::kDynamic, st>>>(map_a, map_b, map_out, map_out2, p); break;
         }
     } else {
@@ -1301,6 +1526,8 @@ static fp8_status_t run_gemm(fp8_ctx *ctx, const uint8_t *a, int a_fmt, bool a_m
         case 1: gemm_kernel<kBN, kStagesAct, 1><<<grid, kGemmThreads, kActDyn, st>>>(map_a, map_b, map_out, map_out2, p); break;
         case 2: gemm_kernel<kBN, kStagesAct, 2><<<grid, kGemmThreads, kActDyn, st>>>(map_a, map_b, map_out, map_out2, p); break;
         case 3: gemm_kernel<kBN, kStagesAct, 3><<<grid, kGemmThreads, kActDyn, st>>>(map_a, map_b, map_out, map_out2, p); break;
+        case 4: gemm_kernel<kBN, kStagesAct, 4><<<grid, kGemmThreads, kActDyn, st>>>(map_a, map_b, map_out, map_out2, p); break;
+        case 5: gemm_kernel<kBN, kStagesAct, 5><<<grid, kGemmThreads, kActDyn, st>>>(map_a, map_b, map_out, map_out2, p); break;
         default: {
             // may start while the launch before it drains (its own first instruction that reads memory waits)
             cudaLaunchAttribute attr[1];
@@ -1388,16 +1615,18 @@ fp8_status_t fp8_linear_fwd_act(fp8_ctx *ctx, const uint8_t *x8, const int32_t *
 {
     using namespace fp8lin;
     if (!ctx || !x8 || !d_bx || !w8 || !d_bw || !y_act) return FP8_ERR_NULL;
-    if ((int)conv < 0 || (int)conv > 1 || (int)bias_dt < 0 || (int)bias_dt > 2 || (int)act != (int)FP8_ACT_GELU)
+    if ((int)conv < 0 || (int)conv > 1 || (int)bias_dt < 0 || (int)bias_dt > 2 ||
+        ((int)act != (int)FP8_ACT_GELU && (int)act != (int)FP8_ACT_SWIGLU))
         return FP8_ERR_DTYPE;
     if (bias_vec && !out_dtype_ok(bias_dt)) return FP8_ERR_UNSUPPORTED;
     if (T <= 0 || K <= 0 || N <= 0) return FP8_ERR_SHAPE;
+    const bool swiglu = act == FP8_ACT_SWIGLU;
     if (!aligned16(x8) || !aligned16(w8) || (K % 16) != 0 || !aligned16(y_act) || (y_pre && !aligned16(y_pre)) ||
-        (N % 8) != 0)
+        (N % (swiglu ? 64 : 8)) != 0)
         return FP8_ERR_ALIGN;
     int delta = 2 * format_delta(FP8_E4, conv);
     return run_gemm(ctx, x8, FP8_E4, false, d_bx, w8, FP8_E4, false, d_bw, delta, bias_vec, bias_dt, y_pre, FP8_BF16,
-                    d_amax_act, T, N, K, (cudaStream_t)stream, 1, y_act);
+                    d_amax_act, T, N, K, (cudaStream_t)stream, swiglu ? 4 : 1, y_act);
 }
 
 fp8_status_t fp8_linear_dgrad(fp8_ctx *ctx, const uint8_t *dy8, const int32_t *d_bg, const uint8_t *w8,
@@ -1428,16 +1657,18 @@ fp8_status_t fp8_linear_dgrad_act(fp8_ctx *ctx, const uint8_t *dy8, const int32_
 {
     using namespace fp8lin;
     if (!ctx || !dy8 || !d_bg || (!w8 && !w8_t) || !d_bw || !y_pre || !dx_act) return FP8_ERR_NULL;
-    if ((int)conv < 0 || (int)conv > 1 || (int)act != (int)FP8_ACT_GELU) return FP8_ERR_DTYPE;
+    if ((int)conv < 0 || (int)conv > 1 || ((int)act != (int)FP8_ACT_GELU && (int)act != (int)FP8_ACT_SWIGLU))
+        return FP8_ERR_DTYPE;
     if (T <= 0 || K <= 0 || N <= 0) return FP8_ERR_SHAPE;
     const bool w_mn = (w8_t == nullptr);
     const uint8_t *w = w_mn ? w8 : w8_t;
+    const bool swiglu = act == FP8_ACT_SWIGLU;
     if (!aligned16(dy8) || !aligned16(w) || (N % 16) != 0 || (w_mn && (K % 16) != 0) || !aligned16(y_pre) ||
-        !aligned16(dx_act) || (dx && !aligned16(dx)) || (K % 8) != 0)
+        !aligned16(dx_act) || (dx && !aligned16(dx)) || (K % (swiglu ? 32 : 8)) != 0)
         return FP8_ERR_ALIGN;
     int delta = format_delta(FP8_E5, conv) + format_delta(FP8_E4, conv);
     return run_gemm(ctx, dy8, FP8_E5, false, d_bg, w, FP8_E4, w_mn, d_bw, delta, nullptr, 0, dx, FP8_BF16, d_amax_act, T,
-                    K, N, (cudaStream_t)stream, 2, dx_act, y_pre);
+                    K, N, (cudaStream_t)stream, swiglu ? 5 : 2, dx_act, y_pre);
 }
 
 fp8_status_t fp8_linear_fwd_q(fp8_ctx *ctx, const uint8_t *x8, const int32_t *d_bx, const uint8_t *w8,
@@ -1447,18 +1678,19 @@ fp8_status_t fp8_linear_fwd_q(fp8_ctx *ctx, const uint8_t *x8, const int32_t *d_
 {
     using namespace fp8lin;
     if (!ctx || !x8 || !d_bx || !w8 || !d_bw || !z8 || !d_bz) return FP8_ERR_NULL;
-    if ((int)conv < 0 || (int)conv > 1 || (int)bias_dt < 0 || (int)bias_dt > 2 ||
-        ((int)act != (int)FP8_ACT_NONE && (int)act != (int)FP8_ACT_GELU))
+    if ((int)conv < 0 || (int)conv > 1 || (int)bias_dt < 0 || (int)bias_dt > 2 || (int)act < (int)FP8_ACT_NONE ||
+        (int)act > (int)FP8_ACT_SWIGLU)
         return FP8_ERR_DTYPE;
     if (bias_vec && !out_dtype_ok(bias_dt)) return FP8_ERR_UNSUPPORTED;
     if (act == FP8_ACT_NONE && y_pre) return FP8_ERR_UNSUPPORTED;  // without an activation z is the output itself
     if (T <= 0 || K <= 0 || N <= 0) return FP8_ERR_SHAPE;
     if (!aligned16(x8) || !aligned16(w8) || (K % 16) != 0 || !aligned16(z8) || (z && !aligned16(z)) ||
-        (y_pre && !aligned16(y_pre)) || (N % 16) != 0)
+        (y_pre && !aligned16(y_pre)) || (N % (act == FP8_ACT_SWIGLU ? 64 : 16)) != 0)
         return FP8_ERR_ALIGN;
     int delta = 2 * format_delta(FP8_E4, conv);
+    const int kind = act == FP8_ACT_GELU ? 1 : (act == FP8_ACT_SWIGLU ? 4 : 3);
     return run_gemm(ctx, x8, FP8_E4, false, d_bx, w8, FP8_E4, false, d_bw, delta, bias_vec, bias_dt, y_pre, FP8_BF16,
-                    d_amax_z, T, N, K, (cudaStream_t)stream, act == FP8_ACT_GELU ? 1 : 3, z, nullptr, z8, d_bz, FP8_E4,
+                    d_amax_z, T, N, K, (cudaStream_t)stream, kind, z, nullptr, z8, d_bz, FP8_E4,
                     format_delta(FP8_E4, conv));
 }
 
@@ -1469,20 +1701,20 @@ fp8_status_t fp8_linear_dgrad_q(fp8_ctx *ctx, const uint8_t *dy8, const int32_t 
 {
     using namespace fp8lin;
     if (!ctx || !dy8 || !d_bg || (!w8 && !w8_t) || !d_bw || !g8 || !d_bq) return FP8_ERR_NULL;
-    if ((int)conv < 0 || (int)conv > 1 || ((int)act != (int)FP8_ACT_NONE && (int)act != (int)FP8_ACT_GELU))
+    if ((int)conv < 0 || (int)conv > 1 || (int)act < (int)FP8_ACT_NONE || (int)act > (int)FP8_ACT_SWIGLU)
         return FP8_ERR_DTYPE;
-    if (act == FP8_ACT_GELU && !y_pre) return FP8_ERR_NULL;
+    if (act != FP8_ACT_NONE && !y_pre) return FP8_ERR_NULL;
     if (act == FP8_ACT_NONE && (y_pre || dx)) return FP8_ERR_UNSUPPORTED;  // g is the input gradient itself
     if (T <= 0 || K <= 0 || N <= 0) return FP8_ERR_SHAPE;
     const bool w_mn = (w8_t == nullptr);
     const uint8_t *w = w_mn ? w8 : w8_t;
-    if (!aligned16(dy8) || !aligned16(w) || (N % 16) != 0 || (K % 16) != 0 || (y_pre && !aligned16(y_pre)) ||
-        !aligned16(g8) || (g && !aligned16(g)) || (dx && !aligned16(dx)))
+    if (!aligned16(dy8) || !aligned16(w) || (N % 16) != 0 || (K % (act == FP8_ACT_SWIGLU ? 32 : 16)) != 0 ||
+        (y_pre && !aligned16(y_pre)) || !aligned16(g8) || (g && !aligned16(g)) || (dx && !aligned16(dx)))
         return FP8_ERR_ALIGN;
     int delta = format_delta(FP8_E5, conv) + format_delta(FP8_E4, conv);
+    const int kind = act == FP8_ACT_GELU ? 2 : (act == FP8_ACT_SWIGLU ? 5 : 3);
     return run_gemm(ctx, dy8, FP8_E5, false, d_bg, w, FP8_E4, w_mn, d_bw, delta, nullptr, 0, dx, FP8_BF16, d_amax_g, T, K,
-                    N, (cudaStream_t)stream, act == FP8_ACT_GELU ? 2 : 3, g, y_pre, g8, d_bq, FP8_E5,
-                    format_delta(FP8_E5, conv));
+                    N, (cudaStream_t)stream, kind, g, y_pre, g8, d_bq, FP8_E5, format_delta(FP8_E5, conv));
 }
 
 fp8_status_t fp8_linear_wgrad(fp8_ctx *ctx, const uint8_t *dy8, const uint8_t *dy8_t, const int32_t *d_bg,

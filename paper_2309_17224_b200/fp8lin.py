@@ -24,6 +24,7 @@ CONV_PAPER, CONV_NATIVE = 0, 1
 BF16, F16, F32 = 0, 1, 2
 ACT_NONE = 0
 ACT_GELU = 1
+ACT_SWIGLU = 2
 FLAG_NONFINITE_AMAX, FLAG_ZERO_AMAX, FLAG_SATURATED, FLAG_TIMEOUT = 1, 2, 4, 8
 
 SYMBOLS = (
@@ -238,7 +239,7 @@ class Context:
     def linear_dgrad_act(self, dy8, d_bg, w8, w8_t, d_bw, y_pre, dx, dx_act, d_amax_act=None, act=ACT_GELU,
                          conv=CONV_PAPER):
         T, N = dy8.shape
-        K = dx_act.shape[1]
+        K = w8.shape[1] if w8 is not None else w8_t.shape[0]
         _check(_lib.fp8_linear_dgrad_act(self._h, _ptr(dy8), _ptr(d_bg), _ptr(w8), _ptr(w8_t), _ptr(d_bw), _ptr(y_pre),
                                          _ptr(dx), _ptr(dx_act), act, _ptr(d_amax_act), T, K, N, conv, _stream()),
                "fp8_linear_dgrad_act")
@@ -255,7 +256,7 @@ class Context:
     def linear_dgrad_q(self, dy8, d_bg, w8, w8_t, d_bw, g8, d_bq, y_pre=None, dx=None, g=None, d_amax_g=None,
                        act=ACT_NONE, conv=CONV_PAPER):
         T, N = dy8.shape
-        K = g8.shape[1]
+        K = w8.shape[1] if w8 is not None else w8_t.shape[0]
         _check(_lib.fp8_linear_dgrad_q(self._h, _ptr(dy8), _ptr(d_bg), _ptr(w8), _ptr(w8_t), _ptr(d_bw), act,
                                        _ptr(y_pre), _ptr(dx), _ptr(g), _ptr(g8), _ptr(d_bq), _ptr(d_amax_g), T, K, N,
                                        conv, _stream()), "fp8_linear_dgrad_q")

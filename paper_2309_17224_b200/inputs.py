@@ -185,3 +185,12 @@ def layer_tensors(wl: Workload, layer_index: int, device="cpu", seed: int = BASE
 def bits(t: torch.Tensor):
     """bf16 tensor -> numpy uint16 bit patterns (host)."""
     return t.detach().contiguous().view(torch.int16).cpu().numpy().view("uint16")
+
+
+def interleave32(gate: torch.Tensor, up: torch.Tensor) -> torch.Tensor:
+    """Rows of `gate` and `up` ([F, ...] each, F a multiple of 32) merged into [2F, ...] in blocks of 32 gate rows
+    followed by their 32 up rows: the weight layout the SwiGLU epilogue expects (pure data movement)."""
+    F = gate.shape[0]
+    assert up.shape == gate.shape and F % 32 == 0
+    rest = gate.shape[1:]
+    return torch.stack((gate.reshape(F // 32, 32, *rest), up.reshape(F // 32, 32, *rest)), dim=1).reshape(2 * F, *rest)

@@ -66,6 +66,14 @@ def gemm(ctx, shapes, iters=20):
                     ("->fp8 (bytes only)", lambda: ctx.linear_fwd_q(a, bias, b, bias, z8, bias)),
                     ("dgrad gelu'->fp8", lambda: ctx.linear_dgrad_q(dy, bias, b, None, bias, g8, bias, y_pre=pre,
                                                                      d_amax_g=amax, act=fp8lin.ACT_GELU)))
+            if N % 64 == 0 and K % 32 == 0:
+                zs = torch.empty((M, N // 2), dtype=torch.uint8, device="cuda")
+                gs = torch.empty((M, 2 * K), dtype=torch.uint8, device="cuda")
+                pre2 = torch.randn((M, 2 * K), device="cuda").to(torch.bfloat16)
+                runs += (("swiglu->fp8", lambda: ctx.linear_fwd_q(a, bias, b, bias, zs, bias, y_pre=y, d_amax_z=amax,
+                                                                  act=fp8lin.ACT_SWIGLU)),
+                         ("dgrad swiglu'->fp8", lambda: ctx.linear_dgrad_q(dy, bias, b, None, bias, gs, bias, y_pre=pre2,
+                                                                           d_amax_g=amax, act=fp8lin.ACT_SWIGLU)))
             for name, fn in runs:
                 for _ in range(3):
                     fn()

@@ -184,3 +184,146 @@ def test_quantised_output_argument_errors(ctx, lib):
     assert e.value.status == lib.ERR_NULL
     ctx.linear_fwd_q(x8, b, w8, b, z8, b, z=y)
     assert bool((y == 0).all()) and bool((z8 == 0).all()) and ctx.device_flags(clear=True) == 0
+
+
+def _interleaved_weight(ctx, F, K, conv, seed):
+    """A gate/up weight pair merged into the 32-row block layout, quantised on the GPU and by the oracle."""
+    gate = I.normal_bf16(F, K, 0.02, seed, 2, "cuda")
+    up = I.normal_bf16(F, K, 0.02, seed, 4, "cuda")
+    return Quantised(ctx, I.interleave32(gate, up).contiguous(), O.E4, conv)
+
+
+@pytest.mark.parametrize("T,K,F", [(256, 768, 384), (144, 272, 96), (400, 1040, 416), (64, 1024, 256), (300, 128, 32)])
+@pytest.mark.parametrize("conv", [O.CONV_PAPER, O.CONV_NATIVE])
+def test_forward_with_swiglu_epilogue(ctx, lib, T, K, F, conv):
+    """z = SiLU(gate) * up out of the forward epilogue (weight rows in blocks of 32 gate, 32 up): the
+    pre-activation meets the forward bar, z is within one bf16 ulp of float64 SwiGLU of the GPU's own
+    pre-activation bits, bytes / amax / saturation as for every quantised output."""
+    N = 2 * F
+    x = I.normal_bf16(T, K, 1.0, 6100 + T, 1, "cuda", outlier_frac=0.01, outlier_scale=50.0)
+    qx = Quantised(ctx, x, O.E4, conv)
+    qw = _interleaved_weight(ctx, F, K, conv, 6100 + T)
+    ref = O.linear_fwd_np(qx.ref, qx.shift, qw.ref, qw.shift)
+    exact = O.scaling_bias(O.amax(OS.swiglu_bits(ref.bf16)), O.E4, conv)
+    kept = None
+    for bias, clip in ((exact, None), (exact + 2, True), (exact - 3, False)):
+        y_pre = torch.full((T, N), float("nan"), dtype=torch.bfloat16, device="cuda")
+        z = torch.full((T, F), float("nan"), dtype=torch.bfloat16, device="cuda")
+        z8 = torch.full((T, F), 0xAA, dtype=torch.uint8, device="cuda")
+        amax_z = torch.full((1,), -1.0, dtype=torch.float32, device="cuda")
+        ctx.linear_fwd_q(qx.y, qx.bias, qw.y, qw.bias, z8, _dev_i32(bias), y_pre=y_pre, z=z, d_amax_z=amax_z,
+                         act=lib.ACT_SWIGLU, conv=conv)
+        assert_bf16_within_one_ulp(bits_of(y_pre), ref)
+        d = np.abs(bf16_ordinal(bits_of(z)) - bf16_ordinal(OS.swiglu_bits(bits_of(y_pre))))
+        assert d.max() <= 1, d.max()
+        if kept is None:
+            kept = bits_of(z)
+        else:
+            assert np.array_equal(bits_of(z), kept)
+        _check_bytes(ctx, lib, z, z8, amax_z, bias, O.E4, conv, clip)
+    # the unquantised twin gives the same z and amax; bytes alone give the same bytes
+    z2 = torch.full((T, F), float("nan"), dtype=torch.bfloat16, device="cuda")
+    amax2 = torch.zeros(1, dtype=torch.float32, device="cuda")
+    ctx.linear_fwd_act(qx.y, qx.bias, qw.y, qw.bias, None, z2, d_amax_act=amax2, act=lib.ACT_SWIGLU, conv=conv)
+    assert np.array_equal(bits_of(z2), kept) and float(amax2.item()) == float(amax_z.item())
+    z8_only = torch.full((T, F), 0x55, dtype=torch.uint8, device="cuda")
+    ctx.linear_fwd_q(qx.y, qx.bias, qw.y, qw.bias, z8_only, _dev_i32(exact - 3), act=lib.ACT_SWIGLU, conv=conv)
+    assert torch.equal(z8_only, z8)
+    assert ctx.device_flags(clear=True) == 0
+
+
+@pytest.mark.parametrize("T,F,N", [(256, 384, 768), (144, 96, 272), (400, 416, 1040), (16, 2048, 48), (300, 32, 128)])
+@pytest.mark.parametrize("layout", ["t", "mn"])
+def test_input_gradient_with_swiglu_backward_epilogue(ctx, lib, T, F, N, layout):
+    """dz[T, F] = dY8 . W8 (the down projection's input gradient); the epilogue turns it into the gradients of the
+    stored gate / up pre-activations [T, 2F] (block layout), their E5 bytes and amax."""
+    conv = O.CONV_PAPER
+    g = I.normal_bf16(T, N, 1e-3, 7100 + T, 3, "cuda")
+    w = I.normal_bf16(N, F, 0.02, 7100 + T, 2, "cuda")
+    qg, qw = Quantised(ctx, g, O.E5, conv), Quantised(ctx, w, O.E4, conv)
+    ref = O.linear_dgrad_np(qg.ref, qg.shift, qw.ref, qw.shift)
+    y_pre = I.normal_bf16(T, 2 * F, 2.0, 17, 9, "cuda")
+    exact = O.scaling_bias(O.amax(OS.f64_to_bf16(OS.swiglu_backward(OS.bf16_to_f64(ref.bf16), bits_of(y_pre)))), O.E5, conv)
+    w8, w8t = (None, qw.y_t) if layout == "t" else (qw.y, None)
+    for bias, clip in ((exact, None), (exact + 2, True), (exact - 4, False)):
+        dz = torch.full((T, F), float("nan"), dtype=torch.bfloat16, device="cuda")
+        gg = torch.full((T, 2 * F), float("nan"), dtype=torch.bfloat16, device="cuda")
+        g8 = torch.full((T, 2 * F), 0xAA, dtype=torch.uint8, device="cuda")
+        amax_g = torch.full((1,), -1.0, dtype=torch.float32, device="cuda")
+        ctx.linear_dgrad_q(qg.y, qg.bias, w8, w8t, qw.bias, g8, _dev_i32(bias), y_pre=y_pre, dx=dz, g=gg,
+                           d_amax_g=amax_g, act=lib.ACT_SWIGLU, conv=conv)
+        assert_bf16_within_one_ulp(bits_of(dz), ref)
+        want = OS.f64_to_bf16(OS.swiglu_backward(OS.bf16_to_f64(bits_of(dz)), bits_of(y_pre)))
+        d = np.abs(bf16_ordinal(bits_of(gg)) - bf16_ordinal(want))
+        assert d.max() <= 1, d.max()
+        _check_bytes(ctx, lib, gg, g8, amax_g, bias, O.E5, conv, clip)
+    gg2 = torch.full((T, 2 * F), float("nan"), dtype=torch.bfloat16, device="cuda")
+    ctx.linear_dgrad_act(qg.y, qg.bias, w8, w8t, qw.bias, y_pre, None, gg2, act=lib.ACT_SWIGLU, conv=conv)
+    assert torch.equal(gg2, gg)
+    assert ctx.device_flags(clear=True) == 0
+
+
+def test_swiglu_argument_errors(ctx, lib):
+    b = torch.zeros(1, dtype=torch.int32, device="cuda")
+    x8 = torch.zeros((32, 64), dtype=torch.uint8, device="cuda")
+    w8 = torch.zeros((96, 64), dtype=torch.uint8, device="cuda")            # N = 96 is not a multiple of 64
+    with pytest.raises(lib.Fp8Error) as e:
+        ctx.linear_fwd_q(x8, b, w8, b, torch.zeros((32, 48), dtype=torch.uint8, device="cuda"), b, act=lib.ACT_SWIGLU)
+    assert e.value.status == lib.ERR_ALIGN
+    dy8 = torch.zeros((32, 64), dtype=torch.uint8, device="cuda")
+    wd = torch.zeros((64, 48), dtype=torch.uint8, device="cuda")            # K = 48 is not a multiple of 32
+    pre = torch.zeros((32, 96), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(lib.Fp8Error) as e:
+        ctx.linear_dgrad_q(dy8, b, wd, None, b, torch.zeros((32, 96), dtype=torch.uint8, device="cuda"), b, y_pre=pre,
+                           act=lib.ACT_SWIGLU)
+    assert e.value.status == lib.ERR_ALIGN
+    with pytest.raises(lib.Fp8Error) as e:
+        ctx.linear_dgrad_q(dy8, b, torch.zeros((64, 64), dtype=torch.uint8, device="cuda"), None, b,
+                           torch.zeros((32, 128), dtype=torch.uint8, device="cuda"), b, act=lib.ACT_SWIGLU)  # no y_pre
+    assert e.value.status == lib.ERR_NULL
+    assert ctx.device_flags(clear=True) == 0
+
+
+def test_llama_mlp_block_forward_and_backward_chain(ctx, lib):
+    """gate_up (SwiGLU epilogue, FP8 bytes out) -> down -> dY -> down's input gradient (SwiGLU backward epilogue,
+    E5 bytes out) -> gate_up's weight and input gradients, all on bytes the epilogues wrote; every matmul is
+    checked against the oracle fed the GPU's own operand bytes, and the interleaved layouts must line up (the
+    gradient bytes [T, 2F] against the interleaved weight [2F, K])."""
+    conv = O.CONV_PAPER
+    T, K, F = 320, 256, 160
+    x = I.normal_bf16(T, K, 1.0, 91, 1, "cuda")
+    qx = Quantised(ctx, x, O.E4, conv)
+    qgu = _interleaved_weight(ctx, F, K, conv, 92)
+    qd = Quantised(ctx, I.normal_bf16(K, F, 0.05, 93, 2, "cuda"), O.E4, conv)      # down: F -> K
+    dev = dict(device="cuda")
+    y_pre = torch.empty((T, 2 * F), dtype=torch.bfloat16, **dev)
+    z = torch.empty((T, F), dtype=torch.bfloat16, **dev)
+    z8 = torch.empty((T, F), dtype=torch.uint8, **dev)
+    amax_z = torch.zeros(1, dtype=torch.float32, **dev)
+    bz = _dev_i32(4)
+    ctx.linear_fwd_q(qx.y, qx.bias, qgu.y, qgu.bias, z8, bz, y_pre=y_pre, z=z, d_amax_z=amax_z, act=lib.ACT_SWIGLU)
+    assert_codes_equal(u8(z8), O.cast(bits_of(z), 4 + 1, O.N_E4), O.N_E4)
+    out = torch.empty((T, K), dtype=torch.bfloat16, **dev)
+    ctx.linear_fwd(z8, bz, qd.y, qd.bias, out)
+    assert_bf16_within_one_ulp(bits_of(out), O.linear_fwd_np(u8(z8), 4 + 1, qd.ref, qd.shift))
+    # backward from a seeded output gradient
+    qdy = Quantised(ctx, I.normal_bf16(T, K, 1e-3, 94, 3, "cuda"), O.E5, conv)
+    g = torch.empty((T, 2 * F), dtype=torch.bfloat16, **dev)
+    g8 = torch.empty((T, 2 * F), dtype=torch.uint8, **dev)
+    dz = torch.empty((T, F), dtype=torch.bfloat16, **dev)
+    amax_g = torch.zeros(1, dtype=torch.float32, **dev)
+    dz_ref = O.linear_dgrad_np(qdy.ref, qdy.shift, qd.ref, qd.shift)
+    bq = O.scaling_bias(O.amax(OS.f64_to_bf16(OS.swiglu_backward(OS.bf16_to_f64(dz_ref.bf16), bits_of(y_pre)))), O.E5) - 1
+    ctx.linear_dgrad_q(qdy.y, qdy.bias, qd.y, None, qd.bias, g8, _dev_i32(bq), y_pre=y_pre, dx=dz, g=g, d_amax_g=amax_g,
+                       act=lib.ACT_SWIGLU)
+    assert_bf16_within_one_ulp(bits_of(dz), dz_ref)
+    assert_codes_equal(u8(g8), O.cast(bits_of(g), bq, O.N_E5), O.N_E5)
+    # gate_up's gradients from those bytes: dW[2F, K] keeps the weight's row layout, dX[T, K]
+    dw = torch.empty((2 * F, K), dtype=torch.bfloat16, **dev)
+    dx = torch.empty((T, K), dtype=torch.bfloat16, **dev)
+    bqt = _dev_i32(bq)
+    ctx.linear_wgrad(g8, None, bqt, qx.y, None, qx.bias, dw, T)
+    ctx.linear_dgrad(g8, bqt, qgu.y, None, qgu.bias, dx)
+    assert_bf16_within_one_ulp(bits_of(dw), O.linear_wgrad_np(u8(g8), bq, qx.ref, qx.shift))
+    assert_bf16_within_one_ulp(bits_of(dx), O.linear_dgrad_np(u8(g8), bq, qgu.ref, qgu.shift))
+    assert ctx.device_flags(clear=True) & ~lib.FLAG_SATURATED == 0

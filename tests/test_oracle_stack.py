@@ -106,3 +106,27 @@ def test_history_mode_uses_the_previous_steps_amax():
     r = big.step(1)
     dec = np.abs(O.decode_table(O.N_E4)[r["x8"][0]])
     assert dec.max() == 448.0 and (dec == 448.0).sum() > 1
+
+
+def test_swiglu_and_its_backward_against_torch_float64():
+    """SwiGLU on the 32-block layout against torch's float64 silu and autograd on de-interleaved tensors."""
+    rng = np.random.default_rng(11)
+    T, F = 24, 96
+    gate = torch.from_numpy(rng.standard_normal((T, F)) * 3).to(torch.bfloat16)
+    up = torch.from_numpy(rng.standard_normal((T, F))).to(torch.bfloat16)
+    gate[0, :6] = torch.tensor([-100.0, -60.0, -20.0, 0.0, 30.0, 90.0], dtype=torch.bfloat16)
+    from paper_2309_17224_b200.inputs import interleave32
+    y = interleave32(gate.T.contiguous(), up.T.contiguous()).T.contiguous()      # [T, 2F] in blocks of 32 columns
+    assert torch.equal(y[:, :32], gate[:, :32]) and torch.equal(y[:, 32:64], up[:, :32]) and torch.equal(y[:, 64:96], gate[:, 32:64])
+    g64 = gate.to(torch.float64).clone().requires_grad_(True)
+    u64 = up.to(torch.float64).clone().requires_grad_(True)
+    z = torch.nn.functional.silu(g64) * u64
+    want = z.detach().to(torch.float32).to(torch.bfloat16)
+    got = S.swiglu_bits(_bits(y))
+    assert np.abs(_ord(got) - _ord(_bits(want))).max() <= 1
+    dz = torch.from_numpy(rng.standard_normal((T, F)))
+    z.backward(dz)
+    back = S.swiglu_backward(dz.numpy(), _bits(y))
+    gi, ui = S._blocks32(2 * F)
+    np.testing.assert_allclose(back[:, gi], g64.grad.numpy(), rtol=1e-11, atol=1e-300)
+    np.testing.assert_allclose(back[:, ui], u64.grad.numpy(), rtol=1e-11, atol=1e-300)

@@ -7,7 +7,9 @@
 //   gemm_pair_kernel  (M > 128)  two CTAs of a cluster own one 256x256 tile;
 //                     tcgen05.mma.cta_group::2, six stages of 32 KB per CTA.
 //   gemm_kernel       (M <= 128: decode, skinny)  one CTA owns a 128x256 tile,
-//                     four stages of 48 KB, optional split of the contraction.
+//                     four stages of 48 KB, optional split of the contraction
+//                     (partial sums in an FP32 workspace, splitk_finalize_kernel
+//                     launched behind it as a programmatic dependent).
 //
 // Roles in both:
 //   warp 0, one lane   TMA producer: 128-byte-swizzled boxes of A and B into a
@@ -22,6 +24,12 @@
 //                      optional activation (second output) and amax, then
 //                      swizzled shared-memory slabs and TMA stores (or direct
 //                      stores for outputs whose rows are not 16-byte multiples).
+// The epilogue comes in six kinds, a template parameter of both kernels so that
+// each instantiation carries only its own arithmetic: plain; GELU forward; GELU
+// backward; identity; SwiGLU forward; SwiGLU backward.  The five fused kinds
+// write a second tensor z next to the (optional) matmul output -- as bf16
+// and / or as FP8 bytes under a bias known before the launch -- and its amax;
+// they run with one stage fewer and four staging slabs per epilogue warp.
 // The two accumulators let the epilogue of tile i overlap the main loop of
 // tile i+1.  An operand may be stored with the contraction index contiguous
 // ("K-major": X8[T,K], W8[N,K] in the forward pass) or with its M / N index

@@ -356,3 +356,45 @@ def test_fused_epilogue_argument_errors(ctx, lib):
     # a valid tiny call still works after the rejected ones
     ctx.linear_fwd_act(x8, b, w8, b, None, y)
     assert bool((y == 0).all()) and ctx.device_flags(clear=True) & lib.FLAG_TIMEOUT == 0
+
+
+@pytest.mark.parametrize("T", [16, 512])
+def test_a_layer_replayed_from_a_cuda_graph_matches_the_eager_run(ctx, lib, T):
+    """Quantise X (amax + bias + cast), forward matmul with output amax, for a decode-size batch (single launch
+    cast, split contraction, finalize and matmul launched as programmatic dependents) and a training-size one:
+    captured once, replayed on fresh inputs, the results must equal the eager calls' bit for bit."""
+    K, N = 2048, 1536
+    w = I.normal_bf16(N, K, 0.02, 55, 2, "cuda")
+    qw = Quantised(ctx, w, O.E4, O.CONV_PAPER)
+    x = torch.empty((T, K), dtype=torch.bfloat16, device="cuda")
+    x8 = torch.empty((T, K), dtype=torch.uint8, device="cuda")
+    ax = torch.zeros(1, dtype=torch.float32, device="cuda")
+    bx = torch.zeros(1, dtype=torch.int32, device="cuda")
+    y = torch.empty((T, N), dtype=torch.bfloat16, device="cuda")
+    ay = torch.zeros(1, dtype=torch.float32, device="cuda")
+
+    def layer():
+        ctx.cast_e4(x, None, d_amax_out=ax, d_bias_out=bx, y=x8)
+        ctx.linear_fwd(x8, bx, qw.y, qw.bias, y, d_amax_y=ay)
+
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        x.copy_(I.normal_bf16(T, K, 1.0, 56, 1, "cuda"))
+        layer()
+        with torch.cuda.graph(g, stream=side):
+            layer()
+    torch.cuda.current_stream().wait_stream(side)
+    for seed, scale in ((57, 1.0), (58, 300.0), (59, 0.004)):
+        x.copy_(I.normal_bf16(T, K, scale, seed, 1, "cuda"))
+        g.replay()
+        torch.cuda.synchronize()
+        got = (y.clone(), x8.clone(), float(ax.item()), int(bx.item()), float(ay.item()))
+        y.zero_(); x8.zero_(); ax.zero_(); bx.zero_(); ay.zero_()
+        layer()
+        torch.cuda.synchronize()
+        assert torch.equal(got[0], y) and torch.equal(got[1], x8)
+        assert got[2:] == (float(ax.item()), int(bx.item()), float(ay.item()))
+        assert got[3] == O.scaling_bias(O.amax(bits_of(x)), O.E4)
+    assert ctx.device_flags(clear=True) & lib.FLAG_TIMEOUT == 0

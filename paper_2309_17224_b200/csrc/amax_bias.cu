@@ -88,6 +88,9 @@ template <int DT>
 __global__ void __launch_bounds__(kAmaxThreads) amax_flat_kernel(const uint4 *__restrict__ x, int64_t nvec, int ntail,
                                                                  AmaxOut o)
 {
+    // the cast launched behind this kernel as a programmatic dependent may take its places as blocks here retire;
+    // it reads nothing before this grid has completed
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     uint32_t acc = 0;
     const int64_t chunk = (int64_t)kAmaxThreads * kAmaxUnroll;
     for (int64_t base = (int64_t)blockIdx.x * chunk; base < nvec; base += (int64_t)gridDim.x * chunk) {
@@ -117,6 +120,7 @@ __global__ void __launch_bounds__(kAmaxThreads) amax_rows_kernel(const void *__r
 {
     constexpr int kPerVec = DT == FP8_F32 ? 4 : 8;
     constexpr int kB = DT == FP8_F32 ? 4 : 2;
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     uint32_t acc = 0;
     for (int64_t r = blockIdx.x; r < rows; r += gridDim.x) {
         int64_t done = 0;

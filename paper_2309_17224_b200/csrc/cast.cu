@@ -65,6 +65,8 @@ __global__ void __launch_bounds__(1024) cast_flat_kernel(const uint4 *__restrict
                                                                  const int32_t *__restrict__ d_bias, int delta,
                                                                  unsigned *d_status, const unsigned *redo)
 {
+    // launched as a programmatic dependent of the amax kernel: nothing it wrote is read before it has completed
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     // as the second launch of a predicted cast: nothing to do when the prediction held
     if (redo != nullptr && *reinterpret_cast<const volatile unsigned *>(redo) == 0u) return;
     const int s = __ldg(d_bias) + delta;
@@ -97,6 +99,7 @@ __global__ void __launch_bounds__(kCastThreads) cast_tile_kernel(const void *__r
     constexpr int kW = InType<DT>::kWords4;  // words per four input elements
     constexpr int kB = InType<DT>::kBytes;
 
+    asm volatile("griddepcontrol.wait;" ::: "memory");  // see cast_flat_kernel
     const int s = __ldg(d_bias) + delta;
     const Pow2Pair p = make_pow2_pair(s);
     bool sat = false;
@@ -185,18 +188,16 @@ static cudaError_t launch_cast(fp8_ctx *ctx, const void *x, int64_t rows, int64_
         int64_t want = (nout + chunk - 1) / chunk;
         int max_blocks = ctx->sm_count * 8;
         int blocks = (int)(want < 1 ? 1 : (want > max_blocks ? max_blocks : want));
-        cast_flat_kernel<FMT, DT><<<blocks, kCastThreads, 0, stream>>>(reinterpret_cast<const uint4 *>(x),
-                                                                       reinterpret_cast<uint4 *>(y), nout, ntail,
-                                                                       d_bias, delta, ctx->d_status, nullptr);
-        return cudaGetLastError();
+        return launch_dependent(cast_flat_kernel<FMT, DT>, blocks, kCastThreads, stream, reinterpret_cast<const uint4 *>(x),
+                                reinterpret_cast<uint4 *>(y), nout, ntail, d_bias, delta, ctx->d_status,
+                                static_cast<const unsigned *>(nullptr));
     }
     int fast_ok = al(x, 4 * kB) && (ld % 4) == 0 && (!y || (al(y, 4) && (cols % 4) == 0)) &&
                   (!y_t || (al(y_t, 4) && (rows % 4) == 0));
     int64_t tiles = ((rows + kTile - 1) / kTile) * ((cols + kTile - 1) / kTile);
     if (tiles > 0x7FFFFFFF) return cudaErrorInvalidValue;
-    cast_tile_kernel<FMT, DT><<<(unsigned)tiles, kCastThreads, 0, stream>>>(x, rows, cols, ld, d_bias, delta, y, y_t,
-                                                                            fast_ok, ctx->d_status);
-    return cudaGetLastError();
+    return launch_dependent(cast_tile_kernel<FMT, DT>, (unsigned)tiles, kCastThreads, stream, x, rows, cols, ld, d_bias, delta,
+                            y, y_t, fast_ok, ctx->d_status);
 }
 
 template <int FMT>

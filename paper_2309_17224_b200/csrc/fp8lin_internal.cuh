@@ -80,6 +80,24 @@ __host__ __device__ inline int bias_from_amax_bits(uint32_t bits, int fmt, int c
     return e_max - e - (frac > frac_max ? 1 : 0) - margin;
 }
 
+// Launch allowed to start while the launch before it on the stream drains (programmatic dependent launch); the
+// kernel itself waits (griddepcontrol.wait) before it touches anything an earlier launch may have written.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_dependent(void (*kernel)(KArgs...), unsigned grid, unsigned block, cudaStream_t stream,
+                                    Args... args)
+{
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(block);
+    cfg.stream = stream;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 cudaError_t launch_amax_bias(fp8_ctx *ctx, const void *x, int dt, int64_t rows, int64_t cols, int64_t ld, float *d_amax,
                              int32_t *d_bias, int fmt, int conv, int margin, cudaStream_t stream);
 

@@ -65,7 +65,9 @@ __global__ void __launch_bounds__(1024) cast_flat_kernel(const uint4 *__restrict
                                                                  const int32_t *__restrict__ d_bias, int delta,
                                                                  unsigned *d_status, const unsigned *redo)
 {
-    // launched as a programmatic dependent of the amax kernel: nothing it wrote is read before it has completed
+    // launched as a programmatic dependent of the amax kernel: nothing it wrote is read before it has completed;
+    // the matmul behind this kernel may in turn take its places as blocks here retire
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     asm volatile("griddepcontrol.wait;" ::: "memory");
     // as the second launch of a predicted cast: nothing to do when the prediction held
     if (redo != nullptr && *reinterpret_cast<const volatile unsigned *>(redo) == 0u) return;
@@ -99,7 +101,8 @@ __global__ void __launch_bounds__(kCastThreads) cast_tile_kernel(const void *__r
     constexpr int kW = InType<DT>::kWords4;  // words per four input elements
     constexpr int kB = InType<DT>::kBytes;
 
-    asm volatile("griddepcontrol.wait;" ::: "memory");  // see cast_flat_kernel
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");  // see cast_flat_kernel
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const int s = __ldg(d_bias) + delta;
     const Pow2Pair p = make_pow2_pair(s);
     bool sat = false;

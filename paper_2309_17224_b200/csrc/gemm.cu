@@ -1149,6 +1149,9 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             uint32_t it = 0;
             bool alive = true;
             const uint32_t leader_full0 = map_to_cta(full_bar(0), 0);
+            // launched as a programmatic dependent of the cast before it: set-up above overlaps that grid's tail,
+            // its bytes are not requested before it has completed
+            asm volatile("griddepcontrol.wait;" ::: "memory");
             for (int tile = pair_id; alive && tile < num_tiles; tile += num_pairs) {
                 int m_blk, n_blk;
                 tile_coords(tile, p, m_blk, n_blk);
@@ -1198,6 +1201,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             }
         }
     } else {
+        asm volatile("griddepcontrol.wait;" ::: "memory");  // the biases (and aux) may come from the launch before
         const int q = warp & 3;
         const int e = -(__ldg(p.d_sa) + __ldg(p.d_sb) + p.delta_sum);
         const Pow2Pair sc = make_pow2_pair(e);
@@ -1525,7 +1529,21 @@ static fp8_status_t run_gemm(fp8_ctx *ctx, const uint8_t *a, int a_fmt, bool a_m
         case 3: gemm_pair_kernel<3><<<grid, kGemmThreads, PairSmemAct::kDynamic, st>>>(map_a, map_b, map_out, map_out2, p); break;
         case 4: gemm_pair_kernel<4><<<grid, kGemmThreads, PairSmemAct::kDynamic, st>>>(map_a, map_b, map_out, map_out2, p); break;
         case 5: gemm_pair_kernel<5><<<grid, kGemmThreads, PairSmemAct::kDynamic, st>>>(map_a, map_b, map_out, map_out2, p); break;
-        default: gemm_pair_kernel<0><<<grid, kGemmThreads, PairSmem::kDynamic, st>>>(map_a, map_b, map_out, map_out2, p); break;
+        default: {
+            cudaLaunchAttribute attr[1];
+            attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+            attr[0].val.programmaticStreamSerializationAllowed = 1;
+            cudaLaunchConfig_t cfg = {};
+            cfg.gridDim = grid;
+            cfg.blockDim = dim3(kGemmThreads);
+            cfg.dynamicSmemBytes = PairSmem::kDynamic;
+            cfg.stream = st;
+            cfg.attrs = attr;
+            cfg.numAttrs = 1;
+            if (cudaLaunchKernelEx(&cfg, gemm_pair_kernel<0>, map_a, map_b, map_out, map_out2, p) != cudaSuccess)
+                return FP8_ERR_CUDA;
+            break;
+        }
         }
     } else {
         int items = tiles * p.splits;

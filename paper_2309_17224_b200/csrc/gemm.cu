@@ -72,6 +72,7 @@ struct GemmParams {
     const int32_t *d_sa, *d_sb;   // paper-convention biases of the two operands
     int delta_sum;                // format shifts to add to them
     int a_mn, b_mn;               // operand stored with its M / N index contiguous (contraction index strided)
+    int a_box_bytes;              // single-CTA kernel: bytes one A load brings (its box holds only the rows that exist)
     const void *bias_vec;         // [N] or NULL
     int bias_dt;
     void *out;
@@ -210,6 +211,12 @@ __device__ __forceinline__ void tile_coords(int tile, const GemmParams &p, int &
     const int r = tile - g * group;
     m_blk = first_m + r % gm;
     n_blk = r / gm;
+}
+
+// Where in its k-range a tile of the single-CTA kernel starts (it wraps around): a different place per tile.
+__device__ __forceinline__ int first_kblock(int m_blk, int n_blk, int len)
+{
+    return (int)(((unsigned)n_blk * 7u + (unsigned)m_blk * 3u) % (unsigned)len);
 }
 
 // One 32-column chunk of one accumulator row: unscale by the exact power of
@@ -863,11 +870,23 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_b)) : "memory");
             uint32_t it = 0;
             bool alive = true;
+            // One row of tiles (decode): every B byte is read exactly once, every A byte by every CTA.  B is marked
+            // to leave L2 first and A to stay: without the hints the few lines of A can lose their place to the
+            // streaming weights and every CTA then fetches them from one DRAM page (measured: 88 -> 140 us for a
+            // 470 MB weight, depending on where the activation happened to be allocated).
+            const bool stream_b = p.tiles_m == 1;
+            const uint64_t keep = l2_policy_evict_last(), drop = l2_policy_evict_first();
             auto load_b = [&](int s, int n_blk, int k) {
                 const uint32_t b_dst = smem_base + s * L::kStageBytes + L::kABytes;
                 if (p.b_mn) {  // two blocks of 128 N values, 16 KB apart
-                    for (int h = 0; h < BN / 128; ++h)
-                        tma_load_2d(b_dst + h * (128 * kBK), &map_b, full_bar(s), n_blk * BN + h * 128, k * kBK);
+                    for (int h = 0; h < BN / 128; ++h) {
+                        if (stream_b)
+                            tma_load_2d_hint(b_dst + h * (128 * kBK), &map_b, full_bar(s), n_blk * BN + h * 128, k * kBK, drop);
+                        else
+                            tma_load_2d(b_dst + h * (128 * kBK), &map_b, full_bar(s), n_blk * BN + h * 128, k * kBK);
+                    }
+                } else if (stream_b) {
+                    tma_load_2d_hint(b_dst, &map_b, full_bar(s), k * kBK, n_blk * BN, drop);
                 } else {
                     tma_load_2d(b_dst, &map_b, full_bar(s), k * kBK, n_blk * BN);
                 }
@@ -879,8 +898,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                 int m_blk, n_blk;
                 tile_coords((int)blockIdx.x / p.splits, p, m_blk, n_blk);
                 const int k0 = ((int)blockIdx.x % p.splits) * p.kb_per_split;
-                const int k1 = min(p.num_k, k0 + min(p.kb_per_split, STAGES));
-                for (int k = k0; k < k1; ++k) {
+                const int k1 = min(p.num_k, k0 + p.kb_per_split);
+                int k = k0 + first_kblock(m_blk, n_blk, k1 - k0);
+                for (int i = 0; i < min(k1 - k0, STAGES); ++i, k = (k + 1 == k1) ? k0 : k + 1) {
                     if (p.b_mn) {
                         for (int h = 0; h < BN / 128; ++h) tma_prefetch_l2_2d(&map_b, n_blk * BN + h * 128, k * kBK);
                     } else {
@@ -894,14 +914,23 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                 tile_coords(item / p.splits, p, m_blk, n_blk);
                 const int k0 = (item % p.splits) * p.kb_per_split;
                 const int k1 = min(p.num_k, k0 + p.kb_per_split);
-                for (int k = k0; k < k1; ++k, ++it) {
+                // The k-blocks of an item are taken in a rotated order that differs from tile to tile: with a few
+                // rows of A, all CTAs walking k in step would ask L2 for the same 128-byte lines at the same time
+                // (measured on 1 to 8 rows: 103-109 us against 83-86 us for a 470 MB weight).
+                int k = k0 + first_kblock(m_blk, n_blk, k1 - k0);
+                for (int i = 0; i < k1 - k0; ++i, ++it, k = (k + 1 == k1) ? k0 : k + 1) {
                     const int s = it % STAGES;
                     const uint32_t ph = (it / STAGES) & 1u;
                     if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p.d_status)) { alive = false; break; }
-                    mbar_expect_tx(full_bar(s), L::kStageBytes);
+                    mbar_expect_tx(full_bar(s), (uint32_t)p.a_box_bytes + L::kBBytes);
                     const uint32_t a_dst = smem_base + s * L::kStageBytes;
-                    if (p.a_mn) tma_load_2d(a_dst, &map_a, full_bar(s), m_blk * kBM, k * kBK);
-                    else tma_load_2d(a_dst, &map_a, full_bar(s), k * kBK, m_blk * kBM);
+                    if (stream_b) {
+                        if (p.a_mn) tma_load_2d_hint(a_dst, &map_a, full_bar(s), m_blk * kBM, k * kBK, keep);
+                        else tma_load_2d_hint(a_dst, &map_a, full_bar(s), k * kBK, m_blk * kBM, keep);
+                    } else {
+                        if (p.a_mn) tma_load_2d(a_dst, &map_a, full_bar(s), m_blk * kBM, k * kBK);
+                        else tma_load_2d(a_dst, &map_a, full_bar(s), k * kBK, m_blk * kBM);
+                    }
                     load_b(s, n_blk, k);
                 }
             }
@@ -1334,6 +1363,8 @@ constexpr int kStages = 4;
 static bool g_force_single = false;  // set from FP8LIN_SINGLE_CTA=1 (A/B comparison of the two kernels)
 static int g_group_m = 0;               // set from FP8LIN_GROUP_M (experiments with the tile order)
 static bool g_no_splitk = false;        // set from FP8LIN_NO_SPLITK=1
+static int g_force_splits = 0;          // set from FP8LIN_SPLITS (experiments with the split count)
+static bool g_no_pdl = false;           // set from FP8LIN_NO_PDL=1 (A/B: matmuls launched without programmatic dependence)
 static bool g_direct_epilogue = false;  // set from FP8LIN_DIRECT_EPILOGUE=1 (A/B comparison of the epilogues)
 static int g_max_pairs = 0;  // CTA pairs that can be resident at once (0: pair kernel unavailable)
 
@@ -1390,6 +1421,10 @@ cudaError_t configure_gemm_kernels(int max_smem_optin)
     g_force_single = env && env[0] == '1';
     env = getenv("FP8LIN_GROUP_M");
     g_group_m = env ? atoi(env) : 0;
+    env = getenv("FP8LIN_NO_PDL");
+    g_no_pdl = env && env[0] == '1';
+    env = getenv("FP8LIN_SPLITS");
+    g_force_splits = env ? atoi(env) : 0;
     env = getenv("FP8LIN_NO_SPLITK");
     g_no_splitk = env && env[0] == '1';
     env = getenv("FP8LIN_DIRECT_EPILOGUE");
@@ -1426,7 +1461,11 @@ static fp8_status_t run_gemm(fp8_ctx *ctx, const uint8_t *a, int a_fmt, bool a_m
     const bool pair = g_max_pairs > 0 && M > kBM && !g_force_single;
     CUtensorMap map_a, map_b;
     // an operand stored [Kc, M or N] is fetched as boxes of 128 contraction rows x 128 bytes
-    const bool ok_a = a_mn ? encode_map(ctx, &map_a, a, Kc, M, kBK) : encode_map(ctx, &map_a, a, M, Kc, kBM);
+    // With a few rows of A (decode) the box covers those rows only, rounded up to the 8-row swizzle atom: the other
+    // rows of the stage keep whatever they held and feed output rows that are never stored.  (A 128-row box on a
+    // one-row tensor cost 6 us of a 89 us launch, and 59 us for some placements of the activation in memory.)
+    const int a_box_rows = (!pair && !a_mn && M < kBM) ? (int)((M + 7) / 8 * 8) : kBM;
+    const bool ok_a = a_mn ? encode_map(ctx, &map_a, a, Kc, M, kBK) : encode_map(ctx, &map_a, a, M, Kc, a_box_rows);
     const bool ok_b = b_mn ? encode_map(ctx, &map_b, b, Kc, N, kBK)
                            : encode_map(ctx, &map_b, b, N, Kc, pair ? kPairHalfN : kBN);
     if (!ok_a || !ok_b) return FP8_ERR_CUDA;
@@ -1434,6 +1473,7 @@ static fp8_status_t run_gemm(fp8_ctx *ctx, const uint8_t *a, int a_fmt, bool a_m
     p.group_m = g_group_m > 0 ? g_group_m : kGroupM;
     p.a_mn = a_mn ? 1 : 0;
     p.b_mn = b_mn ? 1 : 0;
+    p.a_box_bytes = a_box_rows * kBK;
     p.M = (int)M; p.N = (int)N; p.K = (int)Kc;
     p.tiles_m = (int)((M + (pair ? 256 : kBM) - 1) / (pair ? 256 : kBM));
     p.tiles_n = (int)((N + kBN - 1) / kBN);
@@ -1447,20 +1487,19 @@ static fp8_status_t run_gemm(fp8_ctx *ctx, const uint8_t *a, int a_fmt, bool a_m
     if (!pair && !g_no_splitk && !act) {
         const int64_t tiles = (int64_t)p.tiles_m * p.tiles_n;
         if (tiles < 2 * ctx->sm_count && p.num_k >= 8) {
-            // Pick the split count by a byte model of the launch: the busiest CTA streams
-            // ceil(items / SMs) items of kb k-blocks each (one B tile of BN x 128 bytes per k-block; the A
-            // tile is a few rows), every split also writes and re-reads an FP32 partial tile, each item has
-            // a fixed set-up cost and splitting at all costs the finalize launch.  This avoids counts that
-            // leave the last wave nearly empty (448 items on 148 SMs) or move more partial sums than weights.
-            // (Dealing k-blocks evenly to the SMs, stream-K, was measured and lost to this: its extra partial
-            // tiles cost more than the imbalance it removes, because a thin last wave runs at more than its
-            // share of the HBM bandwidth.)
+            // Pick the split count by a byte model of the launch, in bytes at the HBM rate.  The weights stream once
+            // (one B tile of BN x 128 bytes per k-block; the A tile is a few rows) and every split writes and
+            // re-reads an FP32 partial tile: that is the floor when all SMs pull together.  One SM alone draws at
+            // most about 1.6 times its fair share of the HBM rate (measured: 32 to 40 CTAs streaming 2 MB each),
+            // so the busiest CTA's bytes set a second floor, which is what splitting lowers.  Each wave of items
+            // has a fixed set-up cost and splitting at all costs the finalize launch.
             const int64_t by_k = p.num_k / 4;
             const int64_t by_ws = (int64_t)(ctx->partial_bytes / sizeof(float)) / (M * N);
             int64_t cap = by_k < by_ws ? by_k : by_ws;
             if (cap > 64) cap = 64;
             const double sms = (double)ctx->sm_count;
-            const double kb_bytes = (double)kBN * kBK, item_bytes = 24.0e3, finalize_bytes = 24.0e6;
+            const double kb_bytes = (double)kBN * kBK, wave_bytes = 3.5e6, finalize_bytes = 24.0e6, solo = 1.6;
+            const double weights = (double)tiles * p.num_k * kb_bytes;
             double best = 0;
             int64_t best_kb = p.num_k;
             for (int64_t sp = 1; sp <= cap; ++sp) {
@@ -1468,13 +1507,16 @@ static fp8_status_t run_gemm(fp8_ctx *ctx, const uint8_t *a, int a_fmt, bool a_m
                 const int64_t real = (p.num_k + kb - 1) / kb;
                 if (real != sp) continue;
                 const int64_t waves = (tiles * real + ctx->sm_count - 1) / ctx->sm_count;
-                double cost = (double)waves * sms * ((double)kb * kb_bytes + item_bytes);
-                if (real > 1) cost += 8.0 * (double)real * (double)M * (double)N + finalize_bytes;
+                const double partials = real > 1 ? 8.0 * (double)real * (double)M * (double)N : 0.0;
+                const double busiest = (double)waves * (double)kb * kb_bytes * sms / solo;
+                double cost = (weights + partials > busiest ? weights + partials : busiest) + (double)waves * wave_bytes;
+                if (real > 1) cost += finalize_bytes;
                 if (sp == 1 || cost < best) {
                     best = cost;
                     best_kb = kb;
                 }
             }
+            if (g_force_splits > 0) best_kb = (p.num_k + g_force_splits - 1) / g_force_splits;
             p.kb_per_split = (int)best_kb;
             p.splits = (p.num_k + p.kb_per_split - 1) / p.kb_per_split;
         }
@@ -1566,7 +1608,7 @@ static fp8_status_t run_gemm(fp8_ctx *ctx, const uint8_t *a, int a_fmt, bool a_m
             cfg.dynamicSmemBytes = GemmSmem<kBN, kStages>::kDynamic;
             cfg.stream = st;
             cfg.attrs = attr;
-            cfg.numAttrs = 1;
+            cfg.numAttrs = g_no_pdl ? 0 : 1;
             if (cudaLaunchKernelEx(&cfg, gemm_kernel<kBN, kStages, 0>, map_a, map_b, map_out, map_out2, p) != cudaSuccess)
                 return FP8_ERR_CUDA;
             break;

@@ -13,7 +13,13 @@
  *  - `stream` is a cudaStream_t passed as void* (NULL = the legacy default
  *    stream).  Calls are asynchronous and ordered on that stream like any
  *    kernel launch.  Calls that share one fp8_ctx must be issued from one host
- *    thread at a time.
+ *    thread at a time, and decode-size matmuls (at most 128 rows of output:
+ *    they may split the contraction through the context's workspace) that
+ *    share one fp8_ctx must not overlap on the device: keep them on one
+ *    stream, or order the streams with events, or use one context per stream.
+ *    Inside the library a kernel may be launched so that it starts while the
+ *    call before it on the stream is draining; it touches no memory before
+ *    that call has completed, so stream order holds as for any launch.
  *  - Tensors are row-major.  X[T,K] activations, W[N,K] weights (the layout of
  *    a PyTorch nn.Linear), dY[T,N] output gradients; Y[T,N], dX[T,K], dW[N,K].
  *  - FP8 bytes are the native Blackwell encodings (Table 7 rows "(b)": E4M3

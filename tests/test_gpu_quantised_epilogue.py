@@ -327,3 +327,38 @@ def test_llama_mlp_block_forward_and_backward_chain(ctx, lib):
     assert_bf16_within_one_ulp(bits_of(dw), O.linear_wgrad_np(u8(g8), bq, qx.ref, qx.shift))
     assert_bf16_within_one_ulp(bits_of(dx), O.linear_dgrad_np(u8(g8), bq, qgu.ref, qgu.shift))
     assert ctx.device_flags(clear=True) & ~lib.FLAG_SATURATED == 0
+
+
+def test_llama7b_gate_up_with_swiglu_at_benchmark_size_sampled(ctx, lib):
+    """The Llama-2-7B gate_up layer (8192 tokens, 4096 -> 2 x 11008) in the benchmark's launch configuration with the
+    SwiGLU epilogue: pre-activations at sampled positions against the oracle, z and its bytes as relations on the
+    GPU's own stored tensors at the same positions, the amax against a reduction over the whole of z."""
+    T, K, F = 8192, 4096, 11008
+    x = I.normal_bf16(T, K, 1.0, 8100, 1, "cuda", outlier_frac=0.005, outlier_scale=100.0)
+    qx = Quantised(ctx, x, O.E4, O.CONV_PAPER)
+    qw = _interleaved_weight(ctx, F, K, O.CONV_PAPER, 8101)
+    y_pre = torch.empty((T, 2 * F), dtype=torch.bfloat16, device="cuda")
+    z = torch.empty((T, F), dtype=torch.bfloat16, device="cuda")
+    z8 = torch.empty((T, F), dtype=torch.uint8, device="cuda")
+    amax_z = torch.zeros(1, dtype=torch.float32, device="cuda")
+    bias = 1
+    ctx.linear_fwd_q(qx.y, qx.bias, qw.y, qw.bias, z8, _dev_i32(bias), y_pre=y_pre, z=z, d_amax_z=amax_z,
+                     act=lib.ACT_SWIGLU)
+    assert ctx.device_flags(clear=True) & lib.FLAG_TIMEOUT == 0
+    rng = np.random.default_rng(81)
+    rows = np.concatenate([rng.integers(0, T, 3000), [0, T - 1, 0, T - 1]])
+    feat = np.concatenate([rng.integers(0, F, 3000), [0, F - 1, F - 1, 0]])
+    gi, ui = OS._blocks32(2 * F)
+    r_t = torch.from_numpy(rows).cuda()
+    for cols in (gi[feat], ui[feat]):
+        ref = O.linear_samples(O.FWD, qx.ref, O.N_E4, qx.shift, qw.ref, O.N_E4, qw.shift, rows, cols)
+        got = y_pre[r_t, torch.from_numpy(cols).cuda()]
+        assert_bf16_within_one_ulp(bits_of(got.reshape(1, -1))[0], ref)
+    g = OS.bf16_to_f64(bits_of(y_pre[r_t, torch.from_numpy(gi[feat]).cuda()].reshape(1, -1)))
+    u = OS.bf16_to_f64(bits_of(y_pre[r_t, torch.from_numpy(ui[feat]).cuda()].reshape(1, -1)))
+    want = OS.f64_to_bf16(OS.silu(g) * u)
+    zs = z[r_t, torch.from_numpy(feat).cuda()].reshape(1, -1)
+    assert np.abs(bf16_ordinal(bits_of(zs)) - bf16_ordinal(want)).max() <= 1
+    z8s = z8[r_t, torch.from_numpy(feat).cuda()].reshape(1, -1)
+    assert_codes_equal(u8(z8s), O.cast(bits_of(zs), bias + 1, O.N_E4), O.N_E4)
+    assert float(amax_z.item()) == float(z.float().abs().max().item())

@@ -3,6 +3,7 @@
     python -m paper_2309_17224_b200.sweep gemm 8192x8192x16384 8192x8192x4096    # MxNxK forward matmuls
     python -m paper_2309_17224_b200.sweep cast 8192x4096 8192x22016               # amax, cast, amax+cast of bf16 [rows x cols]
     python -m paper_2309_17224_b200.sweep stack 24x1024x4096                      # layers x d x tokens: the SGD stack, three scaling variants
+    python -m paper_2309_17224_b200.sweep mlp 8192x4096x11008                     # tokens x d x ffn: a Llama MLP forward, unfused vs SwiGLU epilogue
     python -m paper_2309_17224_b200.sweep stack 24x1024x4096 --only history --steps 2 --warmup 2 --no-graph   # one variant, short (for profilers)
 
 Prints one line per shape.  Operands of the matmul sweep are random FP8 bytes
@@ -161,6 +162,62 @@ def stack(ctx, shapes, steps=40, warmup=8, only=None, graph=True):
             del st, g
 
 
+def mlp(ctx, shapes, iters=20):
+    """Forward of a gated MLP (x -> SiLU(x Wg^T) * (x Wu^T) -> . Wd^T), every linear in FP8: (a) each linear quantises
+    its input just in time and the gated unit is separate torch kernels; (b) the gate_up matmul's epilogue computes
+    the gated unit and writes the down projection's FP8 input under a bias carried over from the previous call
+    (amax-history scaling).  Weights are quantised once, outside the timed region, in both variants."""
+    from . import inputs as I
+    for T, d, F in shapes:
+        dev = dict(device="cuda")
+        x = torch.randn(T, d, **dev).to(torch.bfloat16)
+        wg, wu = (torch.randn(F, d, **dev) * 0.02).to(torch.bfloat16), (torch.randn(F, d, **dev) * 0.02).to(torch.bfloat16)
+        wd = (torch.randn(d, F, **dev) * 0.02).to(torch.bfloat16)
+        w_gu = torch.cat((wg, wu), 0).contiguous()           # unfused: gate rows then up rows
+        w_il = I.interleave32(wg, wu).contiguous()           # fused: blocks of 32 gate rows, 32 up rows
+        sc_f = torch.zeros(8, dtype=torch.float32, **dev)
+        sc_i = torch.zeros(8, dtype=torch.int32, **dev)
+        u8 = dict(dtype=torch.uint8, **dev)
+        w_gu8, w_il8, wd8 = torch.empty((2 * F, d), **u8), torch.empty((2 * F, d), **u8), torch.empty((d, F), **u8)
+        ctx.ptq_weights(w_gu, fp8lin.CONV_PAPER, w_gu8, None, sc_i[0:1], sc_f[0:1])
+        ctx.ptq_weights(w_il, fp8lin.CONV_PAPER, w_il8, None, sc_i[1:2], sc_f[1:2])
+        ctx.ptq_weights(wd, fp8lin.CONV_PAPER, wd8, None, sc_i[2:3], sc_f[2:3])
+        x8, z8 = torch.empty((T, d), **u8), torch.empty((T, F), **u8)
+        h = torch.empty((T, 2 * F), dtype=torch.bfloat16, **dev)
+        out = torch.empty((T, d), dtype=torch.bfloat16, **dev)
+
+        def unfused():
+            ctx.cast_e4(x, None, d_amax_out=sc_f[3:4], d_bias_out=sc_i[3:4], y=x8)
+            ctx.linear_fwd(x8, sc_i[3:4], w_gu8, sc_i[0:1], h)
+            z = (torch.nn.functional.silu(h[:, :F].float()) * h[:, F:].float()).to(torch.bfloat16)
+            ctx.cast_e4(z, None, d_amax_out=sc_f[4:5], d_bias_out=sc_i[4:5], y=z8)
+            ctx.linear_fwd(z8, sc_i[4:5], wd8, sc_i[2:3], out)
+
+        def fused():
+            ctx.cast_e4(x, None, d_amax_out=sc_f[3:4], d_bias_out=sc_i[3:4], y=x8)
+            ctx.linear_fwd_q(x8, sc_i[3:4], w_il8, sc_i[1:2], z8, sc_i[5:6], d_amax_z=sc_f[5:6], act=fp8lin.ACT_SWIGLU)
+            ctx.linear_fwd(z8, sc_i[5:6], wd8, sc_i[2:3], out)
+            ctx.scaling_bias(sc_f[5:6], fp8lin.E4, fp8lin.CONV_PAPER, 1, sc_i[5:6])   # next call's bias, margin 1
+
+        unfused()
+        sc_i[5:6].copy_(sc_i[4:5] - 1)                       # history for the first fused call
+        res = {}
+        for name, fn in (("unfused", unfused), ("SwiGLU epilogue", fused)):
+            for _ in range(3):
+                fn()
+            torch.cuda.synchronize()
+            s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            s.record()
+            for _ in range(iters):
+                fn()
+            e.record()
+            torch.cuda.synchronize()
+            res[name] = s.elapsed_time(e) / iters
+        flops = 2.0 * T * d * 3 * F
+        print(f"mlp T={T} d={d} ffn={F}: " + " | ".join(f"{k} {v:7.3f} ms {flops / v / 1e9:7.1f} TFLOP/s" for k, v in res.items()),
+              flush=True)
+
+
 def main(argv):
     opts = {"--only": None, "--steps": None, "--warmup": None}
     graph = "--no-graph" not in argv
@@ -170,7 +227,7 @@ def main(argv):
             i = argv.index(key)
             opts[key] = argv[i + 1]
             del argv[i:i + 2]
-    if len(argv) < 2 or argv[0] not in ("gemm", "cast", "stack"):
+    if len(argv) < 2 or argv[0] not in ("gemm", "cast", "stack", "mlp"):
         print(__doc__)
         return 2
     shapes = [tuple(int(v) for v in a.split("x")) for a in argv[1:]]
@@ -179,7 +236,7 @@ def main(argv):
         stack(ctx, shapes, steps=int(opts["--steps"] or 40), warmup=int(opts["--warmup"] or 8), only=opts["--only"],
               graph=graph)
     else:
-        {"gemm": gemm, "cast": cast}[argv[0]](ctx, shapes)
+        {"gemm": gemm, "cast": cast, "mlp": mlp}[argv[0]](ctx, shapes)
     flags = ctx.device_flags()
     if flags & fp8lin.FLAG_TIMEOUT:
         print("a device-side wait expired", file=sys.stderr)

@@ -447,6 +447,7 @@ def main():
                     help="skip the extra timed loop that uses fp8_cast_predicted")
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-mlp-leg", action="store_true", help="skip the chained gated-MLP comparison (c3 only)")
     args = ap.parse_args()
     wl = I.WORKLOADS[args.workload]
     if args.impl == "reference":
@@ -543,6 +544,18 @@ def main():
 
     # ---- the two quantisation kernels, each against its own algorithmic bytes (outside the timed region) ----
     per_kernel = quantisation_kernel_bandwidths(ctx, layers, peaks["hbm_gbs"])
+
+    # ---- the gated MLP of the same model as one chained block, unfused against the fused epilogues ----
+    fused_mlp = None
+    if wl.name == "c3_llama7b" and not args.no_mlp_leg:
+        from paper_2309_17224_b200 import sweep
+        gate_up = next(l for l in wl.layers if l.name == "gate_up")
+        r = sweep.mlp(ctx, [(tokens, gate_up.K, gate_up.N // 2)], iters=10, quiet=True)[-1]
+        fused_mlp = {"block": f"x[{tokens},{gate_up.K}] -> SiLU(x Wg^T) * (x Wu^T) -> . Wd^T, forward + backward, all six matmuls "
+                              "in FP8, every quantisation included",
+                     "unfused_ms": r["unfused_ms"], "fused_ms": r["fused_ms"], "fused_tflops": r["fused_tflops"],
+                     "how": "unfused: just-in-time amax + cast per tensor, gated unit and its backward as torch kernels; fused: "
+                            "fp8_linear_fwd_q / fp8_linear_dgrad_q with the SwiGLU epilogues, amax-history biases (margin 1)"}
 
     # ---- the same steps with the one-pass quantisation (bias guessed from the previous step, verified) ----
     predicted = None
@@ -696,6 +709,7 @@ def main():
                               "against its own bytes; with_bias_prediction is the one-pass variant",
                       "per_kernel": per_kernel},
         "layer_ms": {k: round(v, 4) for k, v in timers.layer_ms().items()},   # amax + cast + matmuls of one layer
+        "fused_mlp": fused_mlp,
         "with_bias_prediction": predicted,
         "with_cuda_graph": graphed,
         "gemm_ms_per_step": gemm_ms / sampled_steps,

@@ -162,12 +162,14 @@ def stack(ctx, shapes, steps=40, warmup=8, only=None, graph=True):
             del st, g
 
 
-def mlp(ctx, shapes, iters=20):
+def mlp(ctx, shapes, iters=20, quiet=False):
     """Forward of a gated MLP (x -> SiLU(x Wg^T) * (x Wu^T) -> . Wd^T), every linear in FP8: (a) each linear quantises
     its input just in time and the gated unit is separate torch kernels; (b) the gate_up matmul's epilogue computes
     the gated unit and writes the down projection's FP8 input under a bias carried over from the previous call
     (amax-history scaling).  Weights are quantised once, outside the timed region, in both variants."""
     from . import inputs as I
+    results = []
+    say = (lambda *a, **k: None) if quiet else print
     for T, d, F in shapes:
         dev = dict(device="cuda")
         x = torch.randn(T, d, **dev).to(torch.bfloat16)
@@ -214,8 +216,69 @@ def mlp(ctx, shapes, iters=20):
             torch.cuda.synchronize()
             res[name] = s.elapsed_time(e) / iters
         flops = 2.0 * T * d * 3 * F
-        print(f"mlp T={T} d={d} ffn={F}: " + " | ".join(f"{k} {v:7.3f} ms {flops / v / 1e9:7.1f} TFLOP/s" for k, v in res.items()),
-              flush=True)
+        say(f"mlp T={T} d={d} ffn={F} forward: " + " | ".join(f"{k} {v:7.3f} ms {flops / v / 1e9:7.1f} TFLOP/s" for k, v in res.items()),
+            flush=True)
+        results.append({"tokens": T, "d": d, "ffn": F, "pass": "fwd", "unfused_ms": res["unfused"],
+                        "fused_ms": res["SwiGLU epilogue"], "fused_tflops": flops / res["SwiGLU epilogue"] / 1e9})
+        if T < 256:
+            continue
+        # ---- forward + backward of the same block (training step without the optimiser) ----
+        dy = (torch.randn(T, d, **dev) * 1e-3).to(torch.bfloat16)
+        dy8, g8 = torch.empty((T, d), **u8), torch.empty((T, 2 * F), **u8)
+        dz = torch.empty((T, F), dtype=torch.bfloat16, **dev)
+        dx = torch.empty((T, d), dtype=torch.bfloat16, **dev)
+        dw_gu = torch.empty((2 * F, d), dtype=torch.bfloat16, **dev)
+        dw_d = torch.empty((d, F), dtype=torch.bfloat16, **dev)
+        h_il = torch.empty((T, 2 * F), dtype=torch.bfloat16, **dev)
+
+        def unfused_step():
+            unfused()
+            ctx.cast_e5(dy, None, d_amax_out=sc_f[6:7], d_bias_out=sc_i[6:7], y=dy8)
+            ctx.linear_dgrad(dy8, sc_i[6:7], wd8, None, sc_i[2:3], dz)
+            ctx.linear_wgrad(dy8, None, sc_i[6:7], z8, None, sc_i[4:5], dw_d, T)
+            a, u_ = h[:, :F].float(), h[:, F:].float()
+            sg = torch.sigmoid(a)
+            g = torch.cat(((dz.float() * u_ * (sg + a * sg * (1 - sg))), (dz.float() * a * sg)), 1).to(torch.bfloat16)
+            ctx.cast_e5(g, None, d_amax_out=sc_f[7:8], d_bias_out=sc_i[7:8], y=g8)
+            ctx.linear_dgrad(g8, sc_i[7:8], w_gu8, None, sc_i[0:1], dx)
+            ctx.linear_wgrad(g8, None, sc_i[7:8], x8, None, sc_i[3:4], dw_gu, T)
+
+        gb = torch.zeros(2, dtype=torch.int32, **dev)      # history bias of the gate/up gradient, and its next value
+        ga = torch.zeros(1, dtype=torch.float32, **dev)
+
+        def fused_step():
+            ctx.cast_e4(x, None, d_amax_out=sc_f[3:4], d_bias_out=sc_i[3:4], y=x8)
+            ctx.linear_fwd_q(x8, sc_i[3:4], w_il8, sc_i[1:2], z8, sc_i[5:6], y_pre=h_il, d_amax_z=sc_f[5:6],
+                             act=fp8lin.ACT_SWIGLU)
+            ctx.linear_fwd(z8, sc_i[5:6], wd8, sc_i[2:3], out)
+            ctx.cast_e5(dy, None, d_amax_out=sc_f[6:7], d_bias_out=sc_i[6:7], y=dy8)
+            ctx.linear_dgrad_q(dy8, sc_i[6:7], wd8, None, sc_i[2:3], g8, gb[0:1], y_pre=h_il, d_amax_g=ga,
+                               act=fp8lin.ACT_SWIGLU)
+            ctx.linear_wgrad(dy8, None, sc_i[6:7], z8, None, sc_i[5:6], dw_d, T)
+            ctx.linear_dgrad(g8, gb[0:1], w_il8, None, sc_i[1:2], dx)
+            ctx.linear_wgrad(g8, None, gb[0:1], x8, None, sc_i[3:4], dw_gu, T)
+            ctx.scaling_bias(sc_f[5:6], fp8lin.E4, fp8lin.CONV_PAPER, 1, sc_i[5:6])
+            ctx.scaling_bias(ga, fp8lin.E5, fp8lin.CONV_PAPER, 1, gb[0:1])
+
+        unfused_step()
+        gb[0:1].copy_(sc_i[7:8] - 1)
+        res = {}
+        for name, fn in (("unfused", unfused_step), ("SwiGLU epilogues", fused_step)):
+            for _ in range(3):
+                fn()
+            torch.cuda.synchronize()
+            s.record()
+            for _ in range(iters):
+                fn()
+            e.record()
+            torch.cuda.synchronize()
+            res[name] = s.elapsed_time(e) / iters
+        flops *= 3
+        say(f"mlp T={T} d={d} ffn={F} forward + backward: "
+            + " | ".join(f"{k} {v:7.3f} ms {flops / v / 1e9:7.1f} TFLOP/s" for k, v in res.items()), flush=True)
+        results.append({"tokens": T, "d": d, "ffn": F, "pass": "fwd+bwd", "unfused_ms": res["unfused"],
+                        "fused_ms": res["SwiGLU epilogues"], "fused_tflops": flops / res["SwiGLU epilogues"] / 1e9})
+    return results
 
 
 def main(argv):

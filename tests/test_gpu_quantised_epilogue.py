@@ -362,3 +362,39 @@ def test_llama7b_gate_up_with_swiglu_at_benchmark_size_sampled(ctx, lib):
     z8s = z8[r_t, torch.from_numpy(feat).cuda()].reshape(1, -1)
     assert_codes_equal(u8(z8s), O.cast(bits_of(zs), bias + 1, O.N_E4), O.N_E4)
     assert float(amax_z.item()) == float(z.float().abs().max().item())
+
+
+def test_llama7b_down_input_gradient_with_swiglu_backward_at_benchmark_size_sampled(ctx, lib):
+    """The backward twin at benchmark size: dz[8192, 11008] = dY8 . W8 (contraction 4096, weight read in its forward
+    layout) with the SwiGLU backward epilogue producing the [8192, 22016] gate / up gradient, its E5 bytes and amax."""
+    T, N, F = 8192, 4096, 11008
+    qg = Quantised(ctx, I.normal_bf16(T, N, 1e-5, 8200, 3, "cuda"), O.E5, O.CONV_PAPER)
+    qw = Quantised(ctx, I.normal_bf16(N, F, 0.02, 8201, 2, "cuda"), O.E4, O.CONV_PAPER)
+    y_pre = I.normal_bf16(T, 2 * F, 1.5, 8202, 9, "cuda")
+    dz = torch.empty((T, F), dtype=torch.bfloat16, device="cuda")
+    g = torch.empty((T, 2 * F), dtype=torch.bfloat16, device="cuda")
+    g8 = torch.empty((T, 2 * F), dtype=torch.uint8, device="cuda")
+    amax_g = torch.zeros(1, dtype=torch.float32, device="cuda")
+    bias = 28
+    ctx.linear_dgrad_q(qg.y, qg.bias, qw.y, None, qw.bias, g8, _dev_i32(bias), y_pre=y_pre, dx=dz, g=g, d_amax_g=amax_g,
+                       act=lib.ACT_SWIGLU)
+    assert ctx.device_flags(clear=True) & lib.FLAG_TIMEOUT == 0
+    rng = np.random.default_rng(82)
+    rows = np.concatenate([rng.integers(0, T, 3000), [0, T - 1, 0, T - 1]])
+    feat = np.concatenate([rng.integers(0, F, 3000), [0, F - 1, F - 1, 0]])
+    r_t, f_t = torch.from_numpy(rows).cuda(), torch.from_numpy(feat).cuda()
+    ref = O.linear_samples(O.DGRAD, qg.ref, O.N_E5, qg.shift, qw.ref, O.N_E4, qw.shift, rows, feat)
+    dzs = dz[r_t, f_t].reshape(1, -1)
+    assert_bf16_within_one_ulp(bits_of(dzs)[0], ref)
+    gi, ui = OS._blocks32(2 * F)
+    gcol, ucol = torch.from_numpy(gi[feat]).cuda(), torch.from_numpy(ui[feat]).cuda()
+    a = OS.bf16_to_f64(bits_of(y_pre[r_t, gcol].reshape(1, -1)))
+    u = OS.bf16_to_f64(bits_of(y_pre[r_t, ucol].reshape(1, -1)))
+    d = OS.bf16_to_f64(bits_of(dzs))
+    e = np.exp(-np.abs(a))
+    s = np.where(a > 0, 1.0 / (1.0 + e), e / (1.0 + e))
+    for cols, want in ((gcol, d * u * (s + a * s * (1.0 - s))), (ucol, d * OS.silu(a))):
+        got = g[r_t, cols].reshape(1, -1)
+        assert np.abs(bf16_ordinal(bits_of(got)) - bf16_ordinal(OS.f64_to_bf16(want))).max() <= 1
+        assert_codes_equal(u8(g8[r_t, cols].reshape(1, -1)), O.cast(bits_of(got), bias, O.N_E5), O.N_E5)
+    assert float(amax_g.item()) == float(g.float().abs().max().item())

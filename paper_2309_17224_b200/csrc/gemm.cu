@@ -448,11 +448,44 @@ __device__ __forceinline__ void silu_and_grad_f32(float a, float &silu, float &g
     float e;
     const float r = sigmoid_parts(a, e);
     const float sg = a > 0.0f ? r : (e * r) * kTwoM32;
-    silu = a > 0.0f ? a * r : (a * e * r) * kTwoM32;
+    silu = a * sg;  // where sigma is subnormal (a < -87) the product is below every bf16 normal anyway
     grad = fmaf(silu, 1.0f - sg, sg);
 }
 __device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
+
+// Four bf16 values (two packed words, memory order) scaled by the exact power of two and rounded to four FP8 bytes,
+// as cast4 does; instead of testing each value for clipping, the largest scaled magnitude is kept in `peak` and
+// tested once per tile (the epilogue pays for every instruction per element).
+template <int FMT, bool TWO_STEP>
+__device__ __forceinline__ uint32_t quantise4(uint32_t w0, uint32_t w1, const Pow2Pair p, float &peak)
+{
+    float f0 = bf16_lo(w0) * p.first, f1 = bf16_hi(w0) * p.first, f2 = bf16_lo(w1) * p.first, f3 = bf16_hi(w1) * p.first;
+    if (TWO_STEP) {
+        f0 *= p.second; f1 *= p.second; f2 *= p.second; f3 *= p.second;
+    }
+    peak = fmaxf(fmaxf(peak, fabsf(f0)), fmaxf(fmaxf(fabsf(f1), fabsf(f2)), fabsf(f3)));
+    return cvt_pair<FMT>(f1, f0) | (cvt_pair<FMT>(f3, f2) << 16);
+}
+// n words of bf16 pairs -> n/2 words of FP8 bytes
+template <int FMT, int NW>
+__device__ __forceinline__ void quantise_words(const uint32_t (&w)[NW], uint32_t *b8, const Pow2Pair p, bool two_step,
+                                               float &peak)
+{
+    if (two_step) {
+#pragma unroll
+        for (int i = 0; i < NW / 2; ++i) b8[i] = quantise4<FMT, true>(w[2 * i], w[2 * i + 1], p, peak);
+    } else {
+#pragma unroll
+        for (int i = 0; i < NW / 2; ++i) b8[i] = quantise4<FMT, false>(w[2 * i], w[2 * i + 1], p, peak);
+    }
+}
+// the saturation rule of the cast kernels on the largest scaled magnitude
+template <int FMT>
+__device__ __forceinline__ bool peak_clips(float peak)
+{
+    return FMT == FP8_E4 ? peak > 464.0f : peak >= 61440.0f;
+}
 
 // One warp's share (32 rows x BN columns) of a finished accumulator.
 //   t_row        TMEM address of this warp's lanes at the accumulator's first column
@@ -495,9 +528,14 @@ __device__ __forceinline__ void epilogue_tile(const CUtensorMap *map_out, const 
         // per 64 columns), slabs 1 and 3 stage z (alternating per 128 columns); one bulk group per 64 columns.
         static_assert(NSLAB == 4, "SwiGLU epilogue needs four slabs per warp");
         uint32_t dummy = 0, wg[16];
-        bool sat = false;
+        float peak = 0.0f;
         Pow2Pair scq = make_pow2_pair(0);
-        if (p.out8) scq = make_pow2_pair(__ldg(p.d_sq) + p.delta_q);
+        bool scq_two = false;
+        if (p.out8) {
+            const int sq = __ldg(p.d_sq) + p.delta_q;
+            scq = make_pow2_pair(sq);
+            scq_two = sq < -126 || sq > 127;
+        }
         const int64_t ldz = p.ldo >> 1;
 #pragma unroll 1
         for (int c = 0; c < BN; c += 32) {
@@ -544,8 +582,7 @@ __device__ __forceinline__ void epilogue_tile(const CUtensorMap *map_out, const 
             }
             if (p.out8 && row_ok && in_n) {
                 uint32_t b8[8];
-#pragma unroll
-                for (int i = 0; i < 8; ++i) b8[i] = cast4<FP8_E4, true>(wz[2 * i], wz[2 * i + 1], scq, sat);
+                quantise_words<FP8_E4>(wz, b8, scq, scq_two, peak);
                 uint8_t *dst = p.out8 + (int64_t)(row0 + lane) * ldz + zc;
                 reinterpret_cast<uint4 *>(dst)[0] = make_uint4(b8[0], b8[1], b8[2], b8[3]);
                 reinterpret_cast<uint4 *>(dst)[1] = make_uint4(b8[4], b8[5], b8[6], b8[7]);
@@ -561,7 +598,7 @@ __device__ __forceinline__ void epilogue_tile(const CUtensorMap *map_out, const 
                 asm volatile("cp.async.bulk.commit_group;" ::: "memory");
             }
         }
-        if (__any_sync(0xFFFFFFFFu, sat) && lane == 0) atomicOr(p.d_status, (unsigned)FP8_FLAG_SATURATED);
+        if (__any_sync(0xFFFFFFFFu, peak_clips<FP8_E4>(peak)) && lane == 0) atomicOr(p.d_status, (unsigned)FP8_FLAG_SATURATED);
         return;
     }
     if constexpr (ACT == 5) {
@@ -570,9 +607,14 @@ __device__ __forceinline__ void epilogue_tile(const CUtensorMap *map_out, const 
         // slabs 1 and 3 the gradients (alternating per 32 columns); one bulk group per 32 columns.
         static_assert(NSLAB == 4, "SwiGLU epilogue needs four slabs per warp");
         uint32_t dummy = 0;
-        bool sat = false;
+        float peak = 0.0f;
         Pow2Pair scq = make_pow2_pair(0);
-        if (p.out8) scq = make_pow2_pair(__ldg(p.d_sq) + p.delta_q);
+        bool scq_two = false;
+        if (p.out8) {
+            const int sq = __ldg(p.d_sq) + p.delta_q;
+            scq = make_pow2_pair(sq);
+            scq_two = sq < -126 || sq > 127;
+        }
         const int64_t ld2 = p.ldo * 2;
         // the stored pre-activations of a chunk (32 gate values then 32 up values, 128 bytes per row) are requested
         // one chunk ahead, so that their trip from memory overlaps the arithmetic of the chunk before
@@ -641,11 +683,8 @@ __device__ __forceinline__ void epilogue_tile(const CUtensorMap *map_out, const 
             }
             if (p.out8 && ok) {
                 uint32_t b8[16];
-#pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    b8[i] = cast4<FP8_E5, true>(wgr[2 * i], wgr[2 * i + 1], scq, sat);
-                    b8[8 + i] = cast4<FP8_E5, true>(wur[2 * i], wur[2 * i + 1], scq, sat);
-                }
+                quantise_words<FP8_E5>(wgr, b8, scq, scq_two, peak);
+                quantise_words<FP8_E5>(wur, b8 + 8, scq, scq_two, peak);
                 uint4 *dst = reinterpret_cast<uint4 *>(p.out8 + (int64_t)(row0 + lane) * ld2 + 2 * (int64_t)col0);
 #pragma unroll
                 for (int j = 0; j < 4; ++j) dst[j] = make_uint4(b8[4 * j], b8[4 * j + 1], b8[4 * j + 2], b8[4 * j + 3]);
@@ -660,7 +699,7 @@ __device__ __forceinline__ void epilogue_tile(const CUtensorMap *map_out, const 
                 asm volatile("cp.async.bulk.commit_group;" ::: "memory");
             }
         }
-        if (__any_sync(0xFFFFFFFFu, sat) && lane == 0) atomicOr(p.d_status, (unsigned)FP8_FLAG_SATURATED);
+        if (__any_sync(0xFFFFFFFFu, peak_clips<FP8_E5>(peak)) && lane == 0) atomicOr(p.d_status, (unsigned)FP8_FLAG_SATURATED);
         return;
     }
     if (ACT) {
@@ -669,9 +708,14 @@ __device__ __forceinline__ void epilogue_tile(const CUtensorMap *map_out, const 
         // columns and is not unrolled: fully unrolled, the activation arithmetic outgrows the instruction cache.
         constexpr int kPairsOfSlabs = NSLAB / 2;
         uint32_t dummy = 0;
-        bool sat = false;
+        float peak = 0.0f;
         Pow2Pair scq = make_pow2_pair(0);
-        if (p.out8) scq = make_pow2_pair(__ldg(p.d_sq) + p.delta_q);
+        bool scq_two = false;
+        if (p.out8) {
+            const int sq = __ldg(p.d_sq) + p.delta_q;
+            scq = make_pow2_pair(sq);
+            scq_two = sq < -126 || sq > 127;
+        }
         // ACT == 2: the stored pre-activations of a chunk (64 bytes per row) are requested one chunk ahead, so that
         // their trip from memory overlaps the arithmetic of the chunk before
         uint4 aux_next[4];
@@ -748,13 +792,8 @@ __device__ __forceinline__ void epilogue_tile(const CUtensorMap *map_out, const 
                 // the bytes are made from the bf16 values just rounded, as a cast of the stored tensor would;
                 // one row per lane, 32 bytes
                 uint32_t b8[8];
-                if (p.q_fmt == FP8_E4) {
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) b8[i] = cast4<FP8_E4, true>(wa[2 * i], wa[2 * i + 1], scq, sat);
-                } else {
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) b8[i] = cast4<FP8_E5, true>(wa[2 * i], wa[2 * i + 1], scq, sat);
-                }
+                if (p.q_fmt == FP8_E4) quantise_words<FP8_E4>(wa, b8, scq, scq_two, peak);
+                else quantise_words<FP8_E5>(wa, b8, scq, scq_two, peak);
                 uint8_t *dst = p.out8 + (int64_t)(row0 + lane) * p.ldo + col0;
                 if (col0 + 32 <= p.N) {
                     reinterpret_cast<uint4 *>(dst)[0] = make_uint4(b8[0], b8[1], b8[2], b8[3]);
@@ -779,7 +818,8 @@ __device__ __forceinline__ void epilogue_tile(const CUtensorMap *map_out, const 
                 ++slab_count;
             }
         }
-        if (__any_sync(0xFFFFFFFFu, sat) && lane == 0) atomicOr(p.d_status, (unsigned)FP8_FLAG_SATURATED);
+        const bool clipped = p.q_fmt == FP8_E4 ? peak_clips<FP8_E4>(peak) : peak_clips<FP8_E5>(peak);
+        if (__any_sync(0xFFFFFFFFu, clipped) && lane == 0) atomicOr(p.d_status, (unsigned)FP8_FLAG_SATURATED);
         return;
     }
     if (p.out_dt == FP8_BF16) {

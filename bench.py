@@ -667,9 +667,25 @@ def main():
             e2e_step()
         barrier_sync(dist)
         e2e_ms = max_over_ranks(1e3 * (time.perf_counter() - t0) / args.e2e_steps, dist, device)
+        # the host link by itself, both directions at once, on the same pinned buffers: the floor for these bytes
+        torch.cuda.synchronize()
+        pairs = [(d, h) for L, hin in zip(layers, host_in) for d, h in zip([L.x] + ([L.w, L.g] if wl.backward else []), hin)]
+        backs = [(h, d) for L, hout in zip(layers, host_out)
+                 for h, d in zip(hout, [L.y] + ([L.dx, L.dw] if wl.backward else []))]
+        t0 = time.perf_counter()
+        with torch.cuda.stream(s_in):
+            for d, h in pairs:
+                d.copy_(h, non_blocking=True)
+        with torch.cuda.stream(s_out):
+            for h, d in backs:
+                h.copy_(d, non_blocking=True)
+        torch.cuda.synchronize()
+        link_ms = 1e3 * (time.perf_counter() - t0)
         e2e = {"value": world * step_flops / (e2e_ms * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": e2e_ms,
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-               "how": "pinned host buffers; copies in, kernels and copies out on three streams, ordered per layer"}
+               "copies_alone_ms": link_ms,
+               "how": "pinned host buffers; copies in, kernels and copies out on three streams, ordered per layer; "
+                      "copies_alone_ms = the same copies, both directions at once, with no kernels"}
         del host_in, host_out
 
     if rank != 0:

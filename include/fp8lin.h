@@ -93,6 +93,11 @@ FP8_API fp8_status_t fp8_destroy(fp8_ctx *ctx);
 
 FP8_API const char *fp8_status_string(fp8_status_t status);
 
+/* Kernels launched by this library in this process so far (all contexts; host
+ * counter, bumped beside every launch; fp8_amax_noalloc is not counted).  The
+ * difference of two readings is what a span of calls launched. */
+FP8_API fp8_status_t fp8_launch_count(uint64_t *count);
+
 /* Synchronises `stream`, copies the sticky status word to *flags (host) and,
  * if `clear` is non-zero, resets it.  Returns FP8_ERR_DEVICE_TIMEOUT if
  * FP8_FLAG_TIMEOUT was set, else FP8_OK. */

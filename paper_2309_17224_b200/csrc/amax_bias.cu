@@ -190,10 +190,12 @@ static cudaError_t launch_amax_dt(fp8_ctx *ctx, const void *x, int64_t rows, int
         int64_t chunk = (int64_t)kAmaxThreads * kAmaxUnroll;
         int64_t want = (nvec + chunk - 1) / chunk;
         int blocks = (int)(want < 1 ? 1 : (want > max_blocks ? max_blocks : want));
+        count_launch();
         amax_flat_kernel<DT><<<blocks, kAmaxThreads, 0, stream>>>(reinterpret_cast<const uint4 *>(x), nvec, ntail, o);
     } else {
         int vec = (aligned && (ld % kPerVec) == 0) ? 1 : 0;
         int blocks = (int)(rows > max_blocks ? max_blocks : rows);
+        count_launch();
         amax_rows_kernel<DT><<<blocks, kAmaxThreads, 0, stream>>>(x, rows, cols, ld, vec, o);
     }
     return cudaGetLastError();
@@ -229,6 +231,7 @@ fp8_status_t fp8_scaling_bias(fp8_ctx *ctx, const float *d_amax, fp8_format_t fm
 {
     if (!ctx || !d_amax || !d_bias) return FP8_ERR_NULL;
     if ((int)fmt < 0 || (int)fmt > 1 || (int)conv < 0 || (int)conv > 1) return FP8_ERR_DTYPE;
+    fp8lin::count_launch();
     fp8lin::scaling_bias_kernel<<<1, 1, 0, (cudaStream_t)stream>>>(d_amax, (int)fmt, (int)conv, margin, d_bias,
                                                                   ctx->d_status);
     return cudaGetLastError() == cudaSuccess ? FP8_OK : FP8_ERR_CUDA;
@@ -241,6 +244,7 @@ fp8_status_t fp8_amax_history_bias(fp8_ctx *ctx, float *d_history, int32_t len, 
     if (!ctx || !d_history || !d_cursor || !d_amax_new || !d_bias) return FP8_ERR_NULL;
     if ((int)fmt < 0 || (int)fmt > 1 || (int)conv < 0 || (int)conv > 1) return FP8_ERR_DTYPE;
     if (len <= 0 || len > 65536) return FP8_ERR_SHAPE;
+    fp8lin::count_launch();
     fp8lin::amax_history_kernel<<<1, 32, 0, (cudaStream_t)stream>>>(d_history, len, d_cursor, d_amax_new, (int)fmt,
                                                                    (int)conv, margin, d_bias, ctx->d_status);
     return cudaGetLastError() == cudaSuccess ? FP8_OK : FP8_ERR_CUDA;

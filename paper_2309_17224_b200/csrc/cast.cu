@@ -317,6 +317,7 @@ static cudaError_t launch_predicted(fp8_ctx *ctx, const void *x, int64_t n, int 
     int blocks = (int)(want < 1 ? 1 : (want > max_blocks ? max_blocks : want));
     unsigned *slot = take_slot(ctx);
     const int delta = format_delta(FMT, conv);
+    count_launch(verify ? 2 : 1);  // this kernel and, when the guess is verified, the gated second pass below
     cast_predicted_kernel<FMT, DT><<<blocks, kCastThreads, 0, stream>>>(
         reinterpret_cast<const uint4 *>(x), reinterpret_cast<uint4 *>(y), nout, ntail, FMT, conv, margin, delta, slot,
         d_amax, d_bias_in, d_bias_inout, verify, ctx->d_status, ctx->d_predict_stats);
@@ -464,6 +465,7 @@ static cudaError_t launch_small(fp8_ctx *ctx, const void *x, int64_t n, int conv
     attr.val.clusterDim.z = 1;
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
+    count_launch();
     return cudaLaunchKernelEx(&cfg, cast_small_kernel<FMT, DT>, reinterpret_cast<const uint4 *>(x),
                               reinterpret_cast<uint4 *>(y), nvec, ntail, (int)FMT, conv, margin, format_delta(FMT, conv),
                               d_amax, d_bias, ctx->d_status);
@@ -661,7 +663,7 @@ fp8_status_t fp8_range_stats(fp8_ctx *ctx, fp8_format_t fmt, const void *x, fp8_
     if (cudaMemsetAsync(d_counts, 0, 4 * sizeof(unsigned long long), st) != cudaSuccess) return FP8_ERR_CUDA;
     const int delta = format_delta((int)fmt, (int)conv);
     const int blocks = (int)(rows < ctx->sm_count * 8 ? rows : ctx->sm_count * 8);
-#define FP8LIN_STATS(F, D) range_stats_kernel<F, D><<<blocks, 256, 0, st>>>(x, rows, cols, ld, d_bias, delta, d_counts)
+#define FP8LIN_STATS(F, D) count_launch(), range_stats_kernel<F, D><<<blocks, 256, 0, st>>>(x, rows, cols, ld, d_bias, delta, d_counts)
     if (fmt == FP8_E4) {
         if (x_dt == FP8_BF16) FP8LIN_STATS(FP8_E4, FP8_BF16);
         else if (x_dt == FP8_F16) FP8LIN_STATS(FP8_E4, FP8_F16);

@@ -5,9 +5,17 @@
 
 namespace fp8lin {
 cudaError_t configure_gemm_kernels(int max_smem_optin);  // gemm.cu
+std::atomic<unsigned long long> g_kernel_launches{0};
 }
 
 extern "C" {
+
+fp8_status_t fp8_launch_count(uint64_t *count)
+{
+    if (!count) return FP8_ERR_NULL;
+    *count = (uint64_t)fp8lin::g_kernel_launches.load(std::memory_order_relaxed);
+    return FP8_OK;
+}
 
 const char *fp8_status_string(fp8_status_t s)
 {

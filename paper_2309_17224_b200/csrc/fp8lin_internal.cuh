@@ -1,6 +1,8 @@
 // Internal declarations shared by the translation units of libfp8lin.so.
 #pragma once
 
+#include <atomic>
+
 #include <cuda.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -80,6 +82,10 @@ __host__ __device__ inline int bias_from_amax_bits(uint32_t bits, int fmt, int c
     return e_max - e - (frac > frac_max ? 1 : 0) - margin;
 }
 
+// Kernels this library has launched in this process (fp8_launch_count); bumped beside every launch.
+extern std::atomic<unsigned long long> g_kernel_launches;
+inline void count_launch(int n = 1) { g_kernel_launches.fetch_add((unsigned long long)n, std::memory_order_relaxed); }
+
 // Launch allowed to start while the launch before it on the stream drains (programmatic dependent launch); the
 // kernel itself waits (griddepcontrol.wait) before it touches anything an earlier launch may have written.
 template <typename... KArgs, typename... Args>
@@ -95,6 +101,7 @@ inline cudaError_t launch_dependent(void (*kernel)(KArgs...), unsigned grid, uns
     cfg.stream = stream;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
+    count_launch();
     return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 

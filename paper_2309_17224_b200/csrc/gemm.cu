@@ -1602,6 +1602,7 @@ static fp8_status_t run_gemm(fp8_ctx *ctx, const uint8_t *a, int a_fmt, bool a_m
               ((uint32_t)p.b_mn << 16);
     if (d_amax_out && cudaMemsetAsync(d_amax_out, 0, sizeof(float), st) != cudaSuccess) return FP8_ERR_CUDA;
     int tiles = p.tiles_m * p.tiles_n;
+    count_launch(p.splits > 1 ? 2 : 1);
     if (pair) {
         int pairs = tiles < g_max_pairs ? tiles : g_max_pairs;
         const dim3 grid(2 * pairs);
@@ -1708,6 +1709,7 @@ fp8_status_t fp8_selftest_wait_expiry(fp8_ctx *ctx, uint64_t limit_ns, void *str
     if (limit_ns == 0 || limit_ns > 100ull * 1000ull * 1000ull) return FP8_ERR_SHAPE;   // at most 100 ms
     cudaStream_t st = (cudaStream_t)stream;
     unsigned *done = ctx->d_slots + (kReduceSlots - 1) * kSlotWords + 3;   // a word no reduction reads
+    count_launch();
     wait_expiry_probe_kernel<<<1, 64, 0, st>>>((unsigned long long)limit_ns, ctx->d_status, done);
     if (cudaGetLastError() != cudaSuccess) return FP8_ERR_CUDA;
     unsigned host = 0;

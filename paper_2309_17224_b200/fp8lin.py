@@ -10,7 +10,7 @@ from __future__ import annotations
 
 import ctypes
 import os
-from ctypes import c_int, c_int32, c_int64, c_uint, c_void_p, c_float, c_char_p, POINTER, byref
+from ctypes import c_int, c_int32, c_int64, c_uint, c_uint64, c_void_p, c_float, c_char_p, POINTER, byref
 
 import torch
 
@@ -31,7 +31,7 @@ SYMBOLS = (
     "fp8_create", "fp8_destroy", "fp8_status_string", "fp8_device_flags", "fp8_amax", "fp8_scaling_bias",
     "fp8_scaling_bias_host", "fp8_cast_e4", "fp8_cast_e5", "fp8_ptq_weights", "fp8_linear_fwd", "fp8_linear_dgrad",
     "fp8_linear_wgrad", "fp8_amax_noalloc", "fp8_linear_fwd_act", "fp8_cast_predicted", "fp8_prediction_stats",
-    "fp8_linear_dgrad_act", "fp8_selftest_wait_expiry", "fp8_range_stats", "fp8_linear_fwd_q", "fp8_linear_dgrad_q", "fp8_amax_history_bias",
+    "fp8_linear_dgrad_act", "fp8_selftest_wait_expiry", "fp8_range_stats", "fp8_linear_fwd_q", "fp8_linear_dgrad_q", "fp8_amax_history_bias", "fp8_launch_count",
 )
 
 if not os.path.exists(LIB_PATH):
@@ -103,6 +103,13 @@ _DT = {torch.bfloat16: BF16, torch.float16: F16, torch.float32: F32}
 def _ld(x):
     """Leading dimension of a 2-D tensor (torch leaves the stride of a size-1 dimension arbitrary)."""
     return x.stride(0) if x.shape[0] > 1 else x.shape[1]
+
+
+def launch_count() -> int:
+    """Kernels this library has launched in this process so far."""
+    out = c_uint64(0)
+    _check(_lib.fp8_launch_count(byref(out)), "fp8_launch_count")
+    return out.value
 
 
 def scaling_bias_host(amax: float, fmt: int, conv: int = CONV_PAPER, margin: int = 0) -> int:

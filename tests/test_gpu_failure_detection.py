@@ -78,3 +78,29 @@ def test_matmuls_write_nothing_outside_their_outputs(ctx, lib, T, K, N):
             assert_bf16_within_one_ulp(bits_of(outs["y"][1]), O.linear_fwd_np(x8h, bx + 1, w8h, bw + 1))
             assert_bf16_within_one_ulp(bits_of(outs["dx"][1]), O.linear_dgrad_np(g8h, bg, w8h, bw + 1))
             assert_bf16_within_one_ulp(bits_of(outs["dw"][1]), O.linear_wgrad_np(g8h, bg, x8h, bx + 1))
+
+
+def test_launch_count_counts_what_a_call_enqueues(ctx, lib):
+    """fp8_launch_count: two launches for amax + cast of a large tensor, one for a decode-size one, one for a cast
+    under a given bias, one or two for a matmul (two when the contraction is split)."""
+    x = torch.randn(2048, 1024, device="cuda").to(torch.bfloat16)
+    small = torch.randn(4, 1024, device="cuda").to(torch.bfloat16)
+    y, ys = torch.empty((2048, 1024), dtype=torch.uint8, device="cuda"), torch.empty((4, 1024), dtype=torch.uint8, device="cuda")
+    a = torch.zeros(1, dtype=torch.float32, device="cuda")
+    b = torch.zeros(1, dtype=torch.int32, device="cuda")
+    def span(fn):
+        n0 = lib.launch_count()
+        fn()
+        return lib.launch_count() - n0
+    assert span(lambda: ctx.cast_e4(x, None, d_amax_out=a, d_bias_out=b, y=y)) == 2
+    assert span(lambda: ctx.cast_e4(small, None, d_amax_out=a, d_bias_out=b, y=ys)) == 1
+    assert span(lambda: ctx.cast_e4(x, b, y=y)) == 1
+    assert span(lambda: ctx.amax(x, a)) == 1
+    w8 = torch.zeros((1024, 1024), dtype=torch.uint8, device="cuda")
+    out = torch.empty((2048, 1024), dtype=torch.bfloat16, device="cuda")
+    assert span(lambda: ctx.linear_fwd(y, b, w8, b, out)) == 1
+    w_long = torch.zeros((512, 8192), dtype=torch.uint8, device="cuda")
+    x_long = torch.zeros((4, 8192), dtype=torch.uint8, device="cuda")
+    out2 = torch.empty((4, 512), dtype=torch.bfloat16, device="cuda")
+    assert span(lambda: ctx.linear_fwd(x_long, b, w_long, b, out2)) == 2       # two tiles, long contraction: split + finalize
+    torch.cuda.synchronize()

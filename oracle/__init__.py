@@ -139,6 +139,15 @@ def f32_to_bf16_bits(x: np.ndarray) -> np.ndarray:
     return out
 
 
+def f32_to_bf16_bits_np(x: np.ndarray) -> np.ndarray:
+    """float32 -> bf16 bit patterns, round to nearest even (NaN stays NaN), on whole arrays; the same rule as
+    ``orc_f32_to_bf16`` (tests/test_oracle_gemm.py holds the two together)."""
+    u = np.ascontiguousarray(x, dtype=np.float32).view(np.uint32).astype(np.uint64)
+    nan = (u & 0x7FFFFFFF) > 0x7F800000
+    rounded = (u + 0x7FFF + ((u >> 16) & 1)) >> 16
+    return np.where(nan, (u >> 16) | 0x40, rounded).astype(np.uint16)
+
+
 # ----------------------------------------------------------------------------
 # amax, bias, cast
 # ----------------------------------------------------------------------------
@@ -161,8 +170,8 @@ def scaling_bias(amax_value: float, kind: int, conv: int = CONV_PAPER, margin: i
 
 
 def history_bias(amax_window, kind: int, conv: int = CONV_PAPER, margin: int = 0) -> int:
-    """Amax-history scaling (Section 3: rely on the past history of the absolute max): the bias for the next
-    step is Eq. 3 on the largest amax of the window, minus the margin."""
+    """Amax-history scaling (Section 3: scale from earlier steps' amax instead of a second pass over the
+    tensor): the bias for the next step is Eq. 3 on the largest amax of the window, minus the margin."""
     return scaling_bias(max(float(a) for a in amax_window), kind, conv, margin)
 
 
@@ -272,22 +281,20 @@ def linear_samples(kind, a8, fa, s_a, b8, fb, s_b, rows, cols, bias_vec=None) ->
 # ----------------------------------------------------------------------------
 # the same matmul definitions with numpy's float64 matmul as the summation step
 # ----------------------------------------------------------------------------
-# Every product of two FP8 values is a small multiple of a power of two, and
-# sums of up to 2^16 of them stay far inside float64's 53 bits, so the float64
-# sum is exact whatever order a BLAS adds in.  These functions therefore return
-# exactly what the plain C loops return (tests/test_oracle_gemm.py checks that
-# equality); they exist because the C loops need minutes where a 24-layer
-# trajectory or a full-size layer has to be checked.
+# Every product of two FP8 values is a small multiple of a power of two, so a float64 sum of them is exact as long
+# as the terms' exponents span less than float64's 53 bits; with E5 x E4 operands over the formats' full range
+# they can span more, and a BLAS may then differ from the plain C loops by a rounding of the float64 sum (a
+# relative 2^-53 or so of sum |a*b|: nine orders of magnitude inside the 2^-14 bar).  So these functions return
+# what the plain C loops return exactly after the rounding to float32 / bf16 except at a float64-level tie, and to
+# 2^-50 relative in float64 (tests/test_oracle_gemm.py checks both); they exist because the C loops need minutes
+# where a 24-layer trajectory or a full-size layer has to be checked.
 
 class _NpResult:
     def __init__(self, f64, abs_sum):
         self.f64 = f64
         self.abs_sum = abs_sum
         self.f32 = f64.astype(np.float32)
-        u = self.f32.view(np.uint32).astype(np.uint64)
-        nan = (u & 0x7FFFFFFF) > 0x7F800000
-        rounded = (u + 0x7FFF + ((u >> 16) & 1)) >> 16
-        self.bf16 = np.where(nan, (u >> 16) | 0x40, rounded).astype(np.uint16)
+        self.bf16 = f32_to_bf16_bits_np(self.f32)
 
 
 def _matmul_unscale(A, B_t, shift_sum, bias_vec=None):

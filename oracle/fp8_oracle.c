@@ -341,23 +341,27 @@ void orc_linear_samples(int kind, const uint8_t *a8, int fa, int s_a, const uint
                         const int64_t *row, const int64_t *col, int64_t count, double *out64,
                         float *out32, uint16_t *out_bf16, double *out_abs)
 {
-#pragma omp parallel for schedule(static)
+    /* Eq. 4 evaluated once per code of each operand's format; the sums below read these values
+     * in the same order as the full products above. */
+    double va[256], vb[256];
+    for (unsigned c = 0; c < 256; ++c) { va[c] = orc_decode(fa, c); vb[c] = orc_decode(fb, c); }
+#pragma omp parallel for schedule(dynamic, 256)
     for (int64_t i = 0; i < count; ++i) {
         int64_t r = row[i], c = col[i];
         double s = 0.0, t = 0.0;
         if (kind == 0) { /* Y[r=t, c=n] */
             for (int64_t k = 0; k < K; ++k) {
-                double p = orc_decode(fa, a8[r * K + k]) * orc_decode(fb, b8[c * K + k]);
+                double p = va[a8[r * K + k]] * vb[b8[c * K + k]];
                 s += p; t += fabs(p);
             }
         } else if (kind == 1) { /* dX[r=t, c=k] */
             for (int64_t n = 0; n < N; ++n) {
-                double p = orc_decode(fa, a8[r * N + n]) * orc_decode(fb, b8[n * K + c]);
+                double p = va[a8[r * N + n]] * vb[b8[n * K + c]];
                 s += p; t += fabs(p);
             }
         } else { /* dW[r=n, c=k] */
             for (int64_t tt = 0; tt < T; ++tt) {
-                double p = orc_decode(fa, a8[tt * N + r]) * orc_decode(fb, b8[tt * K + c]);
+                double p = va[a8[tt * N + r]] * vb[b8[tt * K + c]];
                 s += p; t += fabs(p);
             }
         }

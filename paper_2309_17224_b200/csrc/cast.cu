@@ -524,7 +524,11 @@ __global__ void __launch_bounds__(256) range_stats_kernel(const void *__restrict
     }
 }
 
+#ifdef FP8LIN_EXPERIMENTS
 static const bool g_no_small_cast = [] { const char *e = getenv("FP8LIN_NO_SMALL_CAST"); return e && e[0] == '1'; }();
+#else
+constexpr bool g_no_small_cast = false;
+#endif
 
 static fp8_status_t cast_entry(int fmt, fp8_ctx *ctx, const void *x, fp8_dtype_t x_dt, int64_t rows, int64_t cols,
                                int64_t ld, const int32_t *d_bias, fp8_conv_t conv, int32_t margin, float *d_amax_out,

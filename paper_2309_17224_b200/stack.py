@@ -69,6 +69,14 @@ class Fp8Stack:
         # per layer: amax / bias of W, X, dY
         self.amax = torch.zeros((layers, 3), dtype=torch.float32, **dev)
         self.bias = torch.zeros((layers, 3), dtype=torch.int32, **dev)
+        # layers whose tensors the current step keeps copies of (inputs and outputs of every library call), for
+        # comparisons made outside this module; empty in normal use
+        self.snap_layers = ()
+        self.snap: Dict[int, Dict[str, torch.Tensor]] = {}
+
+    def _keep(self, l: int, **tensors) -> None:
+        if l in self.snap_layers:
+            self.snap.setdefault(l, {}).update({k: v.clone() for k, v in tensors.items()})
 
     def flops_per_step(self) -> float:
         return 3.0 * 2.0 * self.T * self.d * self.d * self.L
@@ -90,6 +98,7 @@ class Fp8Stack:
                 x, have_amax = self.act, True
             else:
                 c.linear_fwd(self.x8[l], self.bias[l, 1:2], self.w8[l], self.bias[l, 0:1], self.y[l])
+                self._keep(l, x=x, w=w16, x8=self.x8[l], w8=self.w8[l], y=self.y[l])
                 have_amax = False
                 if l + 1 < self.L:
                     x = gelu_bf16(self.y[l])
@@ -112,7 +121,9 @@ class Fp8Stack:
                                    self.gact, d_amax_act=self.amax[l - 1, 2:3])
             else:
                 c.linear_dgrad(self.g8, self.bias[l, 2:3], None, self.w8t[l], self.bias[l, 0:1], self.dx)
+                self._keep(l, dx=self.dx)
             c.linear_wgrad(None, self.g8t, self.bias[l, 2:3], None, self.x8t[l], self.bias[l, 1:2], self.dw, self.T)
+            self._keep(l, g=g, g8=self.g8, dw=self.dw, amax=self.amax[l], bias=self.bias[l])
             self.w32[l].add_(self.dw.to(torch.float32), alpha=-self.lr)
             if l > 0:
                 if self.fused:
@@ -120,7 +131,10 @@ class Fp8Stack:
                 else:
                     g = (self.dx.to(torch.float32) * gelu_grad_f32(self.y[l - 1])).to(torch.bfloat16)
 
-    def step(self, step: int) -> Dict[str, object]:
+    def step(self, step: int, snap_layers=()) -> Dict[str, object]:
+        """One training step.  `snap_layers`: layers whose tensors (every input and output of the library calls of
+        this step) are copied into `self.snap[layer]`."""
+        self.snap_layers, self.snap = tuple(snap_layers), {}
         x = step_input(self.x_base, step)
         out = self.forward(x)
         loss = torch.mean((out.to(torch.float32) - self.target.to(torch.float32)) ** 2)
@@ -151,11 +165,12 @@ class Fp8StackHistory(Fp8Stack):
             c.scaling_bias(self.amax[l, 2:3], fp8lin_E5, CONV_PAPER, self.margin, self.pred[l, 2:3])
         self.have_history = True
 
-    def step(self, step: int) -> Dict[str, object]:
+    def step(self, step: int, snap_layers=()) -> Dict[str, object]:
         if not self.have_history:
             rec = super().step(step)
             self._update_history()
             return rec
+        self.snap_layers, self.snap = tuple(snap_layers), {}
         c, L, T = self.ctx, self.L, self.T
         x = step_input(self.x_base, step)
         # the input of the first layer is the one activation no matmul produces: one pass, predicted bias
@@ -169,6 +184,9 @@ class Fp8StackHistory(Fp8Stack):
                                self.pred[l + 1, 1:2], y_pre=self.y[l], d_amax_z=self.amax[l + 1, 1:2], act=ACT_GELU)
             else:
                 c.linear_fwd(self.x8[l], self.pred[l, 1:2], self.w8[l], self.bias[l, 0:1], self.y[l])
+            self._keep(l, w=w16, x8=self.x8[l], w8=self.w8[l], y=self.y[l], bias_x=self.pred[l, 1:2],
+                       bias_w=self.bias[l, 0:1], **({"x8_next": self.x8[l + 1], "bias_next": self.pred[l + 1, 1:2],
+                                                     "amax_next": self.amax[l + 1, 1:2]} if l + 1 < L else {}))
         out = self.y[L - 1].to(torch.float32)
         loss = torch.mean((out - self.target.to(torch.float32)) ** 2)
         g = ((out - self.target.to(torch.float32)) * (2.0 / (T * self.d))).to(torch.bfloat16)
@@ -181,6 +199,8 @@ class Fp8StackHistory(Fp8Stack):
                 c.linear_dgrad_q(cur, self.pred[l, 2:3], self.w8[l], None, self.bias[l, 0:1], nxt, self.pred[l - 1, 2:3],
                                  y_pre=self.y[l - 1], d_amax_g=self.amax[l - 1, 2:3], act=ACT_GELU)
             c.linear_wgrad(cur, None, self.pred[l, 2:3], self.x8[l], None, self.pred[l, 1:2], self.dw, T)
+            self._keep(l, g8=cur, bias_g=self.pred[l, 2:3], dw=self.dw,
+                       **({"g8_next": nxt, "bias_g_next": self.pred[l - 1, 2:3], "y_below": self.y[l - 1]} if l > 0 else {}))
             self.w32[l].add_(self.dw.to(torch.float32), alpha=-self.lr)
         used = self.bias.clone()
         used[:, 1:3] = self.pred[:, 1:3]

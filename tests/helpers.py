@@ -54,18 +54,61 @@ def bf16_bits_to_f64(b: np.ndarray) -> np.ndarray:
     return (b.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
 
 
-def assert_bf16_within_one_ulp(got_bits: np.ndarray, ref: "O.GemmResult"):
-    """bf16 output within one bf16 ulp of the oracle's rounded value.  Where the
-    sum cancels, one bf16 ulp of the result is finer than the FP32 accumulation
-    bar (2^-14 * sum_k |a*b|); there that bar, plus the half ulp of the output
-    rounding itself, is the one that applies."""
+# The relaxed branch of the bf16 bar (below) is confined to outputs whose sum cancels this far ...
+CANCEL_RATIO = 2.0 ** -10
+# ... and allows this much accumulation error there: 2^-19 * sum|a*b|, about 6.5 times the largest FP32
+# accumulation error measured on the tensor cores in these tests (2^-21.7 * sum|a*b|), far inside the
+# 2^-14 * sum|a*b| bar of the FP32 outputs.
+CANCEL_SLACK = 2.0 ** -19
+# largest share of a tensor's outputs that may need the relaxed branch
+CANCEL_MAX_FRACTION = 0.002   # largest seen on the benchmark-size layers: 2.2e-4
+
+
+def assert_bf16_within_one_ulp(got_bits: np.ndarray, ref: "O.GemmResult", max_fraction: float = CANCEL_MAX_FRACTION):
+    """bf16 output within one bf16 ulp of the oracle's rounded value.
+
+    Where the sum cancels so far that one bf16 ulp of the result is finer than any FP32 accumulation can
+    resolve (|exact| <= 2^-10 * sum_k |a*b|: there half a bf16 ulp is below 2^-19 * sum_k |a*b|), an output may
+    instead lie within 2^-19 * sum_k |a*b| plus the half ulp of its own rounding.  The share of outputs that
+    needed that branch is returned and bounded."""
     d = np.abs(bf16_ordinal(got_bits) - bf16_ordinal(ref.bf16))
     got = bf16_bits_to_f64(got_bits)
     half_ulp = np.abs(ref.f64) * 2.0 ** -8
-    within_acc = np.abs(got - ref.f64) <= ref.abs_sum * 2.0 ** -14 + half_ulp + 2.0 ** -150
-    bad = (d > 1) & ~within_acc
+    cancels = np.abs(ref.f64) <= ref.abs_sum * CANCEL_RATIO
+    within_acc = np.abs(got - ref.f64) <= ref.abs_sum * CANCEL_SLACK + half_ulp + 2.0 ** -150
+    relaxed = (d > 1) & cancels & within_acc
+    bad = (d > 1) & ~relaxed
     if bad.any():
         i = np.argwhere(bad)[0]
         raise AssertionError(f"{bad.sum()} bf16 outputs differ by more than one ulp; first at {i.tolist()}: "
                              f"got {hex(got_bits[tuple(i)])} want {hex(ref.bf16[tuple(i)])}")
-    return float((d > 1).mean())
+    frac = float(relaxed.mean()) if relaxed.size else 0.0
+    assert frac <= max_fraction, f"{frac:.4f} of the outputs needed the cancellation branch (bound {max_fraction})"
+    return frac
+
+
+def tile_sample_positions(rng, R: int, C: int, per_tile: int = 64, tile: int = 128, full_tiles: int = 8):
+    """Output positions that cover a matmul result of R x C: `per_tile` random positions inside EVERY tile x tile
+    block (ragged edge blocks included), every element of at least `full_tiles` whole blocks (the four corners of
+    the block grid, the rest drawn at random), and the complete first and last rows and columns."""
+    tr, tc = (R + tile - 1) // tile, (C + tile - 1) // tile
+    r0 = np.repeat(np.arange(tr) * tile, tc)
+    c0 = np.tile(np.arange(tc) * tile, tr)
+    h = np.minimum(tile, R - r0)
+    w = np.minimum(tile, C - c0)
+    rows = [(r0[:, None] + (rng.random((tr * tc, per_tile)) * h[:, None]).astype(np.int64)).reshape(-1)]
+    cols = [(c0[:, None] + (rng.random((tr * tc, per_tile)) * w[:, None]).astype(np.int64)).reshape(-1)]
+    blocks = {(0, 0), (0, tc - 1), (tr - 1, 0), (tr - 1, tc - 1)}
+    want = min(full_tiles, tr * tc)
+    while len(blocks) < want:
+        blocks.add((int(rng.integers(0, tr)), int(rng.integers(0, tc))))
+    for br, bc in sorted(blocks):
+        rr = np.arange(br * tile, min(R, (br + 1) * tile))
+        cc = np.arange(bc * tile, min(C, (bc + 1) * tile))
+        g = np.meshgrid(rr, cc, indexing="ij")
+        rows.append(g[0].reshape(-1)); cols.append(g[1].reshape(-1))
+    for r in {0, R - 1}:
+        rows.append(np.full(C, r)); cols.append(np.arange(C))
+    for c in {0, C - 1}:
+        rows.append(np.arange(R)); cols.append(np.full(R, c))
+    return np.concatenate(rows).astype(np.int64), np.concatenate(cols).astype(np.int64)

@@ -220,6 +220,26 @@ def test_saturation_flag_and_constant_scale(ctx, lib):
     assert bool((y == 0x7E).all())
 
 
+@pytest.mark.parametrize("top,flag", [(240.0, True), (236.0, True), (233.0, True), (232.0, False), (200.0, False)])
+def test_paper_convention_raises_saturated_when_amax_rounds_to_the_240_code(ctx, lib, top, flag):
+    """Just-in-time FP8-AMAX under the paper convention: a scaled amax in (232, 240] would take the paper format's
+    top code, which has no native byte; the cast emits 224 (byte 0x7E) and raises FP8_FLAG_SATURATED.  Same bytes
+    as the oracle; the native convention raises nothing."""
+    x = (torch.randn((64, 256), device="cuda") * 20.0).clamp(-200, 200).to(torch.bfloat16)
+    x[3, 5], x[60, 255] = top, -top
+    for conv, expect in ((lib.CONV_PAPER, flag), (lib.CONV_NATIVE, False)):
+        ctx.device_flags(clear=True)
+        y = torch.empty(x.shape, dtype=torch.uint8, device="cuda")
+        amax, bias = _dev_scalar(torch.float32), _dev_scalar(torch.int32, 99)
+        ctx.cast_e4(x, None, conv=conv, d_amax_out=amax, d_bias_out=bias, y=y)
+        a, b, ref = O.quantise(bits_of(x), O.E4, conv)
+        assert (float(amax.item()), int(bias.item())) == (a, b) and a == top and (b == 0 or conv == lib.CONV_NATIVE)
+        assert_codes_equal(u8(y), ref, O.N_E4)
+        assert bool(ctx.device_flags(clear=True) & lib.FLAG_SATURATED) == expect
+        if conv == lib.CONV_PAPER and top > 216:
+            assert u8(y)[3, 5] == 0x7E and u8(y)[60, 255] == 0xFE
+
+
 def test_argument_errors(ctx, lib):
     x = torch.zeros((16, 16), dtype=torch.bfloat16, device="cuda")
     y = torch.zeros((16, 16), dtype=torch.uint8, device="cuda")

@@ -9,7 +9,8 @@ import pytest
 import torch
 
 import oracle as O
-from helpers import (assert_bf16_within_one_ulp, assert_codes_equal, assert_gemm_close, bits_of, u8)
+from helpers import (assert_bf16_within_one_ulp, assert_codes_equal, assert_gemm_close, bits_of, tile_sample_positions,
+                     u8)
 from paper_2309_17224_b200 import inputs as I
 
 pytestmark = pytest.mark.gpu
@@ -31,20 +32,22 @@ def ctx(lib):
 class Quantised:
     """One tensor quantised on the GPU (both layouts) and by the oracle."""
 
-    def __init__(self, ctx, x, kind, conv, margin=0):
+    def __init__(self, ctx, x, kind, conv, margin=0, transposed=True):
+        """transposed=False asks for the row-major bytes only, which is what the benchmark's steps do."""
         rows, cols = x.shape
         self.kind, self.conv = kind, conv
         self.amax = torch.zeros(1, dtype=torch.float32, device="cuda")
         self.bias = torch.zeros(1, dtype=torch.int32, device="cuda")
         self.y = torch.empty((rows, cols), dtype=torch.uint8, device="cuda")
-        self.y_t = torch.empty((cols, rows), dtype=torch.uint8, device="cuda")
+        self.y_t = torch.empty((cols, rows), dtype=torch.uint8, device="cuda") if transposed else None
         cast = ctx.cast_e4 if kind == O.E4 else ctx.cast_e5
         cast(x, None, conv=conv, margin=margin, d_amax_out=self.amax, d_bias_out=self.bias, y=self.y, y_t=self.y_t)
-        a, b, ref, ref_t = O.quantise(bits_of(x), kind, conv, margin, transposed=True)
+        a, b, ref = O.quantise(bits_of(x), kind, conv, margin)
         assert float(self.amax.item()) == a and int(self.bias.item()) == b
         fmt = O.native_format(kind)
         assert_codes_equal(u8(self.y), ref, fmt)
-        assert_codes_equal(u8(self.y_t), ref_t, fmt)
+        if transposed:
+            assert_codes_equal(u8(self.y_t), np.ascontiguousarray(ref.T), fmt)
         self.ref, self.ref_bias, self.shift = ref, b, b + O.delta(kind, conv)
 
 
@@ -220,23 +223,20 @@ def test_matmul_argument_errors(ctx, lib):
     assert e.value.status == lib.ERR_NULL
 
 
-def _sample_positions(rng, R, C, n):
-    rows = np.concatenate([rng.integers(0, R, n), [0, R - 1, 0, R - 1]])
-    cols = np.concatenate([rng.integers(0, C, n), [0, C - 1, C - 1, 0]])
-    return rows, cols
-
-
-@pytest.mark.parametrize("wl_name,layer", [("c2_gpt", 0), ("c2_gpt", 3), ("c3_llama7b", 1), ("c3_llama7b", 3)])
+@pytest.mark.parametrize("wl_name,layer", [("c2_gpt", 0), ("c2_gpt", 1), ("c2_gpt", 2), ("c2_gpt", 3),
+                                           ("c3_llama7b", 0), ("c3_llama7b", 1), ("c3_llama7b", 2), ("c3_llama7b", 3)])
 def test_full_size_layers_sampled(ctx, lib, wl_name, layer):
-    """Benchmark-size layers in the benchmark's launch configuration: bytes and
-    biases checked in full, matmul outputs at sampled positions."""
+    """Every layer of the GPT block and of the Llama-2-7B block at benchmark size, in the benchmark's launch
+    configuration (forward layouts, no transposed copies): bytes and biases checked in full; each matmul output
+    at 64 positions in every 128 x 128 block, on eight whole blocks and on its first / last rows and columns."""
     wl = I.WORKLOADS[wl_name]
     l = wl.layers[layer]
     T, K, N = wl.tokens, l.K, l.N
     t = I.layer_tensors(wl, layer, device="cuda")
-    qx = Quantised(ctx, t["x"], O.E4, O.CONV_PAPER)
-    qw = Quantised(ctx, t["w"], O.E4, O.CONV_PAPER)
-    qg = Quantised(ctx, t["g"], O.E5, O.CONV_PAPER)
+    qx = Quantised(ctx, t["x"], O.E4, O.CONV_PAPER, transposed=False)
+    qw = Quantised(ctx, t["w"], O.E4, O.CONV_PAPER, transposed=False)
+    qg = Quantised(ctx, t["g"], O.E5, O.CONV_PAPER, transposed=False)
+    del t
     y = torch.empty((T, N), dtype=torch.bfloat16, device="cuda")
     dx = torch.empty((T, K), dtype=torch.bfloat16, device="cuda")
     dw = torch.empty((N, K), dtype=torch.bfloat16, device="cuda")
@@ -249,10 +249,29 @@ def test_full_size_layers_sampled(ctx, lib, wl_name, layer):
              (O.DGRAD, dx, (qg.ref, O.N_E5, qg.shift, qw.ref, O.N_E4, qw.shift)),
              (O.WGRAD, dw, (qg.ref, O.N_E5, qg.shift, qx.ref, O.N_E4, qx.shift)))
     for kind, out, ops in cases:
-        rows, cols = _sample_positions(rng, out.shape[0], out.shape[1], 4000)
+        rows, cols = tile_sample_positions(rng, out.shape[0], out.shape[1])
         ref = O.linear_samples(kind, *ops, rows, cols)
         got = bits_of(out)[rows, cols]
-        assert_bf16_within_one_ulp(got, ref)
+        frac = assert_bf16_within_one_ulp(got, ref)
+        print(f"[parity] {wl_name}/{l.name} kind {kind}: {rows.size} positions, {frac:.5f} through the cancellation branch")
+
+
+@pytest.mark.parametrize("T,K,N", [(256, 768, 768), (400, 1040, 784), (16, 4096, 1280), (3, 16384, 272)])
+def test_bf16_output_is_the_rounded_fp32_output(ctx, lib, T, K, N):
+    """The bf16 result of a call equals the FP32 result of the same call on the same operands rounded to bf16
+    (nearest even), bit for bit: the two output types differ in the last step of the epilogue only.  Covers the
+    CTA-pair kernel, the single-CTA kernel and the split contraction with its finishing kernel."""
+    qx, qw, qg = _layer(ctx, T, K, N, O.CONV_PAPER, seed=31337 + T)
+    calls = (lambda out: ctx.linear_fwd(qx.y, qx.bias, qw.y, qw.bias, out), (T, N)), \
+            (lambda out: ctx.linear_dgrad(qg.y, qg.bias, qw.y, None, qw.bias, out), (T, K)), \
+            (lambda out: ctx.linear_wgrad(qg.y, None, qg.bias, qx.y, None, qx.bias, out, T), (N, K))
+    for call, shape in calls:
+        o32 = torch.full(shape, float("nan"), dtype=torch.float32, device="cuda")
+        o16 = torch.full(shape, float("nan"), dtype=torch.bfloat16, device="cuda")
+        call(o32)
+        call(o16)
+        assert np.array_equal(bits_of(o16), O.f32_to_bf16_bits_np(o32.cpu().numpy()))
+    assert ctx.device_flags(clear=True) & lib.FLAG_TIMEOUT == 0
 
 
 @pytest.mark.parametrize("T,K,N", [(1, 2048, 768), (16, 4096, 1280), (64, 8192, 512), (100, 1024, 2304),
@@ -299,37 +318,58 @@ def test_decode_shapes_dgrad_from_row_major_weights(ctx, lib, T, N, K):
     assert ctx.device_flags(clear=True) & lib.FLAG_TIMEOUT == 0
 
 
-@pytest.mark.parametrize("layer,tokens", [(1, 1), (0, 16), (1, 64), (3, 64)])
+class _PtqLayer:
+    """One weight tensor of config 4 quantised once on the GPU (fp8_ptq_weights) and once by the oracle; bytes,
+    amax and bias compared in full here, then shared by every token count."""
+
+    def __init__(self, ctx, lib, layer):
+        wl = I.WORKLOADS["c4_llama70b_ptq"]
+        l = wl.layers[layer]
+        self.K, self.N, self.name = l.K, l.N, l.name
+        w = I.layer_tensors(wl, layer, device="cuda", tokens=16, want=("w",))["w"]
+        self.w8 = torch.empty((l.N, l.K), dtype=torch.uint8, device="cuda")
+        self.amax = torch.zeros(1, dtype=torch.float32, device="cuda")
+        self.bias = torch.zeros(1, dtype=torch.int32, device="cuda")
+        ctx.ptq_weights(w, lib.CONV_PAPER, self.w8, None, self.bias, self.amax)
+        a, b, ref = O.quantise(bits_of(w), O.E4)
+        del w
+        assert float(self.amax.item()) == a and int(self.bias.item()) == b
+        assert_codes_equal(u8(self.w8), ref, O.N_E4)
+        self.ref, self.shift = ref, b + 1
+
+
+_ptq_cache = {}
+
+
+def _ptq_layer(ctx, lib, layer):
+    if layer not in _ptq_cache:
+        _ptq_cache.clear()            # one layer's bytes at a time (the largest holds 470 MB on each side)
+        _ptq_cache[layer] = _PtqLayer(ctx, lib, layer)
+    return _ptq_cache[layer]
+
+
+@pytest.mark.parametrize("layer,tokens", [(l, t) for l in (0, 1, 2, 3) for t in (1, 16, 64, 2048)])
 def test_llama70b_ptq_inference_layers(ctx, lib, layer, tokens):
-    """Config 4: weights quantised once (post-training quantisation), forward
-    only, decode-size batches.  Weight bytes are checked on sampled rows (the
-    bias comes from the amax of the whole tensor), outputs at sampled positions."""
+    """Config 4: weights quantised once (post-training quantisation, Section 3.1), forward only; every layer at
+    every token count of the config (decode 1 / 16 / 64, prefill 2048).  Weight bytes are checked in full, the
+    activation's bytes in full, the output at 64 positions per 128 x 128 block, on eight whole blocks and on its
+    first / last rows and columns."""
     wl = I.WORKLOADS["c4_llama70b_ptq"]
-    l = wl.layers[layer]
-    K, N = l.K, l.N
-    t = I.layer_tensors(wl, layer, device="cuda", tokens=tokens)
-    w8 = torch.empty((N, K), dtype=torch.uint8, device="cuda")
-    amax_w = torch.zeros(1, dtype=torch.float32, device="cuda")
-    bias_w = torch.zeros(1, dtype=torch.int32, device="cuda")
-    ctx.ptq_weights(t["w"], lib.CONV_PAPER, w8, None, bias_w, amax_w)
-    wb = bits_of(t["w"])
-    a = O.amax(wb)
-    b = O.scaling_bias(a, O.E4)
-    assert float(amax_w.item()) == a and int(bias_w.item()) == b
-    rng = np.random.default_rng(layer * 100 + tokens)
-    rows = np.sort(rng.choice(N, size=256, replace=False))
-    w8_rows = O.cast(wb[rows], b + 1, O.N_E4)
-    assert_codes_equal(u8(w8)[rows], w8_rows, O.N_E4)
-    qx = Quantised(ctx, t["x"], O.E4, O.CONV_PAPER)
-    y = torch.empty((tokens, N), dtype=torch.bfloat16, device="cuda")
-    ctx.linear_fwd(qx.y, qx.bias, w8, bias_w, y)
+    pw = _ptq_layer(ctx, lib, layer)
+    x = I.layer_tensors(wl, layer, device="cuda", tokens=tokens, want=("x",))["x"]
+    qx = Quantised(ctx, x, O.E4, O.CONV_PAPER, transposed=False)
+    y = torch.empty((tokens, pw.N), dtype=torch.bfloat16, device="cuda")
+    ctx.linear_fwd(qx.y, qx.bias, pw.w8, pw.bias, y)
     assert ctx.device_flags(clear=True) & lib.FLAG_TIMEOUT == 0
-    # outputs in the sampled weight rows: the oracle sees only those rows of W8
-    ti = rng.integers(0, tokens, 3000)
-    ni = rng.integers(0, len(rows), 3000)
-    ref = O.linear_samples(O.FWD, qx.ref, O.N_E4, qx.shift, w8_rows, O.N_E4, b + 1, ti, ni)
-    got = bits_of(y)[ti, rows[ni]]
-    assert_bf16_within_one_ulp(got, ref)
+    rng = np.random.default_rng(layer * 100 + tokens)
+    rows, cols = tile_sample_positions(rng, tokens, pw.N)
+    ref = O.linear_samples(O.FWD, qx.ref, O.N_E4, qx.shift, pw.ref, O.N_E4, pw.shift, rows, cols)
+    frac = assert_bf16_within_one_ulp(bits_of(y)[rows, cols], ref)
+    print(f"[parity] c4/{pw.name} T={tokens}: {rows.size} positions, {frac:.5f} through the cancellation branch")
+
+
+def test_ptq_cache_is_released():
+    _ptq_cache.clear()
 
 
 def test_fused_epilogue_argument_errors(ctx, lib):

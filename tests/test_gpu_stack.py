@@ -4,17 +4,23 @@ stack of FP8 linears (d = 1024, 4096 tokens) whose input scale drifts as
 
 What is compared with what:
   * every step: the bias of the first layer's input against the oracle's bias
-    of the seeded, drifted input (the drift law; nothing from the GPU feeds the
-    oracle);
+    of the seeded, drifted input (the drift law);
   * steps 0, 1, 50, 199: the first layer's input bytes against the oracle's cast;
-  * steps 0 and 1: the oracle runs the whole trajectory from the seeded tensors.
-    Each GPU linear is then given the ORACLE's tensors for three layers of the
-    stack and must reproduce the oracle's bytes bit for bit and its outputs to
-    one bf16 ulp; the free-running GPU trajectory must agree with the oracle's
-    in loss and (away from power-of-two boundaries) in every bias;
-  * steps 50 and 199, where no oracle trajectory can exist: the defining
-    inequality of Eq. 3 for every bias the GPU produced, finite loss, no
-    device time-out.
+  * steps 0, 1, 50 and 199, layers 0, 12 and 23, teacher-forced: the run keeps
+    the bf16 tensors each linear actually saw at that step (input, weight after
+    that many SGD updates, output gradient) and everything the library made of
+    them; the oracle is given those same bf16 tensors and must agree on amax,
+    bias and FP8 bytes bit for bit and on Y, dX, dW to one bf16 ulp.  (A matmul
+    output that differs within tolerance can move the next tensor's amax across
+    a power of two, so two free-running trajectories cannot be compared byte for
+    byte; each op on identical inputs can.)
+  * steps 0 and 1: the oracle also runs the whole trajectory from the seeded
+    tensors.  Each GPU linear is given the ORACLE's tensors for three layers of
+    the stack and must reproduce the oracle's bytes and outputs; the
+    free-running GPU trajectory must agree with the oracle's in loss and (away
+    from power-of-two boundaries) in every bias;
+  * steps 50 and 199 besides: the defining inequality of Eq. 3 for every bias
+    the GPU produced, finite loss, no device time-out.
 """
 from fractions import Fraction
 
@@ -31,6 +37,7 @@ pytestmark = pytest.mark.gpu
 
 CHECK_STEPS = (0, 1, 50, 199)
 LAYERS, D, TOKENS, STEPS = 24, 1024, 4096, 200
+SNAP_LAYERS = (0, LAYERS // 2, LAYERS - 1)
 
 
 @pytest.fixture(scope="module")
@@ -41,15 +48,16 @@ def run():
     seeded = {"w": [bits_of(w.to(torch.bfloat16)) for w in st.w32], "x_base": bits_of(st.x_base),
               "target": bits_of(st.target)}
     trace = []
-    x8_at = {}
+    x8_at, snaps = {}, {}
     for step in range(STEPS):
-        r = st.step(step)
+        r = st.step(step, snap_layers=SNAP_LAYERS if step in CHECK_STEPS else ())
         trace.append(r)
         if step in CHECK_STEPS:
             x8_at[step] = u8(st.x8[0])
+            snaps[step] = {l: {k: v.cpu() for k, v in d.items()} for l, d in st.snap.items()}
     torch.cuda.synchronize()
     flags = ctx.device_flags(clear=True)
-    out = {"lib": fp8lin, "ctx": ctx, "stack": st, "seeded": seeded, "x8_at": x8_at, "flags": flags,
+    out = {"lib": fp8lin, "ctx": ctx, "stack": st, "seeded": seeded, "x8_at": x8_at, "flags": flags, "snaps": snaps,
            "loss": [float(r["loss"].item()) for r in trace],
            "bias": np.stack([r["bias"].cpu().numpy() for r in trace]),
            "amax": np.stack([r["amax"].cpu().numpy() for r in trace])}
@@ -105,6 +113,28 @@ def test_gradient_biases_move_with_the_drift(run):
     bg = run["bias"][:, :, 2]
     assert bg.min() > run["bias"][:, :, 0].max()
     assert len(np.unique(bg[:, 0])) >= 3
+
+
+@pytest.mark.parametrize("step", CHECK_STEPS)
+def test_checked_steps_teacher_forced_against_the_oracle(run, step):
+    """Config 5's comparison at steps 0, 1, 50 and 199: for the first, the middle and the last layer, the oracle
+    quantises the very bf16 tensors the GPU linear saw at that step and multiplies the resulting bytes; amax, bias
+    and bytes must be equal, Y, dX and dW within one bf16 ulp."""
+    for l in SNAP_LAYERS:
+        sn = run["snaps"][step][l]
+        got_amax, got_bias = sn["amax"].tolist(), sn["bias"].tolist()
+        aw, bw, w8 = O.quantise(bits_of(sn["w"]), O.E4)
+        ax, bx, x8 = O.quantise(bits_of(sn["x"]), O.E4)
+        ag, bg, g8 = O.quantise(bits_of(sn["g"]), O.E5)
+        assert got_amax == [aw, ax, ag] and got_bias == [bw, bx, bg], (step, l)
+        assert_codes_equal(u8(sn["w8"]), w8, O.N_E4)
+        assert_codes_equal(u8(sn["x8"]), x8, O.N_E4)
+        assert_codes_equal(u8(sn["g8"]), g8, O.N_E5)
+        assert_bf16_within_one_ulp(bits_of(sn["y"]), O.linear_fwd_np(x8, bx + 1, w8, bw + 1))
+        assert_bf16_within_one_ulp(bits_of(sn["dx"]), O.linear_dgrad_np(g8, bg, w8, bw + 1))
+        assert_bf16_within_one_ulp(bits_of(sn["dw"]), O.linear_wgrad_np(g8, bg, x8, bx + 1))
+    if step >= 50:
+        assert run["bias"][step, 0, 1] != run["bias"][0, 0, 1]   # the input scale has drifted since step 0
 
 
 def test_steps_0_and_1_against_the_oracle_trajectory(run):
@@ -167,11 +197,22 @@ def test_history_scaling_stack_against_the_oracle_trajectory():
         orc = OS.OracleStack([bits_of(w.to(torch.bfloat16)) for w in st.w32], bits_of(st.x_base), bits_of(st.target),
                              lr=1e-3, history=True, margin=margin)
         for step in range(steps):
-            r = st.step(step)
+            r = st.step(step, snap_layers=(0, L // 2, L - 1) if step == steps - 1 else ())
             flags = ctx.device_flags(clear=True)
             assert flags & fp8lin.FLAG_TIMEOUT == 0
             if step > 0:
                 assert flags & fp8lin.FLAG_SATURATED == 0
+            if step == steps - 1:
+                # teacher-forced: the oracle multiplies the bytes the GPU matmuls were given at this step, under the
+                # biases they were given, and quantises the weight the GPU quantised
+                for l, sn in st.snap.items():
+                    sn = {k: v.cpu() for k, v in sn.items()}
+                    aw, bw, w8 = O.quantise(bits_of(sn["w"]), O.E4)
+                    assert int(sn["bias_w"].item()) == bw
+                    assert_codes_equal(u8(sn["w8"]), w8, O.N_E4)
+                    bx, bg = int(sn["bias_x"].item()), int(sn["bias_g"].item())
+                    assert_bf16_within_one_ulp(bits_of(sn["y"]), O.linear_fwd_np(u8(sn["x8"]), bx + 1, w8, bw + 1))
+                    assert_bf16_within_one_ulp(bits_of(sn["dw"]), O.linear_wgrad_np(u8(sn["g8"]), bg, u8(sn["x8"]), bx + 1))
             rec = orc.step(step)
             assert abs(float(r["loss"].item()) - rec["loss"]) <= 2e-3 * rec["loss"], step
             got = r["bias"].cpu().numpy()

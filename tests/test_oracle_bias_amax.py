@@ -148,3 +148,19 @@ def test_history_bias_is_eq3_on_the_window_maximum():
             assert all(Fraction(a) * Fraction(2) ** b <= mx for a in window)
             assert Fraction(max(window)) * Fraction(2) ** (b + 1) > mx
             assert O.history_bias(window, kind, O.CONV_PAPER, 3) == b - 3
+
+
+def test_paper_e4_top_code_has_no_native_byte():
+    """Table 7 row (a) puts the E4 maximum at 240; read as a native byte its code is NaN.  A tensor whose scaled
+    amax lands in (232, 240] therefore carries 224 (byte 0x7E) for its largest elements under the paper
+    convention, and is untouched under the native convention (max_num 448 leaves it one binade of headroom)."""
+    for top, want in ((236.0, 0x7E), (240.0, 0x7E), (232.0, 0x7E), (231.0, 0x7E), (228.0, 0x7E), (216.0, 0x7E),
+                      (215.0, 0x7D)):
+        x = np.array([[top, -top, 1.0, 0.5]], dtype=np.float32)
+        a, b, y = O.quantise(x, O.E4, O.CONV_PAPER)
+        assert (a, b) == (top, 0)
+        assert y[0, 0] == want and y[0, 1] == (want | 0x80)
+    # what the byte means in paper units: native value / 2
+    assert O.decode(O.N_E4, 0x7E) / 2 == 224.0
+    a, b, y = O.quantise(np.array([[236.0, 1.0]], dtype=np.float32), O.E4, O.CONV_NATIVE)
+    assert b == 0 and O.decode(O.N_E4, int(y[0, 0])) == 240.0   # 236 rounds to 240 on the native grid, no clipping

@@ -5,7 +5,8 @@
  *
  * Conventions that hold for every entry point
  * -------------------------------------------
- *  - Every call returns an fp8_status_t.  Nothing throws, nothing is printed.
+ *  - Every call returns an fp8_status_t.  Nothing throws, nothing is printed
+ *    and no environment variable is read.
  *  - All tensor pointers are DEVICE pointers owned by the caller; the library
  *    never allocates, frees or retains them.  "d_" marks a device scalar.
  *    The only host pointers are the fp8_ctx handle, `flags` of
@@ -74,7 +75,13 @@ typedef enum { FP8_BF16 = 0, FP8_F16 = 1, FP8_F32 = 2 } fp8_dtype_t;
 /* Sticky device status bits. */
 #define FP8_FLAG_NONFINITE_AMAX 1u /* an amax was inf or NaN; its bias was set to 0 */
 #define FP8_FLAG_ZERO_AMAX 2u      /* an amax was 0; its bias was set to 0 */
-#define FP8_FLAG_SATURATED 4u      /* a cast clipped at least one value (finite or infinite) to the format's maximum */
+#define FP8_FLAG_SATURATED 4u      /* a cast clipped at least one value (finite or infinite) to the format's maximum.
+                                    * Under (FP8_E4, FP8_CONV_PAPER) this also fires for a just-in-time FP8-AMAX
+                                    * cast whose scaled amax lands in (232, 240]: Eq. 3 places it at or below the
+                                    * paper format's 240, the one magnitude code with no native counterpart, and
+                                    * the bytes carry 224 instead (about one tensor in twenty; the largest
+                                    * elements lose at most 6.7 %).  FP8_CONV_NATIVE never clips a finite
+                                    * just-in-time cast. */
 #define FP8_FLAG_TIMEOUT 8u        /* a bounded wait inside a kernel expired; that kernel's output is invalid */
 
 typedef struct fp8_ctx fp8_ctx;
@@ -86,8 +93,8 @@ typedef struct fp8_ctx fp8_ctx;
  * shared-memory limit of the matmul kernels.  It must not be called during
  * stream capture.  The context-taking calls that enqueue work (fp8_amax,
  * fp8_scaling_bias, fp8_cast_*, fp8_ptq_weights, fp8_linear_*) neither
- * synchronise nor allocate, and bench.py replays a whole step of them from a
- * CUDA graph. */
+ * synchronise nor allocate, so a whole step of them can be captured into a
+ * CUDA graph and replayed. */
 FP8_API fp8_status_t fp8_create(fp8_ctx **ctx, int device);
 FP8_API fp8_status_t fp8_destroy(fp8_ctx *ctx);
 
@@ -152,9 +159,9 @@ FP8_API fp8_status_t fp8_amax_noalloc(const void *x, fp8_dtype_t x_dt, int64_t r
 FP8_API fp8_status_t fp8_scaling_bias(fp8_ctx *ctx, const float *d_amax, fp8_format_t fmt, fp8_conv_t conv,
                               int32_t margin, int32_t *d_bias, void *stream);
 
-/* Amax history (Section 3: "rely on the past history of absolute max" where a
- * second pass over memory is too costly): a ring of the last `len` amax values of
- * one tensor.  The call stores *d_amax_new at the cursor, advances the cursor
+/* Amax history (Section 3: where a second pass over memory is too costly, the
+ * scale may come from the amax of earlier steps): a ring of the last `len` amax
+ * values of one tensor.  The call stores *d_amax_new at the cursor, advances the cursor
  * (wrapping), and writes to *d_bias the bias Eq. 3 gives for the LARGEST entry of
  * the ring, minus `margin` -- the bias to quantise that tensor with at the next
  * step.  A ring that starts zero-filled ignores its unused entries; an all-zero
@@ -213,6 +220,41 @@ FP8_API fp8_status_t fp8_cast_e5(fp8_ctx *ctx, const void *x, fp8_dtype_t x_dt, 
 FP8_API fp8_status_t fp8_cast_predicted(fp8_ctx *ctx, fp8_format_t fmt, const void *x, fp8_dtype_t x_dt, int64_t rows,
                                         int64_t cols, int64_t ld, fp8_conv_t conv, int32_t margin, float *d_amax_out,
                                         int32_t *d_bias_inout, uint8_t *y, void *stream);
+
+/* FP8-AMAX quantisation of several tensors in one call (Eq. 3, Eq. 1 and the casts of Sections 2.1 / 2.2,
+ * per tensor; the grouping itself has no counterpart in the paper).  Every linear of a step quantises its
+ * weight, and a step usually has several tensors ready at once (all weights after the optimiser update; in a
+ * benchmark also the activations and gradients).  Launched one by one, kernels over tens of megabytes spend a
+ * sizeable share of their time ramping up and draining; this call walks the chunks of all tensors with one
+ * persistent grid per pass, two launches for the whole group.
+ *   items      HOST array of `count` descriptors (read during the call, not retained); each tensor gets its own
+ *              amax and bias, exactly as fp8_cast_e4 / fp8_cast_e5 with d_bias = NULL would give:
+ *                x, x_dt, rows, cols, ld   the input tensor
+ *                fmt, margin               target format and the margin subtracted from its Eq. 3 bias
+ *                d_amax                    out, device float
+ *                d_bias                    out, device int32; with predicted != 0 also IN: the guess
+ *                y                         out [rows, cols] bytes, row-major
+ *   predicted  0: just in time -- one pass takes every amax and bias, a second casts (5 bytes moved per 16-bit
+ *              element).  Non-zero: one pass casts every tensor with the guess found in its d_bias (typically the
+ *              value the previous step left there) while taking its amax; tensors whose guess turns out wrong
+ *              are cast again by the second launch, the others are not touched again (3 bytes per element when
+ *              all guesses hold; fp8_prediction_stats counts hits and misses).  Results are identical in both
+ *              modes, whatever the guesses.
+ * Tensors with ld == cols and 16-byte aligned x and y are grouped (up to FP8_GROUP_MAX per pair of launches, more
+ * are taken in several rounds); any other tensor in the list is handed to fp8_cast_e4 / _e5 / _predicted. */
+#define FP8_GROUP_MAX 16
+typedef struct {
+    const void *x;
+    fp8_dtype_t x_dt;
+    int64_t rows, cols, ld;
+    fp8_format_t fmt;
+    int32_t margin;
+    float *d_amax;
+    int32_t *d_bias;
+    uint8_t *y;
+} fp8_group_item_t;
+FP8_API fp8_status_t fp8_cast_group(fp8_ctx *ctx, const fp8_group_item_t *items, int32_t count, fp8_conv_t conv,
+                                    int32_t predicted, void *stream);
 
 /* Synchronises `stream` and returns how many guesses of fp8_cast_predicted held / did not hold since the
  * context was created or the counters were last cleared. */

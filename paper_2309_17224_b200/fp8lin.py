@@ -31,7 +31,7 @@ SYMBOLS = (
     "fp8_create", "fp8_destroy", "fp8_status_string", "fp8_device_flags", "fp8_amax", "fp8_scaling_bias",
     "fp8_scaling_bias_host", "fp8_cast_e4", "fp8_cast_e5", "fp8_ptq_weights", "fp8_linear_fwd", "fp8_linear_dgrad",
     "fp8_linear_wgrad", "fp8_amax_noalloc", "fp8_linear_fwd_act", "fp8_cast_predicted", "fp8_prediction_stats",
-    "fp8_linear_dgrad_act", "fp8_selftest_wait_expiry", "fp8_range_stats", "fp8_linear_fwd_q", "fp8_linear_dgrad_q", "fp8_amax_history_bias", "fp8_launch_count",
+    "fp8_linear_dgrad_act", "fp8_selftest_wait_expiry", "fp8_range_stats", "fp8_linear_fwd_q", "fp8_linear_dgrad_q", "fp8_amax_history_bias", "fp8_launch_count", "fp8_cast_group",
 )
 
 if not os.path.exists(LIB_PATH):
@@ -69,6 +69,15 @@ _lib.fp8_linear_fwd_q.argtypes = [_P, _P, _P, _P, _P, _P, c_int, c_int, _P, _P, 
 _lib.fp8_linear_dgrad_q.argtypes = [_P, _P, _P, _P, _P, _P, c_int, _P, _P, _P, _P, _P, _P, c_int64, c_int64, c_int64,
                                     c_int, _P]
 _lib.fp8_linear_wgrad.argtypes = [_P, _P, _P, _P, _P, _P, _P, _P, c_int, c_int64, c_int64, c_int64, c_int, _P]
+
+
+class GroupItem(ctypes.Structure):
+    """``fp8_group_item_t``."""
+    _fields_ = [("x", c_void_p), ("x_dt", c_int), ("rows", c_int64), ("cols", c_int64), ("ld", c_int64),
+                ("fmt", c_int), ("margin", c_int32), ("d_amax", c_void_p), ("d_bias", c_void_p), ("y", c_void_p)]
+
+
+_lib.fp8_cast_group.argtypes = [_P, POINTER(GroupItem), c_int32, c_int, c_int32, _P]
 for _name in SYMBOLS:
     if _name != "fp8_status_string":
         getattr(_lib, _name).restype = c_int
@@ -127,6 +136,18 @@ def amax_noalloc(x, d_amax, rows=None, cols=None, ld=None):
     cols = x.shape[1] if cols is None else cols
     ld = _ld(x) if ld is None else ld
     _check(_lib.fp8_amax_noalloc(_ptr(x), _DT[x.dtype], rows, cols, ld, _ptr(d_amax), _stream()), "fp8_amax_noalloc")
+
+
+def group_items(tensors):
+    """A ctypes array of ``fp8_group_item_t`` from (fmt, x, d_amax, d_bias, y[, margin]) tuples; build it once
+    and hand it to ``Context.cast_group`` every step (the tensors must stay alive)."""
+    arr = (GroupItem * len(tensors))()
+    for it, t in zip(arr, tensors):
+        fmt, x, d_amax, d_bias, y = t[:5]
+        it.x, it.x_dt, it.rows, it.cols, it.ld = x.data_ptr(), _DT[x.dtype], x.shape[0], x.shape[1], _ld(x)
+        it.fmt, it.margin = fmt, (t[5] if len(t) > 5 else 0)
+        it.d_amax, it.d_bias, it.y = d_amax.data_ptr(), d_bias.data_ptr(), y.data_ptr()
+    return arr
 
 
 class Context:
@@ -200,6 +221,12 @@ class Context:
         ld = _ld(x) if ld is None else ld
         _check(_lib.fp8_cast_predicted(self._h, fmt, _ptr(x), _DT[x.dtype], rows, cols, ld, conv, margin,
                                        _ptr(d_amax_out), _ptr(d_bias_inout), _ptr(y), _stream()), "fp8_cast_predicted")
+
+    def cast_group(self, items, conv=CONV_PAPER, predicted=False):
+        """``fp8_cast_group``.  `items`: a ``group_items(...)`` array, or a list of (fmt, x, d_amax, d_bias, y[, margin])
+        tuples that is marshalled on the spot."""
+        arr = items if isinstance(items, ctypes.Array) else group_items(items)
+        _check(_lib.fp8_cast_group(self._h, arr, len(arr), conv, 1 if predicted else 0, _stream()), "fp8_cast_group")
 
     def prediction_stats(self, clear: bool = True):
         hits, misses = c_uint(0), c_uint(0)

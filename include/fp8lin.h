@@ -117,6 +117,16 @@ FP8_API fp8_status_t fp8_device_flags(fp8_ctx *ctx, void *stream, unsigned *flag
  * is cleared, and the context stays usable.  Synchronises `stream`. */
 FP8_API fp8_status_t fp8_selftest_wait_expiry(fp8_ctx *ctx, uint64_t limit_ns, void *stream);
 
+/* Measurement aid (no counterpart in the paper): the tensor-pipe ceiling of the CTA-pair matmul kernel on this
+ * device.  Runs that kernel for an M x N x K problem (M > 128) with its operand loads switched off: the shared-memory
+ * stages are filled once with a fixed pattern of finite E4M3 bytes and every tcgen05.mma reads them as they stand;
+ * barriers, instruction stream, accumulators, epilogue and output stores are those of fp8_linear_fwd.  Timed by the
+ * caller with CUDA events, 2 M N K / time is what the kernel would reach if moving operands cost nothing -- the
+ * denominator that isolates the operand feed.  `out` [M, N] bf16 (16-byte aligned, N % 8 == 0) receives
+ * meaningless values; `d_zero` is a device int32 holding 0 (it stands in for the two biases). */
+FP8_API fp8_status_t fp8_selftest_mma_ceiling(fp8_ctx *ctx, void *out, const int32_t *d_zero, int64_t M, int64_t N,
+                                              int64_t K, void *stream);
+
 /* amax = max(|x|) over the whole tensor (Eq. 3, first line).
  *   x       [rows, cols] with leading dimension ld (elements), dtype x_dt
  *           (FP8_BF16, FP8_F16 or FP8_F32)
@@ -172,6 +182,31 @@ FP8_API fp8_status_t fp8_scaling_bias(fp8_ctx *ctx, const float *d_amax, fp8_for
 FP8_API fp8_status_t fp8_amax_history_bias(fp8_ctx *ctx, float *d_history, int32_t len, int32_t *d_cursor,
                                            const float *d_amax_new, fp8_format_t fmt, fp8_conv_t conv, int32_t margin,
                                            int32_t *d_bias, void *stream);
+
+/* Bias log and bias mode (Appendix G plots, per tensor, the mode of the scaling bias over the data samples;
+ * Appendix I its evolution per layer and step).  The log is a ring of records in device memory that the CALLER
+ * owns and drains (a plain device-to-host copy of `capacity` records plus the head counter); nothing here
+ * synchronises.
+ *   fp8_bias_log_append  appends `count` records {step, first_tensor_id + i, d_amax[i], d_bias[i]}, i < count,
+ *                        at the head of the ring (record n lives in slot n mod capacity; *d_head, a device
+ *                        uint64 that starts at 0, counts every record ever appended).  d_amax / d_bias are
+ *                        device arrays, e.g. the amax and bias words of all tensors of a step.  count <= capacity.
+ *   fp8_bias_mode        over the records currently in the ring that carry `tensor_id` and a step in
+ *                        [step_lo, step_hi]: *d_mode = their most frequent bias (the smaller value on a tie; 0
+ *                        when there is none), *d_count = how often it occurs, *d_samples (may be NULL) = how
+ *                        many records matched. */
+typedef struct {
+    int32_t step;
+    int32_t tensor_id;
+    float amax;
+    int32_t bias;
+} fp8_bias_record_t;
+FP8_API fp8_status_t fp8_bias_log_append(fp8_ctx *ctx, fp8_bias_record_t *d_ring, int32_t capacity, uint64_t *d_head,
+                                         int32_t step, int32_t first_tensor_id, const float *d_amax, const int32_t *d_bias,
+                                         int32_t count, void *stream);
+FP8_API fp8_status_t fp8_bias_mode(fp8_ctx *ctx, const fp8_bias_record_t *d_ring, int32_t capacity, const uint64_t *d_head,
+                                   int32_t tensor_id, int32_t step_lo, int32_t step_hi, int32_t *d_mode, int32_t *d_count,
+                                   int32_t *d_samples, void *stream);
 
 /* The same integer rule on the host (no device work, no ctx). */
 FP8_API fp8_status_t fp8_scaling_bias_host(float amax, fp8_format_t fmt, fp8_conv_t conv, int32_t margin, int32_t *bias);
@@ -232,16 +267,21 @@ FP8_API fp8_status_t fp8_cast_predicted(fp8_ctx *ctx, fp8_format_t fmt, const vo
  *                x, x_dt, rows, cols, ld   the input tensor
  *                fmt, margin               target format and the margin subtracted from its Eq. 3 bias
  *                d_amax                    out, device float
- *                d_bias                    out, device int32; with predicted != 0 also IN: the guess
+ *                d_bias                    out, device int32; IN as well in the modes that start from a given bias
  *                y                         out [rows, cols] bytes, row-major
- *   predicted  0: just in time -- one pass takes every amax and bias, a second casts (5 bytes moved per 16-bit
- *              element).  Non-zero: one pass casts every tensor with the guess found in its d_bias (typically the
+ *   mode       FP8_GROUP_AMAX_CAST: just in time -- one pass takes every amax and bias, a second casts (5 bytes
+ *              moved per 16-bit element).
+ *              FP8_GROUP_PREDICTED: one pass casts every tensor with the guess found in its d_bias (typically the
  *              value the previous step left there) while taking its amax; tensors whose guess turns out wrong
  *              are cast again by the second launch, the others are not touched again (3 bytes per element when
- *              all guesses hold; fp8_prediction_stats counts hits and misses).  Results are identical in both
- *              modes, whatever the guesses.
- * Tensors with ld == cols and 16-byte aligned x and y are grouped (up to FP8_GROUP_MAX per pair of launches, more
- * are taken in several rounds); any other tensor in the list is handed to fp8_cast_e4 / _e5 / _predicted. */
+ *              all guesses hold; fp8_prediction_stats counts hits and misses).  Same results as
+ *              FP8_GROUP_AMAX_CAST, whatever the guesses.
+ *              FP8_GROUP_AMAX_ONLY: the first pass alone: d_amax and d_bias of every tensor (y may be NULL).
+ *              FP8_GROUP_CAST_ONLY: the second pass alone, with the biases found in d_bias (chosen by the caller:
+ *              FP8-CSCALE, or biases from an amax history); d_amax is not touched and may be NULL.
+ * Tensors with ld == cols and 16-byte aligned x and y are grouped (up to FP8_GROUP_MAX of one input type per pair
+ * of launches; more, or mixed types, are taken in several rounds); any other tensor in the list is handed to
+ * fp8_amax / fp8_cast_e4 / _e5 / _predicted. */
 #define FP8_GROUP_MAX 16
 typedef struct {
     const void *x;
@@ -253,8 +293,9 @@ typedef struct {
     int32_t *d_bias;
     uint8_t *y;
 } fp8_group_item_t;
+typedef enum { FP8_GROUP_AMAX_CAST = 0, FP8_GROUP_PREDICTED = 1, FP8_GROUP_AMAX_ONLY = 2, FP8_GROUP_CAST_ONLY = 3 } fp8_group_mode_t;
 FP8_API fp8_status_t fp8_cast_group(fp8_ctx *ctx, const fp8_group_item_t *items, int32_t count, fp8_conv_t conv,
-                                    int32_t predicted, void *stream);
+                                    fp8_group_mode_t mode, void *stream);
 
 /* Synchronises `stream` and returns how many guesses of fp8_cast_predicted held / did not hold since the
  * context was created or the counters were last cleared. */

@@ -175,6 +175,18 @@ def history_bias(amax_window, kind: int, conv: int = CONV_PAPER, margin: int = 0
     return scaling_bias(max(float(a) for a in amax_window), kind, conv, margin)
 
 
+def bias_mode(biases):
+    """The statistic Appendix G plots per tensor: the mode of its scaling bias over the samples.  Returns
+    (mode, how often it occurs); the smaller bias on a tie, (0, 0) for no samples."""
+    counts = {}
+    for b in biases:
+        counts[int(b)] = counts.get(int(b), 0) + 1
+    if not counts:
+        return 0, 0
+    top = max(counts.values())
+    return min(b for b, c in counts.items() if c == top), top
+
+
 def cast(x_bits: np.ndarray, shift: int, fmt: int, transposed: bool = False):
     """codes = encode_fmt(x * 2^shift); returns y[rows, cols] and, if asked,
     also y_t[cols, rows]."""

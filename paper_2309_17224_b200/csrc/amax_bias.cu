@@ -175,6 +175,60 @@ __global__ void amax_history_kernel(float *__restrict__ d_history, int len, int3
     }
 }
 
+// Append `count` records {step, first_id + i, amax[i], bias[i]} to a ring of `capacity` records; *d_head counts
+// every record ever appended (the slot of record n is n mod capacity).
+__global__ void bias_log_kernel(fp8_bias_record_t *__restrict__ ring, int capacity, unsigned long long *d_head, int step,
+                                int first_id, const float *__restrict__ d_amax, const int32_t *__restrict__ d_bias,
+                                int count)
+{
+    const unsigned long long head = *d_head;
+    for (int i = threadIdx.x; i < count; i += blockDim.x) {
+        fp8_bias_record_t r;
+        r.step = step;
+        r.tensor_id = first_id + i;
+        r.amax = d_amax[i];
+        r.bias = d_bias[i];
+        ring[(head + (unsigned long long)i) % (unsigned long long)capacity] = r;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) *d_head = head + (unsigned long long)count;
+}
+
+// Mode of one tensor's bias over the records of the ring whose step lies in [step_lo, step_hi]: a histogram over
+// every value Eq. 3 can produce for a 32-bit float amax (|bias| <= 165 with margins up to 16; others are counted
+// but cannot win), the most frequent value wins, the smaller one on a tie.
+constexpr int kModeLo = -192, kModeBins = 385;
+__global__ void bias_mode_kernel(const fp8_bias_record_t *__restrict__ ring, int capacity,
+                                 const unsigned long long *__restrict__ d_head, int tensor_id, int step_lo, int step_hi,
+                                 int32_t *__restrict__ d_mode, int32_t *__restrict__ d_count, int32_t *__restrict__ d_samples)
+{
+    __shared__ unsigned hist[kModeBins];
+    __shared__ unsigned samples;
+    for (int i = threadIdx.x; i < kModeBins; i += blockDim.x) hist[i] = 0u;
+    if (threadIdx.x == 0) samples = 0u;
+    __syncthreads();
+    const unsigned long long head = *d_head;
+    const int valid = head < (unsigned long long)capacity ? (int)head : capacity;
+    for (int i = threadIdx.x; i < valid; i += blockDim.x) {
+        const fp8_bias_record_t r = ring[i];
+        if (r.tensor_id == tensor_id && r.step >= step_lo && r.step <= step_hi) {
+            atomicAdd(&samples, 1u);
+            const int b = r.bias - kModeLo;
+            if (b >= 0 && b < kModeBins) atomicAdd(&hist[b], 1u);
+        }
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        unsigned best = 0u;
+        int mode = 0;
+        for (int i = 0; i < kModeBins; ++i)
+            if (hist[i] > best) { best = hist[i]; mode = i + kModeLo; }
+        *d_mode = mode;
+        *d_count = (int32_t)best;
+        if (d_samples) *d_samples = (int32_t)samples;
+    }
+}
+
 template <int DT>
 static cudaError_t launch_amax_dt(fp8_ctx *ctx, const void *x, int64_t rows, int64_t cols, int64_t ld, AmaxOut o,
                                   cudaStream_t stream)
@@ -247,6 +301,33 @@ fp8_status_t fp8_amax_history_bias(fp8_ctx *ctx, float *d_history, int32_t len, 
     fp8lin::count_launch();
     fp8lin::amax_history_kernel<<<1, 32, 0, (cudaStream_t)stream>>>(d_history, len, d_cursor, d_amax_new, (int)fmt,
                                                                    (int)conv, margin, d_bias, ctx->d_status);
+    return cudaGetLastError() == cudaSuccess ? FP8_OK : FP8_ERR_CUDA;
+}
+
+fp8_status_t fp8_bias_log_append(fp8_ctx *ctx, fp8_bias_record_t *d_ring, int32_t capacity, uint64_t *d_head, int32_t step,
+                                 int32_t first_tensor_id, const float *d_amax, const int32_t *d_bias, int32_t count,
+                                 void *stream)
+{
+    if (!ctx || !d_ring || !d_head || !d_amax || !d_bias) return FP8_ERR_NULL;
+    if (capacity <= 0 || count <= 0 || count > capacity) return FP8_ERR_SHAPE;
+    if ((reinterpret_cast<uintptr_t>(d_ring) & 3u) || (reinterpret_cast<uintptr_t>(d_head) & 7u)) return FP8_ERR_ALIGN;
+    fp8lin::count_launch();
+    fp8lin::bias_log_kernel<<<1, 128, 0, (cudaStream_t)stream>>>(d_ring, capacity,
+                                                                reinterpret_cast<unsigned long long *>(d_head), step,
+                                                                first_tensor_id, d_amax, d_bias, count);
+    return cudaGetLastError() == cudaSuccess ? FP8_OK : FP8_ERR_CUDA;
+}
+
+fp8_status_t fp8_bias_mode(fp8_ctx *ctx, const fp8_bias_record_t *d_ring, int32_t capacity, const uint64_t *d_head,
+                           int32_t tensor_id, int32_t step_lo, int32_t step_hi, int32_t *d_mode, int32_t *d_count,
+                           int32_t *d_samples, void *stream)
+{
+    if (!ctx || !d_ring || !d_head || !d_mode || !d_count) return FP8_ERR_NULL;
+    if (capacity <= 0 || step_lo > step_hi) return FP8_ERR_SHAPE;
+    fp8lin::count_launch();
+    fp8lin::bias_mode_kernel<<<1, 256, 0, (cudaStream_t)stream>>>(d_ring, capacity,
+                                                                 reinterpret_cast<const unsigned long long *>(d_head),
+                                                                 tensor_id, step_lo, step_hi, d_mode, d_count, d_samples);
     return cudaGetLastError() == cudaSuccess ? FP8_OK : FP8_ERR_CUDA;
 }
 

@@ -94,6 +94,7 @@ struct GemmParams {
     unsigned *d_amax_bits;        // or NULL
     unsigned *d_status;
     uint32_t idesc;
+    int no_loads;                 // measurement aid (fp8_selftest_mma_ceiling): the CTA-pair kernel issues no operand loads
 };
 
 // ---------------------------------------------------------------------------
@@ -1088,12 +1089,16 @@ constexpr int kPairHalfN = 128;    // B rows each CTA loads
 
 constexpr int kPairStagesAct = 5;  // the kernels with a second output trade one stage for two more slabs per warp
 
-template <int STAGES, int SLABS>
+// NHALF = 1: the 256 x 256 pair tile, two accumulators in tensor memory (the epilogue of one tile overlaps the main
+// loop of the next).  NHALF = 2: a 256 x 512 pair tile held as ONE accumulator of two 256-column halves: each CTA
+// loads its 128 rows of A once per k-block and 2 x 128 rows of B, 48 KB for twice the multiply-adds of the 32 KB
+// of the narrow tile -- three quarters of the bytes that cross from L2 into shared memory per FLOP.
+template <int STAGES, int SLABS, int NHALF = 1>
 struct PairSmemT {
     static constexpr int kStages = STAGES;
     static constexpr int kSlabs = SLABS;
     static constexpr int kABytes = kBM * kBK;
-    static constexpr int kBBytes = kPairHalfN * kBK;
+    static constexpr int kBBytes = NHALF * kPairHalfN * kBK;
     static constexpr int kStageBytes = kABytes + kBBytes;
     static constexpr int kEpiOffset = STAGES * kStageBytes;
     static constexpr int kBarOffset = kEpiOffset + 4 * SLABS * kSlabBytes;
@@ -1104,6 +1109,8 @@ struct PairSmemT {
 };
 using PairSmem = PairSmemT<kPairStages, kPairSlabs>;
 using PairSmemAct = PairSmemT<kPairStagesAct, kActSlabs>;
+constexpr int kWideStages = 4;
+using PairSmemWide = PairSmemT<kWideStages, kPairSlabs, 2>;
 
 __device__ __forceinline__ uint32_t cluster_ctarank()
 {
@@ -1169,15 +1176,17 @@ __host__ __device__ inline uint32_t make_idesc_pair(int a_fmt, int b_fmt)
            ((uint32_t)(256 >> 4) << 24);
 }
 
-// tiles here are 256 x 256; p.tiles_m / p.tiles_n count those
-template <int ACT>
+// tiles here are 256 x (256 * NHALF); p.tiles_m / p.tiles_n count those
+template <int ACT, int NHALF = 1>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1)
 gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                  const __grid_constant__ CUtensorMap map_out, const __grid_constant__ CUtensorMap map_out2,
                  const GemmParams p)
 {
-    using L = PairSmemT<ACT ? kPairStagesAct : kPairStages, ACT ? kActSlabs : kPairSlabs>;
+    static_assert(NHALF == 1 || ACT == 0, "the wide tile carries the plain epilogue only");
+    using L = PairSmemT<NHALF == 2 ? kWideStages : (ACT ? kPairStagesAct : kPairStages), ACT ? kActSlabs : kPairSlabs, NHALF>;
     constexpr int kStagesL = L::kStages;
+    constexpr int kTileN = kPairBN * NHALF;
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const uint32_t smem_base = smem_u32(smem);
@@ -1207,6 +1216,13 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
     }
+    if (p.no_loads) {
+        // the stages keep one fixed pattern for the whole run: finite E4M3 bytes of magnitude below 2
+        uint32_t *w = reinterpret_cast<uint32_t *>(smem);
+        for (int i = threadIdx.x; i < kStagesL * L::kStageBytes / 4; i += kGemmThreads)
+            w[i] = ((uint32_t)i * 2654435761u + 0x9E3779B9u * (rank + 1u)) & 0xBFBFBFBFu;
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
     tc_fence_before();
     __syncthreads();
     cluster_sync_all();  // both CTAs' barriers exist before anyone signals across
@@ -1231,15 +1247,24 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                     const uint32_t leader_full = leader_full0 + 8u * s;
                     const uint32_t ph = (it / kStagesL) & 1u;
                     if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p.d_status)) { alive = false; break; }
+                    if (p.no_loads) {   // the stage is "full" as it stands
+                        if (rank == 0) mbar_arrive(full_bar(s));
+                        continue;
+                    }
                     // only the leader arrives, announcing the bytes of all four loads of the pair; the
                     // peer's bytes may land first (the pending arrival keeps the phase open)
                     if (rank == 0) mbar_expect_tx(full_bar(s), 2 * L::kStageBytes);
                     const uint32_t a_dst = smem_base + s * L::kStageBytes;
-                    const int a_row = m_blk * 256 + (int)rank * kBM, b_row = n_blk * kPairBN + (int)rank * kPairHalfN;
+                    const int a_row = m_blk * 256 + (int)rank * kBM;
                     if (p.a_mn) tma_load_2d_pair(a_dst, &map_a, leader_full, a_row, k * kBK);
                     else tma_load_2d_pair(a_dst, &map_a, leader_full, k * kBK, a_row);
-                    if (p.b_mn) tma_load_2d_pair(a_dst + L::kABytes, &map_b, leader_full, b_row, k * kBK);
-                    else tma_load_2d_pair(a_dst + L::kABytes, &map_b, leader_full, k * kBK, b_row);
+#pragma unroll
+                    for (int h = 0; h < NHALF; ++h) {   // this CTA's 128 of the 256 B rows of each half of the tile
+                        const int b_row = n_blk * kTileN + h * kPairBN + (int)rank * kPairHalfN;
+                        const uint32_t b_dst = a_dst + L::kABytes + h * (kPairHalfN * kBK);
+                        if (p.b_mn) tma_load_2d_pair(b_dst, &map_b, leader_full, b_row, k * kBK);
+                        else tma_load_2d_pair(b_dst, &map_b, leader_full, k * kBK, b_row);
+                    }
                 }
             }
         }
@@ -1250,24 +1275,52 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             // the bounded waits below start counting only once the launch before this one has completed
             asm volatile("griddepcontrol.wait;" ::: "memory");
             for (int tile = pair_id; alive && tile < num_tiles; tile += num_pairs, ++t) {
-                const int buf = t & 1;
-                const uint32_t acc_ph = (t >> 1) & 1u;
+                // narrow tile: two accumulators used in turn; wide tile: one accumulator whose two halves are
+                // released (and waited for) separately, barrier b standing for half b
+                const int buf = NHALF == 2 ? 0 : (t & 1);
+                const uint32_t acc_ph = NHALF == 2 ? (t & 1u) : ((t >> 1) & 1u);
                 if (!mbar_wait(acc_empty_bar(buf), acc_ph ^ 1u, abort_flag, p.d_status)) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + buf * kPairBN;
-                for (int k = 0; k < p.num_k; ++k, ++it) {
+                auto issue = [&](int s, int k, int h) {
+                    const uint32_t a_addr = smem_base + s * L::kStageBytes;
+                    const uint32_t b_addr = a_addr + L::kABytes + h * (kPairHalfN * kBK);
+                    const uint64_t da = p.a_mn ? smem_desc_mn128(a_addr, 128 * kBK) : smem_desc_k128(a_addr);
+                    const uint64_t db = p.b_mn ? smem_desc_mn128(b_addr, 128 * kBK) : smem_desc_k128(b_addr);
+                    // per instruction (K = 32): 32 bytes along a 128-byte row, or 32 rows = 4096 bytes
+                    const uint32_t step_a = p.a_mn ? 256u : 2u, step_b = p.b_mn ? 256u : 2u;
+#pragma unroll
+                    for (int j = 0; j < kBK / kUmmaK; ++j)
+                        umma_f8_pair(d_tmem + h * kPairBN, da + step_a * j, db + step_b * j, p.idesc, (k > 0 || j > 0) ? 1u : 0u);
+                };
+                int k = 0;
+                if (NHALF == 2) {
+                    // The epilogue of the previous tile drains half 0, then half 1.  The first k-blocks of this tile
+                    // run on half 0 alone while half 1 is still being read; their stages stay held until half 1 has
+                    // used them too.
+                    const int ahead = min(p.num_k, kStagesL - 1);
+                    for (int a = 0; alive && a < ahead; ++a) {
+                        const uint32_t ia = it + a;
+                        if (!mbar_wait(full_bar(ia % kStagesL), (ia / kStagesL) & 1u, abort_flag, p.d_status)) { alive = false; break; }
+                        tc_fence_after();
+                        issue(ia % kStagesL, a, 0);
+                    }
+                    if (alive && !mbar_wait(acc_empty_bar(1), acc_ph ^ 1u, abort_flag, p.d_status)) alive = false;
+                    if (!alive) break;
+                    tc_fence_after();
+                    for (int a = 0; a < ahead; ++a, ++it) {
+                        issue(it % kStagesL, a, 1);
+                        umma_commit_pair(empty_bar(it % kStagesL));
+                    }
+                    k = ahead;
+                }
+                for (; k < p.num_k; ++k, ++it) {
                     const int s = it % kStagesL;
                     const uint32_t ph = (it / kStagesL) & 1u;
                     if (!mbar_wait(full_bar(s), ph, abort_flag, p.d_status)) { alive = false; break; }
                     tc_fence_after();
-                    const uint32_t a_addr = smem_base + s * L::kStageBytes;
-                    const uint64_t da = p.a_mn ? smem_desc_mn128(a_addr, 128 * kBK) : smem_desc_k128(a_addr);
-                    const uint64_t db = p.b_mn ? smem_desc_mn128(a_addr + L::kABytes, 128 * kBK)
-                                               : smem_desc_k128(a_addr + L::kABytes);
-                    const uint32_t step_a = p.a_mn ? 256u : 2u, step_b = p.b_mn ? 256u : 2u;
 #pragma unroll
-                    for (int j = 0; j < kBK / kUmmaK; ++j)
-                        umma_f8_pair(d_tmem, da + step_a * j, db + step_b * j, p.idesc, (k > 0 || j > 0) ? 1u : 0u);
+                    for (int h = 0; h < NHALF; ++h) issue(s, k, h);
                     umma_commit_pair(empty_bar(s));
                 }
                 if (alive) umma_commit_pair(acc_full_bar(buf));
@@ -1286,14 +1339,18 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
         for (int tile = pair_id; tile < num_tiles; tile += num_pairs, ++t) {
             int m_blk, n_blk;
             tile_coords(tile, p, m_blk, n_blk);
-            const int buf = t & 1;
-            const uint32_t acc_ph = (t >> 1) & 1u;
+            const int buf = NHALF == 2 ? 0 : (t & 1);
+            const uint32_t acc_ph = NHALF == 2 ? (t & 1u) : ((t >> 1) & 1u);
             const bool ready = mbar_wait(acc_full_bar(buf), acc_ph, abort_flag, p.d_status);
             if (!__all_sync(0xFFFFFFFFu, ready)) break;
             tc_fence_after();
             const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + buf * kPairBN;
-            epilogue_tile<kPairBN, ACT, L::kSlabs>(&map_out, &map_out2, t_row, m_blk * 256 + (int)rank * kBM + q * 32, n_blk * kPairBN, p, sc,
-                                   two_step, amax_bits, warp_slabs, slab_count, leader_acc_empty0 + 8u * buf, true, lane);
+#pragma unroll 1
+            for (int h = 0; h < NHALF; ++h)   // the wide tile: half 0 is handed back to the MMA thread before half 1 is read
+                epilogue_tile<kPairBN, ACT, L::kSlabs>(&map_out, &map_out2, t_row + h * kPairBN,
+                                                       m_blk * 256 + (int)rank * kBM + q * 32, n_blk * kTileN + h * kPairBN, p,
+                                                       sc, two_step, amax_bits, warp_slabs, slab_count,
+                                                       leader_acc_empty0 + 8u * (NHALF == 2 ? h : buf), true, lane);
         }
         if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
         if (p.d_amax_bits) {
@@ -1411,7 +1468,13 @@ static bool g_no_splitk = false;        // set from FP8LIN_NO_SPLITK=1
 static int g_force_splits = 0;          // set from FP8LIN_SPLITS (experiments with the split count)
 static bool g_no_pdl = false;           // set from FP8LIN_NO_PDL=1 (A/B: matmuls launched without programmatic dependence)
 static bool g_direct_epilogue = false;  // set from FP8LIN_DIRECT_EPILOGUE=1 (A/B comparison of the epilogues)
+static int g_force_wide = -1;           // set from FP8LIN_WIDE=0/1 (A/B: never / always the 256 x 512 pair tile)
 static int g_max_pairs = 0;  // CTA pairs that can be resident at once (0: pair kernel unavailable)
+
+#ifndef FP8LIN_WIDE_DEFAULT
+#define FP8LIN_WIDE_DEFAULT 1
+#endif
+constexpr bool kWideTileDefault = FP8LIN_WIDE_DEFAULT != 0;
 
 constexpr int kStagesAct = 3;  // single-CTA kernels with a second output: fewer stages, two more slabs per warp
 
@@ -1424,6 +1487,9 @@ static cudaError_t set_smem_attributes()
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, LS::kDynamic);
     if (e == cudaSuccess)
         e = cudaFuncSetAttribute(gemm_pair_kernel<ACT>, cudaFuncAttributeMaxDynamicSharedMemorySize, LP::kDynamic);
+    if (e == cudaSuccess && ACT == 0)
+        e = cudaFuncSetAttribute(gemm_pair_kernel<0, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 PairSmemWide::kDynamic);
     return e;
 }
 
@@ -1432,7 +1498,7 @@ cudaError_t configure_gemm_kernels(int max_smem_optin)
     using L = GemmSmem<kBN, kStages>;
     using LA = GemmSmem<kBN, kStagesAct, kActSlabs>;
     if (L::kDynamic > max_smem_optin || PairSmem::kDynamic > max_smem_optin || LA::kDynamic > max_smem_optin ||
-        PairSmemAct::kDynamic > max_smem_optin)
+        PairSmemAct::kDynamic > max_smem_optin || PairSmemWide::kDynamic > max_smem_optin)
         return cudaErrorInvalidValue;
     cudaError_t e = set_smem_attributes<0>();
     if (e == cudaSuccess) e = set_smem_attributes<1>();
@@ -1475,6 +1541,8 @@ cudaError_t configure_gemm_kernels(int max_smem_optin)
     g_no_splitk = env && env[0] == '1';
     env = getenv("FP8LIN_DIRECT_EPILOGUE");
     g_direct_epilogue = env && env[0] == '1';
+    env = getenv("FP8LIN_WIDE");
+    g_force_wide = env ? atoi(env) : -1;
     if (getenv("FP8LIN_DEBUG")) fprintf(stderr, "fp8lin: %d SMs, %d resident CTA pairs, pair kernel %s\n", sms, clusters,
                                         g_force_single ? "off" : "on");
 #endif
@@ -1495,6 +1563,21 @@ static bool encode_map(fp8_ctx *ctx, CUtensorMap *map, const void *base, int64_t
     return r == CUDA_SUCCESS;
 }
 
+// Which pair tile a plain matmul takes.  The 256 x 512 tile moves three quarters of the operand bytes per FLOP but
+// cannot overlap a tile's epilogue with the next tile's main loop beyond its first k-blocks, and its tiles are
+// twice as coarse: it must not add a wave, nor waste much of its width beyond N.
+static bool use_wide_tile(int64_t M, int64_t N, int64_t Kc)
+{
+    if (g_force_wide >= 0) return g_force_wide != 0;
+    if (g_max_pairs <= 0) return false;
+    const int64_t tm = (M + 255) / 256;
+    const int64_t narrow = tm * ((N + 255) / 256), wide_t = tm * ((N + 511) / 512);
+    const int64_t waves_n = (narrow + g_max_pairs - 1) / g_max_pairs, waves_w = (wide_t + g_max_pairs - 1) / g_max_pairs;
+    const bool no_extra_wave = 2 * waves_w <= waves_n + (waves_n >= 8 ? 1 : 0);
+    const bool little_waste = ((N + 511) / 512) * 512 - N <= N / 32;
+    return kWideTileDefault && Kc >= 2048 && no_extra_wave && little_waste;
+}
+
 // D[M,N] = A * B^T over a contraction of length Kc, unscaled by 2^-(bias_a + bias_b + delta_sum).
 // A is stored [M, Kc] (a_mn = false) or [Kc, M] (a_mn = true); B is stored [N, Kc] or [Kc, N] likewise.
 static fp8_status_t run_gemm(fp8_ctx *ctx, const uint8_t *a, int a_fmt, bool a_mn, const int32_t *d_ba,
@@ -1502,7 +1585,7 @@ static fp8_status_t run_gemm(fp8_ctx *ctx, const uint8_t *a, int a_fmt, bool a_m
                              const void *bias_vec, int bias_dt, void *out, int out_dt, float *d_amax_out, int64_t M,
                              int64_t N, int64_t Kc, cudaStream_t st, int act = 0, void *out_act = nullptr,
                              const void *aux = nullptr, uint8_t *out8 = nullptr, const int32_t *d_sq = nullptr,
-                             int q_fmt = 0, int delta_q = 0)
+                             int q_fmt = 0, int delta_q = 0, bool no_loads = false)
 {
     if (M > 0x7FFFFFFF / 2 || N > 0x7FFFFFFF / 2 || Kc > 0x7FFFFFFF / 2) return FP8_ERR_SHAPE;
     const bool pair = g_max_pairs > 0 && M > kBM && !g_force_single;
@@ -1522,8 +1605,9 @@ static fp8_status_t run_gemm(fp8_ctx *ctx, const uint8_t *a, int a_fmt, bool a_m
     p.b_mn = b_mn ? 1 : 0;
     p.a_box_bytes = a_box_rows * kBK;
     p.M = (int)M; p.N = (int)N; p.K = (int)Kc;
+    const bool wide = pair && act == 0 && use_wide_tile(M, N, Kc);
     p.tiles_m = (int)((M + (pair ? 256 : kBM) - 1) / (pair ? 256 : kBM));
-    p.tiles_n = (int)((N + kBN - 1) / kBN);
+    p.tiles_n = (int)((N + (wide ? 2 * kBN : kBN) - 1) / (wide ? 2 * kBN : kBN));
     p.num_k = (int)((Kc + kBK - 1) / kBK);
     if ((int64_t)p.tiles_m * p.tiles_n > 0x7FFFFFFF) return FP8_ERR_SHAPE;
     // Few output tiles and a long contraction (the decode regime): split the contraction so that every SM
@@ -1581,6 +1665,8 @@ static fp8_status_t run_gemm(fp8_ctx *ctx, const uint8_t *a, int a_fmt, bool a_m
     p.d_sq = d_sq;
     p.q_fmt = q_fmt;
     p.delta_q = delta_q;
+    p.no_loads = no_loads ? 1 : 0;
+    if (no_loads && !pair) return FP8_ERR_UNSUPPORTED;
     CUtensorMap map_out = map_a;  // placeholder when the staged epilogue is off (never dereferenced then)
     CUtensorMap map_out2 = map_a;
     auto encode_out = [&](CUtensorMap *m, void *base, int64_t cols) {
@@ -1626,12 +1712,13 @@ static fp8_status_t run_gemm(fp8_ctx *ctx, const uint8_t *a, int a_fmt, bool a_m
             cudaLaunchConfig_t cfg = {};
             cfg.gridDim = grid;
             cfg.blockDim = dim3(kGemmThreads);
-            cfg.dynamicSmemBytes = PairSmem::kDynamic;
+            cfg.dynamicSmemBytes = wide ? PairSmemWide::kDynamic : PairSmem::kDynamic;
             cfg.stream = st;
             cfg.attrs = attr;
             cfg.numAttrs = 1;
-            if (cudaLaunchKernelEx(&cfg, gemm_pair_kernel<0>, map_a, map_b, map_out, map_out2, p) != cudaSuccess)
-                return FP8_ERR_CUDA;
+            cudaError_t le = wide ? cudaLaunchKernelEx(&cfg, gemm_pair_kernel<0, 2>, map_a, map_b, map_out, map_out2, p)
+                                  : cudaLaunchKernelEx(&cfg, gemm_pair_kernel<0>, map_a, map_b, map_out, map_out2, p);
+            if (le != cudaSuccess) return FP8_ERR_CUDA;
             break;
         }
         }
@@ -1707,6 +1794,19 @@ fp8_status_t fp8_linear_fwd(fp8_ctx *ctx, const uint8_t *x8, const int32_t *d_bx
     int delta = 2 * format_delta(FP8_E4, conv);
     return run_gemm(ctx, x8, FP8_E4, false, d_bx, w8, FP8_E4, false, d_bw, delta, bias_vec, bias_dt, y, y_dt, d_amax_y,
                     T, N, K, (cudaStream_t)stream);
+}
+
+fp8_status_t fp8_selftest_mma_ceiling(fp8_ctx *ctx, void *out, const int32_t *d_zero, int64_t M, int64_t N, int64_t K,
+                                      void *stream)
+{
+    using namespace fp8lin;
+    if (!ctx || !out || !d_zero) return FP8_ERR_NULL;
+    if (M <= kBM || N <= 0 || K <= 0) return FP8_ERR_SHAPE;
+    if (!aligned16(out) || (N % 8) != 0 || (K % 16) != 0) return FP8_ERR_ALIGN;
+    // the operand maps are encoded (over the output buffer's address) but never used: no load is issued
+    return run_gemm(ctx, static_cast<const uint8_t *>(out), FP8_E4, false, d_zero, static_cast<const uint8_t *>(out),
+                    FP8_E4, false, d_zero, 0, nullptr, 0, out, FP8_BF16, nullptr, M, N, K, (cudaStream_t)stream, 0, nullptr,
+                    nullptr, nullptr, nullptr, 0, 0, true);
 }
 
 fp8_status_t fp8_selftest_wait_expiry(fp8_ctx *ctx, uint64_t limit_ns, void *stream)

@@ -173,7 +173,7 @@ __device__ __forceinline__ GroupItem get_item(const GroupParams &gp, int i)
 // amax passes count from the front of the first tensor; the cast pass counts from the back of the last one, so that
 // what the amax pass read last (and may still be in L2) is read first.
 template <int MODE, int DT>
-__global__ void __launch_bounds__(kCastThreads, 6) group_kernel(const __grid_constant__ GroupParams gp, int gate)
+__global__ void __launch_bounds__(kCastThreads, 5) group_kernel(const __grid_constant__ GroupParams gp, int gate)
 {
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (MODE == kCast) asm volatile("griddepcontrol.wait;" ::: "memory");   // biases / redo flags of the launch before
@@ -209,7 +209,7 @@ __global__ void __launch_bounds__(kCastThreads, 6) group_kernel(const __grid_con
 static bool group_shape_ok(const fp8_group_item_t &t)
 {
     auto al16 = [](const void *q) { return (reinterpret_cast<uintptr_t>(q) & 15u) == 0; };
-    return t.ld == t.cols && al16(t.x) && al16(t.y);
+    return t.ld == t.cols && al16(t.x) && al16(t.y);   // a NULL y (amax only) passes
 }
 
 }  // namespace fp8lin
@@ -217,15 +217,17 @@ static bool group_shape_ok(const fp8_group_item_t &t)
 extern "C" {
 
 fp8_status_t fp8_cast_group(fp8_ctx *ctx, const fp8_group_item_t *items, int32_t count, fp8_conv_t conv,
-                            int32_t predicted, void *stream)
+                            fp8_group_mode_t mode, void *stream)
 {
     using namespace fp8lin;
     if (!ctx || !items) return FP8_ERR_NULL;
     if (count <= 0) return FP8_ERR_SHAPE;
-    if ((int)conv < 0 || (int)conv > 1) return FP8_ERR_DTYPE;
+    if ((int)conv < 0 || (int)conv > 1 || (int)mode < 0 || (int)mode > 3) return FP8_ERR_DTYPE;
+    const bool predicted = mode == FP8_GROUP_PREDICTED;
+    const bool want_amax = mode != FP8_GROUP_CAST_ONLY, want_cast = mode != FP8_GROUP_AMAX_ONLY;
     for (int i = 0; i < count; ++i) {
         const fp8_group_item_t &t = items[i];
-        if (!t.x || !t.y || !t.d_amax || !t.d_bias) return FP8_ERR_NULL;
+        if (!t.x || (want_cast && !t.y) || (want_amax && !t.d_amax) || !t.d_bias) return FP8_ERR_NULL;
         if ((int)t.fmt < 0 || (int)t.fmt > 1 || (int)t.x_dt < 0 || (int)t.x_dt > 2) return FP8_ERR_DTYPE;
         if (t.rows <= 0 || t.cols <= 0 || t.ld < t.cols) return FP8_ERR_SHAPE;
         if (reinterpret_cast<uintptr_t>(t.x) & (t.x_dt == FP8_F32 ? 3u : 1u)) return FP8_ERR_ALIGN;
@@ -236,12 +238,22 @@ fp8_status_t fp8_cast_group(fp8_ctx *ctx, const fp8_group_item_t *items, int32_t
         // tensors outside the grouped kernels' shape rules go through the single-tensor entry points
         if (!group_shape_ok(items[i])) {
             const fp8_group_item_t &t = items[i];
-            fp8_status_t s = predicted ? fp8_cast_predicted(ctx, t.fmt, t.x, t.x_dt, t.rows, t.cols, t.ld, conv, t.margin,
-                                                            t.d_amax, t.d_bias, t.y, stream)
-                             : t.fmt == FP8_E4 ? fp8_cast_e4(ctx, t.x, t.x_dt, t.rows, t.cols, t.ld, nullptr, conv, t.margin,
-                                                             t.d_amax, t.d_bias, t.y, nullptr, stream)
-                                               : fp8_cast_e5(ctx, t.x, t.x_dt, t.rows, t.cols, t.ld, nullptr, conv, t.margin,
-                                                             t.d_amax, t.d_bias, t.y, nullptr, stream);
+            fp8_status_t s;
+            if (predicted) {
+                s = fp8_cast_predicted(ctx, t.fmt, t.x, t.x_dt, t.rows, t.cols, t.ld, conv, t.margin, t.d_amax, t.d_bias, t.y,
+                                       stream);
+            } else if (mode == FP8_GROUP_AMAX_ONLY) {
+                s = launch_amax_bias(ctx, t.x, (int)t.x_dt, t.rows, t.cols, t.ld, t.d_amax, t.d_bias, (int)t.fmt, (int)conv,
+                                     t.margin, (cudaStream_t)stream) == cudaSuccess ? FP8_OK : FP8_ERR_CUDA;
+            } else {
+                const int32_t *given = mode == FP8_GROUP_CAST_ONLY ? t.d_bias : nullptr;
+                float *ao = given ? nullptr : t.d_amax;
+                int32_t *bo = given ? nullptr : t.d_bias;
+                s = t.fmt == FP8_E4 ? fp8_cast_e4(ctx, t.x, t.x_dt, t.rows, t.cols, t.ld, given, conv, t.margin, ao, bo, t.y,
+                                                  nullptr, stream)
+                                    : fp8_cast_e5(ctx, t.x, t.x_dt, t.rows, t.cols, t.ld, given, conv, t.margin, ao, bo, t.y,
+                                                  nullptr, stream);
+            }
             if (s != FP8_OK) return s;
             ++i;
             continue;
@@ -273,17 +285,20 @@ fp8_status_t fp8_cast_group(fp8_ctx *ctx, const fp8_group_item_t *items, int32_t
             g.d_bias = t.d_bias;
             ++i;
         }
-        const int64_t cap = (int64_t)ctx->sm_count * 6;   // the blocks that are resident at once (launch bounds)
+        const int64_t cap = (int64_t)ctx->sm_count * 5;   // the blocks that are resident at once (launch bounds)
         const unsigned blocks = (unsigned)(gp.total_chunks < cap ? gp.total_chunks : cap);
-        count_launch(2);
+        count_launch((want_amax ? 1 : 0) + (want_cast ? 1 : 0));
+        if (want_amax) {
 #define FP8LIN_FIRST(D) \
     if (predicted) group_kernel<kBoth, D><<<blocks, kCastThreads, 0, st>>>(gp, 0); \
     else group_kernel<kAmax, D><<<blocks, kCastThreads, 0, st>>>(gp, 0)
-        if (dt == FP8_BF16) { FP8LIN_FIRST(FP8_BF16); }
-        else if (dt == FP8_F16) { FP8LIN_FIRST(FP8_F16); }
-        else { FP8LIN_FIRST(FP8_F32); }
+            if (dt == FP8_BF16) { FP8LIN_FIRST(FP8_BF16); }
+            else if (dt == FP8_F16) { FP8LIN_FIRST(FP8_F16); }
+            else { FP8LIN_FIRST(FP8_F32); }
 #undef FP8LIN_FIRST
-        if (cudaGetLastError() != cudaSuccess) return FP8_ERR_CUDA;
+            if (cudaGetLastError() != cudaSuccess) return FP8_ERR_CUDA;
+        }
+        if (!want_cast) continue;
         cudaLaunchAttribute attr[1];
         attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
         attr[0].val.programmaticStreamSerializationAllowed = 1;

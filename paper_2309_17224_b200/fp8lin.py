@@ -22,6 +22,7 @@ ERR_NULL, ERR_SHAPE, ERR_ALIGN, ERR_DTYPE, ERR_UNSUPPORTED, ERR_CUDA, ERR_DEVICE
 E4, E5 = 0, 1
 CONV_PAPER, CONV_NATIVE = 0, 1
 BF16, F16, F32 = 0, 1, 2
+GROUP_AMAX_CAST, GROUP_PREDICTED, GROUP_AMAX_ONLY, GROUP_CAST_ONLY = 0, 1, 2, 3
 ACT_NONE = 0
 ACT_GELU = 1
 ACT_SWIGLU = 2
@@ -31,7 +32,7 @@ SYMBOLS = (
     "fp8_create", "fp8_destroy", "fp8_status_string", "fp8_device_flags", "fp8_amax", "fp8_scaling_bias",
     "fp8_scaling_bias_host", "fp8_cast_e4", "fp8_cast_e5", "fp8_ptq_weights", "fp8_linear_fwd", "fp8_linear_dgrad",
     "fp8_linear_wgrad", "fp8_amax_noalloc", "fp8_linear_fwd_act", "fp8_cast_predicted", "fp8_prediction_stats",
-    "fp8_linear_dgrad_act", "fp8_selftest_wait_expiry", "fp8_range_stats", "fp8_linear_fwd_q", "fp8_linear_dgrad_q", "fp8_amax_history_bias", "fp8_launch_count", "fp8_cast_group",
+    "fp8_linear_dgrad_act", "fp8_selftest_wait_expiry", "fp8_range_stats", "fp8_linear_fwd_q", "fp8_linear_dgrad_q", "fp8_amax_history_bias", "fp8_launch_count", "fp8_cast_group", "fp8_selftest_mma_ceiling", "fp8_bias_log_append", "fp8_bias_mode",
 )
 
 if not os.path.exists(LIB_PATH):
@@ -48,6 +49,9 @@ _lib.fp8_status_string.argtypes = [c_int]
 _lib.fp8_status_string.restype = c_char_p
 _lib.fp8_device_flags.argtypes = [_P, _P, POINTER(c_uint), c_int]
 _lib.fp8_selftest_wait_expiry.argtypes = [_P, ctypes.c_uint64, _P]
+_lib.fp8_selftest_mma_ceiling.argtypes = [_P, _P, _P, c_int64, c_int64, c_int64, _P]
+_lib.fp8_bias_log_append.argtypes = [_P, _P, c_int32, _P, c_int32, c_int32, _P, _P, c_int32, _P]
+_lib.fp8_bias_mode.argtypes = [_P, _P, c_int32, _P, c_int32, c_int32, c_int32, _P, _P, _P, _P]
 _lib.fp8_amax.argtypes = [_P, _P, c_int, c_int64, c_int64, c_int64, _P, _P]
 _lib.fp8_amax_noalloc.argtypes = [_P, c_int, c_int64, c_int64, c_int64, _P, _P]
 _lib.fp8_scaling_bias.argtypes = [_P, _P, c_int, c_int, c_int32, _P, _P]
@@ -146,7 +150,8 @@ def group_items(tensors):
         fmt, x, d_amax, d_bias, y = t[:5]
         it.x, it.x_dt, it.rows, it.cols, it.ld = x.data_ptr(), _DT[x.dtype], x.shape[0], x.shape[1], _ld(x)
         it.fmt, it.margin = fmt, (t[5] if len(t) > 5 else 0)
-        it.d_amax, it.d_bias, it.y = d_amax.data_ptr(), d_bias.data_ptr(), y.data_ptr()
+        it.d_amax = d_amax.data_ptr() if d_amax is not None else None
+        it.d_bias, it.y = d_bias.data_ptr(), (y.data_ptr() if y is not None else None)
     return arr
 
 
@@ -181,6 +186,11 @@ class Context:
         """Make one bounded device-side wait run out on purpose (raises FP8_FLAG_TIMEOUT, no fault)."""
         _check(_lib.fp8_selftest_wait_expiry(self._h, ctypes.c_uint64(limit_ns), _stream()), "fp8_selftest_wait_expiry")
 
+    def selftest_mma_ceiling(self, out, d_zero, K: int):
+        """The CTA-pair matmul kernel on an out.shape[0] x out.shape[1] x K problem with its operand loads off."""
+        _check(_lib.fp8_selftest_mma_ceiling(self._h, _ptr(out), _ptr(d_zero), out.shape[0], out.shape[1], K, _stream()),
+               "fp8_selftest_mma_ceiling")
+
     # -- amax / bias ------------------------------------------------------------
     def amax(self, x, d_amax, rows=None, cols=None, ld=None):
         rows = x.shape[0] if rows is None else rows
@@ -195,6 +205,17 @@ class Context:
     def amax_history_bias(self, d_history, d_cursor, d_amax_new, fmt, d_bias, conv=CONV_PAPER, margin=0):
         _check(_lib.fp8_amax_history_bias(self._h, _ptr(d_history), d_history.numel(), _ptr(d_cursor), _ptr(d_amax_new),
                                           fmt, conv, margin, _ptr(d_bias), _stream()), "fp8_amax_history_bias")
+
+    # -- bias log ---------------------------------------------------------------
+    def bias_log_append(self, d_ring, d_head, step, first_tensor_id, d_amax, d_bias):
+        """``fp8_bias_log_append``: d_ring is an int32 tensor [capacity, 4] (one ``fp8_bias_record_t`` per row: step,
+        tensor id, amax bits, bias), d_head an int64 scalar tensor; d_amax / d_bias are 1-D device arrays."""
+        _check(_lib.fp8_bias_log_append(self._h, _ptr(d_ring), d_ring.shape[0], _ptr(d_head), step, first_tensor_id,
+                                        _ptr(d_amax), _ptr(d_bias), d_amax.numel(), _stream()), "fp8_bias_log_append")
+
+    def bias_mode(self, d_ring, d_head, tensor_id, step_lo, step_hi, d_mode, d_count, d_samples=None):
+        _check(_lib.fp8_bias_mode(self._h, _ptr(d_ring), d_ring.shape[0], _ptr(d_head), tensor_id, step_lo, step_hi,
+                                  _ptr(d_mode), _ptr(d_count), _ptr(d_samples), _stream()), "fp8_bias_mode")
 
     # -- cast -------------------------------------------------------------------
     def _cast(self, fn, name, x, d_bias, conv, margin, d_amax_out, d_bias_out, y, y_t, rows, cols, ld):
@@ -222,11 +243,14 @@ class Context:
         _check(_lib.fp8_cast_predicted(self._h, fmt, _ptr(x), _DT[x.dtype], rows, cols, ld, conv, margin,
                                        _ptr(d_amax_out), _ptr(d_bias_inout), _ptr(y), _stream()), "fp8_cast_predicted")
 
-    def cast_group(self, items, conv=CONV_PAPER, predicted=False):
+    def cast_group(self, items, conv=CONV_PAPER, predicted=False, mode=None):
         """``fp8_cast_group``.  `items`: a ``group_items(...)`` array, or a list of (fmt, x, d_amax, d_bias, y[, margin])
-        tuples that is marshalled on the spot."""
+        tuples that is marshalled on the spot.  `mode`: one of the GROUP_* constants (default: GROUP_PREDICTED if
+        `predicted` else GROUP_AMAX_CAST)."""
         arr = items if isinstance(items, ctypes.Array) else group_items(items)
-        _check(_lib.fp8_cast_group(self._h, arr, len(arr), conv, 1 if predicted else 0, _stream()), "fp8_cast_group")
+        if mode is None:
+            mode = GROUP_PREDICTED if predicted else GROUP_AMAX_CAST
+        _check(_lib.fp8_cast_group(self._h, arr, len(arr), conv, mode, _stream()), "fp8_cast_group")
 
     def prediction_stats(self, clear: bool = True):
         hits, misses = c_uint(0), c_uint(0)

@@ -44,9 +44,13 @@ def gelu_grad_f32(y: torch.Tensor) -> torch.Tensor:
 
 class Fp8Stack:
     def __init__(self, ctx, layers: int = 24, d: int = 1024, tokens: int = 4096, lr: float = 1e-3,
-                 seed: int = I.BASE_SEED, device="cuda", w_std: float = 0.02, fused_activation: bool = False):
+                 seed: int = I.BASE_SEED, device="cuda", w_std: float = 0.02, fused_activation: bool = False,
+                 log_steps: int = 0):
         """fused_activation: GELU runs in the forward matmul's epilogue, which also emits the amax of the
-        activated tensor, so the next layer's input is quantised in one pass (no amax pass, no GELU kernel)."""
+        activated tensor, so the next layer's input is quantised in one pass (no amax pass, no GELU kernel).
+        log_steps > 0: every step appends the (amax, bias) of all 3 x layers tensors to a device-side ring that
+        holds the last `log_steps` steps (``fp8_bias_log_append``); see ``bias_records`` / ``write_bias_csv`` /
+        ``bias_modes``."""
         self.ctx, self.L, self.d, self.T, self.lr = ctx, layers, d, tokens, lr
         self.fused = fused_activation
         dev = dict(device=device)
@@ -69,6 +73,9 @@ class Fp8Stack:
         # per layer: amax / bias of W, X, dY
         self.amax = torch.zeros((layers, 3), dtype=torch.float32, **dev)
         self.bias = torch.zeros((layers, 3), dtype=torch.int32, **dev)
+        # bias log: one record {step, tensor id = 3 * layer + (0 W, 1 X, 2 dY), amax, bias} per tensor and step
+        self.log_ring = torch.zeros((log_steps * 3 * layers, 4), dtype=torch.int32, **dev) if log_steps > 0 else None
+        self.log_head = torch.zeros(1, dtype=torch.int64, **dev)
         # layers whose tensors the current step keeps copies of (inputs and outputs of every library call), for
         # comparisons made outside this module; empty in normal use
         self.snap_layers = ()
@@ -139,7 +146,49 @@ class Fp8Stack:
         out = self.forward(x)
         loss = torch.mean((out.to(torch.float32) - self.target.to(torch.float32)) ** 2)
         self.backward_and_update()
+        self._log(step, self.bias)
         return {"loss": loss, "bias": self.bias.clone(), "amax": self.amax.clone()}
+
+    # -- bias log (Appendix G / Appendix I style statistics) ---------------------------------------------------
+    def _log(self, step: int, bias_used: torch.Tensor) -> None:
+        if self.log_ring is not None:
+            self.ctx.bias_log_append(self.log_ring, self.log_head, step, 0, self.amax.view(-1),
+                                     bias_used.contiguous().view(-1))
+
+    def bias_records(self):
+        """The records currently in the ring, oldest first, as a list of (step, layer, tensor, amax, bias) with
+        tensor in {"W", "X", "dY"}.  Synchronises."""
+        if self.log_ring is None:
+            return []
+        ring = self.log_ring.cpu()
+        head = int(self.log_head.item())
+        cap = ring.shape[0]
+        order = range(head - min(head, cap), head)
+        amax = ring[:, 2].contiguous().view(torch.float32)
+        out = []
+        for n in order:
+            r = ring[n % cap]
+            tid = int(r[1])
+            out.append((int(r[0]), tid // 3, ("W", "X", "dY")[tid % 3], float(amax[n % cap]), int(r[3])))
+        return out
+
+    def write_bias_csv(self, path: str) -> int:
+        """step,layer,tensor,amax,bias for every record in the ring; returns the number of rows written."""
+        rows = self.bias_records()
+        with open(path, "w") as fh:
+            fh.write("step,layer,tensor,amax,bias\n")
+            for step, layer, tensor, amax, bias in rows:
+                fh.write(f"{step},{layer},{tensor},{amax!r},{bias}\n")
+        return len(rows)
+
+    def bias_modes(self, step_lo: int, step_hi: int) -> torch.Tensor:
+        """[layers, 3, 2] int32: per tensor, the mode of its bias over the logged steps in [step_lo, step_hi] and how
+        often it occurred (``fp8_bias_mode``)."""
+        out = torch.zeros((self.L, 3, 2), dtype=torch.int32, device=self.log_ring.device)
+        for l in range(self.L):
+            for j in range(3):
+                self.ctx.bias_mode(self.log_ring, self.log_head, 3 * l + j, step_lo, step_hi, out[l, j, 0:1], out[l, j, 1:2])
+        return out
 
 
 class Fp8StackHistory(Fp8Stack):
@@ -205,5 +254,6 @@ class Fp8StackHistory(Fp8Stack):
         used = self.bias.clone()
         used[:, 1:3] = self.pred[:, 1:3]
         rec = {"loss": loss, "bias": used, "amax": self.amax.clone()}
+        self._log(step, used)
         self._update_history()
         return rec

@@ -437,3 +437,38 @@ def test_amax_history_ring(ctx, lib, length, kind):
     with pytest.raises(lib.Fp8Error) as e:
         ctx.amax_history_bias(hist[:0], cursor, new, kind, bias)
     assert e.value.status in (lib.ERR_SHAPE, lib.ERR_NULL)
+
+
+def test_bias_log_ring_wraps_and_mode_breaks_ties_downwards(ctx, lib):
+    """fp8_bias_log_append on a ring of 10 records through several wraps, fp8_bias_mode on what the ring holds."""
+    ring = torch.zeros((10, 4), dtype=torch.int32, device="cuda")
+    head = torch.zeros(1, dtype=torch.int64, device="cuda")
+    kept = []          # what a ring of 10 must hold
+    biases = [[3, 7, -2], [3, 6, -2], [4, 6, -1], [4, 7, -1], [5, 7, -2], [3, 7, -2], [9, 9, 9]]
+    for step, b in enumerate(biases):
+        amax = torch.tensor([1.5 + step, 0.25, 100.0 * (step + 1)], dtype=torch.float32, device="cuda")
+        ctx.bias_log_append(ring, head, step, 40, amax, torch.tensor(b, dtype=torch.int32, device="cuda"))
+        kept += [(step, 40 + i, float(amax[i].item()), b[i]) for i in range(3)]
+    n = len(kept)
+    assert int(head.item()) == n
+    host = ring.cpu()
+    amax_f = host[:, 2].contiguous().view(torch.float32)
+    for k in range(n - 10, n):
+        r = host[k % 10]
+        assert (int(r[0]), int(r[1]), float(amax_f[k % 10]), int(r[3])) == kept[k]
+    mode, count, samples = (torch.zeros(1, dtype=torch.int32, device="cuda") for _ in range(3))
+    live = kept[n - 10:]
+    for tid in (40, 41, 42, 43):
+        for lo, hi in ((0, 99), (4, 5), (6, 6), (50, 60)):
+            ctx.bias_mode(ring, head, tid, lo, hi, mode, count, samples)
+            seq = [b for (s_, t_, _, b) in live if t_ == tid and lo <= s_ <= hi]
+            assert (int(mode.item()), int(count.item())) == O.bias_mode(seq) and int(samples.item()) == len(seq)
+    # a tie: biases 4 and 6 twice each -> the smaller
+    ring.zero_(); head.zero_()
+    for step, b in enumerate((6, 4, 6, 4, 9)):
+        ctx.bias_log_append(ring, head, step, 0, torch.ones(1, device="cuda"), torch.tensor([b], dtype=torch.int32, device="cuda"))
+    ctx.bias_mode(ring, head, 0, 0, 10, mode, count)
+    assert (int(mode.item()), int(count.item())) == (4, 2)
+    with pytest.raises(lib.Fp8Error) as e:
+        ctx.bias_log_append(ring, head, 0, 0, torch.ones(11, device="cuda"), torch.ones(11, dtype=torch.int32, device="cuda"))
+    assert e.value.status == lib.ERR_SHAPE

@@ -164,3 +164,19 @@ def test_paper_e4_top_code_has_no_native_byte():
     assert O.decode(O.N_E4, 0x7E) / 2 == 224.0
     a, b, y = O.quantise(np.array([[236.0, 1.0]], dtype=np.float32), O.E4, O.CONV_NATIVE)
     assert b == 0 and O.decode(O.N_E4, int(y[0, 0])) == 240.0   # 236 rounds to 240 on the native grid, no clipping
+
+
+def test_bias_mode_of_hand_made_sequences():
+    """Appendix G's per-tensor statistic: the most frequent bias; the smaller value on a tie."""
+    assert O.bias_mode([7, 7, 6, 7, 8, 6]) == (7, 3)
+    assert O.bias_mode([5, 6, 6, 5]) == (5, 2)            # tie -> smaller
+    assert O.bias_mode([-3, -4, -4, -3, 2]) == (-4, 2)    # tie between negatives -> smaller
+    assert O.bias_mode([19]) == (19, 1)
+    assert O.bias_mode([]) == (0, 0)
+    # against a library routine on random draws: scipy's mode also returns the smallest of the most frequent values
+    from scipy import stats
+    rng = np.random.default_rng(4)
+    for _ in range(20):
+        seq = rng.integers(-6, 7, size=int(rng.integers(1, 40)))
+        m = stats.mode(seq, keepdims=False)
+        assert O.bias_mode(seq) == (int(m.mode), int(m.count))

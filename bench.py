@@ -20,6 +20,7 @@ Single-kernel legs (one line of text per shape, no JSON):
     python bench.py --leg cast  --shapes 8192x4096 8192x22016              # amax, cast, amax+cast of bf16 [rows x cols]
     python bench.py --leg stack --shapes 24x1024x4096                      # layers x d x tokens: the SGD stack
     python bench.py --leg mlp   --shapes 8192x4096x11008                   # tokens x d x ffn: a gated MLP, unfused vs fused
+    python bench.py --leg group --workload c2_gpt                          # fp8_cast_group over a workload's tensors, each mode
 """
 from __future__ import annotations
 
@@ -790,17 +791,45 @@ def leg_mlp(ctx, fp8lin, shapes, iters=20, quiet=False):
     return results
 
 
+def leg_group(ctx, fp8lin, wl, reps=3):
+    """fp8_cast_group over every tensor a step of the workload quantises, one launch pair at a time: the amax pass,
+    the cast pass, the one-pass mode (every guess holds) and the two-pass mode."""
+    layers = [LayerState(wl, li, "cuda", I.BASE_SEED, wl.backward) for li in range(len(wl.layers))]
+    tensors = [it for L in layers for it in L.quant_items()]
+    items = fp8lin.group_items(tensors)
+    elems = sum(t[1].numel() for t in tensors)
+    ctx.cast_group(items)
+    line = f"group {wl.name}: {len(tensors)} tensors, {elems / 1e6:.0f} M elements:"
+    for name, bpe, mode in (("amax pass", 2, fp8lin.GROUP_AMAX_ONLY), ("cast pass", 3, fp8lin.GROUP_CAST_ONLY),
+                            ("one pass", 3, fp8lin.GROUP_PREDICTED), ("two passes", 5, fp8lin.GROUP_AMAX_CAST)):
+        ms = []
+        for r in range(reps + 1):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda._sleep(200000)
+            a.record()
+            ctx.cast_group(items, mode=mode)
+            b.record()
+            torch.cuda.synchronize()
+            if r:
+                ms.append(a.elapsed_time(b))
+        t = sum(ms) / len(ms)
+        line += f" | {name} {t * 1e3:6.1f} us {elems * bpe / t / 1e6:6.0f} GB/s on {bpe} B/element"
+    print(line, flush=True)
+
+
 def run_leg(args):
     from paper_2309_17224_b200 import build as B
     B.build()
     from paper_2309_17224_b200 import fp8lin
     shapes = [tuple(int(v) for v in a.split("x")) for a in args.shapes]
-    if not shapes:
+    if not shapes and args.leg != "group":
         print(__doc__)
         return 2
     torch.cuda.set_device(0)
     ctx = fp8lin.Context(0)
-    if args.leg == "gemm":
+    if args.leg == "group":
+        leg_group(ctx, fp8lin, I.WORKLOADS[args.workload])
+    elif args.leg == "gemm":
         leg_gemm(ctx, fp8lin, shapes, fused=not args.plain_only)
     elif args.leg == "cast":
         leg_cast(ctx, fp8lin, shapes)
@@ -876,10 +905,11 @@ def main():
     ap.add_argument("--no-extra-legs", action="store_true",
                     help="skip every leg beside the headline: other quantisation modes, moving gradients, sustained "
                          "run, tensor-pipe ceiling, fused MLP, other workloads")
+    ap.add_argument("--no-ceiling-leg", action="store_true", help="skip the tensor-pipe ceiling measurement")
     ap.add_argument("--sustain-seconds", type=float, default=3.0)
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--leg", default="step", choices=["step", "gemm", "cast", "stack", "mlp"])
+    ap.add_argument("--leg", default="step", choices=["step", "gemm", "cast", "stack", "mlp", "group"])
     ap.add_argument("--shapes", nargs="*", default=[])
     ap.add_argument("--only", default=None, help="--leg stack: run only the variant whose name contains this")
     ap.add_argument("--plain-only", action="store_true", help="--leg gemm: skip the fused epilogues")
@@ -991,6 +1021,33 @@ def main():
                                "cast >= 0.80 of HBM peak (amax_cast.per_kernel.*.frac); frac is against 2 x the cuBLAS "
                                "bf16 rate measured on this pool")
 
+    # ---- what the matmul kernel reaches when moving operands costs nothing ----
+    ceiling = None
+    if not args.no_ceiling_leg and not decode and rank == 0:
+        try:
+            big = max(layers, key=lambda L: L.T * L.N * L.K)
+            zero = torch.zeros(1, dtype=torch.int32, device=device)
+            c_sampler = ClockSampler(local)
+            shapes = {"long_k": (8192, 8192, 16384), "largest_layer_fwd": (big.T, big.N, big.K)}
+            ceiling = {"how": "fp8_selftest_mma_ceiling: gemm_pair_kernel with its operand loads off (barriers, MMAs, "
+                              "epilogue and stores as usual), 10 launches back to back right after the timed region, beside "
+                              "the same shape with loads; when the power cap already holds the clock down the two meet: "
+                              "the limit is then the power of the tensor pipe, not the operand feed"}
+            for name, (M, N, K) in shapes.items():
+                out = torch.empty((M, N), dtype=torch.bfloat16, device=device)
+                a8 = torch.randint(0, 0x78, (M, K), dtype=torch.uint8, device=device)
+                b8 = torch.randint(0, 0x78, (N, K), dtype=torch.uint8, device=device)
+                t_off = _time_burst(lambda: ctx.selftest_mma_ceiling(out, zero, K), 10, warm=2)
+                t_on = _time_burst(lambda: ctx.linear_fwd(a8, zero, b8, zero, out), 10, warm=2)
+                ceiling[name] = {"shape_mnk": [M, N, K], "loads_off_tflops": 2.0 * M * N * K / t_off / 1e9,
+                                 "with_loads_tflops": 2.0 * M * N * K / t_on / 1e9}
+                del out, a8, b8
+            ceiling["clocks"] = c_sampler.stop()
+            roofline["ceiling"] = ceiling
+        except Exception as exc:
+            roofline["ceiling"] = {"error": str(exc)[:200]}
+            torch.cuda.synchronize()
+
     extra = not args.no_extra_legs
     # ---- the quantisation kernels, each against its own algorithmic bytes (outside the timed region) ----
     per_kernel = quantisation_kernel_bandwidths(ctx, fp8lin, layers, peaks["hbm_gbs"])
@@ -1097,31 +1154,6 @@ def main():
             sustained["frac_of_2x_sustained_bf16"] = sustained["value"] / world / (2.0 * peaks["bf16_tflops_sustained"])
             sustained["note"] = ("whole step (quantisation included) against 2 x the sustained cuBLAS bf16 rate; "
                                  "ms_times_sm_ghz compares runs at different clocks")
-
-    # ---- what the matmul kernel reaches when moving operands costs nothing ----
-    ceiling = None
-    if extra and not decode and rank == 0:
-        try:
-            big = max(layers, key=lambda L: L.T * L.N * L.K)
-            zero = torch.zeros(1, dtype=torch.int32, device=device)
-            c_sampler = ClockSampler(local)
-            shapes = {"long_k": (8192, 8192, 16384), "largest_layer_fwd": (big.T, big.N, big.K)}
-            ceiling = {"how": "fp8_selftest_mma_ceiling: gemm_pair_kernel with its operand loads off (barriers, MMAs, "
-                              "epilogue and stores as usual), 20 launches back to back, beside the same shape with loads"}
-            for name, (M, N, K) in shapes.items():
-                out = torch.empty((M, N), dtype=torch.bfloat16, device=device)
-                a8 = torch.randint(0, 0x78, (M, K), dtype=torch.uint8, device=device)
-                b8 = torch.randint(0, 0x78, (N, K), dtype=torch.uint8, device=device)
-                t_off = _time_burst(lambda: ctx.selftest_mma_ceiling(out, zero, K), 20)
-                t_on = _time_burst(lambda: ctx.linear_fwd(a8, zero, b8, zero, out), 20)
-                ceiling[name] = {"shape_mnk": [M, N, K], "loads_off_tflops": 2.0 * M * N * K / t_off / 1e9,
-                                 "with_loads_tflops": 2.0 * M * N * K / t_on / 1e9}
-                del out, a8, b8
-            ceiling["clocks"] = c_sampler.stop()
-            roofline["ceiling"] = ceiling
-        except Exception as exc:
-            roofline["ceiling"] = {"error": str(exc)[:200]}
-            torch.cuda.synchronize()
 
     # ---- the gated MLP of the same model as one chained block, unfused against the fused epilogues ----
     fused_mlp = None

@@ -363,6 +363,7 @@ cast_small_kernel(const uint4 *__restrict__ x, uint4 *__restrict__ y, int64_t nv
     // A matmul launched behind this kernel as a programmatic dependent may take its places now and start
     // streaming its weights; it waits for this grid to complete before it touches anything written here.
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");   // the tensor may come from the launch before this one
 
     uint4 v[kSmallVecs];
     uint32_t acc = 0;
@@ -458,13 +459,16 @@ static cudaError_t launch_small(fp8_ctx *ctx, const void *x, int64_t n, int conv
     cfg.blockDim = dim3(kSmallThreads, 1, 1);
     cfg.dynamicSmemBytes = 0;
     cfg.stream = stream;
-    cudaLaunchAttribute attr;
-    attr.id = cudaLaunchAttributeClusterDimension;
-    attr.val.clusterDim.x = (unsigned)ctas;
-    attr.val.clusterDim.y = 1;
-    attr.val.clusterDim.z = 1;
-    cfg.attrs = &attr;
-    cfg.numAttrs = 1;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)ctas;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    // may be set up while the launch before it drains; it reads nothing before that launch has completed
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
     count_launch();
     return cudaLaunchKernelEx(&cfg, cast_small_kernel<FMT, DT>, reinterpret_cast<const uint4 *>(x),
                               reinterpret_cast<uint4 *>(y), nvec, ntail, (int)FMT, conv, margin, format_delta(FMT, conv),

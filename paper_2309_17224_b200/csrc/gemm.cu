@@ -1200,7 +1200,9 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();
-    const int num_tiles = p.tiles_m * p.tiles_n;
+    // an item is one output tile, or one slice of its contraction when the launch splits it (few tiles, long
+    // contraction: partial sums go to the FP32 workspace and splitk_finalize_kernel adds them up)
+    const int num_tiles = p.tiles_m * p.tiles_n * p.splits;
     const int pair_id = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
 
     if (threadIdx.x == 0) {
@@ -1228,6 +1230,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
     cluster_sync_all();  // both CTAs' barriers exist before anyone signals across
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    if (p.splits > 1) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the finalize kernel may take its places
 
     if (warp == 0) {
         if (lane == 0) {
@@ -1241,8 +1244,9 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             asm volatile("griddepcontrol.wait;" ::: "memory");
             for (int tile = pair_id; alive && tile < num_tiles; tile += num_pairs) {
                 int m_blk, n_blk;
-                tile_coords(tile, p, m_blk, n_blk);
-                for (int k = 0; k < p.num_k; ++k, ++it) {
+                tile_coords(tile / p.splits, p, m_blk, n_blk);
+                const int k0 = (tile % p.splits) * p.kb_per_split, k1 = min(p.num_k, k0 + p.kb_per_split);
+                for (int k = k0; k < k1; ++k, ++it) {
                     const int s = it % kStagesL;
                     const uint32_t leader_full = leader_full0 + 8u * s;
                     const uint32_t ph = (it / kStagesL) & 1u;
@@ -1282,6 +1286,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                 if (!mbar_wait(acc_empty_bar(buf), acc_ph ^ 1u, abort_flag, p.d_status)) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + buf * kPairBN;
+                const int k0 = (tile % p.splits) * p.kb_per_split, k1 = min(p.num_k, k0 + p.kb_per_split);
                 auto issue = [&](int s, int k, int h) {
                     const uint32_t a_addr = smem_base + s * L::kStageBytes;
                     const uint32_t b_addr = a_addr + L::kABytes + h * (kPairHalfN * kBK);
@@ -1291,30 +1296,30 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                     const uint32_t step_a = p.a_mn ? 256u : 2u, step_b = p.b_mn ? 256u : 2u;
 #pragma unroll
                     for (int j = 0; j < kBK / kUmmaK; ++j)
-                        umma_f8_pair(d_tmem + h * kPairBN, da + step_a * j, db + step_b * j, p.idesc, (k > 0 || j > 0) ? 1u : 0u);
+                        umma_f8_pair(d_tmem + h * kPairBN, da + step_a * j, db + step_b * j, p.idesc, (k > k0 || j > 0) ? 1u : 0u);
                 };
-                int k = 0;
+                int k = k0;
                 if (NHALF == 2) {
                     // The epilogue of the previous tile drains half 0, then half 1.  The first k-blocks of this tile
                     // run on half 0 alone while half 1 is still being read; their stages stay held until half 1 has
                     // used them too.
-                    const int ahead = min(p.num_k, kStagesL - 1);
+                    const int ahead = min(k1 - k0, kStagesL - 1);
                     for (int a = 0; alive && a < ahead; ++a) {
                         const uint32_t ia = it + a;
                         if (!mbar_wait(full_bar(ia % kStagesL), (ia / kStagesL) & 1u, abort_flag, p.d_status)) { alive = false; break; }
                         tc_fence_after();
-                        issue(ia % kStagesL, a, 0);
+                        issue(ia % kStagesL, k0 + a, 0);
                     }
                     if (alive && !mbar_wait(acc_empty_bar(1), acc_ph ^ 1u, abort_flag, p.d_status)) alive = false;
                     if (!alive) break;
                     tc_fence_after();
                     for (int a = 0; a < ahead; ++a, ++it) {
-                        issue(it % kStagesL, a, 1);
+                        issue(it % kStagesL, k0 + a, 1);
                         umma_commit_pair(empty_bar(it % kStagesL));
                     }
-                    k = ahead;
+                    k = k0 + ahead;
                 }
-                for (; k < p.num_k; ++k, ++it) {
+                for (; k < k1; ++k, ++it) {
                     const int s = it % kStagesL;
                     const uint32_t ph = (it / kStagesL) & 1u;
                     if (!mbar_wait(full_bar(s), ph, abort_flag, p.d_status)) { alive = false; break; }
@@ -1336,9 +1341,21 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
         const uint32_t warp_slabs = smem_base + L::kEpiOffset + q * L::kSlabs * kSlabBytes;
         const uint32_t leader_acc_empty0 = map_to_cta(acc_empty_bar(0), 0);
         uint32_t t = 0;
+        // with a split contraction every item leaves its raw FP32 partial sum in the workspace
+        GemmParams pp = p;
+        if (p.splits > 1) {
+            pp.out_dt = FP8_F32;
+            pp.bias_vec = nullptr;
+            pp.d_amax_bits = nullptr;
+            pp.tma_out = 0;
+            pp.vec_ok = (p.N % 4) == 0;
+            pp.ldo = p.N;
+        }
+        const Pow2Pair sc_one = make_pow2_pair(0);
         for (int tile = pair_id; tile < num_tiles; tile += num_pairs, ++t) {
             int m_blk, n_blk;
-            tile_coords(tile, p, m_blk, n_blk);
+            tile_coords(tile / p.splits, p, m_blk, n_blk);
+            if (p.splits > 1) pp.out = p.partial + (int64_t)(tile % p.splits) * p.M * p.N;
             const int buf = NHALF == 2 ? 0 : (t & 1);
             const uint32_t acc_ph = NHALF == 2 ? (t & 1u) : ((t >> 1) & 1u);
             const bool ready = mbar_wait(acc_full_bar(buf), acc_ph, abort_flag, p.d_status);
@@ -1348,8 +1365,9 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
 #pragma unroll 1
             for (int h = 0; h < NHALF; ++h)   // the wide tile: half 0 is handed back to the MMA thread before half 1 is read
                 epilogue_tile<kPairBN, ACT, L::kSlabs>(&map_out, &map_out2, t_row + h * kPairBN,
-                                                       m_blk * 256 + (int)rank * kBM + q * 32, n_blk * kTileN + h * kPairBN, p,
-                                                       sc, two_step, amax_bits, warp_slabs, slab_count,
+                                                       m_blk * 256 + (int)rank * kBM + q * 32, n_blk * kTileN + h * kPairBN, pp,
+                                                       p.splits > 1 ? sc_one : sc, p.splits > 1 ? false : two_step, amax_bits,
+                                                       warp_slabs, slab_count,
                                                        leader_acc_empty0 + 8u * (NHALF == 2 ? h : buf), true, lane);
         }
         if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
@@ -1378,7 +1396,9 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
 template <int VEC>
 __global__ void __launch_bounds__(256) splitk_finalize_kernel(const GemmParams p)
 {
-    // launched as a programmatic dependent of the matmul kernel: nothing of that grid's output is read before this
+    // launched as a programmatic dependent of the matmul kernel: nothing of that grid's output is read before this;
+    // the launch behind this one may take its places as blocks here retire (it waits the same way)
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     asm volatile("griddepcontrol.wait;" ::: "memory");
     const int64_t total = (int64_t)p.M * p.N;
     const int e = -(__ldg(p.d_sa) + __ldg(p.d_sb) + p.delta_sum);
@@ -1647,8 +1667,28 @@ static fp8_status_t run_gemm(fp8_ctx *ctx, const uint8_t *a, int a_fmt, bool a_m
                     best_kb = kb;
                 }
             }
-            if (g_force_splits > 0) best_kb = (p.num_k + g_force_splits - 1) / g_force_splits;
+            if (g_force_splits > 0) {   // an experiment's count, still bounded by the workspace
+                const int64_t forced = g_force_splits < by_ws ? g_force_splits : (by_ws > 0 ? by_ws : 1);
+                best_kb = (p.num_k + forced - 1) / forced;
+            }
             p.kb_per_split = (int)best_kb;
+            p.splits = (p.num_k + p.kb_per_split - 1) / p.kb_per_split;
+        }
+    }
+    if (pair && !g_no_splitk && !act && !no_loads) {
+        // Fewer tiles than CTA pairs and a long contraction: slice it so that most pairs have work.  The second
+        // launch and the trip of the partial sums through memory cost 6-7 us, so a slice keeps at least sixteen
+        // k-blocks (measured: 1024 x 1024 x 8192 27 -> 22 us, 512 x 512 x 16384 46 -> 20 us; at 32 k-blocks or fewer
+        // per tile the unsplit launch wins); the partial sums must fit the workspace.
+        const int64_t tiles = (int64_t)p.tiles_m * p.tiles_n;
+        int64_t sp = g_max_pairs / tiles;
+        const int64_t by_k = p.num_k / 16, by_ws = (int64_t)(ctx->partial_bytes / sizeof(float)) / (M * N);
+        if (sp > by_k) sp = by_k;
+        if (sp > 16) sp = 16;
+        if (g_force_splits > 0) sp = g_force_splits;
+        if (sp > by_ws) sp = by_ws;   // never beyond the workspace, whatever asked for the count
+        if (sp > 1) {
+            p.kb_per_split = (int)((p.num_k + sp - 1) / sp);
             p.splits = (p.num_k + p.kb_per_split - 1) / p.kb_per_split;
         }
     }
@@ -1697,7 +1737,8 @@ static fp8_status_t run_gemm(fp8_ctx *ctx, const uint8_t *a, int a_fmt, bool a_m
     int tiles = p.tiles_m * p.tiles_n;
     count_launch(p.splits > 1 ? 2 : 1);
     if (pair) {
-        int pairs = tiles < g_max_pairs ? tiles : g_max_pairs;
+        const int items = tiles * p.splits;
+        int pairs = items < g_max_pairs ? items : g_max_pairs;
         const dim3 grid(2 * pairs);
         switch (act) {
         case 1: gemm_pair_kernel<1><<<grid, kGemmThreads, PairSmemAct::kDynamic, st>>>(map_a, map_b, map_out, map_out2, p); break;
@@ -1749,25 +1790,25 @@ static fp8_status_t run_gemm(fp8_ctx *ctx, const uint8_t *a, int a_fmt, bool a_m
             break;
         }
         }
-        if (p.splits > 1) {
-            if (cudaGetLastError() != cudaSuccess) return FP8_ERR_CUDA;
-            const bool vec = p.vec_ok && (N % 4) == 0;
-            int64_t threads = vec ? M * N / 4 : M * N;
-            int64_t blocks = (threads + 255) / 256;
-            if (blocks > (int64_t)ctx->sm_count * 16) blocks = (int64_t)ctx->sm_count * 16;
-            cudaLaunchAttribute attr[1];
-            attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-            attr[0].val.programmaticStreamSerializationAllowed = 1;
-            cudaLaunchConfig_t cfg = {};
-            cfg.gridDim = dim3((unsigned)blocks);
-            cfg.blockDim = dim3(256);
-            cfg.stream = st;
-            cfg.attrs = attr;
-            cfg.numAttrs = 1;
-            cudaError_t le = vec ? cudaLaunchKernelEx(&cfg, splitk_finalize_kernel<4>, p)
-                                 : cudaLaunchKernelEx(&cfg, splitk_finalize_kernel<1>, p);
-            if (le != cudaSuccess) return FP8_ERR_CUDA;
-        }
+    }
+    if (p.splits > 1) {
+        if (cudaGetLastError() != cudaSuccess) return FP8_ERR_CUDA;
+        const bool vec = p.vec_ok && (N % 4) == 0;
+        int64_t threads = vec ? M * N / 4 : M * N;
+        int64_t blocks = (threads + 255) / 256;
+        if (blocks > (int64_t)ctx->sm_count * 16) blocks = (int64_t)ctx->sm_count * 16;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)blocks);
+        cfg.blockDim = dim3(256);
+        cfg.stream = st;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        cudaError_t le = vec ? cudaLaunchKernelEx(&cfg, splitk_finalize_kernel<4>, p)
+                             : cudaLaunchKernelEx(&cfg, splitk_finalize_kernel<1>, p);
+        if (le != cudaSuccess) return FP8_ERR_CUDA;
     }
     return cudaGetLastError() == cudaSuccess ? FP8_OK : FP8_ERR_CUDA;
 }

@@ -3,11 +3,11 @@
 //
 // The tensors a step quantises are tens to hundreds of megabytes each; launched one by one, every kernel pays its
 // own ramp-up and its own thin last wave, which at these sizes is 10-40 % of its run time.  Here the tensors of a
-// group are cut into chunks of 8192 elements, the chunks of all tensors are numbered in one sequence and a
+// group are cut into chunks of a few thousand elements, the chunks of all tensors are numbered in one sequence and a
 // persistent grid walks that sequence with a grid stride, so the whole group has one ramp and one tail.  Each
-// tensor keeps its own reduction slot: a block folds its running maximum into the slot when it moves on to the
-// next tensor, adds the number of chunks it did, and the block that completes the count publishes that tensor's
-// amax and bias.
+// tensor keeps its own reduction slot: a block notes its maximum of a tensor when it moves on to the next one, folds
+// all its notes into the slots at the end (one thread per tensor), adds the number of chunks it did, and the block
+// that completes a tensor's count publishes that tensor's amax and bias.
 //
 // Two modes, both bit-identical to fp8_cast_e4 / fp8_cast_e5 with d_bias = NULL per tensor:
 //   just in time   group_kernel<kAmax> over all tensors, then group_kernel<kCast> (a programmatic dependent) over
@@ -22,8 +22,13 @@
 namespace fp8lin {
 
 constexpr int kGroupMax = FP8_GROUP_MAX;
-constexpr int kChunkElems = 8192;             // elements per chunk
-constexpr int kChunkOut = kChunkElems / 16;   // 16-byte output vectors per chunk: two per thread
+// Measured on the twelve tensors of a Llama-2-7B step (1.5 GB of bf16): four output vectors per thread and chunk
+// (eight 16-byte loads in flight per thread), three resident blocks per SM for the read-only pass and two for the
+// passes that also write, streaming stores: amax 7.0 TB/s, cast 6.7 TB/s, one pass 6.3 TB/s.  More blocks per SM
+// cost the writing passes up to a third of their bandwidth (5 per SM: 5.8 TB/s).
+constexpr int kUnroll = 4;                               // 16-byte output vectors per thread and chunk
+__host__ __device__ constexpr int group_blocks_per_sm(int mode) { return mode == 0 ? 3 : 2; }
+constexpr int kChunkOut = kUnroll * kCastThreads;       // 16-byte output vectors per chunk
 
 struct GroupItem {
     const uint4 *x;
@@ -51,7 +56,7 @@ __device__ __forceinline__ uint32_t fold_any(int dt, uint32_t acc, uint32_t w)
     return dt == FP8_F32 ? max(acc, w & 0x7FFFFFFFu) : __vmaxu2(acc, w & 0x7FFF7FFFu);
 }
 
-// One chunk of one tensor: thread t owns output vectors c * 512 + t and c * 512 + 256 + t.
+// One chunk of one tensor: thread t owns output vectors c * kChunkOut + t + u * 256, u < kUnroll.
 template <int MODE, int FMT, int DT, bool TWO_STEP>
 __device__ __forceinline__ void chunk_body(const uint4 *__restrict__ gx, uint4 *__restrict__ gy, int64_t n, int64_t c,
                                            Pow2Pair p, uint32_t &acc, bool &sat)
@@ -59,17 +64,19 @@ __device__ __forceinline__ void chunk_body(const uint4 *__restrict__ gx, uint4 *
     constexpr int kIn = InType<DT>::kBytes;   // input vectors per output vector
     constexpr int kW = InType<DT>::kWords4;
     const int64_t nout = n / 16;
-    const int64_t idx[2] = {c * kChunkOut + threadIdx.x, c * kChunkOut + threadIdx.x + kCastThreads};
-    uint4 v[2][kIn];
+    int64_t idx[kUnroll];
 #pragma unroll
-    for (int u = 0; u < 2; ++u)
+    for (int u = 0; u < kUnroll; ++u) idx[u] = c * kChunkOut + threadIdx.x + u * kCastThreads;
+    uint4 v[kUnroll][kIn];
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u)
         if (idx[u] < nout) {
 #pragma unroll
             for (int j = 0; j < kIn; ++j)
                 v[u][j] = MODE == kAmax ? __ldg(gx + kIn * idx[u] + j) : __ldcs(gx + kIn * idx[u] + j);
         }
 #pragma unroll
-    for (int u = 0; u < 2; ++u)
+    for (int u = 0; u < kUnroll; ++u)
         if (idx[u] < nout) {
             const uint32_t *w = reinterpret_cast<const uint32_t *>(&v[u][0]);
             if (MODE != kCast) {
@@ -82,7 +89,7 @@ __device__ __forceinline__ void chunk_body(const uint4 *__restrict__ gx, uint4 *
                 o.y = cast4w<FMT, DT, TWO_STEP>(w + 1 * kW, p, sat);
                 o.z = cast4w<FMT, DT, TWO_STEP>(w + 2 * kW, p, sat);
                 o.w = cast4w<FMT, DT, TWO_STEP>(w + 3 * kW, p, sat);
-                gy[idx[u]] = o;
+                __stcs(gy + idx[u], o);   // the bytes are read next by a matmul, long after this pass
             }
         }
     // the elements past the last whole output vector belong to the tensor's first chunk
@@ -111,46 +118,66 @@ __device__ __forceinline__ void item_loop(const GroupItem &g, int64_t c, int64_t
     }
 }
 
-// A block leaves tensor `g` after `done` chunks: fold its maximum into the tensor's slot; the block that completes
-// the tensor's chunk count publishes amax and bias (and, in the predicted mode, the verdict on the guess).
-template <int MODE>
-__device__ __forceinline__ void leave_item(const GroupItem &g, int conv, unsigned *d_status, unsigned *d_stats,
-                                           uint32_t acc, bool sat, unsigned done, int guess)
+// What a block found in the tensors it walked, kept in shared memory until the end of the kernel: the block's
+// maximum, how many chunks it did, whether a value clipped, the guess it cast with.
+struct BlockNotes {
+    uint32_t max_key[kGroupMax];
+    unsigned done[kGroupMax];
+    unsigned sat[kGroupMax];
+    int guess[kGroupMax];
+};
+
+// A block leaves tensor `item` after `done` chunks: reduce its maximum across the block and note it.
+__device__ __forceinline__ void note_item(BlockNotes &notes, int item, int dt, uint32_t acc, bool sat, unsigned done, int guess)
 {
     __shared__ uint32_t warp_max[kCastThreads / 32];
-    uint32_t m = g.dt == FP8_F32 ? acc : max(acc & 0xFFFFu, acc >> 16);
+    uint32_t m = dt == FP8_F32 ? acc : max(acc & 0xFFFFu, acc >> 16);
     m = __reduce_max_sync(0xFFFFFFFFu, m);
     if ((threadIdx.x & 31) == 0) warp_max[threadIdx.x >> 5] = m;
     const int any_sat = __syncthreads_or(sat);
     if (threadIdx.x == 0) {
 #pragma unroll
         for (int i = 1; i < kCastThreads / 32; ++i) m = max(m, warp_max[i]);
-        atomicMax(&g.slot[0], m);
-        if (MODE == kBoth && any_sat) atomicOr(&g.slot[2], 1u);
-        __threadfence();
-        if (atomicAdd(&g.slot[1], done) + done == (unsigned)g.chunks) {
-            __threadfence();
-            const uint32_t total = atomicExch(&g.slot[0], 0u);
-            const unsigned was_sat = atomicExch(&g.slot[2], 0u);
-            g.slot[1] = 0u;
-            uint32_t fbits;
-            if (g.dt == FP8_F32) fbits = total;
-            else if (g.dt == FP8_BF16) fbits = total << 16;
-            else { float f; asm("cvt.f32.f16 %0, %1;" : "=f"(f) : "h"((uint16_t)total)); fbits = __float_as_uint(f); }
-            *g.d_amax = __uint_as_float(fbits);
-            unsigned flags = 0;
-            const int b = bias_from_amax_bits(fbits, g.fmt, conv, g.margin, &flags);
-            *g.d_bias = b;
-            if (MODE == kBoth) {
-                const bool hit = b == guess;
-                g.slot[3] = hit ? 0u : 1u;   // read by the gated second launch
-                atomicAdd(&d_stats[hit ? 0 : 1], 1u);
-                if (hit && was_sat) flags |= FP8_FLAG_SATURATED;   // clipping under a wrong guess says nothing
-            }
-            if (flags) atomicOr(d_status, flags);
-        }
+        notes.max_key[item] = m;
+        notes.done[item] = done;
+        notes.sat[item] = any_sat ? 1u : 0u;
+        notes.guess[item] = guess;
     }
     __syncthreads();   // warp_max is reused by the next tensor
+}
+
+// End of the kernel: one thread per tensor folds the block's note into the tensor's slot (all tensors at once, so
+// the block pays one round trip to the atomics and not one per tensor); the thread that completes a tensor's chunk
+// count publishes its amax and bias and, in the predicted mode, the verdict on the guess.
+template <int MODE>
+__device__ __forceinline__ void publish_item(const GroupItem &g, const BlockNotes &notes, int item, int conv,
+                                             unsigned *d_status, unsigned *d_stats)
+{
+    const unsigned done = notes.done[item];
+    if (done == 0u) return;
+    atomicMax(&g.slot[0], notes.max_key[item]);
+    if (MODE == kBoth && notes.sat[item]) atomicOr(&g.slot[2], 1u);
+    __threadfence();
+    if (atomicAdd(&g.slot[1], done) + done != (unsigned)g.chunks) return;
+    __threadfence();
+    const uint32_t total = atomicExch(&g.slot[0], 0u);
+    const unsigned was_sat = atomicExch(&g.slot[2], 0u);
+    g.slot[1] = 0u;
+    uint32_t fbits;
+    if (g.dt == FP8_F32) fbits = total;
+    else if (g.dt == FP8_BF16) fbits = total << 16;
+    else { float f; asm("cvt.f32.f16 %0, %1;" : "=f"(f) : "h"((uint16_t)total)); fbits = __float_as_uint(f); }
+    *g.d_amax = __uint_as_float(fbits);
+    unsigned flags = 0;
+    const int b = bias_from_amax_bits(fbits, g.fmt, conv, g.margin, &flags);
+    *g.d_bias = b;
+    if (MODE == kBoth) {
+        const bool hit = b == notes.guess[item];
+        g.slot[3] = hit ? 0u : 1u;   // read by the gated second launch
+        atomicAdd(&d_stats[hit ? 0 : 1], 1u);
+        if (hit && was_sat) flags |= FP8_FLAG_SATURATED;   // clipping under a wrong guess says nothing
+    }
+    if (flags) atomicOr(d_status, flags);
 }
 
 // Item `i` of the parameter block.  Kernel parameters cannot be indexed by a run-time value without the compiler
@@ -173,12 +200,17 @@ __device__ __forceinline__ GroupItem get_item(const GroupParams &gp, int i)
 // amax passes count from the front of the first tensor; the cast pass counts from the back of the last one, so that
 // what the amax pass read last (and may still be in L2) is read first.
 template <int MODE, int DT>
-__global__ void __launch_bounds__(kCastThreads, 5) group_kernel(const __grid_constant__ GroupParams gp, int gate)
+__global__ void __launch_bounds__(kCastThreads, group_blocks_per_sm(MODE)) group_kernel(const __grid_constant__ GroupParams gp, int gate)
 {
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (MODE == kCast) asm volatile("griddepcontrol.wait;" ::: "memory");   // biases / redo flags of the launch before
     const int64_t grid = gridDim.x, b = blockIdx.x;
     bool any_sat = false;
+    __shared__ BlockNotes notes;
+    if (MODE != kCast) {
+        if (threadIdx.x < kGroupMax) notes.done[threadIdx.x] = 0u;
+        __syncthreads();
+    }
     for (int n = 0; n < gp.count; ++n) {
         const int item = MODE == kCast ? gp.count - 1 - n : n;
         const GroupItem g = get_item(gp, item);
@@ -201,9 +233,13 @@ __global__ void __launch_bounds__(kCastThreads, 5) group_kernel(const __grid_con
         if (MODE == kCast) item_loop<MODE, DT>(g, g.chunks - 1 - j0, -grid, iters, p, acc, sat);
         else item_loop<MODE, DT>(g, j0, grid, iters, p, acc, sat);
         if (MODE == kCast) any_sat = any_sat || sat;
-        else leave_item<MODE>(g, gp.conv, gp.d_status, gp.d_stats, acc, sat, (unsigned)iters, guess);
+        else note_item(notes, item, g.dt, acc, sat, (unsigned)iters, guess);
     }
-    if (MODE == kCast && __syncthreads_or(any_sat) && threadIdx.x == 0) atomicOr(gp.d_status, (unsigned)FP8_FLAG_SATURATED);
+    if (MODE == kCast) {
+        if (__syncthreads_or(any_sat) && threadIdx.x == 0) atomicOr(gp.d_status, (unsigned)FP8_FLAG_SATURATED);
+    } else if ((int)threadIdx.x < gp.count) {   // note_item ended on a barrier: the notes are complete
+        publish_item<MODE>(get_item(gp, threadIdx.x), notes, threadIdx.x, gp.conv, gp.d_status, gp.d_stats);
+    }
 }
 
 static bool group_shape_ok(const fp8_group_item_t &t)
@@ -285,13 +321,15 @@ fp8_status_t fp8_cast_group(fp8_ctx *ctx, const fp8_group_item_t *items, int32_t
             g.d_bias = t.d_bias;
             ++i;
         }
-        const int64_t cap = (int64_t)ctx->sm_count * 5;   // the blocks that are resident at once (launch bounds)
-        const unsigned blocks = (unsigned)(gp.total_chunks < cap ? gp.total_chunks : cap);
+        auto grid_for = [&](int mode) {   // the blocks that are resident at once (launch bounds)
+            const int64_t cap = (int64_t)ctx->sm_count * group_blocks_per_sm(mode);
+            return (unsigned)(gp.total_chunks < cap ? gp.total_chunks : cap);
+        };
         count_launch((want_amax ? 1 : 0) + (want_cast ? 1 : 0));
         if (want_amax) {
 #define FP8LIN_FIRST(D) \
-    if (predicted) group_kernel<kBoth, D><<<blocks, kCastThreads, 0, st>>>(gp, 0); \
-    else group_kernel<kAmax, D><<<blocks, kCastThreads, 0, st>>>(gp, 0)
+    if (predicted) group_kernel<kBoth, D><<<grid_for(kBoth), kCastThreads, 0, st>>>(gp, 0); \
+    else group_kernel<kAmax, D><<<grid_for(kAmax), kCastThreads, 0, st>>>(gp, 0)
             if (dt == FP8_BF16) { FP8LIN_FIRST(FP8_BF16); }
             else if (dt == FP8_F16) { FP8LIN_FIRST(FP8_F16); }
             else { FP8LIN_FIRST(FP8_F32); }
@@ -303,7 +341,7 @@ fp8_status_t fp8_cast_group(fp8_ctx *ctx, const fp8_group_item_t *items, int32_t
         attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
         attr[0].val.programmaticStreamSerializationAllowed = 1;
         cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3(blocks);
+        cfg.gridDim = dim3(grid_for(kCast));
         cfg.blockDim = dim3(kCastThreads);
         cfg.stream = st;
         cfg.attrs = attr;

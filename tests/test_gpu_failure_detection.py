@@ -103,4 +103,9 @@ def test_launch_count_counts_what_a_call_enqueues(ctx, lib):
     x_long = torch.zeros((4, 8192), dtype=torch.uint8, device="cuda")
     out2 = torch.empty((4, 512), dtype=torch.bfloat16, device="cuda")
     assert span(lambda: ctx.linear_fwd(x_long, b, w_long, b, out2)) == 2       # two tiles, long contraction: split + finalize
+    # the CTA-pair kernel splits too when tiles are few and the contraction is very long
+    x_pair = torch.zeros((512, 16384), dtype=torch.uint8, device="cuda")
+    w_pair = torch.zeros((512, 16384), dtype=torch.uint8, device="cuda")
+    out3 = torch.empty((512, 512), dtype=torch.bfloat16, device="cuda")
+    assert span(lambda: ctx.linear_fwd(x_pair, b, w_pair, b, out3)) == 2
     torch.cuda.synchronize()

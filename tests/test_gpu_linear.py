@@ -59,6 +59,7 @@ def _layer(ctx, T, K, N, conv, seed, x_std=1.0, w_std=0.02, g_std=1e-3, margin=0
 
 
 SHAPES = [
+    (272, 8208, 304),    # few tiles of the CTA-pair kernel, long ragged contraction: sliced, partial sums, finalize
     (256, 768, 768),     # config 1
     (128, 128, 256),     # exactly one tile, one k-block
     (128, 16, 256),      # shortest contraction the API allows
@@ -256,7 +257,7 @@ def test_full_size_layers_sampled(ctx, lib, wl_name, layer):
         print(f"[parity] {wl_name}/{l.name} kind {kind}: {rows.size} positions, {frac:.5f} through the cancellation branch")
 
 
-@pytest.mark.parametrize("T,K,N", [(256, 768, 768), (400, 1040, 784), (16, 4096, 1280), (3, 16384, 272)])
+@pytest.mark.parametrize("T,K,N", [(256, 768, 768), (400, 1040, 784), (16, 4096, 1280), (3, 16384, 272), (272, 8208, 304)])
 def test_bf16_output_is_the_rounded_fp32_output(ctx, lib, T, K, N):
     """The bf16 result of a call equals the FP32 result of the same call on the same operands rounded to bf16
     (nearest even), bit for bit: the two output types differ in the last step of the epilogue only.  Covers the

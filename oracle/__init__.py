@@ -332,3 +332,52 @@ def linear_dgrad_np(dy8, s_g, w8, s_w, fg=N_E5, fw=N_E4):
 def linear_wgrad_np(dy8, s_g, x8, s_x, fg=N_E5, fx=N_E4):
     """dW = (dY8^T . X8) * 2^-(s_g+s_x)."""
     return _matmul_unscale(decode_table(fg)[_u8(dy8)].T, decode_table(fx)[_u8(x8)], int(s_g) + int(s_x))
+
+
+# ----------------------------------------------------------------------------
+# FP16 accumulation (Fig. 3b and Section 2.4)
+# ----------------------------------------------------------------------------
+# The paper's own matmul takes FP8 inputs, accumulates the partial results in FP16 and outputs FP16 (Fig. 3b);
+# Section 2.4 explains that this is where loss scaling comes back in, and Section 3.2 that the two backward matmuls
+# can overflow FP16 unless a margin lowers the bias of the E5 operand.  The paper does not say how many products
+# the hardware adds before it rounds to FP16.  Reading taken here, with the granularity an explicit argument:
+# the products of `chunk` consecutive contraction indices are summed exactly; every such partial sum is added to
+# a running FP16 accumulator with one rounding to FP16 (nearest even; beyond 65504 the accumulator becomes
+# infinite and stays so); the FP16 accumulator is then unscaled by 2^-(s_a + s_b) in FP16 (Eq. 2 on the FP16
+# output: exact unless the result leaves FP16's normal range, where it rounds once or becomes infinite / zero).
+# chunk = 1 is a purely sequential FP16 accumulation.
+
+class Fp16AccResult:
+    def __init__(self, f16):
+        self.f16 = f16                          # numpy float16: what an FP16 output tensor would hold
+        self.f64 = f16.astype(np.float64)
+        self.overflowed = ~np.isfinite(self.f64)
+
+
+def _matmul_fp16acc(A, B_t, shift_sum, chunk):
+    """A [M, Kc] and B_t [Kc, N] decoded to float64; Kc is the contraction."""
+    assert chunk >= 1
+    M, Kc = A.shape
+    acc = np.zeros((M, B_t.shape[1]), dtype=np.float16)
+    for k0 in range(0, Kc, chunk):
+        partial = A[:, k0:k0 + chunk] @ B_t[k0:k0 + chunk, :]          # exact: few terms, each a short dyadic number
+        with np.errstate(over="ignore", invalid="ignore"):
+            acc = (acc.astype(np.float64) + partial).astype(np.float16)    # one rounding to FP16 per chunk
+    with np.errstate(over="ignore", under="ignore"):
+        out = np.ldexp(acc.astype(np.float64), -int(shift_sum)).astype(np.float16)
+    return Fp16AccResult(out)
+
+
+def linear_fwd_fp16acc(x8, s_x, w8, s_w, chunk=128, fx=N_E4, fw=N_E4):
+    """Y = FP16-accumulated (X8 . W8^T), unscaled in FP16."""
+    return _matmul_fp16acc(decode_table(fx)[_u8(x8)], decode_table(fw)[_u8(w8)].T, int(s_x) + int(s_w), chunk)
+
+
+def linear_dgrad_fp16acc(dy8, s_g, w8, s_w, chunk=128, fg=N_E5, fw=N_E4):
+    """dX = FP16-accumulated (dY8 . W8), unscaled in FP16."""
+    return _matmul_fp16acc(decode_table(fg)[_u8(dy8)], decode_table(fw)[_u8(w8)], int(s_g) + int(s_w), chunk)
+
+
+def linear_wgrad_fp16acc(dy8, s_g, x8, s_x, chunk=128, fg=N_E5, fx=N_E4):
+    """dW = FP16-accumulated (dY8^T . X8), unscaled in FP16."""
+    return _matmul_fp16acc(decode_table(fg)[_u8(dy8)].T, decode_table(fx)[_u8(x8)], int(s_g) + int(s_x), chunk)

@@ -2,18 +2,18 @@
 //
 // amax is a selection, not arithmetic: on the bit patterns of bf16, fp16 and
 // fp32 alike |x| orders like the unsigned integer with the sign bit cleared,
-// with NaN > inf > finite.  For the 16-bit types the kernel keeps two lanes
-// per register (one packed max per 32-bit word); it reduces by
+// with NaN > inf > finite.  For the 16-bit types the kernels keep two lanes
+// per register (one packed max per 32-bit word); they reduce by
 // warp shuffle, then per block, then across the grid through one atomicMax per
 // block on a context-owned slot; the last block to arrive publishes the result
 // (and, when asked, the bias) and leaves the slot zeroed for the next call.
-// HBM-bound: 2 bytes read per element, nothing written.
+// HBM-bound: 2 bytes read per element, nothing written.  Contiguous tensors take
+// the streaming kernel of group.cu; this file holds the strided form.
 #include "fp8lin_internal.cuh"
 
 namespace fp8lin {
 
 constexpr int kAmaxThreads = 256;
-constexpr int kAmaxUnroll = 4;  // 16-byte loads in flight per thread
 
 struct AmaxOut {
     unsigned *slot;      // {running max, arrival counter}
@@ -81,36 +81,6 @@ __device__ __forceinline__ void amax_finish(uint32_t acc, const AmaxOut &o)
             }
         }
     }
-}
-
-// Contiguous tensor seen as nvec 16-byte vectors plus a scalar tail of ntail elements.
-template <int DT>
-__global__ void __launch_bounds__(kAmaxThreads) amax_flat_kernel(const uint4 *__restrict__ x, int64_t nvec, int ntail,
-                                                                 AmaxOut o)
-{
-    // the cast launched behind this kernel as a programmatic dependent may take its places as blocks here retire;
-    // it reads nothing before this grid has completed
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    uint32_t acc = 0;
-    const int64_t chunk = (int64_t)kAmaxThreads * kAmaxUnroll;
-    for (int64_t base = (int64_t)blockIdx.x * chunk; base < nvec; base += (int64_t)gridDim.x * chunk) {
-        uint4 v[kAmaxUnroll];
-#pragma unroll
-        for (int j = 0; j < kAmaxUnroll; ++j) {
-            int64_t i = base + threadIdx.x + (int64_t)j * kAmaxThreads;
-            v[j] = (i < nvec) ? __ldg(x + i) : make_uint4(0, 0, 0, 0);
-        }
-#pragma unroll
-        for (int j = 0; j < kAmaxUnroll; ++j) {
-            acc = fold_word<DT>(acc, v[j].x);
-            acc = fold_word<DT>(acc, v[j].y);
-            acc = fold_word<DT>(acc, v[j].z);
-            acc = fold_word<DT>(acc, v[j].w);
-        }
-    }
-    constexpr int kPerVec = DT == FP8_F32 ? 4 : 8;
-    if (blockIdx.x == 0 && (int)threadIdx.x < ntail) acc = fold_elem<DT>(acc, x, nvec * kPerVec + threadIdx.x);
-    amax_finish<DT>(acc, o);
 }
 
 // General [rows, cols] with leading dimension ld; vec != 0 promises 16-byte aligned rows.
@@ -230,38 +200,30 @@ __global__ void bias_mode_kernel(const fp8_bias_record_t *__restrict__ ring, int
 }
 
 template <int DT>
-static cudaError_t launch_amax_dt(fp8_ctx *ctx, const void *x, int64_t rows, int64_t cols, int64_t ld, AmaxOut o,
-                                  cudaStream_t stream)
+static cudaError_t launch_amax_rows(fp8_ctx *ctx, const void *x, int64_t rows, int64_t cols, int64_t ld, AmaxOut o,
+                                    cudaStream_t stream)
 {
     constexpr int kPerVec = DT == FP8_F32 ? 4 : 8;
     const bool aligned = (reinterpret_cast<uintptr_t>(x) & 15u) == 0;
-    // six blocks of 256 threads per SM: measured 6-8 % faster than eight on tensors of 180-360 MB, equal below
     const int max_blocks = ctx->sm_count * 6;
-    if (ld == cols && aligned) {
-        int64_t n = rows * cols;
-        int64_t nvec = n / kPerVec;
-        int ntail = (int)(n - nvec * kPerVec);
-        int64_t chunk = (int64_t)kAmaxThreads * kAmaxUnroll;
-        int64_t want = (nvec + chunk - 1) / chunk;
-        int blocks = (int)(want < 1 ? 1 : (want > max_blocks ? max_blocks : want));
-        count_launch();
-        amax_flat_kernel<DT><<<blocks, kAmaxThreads, 0, stream>>>(reinterpret_cast<const uint4 *>(x), nvec, ntail, o);
-    } else {
-        int vec = (aligned && (ld % kPerVec) == 0) ? 1 : 0;
-        int blocks = (int)(rows > max_blocks ? max_blocks : rows);
-        count_launch();
-        amax_rows_kernel<DT><<<blocks, kAmaxThreads, 0, stream>>>(x, rows, cols, ld, vec, o);
-    }
+    int vec = (aligned && (ld % kPerVec) == 0) ? 1 : 0;
+    int blocks = (int)(rows > max_blocks ? max_blocks : rows);
+    count_launch();
+    amax_rows_kernel<DT><<<blocks, kAmaxThreads, 0, stream>>>(x, rows, cols, ld, vec, o);
     return cudaGetLastError();
 }
 
 cudaError_t launch_amax_bias(fp8_ctx *ctx, const void *x, int dt, int64_t rows, int64_t cols, int64_t ld, float *d_amax,
                              int32_t *d_bias, int fmt, int conv, int margin, cudaStream_t stream)
 {
+    // contiguous and 16-byte aligned: the streaming kernel shared with fp8_cast_group, on one tensor
+    if (ld == cols && (reinterpret_cast<uintptr_t>(x) & 15u) == 0 &&
+        (rows * cols / 16) / 1024 < 0x7FFFFFFF)
+        return launch_amax_flat(ctx, x, dt, rows * cols, d_amax, d_bias, fmt, conv, margin, stream);
     AmaxOut o{take_slot(ctx), d_amax, d_bias, ctx->d_status, fmt, conv, margin};
-    if (dt == FP8_BF16) return launch_amax_dt<FP8_BF16>(ctx, x, rows, cols, ld, o, stream);
-    if (dt == FP8_F16) return launch_amax_dt<FP8_F16>(ctx, x, rows, cols, ld, o, stream);
-    return launch_amax_dt<FP8_F32>(ctx, x, rows, cols, ld, o, stream);
+    if (dt == FP8_BF16) return launch_amax_rows<FP8_BF16>(ctx, x, rows, cols, ld, o, stream);
+    if (dt == FP8_F16) return launch_amax_rows<FP8_F16>(ctx, x, rows, cols, ld, o, stream);
+    return launch_amax_rows<FP8_F32>(ctx, x, rows, cols, ld, o, stream);
 }
 
 }  // namespace fp8lin

@@ -7,79 +7,20 @@
 // either way) and the rounding is one hardware cvt.rn.satfinite per pair.
 //
 // Kernels, all HBM-bound (2 B read per 16-bit element + 1 B written per element and layout):
-//   cast_flat_kernel       contiguous tensor, row-major output; 16 elements per thread per step.
+//   (group.cu)             contiguous tensor, row-major output: the streaming kernels shared with
+//                          fp8_cast_group -- cast, amax + cast in one pass (fp8_cast_predicted, delayed scaling).
 //   cast_tile_kernel       128x128 tiles, optional row-major output and optional transposed output
 //                          staged through shared memory so that both are written in 128-byte rows;
 //                          also the guarded path for ragged or strided tensors.
-//   cast_predicted_kernel  the flat cast with the amax of the same pass: FP8-AMAX in one pass when
-//                          the bias guess holds (fp8_cast_predicted), and delayed scaling.
 //   cast_small_kernel      decode-size tensors: one cluster keeps the tensor in registers between
 //                          its amax and its cast, one launch.
-// The flat and tile kernels walk the tensor from its end to its start: when the amax pass has just
-// streamed it front to back, the part most recently read is the part most likely still in L2.
+// The cast kernels walk the tensor from its end to its start: when the amax pass has just streamed
+// it front to back, the part most recently read is the part most likely still in L2.
 #include <cstdlib>
 
 #include "cast_common.cuh"
 
 namespace fp8lin {
-
-// ---------------------------------------------------------------------------
-// contiguous, row-major output only
-// ---------------------------------------------------------------------------
-
-template <int FMT, int DT, bool TWO_STEP>
-__device__ __forceinline__ void cast_flat_body(const uint4 *__restrict__ x, uint4 *__restrict__ y, int64_t nout,
-                                               Pow2Pair p, bool &sat)
-{
-    // nout = number of 16-byte output vectors; each consumes kIn input vectors (16 elements).
-    constexpr int kIn = InType<DT>::kBytes;  // 2 vectors of 16-bit elements, 4 of fp32
-    const int64_t chunk = (int64_t)blockDim.x * 2;
-    const int64_t nchunks = (nout + chunk - 1) / chunk;
-    for (int64_t c = nchunks - 1 - blockIdx.x; c >= 0; c -= gridDim.x) {
-        int64_t idx[2] = {c * chunk + threadIdx.x, c * chunk + threadIdx.x + blockDim.x};
-        uint4 v[2][kIn];
-#pragma unroll
-        for (int u = 0; u < 2; ++u)
-            if (idx[u] < nout) {
-#pragma unroll
-                for (int j = 0; j < kIn; ++j) v[u][j] = __ldcs(x + kIn * idx[u] + j);
-            }
-#pragma unroll
-        for (int u = 0; u < 2; ++u)
-            if (idx[u] < nout) {
-                const uint32_t *w = reinterpret_cast<const uint32_t *>(&v[u][0]);
-                constexpr int kW = InType<DT>::kWords4;
-                uint4 o;
-                o.x = cast4w<FMT, DT, TWO_STEP>(w + 0 * kW, p, sat);
-                o.y = cast4w<FMT, DT, TWO_STEP>(w + 1 * kW, p, sat);
-                o.z = cast4w<FMT, DT, TWO_STEP>(w + 2 * kW, p, sat);
-                o.w = cast4w<FMT, DT, TWO_STEP>(w + 3 * kW, p, sat);
-                y[idx[u]] = o;
-            }
-    }
-}
-
-template <int FMT, int DT>
-__global__ void __launch_bounds__(1024) cast_flat_kernel(const uint4 *__restrict__ x, uint4 *__restrict__ y,
-                                                                 int64_t nout, int ntail,
-                                                                 const int32_t *__restrict__ d_bias, int delta,
-                                                                 unsigned *d_status, const unsigned *redo)
-{
-    // launched as a programmatic dependent of the amax kernel: nothing it wrote is read before it has completed;
-    // the matmul behind this kernel may in turn take its places as blocks here retire
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    asm volatile("griddepcontrol.wait;" ::: "memory");
-    // as the second launch of a predicted cast: nothing to do when the prediction held
-    if (redo != nullptr && *reinterpret_cast<const volatile unsigned *>(redo) == 0u) return;
-    const int s = __ldg(d_bias) + delta;
-    const Pow2Pair p = make_pow2_pair(s);
-    bool sat = false;
-    if (s >= -126 && s <= 127) cast_flat_body<FMT, DT, false>(x, y, nout, p, sat);
-    else cast_flat_body<FMT, DT, true>(x, y, nout, p, sat);
-    if (blockIdx.x == 0 && (int)threadIdx.x < ntail)
-        reinterpret_cast<uint8_t *>(y)[nout * 16 + threadIdx.x] = cast1<FMT, DT, true>(x, nout * 16 + threadIdx.x, p, sat);
-    if (__syncthreads_or(sat) && threadIdx.x == 0) atomicOr(d_status, FP8_FLAG_SATURATED);
-}
 
 // ---------------------------------------------------------------------------
 // tiled, with optional transposed output
@@ -183,18 +124,8 @@ static cudaError_t launch_cast(fp8_ctx *ctx, const void *x, int64_t rows, int64_
 {
     auto al = [](const void *p, unsigned a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; };
     constexpr int kB = InType<DT>::kBytes;
-    if (!y_t && ld == cols && al(x, 16) && al(y, 16)) {
-        int64_t n = rows * cols;
-        int64_t nout = n / 16;
-        int ntail = (int)(n - nout * 16);
-        int64_t chunk = (int64_t)kCastThreads * 2;
-        int64_t want = (nout + chunk - 1) / chunk;
-        int max_blocks = ctx->sm_count * 8;
-        int blocks = (int)(want < 1 ? 1 : (want > max_blocks ? max_blocks : want));
-        return launch_dependent(cast_flat_kernel<FMT, DT>, blocks, kCastThreads, stream, reinterpret_cast<const uint4 *>(x),
-                                reinterpret_cast<uint4 *>(y), nout, ntail, d_bias, delta, ctx->d_status,
-                                static_cast<const unsigned *>(nullptr));
-    }
+    if (!y_t && ld == cols && al(x, 16) && al(y, 16))   // the streaming kernel shared with fp8_cast_group, on one tensor
+        return launch_cast_flat(ctx, x, DT, rows * cols, d_bias, FMT, delta, y, stream);
     int fast_ok = al(x, 4 * kB) && (ld % 4) == 0 && (!y || (al(y, 4) && (cols % 4) == 0)) &&
                   (!y_t || (al(y_t, 4) && (rows % 4) == 0));
     int64_t tiles = ((rows + kTile - 1) / kTile) * ((cols + kTile - 1) / kTile);
@@ -226,110 +157,12 @@ static cudaError_t launch_cast_dt(int dt, fp8_ctx *ctx, const void *x, int64_t r
 // Traffic: 2 B read + 1 B written per element when the guess holds, twice that when it does not.
 
 template <int FMT, int DT>
-__global__ void __launch_bounds__(kCastThreads)
-cast_predicted_kernel(const uint4 *__restrict__ x, uint4 *__restrict__ y, int64_t nout, int ntail, int fmt, int conv,
-                      int margin, int delta, unsigned *slot, float *d_amax, const int32_t *d_bias_in,
-                      int32_t *d_bias_out, int verify, unsigned *d_status, unsigned *d_stats)
-{
-    // verify != 0: d_bias_in is a guess to be checked (fp8_cast_predicted).  verify == 0: d_bias_in is the bias to
-    // use, full stop, and the amax / bias of this tensor are by-products for the next step (delayed scaling).
-    constexpr int kIn = InType<DT>::kBytes;
-    constexpr int kW = InType<DT>::kWords4;
-    const int guess = *reinterpret_cast<const volatile int32_t *>(d_bias_in);
-    const Pow2Pair p = make_pow2_pair(guess + delta);
-    bool sat = false;
-    uint32_t acc = 0;
-    const int64_t chunk = (int64_t)kCastThreads * 2;
-    const int64_t nchunks = (nout + chunk - 1) / chunk;
-    for (int64_t c = blockIdx.x; c < nchunks; c += gridDim.x) {
-        int64_t idx[2] = {c * chunk + threadIdx.x, c * chunk + threadIdx.x + kCastThreads};
-        uint4 v[2][kIn];
-#pragma unroll
-        for (int u = 0; u < 2; ++u)
-            if (idx[u] < nout) {
-#pragma unroll
-                for (int j = 0; j < kIn; ++j) v[u][j] = __ldcs(x + kIn * idx[u] + j);
-            }
-#pragma unroll
-        for (int u = 0; u < 2; ++u)
-            if (idx[u] < nout) {
-                const uint32_t *w = reinterpret_cast<const uint32_t *>(&v[u][0]);
-#pragma unroll
-                for (int j = 0; j < 4 * kIn; ++j)
-                    acc = DT == FP8_F32 ? max(acc, w[j] & 0x7FFFFFFFu) : __vmaxu2(acc, w[j] & 0x7FFF7FFFu);
-                uint4 o;
-                o.x = cast4w<FMT, DT, true>(w + 0 * kW, p, sat);
-                o.y = cast4w<FMT, DT, true>(w + 1 * kW, p, sat);
-                o.z = cast4w<FMT, DT, true>(w + 2 * kW, p, sat);
-                o.w = cast4w<FMT, DT, true>(w + 3 * kW, p, sat);
-                y[idx[u]] = o;
-            }
-    }
-    if (blockIdx.x == 0 && (int)threadIdx.x < ntail) {
-        const int64_t i = nout * 16 + threadIdx.x;
-        if (DT == FP8_F32) acc = max(acc, reinterpret_cast<const uint32_t *>(x)[i] & 0x7FFFFFFFu);
-        else acc = __vmaxu2(acc, (uint32_t)reinterpret_cast<const uint16_t *>(x)[i] & 0x7FFFu);
-        reinterpret_cast<uint8_t *>(y)[i] = cast1<FMT, DT, true>(x, i, p, sat);
-    }
-    // grid-wide max; the last block compares the true bias with the guess
-    __shared__ uint32_t warp_max[kCastThreads / 32];
-    uint32_t m = DT == FP8_F32 ? acc : max(acc & 0xFFFFu, acc >> 16);
-    m = __reduce_max_sync(0xFFFFFFFFu, m);
-    if ((threadIdx.x & 31) == 0) warp_max[threadIdx.x >> 5] = m;
-    const int any_sat = __syncthreads_or(sat);
-    if (threadIdx.x == 0) {
-        for (int i = 1; i < kCastThreads / 32; ++i) m = max(m, warp_max[i]);
-        atomicMax(&slot[0], m);
-        if (any_sat) atomicOr(&slot[2], 1u);
-        __threadfence();
-        if (atomicAdd(&slot[1], 1u) + 1u == gridDim.x) {
-            __threadfence();
-            const uint32_t total = atomicExch(&slot[0], 0u);
-            const unsigned was_sat = atomicExch(&slot[2], 0u);
-            slot[1] = 0u;
-            uint32_t fbits;
-            if (DT == FP8_F32) fbits = total;
-            else if (DT == FP8_BF16) fbits = total << 16;
-            else { float f; asm("cvt.f32.f16 %0, %1;" : "=f"(f) : "h"((uint16_t)total)); fbits = __float_as_uint(f); }
-            *d_amax = __uint_as_float(fbits);
-            unsigned flags = 0;
-            const int b = bias_from_amax_bits(fbits, fmt, conv, margin, &flags);
-            const bool hit = (b == guess) || !verify;
-            *d_bias_out = b;
-            slot[3] = hit ? 0u : 1u;               // read by the gated second launch
-            if (verify) atomicAdd(&d_stats[hit ? 0 : 1], 1u);
-            if (hit && was_sat) flags |= FP8_FLAG_SATURATED;   // clipping under a wrong guess says nothing
-            if (flags) atomicOr(d_status, flags);
-        }
-    }
-}
-
-template <int FMT, int DT>
 static cudaError_t launch_predicted(fp8_ctx *ctx, const void *x, int64_t n, int conv, int margin, float *d_amax,
                                     const int32_t *d_bias_in, int32_t *d_bias_inout, int verify, uint8_t *y,
                                     cudaStream_t stream)
 {
-    int64_t nout = n / 16;
-    int ntail = (int)(n - nout * 16);
-    int64_t chunk = (int64_t)kCastThreads * 2;
-    int64_t want = (nout + chunk - 1) / chunk;
-    int max_blocks = ctx->sm_count * 8;
-    int blocks = (int)(want < 1 ? 1 : (want > max_blocks ? max_blocks : want));
-    unsigned *slot = take_slot(ctx);
-    const int delta = format_delta(FMT, conv);
-    count_launch(verify ? 2 : 1);  // this kernel and, when the guess is verified, the gated second pass below
-    cast_predicted_kernel<FMT, DT><<<blocks, kCastThreads, 0, stream>>>(
-        reinterpret_cast<const uint4 *>(x), reinterpret_cast<uint4 *>(y), nout, ntail, FMT, conv, margin, delta, slot,
-        d_amax, d_bias_in, d_bias_inout, verify, ctx->d_status, ctx->d_predict_stats);
-    if (cudaGetLastError() != cudaSuccess) return cudaErrorUnknown;
-    if (!verify) return cudaSuccess;
-    // the gated second launch: few, large blocks (same threads per SM), so that it costs little when it has nothing to do
-    int64_t want2 = (nout + 2047) / 2048;
-    int blocks2 = (int)(want2 < 1 ? 1 : (want2 > 2 * ctx->sm_count ? 2 * ctx->sm_count : want2));
-    cast_flat_kernel<FMT, DT><<<blocks2, 1024, 0, stream>>>(reinterpret_cast<const uint4 *>(x),
-                                                            reinterpret_cast<uint4 *>(y), nout, ntail, d_bias_inout,
-                                                            delta, ctx->d_status, slot + 3);
-    return cudaGetLastError();
+    // the one-pass kernel of group.cu on one tensor, followed (when the guess is verified) by the gated cast pass
+    return launch_one_pass_flat(ctx, x, DT, n, FMT, conv, margin, d_amax, d_bias_in, d_bias_inout, verify, y, stream);
 }
 
 // ---------------------------------------------------------------------------

@@ -108,6 +108,15 @@ inline cudaError_t launch_dependent(void (*kernel)(KArgs...), unsigned grid, uns
 cudaError_t launch_amax_bias(fp8_ctx *ctx, const void *x, int dt, int64_t rows, int64_t cols, int64_t ld, float *d_amax,
                              int32_t *d_bias, int fmt, int conv, int margin, cudaStream_t stream);
 
+// group.cu: the streaming kernels of fp8_cast_group applied to one contiguous, 16-byte aligned tensor of n elements
+cudaError_t launch_amax_flat(fp8_ctx *ctx, const void *x, int dt, int64_t n, float *d_amax, int32_t *d_bias, int fmt,
+                             int conv, int margin, cudaStream_t st);
+cudaError_t launch_cast_flat(fp8_ctx *ctx, const void *x, int dt, int64_t n, const int32_t *d_bias, int fmt, int delta,
+                             uint8_t *y, cudaStream_t st);
+cudaError_t launch_one_pass_flat(fp8_ctx *ctx, const void *x, int dt, int64_t n, int fmt, int conv, int margin,
+                                 float *d_amax, const int32_t *d_bias_in, int32_t *d_bias_out, int verify, uint8_t *y,
+                                 cudaStream_t st);
+
 }  // namespace fp8lin
 
 // ---------------------------------------------------------------------------

@@ -26,9 +26,19 @@ constexpr int kGroupMax = FP8_GROUP_MAX;
 // (eight 16-byte loads in flight per thread), three resident blocks per SM for the read-only pass and two for the
 // passes that also write, streaming stores: amax 7.0 TB/s, cast 6.7 TB/s, one pass 6.3 TB/s.  More blocks per SM
 // cost the writing passes up to a third of their bandwidth (5 per SM: 5.8 TB/s).
-constexpr int kUnroll = 4;                               // 16-byte output vectors per thread and chunk
-__host__ __device__ constexpr int group_blocks_per_sm(int mode) { return mode == 0 ? 3 : 2; }
-constexpr int kChunkOut = kUnroll * kCastThreads;       // 16-byte output vectors per chunk
+// (FP32 inputs bring twice the bytes per output vector: two output vectors per thread keep them in registers.)
+#ifndef FP8LIN_GROUP_UNROLL
+#define FP8LIN_GROUP_UNROLL 4
+#endif
+#ifndef FP8LIN_GROUP_AMAX_BLOCKS
+#define FP8LIN_GROUP_AMAX_BLOCKS 3
+#endif
+#ifndef FP8LIN_GROUP_CAST_BLOCKS
+#define FP8LIN_GROUP_CAST_BLOCKS 2
+#endif
+__host__ __device__ constexpr int group_unroll(int dt) { return dt == FP8_F32 ? 2 : FP8LIN_GROUP_UNROLL; }   // output vectors per thread and chunk
+__host__ __device__ constexpr int group_blocks_per_sm(int mode) { return mode == 0 ? FP8LIN_GROUP_AMAX_BLOCKS : FP8LIN_GROUP_CAST_BLOCKS; }
+__host__ __device__ constexpr int group_chunk_out(int dt) { return group_unroll(dt) * kCastThreads; }   // output vectors per chunk
 
 struct GroupItem {
     const uint4 *x;
@@ -39,11 +49,13 @@ struct GroupItem {
     int dt, fmt, margin, delta;
     unsigned *slot;        // {running max, chunks done, saturation seen, redo}
     float *d_amax;
-    int32_t *d_bias;
+    const int32_t *d_bias_in;   // the bias a casting pass applies (a guess, in the one-pass mode)
+    int32_t *d_bias;            // where the amax passes write the Eq. 3 bias (may be NULL: amax only)
 };
 
 struct GroupParams {
     int count, conv;
+    int verify;            // one-pass mode: the given bias is a guess to be checked (else it is simply the bias to use)
     int64_t total_chunks;
     unsigned *d_status, *d_stats;
     GroupItem it[kGroupMax];
@@ -56,13 +68,15 @@ __device__ __forceinline__ uint32_t fold_any(int dt, uint32_t acc, uint32_t w)
     return dt == FP8_F32 ? max(acc, w & 0x7FFFFFFFu) : __vmaxu2(acc, w & 0x7FFF7FFFu);
 }
 
-// One chunk of one tensor: thread t owns output vectors c * kChunkOut + t + u * 256, u < kUnroll.
+// One chunk of one tensor: thread t owns output vectors c * chunk + t + u * 256, u < group_unroll(DT).
 template <int MODE, int FMT, int DT, bool TWO_STEP>
 __device__ __forceinline__ void chunk_body(const uint4 *__restrict__ gx, uint4 *__restrict__ gy, int64_t n, int64_t c,
                                            Pow2Pair p, uint32_t &acc, bool &sat)
 {
     constexpr int kIn = InType<DT>::kBytes;   // input vectors per output vector
     constexpr int kW = InType<DT>::kWords4;
+    constexpr int kUnroll = group_unroll(DT);
+    constexpr int kChunkOut = group_chunk_out(DT);
     const int64_t nout = n / 16;
     int64_t idx[kUnroll];
 #pragma unroll
@@ -150,7 +164,7 @@ __device__ __forceinline__ void note_item(BlockNotes &notes, int item, int dt, u
 // the block pays one round trip to the atomics and not one per tensor); the thread that completes a tensor's chunk
 // count publishes its amax and bias and, in the predicted mode, the verdict on the guess.
 template <int MODE>
-__device__ __forceinline__ void publish_item(const GroupItem &g, const BlockNotes &notes, int item, int conv,
+__device__ __forceinline__ void publish_item(const GroupItem &g, const BlockNotes &notes, int item, int conv, int verify,
                                              unsigned *d_status, unsigned *d_stats)
 {
     const unsigned done = notes.done[item];
@@ -170,11 +184,12 @@ __device__ __forceinline__ void publish_item(const GroupItem &g, const BlockNote
     *g.d_amax = __uint_as_float(fbits);
     unsigned flags = 0;
     const int b = bias_from_amax_bits(fbits, g.fmt, conv, g.margin, &flags);
+    if (g.d_bias == nullptr) return;   // amax alone was asked for: no bias, no flags
     *g.d_bias = b;
     if (MODE == kBoth) {
-        const bool hit = b == notes.guess[item];
+        const bool hit = b == notes.guess[item] || !verify;
         g.slot[3] = hit ? 0u : 1u;   // read by the gated second launch
-        atomicAdd(&d_stats[hit ? 0 : 1], 1u);
+        if (verify) atomicAdd(&d_stats[hit ? 0 : 1], 1u);
         if (hit && was_sat) flags |= FP8_FLAG_SATURATED;   // clipping under a wrong guess says nothing
     }
     if (flags) atomicOr(d_status, flags);
@@ -225,7 +240,7 @@ __global__ void __launch_bounds__(kCastThreads, group_blocks_per_sm(MODE)) group
         Pow2Pair p = make_pow2_pair(0);
         if (MODE != kAmax) {
             if (MODE == kCast && gate && *reinterpret_cast<const volatile unsigned *>(&g.slot[3]) == 0u) continue;
-            guess = *reinterpret_cast<const volatile int32_t *>(g.d_bias);
+            guess = *reinterpret_cast<const volatile int32_t *>(g.d_bias_in);
             p = make_pow2_pair(guess + g.delta);
         }
         uint32_t acc = 0;
@@ -238,8 +253,97 @@ __global__ void __launch_bounds__(kCastThreads, group_blocks_per_sm(MODE)) group
     if (MODE == kCast) {
         if (__syncthreads_or(any_sat) && threadIdx.x == 0) atomicOr(gp.d_status, (unsigned)FP8_FLAG_SATURATED);
     } else if ((int)threadIdx.x < gp.count) {   // note_item ended on a barrier: the notes are complete
-        publish_item<MODE>(get_item(gp, threadIdx.x), notes, threadIdx.x, gp.conv, gp.d_status, gp.d_stats);
+        publish_item<MODE>(get_item(gp, threadIdx.x), notes, threadIdx.x, gp.conv, gp.verify, gp.d_status, gp.d_stats);
     }
+}
+
+// One pass over up to kGroupMax tensors of one input type.  `first`: kAmax, kBoth or kCast launched as an ordinary
+// kernel; a kCast pass behind another pass of the same call is launched as its programmatic dependent.
+static cudaError_t launch_pass(fp8_ctx *ctx, const GroupParams &gp, int dt, int mode, int gate, bool dependent, cudaStream_t st)
+{
+    const int64_t cap = (int64_t)ctx->sm_count * group_blocks_per_sm(mode);   // the blocks resident at once (launch bounds)
+    const unsigned blocks = (unsigned)(gp.total_chunks < cap ? gp.total_chunks : cap);
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(blocks);
+    cfg.blockDim = dim3(kCastThreads);
+    cfg.stream = st;
+    cfg.attrs = attr;
+    cfg.numAttrs = dependent ? 1 : 0;
+    count_launch();
+#define FP8LIN_PASS(M) \
+    (dt == FP8_BF16  ? cudaLaunchKernelEx(&cfg, group_kernel<M, FP8_BF16>, gp, gate) \
+     : dt == FP8_F16 ? cudaLaunchKernelEx(&cfg, group_kernel<M, FP8_F16>, gp, gate) \
+                     : cudaLaunchKernelEx(&cfg, group_kernel<M, FP8_F32>, gp, gate))
+    if (mode == kAmax) return FP8LIN_PASS(kAmax);
+    if (mode == kBoth) return FP8LIN_PASS(kBoth);
+    return FP8LIN_PASS(kCast);
+#undef FP8LIN_PASS
+}
+
+static void add_item(fp8_ctx *ctx, GroupParams &gp, const void *x, void *y, int64_t n, int dt, int fmt, int margin, int conv,
+                     float *d_amax, const int32_t *d_bias_in, int32_t *d_bias_out)
+{
+    GroupItem &g = gp.it[gp.count++];
+    g.x = reinterpret_cast<const uint4 *>(x);
+    g.y = reinterpret_cast<uint4 *>(y);
+    g.n = n;
+    g.first_chunk = gp.total_chunks;
+    g.chunks = (n / 16 + group_chunk_out(dt) - 1) / group_chunk_out(dt);
+    if (g.chunks < 1) g.chunks = 1;
+    gp.total_chunks += g.chunks;
+    g.dt = dt;
+    g.fmt = fmt;
+    g.margin = margin;
+    g.delta = format_delta(fmt, conv);
+    g.slot = take_slot(ctx);
+    g.d_amax = d_amax;
+    g.d_bias_in = d_bias_in;
+    g.d_bias = d_bias_out;
+}
+
+static GroupParams empty_group(fp8_ctx *ctx, int conv, int verify)
+{
+    GroupParams gp;
+    gp.count = 0;
+    gp.conv = conv;
+    gp.verify = verify;
+    gp.total_chunks = 0;
+    gp.d_status = ctx->d_status;
+    gp.d_stats = ctx->d_predict_stats;
+    return gp;
+}
+
+// The same kernels for ONE contiguous, 16-byte aligned tensor (the single-tensor entry points route here).
+cudaError_t launch_amax_flat(fp8_ctx *ctx, const void *x, int dt, int64_t n, float *d_amax, int32_t *d_bias, int fmt,
+                             int conv, int margin, cudaStream_t st)
+{
+    GroupParams gp = empty_group(ctx, conv, 0);
+    add_item(ctx, gp, x, nullptr, n, dt, fmt, margin, conv, d_amax, d_bias, d_bias);
+    return launch_pass(ctx, gp, dt, kAmax, 0, false, st);
+}
+
+cudaError_t launch_cast_flat(fp8_ctx *ctx, const void *x, int dt, int64_t n, const int32_t *d_bias, int fmt, int delta,
+                             uint8_t *y, cudaStream_t st)
+{
+    GroupParams gp = empty_group(ctx, FP8_CONV_PAPER, 0);
+    add_item(ctx, gp, x, y, n, dt, fmt, 0, FP8_CONV_PAPER, nullptr, d_bias, nullptr);
+    gp.it[0].delta = delta;   // the format shift comes from the caller; a cast pass needs nothing else of the convention
+    return launch_pass(ctx, gp, dt, kCast, 0, true, st);   // may follow an amax pass as its programmatic dependent
+}
+
+cudaError_t launch_one_pass_flat(fp8_ctx *ctx, const void *x, int dt, int64_t n, int fmt, int conv, int margin,
+                                 float *d_amax, const int32_t *d_bias_in, int32_t *d_bias_out, int verify, uint8_t *y,
+                                 cudaStream_t st)
+{
+    GroupParams gp = empty_group(ctx, conv, verify);
+    add_item(ctx, gp, x, y, n, dt, fmt, margin, conv, d_amax, d_bias_in, d_bias_out);
+    cudaError_t e = launch_pass(ctx, gp, dt, kBoth, 0, false, st);
+    if (e != cudaSuccess || !verify) return e;
+    gp.it[0].d_bias_in = d_bias_out;   // the redo, if any, uses the bias the first pass published
+    return launch_pass(ctx, gp, dt, kCast, 1, true, st);
 }
 
 static bool group_shape_ok(const fp8_group_item_t &t)
@@ -280,7 +384,7 @@ fp8_status_t fp8_cast_group(fp8_ctx *ctx, const fp8_group_item_t *items, int32_t
                                        stream);
             } else if (mode == FP8_GROUP_AMAX_ONLY) {
                 s = launch_amax_bias(ctx, t.x, (int)t.x_dt, t.rows, t.cols, t.ld, t.d_amax, t.d_bias, (int)t.fmt, (int)conv,
-                                     t.margin, (cudaStream_t)stream) == cudaSuccess ? FP8_OK : FP8_ERR_CUDA;
+                                     t.margin, st) == cudaSuccess ? FP8_OK : FP8_ERR_CUDA;
             } else {
                 const int32_t *given = mode == FP8_GROUP_CAST_ONLY ? t.d_bias : nullptr;
                 float *ao = given ? nullptr : t.d_amax;
@@ -294,63 +398,16 @@ fp8_status_t fp8_cast_group(fp8_ctx *ctx, const fp8_group_item_t *items, int32_t
             ++i;
             continue;
         }
-        GroupParams gp;
-        gp.count = 0;
-        gp.conv = (int)conv;
-        gp.total_chunks = 0;
-        gp.d_status = ctx->d_status;
-        gp.d_stats = ctx->d_predict_stats;
+        GroupParams gp = empty_group(ctx, (int)conv, predicted ? 1 : 0);
         const int dt = (int)items[i].x_dt;   // one input type per pair of launches
         while (i < count && gp.count < kGroupMax && group_shape_ok(items[i]) && (int)items[i].x_dt == dt) {
             const fp8_group_item_t &t = items[i];
-            GroupItem &g = gp.it[gp.count++];
-            g.x = reinterpret_cast<const uint4 *>(t.x);
-            g.y = reinterpret_cast<uint4 *>(t.y);
-            g.n = t.rows * t.cols;
-            g.first_chunk = gp.total_chunks;
-            g.chunks = (g.n / 16 + kChunkOut - 1) / kChunkOut;
-            if (g.chunks < 1) g.chunks = 1;
-            if (g.chunks > 0x7FFFFFFF) return FP8_ERR_SHAPE;
-            gp.total_chunks += g.chunks;
-            g.dt = (int)t.x_dt;
-            g.fmt = (int)t.fmt;
-            g.margin = t.margin;
-            g.delta = format_delta((int)t.fmt, (int)conv);
-            g.slot = take_slot(ctx);
-            g.d_amax = t.d_amax;
-            g.d_bias = t.d_bias;
+            if ((t.rows * t.cols / 16 + group_chunk_out(dt) - 1) / group_chunk_out(dt) > 0x7FFFFFFF) return FP8_ERR_SHAPE;
+            add_item(ctx, gp, t.x, t.y, t.rows * t.cols, dt, (int)t.fmt, t.margin, (int)conv, t.d_amax, t.d_bias, t.d_bias);
             ++i;
         }
-        auto grid_for = [&](int mode) {   // the blocks that are resident at once (launch bounds)
-            const int64_t cap = (int64_t)ctx->sm_count * group_blocks_per_sm(mode);
-            return (unsigned)(gp.total_chunks < cap ? gp.total_chunks : cap);
-        };
-        count_launch((want_amax ? 1 : 0) + (want_cast ? 1 : 0));
-        if (want_amax) {
-#define FP8LIN_FIRST(D) \
-    if (predicted) group_kernel<kBoth, D><<<grid_for(kBoth), kCastThreads, 0, st>>>(gp, 0); \
-    else group_kernel<kAmax, D><<<grid_for(kAmax), kCastThreads, 0, st>>>(gp, 0)
-            if (dt == FP8_BF16) { FP8LIN_FIRST(FP8_BF16); }
-            else if (dt == FP8_F16) { FP8LIN_FIRST(FP8_F16); }
-            else { FP8LIN_FIRST(FP8_F32); }
-#undef FP8LIN_FIRST
-            if (cudaGetLastError() != cudaSuccess) return FP8_ERR_CUDA;
-        }
-        if (!want_cast) continue;
-        cudaLaunchAttribute attr[1];
-        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        attr[0].val.programmaticStreamSerializationAllowed = 1;
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3(grid_for(kCast));
-        cfg.blockDim = dim3(kCastThreads);
-        cfg.stream = st;
-        cfg.attrs = attr;
-        cfg.numAttrs = 1;
-        const int gate = predicted ? 1 : 0;
-        cudaError_t le = dt == FP8_BF16  ? cudaLaunchKernelEx(&cfg, group_kernel<kCast, FP8_BF16>, gp, gate)
-                         : dt == FP8_F16 ? cudaLaunchKernelEx(&cfg, group_kernel<kCast, FP8_F16>, gp, gate)
-                                         : cudaLaunchKernelEx(&cfg, group_kernel<kCast, FP8_F32>, gp, gate);
-        if (le != cudaSuccess) return FP8_ERR_CUDA;
+        if (want_amax && launch_pass(ctx, gp, dt, predicted ? kBoth : kAmax, 0, false, st) != cudaSuccess) return FP8_ERR_CUDA;
+        if (want_cast && launch_pass(ctx, gp, dt, kCast, predicted ? 1 : 0, true, st) != cudaSuccess) return FP8_ERR_CUDA;
     }
     return FP8_OK;
 }

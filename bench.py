@@ -51,8 +51,8 @@ ORACLE_SAMPLE_LAYER = 1  # the square attention-output projection
 NOMINAL_FP8_TFLOPS = 4500.0         # dense FP8, the vendor's figure for the part
 FP8_FLOP_PER_CLK_PER_SM = 16384.0   # 8192 multiply-adds per clock per SM: nominal peak / (148 SMs x 1.856 GHz)
 # dram__bytes_read.sum + dram__bytes_write.sum per matmul launch, from one ncu capture of one step of the
-# workload (profiles/gemm_pair_kernel.md, table (c)); keyed by (workload, tokens)
-GEMM_DRAM_BYTES_PER_LAUNCH = {("c3_llama7b", 8192): 371.8e6}
+# workload (profiles/launch_list_c3_llama7b.md, second table); keyed by (workload, tokens)
+GEMM_DRAM_BYTES_PER_LAUNCH = {("c3_llama7b", 8192): 383.5e6}
 
 
 def load_peaks():

@@ -222,12 +222,20 @@ __global__ void __launch_bounds__(kCastThreads, group_blocks_per_sm(MODE)) group
     const int64_t grid = gridDim.x, b = blockIdx.x;
     bool any_sat = false;
     __shared__ BlockNotes notes;
-    if (MODE != kCast) {
-        if (threadIdx.x < kGroupMax) notes.done[threadIdx.x] = 0u;
-        __syncthreads();
+    // the bias every tensor is cast with and, for the gated pass, its redo flag: fetched by one thread per tensor at
+    // once (a block that fetched them tensor by tensor would pay one trip to L2 per tensor before touching its data)
+    __shared__ int given_bias[kGroupMax];
+    __shared__ unsigned redo[kGroupMax];
+    if ((int)threadIdx.x < gp.count) {
+        const GroupItem g = get_item(gp, threadIdx.x);
+        notes.done[threadIdx.x] = 0u;
+        if (MODE != kAmax) given_bias[threadIdx.x] = *reinterpret_cast<const volatile int32_t *>(g.d_bias_in);
+        if (MODE == kCast) redo[threadIdx.x] = gate ? *reinterpret_cast<const volatile unsigned *>(&g.slot[3]) : 1u;
     }
+    __syncthreads();
     for (int n = 0; n < gp.count; ++n) {
         const int item = MODE == kCast ? gp.count - 1 - n : n;
+        if (MODE == kCast && redo[item] == 0u) continue;
         const GroupItem g = get_item(gp, item);
         // sequence numbers of this tensor's chunks: [lo, lo + chunks); number lo + j is tensor-local chunk j in the
         // forward passes and chunk (chunks - 1 - j) in the backward pass
@@ -239,8 +247,7 @@ __global__ void __launch_bounds__(kCastThreads, group_blocks_per_sm(MODE)) group
         int guess = 0;
         Pow2Pair p = make_pow2_pair(0);
         if (MODE != kAmax) {
-            if (MODE == kCast && gate && *reinterpret_cast<const volatile unsigned *>(&g.slot[3]) == 0u) continue;
-            guess = *reinterpret_cast<const volatile int32_t *>(g.d_bias_in);
+            guess = given_bias[item];
             p = make_pow2_pair(guess + g.delta);
         }
         uint32_t acc = 0;

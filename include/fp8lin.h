@@ -433,6 +433,26 @@ FP8_API fp8_status_t fp8_linear_wgrad(fp8_ctx *ctx, const uint8_t *dy8, const ui
                               const uint8_t *x8, const uint8_t *x8_t, const int32_t *d_bx, void *dw,
                               fp8_dtype_t dw_dt, int64_t T, int64_t K, int64_t N, fp8_conv_t conv, void *stream);
 
+/* The paper's own accumulation regime, emulated (Fig. 3b: FP8 inputs, partial results accumulated in FP16, FP16
+ * output; Section 2.4: why loss scaling returns with FP16 accumulation; Section 3.2: the margin that keeps the two
+ * backward matmuls from overflowing FP16).  The paper does not say how many products its hardware adds before it
+ * rounds; here the granularity is the argument `chunk`: the products of `chunk` consecutive contraction indices
+ * (a multiple of 128) are accumulated on the tensor cores in FP32 -- exact to 2^-21 of their absolute sum -- each such
+ * partial sum is added to a running FP16 accumulator with one rounding to FP16 (beyond 65504 it becomes infinite and
+ * stays so), and the FP16 result is unscaled in FP16 (Eq. 2 applied to the FP16 output: one more rounding only where
+ * the result leaves FP16's normal range).  For studying margins and loss scales, not for speed (an eighth of the plain
+ * matmul's rate at chunk = 128, two thirds at chunk = 2048).  Operands in their forward layouts:
+ *   FP8_MM_FWD    a8 = X8[T,K] (E4), b8 = W8[N,K] (E4)  ->  out = Y[T,N]
+ *   FP8_MM_DGRAD  a8 = dY8[T,N] (E5), b8 = W8[N,K] (E4)  ->  out = dX[T,K]
+ *   FP8_MM_WGRAD  a8 = dY8[T,N] (E5), b8 = X8[T,K] (E4)  ->  out = dW[N,K]
+ *   d_ba, d_bb    device int32 paper-convention biases of a8 and b8
+ *   out           contiguous, 16-byte aligned, dtype FP8_F16 (IEEE half) or FP8_F32 (exactly the FP16 values)
+ * K % 16 == 0, N % 16 == 0, and the output's row length a multiple of 8. */
+typedef enum { FP8_MM_FWD = 0, FP8_MM_DGRAD = 1, FP8_MM_WGRAD = 2 } fp8_matmul_t;
+FP8_API fp8_status_t fp8_linear_f16acc(fp8_ctx *ctx, fp8_matmul_t kind, const uint8_t *a8, const int32_t *d_ba,
+                                       const uint8_t *b8, const int32_t *d_bb, void *out, fp8_dtype_t out_dt, int32_t chunk,
+                                       int64_t T, int64_t K, int64_t N, fp8_conv_t conv, void *stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -348,10 +348,13 @@ def linear_wgrad_np(dy8, s_g, x8, s_x, fg=N_E5, fx=N_E4):
 # chunk = 1 is a purely sequential FP16 accumulation.
 
 class Fp16AccResult:
-    def __init__(self, f16):
+    def __init__(self, f16, peak, shift_sum):
         self.f16 = f16                          # numpy float16: what an FP16 output tensor would hold
         self.f64 = f16.astype(np.float64)
         self.overflowed = ~np.isfinite(self.f64)
+        # largest magnitude the running FP16 sum went through, in the output's (unscaled) units: one FP16 step at
+        # THAT magnitude is the resolution of the whole accumulation, however small the final value is
+        self.peak = np.ldexp(peak, -int(shift_sum))
 
 
 def _matmul_fp16acc(A, B_t, shift_sum, chunk):
@@ -359,13 +362,15 @@ def _matmul_fp16acc(A, B_t, shift_sum, chunk):
     assert chunk >= 1
     M, Kc = A.shape
     acc = np.zeros((M, B_t.shape[1]), dtype=np.float16)
+    peak = np.zeros(acc.shape, dtype=np.float64)
     for k0 in range(0, Kc, chunk):
         partial = A[:, k0:k0 + chunk] @ B_t[k0:k0 + chunk, :]          # exact: few terms, each a short dyadic number
         with np.errstate(over="ignore", invalid="ignore"):
             acc = (acc.astype(np.float64) + partial).astype(np.float16)    # one rounding to FP16 per chunk
+        peak = np.maximum(peak, np.abs(acc.astype(np.float64)))
     with np.errstate(over="ignore", under="ignore"):
         out = np.ldexp(acc.astype(np.float64), -int(shift_sum)).astype(np.float16)
-    return Fp16AccResult(out)
+    return Fp16AccResult(out, peak, shift_sum)
 
 
 def linear_fwd_fp16acc(x8, s_x, w8, s_w, chunk=128, fx=N_E4, fw=N_E4):

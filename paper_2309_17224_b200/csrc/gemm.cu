@@ -868,13 +868,93 @@ __device__ __forceinline__ void epilogue_tile(const CUtensorMap *map_out, const 
     }
 }
 
+// The i-th work item of a CTA of the single-CTA kernel: an output tile and a slice [k0, k1) of its contraction.
+// Ordinary launches deal (tile, slice) pairs round-robin to the CTAs.  The FP16-accumulation kind (ACT == 6) keeps
+// all slices of a tile on one CTA, in order: its epilogue folds them into a running FP16 sum one after the other.
+template <int ACT>
+__device__ __forceinline__ bool item_at(const GemmParams &p, int i, int &tile, int &split)
+{
+    if (ACT == 6) {
+        tile = (int)blockIdx.x + (i / p.splits) * (int)gridDim.x;
+        split = i % p.splits;
+        return tile < p.tiles_m * p.tiles_n;
+    }
+    const int item = (int)blockIdx.x + i * (int)gridDim.x;
+    tile = item / p.splits;
+    split = item % p.splits;
+    return item < p.tiles_m * p.tiles_n * p.splits;
+}
+
+// FP16 accumulation (Fig. 3b, Section 2.4): the accumulator of one slice (the exact-to-FP32 sum of `chunk` products
+// per output) is added to a running FP16 sum with one rounding to FP16 per slice; after the last slice the FP16 sum
+// is unscaled in FP16 (Eq. 2 on an FP16 output) and stored.  The running sums of the CTA's 128 x 256 tile live in
+// shared memory as [32-column chunk][16-byte piece][row]: a warp's 32 rows are 512 contiguous bytes, no conflicts.
+template <int BN>
+__device__ __forceinline__ void epilogue_f16acc(uint32_t t_row, int row, int col_base, const GemmParams &p, const Pow2Pair sc,
+                                                uint32_t acc_smem, int local_row, bool first, bool last,
+                                                uint32_t release_bar, int lane)
+{
+#pragma unroll 1
+    for (int c = 0; c < BN; c += 32) {
+        uint32_t r[32];
+        tmem_ld_x32(t_row + c, r);
+        tmem_ld_wait();
+        if (c + 32 >= BN) {
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(release_bar);
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const uint32_t addr = acc_smem + (uint32_t)((((c >> 5) * 4 + j) * kBM + local_row) * 16);
+            uint32_t h[4] = {0u, 0u, 0u, 0u};
+            if (!first) asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(h[0]), "=r"(h[1]), "=r"(h[2]), "=r"(h[3]) : "r"(addr));
+            float out[8];
+#pragma unroll
+            for (int w = 0; w < 4; ++w) {
+                float lo, hi;
+                asm("{ .reg .b16 l, u; mov.b32 {l, u}, %2; cvt.f32.f16 %0, l; cvt.f32.f16 %1, u; }" : "=f"(lo), "=f"(hi) : "r"(h[w]));
+                lo += __uint_as_float(r[8 * j + 2 * w]);       // running FP16 sum + this slice's partial sum ...
+                hi += __uint_as_float(r[8 * j + 2 * w + 1]);
+                asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(h[w]) : "f"(hi), "f"(lo));   // ... rounded to FP16, once per slice
+                if (last) {
+                    asm("{ .reg .b16 l, u; mov.b32 {l, u}, %2; cvt.f32.f16 %0, l; cvt.f32.f16 %1, u; }" : "=f"(lo), "=f"(hi) : "r"(h[w]));
+                    out[2 * w] = lo * sc.first * sc.second;    // exact power of two; the FP16 rounding below is the only one
+                    out[2 * w + 1] = hi * sc.first * sc.second;
+                }
+            }
+            if (!last) {
+                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(h[0]), "r"(h[1]), "r"(h[2]), "r"(h[3]) : "memory");
+                continue;
+            }
+            const int col0 = col_base + c + 8 * j;
+            if (row >= p.M || col0 >= p.N) continue;   // N is a multiple of 8: a piece is whole or absent
+            uint32_t o16[4];
+#pragma unroll
+            for (int w = 0; w < 4; ++w) asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(o16[w]) : "f"(out[2 * w + 1]), "f"(out[2 * w]));
+            if (p.out_dt == FP8_F16) {
+                *reinterpret_cast<uint4 *>(reinterpret_cast<uint16_t *>(p.out) + (int64_t)row * p.ldo + col0) =
+                    make_uint4(o16[0], o16[1], o16[2], o16[3]);
+            } else {   // FP32 holding exactly the FP16 values
+                float f[8];
+#pragma unroll
+                for (int w = 0; w < 4; ++w)
+                    asm("{ .reg .b16 l, u; mov.b32 {l, u}, %2; cvt.f32.f16 %0, l; cvt.f32.f16 %1, u; }" : "=f"(f[2 * w]), "=f"(f[2 * w + 1]) : "r"(o16[w]));
+                float4 *dst = reinterpret_cast<float4 *>(reinterpret_cast<float *>(p.out) + (int64_t)row * p.ldo + col0);
+                dst[0] = make_float4(f[0], f[1], f[2], f[3]);
+                dst[1] = make_float4(f[4], f[5], f[6], f[7]);
+            }
+        }
+    }
+}
+
 template <int BN, int STAGES, int ACT>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
             const __grid_constant__ CUtensorMap map_out, const __grid_constant__ CUtensorMap map_out2,
             const GemmParams p)
 {
-    using L = GemmSmem<BN, STAGES, ACT ? kActSlabs : kSingleSlabs>;
+    using L = GemmSmem<BN, STAGES, ACT ? kActSlabs : kSingleSlabs>;   // ACT == 6: the 64 KB of the four slabs per warp hold the FP16 sums
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const uint32_t smem_base = smem_u32(smem);
@@ -887,7 +967,6 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int num_items = p.tiles_m * p.tiles_n * p.splits;  // (tile, k-split) pairs
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
@@ -935,10 +1014,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             // When this grid runs as a programmatic dependent of the launch before it (a decode-size cast), nothing
             // that launch may have written is read before it has completed; but the first ring of B tiles (the
             // weights, in decode) is already pulled towards L2, which holds no stale data whoever writes them.
-            if ((int)blockIdx.x < num_items) {
+            int tile0, split0;
+            if (item_at<ACT>(p, 0, tile0, split0)) {
                 int m_blk, n_blk;
-                tile_coords((int)blockIdx.x / p.splits, p, m_blk, n_blk);
-                const int k0 = ((int)blockIdx.x % p.splits) * p.kb_per_split;
+                tile_coords(tile0, p, m_blk, n_blk);
+                const int k0 = split0 * p.kb_per_split;
                 const int k1 = min(p.num_k, k0 + p.kb_per_split);
                 int k = k0 + first_kblock(m_blk, n_blk, k1 - k0);
                 for (int i = 0; i < min(k1 - k0, STAGES); ++i, k = (k + 1 == k1) ? k0 : k + 1) {
@@ -950,10 +1030,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                 }
             }
             asm volatile("griddepcontrol.wait;" ::: "memory");
-            for (int item = blockIdx.x; alive && item < num_items; item += gridDim.x) {
+            int tile, split;
+            for (int i = 0; alive && item_at<ACT>(p, i, tile, split); ++i) {
                 int m_blk, n_blk;
-                tile_coords(item / p.splits, p, m_blk, n_blk);
-                const int k0 = (item % p.splits) * p.kb_per_split;
+                tile_coords(tile, p, m_blk, n_blk);
+                const int k0 = split * p.kb_per_split;
                 const int k1 = min(p.num_k, k0 + p.kb_per_split);
                 // The k-blocks of an item are taken in a rotated order that differs from tile to tile: with a few
                 // rows of A, all CTAs walking k in step would ask L2 for the same 128-byte lines at the same time
@@ -982,8 +1063,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             bool alive = true;
             // the bounded waits below start counting only once the launch before this one has completed
             asm volatile("griddepcontrol.wait;" ::: "memory");
-            for (int item = blockIdx.x; alive && item < num_items; item += gridDim.x, ++t) {
-                const int k0 = (item % p.splits) * p.kb_per_split;
+            int tile, split;
+            for (int i = 0; alive && item_at<ACT>(p, i, tile, split); ++i, ++t) {
+                const int k0 = split * p.kb_per_split;
                 const int k1 = min(p.num_k, k0 + p.kb_per_split);
                 const int buf = t & 1;
                 const uint32_t acc_ph = (t >> 1) & 1u;
@@ -1021,7 +1103,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         uint32_t t = 0;
         // with split-K every item leaves its raw FP32 partial sum in the workspace; a second kernel finishes
         GemmParams pp = p;
-        if (p.splits > 1) {
+        if (ACT != 6 && p.splits > 1) {
             pp.out_dt = FP8_F32;
             pp.bias_vec = nullptr;
             pp.d_amax_bits = nullptr;
@@ -1029,10 +1111,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             pp.vec_ok = (p.N % 4) == 0;
         }
         const Pow2Pair sc_one = make_pow2_pair(0);
-        for (int item = blockIdx.x; item < num_items; item += gridDim.x, ++t) {
+        int tile, split;
+        for (int i = 0; item_at<ACT>(p, i, tile, split); ++i, ++t) {
             int m_blk, n_blk;
-            tile_coords(item / p.splits, p, m_blk, n_blk);
-            if (p.splits > 1) pp.out = p.partial + (int64_t)(item % p.splits) * p.M * p.N;
+            tile_coords(tile, p, m_blk, n_blk);
+            if (ACT != 6 && p.splits > 1) pp.out = p.partial + (int64_t)split * p.M * p.N;
             const int buf = t & 1;
             const uint32_t acc_ph = (t >> 1) & 1u;
             // every lane waits (each needs the ordering), but the warp leaves together
@@ -1040,6 +1123,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             if (!__all_sync(0xFFFFFFFFu, ready)) break;
             tc_fence_after();
             const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + buf * BN;
+            if constexpr (ACT == 6) {
+                epilogue_f16acc<BN>(t_row, m_blk * kBM + q * 32 + lane, n_blk * BN, p, sc, smem_base + L::kEpiOffset, q * 32 + lane,
+                                    split == 0, split == p.splits - 1, acc_empty_bar(buf), lane);
+                continue;
+            }
             epilogue_tile<BN, ACT, L::kSlabs>(&map_out, &map_out2, t_row, m_blk * kBM + q * 32, n_blk * BN, pp, p.splits > 1 ? sc_one : sc,
                               p.splits > 1 ? false : two_step, amax_bits, warp_slabs, slab_count, acc_empty_bar(buf),
                               false, lane);
@@ -1496,6 +1584,7 @@ static int g_max_pairs = 0;  // CTA pairs that can be resident at once (0: pair 
 #endif
 constexpr bool kWideTileDefault = FP8LIN_WIDE_DEFAULT != 0;
 
+constexpr int kStagesF16Acc = 2;  // the FP16-accumulation kind keeps 64 KB of running sums beside its stages
 constexpr int kStagesAct = 3;  // single-CTA kernels with a second output: fewer stages, two more slabs per warp
 
 template <int ACT>
@@ -1526,6 +1615,9 @@ cudaError_t configure_gemm_kernels(int max_smem_optin)
     if (e == cudaSuccess) e = set_smem_attributes<3>();
     if (e == cudaSuccess) e = set_smem_attributes<4>();
     if (e == cudaSuccess) e = set_smem_attributes<5>();
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(gemm_kernel<kBN, kStagesF16Acc, 6>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 GemmSmem<kBN, kStagesF16Acc, kActSlabs>::kDynamic);
     if (e != cudaSuccess) return e;
     int sms = 0, dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess ||
@@ -1605,10 +1697,10 @@ static fp8_status_t run_gemm(fp8_ctx *ctx, const uint8_t *a, int a_fmt, bool a_m
                              const void *bias_vec, int bias_dt, void *out, int out_dt, float *d_amax_out, int64_t M,
                              int64_t N, int64_t Kc, cudaStream_t st, int act = 0, void *out_act = nullptr,
                              const void *aux = nullptr, uint8_t *out8 = nullptr, const int32_t *d_sq = nullptr,
-                             int q_fmt = 0, int delta_q = 0, bool no_loads = false)
+                             int q_fmt = 0, int delta_q = 0, bool no_loads = false, int chunk_kb = 0)
 {
     if (M > 0x7FFFFFFF / 2 || N > 0x7FFFFFFF / 2 || Kc > 0x7FFFFFFF / 2) return FP8_ERR_SHAPE;
-    const bool pair = g_max_pairs > 0 && M > kBM && !g_force_single;
+    const bool pair = g_max_pairs > 0 && M > kBM && !g_force_single && act != 6;
     CUtensorMap map_a, map_b;
     // an operand stored [Kc, M or N] is fetched as boxes of 128 contraction rows x 128 bytes
     // With a few rows of A (decode) the box covers those rows only, rounded up to the 8-row swizzle atom: the other
@@ -1635,6 +1727,10 @@ static fp8_status_t run_gemm(fp8_ctx *ctx, const uint8_t *a, int a_fmt, bool a_m
     p.splits = 1;
     p.kb_per_split = p.num_k;
     p.partial = ctx->d_partial;
+    if (act == 6) {   // FP16 accumulation: one slice per FP16 addition, all slices of a tile on one CTA
+        p.kb_per_split = chunk_kb > 0 ? chunk_kb : 1;
+        p.splits = (p.num_k + p.kb_per_split - 1) / p.kb_per_split;
+    }
     if (!pair && !g_no_splitk && !act) {
         const int64_t tiles = (int64_t)p.tiles_m * p.tiles_n;
         if (tiles < 2 * ctx->sm_count && p.num_k >= 8) {
@@ -1718,7 +1814,9 @@ static fp8_status_t run_gemm(fp8_ctx *ctx, const uint8_t *a, int a_fmt, bool a_m
                                  dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                                  CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
     };
-    if (act) {
+    if (act == 6) {
+        p.tma_out = 0;   // the FP16-accumulation kind stores from registers
+    } else if (act) {
         // the activated output always goes through the staged epilogue (callers have checked its alignment)
         p.tma_out = 1;
         p.vec_ok = 1;
@@ -1735,7 +1833,7 @@ static fp8_status_t run_gemm(fp8_ctx *ctx, const uint8_t *a, int a_fmt, bool a_m
               ((uint32_t)p.b_mn << 16);
     if (d_amax_out && cudaMemsetAsync(d_amax_out, 0, sizeof(float), st) != cudaSuccess) return FP8_ERR_CUDA;
     int tiles = p.tiles_m * p.tiles_n;
-    count_launch(p.splits > 1 ? 2 : 1);
+    count_launch(p.splits > 1 && act != 6 ? 2 : 1);
     if (pair) {
         const int items = tiles * p.splits;
         int pairs = items < g_max_pairs ? items : g_max_pairs;
@@ -1764,10 +1862,11 @@ static fp8_status_t run_gemm(fp8_ctx *ctx, const uint8_t *a, int a_fmt, bool a_m
         }
         }
     } else {
-        int items = tiles * p.splits;
+        int items = act == 6 ? tiles : tiles * p.splits;
         int grid = items < ctx->sm_count ? items : ctx->sm_count;
         constexpr int kActDyn = GemmSmem<kBN, kStagesAct, kActSlabs>::kDynamic;
         switch (act) {
+        case 6: gemm_kernel<kBN, kStagesF16Acc, 6><<<grid, kGemmThreads, GemmSmem<kBN, kStagesF16Acc, kActSlabs>::kDynamic, st>>>(map_a, map_b, map_out, map_out2, p); break;
         case 1: gemm_kernel<kBN, kStagesAct, 1><<<grid, kGemmThreads, kActDyn, st>>>(map_a, map_b, map_out, map_out2, p); break;
         case 2: gemm_kernel<kBN, kStagesAct, 2><<<grid, kGemmThreads, kActDyn, st>>>(map_a, map_b, map_out, map_out2, p); break;
         case 3: gemm_kernel<kBN, kStagesAct, 3><<<grid, kGemmThreads, kActDyn, st>>>(map_a, map_b, map_out, map_out2, p); break;
@@ -1791,7 +1890,7 @@ static fp8_status_t run_gemm(fp8_ctx *ctx, const uint8_t *a, int a_fmt, bool a_m
         }
         }
     }
-    if (p.splits > 1) {
+    if (p.splits > 1 && act != 6) {
         if (cudaGetLastError() != cudaSuccess) return FP8_ERR_CUDA;
         const bool vec = p.vec_ok && (N % 4) == 0;
         int64_t threads = vec ? M * N / 4 : M * N;
@@ -1974,6 +2073,27 @@ fp8_status_t fp8_linear_dgrad_q(fp8_ctx *ctx, const uint8_t *dy8, const int32_t 
     const int kind = act == FP8_ACT_GELU ? 2 : (act == FP8_ACT_SWIGLU ? 5 : 3);
     return run_gemm(ctx, dy8, FP8_E5, false, d_bg, w, FP8_E4, w_mn, d_bw, delta, nullptr, 0, dx, FP8_BF16, d_amax_g, T, K,
                     N, (cudaStream_t)stream, kind, g, y_pre, g8, d_bq, FP8_E5, format_delta(FP8_E5, conv));
+}
+
+fp8_status_t fp8_linear_f16acc(fp8_ctx *ctx, fp8_matmul_t kind, const uint8_t *a8, const int32_t *d_ba, const uint8_t *b8,
+                               const int32_t *d_bb, void *out, fp8_dtype_t out_dt, int32_t chunk, int64_t T, int64_t K,
+                               int64_t N, fp8_conv_t conv, void *stream)
+{
+    using namespace fp8lin;
+    if (!ctx || !a8 || !d_ba || !b8 || !d_bb || !out) return FP8_ERR_NULL;
+    if ((int)kind < 0 || (int)kind > 2 || (int)conv < 0 || (int)conv > 1 || (int)out_dt < 0 || (int)out_dt > 2) return FP8_ERR_DTYPE;
+    if (out_dt != FP8_F16 && out_dt != FP8_F32) return FP8_ERR_UNSUPPORTED;
+    if (T <= 0 || K <= 0 || N <= 0 || chunk <= 0 || (chunk % kBK) != 0) return FP8_ERR_SHAPE;
+    // operands in their forward layouts: X8[T,K], W8[N,K], dY8[T,N]
+    const int64_t rows = kind == FP8_MM_WGRAD ? N : T, cols = kind == FP8_MM_FWD ? N : K;
+    const int64_t contraction = kind == FP8_MM_FWD ? K : (kind == FP8_MM_DGRAD ? N : T);
+    if (!aligned16(a8) || !aligned16(b8) || !aligned16(out) || (K % 16) != 0 || (N % 16) != 0 || (cols % 8) != 0) return FP8_ERR_ALIGN;
+    const int e4 = format_delta(FP8_E4, conv), e5 = format_delta(FP8_E5, conv);
+    const int a_fmt = kind == FP8_MM_FWD ? FP8_E4 : FP8_E5;
+    const int delta = (kind == FP8_MM_FWD ? e4 : e5) + e4;
+    const bool a_mn = kind == FP8_MM_WGRAD, b_mn = kind != FP8_MM_FWD;
+    return run_gemm(ctx, a8, a_fmt, a_mn, d_ba, b8, FP8_E4, b_mn, d_bb, delta, nullptr, 0, out, (int)out_dt, nullptr, rows, cols,
+                    contraction, (cudaStream_t)stream, 6, nullptr, nullptr, nullptr, nullptr, 0, 0, false, chunk / kBK);
 }
 
 fp8_status_t fp8_linear_wgrad(fp8_ctx *ctx, const uint8_t *dy8, const uint8_t *dy8_t, const int32_t *d_bg,

@@ -23,6 +23,7 @@ E4, E5 = 0, 1
 CONV_PAPER, CONV_NATIVE = 0, 1
 BF16, F16, F32 = 0, 1, 2
 GROUP_AMAX_CAST, GROUP_PREDICTED, GROUP_AMAX_ONLY, GROUP_CAST_ONLY = 0, 1, 2, 3
+MM_FWD, MM_DGRAD, MM_WGRAD = 0, 1, 2
 ACT_NONE = 0
 ACT_GELU = 1
 ACT_SWIGLU = 2
@@ -32,7 +33,7 @@ SYMBOLS = (
     "fp8_create", "fp8_destroy", "fp8_status_string", "fp8_device_flags", "fp8_amax", "fp8_scaling_bias",
     "fp8_scaling_bias_host", "fp8_cast_e4", "fp8_cast_e5", "fp8_ptq_weights", "fp8_linear_fwd", "fp8_linear_dgrad",
     "fp8_linear_wgrad", "fp8_amax_noalloc", "fp8_linear_fwd_act", "fp8_cast_predicted", "fp8_prediction_stats",
-    "fp8_linear_dgrad_act", "fp8_selftest_wait_expiry", "fp8_range_stats", "fp8_linear_fwd_q", "fp8_linear_dgrad_q", "fp8_amax_history_bias", "fp8_launch_count", "fp8_cast_group", "fp8_selftest_mma_ceiling", "fp8_bias_log_append", "fp8_bias_mode",
+    "fp8_linear_dgrad_act", "fp8_selftest_wait_expiry", "fp8_range_stats", "fp8_linear_fwd_q", "fp8_linear_dgrad_q", "fp8_amax_history_bias", "fp8_launch_count", "fp8_cast_group", "fp8_selftest_mma_ceiling", "fp8_bias_log_append", "fp8_bias_mode", "fp8_linear_f16acc",
 )
 
 if not os.path.exists(LIB_PATH):
@@ -72,6 +73,7 @@ _lib.fp8_linear_fwd_q.argtypes = [_P, _P, _P, _P, _P, _P, c_int, c_int, _P, _P, 
                                   c_int, _P]
 _lib.fp8_linear_dgrad_q.argtypes = [_P, _P, _P, _P, _P, _P, c_int, _P, _P, _P, _P, _P, _P, c_int64, c_int64, c_int64,
                                     c_int, _P]
+_lib.fp8_linear_f16acc.argtypes = [_P, c_int, _P, _P, _P, _P, _P, c_int, c_int32, c_int64, c_int64, c_int64, c_int, _P]
 _lib.fp8_linear_wgrad.argtypes = [_P, _P, _P, _P, _P, _P, _P, _P, c_int, c_int64, c_int64, c_int64, c_int, _P]
 
 
@@ -318,6 +320,11 @@ class Context:
         _check(_lib.fp8_linear_dgrad_q(self._h, _ptr(dy8), _ptr(d_bg), _ptr(w8), _ptr(w8_t), _ptr(d_bw), act,
                                        _ptr(y_pre), _ptr(dx), _ptr(g), _ptr(g8), _ptr(d_bq), _ptr(d_amax_g), T, K, N,
                                        conv, _stream()), "fp8_linear_dgrad_q")
+
+    def linear_f16acc(self, kind, a8, d_ba, b8, d_bb, out, T, K, N, chunk=128, conv=CONV_PAPER):
+        """``fp8_linear_f16acc``: the matmul of `kind` with FP16 accumulation emulated; out is float16 or float32."""
+        _check(_lib.fp8_linear_f16acc(self._h, kind, _ptr(a8), _ptr(d_ba), _ptr(b8), _ptr(d_bb), _ptr(out), _DT[out.dtype],
+                                      chunk, T, K, N, conv, _stream()), "fp8_linear_f16acc")
 
     def linear_wgrad(self, dy8, dy8_t, d_bg, x8, x8_t, d_bx, dw, T, conv=CONV_PAPER):
         N, K = dw.shape

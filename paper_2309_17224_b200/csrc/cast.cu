@@ -177,7 +177,10 @@ static cudaError_t launch_predicted(fp8_ctx *ctx, const void *x, int64_t n, int 
 
 constexpr int kSmallThreads = 1024;
 constexpr int kSmallVecs = 8;          // 16-byte vectors per thread
-constexpr int kSmallMaxCtas = 2;   // beyond ~128K elements the two-launch path (whole GPU) is faster
+#ifndef FP8LIN_SMALL_MAX_CTAS
+#define FP8LIN_SMALL_MAX_CTAS 2
+#endif
+constexpr int kSmallMaxCtas = FP8LIN_SMALL_MAX_CTAS;   // beyond ~128K elements the two-launch path (whole GPU) is faster
 
 template <int FMT, int DT>
 __global__ void __launch_bounds__(kSmallThreads)

@@ -831,6 +831,7 @@ __device__ __forceinline__ void epilogue_tile(const CUtensorMap *map_out, const 
             tmem_ld_x32(t_row + c + 32, r1);
             tmem_ld_wait();
             if (c + 64 >= BN) release();
+
             const uint32_t slab = warp_slabs + (slab_count % NSLAB) * kSlabBytes;
             ++slab_count;
             slab_acquire<NSLAB>(lane);

@@ -1041,6 +1041,14 @@ def main():
                 t_on = _time_burst(lambda: ctx.linear_fwd(a8, zero, b8, zero, out), 10, warm=2)
                 ceiling[name] = {"shape_mnk": [M, N, K], "loads_off_tflops": 2.0 * M * N * K / t_off / 1e9,
                                  "with_loads_tflops": 2.0 * M * N * K / t_on / 1e9}
+                try:   # context only: the vendor library's FP8 matmul on the same operands, same moment, same clock
+                    one = torch.ones((), dtype=torch.float32, device=device)
+                    af, bf = a8.view(torch.float8_e4m3fn), b8.view(torch.float8_e4m3fn).t()
+                    t_lib = _time_burst(lambda: torch._scaled_mm(af, bf, scale_a=one, scale_b=one, out_dtype=torch.bfloat16),
+                                        10, warm=2)
+                    ceiling[name]["library_fp8_matmul_tflops"] = 2.0 * M * N * K / t_lib / 1e9
+                except Exception:
+                    pass
                 del out, a8, b8
             ceiling["clocks"] = c_sampler.stop()
             roofline["ceiling"] = ceiling

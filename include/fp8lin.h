@@ -10,7 +10,9 @@
  *  - All tensor pointers are DEVICE pointers owned by the caller; the library
  *    never allocates, frees or retains them.  "d_" marks a device scalar.
  *    The only host pointers are the fp8_ctx handle, `flags` of
- *    fp8_device_flags and the arguments of fp8_scaling_bias_host.
+ *    fp8_device_flags, the counters of fp8_prediction_stats and
+ *    fp8_launch_count, the descriptor array of fp8_cast_group and the
+ *    arguments of fp8_scaling_bias_host.
  *  - `stream` is a cudaStream_t passed as void* (NULL = the legacy default
  *    stream).  Calls are asynchronous and ordered on that stream like any
  *    kernel launch.  Calls that share one fp8_ctx must be issued from one host

@@ -1,5 +1,6 @@
 // Grouped FP8-AMAX quantisation: amax -> bias -> scale-and-cast (Eq. 3, Eq. 1, Section 2.1 / 2.2) of several
-// tensors in two launches instead of two per tensor.
+// tensors in two launches instead of two per tensor.  The same kernels, on a group of one, serve every contiguous
+// single-tensor call (fp8_amax, fp8_cast_e4 / _e5, fp8_cast_predicted, delayed scaling).
 //
 // The tensors a step quantises are tens to hundreds of megabytes each; launched one by one, every kernel pays its
 // own ramp-up and its own thin last wave, which at these sizes is 10-40 % of its run time.  Here the tensors of a

@@ -410,7 +410,7 @@ def quantisation_kernel_bandwidths(ctx, fp8lin, layers, peak_gbs, reps=3):
     bias = torch.zeros(1, dtype=torch.int32, device=dev)
     items = fp8lin.group_items(tensors)
     elems = sum(t[1].numel() for t in tensors)
-    out = {"how": f"one launch at a time, {reps} rounds after one untimed, inputs out of L2; grouped kernels walk the step's "
+    out = {"how": f"one launch at a time, {reps} passes after one untimed, inputs out of L2; grouped kernels walk the step's "
                   f"{len(tensors)} tensors ({elems / 1e6:.0f} M elements) per launch"}
 
     def timed_once(fn):
@@ -448,7 +448,7 @@ def quantisation_kernel_bandwidths(ctx, fp8lin, layers, peak_gbs, reps=3):
         for rep in range(reps + 1):
             for fmt, x, _, _, y in tensors:
                 a, b = timed_once(lambda: launch(key, fmt, x, y))
-                if rep > 0:                # the first round loads the kernels
+                if rep > 0:                # the first pass loads the kernels
                     spans.append((x.numel(), a, b))
         torch.cuda.synchronize()
         rates = [n * bpe / (a.elapsed_time(b) * 1e-3) / 1e9 for n, a, b in spans]

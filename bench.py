@@ -52,7 +52,7 @@ NOMINAL_FP8_TFLOPS = 4500.0         # dense FP8, the vendor's figure for the par
 FP8_FLOP_PER_CLK_PER_SM = 16384.0   # 8192 multiply-adds per clock per SM: nominal peak / (148 SMs x 1.856 GHz)
 # dram__bytes_read.sum + dram__bytes_write.sum per matmul launch, from one ncu capture of one step of the
 # workload (profiles/launch_list_c3_llama7b.md, second table); keyed by (workload, tokens)
-GEMM_DRAM_BYTES_PER_LAUNCH = {("c3_llama7b", 8192): 383.5e6}
+GEMM_DRAM_BYTES_PER_LAUNCH = {("c3_llama7b", 8192): 331.3e6}
 
 
 def load_peaks():

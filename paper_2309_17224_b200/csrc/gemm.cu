@@ -55,6 +55,7 @@ constexpr int kBK = 128;          // contraction bytes per stage = one 128-byte 
 constexpr int kUmmaK = 32;        // contraction elements per tcgen05.mma for 8-bit types
 constexpr int kGemmThreads = 192;
 constexpr int kGroupM = 16;       // tile rasterisation: m-blocks per group
+constexpr int64_t kStreamOutBytes = 64ll << 20;   // outputs from this size on are stored with the evict-first mark
 constexpr int kSlabBytes = 32 * 128;            // epilogue staging: 32 rows x 128 bytes, what one warp stores at a time
 constexpr int kSingleSlabs = 2;                 // staging slabs per epilogue warp, single-CTA kernel
 constexpr int kActSlabs = 4;                    // ... of the kernels with a second output: two {output, z} pairs
@@ -67,6 +68,8 @@ struct GemmParams {
     int M, N, K;
     int tiles_m, tiles_n, num_k;
     int group_m;                  // tile rasterisation: m-blocks per group
+    int serpentine;               // pair kernel: every other tile of a pair walks the contraction backwards
+    int out_stream;               // plain epilogue: the output is far larger than L2, its stores are marked evict-first
     int splits, kb_per_split;     // split-K (single-CTA kernel only): k-blocks per split
     float *partial;               // [splits, M, N] FP32 partial sums when splits > 1
     const int32_t *d_sa, *d_sb;   // paper-convention biases of the two operands
@@ -329,6 +332,18 @@ __device__ __forceinline__ void tma_store_2d(const CUtensorMap *map, uint32_t sr
                  : "memory");
     asm volatile("cp.async.bulk.commit_group;" ::: "memory");
 }
+// The same store for an output far larger than L2: its lines are marked to leave L2 first, so that they do not push
+// out operand strips that other CTAs are about to read.
+__device__ __forceinline__ void tma_store_2d_stream(const CUtensorMap *map, uint32_t src, int x, int y)
+{
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group.L2::cache_hint [%0, {%2, %3}], [%1], %4;" ::"l"(
+                     reinterpret_cast<uint64_t>(map)),
+                 "r"(src), "r"(x), "r"(y), "l"(pol)
+                 : "memory");
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
 // 16-byte piece j (0..7) of this lane's 128-byte row, at its 128-byte-swizzle position
 __device__ __forceinline__ void slab_write(uint32_t slab, int lane, int j, uint32_t a, uint32_t b, uint32_t c, uint32_t d)
 {
@@ -347,11 +362,15 @@ __device__ __forceinline__ void slab_acquire(int lane)
     }
     __syncwarp();
 }
-__device__ __forceinline__ void slab_publish(const CUtensorMap *map, uint32_t slab, int lane, int x, int y, bool in_range)
+__device__ __forceinline__ void slab_publish(const CUtensorMap *map, uint32_t slab, int lane, int x, int y, bool in_range,
+                                             bool stream = false)
 {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     __syncwarp();
-    if (lane == 0 && in_range) tma_store_2d(map, slab, x, y);
+    if (lane == 0 && in_range) {
+        if (stream) tma_store_2d_stream(map, slab, x, y);
+        else tma_store_2d(map, slab, x, y);
+    }
 }
 
 // Phi(-|x|), the lower tail of the standard normal distribution, and exp(-x^2 / 2), in about fifteen FP32
@@ -845,7 +864,7 @@ __device__ __forceinline__ void epilogue_tile(const CUtensorMap *map_out, const 
             pack_bf16(v, col_base + c + 32, p, w, amax_bits, row_ok);
 #pragma unroll
             for (int j = 0; j < 4; ++j) slab_write(slab, lane, 4 + j, w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
-            slab_publish(map_out, slab, lane, col_base + c, row0, rows_in && col_base + c < p.N);
+            slab_publish(map_out, slab, lane, col_base + c, row0, rows_in && col_base + c < p.N, p.out_stream != 0);
         }
     } else {
 #pragma unroll 1
@@ -864,7 +883,7 @@ __device__ __forceinline__ void epilogue_tile(const CUtensorMap *map_out, const 
             for (int j = 0; j < 8; ++j)
                 slab_write(slab, lane, j, __float_as_uint(v[4 * j]), __float_as_uint(v[4 * j + 1]),
                            __float_as_uint(v[4 * j + 2]), __float_as_uint(v[4 * j + 3]));
-            slab_publish(map_out, slab, lane, col_base + c, row0, rows_in && col_base + c < p.N);
+            slab_publish(map_out, slab, lane, col_base + c, row0, rows_in && col_base + c < p.N, p.out_stream != 0);
         }
     }
 }
@@ -1106,6 +1125,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         GemmParams pp = p;
         if (ACT != 6 && p.splits > 1) {
             pp.out_dt = FP8_F32;
+            pp.out_stream = 0;   // the partial sums are read back at once
             pp.bias_vec = nullptr;
             pp.d_amax_bits = nullptr;
             pp.tma_out = 0;
@@ -1325,17 +1345,23 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
         if (lane == 0) {
             asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_a)) : "memory");
             asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_b)) : "memory");
-            uint32_t it = 0;
+            uint32_t it = 0, t = 0;
             bool alive = true;
             const uint32_t leader_full0 = map_to_cta(full_bar(0), 0);
             // launched as a programmatic dependent of the cast before it: set-up above overlaps that grid's tail,
             // its bytes are not requested before it has completed
             asm volatile("griddepcontrol.wait;" ::: "memory");
-            for (int tile = pair_id; alive && tile < num_tiles; tile += num_pairs) {
+            for (int tile = pair_id; alive && tile < num_tiles; tile += num_pairs, ++t) {
                 int m_blk, n_blk;
                 tile_coords(tile / p.splits, p, m_blk, n_blk);
                 const int k0 = (tile % p.splits) * p.kb_per_split, k1 = min(p.num_k, k0 + p.kb_per_split);
+                // Every other tile of a pair walks the contraction backwards.  All pairs pass from one tile to the
+                // next at about the same time, and the next tiles share operand strips with the last ones; what L2
+                // still holds of those strips is their far end, which a forward walk would reach last (and evict
+                // on the way there).
+                const bool backwards = (t & 1u) != 0 && p.serpentine;
                 for (int k = k0; k < k1; ++k, ++it) {
+                    const int kc = (backwards ? k0 + k1 - 1 - k : k) * kBK;
                     const int s = it % kStagesL;
                     const uint32_t leader_full = leader_full0 + 8u * s;
                     const uint32_t ph = (it / kStagesL) & 1u;
@@ -1349,14 +1375,14 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                     if (rank == 0) mbar_expect_tx(full_bar(s), 2 * L::kStageBytes);
                     const uint32_t a_dst = smem_base + s * L::kStageBytes;
                     const int a_row = m_blk * 256 + (int)rank * kBM;
-                    if (p.a_mn) tma_load_2d_pair(a_dst, &map_a, leader_full, a_row, k * kBK);
-                    else tma_load_2d_pair(a_dst, &map_a, leader_full, k * kBK, a_row);
+                    if (p.a_mn) tma_load_2d_pair(a_dst, &map_a, leader_full, a_row, kc);
+                    else tma_load_2d_pair(a_dst, &map_a, leader_full, kc, a_row);
 #pragma unroll
                     for (int h = 0; h < NHALF; ++h) {   // this CTA's 128 of the 256 B rows of each half of the tile
                         const int b_row = n_blk * kTileN + h * kPairBN + (int)rank * kPairHalfN;
                         const uint32_t b_dst = a_dst + L::kABytes + h * (kPairHalfN * kBK);
-                        if (p.b_mn) tma_load_2d_pair(b_dst, &map_b, leader_full, b_row, k * kBK);
-                        else tma_load_2d_pair(b_dst, &map_b, leader_full, k * kBK, b_row);
+                        if (p.b_mn) tma_load_2d_pair(b_dst, &map_b, leader_full, b_row, kc);
+                        else tma_load_2d_pair(b_dst, &map_b, leader_full, kc, b_row);
                     }
                 }
             }
@@ -1434,6 +1460,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
         GemmParams pp = p;
         if (p.splits > 1) {
             pp.out_dt = FP8_F32;
+            pp.out_stream = 0;   // the partial sums are read back at once
             pp.bias_vec = nullptr;
             pp.d_amax_bits = nullptr;
             pp.tma_out = 0;
@@ -1577,6 +1604,8 @@ static bool g_no_splitk = false;        // set from FP8LIN_NO_SPLITK=1
 static int g_force_splits = 0;          // set from FP8LIN_SPLITS (experiments with the split count)
 static bool g_no_pdl = false;           // set from FP8LIN_NO_PDL=1 (A/B: matmuls launched without programmatic dependence)
 static bool g_direct_epilogue = false;  // set from FP8LIN_DIRECT_EPILOGUE=1 (A/B comparison of the epilogues)
+static bool g_no_out_stream = false;    // set from FP8LIN_OUT_STREAM=0 (A/B: output stores without the evict-first mark)
+static bool g_no_serpentine = false;    // set from FP8LIN_SERPENTINE=0 (A/B: every tile walks the contraction forwards)
 static int g_force_wide = -1;           // set from FP8LIN_WIDE=0/1 (A/B: never / always the 256 x 512 pair tile)
 static int g_max_pairs = 0;  // CTA pairs that can be resident at once (0: pair kernel unavailable)
 
@@ -1646,6 +1675,10 @@ cudaError_t configure_gemm_kernels(int max_smem_optin)
     g_force_single = env && env[0] == '1';
     env = getenv("FP8LIN_GROUP_M");
     g_group_m = env ? atoi(env) : 0;
+    env = getenv("FP8LIN_OUT_STREAM");
+    g_no_out_stream = env && env[0] == '0';
+    env = getenv("FP8LIN_SERPENTINE");
+    g_no_serpentine = env && env[0] == '0';
     env = getenv("FP8LIN_NO_PDL");
     g_no_pdl = env && env[0] == '1';
     env = getenv("FP8LIN_SPLITS");
@@ -1714,6 +1747,8 @@ static fp8_status_t run_gemm(fp8_ctx *ctx, const uint8_t *a, int a_fmt, bool a_m
     if (!ok_a || !ok_b) return FP8_ERR_CUDA;
     GemmParams p;
     p.group_m = g_group_m > 0 ? g_group_m : kGroupM;
+    p.serpentine = g_no_serpentine ? 0 : 1;
+    p.out_stream = (!g_no_out_stream && (int64_t)M * N * (out_dt == FP8_F32 ? 4 : 2) >= kStreamOutBytes) ? 1 : 0;
     p.a_mn = a_mn ? 1 : 0;
     p.b_mn = b_mn ? 1 : 0;
     p.a_box_bytes = a_box_rows * kBK;

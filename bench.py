@@ -477,6 +477,9 @@ def oracle_sample_tokens(wl, seconds):
     return max(16, min(T, 1024, wl.tokens))
 
 
+ORACLE_SPLIT = {}   # the last oracle_sample_run's time, split into quantisation (3 B per element) and matmuls
+
+
 def oracle_sample_run(wl, seed, tokens=ORACLE_SAMPLE_TOKENS):
     """One bounded sample of the workload on the CPU oracle: the whole path
     (amax, bias, cast of X, W, dY; the three matmuls) for one layer at a
@@ -491,14 +494,20 @@ def oracle_sample_run(wl, seed, tokens=ORACLE_SAMPLE_TOKENS):
     t0 = time.perf_counter()
     _, bx, x8 = O.quantise(xb, O.E4)
     _, bw, w8 = O.quantise(wb, O.E4)
+    elements = xb.size + wb.size
+    if wl.backward:
+        _, bg, g8 = O.quantise(gb, O.E5)
+        elements += gb.size
+    t1 = time.perf_counter()
     O.linear_fwd(x8, bx + 1, w8, bw + 1)
     flops = 2.0 * T * l.K * l.N
     if wl.backward:
-        _, bg, g8 = O.quantise(gb, O.E5)
         O.linear_dgrad(g8, bg, w8, bw + 1)
         O.linear_wgrad(g8, bg, x8, bx + 1)
         flops *= 3
     dt = time.perf_counter() - t0
+    ORACLE_SPLIT.update(quantise_seconds=t1 - t0, quantise_elements=int(elements), matmul_seconds=dt - (t1 - t0),
+                        amax_cast_gbs=3.0 * elements / (t1 - t0) / 1e9, matmul_tflops=flops / (dt - (t1 - t0)) / 1e12)
     what = (f"layer '{l.name}' ({l.K}->{l.N}) of {wl.name} at {T} of {wl.tokens} tokens: amax+bias+cast of X, W"
             f"{', dY' if wl.backward else ''} and {'3 matmuls' if wl.backward else '1 matmul'}, {flops / 1e9:.1f} GFLOP")
     return dt, flops, what, O.num_threads(), l, T
@@ -530,7 +539,7 @@ def reference_arm(args, wl):
                    "tokens": T, "of_tokens": wl.tokens, "layers": [f"{layer.name}:{layer.K}->{layer.N}"],
                    "of_layers": [f"{l.name}:{l.K}->{l.N}" for l in wl.layers],
                    "passes": "fwd+bwd" if wl.backward else "fwd"},
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": what},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": what, **ORACLE_SPLIT},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
@@ -1272,7 +1281,7 @@ def main():
         O.build()
         dt, fl, what, cores, _, _ = oracle_sample_run(wl, I.BASE_SEED, oracle_sample_tokens(wl, 12.0))
         cpu_baseline = {"value": fl / dt / 1e12, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": what,
-                        "seconds": dt}
+                        "seconds": dt, **ORACLE_SPLIT}
 
     quant_note = {
         "group-predicted": "FP8-AMAX for W, X, dY every step, all tensors of the step in one fp8_cast_group call; each tensor "

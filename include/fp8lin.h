@@ -336,6 +336,19 @@ FP8_API fp8_status_t fp8_linear_fwd(fp8_ctx *ctx, const uint8_t *x8, const int32
                             fp8_dtype_t y_dt, float *d_amax_y, int64_t T, int64_t K, int64_t N, fp8_conv_t conv,
                             void *stream);
 
+/* The forward matmul of inference on weights quantised once (Section 3.1: post-training quantisation, the weights'
+ * scaling bias and bytes are fixed, the activations are quantised per call).  Arguments, result and errors are
+ * those of fp8_linear_fwd, bit for bit.  One more condition on the caller, and what it buys: the bytes of w8 must
+ * have been final before the launch that precedes this call on `stream` began (true of weights produced once by
+ * fp8_ptq_weights and then left alone; NOT true when w8 comes out of a cast enqueued just before).  With at most 128
+ * rows the matmul then starts streaming weight tiles while that launch (typically the cast of the few activation
+ * rows) is still running, instead of after it; x8, d_bx, d_bw and bias_vec are still read only once it has
+ * completed.  With more rows the call is fp8_linear_fwd. */
+FP8_API fp8_status_t fp8_linear_infer(fp8_ctx *ctx, const uint8_t *x8, const int32_t *d_bx, const uint8_t *w8,
+                              const int32_t *d_bw, const void *bias_vec, fp8_dtype_t bias_dt, void *y,
+                              fp8_dtype_t y_dt, float *d_amax_y, int64_t T, int64_t K, int64_t N, fp8_conv_t conv,
+                              void *stream);
+
 /* Forward matmul with the activation fused into the epilogue (the paper has no
  * counterpart; it answers Section 3's warning that computing a scale just in
  * time costs a second pass over memory: the next layer's input leaves this

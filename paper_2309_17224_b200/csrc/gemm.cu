@@ -76,6 +76,11 @@ struct GemmParams {
     int delta_sum;                // format shifts to add to them
     int a_mn, b_mn;               // operand stored with its M / N index contiguous (contraction index strided)
     int a_box_bytes;              // single-CTA kernel: bytes one A load brings (its box holds only the rows that exist)
+    int dec_bn, dec_stages, dec_a_bytes;   // decode kernel: tile width, stages, bytes a stage sets aside for A
+    int dec_cluster;              // decode kernel: CTAs of a cluster that share one tile's contraction (1: none)
+    int early_b;                  // decode kernel: B may be read before the launch ahead of this one has completed
+    int col_lo;                   // direct stores skip columns below this one (0 except in the decode kernel's last tile)
+    int dbg;                      // experiments build only: timing variants that give wrong results
     const void *bias_vec;         // [N] or NULL
     int bias_dt;
     void *out;
@@ -283,33 +288,39 @@ __device__ __forceinline__ void amax_f32(const float (&v)[32], int col0, const G
 __device__ __forceinline__ void store_direct(const uint32_t (&r)[32], int row, int col0, const GemmParams &p,
                                              const Pow2Pair sc, bool two_step, uint32_t &amax_bits)
 {
-    if (row >= p.M || col0 >= p.N) return;
+    if (row >= p.M || col0 >= p.N || col0 + 32 <= p.col_lo) return;
     float v[32];
     epilogue_values(r, col0, p, sc, two_step, v);
+    const bool below = col0 < p.col_lo;   // the chunk starts in columns that another tile owns (decode kernel only)
+    if (below) {
+#pragma unroll
+        for (int i = 0; i < 32; ++i)
+            if (col0 + i < p.col_lo) v[i] = 0.0f;   // not stored; keeps them out of the amax
+    }
     if (p.out_dt == FP8_BF16) {
         uint32_t w[16];
         pack_bf16(v, col0, p, w, amax_bits, true);
         uint16_t *dst = reinterpret_cast<uint16_t *>(p.out) + (int64_t)row * p.ldo + col0;
-        if (p.vec_ok && col0 + 32 <= p.N) {
+        if (p.vec_ok && col0 + 32 <= p.N && !below) {
 #pragma unroll
             for (int j = 0; j < 4; ++j)
                 reinterpret_cast<uint4 *>(dst)[j] = make_uint4(w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
         } else {
 #pragma unroll
             for (int i = 0; i < 32; ++i)
-                if (col0 + i < p.N) dst[i] = (uint16_t)((i & 1) ? (w[i >> 1] >> 16) : (w[i >> 1] & 0xFFFFu));
+                if (col0 + i < p.N && col0 + i >= p.col_lo) dst[i] = (uint16_t)((i & 1) ? (w[i >> 1] >> 16) : (w[i >> 1] & 0xFFFFu));
         }
     } else {
         amax_f32(v, col0, p, amax_bits, true);
         float *dst = reinterpret_cast<float *>(p.out) + (int64_t)row * p.ldo + col0;
-        if (p.vec_ok && col0 + 32 <= p.N) {
+        if (p.vec_ok && col0 + 32 <= p.N && !below) {
 #pragma unroll
             for (int j = 0; j < 8; ++j)
                 reinterpret_cast<float4 *>(dst)[j] = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
         } else {
 #pragma unroll
             for (int i = 0; i < 32; ++i)
-                if (col0 + i < p.N) dst[i] = v[i];
+                if (col0 + i < p.N && col0 + i >= p.col_lo) dst[i] = v[i];
         }
     }
 }
@@ -529,6 +540,10 @@ __device__ __forceinline__ void epilogue_tile(const CUtensorMap *map_out, const 
         }
     };
     if (!p.tma_out) {
+        if (row0 >= p.M) {   // none of this warp's rows exists (decode): nothing to read
+            release();
+            return;
+        }
 #pragma unroll 1
         for (int c = 0; c < BN; c += 32) {
             uint32_t r[32];
@@ -1149,9 +1164,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                                     split == 0, split == p.splits - 1, acc_empty_bar(buf), lane);
                 continue;
             }
-            epilogue_tile<BN, ACT, L::kSlabs>(&map_out, &map_out2, t_row, m_blk * kBM + q * 32, n_blk * BN, pp, p.splits > 1 ? sc_one : sc,
-                              p.splits > 1 ? false : two_step, amax_bits, warp_slabs, slab_count, acc_empty_bar(buf),
-                              false, lane);
+            epilogue_tile<BN, ACT, L::kSlabs>(&map_out, &map_out2, t_row, m_blk * kBM + q * 32, n_blk * BN, pp,
+                              p.splits > 1 ? sc_one : sc, p.splits > 1 ? false : two_step, amax_bits, warp_slabs, slab_count,
+                              acc_empty_bar(buf), false, lane);
         }
         if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
         if (p.d_amax_bits) {
@@ -1167,6 +1182,339 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     __syncthreads();
     tc_fence_after();
     if (warp == 1) tmem_dealloc(tmem_base, L::kTmemCols);
+}
+
+
+// ---------------------------------------------------------------------------
+// Decode kernel: at most 128 rows of A, both operands contraction-major, plain epilogue
+// ---------------------------------------------------------------------------
+//
+// The weight-streaming regime (Section 3.1: weights quantised once, a few activation rows per call).  Same pipeline
+// as gemm_kernel, with the tile width and the stage count chosen per launch instead of per instantiation: the host
+// picks a width `bn` (a multiple of 16 up to 256) that gives close to one tile per SM, so that most layers need no
+// split contraction (no partial sums, no second launch), and as many stages as shared memory holds, so that a CTA
+// keeps about 190 KB of weight bytes in flight whatever the width.  A stage is `a_bytes` of A (the rows that exist,
+// rounded up to the 1024-byte swizzle atom; the instruction reads 128 rows, the rest being the head of the B tile
+// behind it, feeding output rows that are never stored) followed by bn x 128 bytes of B.  The few output rows are
+// stored from registers.
+//
+// Where a layer has too few tiles for the SMs, the contraction of a tile is split across the CTAs of a cluster
+// (p.dec_cluster of them, one item each): when all have finished their slices the others write their FP32 sums
+// into the leader's shared memory (its stages are free by then) and the leader adds them in rank order and stores
+// the result: no partial sums in global memory, no second launch.  Two cluster barriers frame the exchange; a CTA
+// whose wait ran out still takes part in both.
+
+__device__ __forceinline__ uint32_t cluster_ctarank()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t rank)
+{
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
+#ifdef FP8LIN_EXPERIMENTS
+// timeline of the decode launches (block 0): entry, dependency wait over, exit; read back by fp8_debug_trace
+__device__ unsigned long long g_trace[3 * 1024];
+__device__ unsigned g_trace_n;
+#endif
+
+constexpr int kDecodeMaxStages = 32;
+constexpr int kDecodeHeader = 1024;   // barriers, tensor-memory slot and abort flag in front of the stages
+constexpr int kDecodeSmemBudget = 225 * 1024;   // header + stages, with the slack for aligning the base
+
+__global__ void __launch_bounds__(kGemmThreads, 1)
+decode_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const GemmParams p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    const uint32_t bar_base = smem_u32(smem);
+    const uint32_t stage_base = bar_base + kDecodeHeader;
+    const int stages = p.dec_stages, bn = p.dec_bn;
+    const uint32_t stage_bytes = (uint32_t)p.dec_a_bytes + (uint32_t)bn * kBK;
+    // First column of tile n.  The last tile of a ragged N is moved back to end at N (it recomputes a few columns of
+    // its neighbour, same values): a box that hangs over the end of the tensor is filled in slowly, and the CTA
+    // that owns it finishes long after the others.
+    auto tile_col = [&](int n_blk) { return min(n_blk * bn, max(p.N - bn, 0)); };
+    auto full_bar = [&](int s) { return bar_base + 8u * s; };
+    auto empty_bar = [&](int s) { return bar_base + 8u * (kDecodeMaxStages + s); };
+    auto acc_full_bar = [&](int b) { return bar_base + 8u * (2 * kDecodeMaxStages + b); };
+    auto acc_empty_bar = [&](int b) { return bar_base + 8u * (2 * kDecodeMaxStages + 2 + b); };
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + (2 * kDecodeMaxStages + 4) * 8);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+    constexpr uint32_t kCols = 512;   // two accumulators of up to 256 columns
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+#ifdef FP8LIN_EXPERIMENTS
+    __shared__ unsigned trace_slot;
+    if (threadIdx.x == 0 && blockIdx.x == 0) {
+        trace_slot = atomicAdd(&g_trace_n, 1u) % 1024u;
+        g_trace[3 * trace_slot] = global_timer_ns();
+    }
+#endif
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < stages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(acc_full_bar(b), 1); mbar_init(acc_empty_bar(b), 4); }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) tmem_alloc(smem_u32(tmem_slot), kCols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    // whatever follows in the stream (the finalize kernel of a split launch, the next small cast) may take its places
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+
+    const int num_items = p.tiles_n * p.splits;
+    if (warp == 0) {
+        if (lane == 0) {
+            asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_a)) : "memory");
+            asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_b)) : "memory");
+            // every B byte is read once, every A byte by every CTA: B leaves L2 first, A stays
+            const uint64_t keep = l2_policy_evict_last(), drop = l2_policy_evict_first();
+            // Ahead of the dependency wait (the launch before this one is the small cast of the activation).  Where the
+            // caller vouches that the weight bytes were final before that launch began (inference on weights quantised
+            // once), the first ring of B tiles is loaded outright and two more rings are pulled towards L2: the weights
+            // stream while the launch before drains and the cast runs.  Otherwise the first ring is only pulled towards
+            // L2, which holds no stale data whoever writes those bytes.
+            const uint32_t tx_bytes = (uint32_t)p.a_box_bytes + (uint32_t)bn * kBK, a_bytes = (uint32_t)p.dec_a_bytes;
+            int early = 0;   // stages whose B tile is already on its way when the loop below starts
+            if ((int)blockIdx.x < num_items) {
+                const int n_blk = (int)blockIdx.x / p.splits, split0 = (int)blockIdx.x % p.splits;
+                const int k0 = split0 * p.kb_per_split, k1 = min(p.num_k, k0 + p.kb_per_split);
+                int k = k0 + first_kblock(0, n_blk, k1 - k0);
+                const int ring = min(k1 - k0, stages);
+                if (p.early_b) {
+                    for (int i = 0; i < ring; ++i, k = (k + 1 == k1) ? k0 : k + 1) {
+                        mbar_expect_tx(full_bar(i), tx_bytes);
+                        tma_load_2d_hint(stage_base + i * stage_bytes + a_bytes, &map_b, full_bar(i), k * kBK, tile_col(n_blk), drop);
+                    }
+                    early = ring;
+                    for (int i = ring; i < min(k1 - k0, 3 * stages); ++i, k = (k + 1 == k1) ? k0 : k + 1)
+                        tma_prefetch_l2_2d(&map_b, k * kBK, tile_col(n_blk));
+                } else {
+                    for (int i = 0; i < ring; ++i, k = (k + 1 == k1) ? k0 : k + 1)
+                        tma_prefetch_l2_2d(&map_b, k * kBK, tile_col(n_blk));
+                }
+            }
+            asm volatile("griddepcontrol.wait;" ::: "memory");
+#ifdef FP8LIN_EXPERIMENTS
+            if (blockIdx.x == 0) g_trace[3 * trace_slot + 1] = global_timer_ns();
+#endif
+            // One thread runs this loop and its latency is the ceiling of what a CTA can stream (a division per k-block
+            // was measured to hold a CTA at 0.25 us per k-block with no loads at all): stage index, phase and
+            // addresses advance by increments.
+            int s = 0;
+            uint32_t ph = 0, full = full_bar(0), empty = empty_bar(0), a_dst = stage_base;
+            bool alive = true;
+            for (int item = blockIdx.x; alive && item < num_items; item += gridDim.x) {
+                const int n_blk = item / p.splits, split = item % p.splits;
+                const int k0 = split * p.kb_per_split, k1 = min(p.num_k, k0 + p.kb_per_split);
+                const int b_row = tile_col(n_blk);
+                // the k-blocks are walked in a rotated order that differs from tile to tile, so that the CTAs do not
+                // all ask L2 for the same few lines of A at the same time
+                int k = k0 + first_kblock(0, n_blk, k1 - k0);
+                for (int i = k1 - k0; i > 0; --i) {
+                    if (!mbar_wait(empty, ph ^ 1u, abort_flag, p.d_status)) { alive = false; break; }
+#ifdef FP8LIN_EXPERIMENTS
+                    if (p.dbg == 5) mbar_arrive(full);   // timing only: no loads
+                    else
+#endif
+                    if (early > 0) {   // announced and half loaded before the dependency wait
+                        --early;
+                        tma_load_2d_hint(a_dst, &map_a, full, k * kBK, 0, keep);
+                    } else {
+                        mbar_expect_tx(full, tx_bytes);
+                        tma_load_2d_hint(a_dst, &map_a, full, k * kBK, 0, keep);
+                        tma_load_2d_hint(a_dst + a_bytes, &map_b, full, k * kBK, b_row, drop);
+                    }
+                    k = (k + 1 == k1) ? k0 : k + 1;
+                    if (++s == stages) {
+                        s = 0; ph ^= 1u; full = full_bar(0); empty = empty_bar(0); a_dst = stage_base;
+                    } else {
+                        full += 8u; empty += 8u; a_dst += stage_bytes;
+                    }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            uint32_t t = 0;
+            bool alive = true;
+            // the bounded waits below start counting only once the launch before this one has completed
+            asm volatile("griddepcontrol.wait;" ::: "memory");
+            const uint64_t desc0 = smem_desc_k128(0);   // everything but the address field
+            const uint32_t a_step = stage_bytes >> 4, b_off = (uint32_t)p.dec_a_bytes >> 4;
+            int s = 0;
+            uint32_t ph = 0, full = full_bar(0), empty = empty_bar(0), a16 = stage_base >> 4;   // addresses in 16-byte units
+            for (int item = blockIdx.x; alive && item < num_items; item += gridDim.x, ++t) {
+                const int split = item % p.splits;
+                const int k0 = split * p.kb_per_split, k1 = min(p.num_k, k0 + p.kb_per_split);
+                const int buf = t & 1;
+                const uint32_t acc_ph = (t >> 1) & 1u;
+                if (!mbar_wait(acc_empty_bar(buf), acc_ph ^ 1u, abort_flag, p.d_status)) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + buf * 256;
+                uint32_t accumulate = 0;
+                for (int i = k1 - k0; i > 0; --i) {
+                    if (!mbar_wait(full, ph, abort_flag, p.d_status)) { alive = false; break; }
+                    tc_fence_after();
+#ifdef FP8LIN_EXPERIMENTS
+                    if (p.dbg == 1 || p.dbg == 5) mbar_arrive(empty);   // timing only: no MMA at all
+                    else
+#endif
+                    {
+                        const uint64_t da = desc0 | (uint64_t)a16, db = desc0 | (uint64_t)(a16 + b_off);
+#pragma unroll
+                        for (int j = 0; j < kBK / kUmmaK; ++j) {   // 32 bytes along a 128-byte row per instruction
+                            umma_f8(d_tmem, da + 2u * j, db + 2u * j, p.idesc, accumulate);
+                            accumulate = 1u;
+                        }
+                        umma_commit(empty);
+                    }
+                    if (++s == stages) {
+                        s = 0; ph ^= 1u; full = full_bar(0); empty = empty_bar(0); a16 = stage_base >> 4;
+                    } else {
+                        full += 8u; empty += 8u; a16 += a_step;
+                    }
+                }
+                if (alive) umma_commit(acc_full_bar(buf));
+            }
+        }
+    } else {
+        asm volatile("griddepcontrol.wait;" ::: "memory");  // the biases may come from the launch before this one
+        const int q = warp & 3;  // TMEM lane quarter this warp may address
+        const int e = -(__ldg(p.d_sa) + __ldg(p.d_sb) + p.delta_sum);
+        const Pow2Pair sc = make_pow2_pair(e), sc_one = make_pow2_pair(0);
+        const bool two_step = (e < -126 || e > 127);
+        uint32_t amax_bits = 0, t = 0;
+        GemmParams pp = p;   // what store_direct sees: the tile's own column range, the partial-sum plane of a split
+        if (p.splits > 1) {
+            pp.out_dt = FP8_F32;
+            pp.bias_vec = nullptr;
+            pp.d_amax_bits = nullptr;
+            pp.vec_ok = (p.N % 4) == 0;
+        }
+        for (int item = blockIdx.x; item < num_items; item += gridDim.x, ++t) {
+            const int n_blk = item / p.splits, split = item % p.splits;
+            if (p.splits > 1) pp.out = p.partial + (int64_t)split * p.M * p.N;
+            const int col_base = tile_col(n_blk);
+            pp.N = min(p.N, col_base + bn);   // columns beyond the tile belong to the next one ...
+            pp.col_lo = n_blk * bn;           // ... and those a moved-back last tile recomputes, to the one before
+            const int buf = t & 1;
+            const uint32_t acc_ph = (t >> 1) & 1u;
+            const bool ready = mbar_wait(acc_full_bar(buf), acc_ph, abort_flag, p.d_status);
+            if (!__all_sync(0xFFFFFFFFu, ready)) break;
+            tc_fence_after();
+            const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + buf * 256;
+            if (p.dec_cluster > 1) break;   // the accumulator stays where it is for the exchange below
+            if (q * 32 < p.M) {   // a warp none of whose rows exists reads nothing
+#pragma unroll 1
+                for (int c = 0; c < bn; c += 32) {
+                    uint32_t r[32];
+                    tmem_ld_x32(t_row + c, r);
+                    tmem_ld_wait();
+                    store_direct(r, q * 32 + lane, col_base + c, pp, p.splits > 1 ? sc_one : sc,
+                                 p.splits > 1 ? false : two_step, amax_bits);
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(acc_empty_bar(buf));
+        }
+        if (p.d_amax_bits && p.splits == 1 && p.dec_cluster <= 1) {
+            amax_bits = __reduce_max_sync(0xFFFFFFFFu, amax_bits);
+            if (lane == 0 && amax_bits) atomicMax(p.d_amax_bits, amax_bits);
+        }
+    }
+
+    __syncwarp();  // the single-lane roles rejoin their warps before the block-wide barrier
+    if (p.dec_cluster > 1) {
+        // Every CTA of the cluster holds the sum over its slice of the contraction in accumulator 0 (its epilogue warps
+        // have seen "accumulator full", or given up).  Rank r > 0 writes rows [0, M) of it to plane r - 1 of a buffer at
+        // the start of the leader's stages, [plane][row][bn floats].
+        const uint32_t rank = cluster_ctarank();
+        const int q = warp & 3, row = q * 32 + lane;
+        const bool epi = warp >= 2, has_rows = q * 32 < p.M;
+        const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16);
+        const uint32_t plane_bytes = (uint32_t)p.M * (uint32_t)bn * 4u;
+        cluster_sync_all();   // all slices summed; the leader's stages are no longer read or written
+        if (epi && rank != 0 && has_rows && !*abort_flag) {
+            const uint32_t dst_row = map_to_cta(stage_base, 0) + (rank - 1) * plane_bytes + (uint32_t)row * (uint32_t)bn * 4u;
+#pragma unroll 1
+            for (int c = 0; c < bn; c += 32) {
+                uint32_t r[32];
+                tmem_ld_x32(t_row + c, r);
+                tmem_ld_wait();
+                if (row < p.M) {
+#pragma unroll
+                    for (int j = 0; j < 8; ++j)
+                        if (c + 4 * j < bn)
+                            asm volatile("st.shared::cluster.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst_row + (uint32_t)(c + 4 * j) * 4u),
+                                         "r"(r[4 * j]), "r"(r[4 * j + 1]), "r"(r[4 * j + 2]), "r"(r[4 * j + 3]) : "memory");
+                }
+            }
+        }
+        cluster_sync_all();   // the planes are written (release / acquire across the cluster)
+        if (epi && rank == 0 && has_rows && !*abort_flag) {
+            const int e = -(__ldg(p.d_sa) + __ldg(p.d_sb) + p.delta_sum);
+            const Pow2Pair sc = make_pow2_pair(e);
+            const bool two_step = (e < -126 || e > 127);
+            const int n_blk = (int)blockIdx.x / p.splits;
+            GemmParams pp = p;
+            const int col_base = tile_col(n_blk);
+            pp.N = min(p.N, col_base + bn);
+            pp.col_lo = n_blk * bn;
+            uint32_t amax_bits = 0;
+            const uint32_t src_row = stage_base + (uint32_t)row * (uint32_t)bn * 4u;
+#pragma unroll 1
+            for (int c = 0; c < bn; c += 32) {
+                uint32_t r[32];
+                tmem_ld_x32(t_row + c, r);
+                tmem_ld_wait();
+                if (row < p.M) {
+                    for (int pl = 0; pl < p.dec_cluster - 1; ++pl) {   // rank order: the sum does not depend on timing
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) {
+                            if (c + 4 * j < bn) {
+                                float4 v;
+                                asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
+                                             : "r"(src_row + (uint32_t)pl * plane_bytes + (uint32_t)(c + 4 * j) * 4u));
+                                r[4 * j] = __float_as_uint(__uint_as_float(r[4 * j]) + v.x);
+                                r[4 * j + 1] = __float_as_uint(__uint_as_float(r[4 * j + 1]) + v.y);
+                                r[4 * j + 2] = __float_as_uint(__uint_as_float(r[4 * j + 2]) + v.z);
+                                r[4 * j + 3] = __float_as_uint(__uint_as_float(r[4 * j + 3]) + v.w);
+                            }
+                        }
+                    }
+                }
+                store_direct(r, row, col_base + c, pp, sc, two_step, amax_bits);
+            }
+            if (p.d_amax_bits) {
+                amax_bits = __reduce_max_sync(0xFFFFFFFFu, amax_bits);
+                if (lane == 0 && amax_bits) atomicMax(p.d_amax_bits, amax_bits);
+            }
+        }
+    }
+    if (*abort_flag) __nanosleep(20000);  // let copies and MMAs already issued drain before the memory is released
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    if (warp == 1) tmem_dealloc(tmem_base, kCols);
+#ifdef FP8LIN_EXPERIMENTS
+    if (threadIdx.x == 0 && blockIdx.x == 0) g_trace[3 * trace_slot + 2] = global_timer_ns();
+#endif
 }
 
 
@@ -1221,23 +1569,6 @@ using PairSmemAct = PairSmemT<kPairStagesAct, kActSlabs>;
 constexpr int kWideStages = 4;
 using PairSmemWide = PairSmemT<kWideStages, kPairSlabs, 2>;
 
-__device__ __forceinline__ uint32_t cluster_ctarank()
-{
-    uint32_t r;
-    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
-    return r;
-}
-__device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t rank)
-{
-    uint32_t r;
-    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank));
-    return r;
-}
-__device__ __forceinline__ void cluster_sync_all()
-{
-    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
-    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
 // arrive (+ expected bytes) on a barrier addressed in the cluster window
 __device__ __forceinline__ void mbar_expect_tx_cluster(uint32_t cluster_bar, uint32_t bytes)
 {
@@ -1604,6 +1935,13 @@ static bool g_no_splitk = false;        // set from FP8LIN_NO_SPLITK=1
 static int g_force_splits = 0;          // set from FP8LIN_SPLITS (experiments with the split count)
 static bool g_no_pdl = false;           // set from FP8LIN_NO_PDL=1 (A/B: matmuls launched without programmatic dependence)
 static bool g_direct_epilogue = false;  // set from FP8LIN_DIRECT_EPILOGUE=1 (A/B comparison of the epilogues)
+constexpr int kDecodeMaxCluster = 8;
+static int g_decode_clusters[kDecodeMaxCluster + 1] = {0};   // clusters of each size that can be resident at once
+static bool g_no_decode_cluster = false; // set from FP8LIN_DECODE_CLUSTER=0 (A/B: split contractions through global memory only)
+static bool g_no_early_b = false;        // set from FP8LIN_EARLY_B=0 (A/B: fp8_linear_infer without its early weight loads)
+static bool g_no_decode_kernel = false; // set from FP8LIN_DECODE_KERNEL=0 (A/B: decode shapes on the fixed-width single-CTA kernel)
+static int g_dbg = 0;                   // set from FP8LIN_DECODE_DBG (timing-only variants of the decode kernel)
+static int g_force_bn = 0;              // set from FP8LIN_DECODE_BN (experiments with the decode tile width)
 static bool g_no_out_stream = false;    // set from FP8LIN_OUT_STREAM=0 (A/B: output stores without the evict-first mark)
 static bool g_no_serpentine = false;    // set from FP8LIN_SERPENTINE=0 (A/B: every tile walks the contraction forwards)
 static int g_force_wide = -1;           // set from FP8LIN_WIDE=0/1 (A/B: never / always the 256 x 512 pair tile)
@@ -1629,6 +1967,7 @@ static cudaError_t set_smem_attributes()
     if (e == cudaSuccess && ACT == 0)
         e = cudaFuncSetAttribute(gemm_pair_kernel<0, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  PairSmemWide::kDynamic);
+
     return e;
 }
 
@@ -1637,7 +1976,8 @@ cudaError_t configure_gemm_kernels(int max_smem_optin)
     using L = GemmSmem<kBN, kStages>;
     using LA = GemmSmem<kBN, kStagesAct, kActSlabs>;
     if (L::kDynamic > max_smem_optin || PairSmem::kDynamic > max_smem_optin || LA::kDynamic > max_smem_optin ||
-        PairSmemAct::kDynamic > max_smem_optin || PairSmemWide::kDynamic > max_smem_optin)
+        PairSmemAct::kDynamic > max_smem_optin || PairSmemWide::kDynamic > max_smem_optin ||
+        kDecodeSmemBudget + 1024 > max_smem_optin)
         return cudaErrorInvalidValue;
     cudaError_t e = set_smem_attributes<0>();
     if (e == cudaSuccess) e = set_smem_attributes<1>();
@@ -1648,7 +1988,28 @@ cudaError_t configure_gemm_kernels(int max_smem_optin)
     if (e == cudaSuccess)
         e = cudaFuncSetAttribute(gemm_kernel<kBN, kStagesF16Acc, 6>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  GemmSmem<kBN, kStagesF16Acc, kActSlabs>::kDynamic);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecodeSmemBudget + 1024);
     if (e != cudaSuccess) return e;
+    for (int cs = 2; cs <= kDecodeMaxCluster; ++cs) {   // how many clusters of each size fit the GPU at once
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = (unsigned)cs;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)(cs * 64));
+        cfg.blockDim = dim3(kGemmThreads);
+        cfg.dynamicSmemBytes = kDecodeSmemBudget + 1024;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        int n = 0;
+        if (cudaOccupancyMaxActiveClusters(&n, decode_kernel, &cfg) != cudaSuccess) {
+            (void)cudaGetLastError();
+            n = 0;
+        }
+        g_decode_clusters[cs] = n;
+    }
     int sms = 0, dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess ||
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
@@ -1675,6 +2036,16 @@ cudaError_t configure_gemm_kernels(int max_smem_optin)
     g_force_single = env && env[0] == '1';
     env = getenv("FP8LIN_GROUP_M");
     g_group_m = env ? atoi(env) : 0;
+    env = getenv("FP8LIN_DECODE_CLUSTER");
+    g_no_decode_cluster = env && env[0] == '0';
+    env = getenv("FP8LIN_EARLY_B");
+    g_no_early_b = env && env[0] == '0';
+    env = getenv("FP8LIN_DECODE_KERNEL");
+    g_no_decode_kernel = env && env[0] == '0';
+    env = getenv("FP8LIN_DECODE_DBG");
+    g_dbg = env ? atoi(env) : 0;
+    env = getenv("FP8LIN_DECODE_BN");
+    g_force_bn = env ? atoi(env) : 0;
     env = getenv("FP8LIN_OUT_STREAM");
     g_no_out_stream = env && env[0] == '0';
     env = getenv("FP8LIN_SERPENTINE");
@@ -1724,6 +2095,93 @@ static bool use_wide_tile(int64_t M, int64_t N, int64_t Kc)
     return kWideTileDefault && Kc >= 2048 && no_extra_wave && little_waste;
 }
 
+// Tile width, split count and stage count of a decode launch, by a time model (microseconds) fitted to measured
+// launches of the four layers of a 70B-class decoder block at 1 and 64 rows.  Items (tile, slice of the contraction)
+// are dealt round-robin, so the CTAs hold q or q + 1 of them: all stream q items together, then the few with one more
+// finish alone.  A CTA streaming among `a` active ones moves bytes at 1 / (1 / solo + a / total): about 42 GB/s each
+// with all 148 pulling (6.2 TB/s together), and no more than its own pipeline allows however few remain, which is why
+// a last wave with a handful of items costs almost as much as a full one and why the width is chosen to give close
+// to a whole number of tiles per SM.  A split contraction adds the finalize launch and the trip of the FP32 partial
+// sums to memory and back; every item costs a little set-up.
+// The contraction of a tile can also be split across the CTAs of a cluster, which exchange their sums through shared
+// memory (no partial sums in global memory, no second launch): one tile per cluster, as many clusters as can be
+// resident, the exchange buffer inside the leader's stages.
+static void choose_decode(const fp8_ctx *ctx, int64_t M, int64_t N, int num_k, int a_bytes, int *bn_out, int *kb_out,
+                          int *stages_out, int *cluster_out)
+{
+    const int sms = ctx->sm_count;
+    const double solo0 = 180e3, total = 8e6;   // bytes per microsecond
+    const double finalize_us = 3.5, partial_rate = 3.8e6, item_us = 0.15, exchange_us = 1.0, exchange_rate = 50e3;
+    // whatever its width, a k-block costs the two single-thread loops (wait, two loads / wait, four MMAs, commit) this much
+    const double kblock_us = 0.36;
+    const int64_t by_ws = (int64_t)(ctx->partial_bytes / sizeof(float)) / (M * N);
+    int64_t cap = num_k / 4 < by_ws ? num_k / 4 : by_ws;
+    if (cap > 64) cap = 64;
+    if (cap < 1 || g_no_splitk) cap = 1;
+    double best = 0;
+    *bn_out = 0;
+    for (int bn = 32; bn <= 256; bn += 16) {
+        const int stage = a_bytes + bn * kBK;
+        int stages = (kDecodeSmemBudget - kDecodeHeader - kBM * kBK) / stage;   // 16 KB spare: the A rows read past a stage
+        if (stages > kDecodeMaxStages) stages = kDecodeMaxStages;
+        if (stages < 3) continue;
+        const double in_flight = (double)stages * bn * kBK;
+        const double solo = solo0 * (in_flight < 192.0 * 1024 ? in_flight / (192.0 * 1024) : 1.0);
+        auto rate = [&](double active) { return 1.0 / (1.0 / solo + active / total); };
+        const int64_t tiles = (N + bn - 1) / bn;
+        for (int64_t sp = 1; sp <= cap; ++sp) {
+            const int64_t kb = (num_k + sp - 1) / sp;
+            const int64_t real = (num_k + kb - 1) / kb;
+            if (real != sp) continue;
+            if (g_force_splits > 0 && real != (g_force_splits < cap ? g_force_splits : cap)) continue;
+            if (g_force_bn > 0 && bn != g_force_bn) continue;
+            const int64_t items = tiles * real;
+            const double item_bytes = (double)kb * bn * kBK;
+            const int64_t q = items / sms, extra = items % sms;
+            const double floor_us = (double)kb * kblock_us;
+            auto item_time = [&](double active) { const double t = item_bytes / rate(active); return t > floor_us ? t : floor_us; };
+            double cost = q > 0 ? (double)q * item_time((double)sms) : 0.0;
+            if (extra > 0) cost += item_time((double)extra);
+            cost += item_us * (double)(q + (extra > 0 ? 1 : 0));
+            if (bn % 32) cost += 0.3;   // the last half chunk of a tile is stored element by element
+            if (real > 1) cost += finalize_us + 8.0 * (double)real * (double)M * (double)N / partial_rate;
+            if (*bn_out == 0 || cost < best) {
+                best = cost;
+                *bn_out = bn;
+                *kb_out = (int)kb;
+                *stages_out = stages;
+                *cluster_out = 1;
+            }
+        }
+        for (int cs = 2; cs <= kDecodeMaxCluster && !g_no_decode_cluster; ++cs) {
+            const int64_t kb = (num_k + cs - 1) / cs;
+            if ((num_k + kb - 1) / kb != cs || kb < 4) continue;
+            if (tiles > g_decode_clusters[cs]) continue;
+            if ((int64_t)(cs - 1) * M * bn * 4 > (int64_t)stages * stage) continue;   // the exchange buffer
+            if (g_force_splits > 0 && cs != g_force_splits) continue;
+            if (g_force_bn > 0 && bn != g_force_bn) continue;
+            const double item_bytes = (double)kb * bn * kBK;
+            double cost = item_bytes / rate((double)(tiles * cs));
+            if (cost < (double)kb * kblock_us) cost = (double)kb * kblock_us;
+            cost += item_us + exchange_us + (double)(cs - 1) * (double)M * bn * 4.0 / exchange_rate;
+            if (bn % 32) cost += 0.3;
+            if (*bn_out == 0 || cost < best) {
+                best = cost;
+                *bn_out = bn;
+                *kb_out = (int)kb;
+                *stages_out = stages;
+                *cluster_out = cs;
+            }
+        }
+    }
+    if (*bn_out == 0) {   // nothing matched a forced count: one tile of 256 columns per item, unsplit
+        *bn_out = 256;
+        *cluster_out = 1;
+        *kb_out = num_k;
+        *stages_out = (kDecodeSmemBudget - kDecodeHeader - kBM * kBK) / (a_bytes + 256 * kBK);
+    }
+}
+
 // D[M,N] = A * B^T over a contraction of length Kc, unscaled by 2^-(bias_a + bias_b + delta_sum).
 // A is stored [M, Kc] (a_mn = false) or [Kc, M] (a_mn = true); B is stored [N, Kc] or [Kc, N] likewise.
 static fp8_status_t run_gemm(fp8_ctx *ctx, const uint8_t *a, int a_fmt, bool a_mn, const int32_t *d_ba,
@@ -1731,7 +2189,7 @@ static fp8_status_t run_gemm(fp8_ctx *ctx, const uint8_t *a, int a_fmt, bool a_m
                              const void *bias_vec, int bias_dt, void *out, int out_dt, float *d_amax_out, int64_t M,
                              int64_t N, int64_t Kc, cudaStream_t st, int act = 0, void *out_act = nullptr,
                              const void *aux = nullptr, uint8_t *out8 = nullptr, const int32_t *d_sq = nullptr,
-                             int q_fmt = 0, int delta_q = 0, bool no_loads = false, int chunk_kb = 0)
+                             int q_fmt = 0, int delta_q = 0, bool no_loads = false, int chunk_kb = 0, bool static_b = false)
 {
     if (M > 0x7FFFFFFF / 2 || N > 0x7FFFFFFF / 2 || Kc > 0x7FFFFFFF / 2) return FP8_ERR_SHAPE;
     const bool pair = g_max_pairs > 0 && M > kBM && !g_force_single && act != 6;
@@ -1741,11 +2199,28 @@ static fp8_status_t run_gemm(fp8_ctx *ctx, const uint8_t *a, int a_fmt, bool a_m
     // rows of the stage keep whatever they held and feed output rows that are never stored.  (A 128-row box on a
     // one-row tensor cost 6 us of a 89 us launch, and 59 us for some placements of the activation in memory.)
     const int a_box_rows = (!pair && !a_mn && M < kBM) ? (int)((M + 7) / 8 * 8) : kBM;
+    // at most 128 rows, both operands contraction-major, plain epilogue: the decode kernel, tile width chosen here
+    const bool decode = !pair && !a_mn && !b_mn && act == 0 && M <= kBM && !g_no_decode_kernel && !no_loads;
+    GemmParams p;
+    p.dec_bn = p.dec_stages = p.dec_a_bytes = 0;
+    p.dec_cluster = 1;
+    p.col_lo = 0;
+    p.early_b = (decode && static_b && !g_no_early_b) ? 1 : 0;
+    p.dbg = g_dbg;
+    int dec_kb = 0;
+    if (decode) {
+        p.dec_a_bytes = a_box_rows * kBK;
+        choose_decode(ctx, M, N, (int)((Kc + kBK - 1) / kBK), p.dec_a_bytes, &p.dec_bn, &dec_kb, &p.dec_stages, &p.dec_cluster);
+#ifdef FP8LIN_EXPERIMENTS
+        if (getenv("FP8LIN_DEBUG"))
+            fprintf(stderr, "fp8lin decode M=%lld N=%lld K=%lld: bn %d, %d k-blocks per item, %d stages, cluster %d\n",
+                    (long long)M, (long long)N, (long long)Kc, p.dec_bn, dec_kb, p.dec_stages, p.dec_cluster);
+#endif
+    }
     const bool ok_a = a_mn ? encode_map(ctx, &map_a, a, Kc, M, kBK) : encode_map(ctx, &map_a, a, M, Kc, a_box_rows);
     const bool ok_b = b_mn ? encode_map(ctx, &map_b, b, Kc, N, kBK)
-                           : encode_map(ctx, &map_b, b, N, Kc, pair ? kPairHalfN : kBN);
+                           : encode_map(ctx, &map_b, b, N, Kc, decode ? p.dec_bn : (pair ? kPairHalfN : kBN));
     if (!ok_a || !ok_b) return FP8_ERR_CUDA;
-    GemmParams p;
     p.group_m = g_group_m > 0 ? g_group_m : kGroupM;
     p.serpentine = g_no_serpentine ? 0 : 1;
     p.out_stream = (!g_no_out_stream && (int64_t)M * N * (out_dt == FP8_F32 ? 4 : 2) >= kStreamOutBytes) ? 1 : 0;
@@ -1767,33 +2242,41 @@ static fp8_status_t run_gemm(fp8_ctx *ctx, const uint8_t *a, int a_fmt, bool a_m
         p.kb_per_split = chunk_kb > 0 ? chunk_kb : 1;
         p.splits = (p.num_k + p.kb_per_split - 1) / p.kb_per_split;
     }
-    if (!pair && !g_no_splitk && !act) {
+    if (decode) {
+        p.tiles_n = (int)((N + p.dec_bn - 1) / p.dec_bn);
+        p.kb_per_split = dec_kb;
+        p.splits = (p.num_k + dec_kb - 1) / dec_kb;
+    }
+    if (!pair && !decode && !g_no_splitk && !act) {
         const int64_t tiles = (int64_t)p.tiles_m * p.tiles_n;
         if (tiles < 2 * ctx->sm_count && p.num_k >= 8) {
-            // Pick the split count by a byte model of the launch, in bytes at the HBM rate.  The weights stream once
-            // (one B tile of BN x 128 bytes per k-block; the A tile is a few rows) and every split writes and
-            // re-reads an FP32 partial tile: that is the floor when all SMs pull together.  One SM alone draws at
-            // most about 1.6 times its fair share of the HBM rate (measured: 32 to 40 CTAs streaming 2 MB each),
-            // so the busiest CTA's bytes set a second floor, which is what splitting lowers.  Each wave of items
-            // has a fixed set-up cost and splitting at all costs the finalize launch.
+            // Pick the split count by a time model of the launch (microseconds), fitted to measured launches of the
+            // four decode layers of a 70B-class model at 1 and 64 rows, 1 to 12 splits.  Items are dealt round-robin,
+            // so the CTAs hold q or q + 1 items: all stream q items together, then the few with one more finish alone.
+            // A CTA streaming among `a` active ones moves bytes at 1 / (1 / solo + a / total): about 42 GB/s each
+            // with all 148 pulling (6.2 TB/s together), and no more than its own pipeline allows however few remain
+            // (which is why a last wave with a handful of items costs almost as much as a full one).  A split
+            // launch adds the finalize kernel and the trip of the FP32 partial sums to memory and back.
             const int64_t by_k = p.num_k / 4;
             const int64_t by_ws = (int64_t)(ctx->partial_bytes / sizeof(float)) / (M * N);
             int64_t cap = by_k < by_ws ? by_k : by_ws;
             if (cap > 64) cap = 64;
             const double sms = (double)ctx->sm_count;
-            const double kb_bytes = (double)kBN * kBK, wave_bytes = 3.5e6, finalize_bytes = 24.0e6, solo = 1.6;
-            const double weights = (double)tiles * p.num_k * kb_bytes;
+            const double solo = 180e3, total = 8e6;            // bytes per microsecond
+            const double finalize_us = 1.0, partial_rate = 3.8e6;
+            auto rate = [&](double active) { return 1.0 / (1.0 / solo + active / total); };
             double best = 0;
             int64_t best_kb = p.num_k;
             for (int64_t sp = 1; sp <= cap; ++sp) {
                 const int64_t kb = (p.num_k + sp - 1) / sp;
                 const int64_t real = (p.num_k + kb - 1) / kb;
                 if (real != sp) continue;
-                const int64_t waves = (tiles * real + ctx->sm_count - 1) / ctx->sm_count;
-                const double partials = real > 1 ? 8.0 * (double)real * (double)M * (double)N : 0.0;
-                const double busiest = (double)waves * (double)kb * kb_bytes * sms / solo;
-                double cost = (weights + partials > busiest ? weights + partials : busiest) + (double)waves * wave_bytes;
-                if (real > 1) cost += finalize_bytes;
+                const int64_t items = tiles * real;
+                const double item_bytes = (double)kb * kBN * kBK;
+                const int64_t q = items / ctx->sm_count, extra = items % ctx->sm_count;
+                double cost = q > 0 ? (double)q * item_bytes / rate(sms) : 0.0;
+                if (extra > 0) cost += item_bytes / rate((double)extra);
+                if (real > 1) cost += finalize_us + 8.0 * (double)real * (double)M * (double)N / partial_rate;
                 if (sp == 1 || cost < best) {
                     best = cost;
                     best_kb = kb;
@@ -1829,7 +2312,7 @@ static fp8_status_t run_gemm(fp8_ctx *ctx, const uint8_t *a, int a_fmt, bool a_m
     p.out = out; p.out_dt = out_dt; p.ldo = N;
     const int64_t esz = out_dt == FP8_BF16 ? 2 : 4;
     p.vec_ok = ((reinterpret_cast<uintptr_t>(out) & 15u) == 0 && (N * esz) % 16 == 0) ? 1 : 0;
-    p.tma_out = (p.vec_ok && !g_direct_epilogue) ? 1 : 0;
+    p.tma_out = (p.vec_ok && !g_direct_epilogue && !decode) ? 1 : 0;
     p.act = act;
     p.aux = aux;
     p.has_out2 = out_act ? 1 : 0;
@@ -1865,11 +2348,12 @@ static fp8_status_t run_gemm(fp8_ctx *ctx, const uint8_t *a, int a_fmt, bool a_m
     }
     p.d_amax_bits = reinterpret_cast<unsigned *>(d_amax_out);
     p.d_status = ctx->d_status;
-    p.idesc = (pair ? make_idesc_pair(a_fmt, b_fmt) : make_idesc(a_fmt, b_fmt, kBN)) | ((uint32_t)p.a_mn << 15) |
+    p.idesc = (pair ? make_idesc_pair(a_fmt, b_fmt) : make_idesc(a_fmt, b_fmt, decode ? p.dec_bn : kBN)) | ((uint32_t)p.a_mn << 15) |
               ((uint32_t)p.b_mn << 16);
     if (d_amax_out && cudaMemsetAsync(d_amax_out, 0, sizeof(float), st) != cudaSuccess) return FP8_ERR_CUDA;
     int tiles = p.tiles_m * p.tiles_n;
-    count_launch(p.splits > 1 && act != 6 ? 2 : 1);
+    const bool finalize = p.splits > 1 && act != 6 && p.dec_cluster <= 1;
+    count_launch(finalize ? 2 : 1);
     if (pair) {
         const int items = tiles * p.splits;
         int pairs = items < g_max_pairs ? items : g_max_pairs;
@@ -1897,6 +2381,24 @@ static fp8_status_t run_gemm(fp8_ctx *ctx, const uint8_t *a, int a_fmt, bool a_m
             break;
         }
         }
+    } else if (decode) {
+        const int items = p.tiles_n * p.splits;
+        cudaLaunchAttribute attr[2];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = (unsigned)p.dec_cluster;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[1].val.programmaticStreamSerializationAllowed = 1;
+        cudaLaunchConfig_t cfg = {};
+        // a cluster launch has one item per CTA (the clusters fit the GPU at once, by choose_decode)
+        cfg.gridDim = dim3((unsigned)(p.dec_cluster > 1 ? items : (items < ctx->sm_count ? items : ctx->sm_count)));
+        cfg.blockDim = dim3(kGemmThreads);
+        cfg.dynamicSmemBytes = kDecodeSmemBudget + 1024;
+        cfg.stream = st;
+        cfg.attrs = attr;
+        cfg.numAttrs = g_no_pdl ? 1 : 2;
+        if (cudaLaunchKernelEx(&cfg, decode_kernel, map_a, map_b, p) != cudaSuccess) return FP8_ERR_CUDA;
     } else {
         int items = act == 6 ? tiles : tiles * p.splits;
         int grid = items < ctx->sm_count ? items : ctx->sm_count;
@@ -1926,7 +2428,7 @@ static fp8_status_t run_gemm(fp8_ctx *ctx, const uint8_t *a, int a_fmt, bool a_m
         }
         }
     }
-    if (p.splits > 1 && act != 6) {
+    if (finalize) {
         if (cudaGetLastError() != cudaSuccess) return FP8_ERR_CUDA;
         const bool vec = p.vec_ok && (N % 4) == 0;
         int64_t threads = vec ? M * N / 4 : M * N;
@@ -1971,6 +2473,38 @@ fp8_status_t fp8_linear_fwd(fp8_ctx *ctx, const uint8_t *x8, const int32_t *d_bx
     return run_gemm(ctx, x8, FP8_E4, false, d_bx, w8, FP8_E4, false, d_bw, delta, bias_vec, bias_dt, y, y_dt, d_amax_y,
                     T, N, K, (cudaStream_t)stream);
 }
+
+fp8_status_t fp8_linear_infer(fp8_ctx *ctx, const uint8_t *x8, const int32_t *d_bx, const uint8_t *w8,
+                              const int32_t *d_bw, const void *bias_vec, fp8_dtype_t bias_dt, void *y,
+                              fp8_dtype_t y_dt, float *d_amax_y, int64_t T, int64_t K, int64_t N, fp8_conv_t conv,
+                              void *stream)
+{
+    using namespace fp8lin;
+    if (!ctx || !x8 || !d_bx || !w8 || !d_bw || !y) return FP8_ERR_NULL;
+    if ((int)conv < 0 || (int)conv > 1 || (int)y_dt < 0 || (int)y_dt > 2 || (int)bias_dt < 0 || (int)bias_dt > 2)
+        return FP8_ERR_DTYPE;
+    if (!out_dtype_ok(y_dt) || (bias_vec && !out_dtype_ok(bias_dt))) return FP8_ERR_UNSUPPORTED;
+    if (T <= 0 || K <= 0 || N <= 0) return FP8_ERR_SHAPE;
+    if (!aligned16(x8) || !aligned16(w8) || (K % 16) != 0 || (reinterpret_cast<uintptr_t>(y) & 3u)) return FP8_ERR_ALIGN;
+    int delta = 2 * format_delta(FP8_E4, conv);
+    return run_gemm(ctx, x8, FP8_E4, false, d_bx, w8, FP8_E4, false, d_bw, delta, bias_vec, bias_dt, y, y_dt, d_amax_y,
+                    T, N, K, (cudaStream_t)stream, 0, nullptr, nullptr, nullptr, nullptr, 0, 0, false, 0, true);
+}
+
+#ifdef FP8LIN_EXPERIMENTS
+__attribute__((visibility("default"))) int fp8_debug_trace(unsigned long long *host_out, int clear)
+{
+    unsigned n = 0;
+    cudaDeviceSynchronize();
+    cudaMemcpyFromSymbol(&n, fp8lin::g_trace_n, sizeof(n));
+    cudaMemcpyFromSymbol(host_out, fp8lin::g_trace, sizeof(unsigned long long) * 3 * 1024);
+    if (clear) {
+        unsigned zero = 0;
+        cudaMemcpyToSymbol(fp8lin::g_trace_n, &zero, sizeof(zero));
+    }
+    return (int)n;
+}
+#endif
 
 fp8_status_t fp8_selftest_mma_ceiling(fp8_ctx *ctx, void *out, const int32_t *d_zero, int64_t M, int64_t N, int64_t K,
                                       void *stream)

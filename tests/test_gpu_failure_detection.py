@@ -82,7 +82,7 @@ def test_matmuls_write_nothing_outside_their_outputs(ctx, lib, T, K, N):
 
 def test_launch_count_counts_what_a_call_enqueues(ctx, lib):
     """fp8_launch_count: two launches for amax + cast of a large tensor, one for a decode-size one, one for a cast
-    under a given bias, one or two for a matmul (two when the contraction is split)."""
+    under a given bias, one or two for a matmul (two when the contraction is split through memory)."""
     x = torch.randn(2048, 1024, device="cuda").to(torch.bfloat16)
     small = torch.randn(4, 1024, device="cuda").to(torch.bfloat16)
     y, ys = torch.empty((2048, 1024), dtype=torch.uint8, device="cuda"), torch.empty((4, 1024), dtype=torch.uint8, device="cuda")
@@ -102,7 +102,9 @@ def test_launch_count_counts_what_a_call_enqueues(ctx, lib):
     w_long = torch.zeros((512, 8192), dtype=torch.uint8, device="cuda")
     x_long = torch.zeros((4, 8192), dtype=torch.uint8, device="cuda")
     out2 = torch.empty((4, 512), dtype=torch.bfloat16, device="cuda")
-    assert span(lambda: ctx.linear_fwd(x_long, b, w_long, b, out2)) == 2       # two tiles, long contraction: split + finalize
+    # few tiles, long contraction: the contraction is split; one launch when the slices of a tile meet inside a
+    # cluster, two when the partial sums go through memory and a second kernel adds them
+    assert span(lambda: ctx.linear_fwd(x_long, b, w_long, b, out2)) in (1, 2)
     # the CTA-pair kernel splits too when tiles are few and the contraction is very long
     x_pair = torch.zeros((512, 16384), dtype=torch.uint8, device="cuda")
     w_pair = torch.zeros((512, 16384), dtype=torch.uint8, device="cuda")

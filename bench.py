@@ -278,11 +278,20 @@ def run_matmuls(ctx, L, timers=None):
             _timed(timers, "gemm", lambda: ctx.linear_wgrad(L.g8, None, bi[2:3], L.x8, None, bi[1:2], L.dw, L.T))
 
 
+def fused_decode(L):
+    """Forward-only layer on at most 128 rows: one launch quantises the activation and multiplies."""
+    return (not L.backward) and L.T <= 128 and not L.transposed and not NO_FUSED_DECODE
+
+
 def run_layer(ctx, L, timers=None, predict=False):
     """One layer of one step with every tensor quantised by its own call (two launches per tensor; one pass with
     predict=True when the bias left by the previous step still holds)."""
     af, bi = L.scal_f, L.scal_i
     E4, E5 = 0, 1
+    if fused_decode(L):
+        # inference on a few rows: the activation is quantised by the matmul's own launch (fp8_linear_infer_cast)
+        _timed(timers, "gemm", lambda: ctx.linear_infer_cast(L.x, af[1:2], bi[1:2], L.x8, L.w8, bi[0:1], L.y))
+        return
     if predict and not L.transposed:
         quant = lambda fmt, x, j, y, yt: ctx.cast_predicted(fmt, x, af[j:j + 1], bi[j:j + 1], y)
     else:
@@ -295,6 +304,8 @@ def run_layer(ctx, L, timers=None, predict=False):
         _timed(timers, "amax_cast", lambda: quant(E5, L.g, 2, L.g8, L.g8t))
     run_matmuls(ctx, L, timers)
 
+
+NO_FUSED_DECODE = False   # --no-fused-decode: decode layers as fp8_cast_e4 + fp8_linear_infer (two launches)
 
 QUANT_MODES = ("group-predicted", "group", "per-tensor", "per-tensor-predicted")
 
@@ -321,9 +332,11 @@ class Step:
             self.group_mode = fp8lin.GROUP_PREDICTED if mode == "group-predicted" else fp8lin.GROUP_AMAX_CAST
 
     def launches_per_step(self):
-        gemms = sum(3 if L.backward else 1 for L in self.layers)
-        tensors = sum(len(L.quant_items()) for L in self.layers)
-        return gemms + (2 if self.items is not None else 2 * tensors)
+        """Kernel launches the library enqueues per step, counted by the library itself (fp8_launch_count)."""
+        import paper_2309_17224_b200.fp8lin as lib
+        n0 = lib.launch_count()
+        self.run()
+        return lib.launch_count() - n0
 
     def run(self, timers=None):
         ctx = self.ctx
@@ -912,6 +925,8 @@ def main():
     ap.add_argument("--transposed-copies", action="store_true",
                     help="also write transposed FP8 copies and contract the backward matmuls over contiguous bytes "
                          "(per-tensor quantisation)")
+    ap.add_argument("--no-fused-decode", action="store_true",
+                    help="forward-only layers on at most 128 rows as fp8_cast_e4 + fp8_linear_infer instead of fp8_linear_infer_cast")
     ap.add_argument("--no-graph-leg", action="store_true", help="skip the extra timed loop that replays a CUDA graph")
     ap.add_argument("--no-extra-legs", action="store_true",
                     help="skip every leg beside the headline: other quantisation modes, moving gradients, sustained "
@@ -925,6 +940,8 @@ def main():
     ap.add_argument("--only", default=None, help="--leg stack: run only the variant whose name contains this")
     ap.add_argument("--plain-only", action="store_true", help="--leg gemm: skip the fused epilogues")
     args = ap.parse_args()
+    global NO_FUSED_DECODE
+    NO_FUSED_DECODE = args.no_fused_decode
     wl = I.WORKLOADS[args.workload]
     if args.impl == "reference":
         return reference_arm(args, wl)
@@ -1003,7 +1020,8 @@ def main():
     weight_bytes = float(sum(l.K * l.N for l in wl.layers))
     sm_count = torch.cuda.get_device_properties(local).multi_processor_count
     if decode:
-        roofline = {"bound": "hbm", "kernel": "gemm_kernel (+ splitk_finalize_kernel)",
+        roofline = {"bound": "hbm", "kernel": "decode_kernel (activation quantised in the same launch)" if fused_decode(layers[0])
+                    else "decode_kernel (+ splitk_finalize_kernel)",
                     "achieved": sampled_steps * weight_bytes / (gemm_ms * 1e-3) / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                     "peak_source": f"{peaks['source']} copy bandwidth", "launches": gemm_launches,
                     "avg_launch_ms": gemm_ms / max(1, gemm_launches),
@@ -1309,10 +1327,10 @@ def main():
         "e2e": e2e,
         "gpu_launches": launches_timed,
         "roofline": roofline,
-        "amax_cast": {"effective_gbs": cast_elems * bytes_per_elem / (cast_ms * 1e-3) / 1e9,
+        "amax_cast": {"effective_gbs": cast_elems * bytes_per_elem / (cast_ms * 1e-3) / 1e9 if cast_ms > 0 else None,
                       "bytes_per_element": bytes_per_elem, "ms_per_step": cast_ms / sampled_steps,
                       "hbm_peak_gbs": peaks["hbm_gbs"],
-                      "frac": cast_elems * bytes_per_elem / (cast_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                      "frac": cast_elems * bytes_per_elem / (cast_ms * 1e-3) / 1e9 / peaks["hbm_gbs"] if cast_ms > 0 else None,
                       "guesses_held_missed": list(guesses),
                       "note": "amax + bias + cast of every tensor of a step as timed inside the step (events on every "
                               "eighth step), against the 3 B/element a single pass must move; per_kernel holds each "

@@ -349,6 +349,20 @@ FP8_API fp8_status_t fp8_linear_infer(fp8_ctx *ctx, const uint8_t *x8, const int
                               fp8_dtype_t y_dt, float *d_amax_y, int64_t T, int64_t K, int64_t N, fp8_conv_t conv,
                               void *stream);
 
+/* Inference on a few rows in one launch (Section 3.1: the activation is quantised per call, the weights once):
+ * FP8-AMAX of the activation (Eq. 3, then Eq. 1 and the E4 cast) followed by the forward matmul.  Results are those
+ * of fp8_cast_e4 (d_bias = NULL, FP8-AMAX) followed by fp8_linear_infer, bit for bit: d_amax_x, d_bx and the bytes
+ * x8 [T, K] are outputs of this call (all three required; x8 16-byte aligned), y as in fp8_linear_fwd.
+ *   x    [T, K] contiguous, dtype x_dt
+ * With an activation of at most 64 KB (one row of 28672 elements, four rows of 8192), bf16 and 16-byte aligned, one
+ * kernel does both steps: every CTA takes the amax of the whole of x, derives the bias and casts x for itself (all
+ * write the same bytes to x8), then multiplies, while its weight tiles have been streaming since the kernel began.
+ * Any other case runs the two calls.  The condition of fp8_linear_infer on w8 applies. */
+FP8_API fp8_status_t fp8_linear_infer_cast(fp8_ctx *ctx, const void *x, fp8_dtype_t x_dt, int32_t margin, float *d_amax_x,
+                                   int32_t *d_bx, uint8_t *x8, const uint8_t *w8, const int32_t *d_bw,
+                                   const void *bias_vec, fp8_dtype_t bias_dt, void *y, fp8_dtype_t y_dt,
+                                   float *d_amax_y, int64_t T, int64_t K, int64_t N, fp8_conv_t conv, void *stream);
+
 /* Forward matmul with the activation fused into the epilogue (the paper has no
  * counterpart; it answers Section 3's warning that computing a scale just in
  * time costs a second pass over memory: the next layer's input leaves this

@@ -6,12 +6,16 @@
 //
 //   gemm_pair_kernel  (M > 128)  two CTAs of a cluster own one 256x256 tile;
 //                     tcgen05.mma.cta_group::2, six stages of 32 KB per CTA.
-//   gemm_kernel       (M <= 128: decode, skinny)  one CTA owns a 128x256 tile,
+//   gemm_kernel       (M <= 128)  one CTA owns a 128x256 tile,
 //                     four stages of 48 KB, optional split of the contraction
 //                     (partial sums in an FP32 workspace, splitk_finalize_kernel
 //                     launched behind it as a programmatic dependent).
+//   decode_kernel     (M <= 128, contraction-major operands, plain epilogue)
+//                     gemm_kernel with tile width, stage count and split chosen
+//                     per launch, a tile's contraction shared by a cluster, and
+//                     optionally the activation quantised by the same launch.
 //
-// Roles in both:
+// Roles in all of them:
 //   warp 0, one lane   TMA producer: 128-byte-swizzled boxes of A and B into a
 //                      ring of shared-memory stages, completion on an mbarrier.
 //   warp 1, one lane   MMA issuer: tcgen05.mma.kind::f8f6f4 (K = 32 per
@@ -79,7 +83,14 @@ struct GemmParams {
     int dec_bn, dec_stages, dec_a_bytes;   // decode kernel: tile width, stages, bytes a stage sets aside for A
     int dec_cluster;              // decode kernel: CTAs of a cluster that share one tile's contraction (1: none)
     int early_b;                  // decode kernel: B may be read before the launch ahead of this one has completed
+    int early_rings;              // ... how many rings of B tiles are requested then (the first into shared memory, the rest into L2)
     int col_lo;                   // direct stores skip columns below this one (0 except in the decode kernel's last tile)
+    // decode kernel, activation quantised in the same launch (NULL / unused otherwise)
+    const uint4 *qx;              // the bf16 activation [M, K], 16-byte vectors
+    uint8_t *qx8;                 // out: its E4 bytes, which the A loads then read
+    float *q_amax;                // out: its amax
+    int32_t *q_bias;              // out: its scaling bias (paper convention)
+    int q_margin, q_conv;
     int dbg;                      // experiments build only: timing variants that give wrong results
     const void *bias_vec;         // [N] or NULL
     int bias_dt;
@@ -1203,6 +1214,15 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
 // into the leader's shared memory (its stages are free by then) and the leader adds them in rank order and stores
 // the result: no partial sums in global memory, no second launch.  Two cluster barriers frame the exchange; a CTA
 // whose wait ran out still takes part in both.
+//
+// With p.qx set the launch also quantises the activation (FP8-AMAX, Eq. 3 and Eq. 1, bit for bit what fp8_cast_e4
+// does), for activations of a few rows (at most 64 KB): after the dependency wait the four epilogue warps of EVERY CTA
+// take the amax of the whole of X, derive the bias, cast the whole of X and write the bytes (every CTA writes the same
+// bytes to the same places; each reads back only what it has itself written), and only then does the producer start
+// the A loads (its weight tiles have been streaming since the kernel began).  No CTA waits for another: the small
+// cast kernel, its launch and two dependency hops leave the critical path at the price of reading 64 KB from L2 per
+// CTA.  (A version that shared the work between the CTAs, with two barriers across the grid, was slower than the
+// separate cast kernel: 177 against 165 us for a four-layer decoder block at one row.)
 
 __device__ __forceinline__ uint32_t cluster_ctarank()
 {
@@ -1224,9 +1244,11 @@ __device__ __forceinline__ void cluster_sync_all()
 
 #ifdef FP8LIN_EXPERIMENTS
 // timeline of the decode launches (block 0): entry, dependency wait over, exit; read back by fp8_debug_trace
-__device__ unsigned long long g_trace[3 * 1024];
+__device__ unsigned long long g_trace[8 * 1024];
 __device__ unsigned g_trace_n;
 #endif
+
+__device__ __forceinline__ void epilogue_warps_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
 constexpr int kDecodeMaxStages = 32;
 constexpr int kDecodeHeader = 1024;   // barriers, tensor-memory slot and abort flag in front of the stages
@@ -1251,6 +1273,9 @@ decode_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
     auto acc_empty_bar = [&](int b) { return bar_base + 8u * (2 * kDecodeMaxStages + 2 + b); };
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + (2 * kDecodeMaxStages + 4) * 8);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+    const uint32_t a_ready_bar = bar_base + 8u * (2 * kDecodeMaxStages + 6);   // fused quantisation: the bytes of A exist
+    int *s_bias_x = reinterpret_cast<int *>(smem + (2 * kDecodeMaxStages + 8) * 8);   // ... and their bias
+    uint32_t *s_max = reinterpret_cast<uint32_t *>(s_bias_x + 1);                     // five words of the amax reduction
     constexpr uint32_t kCols = 512;   // two accumulators of up to 256 columns
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -1258,12 +1283,13 @@ decode_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
     __shared__ unsigned trace_slot;
     if (threadIdx.x == 0 && blockIdx.x == 0) {
         trace_slot = atomicAdd(&g_trace_n, 1u) % 1024u;
-        g_trace[3 * trace_slot] = global_timer_ns();
+        g_trace[8 * trace_slot] = global_timer_ns();
     }
 #endif
     if (threadIdx.x == 0) {
         for (int s = 0; s < stages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
         for (int b = 0; b < 2; ++b) { mbar_init(acc_full_bar(b), 1); mbar_init(acc_empty_bar(b), 4); }
+        mbar_init(a_ready_bar, 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -1301,7 +1327,7 @@ decode_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
                         tma_load_2d_hint(stage_base + i * stage_bytes + a_bytes, &map_b, full_bar(i), k * kBK, tile_col(n_blk), drop);
                     }
                     early = ring;
-                    for (int i = ring; i < min(k1 - k0, 3 * stages); ++i, k = (k + 1 == k1) ? k0 : k + 1)
+                    for (int i = ring; i < min(k1 - k0, p.early_rings * stages); ++i, k = (k + 1 == k1) ? k0 : k + 1)
                         tma_prefetch_l2_2d(&map_b, k * kBK, tile_col(n_blk));
                 } else {
                     for (int i = 0; i < ring; ++i, k = (k + 1 == k1) ? k0 : k + 1)
@@ -1310,7 +1336,7 @@ decode_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
             }
             asm volatile("griddepcontrol.wait;" ::: "memory");
 #ifdef FP8LIN_EXPERIMENTS
-            if (blockIdx.x == 0) g_trace[3 * trace_slot + 1] = global_timer_ns();
+            if (blockIdx.x == 0) g_trace[8 * trace_slot + 1] = global_timer_ns();
 #endif
             // One thread runs this loop and its latency is the ceiling of what a CTA can stream (a division per k-block
             // was measured to hold a CTA at 0.25 us per k-block with no loads at all): stage index, phase and
@@ -1318,6 +1344,13 @@ decode_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
             int s = 0;
             uint32_t ph = 0, full = full_bar(0), empty = empty_bar(0), a_dst = stage_base;
             bool alive = true;
+            if (p.qx) {   // the bytes of A are written by this very CTA's epilogue warps: wait until all of them are
+                alive = mbar_wait(a_ready_bar, 0u, abort_flag, p.d_status);
+                asm volatile("fence.proxy.async.global;" ::: "memory");   // written through the generic proxy, read by TMA
+            }
+#ifdef FP8LIN_EXPERIMENTS
+            if (blockIdx.x == 0) g_trace[8 * trace_slot + 3] = global_timer_ns();
+#endif
             for (int item = blockIdx.x; alive && item < num_items; item += gridDim.x) {
                 const int n_blk = item / p.splits, split = item % p.splits;
                 const int k0 = split * p.kb_per_split, k1 = min(p.num_k, k0 + p.kb_per_split);
@@ -1395,7 +1428,73 @@ decode_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
     } else {
         asm volatile("griddepcontrol.wait;" ::: "memory");  // the biases may come from the launch before this one
         const int q = warp & 3;  // TMEM lane quarter this warp may address
-        const int e = -(__ldg(p.d_sa) + __ldg(p.d_sb) + p.delta_sum);
+        int bias_x;
+        if (p.qx) {
+            // FP8-AMAX of the whole activation by the 128 threads of these warps, in 16-byte vectors
+            const int tid = (int)threadIdx.x - 64;
+            const int64_t v0 = 0, v1 = (int64_t)p.M * p.K / 8;
+            // eight loads in flight per thread at a time: one after the other they cost a trip to L2 each (measured:
+            // 5 us for 16 KB, 14 us for 56 KB)
+            constexpr int kBatch = 8;
+            uint32_t acc = 0;
+            for (int64_t base = v0 + tid; base < v1; base += 128 * kBatch) {
+                uint4 v[kBatch];
+#pragma unroll
+                for (int j = 0; j < kBatch; ++j) {
+                    const int64_t i = base + 128 * j;
+                    v[j] = i < v1 ? __ldcg(p.qx + i) : make_uint4(0u, 0u, 0u, 0u);
+                }
+#pragma unroll
+                for (int j = 0; j < kBatch; ++j) {
+                    acc = __vmaxu2(acc, v[j].x & 0x7FFF7FFFu);
+                    acc = __vmaxu2(acc, v[j].y & 0x7FFF7FFFu);
+                    acc = __vmaxu2(acc, v[j].z & 0x7FFF7FFFu);
+                    acc = __vmaxu2(acc, v[j].w & 0x7FFF7FFFu);
+                }
+            }
+            uint32_t m = __reduce_max_sync(0xFFFFFFFFu, max(acc & 0xFFFFu, acc >> 16));
+            if (lane == 0) s_max[q] = m;
+            epilogue_warps_sync();
+            const uint32_t fbits = max(max(s_max[0], s_max[1]), max(s_max[2], s_max[3])) << 16;   // bf16 bits of the amax, as a float
+            unsigned flags = 0;
+            bias_x = bias_from_amax_bits(fbits, FP8_E4, p.q_conv, p.q_margin, &flags);
+            if (blockIdx.x == 0 && tid == 0) {
+                *p.q_amax = __uint_as_float(fbits);
+                *p.q_bias = bias_x;
+                if (flags) atomicOr(p.d_status, flags);
+            }
+            const Pow2Pair p2 = make_pow2_pair(bias_x + format_delta(FP8_E4, p.q_conv));
+            bool sat = false;
+            for (int64_t base = v0 + tid; base < v1; base += 128 * kBatch) {
+                uint4 v[kBatch];
+#pragma unroll
+                for (int j = 0; j < kBatch; ++j) {
+                    const int64_t i = base + 128 * j;
+                    v[j] = i < v1 ? __ldcg(p.qx + i) : make_uint4(0u, 0u, 0u, 0u);
+                }
+#pragma unroll
+                for (int j = 0; j < kBatch; ++j) {
+                    const int64_t i = base + 128 * j;
+                    if (i >= v1) continue;
+                    const uint32_t w[4] = {v[j].x, v[j].y, v[j].z, v[j].w};
+                    uint2 o;
+                    o.x = cast4w<FP8_E4, FP8_BF16, true>(w, p2, sat);
+                    o.y = cast4w<FP8_E4, FP8_BF16, true>(w + 2, p2, sat);
+                    *reinterpret_cast<uint2 *>(p.qx8 + i * 8) = o;
+                }
+            }
+            if (__any_sync(0xFFFFFFFFu, sat) && lane == 0) atomicOr(p.d_status, (unsigned)FP8_FLAG_SATURATED);
+            asm volatile("fence.proxy.async.global;" ::: "memory");   // the bytes are read back by this CTA's TMA loads
+            __threadfence();
+            epilogue_warps_sync();
+            if (tid == 0) {
+                *s_bias_x = bias_x;
+                mbar_arrive(a_ready_bar);
+            }
+        } else {
+            bias_x = __ldcg(p.d_sa);
+        }
+        const int e = -(bias_x + __ldg(p.d_sb) + p.delta_sum);
         const Pow2Pair sc = make_pow2_pair(e), sc_one = make_pow2_pair(0);
         const bool two_step = (e < -126 || e > 127);
         uint32_t amax_bits = 0, t = 0;
@@ -1418,6 +1517,9 @@ decode_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
             if (!__all_sync(0xFFFFFFFFu, ready)) break;
             tc_fence_after();
             const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + buf * 256;
+#ifdef FP8LIN_EXPERIMENTS
+            if (blockIdx.x == 0 && warp == 2 && lane == 0 && t == 0) g_trace[8 * trace_slot + 4] = global_timer_ns();
+#endif
             if (p.dec_cluster > 1) break;   // the accumulator stays where it is for the exchange below
             if (q * 32 < p.M) {   // a warp none of whose rows exists reads nothing
 #pragma unroll 1
@@ -1442,16 +1544,21 @@ decode_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
     __syncwarp();  // the single-lane roles rejoin their warps before the block-wide barrier
     if (p.dec_cluster > 1) {
         // Every CTA of the cluster holds the sum over its slice of the contraction in accumulator 0 (its epilogue warps
-        // have seen "accumulator full", or given up).  Rank r > 0 writes rows [0, M) of it to plane r - 1 of a buffer at
-        // the start of the leader's stages, [plane][row][bn floats].
+        // have seen "accumulator full", or given up).  Rank r writes rows [0, M) of it to plane r of a buffer at the
+        // start of the leader's stages, [plane][row][bn + 4 floats], and the leader adds the planes in rank order.  With
+        // up to eight rows its 128 epilogue threads share the columns, four each (a row per lane would leave the whole
+        // tile to a few threads: measured 2 to 4 us per launch at one row); with more rows each lane keeps its own row
+        // (its accumulator stays in tensor memory; the column-sharing loop, about a hundred dependent instructions
+        // per four outputs on four warps, took 8 us at 64 rows).
         const uint32_t rank = cluster_ctarank();
         const int q = warp & 3, row = q * 32 + lane;
-        const bool epi = warp >= 2, has_rows = q * 32 < p.M;
+        const bool epi = warp >= 2, share_columns = p.M <= 8;
         const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16);
-        const uint32_t plane_bytes = (uint32_t)p.M * (uint32_t)bn * 4u;
+        const uint32_t row_floats = (uint32_t)bn + 4u;   // padded: the lanes of a warp write 32 different rows at once
+        const uint32_t plane_bytes = (uint32_t)p.M * row_floats * 4u;
         cluster_sync_all();   // all slices summed; the leader's stages are no longer read or written
-        if (epi && rank != 0 && has_rows && !*abort_flag) {
-            const uint32_t dst_row = map_to_cta(stage_base, 0) + (rank - 1) * plane_bytes + (uint32_t)row * (uint32_t)bn * 4u;
+        if (epi && q * 32 < p.M && !*abort_flag && (rank != 0 || share_columns)) {
+            const uint32_t dst_row = map_to_cta(stage_base, 0) + rank * plane_bytes + (uint32_t)row * row_floats * 4u;
 #pragma unroll 1
             for (int c = 0; c < bn; c += 32) {
                 uint32_t r[32];
@@ -1467,8 +1574,11 @@ decode_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
             }
         }
         cluster_sync_all();   // the planes are written (release / acquire across the cluster)
-        if (epi && rank == 0 && has_rows && !*abort_flag) {
-            const int e = -(__ldg(p.d_sa) + __ldg(p.d_sb) + p.delta_sum);
+#ifdef FP8LIN_EXPERIMENTS
+        if (blockIdx.x == 0 && threadIdx.x == 64) g_trace[8 * trace_slot + 5] = global_timer_ns();
+#endif
+        if (epi && rank == 0 && !*abort_flag && !share_columns && q * 32 < p.M) {
+            const int e = -((p.qx ? *s_bias_x : __ldcg(p.d_sa)) + __ldg(p.d_sb) + p.delta_sum);
             const Pow2Pair sc = make_pow2_pair(e);
             const bool two_step = (e < -126 || e > 127);
             const int n_blk = (int)blockIdx.x / p.splits;
@@ -1477,14 +1587,14 @@ decode_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
             pp.N = min(p.N, col_base + bn);
             pp.col_lo = n_blk * bn;
             uint32_t amax_bits = 0;
-            const uint32_t src_row = stage_base + (uint32_t)row * (uint32_t)bn * 4u;
+            const uint32_t src_row = stage_base + (uint32_t)row * row_floats * 4u;
 #pragma unroll 1
             for (int c = 0; c < bn; c += 32) {
                 uint32_t r[32];
                 tmem_ld_x32(t_row + c, r);
                 tmem_ld_wait();
                 if (row < p.M) {
-                    for (int pl = 0; pl < p.dec_cluster - 1; ++pl) {   // rank order: the sum does not depend on timing
+                    for (int pl = 1; pl < p.dec_cluster; ++pl) {   // rank order: the sum does not depend on timing
 #pragma unroll
                         for (int j = 0; j < 8; ++j) {
                             if (c + 4 * j < bn) {
@@ -1506,6 +1616,73 @@ decode_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
                 if (lane == 0 && amax_bits) atomicMax(p.d_amax_bits, amax_bits);
             }
         }
+        if (epi && rank == 0 && !*abort_flag && share_columns) {
+            const int e = -((p.qx ? *s_bias_x : __ldcg(p.d_sa)) + __ldg(p.d_sb) + p.delta_sum);
+            const Pow2Pair sc = make_pow2_pair(e);
+            const bool two_step = (e < -126 || e > 127);
+            const int n_blk = (int)blockIdx.x / p.splits;
+            const int col_base = tile_col(n_blk), col_lo = n_blk * bn, col_hi = min(p.N, col_base + bn);
+            const int quads = bn >> 2;                 // groups of four columns per row
+            uint32_t amax_bits = 0;
+            // ordinary loads (written by other CTAs before the cluster barrier above): the compiler may overlap iterations
+            const float *planes = reinterpret_cast<const float *>(smem + kDecodeHeader);
+            const uint32_t plane_floats = plane_bytes >> 2;
+#pragma unroll 2
+            for (int idx = (int)threadIdx.x - 64; idx < p.M * quads; idx += 128) {
+                const int r_out = idx / quads, c4 = (idx - r_out * quads) << 2, col = col_base + c4;
+                const float *src = planes + (uint32_t)r_out * row_floats + (uint32_t)c4;
+                const float4 first = *reinterpret_cast<const float4 *>(src);
+                float v[4] = {first.x, first.y, first.z, first.w};
+                for (int pl = 1; pl < p.dec_cluster; ++pl) {   // rank order: the sum does not depend on timing
+                    const float4 u = *reinterpret_cast<const float4 *>(src + (uint32_t)pl * plane_floats);
+                    v[0] += u.x; v[1] += u.y; v[2] += u.z; v[3] += u.w;
+                }
+                if (col >= col_hi || col + 4 <= col_lo) continue;
+                uint32_t bits[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    v[i] *= sc.first;
+                    if (two_step) v[i] *= sc.second;
+                    if (p.bias_vec && col + i < p.N)
+                        v[i] += p.bias_dt == FP8_F32 ? __ldg(reinterpret_cast<const float *>(p.bias_vec) + col + i)
+                                                     : __uint_as_float((uint32_t)__ldg(reinterpret_cast<const uint16_t *>(p.bias_vec) + col + i) << 16);
+                    if (p.out_dt == FP8_BF16) {
+                        uint32_t w;
+                        asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(w) : "f"(0.0f), "f"(v[i]));
+                        bits[i] = w & 0xFFFFu;
+                    } else {
+                        bits[i] = __float_as_uint(v[i]);
+                    }
+                }
+                const bool whole = col >= col_lo && col + 4 <= col_hi && p.vec_ok;
+                if (p.out_dt == FP8_BF16) {
+                    uint16_t *dst = reinterpret_cast<uint16_t *>(p.out) + (int64_t)r_out * p.ldo + col;
+                    if (whole) *reinterpret_cast<uint2 *>(dst) = make_uint2(bits[0] | (bits[1] << 16), bits[2] | (bits[3] << 16));
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        if (col + i < col_lo || col + i >= col_hi) continue;
+                        if (!whole) dst[i] = (uint16_t)bits[i];
+                        amax_bits = max(amax_bits, (bits[i] & 0x7FFFu) << 16);
+                    }
+                } else {
+                    float *dst = reinterpret_cast<float *>(p.out) + (int64_t)r_out * p.ldo + col;
+                    if (whole) *reinterpret_cast<uint4 *>(dst) = make_uint4(bits[0], bits[1], bits[2], bits[3]);
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        if (col + i < col_lo || col + i >= col_hi) continue;
+                        if (!whole) dst[i] = __uint_as_float(bits[i]);
+                        amax_bits = max(amax_bits, bits[i] & 0x7FFFFFFFu);
+                    }
+                }
+            }
+            if (p.d_amax_bits) {
+                amax_bits = __reduce_max_sync(0xFFFFFFFFu, amax_bits);
+                if (lane == 0 && amax_bits) atomicMax(p.d_amax_bits, amax_bits);
+            }
+#ifdef FP8LIN_EXPERIMENTS
+            if (blockIdx.x == 0 && threadIdx.x == 64) g_trace[8 * trace_slot + 6] = global_timer_ns();
+#endif
+        }
     }
     if (*abort_flag) __nanosleep(20000);  // let copies and MMAs already issued drain before the memory is released
     tc_fence_before();
@@ -1513,7 +1690,7 @@ decode_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
     tc_fence_after();
     if (warp == 1) tmem_dealloc(tmem_base, kCols);
 #ifdef FP8LIN_EXPERIMENTS
-    if (threadIdx.x == 0 && blockIdx.x == 0) g_trace[3 * trace_slot + 2] = global_timer_ns();
+    if (threadIdx.x == 0 && blockIdx.x == 0) g_trace[8 * trace_slot + 2] = global_timer_ns();
 #endif
 }
 
@@ -1848,7 +2025,10 @@ __global__ void __launch_bounds__(256) splitk_finalize_kernel(const GemmParams p
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     asm volatile("griddepcontrol.wait;" ::: "memory");
     const int64_t total = (int64_t)p.M * p.N;
-    const int e = -(__ldg(p.d_sa) + __ldg(p.d_sb) + p.delta_sum);
+    // Read at L2, not through the read-only path: the matmul ahead of this launch may itself have written A's bias
+    // (activation quantised in the same launch) while this grid was already resident, and a line the read-only path
+    // holds on this SM is not refreshed by the dependency wait (seen: the stale word, once in a few launches).
+    const int e = -(__ldcg(p.d_sa) + __ldcg(p.d_sb) + p.delta_sum);
     const Pow2Pair sc = make_pow2_pair(e);
     uint32_t amax_bits = 0;
     for (int64_t i = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * VEC; i < total;
@@ -1938,6 +2118,8 @@ static bool g_direct_epilogue = false;  // set from FP8LIN_DIRECT_EPILOGUE=1 (A/
 constexpr int kDecodeMaxCluster = 8;
 static int g_decode_clusters[kDecodeMaxCluster + 1] = {0};   // clusters of each size that can be resident at once
 static bool g_no_decode_cluster = false; // set from FP8LIN_DECODE_CLUSTER=0 (A/B: split contractions through global memory only)
+static bool g_no_fused_quant = false;    // set from FP8LIN_FUSED_QUANT=0 (A/B: fp8_linear_infer_cast as its two calls)
+static int g_early_rings = 2;            // rings of B tiles requested ahead of the dependency wait by fp8_linear_infer (FP8LIN_EARLY_RINGS)
 static bool g_no_early_b = false;        // set from FP8LIN_EARLY_B=0 (A/B: fp8_linear_infer without its early weight loads)
 static bool g_no_decode_kernel = false; // set from FP8LIN_DECODE_KERNEL=0 (A/B: decode shapes on the fixed-width single-CTA kernel)
 static int g_dbg = 0;                   // set from FP8LIN_DECODE_DBG (timing-only variants of the decode kernel)
@@ -2038,6 +2220,10 @@ cudaError_t configure_gemm_kernels(int max_smem_optin)
     g_group_m = env ? atoi(env) : 0;
     env = getenv("FP8LIN_DECODE_CLUSTER");
     g_no_decode_cluster = env && env[0] == '0';
+    env = getenv("FP8LIN_FUSED_QUANT");
+    g_no_fused_quant = env && env[0] == '0';
+    env = getenv("FP8LIN_EARLY_RINGS");
+    if (env) g_early_rings = atoi(env);
     env = getenv("FP8LIN_EARLY_B");
     g_no_early_b = env && env[0] == '0';
     env = getenv("FP8LIN_DECODE_KERNEL");
@@ -2060,8 +2246,12 @@ cudaError_t configure_gemm_kernels(int max_smem_optin)
     g_direct_epilogue = env && env[0] == '1';
     env = getenv("FP8LIN_WIDE");
     g_force_wide = env ? atoi(env) : -1;
-    if (getenv("FP8LIN_DEBUG")) fprintf(stderr, "fp8lin: %d SMs, %d resident CTA pairs, pair kernel %s\n", sms, clusters,
-                                        g_force_single ? "off" : "on");
+    if (getenv("FP8LIN_DEBUG")) {
+        fprintf(stderr, "fp8lin: %d SMs, %d resident CTA pairs, pair kernel %s\n", sms, clusters, g_force_single ? "off" : "on");
+        fprintf(stderr, "fp8lin: resident decode clusters of 2..8 CTAs: %d %d %d %d %d %d %d\n", g_decode_clusters[2],
+                g_decode_clusters[3], g_decode_clusters[4], g_decode_clusters[5], g_decode_clusters[6], g_decode_clusters[7],
+                g_decode_clusters[8]);
+    }
 #endif
     return cudaSuccess;
 }
@@ -2113,7 +2303,7 @@ static void choose_decode(const fp8_ctx *ctx, int64_t M, int64_t N, int num_k, i
     const double solo0 = 180e3, total = 8e6;   // bytes per microsecond
     const double finalize_us = 3.5, partial_rate = 3.8e6, item_us = 0.15, exchange_us = 1.0, exchange_rate = 50e3;
     // whatever its width, a k-block costs the two single-thread loops (wait, two loads / wait, four MMAs, commit) this much
-    const double kblock_us = 0.36;
+    const double kblock_us = 0.36, kOverlapLoss = 0.35;
     const int64_t by_ws = (int64_t)(ctx->partial_bytes / sizeof(float)) / (M * N);
     int64_t cap = num_k / 4 < by_ws ? num_k / 4 : by_ws;
     if (cap > 64) cap = 64;
@@ -2139,7 +2329,11 @@ static void choose_decode(const fp8_ctx *ctx, int64_t M, int64_t N, int num_k, i
             const double item_bytes = (double)kb * bn * kBK;
             const int64_t q = items / sms, extra = items % sms;
             const double floor_us = (double)kb * kblock_us;
-            auto item_time = [&](double active) { const double t = item_bytes / rate(active); return t > floor_us ? t : floor_us; };
+            // the two bounds do not hide behind each other completely: the larger plus a share of the smaller
+            auto item_time = [&](double active) {
+                const double t = item_bytes / rate(active);
+                return t > floor_us ? t + kOverlapLoss * floor_us : floor_us + kOverlapLoss * t;
+            };
             double cost = q > 0 ? (double)q * item_time((double)sms) : 0.0;
             if (extra > 0) cost += item_time((double)extra);
             cost += item_us * (double)(q + (extra > 0 ? 1 : 0));
@@ -2153,16 +2347,16 @@ static void choose_decode(const fp8_ctx *ctx, int64_t M, int64_t N, int num_k, i
                 *cluster_out = 1;
             }
         }
-        for (int cs = 2; cs <= kDecodeMaxCluster && !g_no_decode_cluster; ++cs) {
+        for (int cs = 2; cs <= kDecodeMaxCluster && !g_no_decode_cluster; cs *= 2) {   // 2, 4, 8 (three was measured slower than four)
             const int64_t kb = (num_k + cs - 1) / cs;
             if ((num_k + kb - 1) / kb != cs || kb < 4) continue;
             if (tiles > g_decode_clusters[cs]) continue;
-            if ((int64_t)(cs - 1) * M * bn * 4 > (int64_t)stages * stage) continue;   // the exchange buffer
+            if ((int64_t)cs * M * (bn + 4) * 4 > (int64_t)stages * stage) continue;   // the exchange buffer (padded rows)
             if (g_force_splits > 0 && cs != g_force_splits) continue;
             if (g_force_bn > 0 && bn != g_force_bn) continue;
             const double item_bytes = (double)kb * bn * kBK;
-            double cost = item_bytes / rate((double)(tiles * cs));
-            if (cost < (double)kb * kblock_us) cost = (double)kb * kblock_us;
+            const double stream_us = item_bytes / rate((double)(tiles * cs)), floor_us = (double)kb * kblock_us;
+            double cost = stream_us > floor_us ? stream_us + kOverlapLoss * floor_us : floor_us + kOverlapLoss * stream_us;
             cost += item_us + exchange_us + (double)(cs - 1) * (double)M * bn * 4.0 / exchange_rate;
             if (bn % 32) cost += 0.3;
             if (*bn_out == 0 || cost < best) {
@@ -2182,6 +2376,16 @@ static void choose_decode(const fp8_ctx *ctx, int64_t M, int64_t N, int num_k, i
     }
 }
 
+constexpr int64_t kFusedQuantMaxBytes = 64 << 10;
+// The activation of a decode launch, to be quantised by that launch itself (decode kernel only).
+struct FusedQuant {
+    const void *x;     // bf16 [M, Kc], contiguous, 16-byte aligned
+    uint8_t *x8;       // out [M, Kc]; run_gemm's `a` must be this buffer
+    float *d_amax;     // out
+    int32_t *d_bias;   // out; run_gemm's `d_ba` must be this word
+    int margin, conv;
+};
+
 // D[M,N] = A * B^T over a contraction of length Kc, unscaled by 2^-(bias_a + bias_b + delta_sum).
 // A is stored [M, Kc] (a_mn = false) or [Kc, M] (a_mn = true); B is stored [N, Kc] or [Kc, N] likewise.
 static fp8_status_t run_gemm(fp8_ctx *ctx, const uint8_t *a, int a_fmt, bool a_mn, const int32_t *d_ba,
@@ -2189,7 +2393,8 @@ static fp8_status_t run_gemm(fp8_ctx *ctx, const uint8_t *a, int a_fmt, bool a_m
                              const void *bias_vec, int bias_dt, void *out, int out_dt, float *d_amax_out, int64_t M,
                              int64_t N, int64_t Kc, cudaStream_t st, int act = 0, void *out_act = nullptr,
                              const void *aux = nullptr, uint8_t *out8 = nullptr, const int32_t *d_sq = nullptr,
-                             int q_fmt = 0, int delta_q = 0, bool no_loads = false, int chunk_kb = 0, bool static_b = false)
+                             int q_fmt = 0, int delta_q = 0, bool no_loads = false, int chunk_kb = 0, bool static_b = false,
+                             const FusedQuant *fq = nullptr)
 {
     if (M > 0x7FFFFFFF / 2 || N > 0x7FFFFFFF / 2 || Kc > 0x7FFFFFFF / 2) return FP8_ERR_SHAPE;
     const bool pair = g_max_pairs > 0 && M > kBM && !g_force_single && act != 6;
@@ -2205,7 +2410,19 @@ static fp8_status_t run_gemm(fp8_ctx *ctx, const uint8_t *a, int a_fmt, bool a_m
     p.dec_bn = p.dec_stages = p.dec_a_bytes = 0;
     p.dec_cluster = 1;
     p.col_lo = 0;
+    p.qx = nullptr;
+    if (fq) {
+        // beyond 64 KB of activation (or outside the decode kernel) the caller quantises with a call of its own
+        if (!decode || M * Kc * 2 > kFusedQuantMaxBytes) return FP8_ERR_UNSUPPORTED;
+        p.qx = static_cast<const uint4 *>(fq->x);
+        p.qx8 = fq->x8;
+        p.q_amax = fq->d_amax;
+        p.q_bias = fq->d_bias;
+        p.q_margin = fq->margin;
+        p.q_conv = fq->conv;
+    }
     p.early_b = (decode && static_b && !g_no_early_b) ? 1 : 0;
+    p.early_rings = g_early_rings;
     p.dbg = g_dbg;
     int dec_kb = 0;
     if (decode) {
@@ -2497,7 +2714,7 @@ __attribute__((visibility("default"))) int fp8_debug_trace(unsigned long long *h
     unsigned n = 0;
     cudaDeviceSynchronize();
     cudaMemcpyFromSymbol(&n, fp8lin::g_trace_n, sizeof(n));
-    cudaMemcpyFromSymbol(host_out, fp8lin::g_trace, sizeof(unsigned long long) * 3 * 1024);
+    cudaMemcpyFromSymbol(host_out, fp8lin::g_trace, sizeof(unsigned long long) * 8 * 1024);
     if (clear) {
         unsigned zero = 0;
         cudaMemcpyToSymbol(fp8lin::g_trace_n, &zero, sizeof(zero));
@@ -2505,6 +2722,33 @@ __attribute__((visibility("default"))) int fp8_debug_trace(unsigned long long *h
     return (int)n;
 }
 #endif
+
+fp8_status_t fp8_linear_infer_cast(fp8_ctx *ctx, const void *x, fp8_dtype_t x_dt, int32_t margin, float *d_amax_x,
+                                   int32_t *d_bx, uint8_t *x8, const uint8_t *w8, const int32_t *d_bw, const void *bias_vec,
+                                   fp8_dtype_t bias_dt, void *y, fp8_dtype_t y_dt, float *d_amax_y, int64_t T, int64_t K,
+                                   int64_t N, fp8_conv_t conv, void *stream)
+{
+    using namespace fp8lin;
+    if (!ctx || !x || !d_amax_x || !d_bx || !x8 || !w8 || !d_bw || !y) return FP8_ERR_NULL;
+    if ((int)conv < 0 || (int)conv > 1 || (int)y_dt < 0 || (int)y_dt > 2 || (int)bias_dt < 0 || (int)bias_dt > 2 ||
+        (int)x_dt < 0 || (int)x_dt > 2)
+        return FP8_ERR_DTYPE;
+    if (!out_dtype_ok(y_dt) || (bias_vec && !out_dtype_ok(bias_dt))) return FP8_ERR_UNSUPPORTED;
+    if (T <= 0 || K <= 0 || N <= 0) return FP8_ERR_SHAPE;
+    if (!aligned16(x8) || !aligned16(w8) || (K % 16) != 0 || (reinterpret_cast<uintptr_t>(y) & 3u)) return FP8_ERR_ALIGN;
+    const int delta = 2 * format_delta(FP8_E4, conv);
+    if (x_dt == FP8_BF16 && aligned16(x) && T <= kBM && g_max_pairs >= 0 && !g_no_fused_quant) {
+        const FusedQuant fq = {x, x8, d_amax_x, d_bx, margin, (int)conv};
+        const fp8_status_t st = run_gemm(ctx, x8, FP8_E4, false, d_bx, w8, FP8_E4, false, d_bw, delta, bias_vec, bias_dt, y,
+                                         y_dt, d_amax_y, T, N, K, (cudaStream_t)stream, 0, nullptr, nullptr, nullptr,
+                                         nullptr, 0, 0, false, 0, true, &fq);
+        if (st != FP8_ERR_UNSUPPORTED) return st;
+    }
+    // any other case: the two calls this one stands for
+    const fp8_status_t st = fp8_cast_e4(ctx, x, x_dt, T, K, K, nullptr, conv, margin, d_amax_x, d_bx, x8, nullptr, stream);
+    if (st != FP8_OK) return st;
+    return fp8_linear_infer(ctx, x8, d_bx, w8, d_bw, bias_vec, bias_dt, y, y_dt, d_amax_y, T, K, N, conv, stream);
+}
 
 fp8_status_t fp8_selftest_mma_ceiling(fp8_ctx *ctx, void *out, const int32_t *d_zero, int64_t M, int64_t N, int64_t K,
                                       void *stream)

@@ -33,7 +33,7 @@ SYMBOLS = (
     "fp8_create", "fp8_destroy", "fp8_status_string", "fp8_device_flags", "fp8_amax", "fp8_scaling_bias",
     "fp8_scaling_bias_host", "fp8_cast_e4", "fp8_cast_e5", "fp8_ptq_weights", "fp8_linear_fwd", "fp8_linear_dgrad",
     "fp8_linear_wgrad", "fp8_amax_noalloc", "fp8_linear_fwd_act", "fp8_cast_predicted", "fp8_prediction_stats",
-    "fp8_linear_dgrad_act", "fp8_selftest_wait_expiry", "fp8_range_stats", "fp8_linear_fwd_q", "fp8_linear_dgrad_q", "fp8_amax_history_bias", "fp8_launch_count", "fp8_cast_group", "fp8_selftest_mma_ceiling", "fp8_bias_log_append", "fp8_bias_mode", "fp8_linear_f16acc", "fp8_linear_infer",
+    "fp8_linear_dgrad_act", "fp8_selftest_wait_expiry", "fp8_range_stats", "fp8_linear_fwd_q", "fp8_linear_dgrad_q", "fp8_amax_history_bias", "fp8_launch_count", "fp8_cast_group", "fp8_selftest_mma_ceiling", "fp8_bias_log_append", "fp8_bias_mode", "fp8_linear_f16acc", "fp8_linear_infer", "fp8_linear_infer_cast",
 )
 
 if not os.path.exists(LIB_PATH):
@@ -66,6 +66,8 @@ _lib.fp8_range_stats.argtypes = [_P, c_int, _P, c_int, c_int64, c_int64, c_int64
 _lib.fp8_ptq_weights.argtypes = [_P, _P, c_int, c_int64, c_int64, c_int64, c_int, _P, _P, _P, _P, _P]
 _lib.fp8_linear_fwd.argtypes = [_P, _P, _P, _P, _P, _P, c_int, _P, c_int, _P, c_int64, c_int64, c_int64, c_int, _P]
 _lib.fp8_linear_infer.argtypes = _lib.fp8_linear_fwd.argtypes
+_lib.fp8_linear_infer_cast.argtypes = [_P, _P, c_int, c_int, _P, _P, _P, _P, _P, _P, c_int, _P, c_int, _P, c_int64, c_int64,
+                                       c_int64, c_int, _P]
 _lib.fp8_linear_fwd_act.argtypes = [_P, _P, _P, _P, _P, _P, c_int, _P, _P, c_int, _P, c_int64, c_int64, c_int64, c_int, _P]
 _lib.fp8_linear_dgrad.argtypes = [_P, _P, _P, _P, _P, _P, _P, c_int, _P, c_int64, c_int64, c_int64, c_int, _P]
 _lib.fp8_linear_dgrad_act.argtypes = [_P, _P, _P, _P, _P, _P, _P, _P, _P, c_int, _P, c_int64, c_int64, c_int64, c_int, _P]
@@ -290,6 +292,15 @@ class Context:
         _check(_lib.fp8_linear_infer(self._h, _ptr(x8), _ptr(d_bx), _ptr(w8), _ptr(d_bw), _ptr(bias_vec), bias_dt,
                                      _ptr(y), _DT[y.dtype], _ptr(d_amax_y), T, K, N, conv, _stream()),
                "fp8_linear_infer")
+
+    def linear_infer_cast(self, x, d_amax_x, d_bx, x8, w8, d_bw, y, margin=0, bias_vec=None, d_amax_y=None, conv=CONV_PAPER):
+        """``fp8_linear_infer_cast``: FP8-AMAX of the activation x and the forward matmul on weights quantised once."""
+        T, K = x.shape
+        N = w8.shape[0]
+        bias_dt = _DT[bias_vec.dtype] if bias_vec is not None else BF16
+        _check(_lib.fp8_linear_infer_cast(self._h, _ptr(x), _DT[x.dtype], margin, _ptr(d_amax_x), _ptr(d_bx), _ptr(x8),
+                                          _ptr(w8), _ptr(d_bw), _ptr(bias_vec), bias_dt, _ptr(y), _DT[y.dtype],
+                                          _ptr(d_amax_y), T, K, N, conv, _stream()), "fp8_linear_infer_cast")
 
     def linear_fwd_act(self, x8, d_bx, w8, d_bw, y_pre, y_act, bias_vec=None, d_amax_act=None, act=ACT_GELU,
                        conv=CONV_PAPER):

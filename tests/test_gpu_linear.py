@@ -310,6 +310,83 @@ def test_decode_shapes_split_k(ctx, lib, T, K, N):
     assert ctx.device_flags(clear=True) & lib.FLAG_TIMEOUT == 0
 
 
+def _infer_cast(ctx, x, w8, d_bw, dt, conv=O.CONV_PAPER, margin=0, bias_vec=None):
+    """fp8_linear_infer_cast on fresh outputs (poisoned first): amax, bias, bytes of x and the product."""
+    T, K = x.shape
+    x8 = torch.full((T, K), 0x55, dtype=torch.uint8, device="cuda")
+    amax = torch.full((1,), -1.0, dtype=torch.float32, device="cuda")
+    bias = torch.full((1,), 77, dtype=torch.int32, device="cuda")
+    y = torch.full((T, w8.shape[0]), float("nan"), dtype=dt, device="cuda")
+    amax_y = torch.zeros(1, dtype=torch.float32, device="cuda")
+    ctx.linear_infer_cast(x, amax, bias, x8, w8, d_bw, y, margin=margin, bias_vec=bias_vec, d_amax_y=amax_y, conv=conv)
+    return x8, amax, bias, y, amax_y
+
+
+@pytest.mark.parametrize("T,K,N", [(1, 2048, 768), (1, 28672, 1024), (4, 8192, 1280), (3, 1024, 272), (2, 16384, 512),
+                                   (5, 2064, 784), (16, 4096, 1280), (64, 8192, 512), (128, 4096, 4096), (33, 1024, 18944)])
+@pytest.mark.parametrize("conv", [O.CONV_PAPER, O.CONV_NATIVE])
+def test_inference_call_that_quantises_its_activation(ctx, lib, T, K, N, conv):
+    """fp8_linear_infer_cast: one call for FP8-AMAX of the activation and the forward matmul (Section 3.1).  amax,
+    bias and bytes of x must be the oracle's bit for bit, the product must meet the forward bars and carry the same
+    bits as fp8_cast_e4 followed by fp8_linear_infer, both for activations small enough for the single launch
+    (at most 64 KB) and for larger ones."""
+    x = I.normal_bf16(T, K, 1.0, 53, 1, "cuda", outlier_frac=0.005, outlier_scale=100.0)
+    w = I.normal_bf16(N, K, 0.015, 53, 2, "cuda")
+    qx, qw = Quantised(ctx, x, O.E4, conv, transposed=False), Quantised(ctx, w, O.E4, conv, transposed=False)
+    bv = (torch.randn(N, device="cuda") * 0.1).to(torch.bfloat16)
+    ref = O.linear_fwd(qx.ref, qx.shift, qw.ref, qw.shift, bias_vec=bv.double().cpu().numpy())
+    for dt in (torch.float32, torch.bfloat16):
+        for _ in range(2):   # a second call finds the context's scratch as the first left it
+            x8, amax, bias, y, amax_y = _infer_cast(ctx, x, qw.y, qw.bias, dt, conv=conv, bias_vec=bv)
+            assert float(amax.item()) == float(qx.amax.item()) and int(bias.item()) == qx.ref_bias
+            assert_codes_equal(u8(x8), qx.ref, O.N_E4)
+            if dt == torch.float32:
+                assert_gemm_close(y.cpu().numpy(), ref)
+            else:
+                assert_bf16_within_one_ulp(bits_of(y), ref)
+            assert float(amax_y.item()) == float(y.float().abs().max().item())
+            y2 = torch.full((T, N), float("nan"), dtype=dt, device="cuda")
+            ctx.linear_infer(qx.y, qx.bias, qw.y, qw.bias, y2, bias_vec=bv, conv=conv)
+            as_int = torch.int16 if dt == torch.bfloat16 else torch.int32
+            assert torch.equal(y.view(as_int), y2.view(as_int))
+    assert ctx.device_flags(clear=True) & lib.FLAG_TIMEOUT == 0
+
+
+def test_inference_call_margin_specials_and_other_input_types(ctx, lib):
+    """The margin of Section 3.2 reaches the bias; an all-zero activation gives bias 0 and the ZERO_AMAX flag as
+    fp8_cast_e4 does; FP16 / FP32 activations and unaligned ones take the two-call route with the same results."""
+    T, K, N = 2, 4096, 512
+    w = I.normal_bf16(N, K, 0.02, 59, 2, "cuda")
+    qw = Quantised(ctx, w, O.E4, O.CONV_PAPER, transposed=False)
+    x = I.normal_bf16(T, K, 3.0, 59, 1, "cuda")
+    a, b, ref8 = O.quantise(bits_of(x), O.E4, O.CONV_PAPER, 3)
+    x8, amax, bias, y, _ = _infer_cast(ctx, x, qw.y, qw.bias, torch.float32, margin=3)
+    assert float(amax.item()) == a and int(bias.item()) == b
+    assert_codes_equal(u8(x8), ref8, O.N_E4)
+    assert_gemm_close(y.cpu().numpy(), O.linear_fwd(ref8, b + 1, qw.ref, qw.shift))
+    ctx.device_flags(clear=True)
+    z = torch.zeros((T, K), dtype=torch.bfloat16, device="cuda")
+    x8, amax, bias, y, _ = _infer_cast(ctx, z, qw.y, qw.bias, torch.float32)
+    assert float(amax.item()) == 0.0 and int(bias.item()) == 0 and not x8.any() and not y.any()
+    assert ctx.device_flags(clear=True) & lib.FLAG_ZERO_AMAX
+    for xin in (x.to(torch.float16), x.float(), torch.cat([x.flatten()[:1], x.flatten()])[1:].view(T, K)):
+        a, b, ref8 = O.quantise(bits_of(xin.to(torch.bfloat16)), O.E4) if xin.dtype == torch.bfloat16 else (None, None, None)
+        x8, amax, bias, y, _ = _infer_cast(ctx, xin, qw.y, qw.bias, torch.bfloat16)
+        x8b = torch.empty_like(x8)
+        amax_b, bias_b = torch.zeros_like(amax), torch.zeros_like(bias)
+        ctx.cast_e4(xin, None, d_amax_out=amax_b, d_bias_out=bias_b, y=x8b)
+        y_b = torch.empty_like(y)
+        ctx.linear_infer(x8b, bias_b, qw.y, qw.bias, y_b)
+        assert torch.equal(x8, x8b) and torch.equal(amax, amax_b) and torch.equal(bias, bias_b)
+        assert torch.equal(y.view(torch.int16), y_b.view(torch.int16))
+        if ref8 is not None:
+            assert_codes_equal(u8(x8), ref8, O.N_E4)
+    with pytest.raises(lib.Fp8Error) as e:
+        ctx.linear_infer_cast(x, amax, None, x8, qw.y, qw.bias, y)
+    assert e.value.status == lib.ERR_NULL
+    assert ctx.device_flags(clear=True) & lib.FLAG_TIMEOUT == 0
+
+
 @pytest.mark.parametrize("T,N,K", [(16, 4096, 1024), (2, 8208, 528)])
 def test_decode_shapes_dgrad_from_row_major_weights(ctx, lib, T, N, K):
     """The same split contraction with the weight read in its forward layout
@@ -370,6 +447,12 @@ def test_llama70b_ptq_inference_layers(ctx, lib, layer, tokens):
     ctx.linear_infer(qx.y, qx.bias, pw.w8, pw.bias, y_inf)     # what the benchmark's forward-only workloads call
     assert ctx.device_flags(clear=True) & lib.FLAG_TIMEOUT == 0
     assert torch.equal(y.view(torch.int16), y_inf.view(torch.int16))
+    if tokens <= 128:   # the benchmark's decode step: activation quantised by the matmul's own call
+        x8, amax, bias, y_q, _ = _infer_cast(ctx, x, pw.w8, pw.bias, torch.bfloat16)
+        assert float(amax.item()) == float(qx.amax.item()) and int(bias.item()) == qx.ref_bias
+        assert_codes_equal(u8(x8), qx.ref, O.N_E4)
+        assert torch.equal(y.view(torch.int16), y_q.view(torch.int16))
+        assert ctx.device_flags(clear=True) & lib.FLAG_TIMEOUT == 0
     rng = np.random.default_rng(layer * 100 + tokens)
     rows, cols = tile_sample_positions(rng, tokens, pw.N)
     ref = O.linear_samples(O.FWD, qx.ref, O.N_E4, qx.shift, pw.ref, O.N_E4, pw.shift, rows, cols)

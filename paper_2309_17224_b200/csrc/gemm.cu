@@ -1878,15 +1878,29 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                         if (rank == 0) mbar_arrive(full_bar(s));
                         continue;
                     }
+#ifdef FP8LIN_EXPERIMENTS
+                    // timing only (wrong results): every other trip round the ring re-uses what the stages hold, in
+                    // whole (11) or for B alone (12) or A alone (13): what fewer bytes from L2 would be worth
+                    const bool reuse = ((it / kStagesL) & 1u) != 0;
+                    if (reuse && p.dbg == 11) {
+                        if (rank == 0) mbar_arrive(full_bar(s));
+                        continue;
+                    }
+                    const bool skip_a = reuse && p.dbg == 13, skip_b = reuse && p.dbg == 12;
+                    if (rank == 0) mbar_expect_tx(full_bar(s), skip_a ? 2 * (L::kStageBytes - L::kABytes) : (skip_b ? 2 * L::kABytes : 2 * L::kStageBytes));
+#else
+                    constexpr bool skip_a = false, skip_b = false;
                     // only the leader arrives, announcing the bytes of all four loads of the pair; the
                     // peer's bytes may land first (the pending arrival keeps the phase open)
                     if (rank == 0) mbar_expect_tx(full_bar(s), 2 * L::kStageBytes);
+#endif
                     const uint32_t a_dst = smem_base + s * L::kStageBytes;
                     const int a_row = m_blk * 256 + (int)rank * kBM;
-                    if (p.a_mn) tma_load_2d_pair(a_dst, &map_a, leader_full, a_row, kc);
+                    if (skip_a) {}
+                    else if (p.a_mn) tma_load_2d_pair(a_dst, &map_a, leader_full, a_row, kc);
                     else tma_load_2d_pair(a_dst, &map_a, leader_full, kc, a_row);
 #pragma unroll
-                    for (int h = 0; h < NHALF; ++h) {   // this CTA's 128 of the 256 B rows of each half of the tile
+                    for (int h = 0; h < NHALF && !skip_b; ++h) {   // this CTA's 128 of the 256 B rows of each half of the tile
                         const int b_row = n_blk * kTileN + h * kPairBN + (int)rank * kPairHalfN;
                         const uint32_t b_dst = a_dst + L::kABytes + h * (kPairHalfN * kBK);
                         if (p.b_mn) tma_load_2d_pair(b_dst, &map_b, leader_full, b_row, kc);

@@ -44,7 +44,7 @@ __global__ void __launch_bounds__(kCastThreads) cast_tile_kernel(const void *__r
 
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");  // see cast_flat_kernel
     asm volatile("griddepcontrol.wait;" ::: "memory");
-    const int s = __ldg(d_bias) + delta;
+    const int s = __ldcg(d_bias) + delta;   // at L2: the word may come from the launch before this one (see ptx.cuh)
     const Pow2Pair p = make_pow2_pair(s);
     bool sat = false;
 

@@ -578,7 +578,7 @@ __device__ __forceinline__ void epilogue_tile(const CUtensorMap *map_out, const 
         Pow2Pair scq = make_pow2_pair(0);
         bool scq_two = false;
         if (p.out8) {
-            const int sq = __ldg(p.d_sq) + p.delta_q;
+            const int sq = __ldcg(p.d_sq) + p.delta_q;
             scq = make_pow2_pair(sq);
             scq_two = sq < -126 || sq > 127;
         }
@@ -657,7 +657,7 @@ __device__ __forceinline__ void epilogue_tile(const CUtensorMap *map_out, const 
         Pow2Pair scq = make_pow2_pair(0);
         bool scq_two = false;
         if (p.out8) {
-            const int sq = __ldg(p.d_sq) + p.delta_q;
+            const int sq = __ldcg(p.d_sq) + p.delta_q;
             scq = make_pow2_pair(sq);
             scq_two = sq < -126 || sq > 127;
         }
@@ -758,7 +758,7 @@ __device__ __forceinline__ void epilogue_tile(const CUtensorMap *map_out, const 
         Pow2Pair scq = make_pow2_pair(0);
         bool scq_two = false;
         if (p.out8) {
-            const int sq = __ldg(p.d_sq) + p.delta_q;
+            const int sq = __ldcg(p.d_sq) + p.delta_q;
             scq = make_pow2_pair(sq);
             scq_two = sq < -126 || sq > 127;
         }
@@ -1141,7 +1141,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         // ------------------------------- epilogue -------------------------------
         asm volatile("griddepcontrol.wait;" ::: "memory");  // the biases may come from the launch before this one
         const int q = warp & 3;  // TMEM lane quarter this warp may address
-        const int e = -(__ldg(p.d_sa) + __ldg(p.d_sb) + p.delta_sum);
+        const int e = -(__ldcg(p.d_sa) + __ldcg(p.d_sb) + p.delta_sum);
         const Pow2Pair sc = make_pow2_pair(e);
         const bool two_step = (e < -126 || e > 127);
         uint32_t amax_bits = 0, slab_count = 0;
@@ -1494,7 +1494,7 @@ decode_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
         } else {
             bias_x = __ldcg(p.d_sa);
         }
-        const int e = -(bias_x + __ldg(p.d_sb) + p.delta_sum);
+        const int e = -(bias_x + __ldcg(p.d_sb) + p.delta_sum);
         const Pow2Pair sc = make_pow2_pair(e), sc_one = make_pow2_pair(0);
         const bool two_step = (e < -126 || e > 127);
         uint32_t amax_bits = 0, t = 0;
@@ -1578,7 +1578,7 @@ decode_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
         if (blockIdx.x == 0 && threadIdx.x == 64) g_trace[8 * trace_slot + 5] = global_timer_ns();
 #endif
         if (epi && rank == 0 && !*abort_flag && !share_columns && q * 32 < p.M) {
-            const int e = -((p.qx ? *s_bias_x : __ldcg(p.d_sa)) + __ldg(p.d_sb) + p.delta_sum);
+            const int e = -((p.qx ? *s_bias_x : __ldcg(p.d_sa)) + __ldcg(p.d_sb) + p.delta_sum);
             const Pow2Pair sc = make_pow2_pair(e);
             const bool two_step = (e < -126 || e > 127);
             const int n_blk = (int)blockIdx.x / p.splits;
@@ -1617,7 +1617,7 @@ decode_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
             }
         }
         if (epi && rank == 0 && !*abort_flag && share_columns) {
-            const int e = -((p.qx ? *s_bias_x : __ldcg(p.d_sa)) + __ldg(p.d_sb) + p.delta_sum);
+            const int e = -((p.qx ? *s_bias_x : __ldcg(p.d_sa)) + __ldcg(p.d_sb) + p.delta_sum);
             const Pow2Pair sc = make_pow2_pair(e);
             const bool two_step = (e < -126 || e > 127);
             const int n_blk = (int)blockIdx.x / p.splits;
@@ -1971,7 +1971,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
     } else {
         asm volatile("griddepcontrol.wait;" ::: "memory");  // the biases (and aux) may come from the launch before
         const int q = warp & 3;
-        const int e = -(__ldg(p.d_sa) + __ldg(p.d_sb) + p.delta_sum);
+        const int e = -(__ldcg(p.d_sa) + __ldcg(p.d_sb) + p.delta_sum);
         const Pow2Pair sc = make_pow2_pair(e);
         const bool two_step = (e < -126 || e > 127);
         uint32_t amax_bits = 0, slab_count = 0;

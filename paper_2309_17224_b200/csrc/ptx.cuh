@@ -5,6 +5,13 @@
 
 namespace fp8lin {
 
+// Programmatic dependent launches and the read-only data path.  A kernel launched as a programmatic dependent is
+// resident while the launch before it still runs, and orders itself behind that launch with griddepcontrol.wait.
+// A word that the earlier launch may write (a scaling bias, a redo flag) must then be read with an ordinary load
+// at L2 (__ldcg) or a volatile one, never through the read-only path (__ldg, or a plain load from a
+// const __restrict__ pointer): such a load promises that the word does not change while the kernel runs, so it
+// may be issued ahead of the wait, and it was seen to return the word as it stood before the earlier launch wrote it.
+
 // Upper bound of every device-side wait; on expiry the waiting kernel raises FP8_FLAG_TIMEOUT and returns.
 constexpr unsigned long long kWaitLimitNs = 1000ull * 1000ull * 1000ull;
 

@@ -387,6 +387,49 @@ def test_inference_call_margin_specials_and_other_input_types(ctx, lib):
     assert ctx.device_flags(clear=True) & lib.FLAG_TIMEOUT == 0
 
 
+@pytest.mark.parametrize("T,K,N", [(256, 768, 768), (2048, 1024, 1024), (16, 4096, 1280), (1, 8192, 1024), (1, 28672, 1024)])
+def test_calls_chained_without_host_synchronisation_see_each_others_results(ctx, lib, T, K, N):
+    """Inside a step the library's kernels follow each other as programmatic dependent launches: a kernel is resident
+    while the one before it still runs and must not read a bias before that one has written it.  Quantise and multiply
+    back to back with no host synchronisation in between, the bias words and bytes poisoned before every round, through
+    each quantisation route (two launches, one pass with a wrong guess, the grouped call in both modes); every round
+    must give the bits of a run that synchronises between the calls."""
+    x = I.normal_bf16(T, K, 1.0, 61, 1, "cuda", outlier_frac=0.01, outlier_scale=50.0)
+    w = I.normal_bf16(N, K, 0.02, 61, 2, "cuda")
+    qx, qw = Quantised(ctx, x, O.E4, O.CONV_PAPER, transposed=False), Quantised(ctx, w, O.E4, O.CONV_PAPER, transposed=False)
+    y_ref = torch.empty((T, N), dtype=torch.bfloat16, device="cuda")
+    ctx.linear_fwd(qx.y, qx.bias, qw.y, qw.bias, y_ref)
+    torch.cuda.synchronize()
+    x8, w8 = torch.empty_like(qx.y), torch.empty_like(qw.y)
+    amax = torch.zeros(2, dtype=torch.float32, device="cuda")
+    bias = torch.zeros(2, dtype=torch.int32, device="cuda")
+    y = torch.empty_like(y_ref)
+
+    def two_launches():
+        ctx.cast_e4(w, None, d_amax_out=amax[0:1], d_bias_out=bias[0:1], y=w8)
+        ctx.cast_e4(x, None, d_amax_out=amax[1:2], d_bias_out=bias[1:2], y=x8)
+
+    def one_pass_wrong_guess():
+        ctx.cast_predicted(lib.E4, w, amax[0:1], bias[0:1], w8)
+        ctx.cast_predicted(lib.E4, x, amax[1:2], bias[1:2], x8)
+
+    items = [(lib.E4, w, amax[0:1], bias[0:1], w8), (lib.E4, x, amax[1:2], bias[1:2], x8)]
+    routes = (two_launches, one_pass_wrong_guess, lambda: ctx.cast_group(items), lambda: ctx.cast_group(items, predicted=True))
+    for route in routes:
+        for rnd in range(12):
+            bias.fill_(60 + rnd)     # an absurd bias: a matmul that read it would be off by dozens of powers of two
+            x8.fill_(0x55)
+            w8.fill_(0x55)
+            y.fill_(float("nan"))
+            route()
+            ctx.linear_fwd(x8, bias[1:2], w8, bias[0:1], y)
+            torch.cuda.synchronize()
+            assert int(bias[0].item()) == qw.ref_bias and int(bias[1].item()) == qx.ref_bias
+            assert torch.equal(x8, qx.y) and torch.equal(w8, qw.y)
+            assert torch.equal(y.view(torch.int16), y_ref.view(torch.int16)), f"round {rnd}"
+    assert ctx.device_flags(clear=True) & lib.FLAG_TIMEOUT == 0
+
+
 @pytest.mark.parametrize("T,N,K", [(16, 4096, 1024), (2, 8208, 528)])
 def test_decode_shapes_dgrad_from_row_major_weights(ctx, lib, T, N, K):
     """The same split contraction with the weight read in its forward layout

@@ -50,9 +50,9 @@ EVENT_EVERY = 8   # per-kernel CUDA-event pairs are recorded on every eighth tim
 ORACLE_SAMPLE_LAYER = 1  # the square attention-output projection
 NOMINAL_FP8_TFLOPS = 4500.0         # dense FP8, the vendor's figure for the part
 FP8_FLOP_PER_CLK_PER_SM = 16384.0   # 8192 multiply-adds per clock per SM: nominal peak / (148 SMs x 1.856 GHz)
-# dram__bytes_read.sum + dram__bytes_write.sum per matmul launch, from one ncu capture of one step of the
-# workload (profiles/launch_list_c3_llama7b.md, second table); keyed by (workload, tokens)
-GEMM_DRAM_BYTES_PER_LAUNCH = {("c3_llama7b", 8192): 331.3e6}
+# dram__bytes_read.sum + dram__bytes_write.sum per matmul launch, from one ncu capture of the workload's steps
+# (profiles/launch_list_c3_llama7b.md); keyed by (workload, tokens, one launch per step or one per matmul)
+GEMM_DRAM_BYTES_PER_LAUNCH = {("c3_llama7b", 8192, "per-call"): 331.3e6, ("c3_llama7b", 8192, "group"): 4722.9e6}
 
 
 def load_peaks():
@@ -322,14 +322,27 @@ class Step:
     Decode-size batches (at most 128 tokens) always take the per-tensor path: their activations fit the
     single-launch register-resident kernel, which chains into the matmul behind it."""
 
-    def __init__(self, ctx, fp8lin, layers, mode, tokens):
+    def __init__(self, ctx, fp8lin, layers, mode, tokens, matmuls="group"):
+        """matmuls: "group" = all matmuls of the step in one fp8_linear_group call (the layers of a step are
+        independent here: every operand is quantised before the first matmul), "per-call" = one call each."""
         self.ctx, self.layers = ctx, layers
         grouped = mode.startswith("group") and tokens > 128 and not any(L.transposed for L in layers)
         self.mode = mode if grouped or not mode.startswith("group") else "per-tensor"
         self.items = None
+        self.mm_items = None
         if grouped:
             self.items = fp8lin.group_items([it for L in layers for it in L.quant_items()])
             self.group_mode = fp8lin.GROUP_PREDICTED if mode == "group-predicted" else fp8lin.GROUP_AMAX_CAST
+            if matmuls == "group":
+                mm = []
+                for L in layers:
+                    bi = L.scal_i
+                    mm.append((fp8lin.MATMUL_FWD, L.x8, bi[1:2], L.w8, bi[0:1], L.y))
+                    if L.backward:
+                        mm.append((fp8lin.MATMUL_DGRAD, L.g8, bi[2:3], L.w8, bi[0:1], L.dx))
+                        mm.append((fp8lin.MATMUL_WGRAD, L.g8, bi[2:3], L.x8, bi[1:2], L.dw))
+                self.mm_items = fp8lin.matmul_items(mm)
+        self.matmuls = "group" if self.mm_items is not None else "per-call"
 
     def launches_per_step(self):
         """Kernel launches the library enqueues per step, counted by the library itself (fp8_launch_count)."""
@@ -342,6 +355,9 @@ class Step:
         ctx = self.ctx
         if self.items is not None:
             _timed(timers, "amax_cast", lambda: ctx.cast_group(self.items, mode=self.group_mode))
+            if self.mm_items is not None:
+                _timed(timers, "gemm", lambda: ctx.linear_group(self.mm_items))
+                return
             for L in self.layers:
                 if timers is not None:
                     la, lb = timers.layer_span(L.name)
@@ -922,6 +938,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--quant", default="group-predicted", choices=QUANT_MODES,
                     help="how the step quantises its tensors (see class Step)")
+    ap.add_argument("--matmuls", default="group", choices=("group", "per-call"),
+                    help="all matmuls of a step in one fp8_linear_group call, or one call each")
     ap.add_argument("--transposed-copies", action="store_true",
                     help="also write transposed FP8 copies and contract the backward matmuls over contiguous bytes "
                          "(per-tensor quantisation)")
@@ -968,7 +986,8 @@ def main():
     if not wl.backward:  # post-training quantisation, once, outside the timed region
         for L in layers:
             ctx.ptq_weights(L.w, fp8lin.CONV_PAPER, L.w8, None, L.scal_i[0:1], L.scal_f[0:1])
-    step = Step(ctx, fp8lin, layers, quant, tokens)
+    step = Step(ctx, fp8lin, layers, quant, tokens, args.matmuls)
+    step_matmuls = step.matmuls
 
     ctx.prediction_stats(clear=True)
     for _ in range(warmup):
@@ -1028,7 +1047,9 @@ def main():
                     "algorithmic_bytes_per_launch": weight_bytes / max(1, gemm_launches / sampled_steps),
                     "timed_on": f"every {EVENT_EVERY}th step of the timed region ({sampled_steps} steps)", "traffic": None}
     else:
-        roofline = {"bound": "tensor", "kernel": "gemm_pair_kernel", "achieved": gemm_tflops, "peak": fp8_peak,
+        roofline = {"bound": "tensor",
+                    "kernel": "gemm_pair_group_kernel (all matmuls of the step in one launch)" if step.matmuls == "group"
+                    else "gemm_pair_kernel", "achieved": gemm_tflops, "peak": fp8_peak,
                     "unit": "TFLOP/s",
                     "peak_source": f"2 x {peaks['source']} {peak_kind} bf16 cuBLAS "
                                    f"({peaks['bf16_tflops' if held_max else 'bf16_tflops_sustained']} TFLOP/s); "
@@ -1036,7 +1057,7 @@ def main():
                     "launches": gemm_launches, "avg_launch_ms": gemm_ms / max(1, gemm_launches),
                     "algorithmic_bytes_per_launch": sum(L.gemm_bytes() for L in layers) / max(1, gemm_launches / sampled_steps),
                     "timed_on": f"every {EVENT_EVERY}th step of the timed region ({sampled_steps} steps)",
-                    "traffic": GEMM_DRAM_BYTES_PER_LAUNCH.get((wl.name, tokens))}
+                    "traffic": GEMM_DRAM_BYTES_PER_LAUNCH.get((wl.name, tokens, step.matmuls))}
     roofline["frac"] = roofline["achieved"] / roofline["peak"]
     if not decode:
         # the same achieved rate against the two other denominators in use: the vendor's dense-FP8 figure (what the
@@ -1091,11 +1112,9 @@ def main():
 
     # ---- the same step under the other quantisation modes (same per-kernel event schedule as the headline) ----
     other_modes = {}
+    layer_ms = timers.layer_ms()   # empty when the step's matmuls are one call; then taken from the per-call leg
     if extra and not decode and not args.transposed_copies:
-        for mode in QUANT_MODES:
-            if mode == step.mode:
-                continue
-            st = Step(ctx, fp8lin, layers, mode, tokens)
+        def time_variant(st):
             for _ in range(3):
                 st.run()
             ctx.prediction_stats(clear=True)
@@ -1110,11 +1129,21 @@ def main():
             barrier_sync(dist)
             m_ms = max_over_ranks(a.elapsed_time(b), dist, device) / m_steps
             m_sampled = (m_steps + EVENT_EVERY - 1) // EVENT_EVERY
-            other_modes[mode] = {"value": whole_job_value(world, step_flops, m_ms), "unit": UNIT, "ms_per_step": m_ms,
-                                 "steps": m_steps, "amax_cast_ms_per_step": tm.total_ms("amax_cast") / m_sampled,
-                                 "launches_per_step": st.launches_per_step()}
-            if "predicted" in mode:
-                other_modes[mode]["guesses_held_missed"] = list(ctx.prediction_stats(clear=True))
+            out = {"value": whole_job_value(world, step_flops, m_ms), "unit": UNIT, "ms_per_step": m_ms,
+                   "steps": m_steps, "amax_cast_ms_per_step": tm.total_ms("amax_cast") / m_sampled,
+                   "gemm_ms_per_step": tm.total_ms("gemm") / m_sampled, "matmuls": st.matmuls,
+                   "launches_per_step": st.launches_per_step()}
+            if "predicted" in st.mode:
+                out["guesses_held_missed"] = list(ctx.prediction_stats(clear=True))
+            return out, tm
+
+        if step.matmuls == "group":   # the headline's quantisation with one call per matmul: what the one launch buys
+            other_modes["per-call matmuls"], tm_calls = time_variant(Step(ctx, fp8lin, layers, step.mode, tokens, "per-call"))
+            layer_ms = tm_calls.layer_ms()
+        for mode in QUANT_MODES:
+            if mode == step.mode:
+                continue
+            other_modes[mode], _ = time_variant(Step(ctx, fp8lin, layers, mode, tokens, args.matmuls))
 
     # ---- gradients whose magnitude moves every step: what a wrong guess costs ----
     moving = None
@@ -1320,6 +1349,9 @@ def main():
                    "passes": "fwd+bwd" if wl.backward else "fwd (weights quantised once at load)",
                    "scaling_bias": quant_note if wl.backward else "FP8-AMAX for X every step; " + quant_note,
                    "quantisation_mode": "per-tensor" if decode and quant.startswith("group") else quant,
+                   "matmuls": "all matmuls of the step in one fp8_linear_group call (one persistent launch; the layers of "
+                              "a step are independent here)" if step_matmuls == "group" else "one call per matmul",
+
                    "l2": "inputs larger than L2 (each layer's tensors exceed 126 MB); no flush between steps",
                    "fp8_layouts": "row-major + transposed copy" if args.transposed_copies else "row-major only",
                    "parallelism": "replicas" if world > 1 else "single"},
@@ -1337,7 +1369,7 @@ def main():
                               "kernel alone against its own bytes; other_modes and moving_gradients the same step under "
                               "the other quantisation paths and with biases that move",
                       "per_kernel": per_kernel},
-        "layer_matmul_ms": {k: round(v, 4) for k, v in timers.layer_ms().items()},
+        "layer_matmul_ms": {k: round(v, 4) for k, v in layer_ms.items()},
         "other_modes": other_modes,
         "moving_gradients": moving,
         "with_cuda_graph": graphed,

@@ -363,6 +363,39 @@ FP8_API fp8_status_t fp8_linear_infer_cast(fp8_ctx *ctx, const void *x, fp8_dtyp
                                    const void *bias_vec, fp8_dtype_t bias_dt, void *y, fp8_dtype_t y_dt,
                                    float *d_amax_y, int64_t T, int64_t K, int64_t N, fp8_conv_t conv, void *stream);
 
+/* Several independent matmuls in one launch (the paper has no counterpart; Section 2.2 is where they come from: the
+ * input-gradient and weight-gradient matmuls of a layer share dY8 and do not depend on each other, nor do the
+ * matmuls of different layers whose operands are ready).  Each item is one fp8_linear_fwd, fp8_linear_dgrad or
+ * fp8_linear_wgrad call on row-major operands, with that call's meaning, checks and results (the FP32 sums may be
+ * taken in another order than the member's own launch would take them: same bars, not always the same last bit):
+ *   FP8_MATMUL_FWD    a8 = x8 [T, K] (E4),  b8 = w8 [N, K] (E4), out = Y [T, N]; bias_vec / bias_dt as in fp8_linear_fwd
+ *   FP8_MATMUL_DGRAD  a8 = dy8 [T, N] (E5), b8 = w8 [N, K] (E4), out = dX [T, K]   (fp8_linear_dgrad with w8_t = NULL)
+ *   FP8_MATMUL_WGRAD  a8 = dy8 [T, N] (E5), b8 = x8 [T, K] (E4), out = dW [N, K]   (fp8_linear_wgrad with both
+ *                     transposed copies NULL); d_amax_out must be NULL
+ *   d_ba, d_bb        device int32 biases of a8 and b8;  out_dt FP8_BF16 or FP8_F32;  d_amax_out NULL or the amax of out
+ * No item may read what another item of the same call writes.  `items` is a HOST array, read during the call only.
+ * With at most 16 items, all of more than 128 output rows, one persistent kernel walks the output tiles of all
+ * items in one sequence (shortest contractions first), so the launch pays one ramp and one drain and the last wave
+ * of one matmul is filled with the first tiles of the next; any other group runs as its members' own calls, in
+ * order.  Argument errors of any member are returned before anything of a one-launch group is enqueued. */
+typedef enum { FP8_MATMUL_FWD = 0, FP8_MATMUL_DGRAD = 1, FP8_MATMUL_WGRAD = 2 } fp8_matmul_kind_t;
+typedef struct {
+    int32_t kind;            /* fp8_matmul_kind_t */
+    int32_t bias_dt;         /* fp8_dtype_t of bias_vec (FWD) */
+    const uint8_t *a8;
+    const int32_t *d_ba;
+    const uint8_t *b8;
+    const int32_t *d_bb;
+    const void *bias_vec;    /* FWD: NULL or [N]; otherwise NULL */
+    void *out;
+    float *d_amax_out;
+    int32_t out_dt;          /* fp8_dtype_t */
+    int32_t reserved;        /* 0 */
+    int64_t T, K, N;         /* of the layer: tokens, in-features, out-features */
+} fp8_matmul_item_t;
+FP8_API fp8_status_t fp8_linear_group(fp8_ctx *ctx, const fp8_matmul_item_t *items, int32_t count, fp8_conv_t conv,
+                              void *stream);
+
 /* Forward matmul with the activation fused into the epilogue (the paper has no
  * counterpart; it answers Section 3's warning that computing a scale just in
  * time costs a second pass over memory: the next layer's input leaves this

@@ -389,8 +389,13 @@ __device__ __forceinline__ void slab_publish(const CUtensorMap *map, uint32_t sl
 {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     __syncwarp();
-    if (lane == 0 && in_range) {
-        if (stream) tma_store_2d_stream(map, slab, x, y);
+    if (lane == 0) {
+        // One bulk group per slab use, store or no store: slab_acquire counts groups.  (A chunk beyond the last column
+        // of a ragged tile used to commit nothing, so the count ran ahead and a slab could be rewritten while the
+        // store of the tile's last real chunk was still reading it: seen as zeros in the last columns of a tensor,
+        // in a few per cent of launches on a busy GPU.)
+        if (!in_range) asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+        else if (stream) tma_store_2d_stream(map, slab, x, y);
         else tma_store_2d(map, slab, x, y);
     }
 }
@@ -2027,6 +2032,225 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
 }
 
 
+// ---------------------------------------------------------------------------
+// CTA-pair kernel over a list of independent problems (fp8_linear_group)
+// ---------------------------------------------------------------------------
+//
+// The plain CTA-pair kernel with one more level in its tile loop: the tiles of up to kGroupGemmMax matmuls are
+// numbered in one sequence (problem after problem, each in its own rasterisation order) and pair q takes numbers
+// q, q + pairs, q + 2 pairs, ...  One launch therefore pays one prologue and one drain for all of them, and the last
+// wave of one problem is filled up with the first tiles of the next.  Per tile the three roles look up the problem
+// the number falls in (the lists are short and the numbers only grow, so the index only moves forward) and take its
+// shapes, layouts, instruction descriptor, tensor maps, biases and output from that entry.  Everything else -- stage
+// ring, barriers, accumulator hand-over, epilogue -- is the pair kernel's, and carries on across problem boundaries
+// without a pause.  Plain epilogue only, no split contraction.  A tile walks the contraction backwards when its
+// number within its own problem falls in an odd round of the pairs, which is the direction the single launch of that
+// problem would give it (same sums in the same order: same bits).
+
+constexpr int kGroupGemmMax = 16;
+
+struct GroupGemmParams {
+    CUtensorMap map_a[kGroupGemmMax], map_b[kGroupGemmMax], map_out[kGroupGemmMax];
+    GemmParams p[kGroupGemmMax];
+    int first_tile[kGroupGemmMax + 1];   // tile numbers of problem i: [first_tile[i], first_tile[i + 1])
+    int count;
+};
+
+template <int NHALF>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1)
+gemm_pair_group_kernel(const __grid_constant__ GroupGemmParams gg)
+{
+    using L = PairSmemT<NHALF == 2 ? kWideStages : kPairStages, kPairSlabs, NHALF>;
+    constexpr int kStagesL = L::kStages;
+    constexpr int kTileN = kPairBN * NHALF;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    const uint32_t smem_base = smem_u32(smem);
+    const uint32_t bar_base = smem_base + L::kBarOffset;
+    auto full_bar = [&](int s) { return bar_base + 8u * s; };
+    auto empty_bar = [&](int s) { return bar_base + 8u * (kStagesL + s); };
+    auto acc_full_bar = [&](int b) { return bar_base + 8u * (2 * kStagesL + b); };
+    auto acc_empty_bar = [&](int b) { return bar_base + 8u * (2 * kStagesL + 2 + b); };
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + L::kBarOffset + L::kNumBars * 8);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank();
+    const int num_tiles = gg.first_tile[gg.count];
+    const int pair_id = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
+    unsigned *const d_status = gg.p[0].d_status;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStagesL; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(acc_full_bar(b), 1); mbar_init(acc_empty_bar(b), 8); }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                     "r"((uint32_t)L::kTmemCols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();  // both CTAs' barriers exist before anyone signals across
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            uint32_t it = 0;
+            bool alive = true;
+            const uint32_t leader_full0 = map_to_cta(full_bar(0), 0);
+            asm volatile("griddepcontrol.wait;" ::: "memory");
+            int pi = 0;
+            for (int tile = pair_id; alive && tile < num_tiles; tile += num_pairs) {
+                while (tile >= gg.first_tile[pi + 1]) ++pi;
+                const GemmParams &p = gg.p[pi];
+                const CUtensorMap *map_a = &gg.map_a[pi], *map_b = &gg.map_b[pi];
+                const int local = tile - gg.first_tile[pi];
+                int m_blk, n_blk;
+                tile_coords(local, p, m_blk, n_blk);
+                const bool backwards = ((local / num_pairs) & 1) != 0 && p.serpentine;
+                for (int k = 0; k < p.num_k; ++k, ++it) {
+                    const int kc = (backwards ? p.num_k - 1 - k : k) * kBK;
+                    const int s = it % kStagesL;
+                    const uint32_t leader_full = leader_full0 + 8u * s;
+                    const uint32_t ph = (it / kStagesL) & 1u;
+                    if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, d_status)) { alive = false; break; }
+                    if (rank == 0) mbar_expect_tx(full_bar(s), 2 * L::kStageBytes);
+                    const uint32_t a_dst = smem_base + s * L::kStageBytes;
+                    const int a_row = m_blk * 256 + (int)rank * kBM;
+                    if (p.a_mn) tma_load_2d_pair(a_dst, map_a, leader_full, a_row, kc);
+                    else tma_load_2d_pair(a_dst, map_a, leader_full, kc, a_row);
+#pragma unroll
+                    for (int h = 0; h < NHALF; ++h) {
+                        const int b_row = n_blk * kTileN + h * kPairBN + (int)rank * kPairHalfN;
+                        const uint32_t b_dst = a_dst + L::kABytes + h * (kPairHalfN * kBK);
+                        if (p.b_mn) tma_load_2d_pair(b_dst, map_b, leader_full, b_row, kc);
+                        else tma_load_2d_pair(b_dst, map_b, leader_full, kc, b_row);
+                    }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0 && rank == 0) {
+            uint32_t it = 0, t = 0;
+            bool alive = true;
+            asm volatile("griddepcontrol.wait;" ::: "memory");
+            int pi = 0;
+            for (int tile = pair_id; alive && tile < num_tiles; tile += num_pairs, ++t) {
+                while (tile >= gg.first_tile[pi + 1]) ++pi;
+                const GemmParams &p = gg.p[pi];
+                const int buf = NHALF == 2 ? 0 : (t & 1);
+                const uint32_t acc_ph = NHALF == 2 ? (t & 1u) : ((t >> 1) & 1u);
+                if (!mbar_wait(acc_empty_bar(buf), acc_ph ^ 1u, abort_flag, d_status)) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + buf * kPairBN;
+                const int k1 = p.num_k;
+                const uint32_t idesc = p.idesc;
+                const bool a_mn = p.a_mn != 0, b_mn = p.b_mn != 0;
+                auto issue = [&](int s, int k, int h) {
+                    const uint32_t a_addr = smem_base + s * L::kStageBytes;
+                    const uint32_t b_addr = a_addr + L::kABytes + h * (kPairHalfN * kBK);
+                    const uint64_t da = a_mn ? smem_desc_mn128(a_addr, 128 * kBK) : smem_desc_k128(a_addr);
+                    const uint64_t db = b_mn ? smem_desc_mn128(b_addr, 128 * kBK) : smem_desc_k128(b_addr);
+                    const uint32_t step_a = a_mn ? 256u : 2u, step_b = b_mn ? 256u : 2u;
+#pragma unroll
+                    for (int j = 0; j < kBK / kUmmaK; ++j)
+                        umma_f8_pair(d_tmem + h * kPairBN, da + step_a * j, db + step_b * j, idesc, (k > 0 || j > 0) ? 1u : 0u);
+                };
+                int k = 0;
+                if (NHALF == 2) {   // as in the pair kernel: the first k-blocks run on half 0 while half 1 is still being read
+                    const int ahead = min(k1, kStagesL - 1);
+                    for (int a = 0; alive && a < ahead; ++a) {
+                        const uint32_t ia = it + a;
+                        if (!mbar_wait(full_bar(ia % kStagesL), (ia / kStagesL) & 1u, abort_flag, d_status)) { alive = false; break; }
+                        tc_fence_after();
+                        issue(ia % kStagesL, a, 0);
+                    }
+                    if (alive && !mbar_wait(acc_empty_bar(1), acc_ph ^ 1u, abort_flag, d_status)) alive = false;
+                    if (!alive) break;
+                    tc_fence_after();
+                    for (int a = 0; a < ahead; ++a, ++it) {
+                        issue(it % kStagesL, a, 1);
+                        umma_commit_pair(empty_bar(it % kStagesL));
+                    }
+                    k = ahead;
+                }
+                for (; k < k1; ++k, ++it) {
+                    const int s = it % kStagesL;
+                    const uint32_t ph = (it / kStagesL) & 1u;
+                    if (!mbar_wait(full_bar(s), ph, abort_flag, d_status)) { alive = false; break; }
+                    tc_fence_after();
+#pragma unroll
+                    for (int h = 0; h < NHALF; ++h) issue(s, k, h);
+                    umma_commit_pair(empty_bar(s));
+                }
+                if (alive) umma_commit_pair(acc_full_bar(buf));
+            }
+        }
+    } else {
+        asm volatile("griddepcontrol.wait;" ::: "memory");  // the biases may come from the launch before
+        const int q = warp & 3;
+        uint32_t amax_bits = 0, slab_count = 0;
+        const uint32_t warp_slabs = smem_base + L::kEpiOffset + q * L::kSlabs * kSlabBytes;
+        const uint32_t leader_acc_empty0 = map_to_cta(acc_empty_bar(0), 0);
+        uint32_t t = 0;
+        int pi = 0, cur = -1;
+        Pow2Pair sc = make_pow2_pair(0);
+        bool two_step = false;
+        // the output amax of a problem is folded into its word when this warp moves on to the next problem
+        auto flush_amax = [&](int done) {
+            if (done >= 0 && gg.p[done].d_amax_bits) {
+                amax_bits = __reduce_max_sync(0xFFFFFFFFu, amax_bits);
+                if (lane == 0 && amax_bits) atomicMax(gg.p[done].d_amax_bits, amax_bits);
+            }
+            amax_bits = 0;
+        };
+        for (int tile = pair_id; tile < num_tiles; tile += num_pairs, ++t) {
+            while (tile >= gg.first_tile[pi + 1]) ++pi;
+            const GemmParams &p = gg.p[pi];
+            if (pi != cur) {
+                flush_amax(cur);
+                cur = pi;
+                const int e = -(__ldcg(p.d_sa) + __ldcg(p.d_sb) + p.delta_sum);
+                sc = make_pow2_pair(e);
+                two_step = (e < -126 || e > 127);
+            }
+            int m_blk, n_blk;
+            tile_coords(tile - gg.first_tile[pi], p, m_blk, n_blk);
+            const int buf = NHALF == 2 ? 0 : (t & 1);
+            const uint32_t acc_ph = NHALF == 2 ? (t & 1u) : ((t >> 1) & 1u);
+            const bool ready = mbar_wait(acc_full_bar(buf), acc_ph, abort_flag, d_status);
+            if (!__all_sync(0xFFFFFFFFu, ready)) break;
+            tc_fence_after();
+            const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + buf * kPairBN;
+#pragma unroll 1
+            for (int h = 0; h < NHALF; ++h)
+                epilogue_tile<kPairBN, 0, L::kSlabs>(&gg.map_out[pi], &gg.map_out[pi], t_row + h * kPairBN,
+                                                     m_blk * 256 + (int)rank * kBM + q * 32, n_blk * kTileN + h * kPairBN, p,
+                                                     sc, two_step, amax_bits, warp_slabs, slab_count,
+                                                     leader_acc_empty0 + 8u * (NHALF == 2 ? h : buf), true, lane);
+        }
+        if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+        flush_amax(cur);
+    }
+
+    __syncwarp();
+    if (*abort_flag) __nanosleep(20000);
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();  // neither CTA releases shared or tensor memory while its peer may still touch it
+    tc_fence_after();
+    if (warp == 1)
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)L::kTmemCols)
+                     : "memory");
+}
+
+
 // Second half of a split-K matmul: add the partial sums in a fixed order, then
 // the same unscale / bias / rounding / amax as the fused epilogue.
 // VEC = 4: four adjacent columns per thread through 16-byte loads (N a multiple of 4, output 16-byte aligned), all
@@ -2141,6 +2365,8 @@ static int g_force_bn = 0;              // set from FP8LIN_DECODE_BN (experiment
 static bool g_no_out_stream = false;    // set from FP8LIN_OUT_STREAM=0 (A/B: output stores without the evict-first mark)
 static bool g_no_serpentine = false;    // set from FP8LIN_SERPENTINE=0 (A/B: every tile walks the contraction forwards)
 static int g_force_wide = -1;           // set from FP8LIN_WIDE=0/1 (A/B: never / always the 256 x 512 pair tile)
+static bool g_no_group_gemm = false;    // set from FP8LIN_GROUP_GEMM=0 (A/B: fp8_linear_group as its members' own launches)
+static int g_group_order = 0;           // set from FP8LIN_GROUP_ORDER (experiments: 0 shortest contraction first, 1 longest first, 2 as given)
 static int g_max_pairs = 0;  // CTA pairs that can be resident at once (0: pair kernel unavailable)
 
 #ifndef FP8LIN_WIDE_DEFAULT
@@ -2186,6 +2412,11 @@ cudaError_t configure_gemm_kernels(int max_smem_optin)
                                  GemmSmem<kBN, kStagesF16Acc, kActSlabs>::kDynamic);
     if (e == cudaSuccess)
         e = cudaFuncSetAttribute(decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecodeSmemBudget + 1024);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(gemm_pair_group_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, PairSmem::kDynamic);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(gemm_pair_group_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 PairSmemWide::kDynamic);
     if (e != cudaSuccess) return e;
     for (int cs = 2; cs <= kDecodeMaxCluster; ++cs) {   // how many clusters of each size fit the GPU at once
         cudaLaunchAttribute attr[1];
@@ -2260,6 +2491,10 @@ cudaError_t configure_gemm_kernels(int max_smem_optin)
     g_direct_epilogue = env && env[0] == '1';
     env = getenv("FP8LIN_WIDE");
     g_force_wide = env ? atoi(env) : -1;
+    env = getenv("FP8LIN_GROUP_GEMM");
+    g_no_group_gemm = env && env[0] == '0';
+    env = getenv("FP8LIN_GROUP_ORDER");
+    g_group_order = env ? atoi(env) : 0;
     if (getenv("FP8LIN_DEBUG")) {
         fprintf(stderr, "fp8lin: %d SMs, %d resident CTA pairs, pair kernel %s\n", sms, clusters, g_force_single ? "off" : "on");
         fprintf(stderr, "fp8lin: resident decode clusters of 2..8 CTAs: %d %d %d %d %d %d %d\n", g_decode_clusters[2],
@@ -2400,6 +2635,14 @@ struct FusedQuant {
     int margin, conv;
 };
 
+// Where run_gemm leaves a prepared problem instead of launching it (fp8_linear_group): entry `index` of `gg`, in
+// the tile shape the whole group uses.
+struct GroupSlot {
+    GroupGemmParams *gg;
+    int index;
+    bool wide;
+};
+
 // D[M,N] = A * B^T over a contraction of length Kc, unscaled by 2^-(bias_a + bias_b + delta_sum).
 // A is stored [M, Kc] (a_mn = false) or [Kc, M] (a_mn = true); B is stored [N, Kc] or [Kc, N] likewise.
 static fp8_status_t run_gemm(fp8_ctx *ctx, const uint8_t *a, int a_fmt, bool a_mn, const int32_t *d_ba,
@@ -2408,10 +2651,11 @@ static fp8_status_t run_gemm(fp8_ctx *ctx, const uint8_t *a, int a_fmt, bool a_m
                              int64_t N, int64_t Kc, cudaStream_t st, int act = 0, void *out_act = nullptr,
                              const void *aux = nullptr, uint8_t *out8 = nullptr, const int32_t *d_sq = nullptr,
                              int q_fmt = 0, int delta_q = 0, bool no_loads = false, int chunk_kb = 0, bool static_b = false,
-                             const FusedQuant *fq = nullptr)
+                             const FusedQuant *fq = nullptr, GroupSlot *slot = nullptr)
 {
     if (M > 0x7FFFFFFF / 2 || N > 0x7FFFFFFF / 2 || Kc > 0x7FFFFFFF / 2) return FP8_ERR_SHAPE;
     const bool pair = g_max_pairs > 0 && M > kBM && !g_force_single && act != 6;
+    if (slot && (!pair || act != 0 || no_loads || fq)) return FP8_ERR_UNSUPPORTED;
     CUtensorMap map_a, map_b;
     // an operand stored [Kc, M or N] is fetched as boxes of 128 contraction rows x 128 bytes
     // With a few rows of A (decode) the box covers those rows only, rounded up to the 8-row swizzle atom: the other
@@ -2459,7 +2703,7 @@ static fp8_status_t run_gemm(fp8_ctx *ctx, const uint8_t *a, int a_fmt, bool a_m
     p.b_mn = b_mn ? 1 : 0;
     p.a_box_bytes = a_box_rows * kBK;
     p.M = (int)M; p.N = (int)N; p.K = (int)Kc;
-    const bool wide = pair && act == 0 && use_wide_tile(M, N, Kc);
+    const bool wide = pair && act == 0 && (slot ? slot->wide : use_wide_tile(M, N, Kc));
     p.tiles_m = (int)((M + (pair ? 256 : kBM) - 1) / (pair ? 256 : kBM));
     p.tiles_n = (int)((N + (wide ? 2 * kBN : kBN) - 1) / (wide ? 2 * kBN : kBN));
     p.num_k = (int)((Kc + kBK - 1) / kBK);
@@ -2521,7 +2765,7 @@ static fp8_status_t run_gemm(fp8_ctx *ctx, const uint8_t *a, int a_fmt, bool a_m
             p.splits = (p.num_k + p.kb_per_split - 1) / p.kb_per_split;
         }
     }
-    if (pair && !g_no_splitk && !act && !no_loads) {
+    if (pair && !g_no_splitk && !act && !no_loads && !slot) {
         // Fewer tiles than CTA pairs and a long contraction: slice it so that most pairs have work.  The second
         // launch and the trip of the partial sums through memory cost 6-7 us, so a slice keeps at least sixteen
         // k-blocks (measured: 1024 x 1024 x 8192 27 -> 22 us, 512 x 512 x 16384 46 -> 20 us; at 32 k-blocks or fewer
@@ -2582,6 +2826,14 @@ static fp8_status_t run_gemm(fp8_ctx *ctx, const uint8_t *a, int a_fmt, bool a_m
     p.idesc = (pair ? make_idesc_pair(a_fmt, b_fmt) : make_idesc(a_fmt, b_fmt, decode ? p.dec_bn : kBN)) | ((uint32_t)p.a_mn << 15) |
               ((uint32_t)p.b_mn << 16);
     if (d_amax_out && cudaMemsetAsync(d_amax_out, 0, sizeof(float), st) != cudaSuccess) return FP8_ERR_CUDA;
+    if (slot) {   // prepared, not launched: the group's one launch runs it
+        GroupGemmParams &g = *slot->gg;
+        g.p[slot->index] = p;
+        g.map_a[slot->index] = map_a;
+        g.map_b[slot->index] = map_b;
+        g.map_out[slot->index] = map_out;
+        return FP8_OK;
+    }
     int tiles = p.tiles_m * p.tiles_n;
     const bool finalize = p.splits > 1 && act != 6 && p.dec_cluster <= 1;
     count_launch(finalize ? 2 : 1);
@@ -2688,10 +2940,10 @@ static bool out_dtype_ok(int dt) { return dt == FP8_BF16 || dt == FP8_F32; }
 
 extern "C" {
 
-fp8_status_t fp8_linear_fwd(fp8_ctx *ctx, const uint8_t *x8, const int32_t *d_bx, const uint8_t *w8,
-                            const int32_t *d_bw, const void *bias_vec, fp8_dtype_t bias_dt, void *y,
-                            fp8_dtype_t y_dt, float *d_amax_y, int64_t T, int64_t K, int64_t N, fp8_conv_t conv,
-                            void *stream)
+static fp8_status_t linear_fwd_impl(fp8_ctx *ctx, const uint8_t *x8, const int32_t *d_bx, const uint8_t *w8,
+                                    const int32_t *d_bw, const void *bias_vec, fp8_dtype_t bias_dt, void *y,
+                                    fp8_dtype_t y_dt, float *d_amax_y, int64_t T, int64_t K, int64_t N, fp8_conv_t conv,
+                                    void *stream, fp8lin::GroupSlot *slot)
 {
     using namespace fp8lin;
     if (!ctx || !x8 || !d_bx || !w8 || !d_bw || !y) return FP8_ERR_NULL;
@@ -2702,7 +2954,16 @@ fp8_status_t fp8_linear_fwd(fp8_ctx *ctx, const uint8_t *x8, const int32_t *d_bx
     if (!aligned16(x8) || !aligned16(w8) || (K % 16) != 0 || (reinterpret_cast<uintptr_t>(y) & 3u)) return FP8_ERR_ALIGN;
     int delta = 2 * format_delta(FP8_E4, conv);
     return run_gemm(ctx, x8, FP8_E4, false, d_bx, w8, FP8_E4, false, d_bw, delta, bias_vec, bias_dt, y, y_dt, d_amax_y,
-                    T, N, K, (cudaStream_t)stream);
+                    T, N, K, (cudaStream_t)stream, 0, nullptr, nullptr, nullptr, nullptr, 0, 0, false, 0, false, nullptr,
+                    slot);
+}
+
+fp8_status_t fp8_linear_fwd(fp8_ctx *ctx, const uint8_t *x8, const int32_t *d_bx, const uint8_t *w8,
+                            const int32_t *d_bw, const void *bias_vec, fp8_dtype_t bias_dt, void *y,
+                            fp8_dtype_t y_dt, float *d_amax_y, int64_t T, int64_t K, int64_t N, fp8_conv_t conv,
+                            void *stream)
+{
+    return linear_fwd_impl(ctx, x8, d_bx, w8, d_bw, bias_vec, bias_dt, y, y_dt, d_amax_y, T, K, N, conv, stream, nullptr);
 }
 
 fp8_status_t fp8_linear_infer(fp8_ctx *ctx, const uint8_t *x8, const int32_t *d_bx, const uint8_t *w8,
@@ -2815,9 +3076,10 @@ fp8_status_t fp8_linear_fwd_act(fp8_ctx *ctx, const uint8_t *x8, const int32_t *
                     d_amax_act, T, N, K, (cudaStream_t)stream, swiglu ? 4 : 1, y_act);
 }
 
-fp8_status_t fp8_linear_dgrad(fp8_ctx *ctx, const uint8_t *dy8, const int32_t *d_bg, const uint8_t *w8,
-                              const uint8_t *w8_t, const int32_t *d_bw, void *dx, fp8_dtype_t dx_dt,
-                              float *d_amax_dx, int64_t T, int64_t K, int64_t N, fp8_conv_t conv, void *stream)
+static fp8_status_t linear_dgrad_impl(fp8_ctx *ctx, const uint8_t *dy8, const int32_t *d_bg, const uint8_t *w8,
+                                      const uint8_t *w8_t, const int32_t *d_bw, void *dx, fp8_dtype_t dx_dt,
+                                      float *d_amax_dx, int64_t T, int64_t K, int64_t N, fp8_conv_t conv, void *stream,
+                                      fp8lin::GroupSlot *slot)
 {
     using namespace fp8lin;
     if (!ctx || !dy8 || !d_bg || (!w8 && !w8_t) || !d_bw || !dx) return FP8_ERR_NULL;
@@ -2833,7 +3095,14 @@ fp8_status_t fp8_linear_dgrad(fp8_ctx *ctx, const uint8_t *dy8, const int32_t *d
         return FP8_ERR_ALIGN;
     int delta = format_delta(FP8_E5, conv) + format_delta(FP8_E4, conv);
     return run_gemm(ctx, dy8, FP8_E5, false, d_bg, w, FP8_E4, w_mn, d_bw, delta, nullptr, 0, dx, dx_dt, d_amax_dx, T, K,
-                    N, (cudaStream_t)stream);
+                    N, (cudaStream_t)stream, 0, nullptr, nullptr, nullptr, nullptr, 0, 0, false, 0, false, nullptr, slot);
+}
+
+fp8_status_t fp8_linear_dgrad(fp8_ctx *ctx, const uint8_t *dy8, const int32_t *d_bg, const uint8_t *w8,
+                              const uint8_t *w8_t, const int32_t *d_bw, void *dx, fp8_dtype_t dx_dt,
+                              float *d_amax_dx, int64_t T, int64_t K, int64_t N, fp8_conv_t conv, void *stream)
+{
+    return linear_dgrad_impl(ctx, dy8, d_bg, w8, w8_t, d_bw, dx, dx_dt, d_amax_dx, T, K, N, conv, stream, nullptr);
 }
 
 fp8_status_t fp8_linear_dgrad_act(fp8_ctx *ctx, const uint8_t *dy8, const int32_t *d_bg, const uint8_t *w8,
@@ -2924,9 +3193,10 @@ fp8_status_t fp8_linear_f16acc(fp8_ctx *ctx, fp8_matmul_t kind, const uint8_t *a
                     contraction, (cudaStream_t)stream, 6, nullptr, nullptr, nullptr, nullptr, 0, 0, false, chunk / kBK);
 }
 
-fp8_status_t fp8_linear_wgrad(fp8_ctx *ctx, const uint8_t *dy8, const uint8_t *dy8_t, const int32_t *d_bg,
-                              const uint8_t *x8, const uint8_t *x8_t, const int32_t *d_bx, void *dw,
-                              fp8_dtype_t dw_dt, int64_t T, int64_t K, int64_t N, fp8_conv_t conv, void *stream)
+static fp8_status_t linear_wgrad_impl(fp8_ctx *ctx, const uint8_t *dy8, const uint8_t *dy8_t, const int32_t *d_bg,
+                                      const uint8_t *x8, const uint8_t *x8_t, const int32_t *d_bx, void *dw,
+                                      fp8_dtype_t dw_dt, int64_t T, int64_t K, int64_t N, fp8_conv_t conv, void *stream,
+                                      fp8lin::GroupSlot *slot)
 {
     using namespace fp8lin;
     if (!ctx || (!dy8 && !dy8_t) || !d_bg || (!x8 && !x8_t) || !d_bx || !dw) return FP8_ERR_NULL;
@@ -2942,7 +3212,113 @@ fp8_status_t fp8_linear_wgrad(fp8_ctx *ctx, const uint8_t *dy8, const uint8_t *d
         return FP8_ERR_ALIGN;
     int delta = format_delta(FP8_E5, conv) + format_delta(FP8_E4, conv);
     return run_gemm(ctx, g, FP8_E5, g_mn, d_bg, xx, FP8_E4, x_mn, d_bx, delta, nullptr, 0, dw, dw_dt, nullptr, N, K, T,
-                    (cudaStream_t)stream);
+                    (cudaStream_t)stream, 0, nullptr, nullptr, nullptr, nullptr, 0, 0, false, 0, false, nullptr, slot);
+}
+
+fp8_status_t fp8_linear_wgrad(fp8_ctx *ctx, const uint8_t *dy8, const uint8_t *dy8_t, const int32_t *d_bg,
+                              const uint8_t *x8, const uint8_t *x8_t, const int32_t *d_bx, void *dw,
+                              fp8_dtype_t dw_dt, int64_t T, int64_t K, int64_t N, fp8_conv_t conv, void *stream)
+{
+    return linear_wgrad_impl(ctx, dy8, dy8_t, d_bg, x8, x8_t, d_bx, dw, dw_dt, T, K, N, conv, stream, nullptr);
+}
+
+// One matmul of a group, through the same checks and set-up as its own entry point.
+static fp8_status_t group_item_call(fp8_ctx *ctx, const fp8_matmul_item_t &m, fp8_conv_t conv, void *stream,
+                                    fp8lin::GroupSlot *slot)
+{
+    switch (m.kind) {
+    case FP8_MATMUL_FWD:
+        return linear_fwd_impl(ctx, m.a8, m.d_ba, m.b8, m.d_bb, m.bias_vec, (fp8_dtype_t)m.bias_dt, m.out,
+                               (fp8_dtype_t)m.out_dt, m.d_amax_out, m.T, m.K, m.N, conv, stream, slot);
+    case FP8_MATMUL_DGRAD:
+        return linear_dgrad_impl(ctx, m.a8, m.d_ba, m.b8, nullptr, m.d_bb, m.out, (fp8_dtype_t)m.out_dt, m.d_amax_out, m.T,
+                                 m.K, m.N, conv, stream, slot);
+    case FP8_MATMUL_WGRAD:
+        if (m.d_amax_out) return FP8_ERR_UNSUPPORTED;
+        return linear_wgrad_impl(ctx, m.a8, nullptr, m.d_ba, m.b8, nullptr, m.d_bb, m.out, (fp8_dtype_t)m.out_dt, m.T, m.K,
+                                 m.N, conv, stream, slot);
+    default: return FP8_ERR_DTYPE;
+    }
+}
+
+fp8_status_t fp8_linear_group(fp8_ctx *ctx, const fp8_matmul_item_t *items, int32_t count, fp8_conv_t conv, void *stream)
+{
+    using namespace fp8lin;
+    if (!ctx || !items) return FP8_ERR_NULL;
+    if (count <= 0) return FP8_ERR_SHAPE;
+    if ((int)conv < 0 || (int)conv > 1) return FP8_ERR_DTYPE;
+    // rows, columns and contraction length of each item as a matmul
+    auto dims = [](const fp8_matmul_item_t &m, int64_t &M, int64_t &N, int64_t &Kc) {
+        if (m.kind == FP8_MATMUL_FWD) { M = m.T; N = m.N; Kc = m.K; }
+        else if (m.kind == FP8_MATMUL_DGRAD) { M = m.T; N = m.K; Kc = m.N; }
+        else { M = m.N; N = m.K; Kc = m.T; }
+    };
+    bool one_launch = count <= kGroupGemmMax && g_max_pairs > 0 && !g_force_single && !g_no_group_gemm;
+    bool wide = kWideTileDefault && g_force_wide != 0;
+    for (int i = 0; i < count; ++i) {
+        if (items[i].kind < 0 || items[i].kind > 2) return FP8_ERR_DTYPE;
+        if (items[i].T <= 0 || items[i].K <= 0 || items[i].N <= 0) return FP8_ERR_SHAPE;
+        int64_t M, N, Kc;
+        dims(items[i], M, N, Kc);
+        if (M <= kBM) one_launch = false;   // a decode-size member: its own kernel, its own launch
+        if (Kc < 2048 || ((N + 511) / 512) * 512 - N > N / 32) wide = false;   // the wide tile would waste its width
+    }
+    if (g_force_wide == 1) wide = true;
+    if (!one_launch) {
+        for (int i = 0; i < count; ++i) {
+            const fp8_status_t st = group_item_call(ctx, items[i], conv, stream, nullptr);
+            if (st != FP8_OK) return st;
+        }
+        return FP8_OK;
+    }
+    // Shortest contractions first.  Where one problem ends and the next begins some pairs are a tile ahead of the
+    // others, by the difference of the two tile times, and stay so; pairs that share operand strips hit in L2 only while
+    // they walk them at about the same time.  In this order the large differences come last (measured on the twelve
+    // matmuls of a 7B-class step: 3.22 ms and 3.3 GB read from DRAM, against 3.27 ms and 4.6 GB longest first, 3.29 ms
+    // in the caller's order, 3.38 ms as twelve launches).
+    int order[kGroupGemmMax];
+    for (int i = 0; i < count; ++i) order[i] = i;
+    for (int i = 1; i < count; ++i) {   // insertion sort, stable
+        int64_t Mi, Ni, Ki;
+        const int oi = order[i];
+        dims(items[oi], Mi, Ni, Ki);
+        int j = i;
+        for (; j > 0; --j) {
+            int64_t Mj, Nj, Kj;
+            dims(items[order[j - 1]], Mj, Nj, Kj);
+            if (g_group_order == 2 || (g_group_order == 1 ? Kj >= Ki : Kj <= Ki)) break;
+            order[j] = order[j - 1];
+        }
+        order[j] = oi;
+    }
+    static thread_local GroupGemmParams gg;   // about 11 KB: filled per call, copied by the launch
+    gg.count = count;
+    gg.first_tile[0] = 0;
+    for (int i = 0; i < count; ++i) {
+        GroupSlot slot = {&gg, i, wide};
+        const fp8_status_t st = group_item_call(ctx, items[order[i]], conv, stream, &slot);
+        if (st != FP8_OK) return st;   // argument errors surface before anything of the group is launched
+        const int64_t tiles = (int64_t)gg.p[i].tiles_m * gg.p[i].tiles_n + gg.first_tile[i];
+        if (tiles > 0x7FFFFFFF) return FP8_ERR_SHAPE;
+        gg.first_tile[i + 1] = (int)tiles;
+    }
+    const int total = gg.first_tile[count];
+    const int pairs = total < g_max_pairs ? total : g_max_pairs;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2u * (unsigned)pairs);
+    cfg.blockDim = dim3(kGemmThreads);
+    cfg.dynamicSmemBytes = wide ? PairSmemWide::kDynamic : PairSmem::kDynamic;
+    cfg.stream = (cudaStream_t)stream;
+    cfg.attrs = attr;
+    cfg.numAttrs = g_no_pdl ? 0 : 1;
+    count_launch();
+    const cudaError_t le = wide ? cudaLaunchKernelEx(&cfg, gemm_pair_group_kernel<2>, gg)
+                                : cudaLaunchKernelEx(&cfg, gemm_pair_group_kernel<1>, gg);
+    if (le != cudaSuccess) return FP8_ERR_CUDA;
+    return cudaGetLastError() == cudaSuccess ? FP8_OK : FP8_ERR_CUDA;
 }
 
 }  // extern "C"

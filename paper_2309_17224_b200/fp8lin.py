@@ -33,7 +33,7 @@ SYMBOLS = (
     "fp8_create", "fp8_destroy", "fp8_status_string", "fp8_device_flags", "fp8_amax", "fp8_scaling_bias",
     "fp8_scaling_bias_host", "fp8_cast_e4", "fp8_cast_e5", "fp8_ptq_weights", "fp8_linear_fwd", "fp8_linear_dgrad",
     "fp8_linear_wgrad", "fp8_amax_noalloc", "fp8_linear_fwd_act", "fp8_cast_predicted", "fp8_prediction_stats",
-    "fp8_linear_dgrad_act", "fp8_selftest_wait_expiry", "fp8_range_stats", "fp8_linear_fwd_q", "fp8_linear_dgrad_q", "fp8_amax_history_bias", "fp8_launch_count", "fp8_cast_group", "fp8_selftest_mma_ceiling", "fp8_bias_log_append", "fp8_bias_mode", "fp8_linear_f16acc", "fp8_linear_infer", "fp8_linear_infer_cast",
+    "fp8_linear_dgrad_act", "fp8_selftest_wait_expiry", "fp8_range_stats", "fp8_linear_fwd_q", "fp8_linear_dgrad_q", "fp8_amax_history_bias", "fp8_launch_count", "fp8_cast_group", "fp8_selftest_mma_ceiling", "fp8_bias_log_append", "fp8_bias_mode", "fp8_linear_f16acc", "fp8_linear_infer", "fp8_linear_infer_cast", "fp8_linear_group",
 )
 
 if not os.path.exists(LIB_PATH):
@@ -87,6 +87,16 @@ class GroupItem(ctypes.Structure):
 
 
 _lib.fp8_cast_group.argtypes = [_P, POINTER(GroupItem), c_int32, c_int, c_int32, _P]
+
+
+class MatmulItem(ctypes.Structure):
+    """``fp8_matmul_item_t``."""
+    _fields_ = [("kind", c_int32), ("bias_dt", c_int32), ("a8", c_void_p), ("d_ba", c_void_p), ("b8", c_void_p),
+                ("d_bb", c_void_p), ("bias_vec", c_void_p), ("out", c_void_p), ("d_amax_out", c_void_p),
+                ("out_dt", c_int32), ("reserved", c_int32), ("T", c_int64), ("K", c_int64), ("N", c_int64)]
+
+
+_lib.fp8_linear_group.argtypes = [_P, POINTER(MatmulItem), c_int32, c_int, _P]
 for _name in SYMBOLS:
     if _name != "fp8_status_string":
         getattr(_lib, _name).restype = c_int
@@ -157,6 +167,33 @@ def group_items(tensors):
         it.fmt, it.margin = fmt, (t[5] if len(t) > 5 else 0)
         it.d_amax = d_amax.data_ptr() if d_amax is not None else None
         it.d_bias, it.y = d_bias.data_ptr(), (y.data_ptr() if y is not None else None)
+    return arr
+
+
+MATMUL_FWD, MATMUL_DGRAD, MATMUL_WGRAD = 0, 1, 2
+
+
+def matmul_items(matmuls):
+    """A ctypes array of ``fp8_matmul_item_t`` from (kind, a8, d_ba, b8, d_bb, out[, bias_vec[, d_amax_out]]) tuples
+    (row-major operands: FWD x8, w8 -> y; DGRAD dy8, w8 -> dx; WGRAD dy8, x8 -> dw); build it once and hand it to
+    ``Context.linear_group`` every step (the tensors must stay alive)."""
+    arr = (MatmulItem * len(matmuls))()
+    for it, m in zip(arr, matmuls):
+        kind, a8, d_ba, b8, d_bb, out = m[:6]
+        bias_vec = m[6] if len(m) > 6 else None
+        d_amax_out = m[7] if len(m) > 7 else None
+        if kind == MATMUL_FWD:
+            (T, K), N = a8.shape, b8.shape[0]
+        elif kind == MATMUL_DGRAD:
+            (T, N), K = a8.shape, b8.shape[1]
+        else:
+            (T, N), K = a8.shape, b8.shape[1]
+        it.kind, it.T, it.K, it.N = kind, T, K, N
+        it.a8, it.d_ba, it.b8, it.d_bb = a8.data_ptr(), d_ba.data_ptr(), b8.data_ptr(), d_bb.data_ptr()
+        it.bias_vec = bias_vec.data_ptr() if bias_vec is not None else None
+        it.bias_dt = _DT[bias_vec.dtype] if bias_vec is not None else BF16
+        it.out, it.out_dt = out.data_ptr(), _DT[out.dtype]
+        it.d_amax_out = d_amax_out.data_ptr() if d_amax_out is not None else None
     return arr
 
 
@@ -301,6 +338,12 @@ class Context:
         _check(_lib.fp8_linear_infer_cast(self._h, _ptr(x), _DT[x.dtype], margin, _ptr(d_amax_x), _ptr(d_bx), _ptr(x8),
                                           _ptr(w8), _ptr(d_bw), _ptr(bias_vec), bias_dt, _ptr(y), _DT[y.dtype],
                                           _ptr(d_amax_y), T, K, N, conv, _stream()), "fp8_linear_infer_cast")
+
+    def linear_group(self, items, conv=CONV_PAPER):
+        """``fp8_linear_group``: independent matmuls in one launch.  `items`: a ``matmul_items(...)`` array or the list
+        of tuples it is built from."""
+        arr = items if isinstance(items, ctypes.Array) else matmul_items(items)
+        _check(_lib.fp8_linear_group(self._h, arr, len(arr), conv, _stream()), "fp8_linear_group")
 
     def linear_fwd_act(self, x8, d_bx, w8, d_bw, y_pre, y_act, bias_vec=None, d_amax_act=None, act=ACT_GELU,
                        conv=CONV_PAPER):

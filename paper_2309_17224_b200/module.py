@@ -95,13 +95,20 @@ class _Fp8LinearFn(torch.autograd.Function):
         dx = dw = db = None
         if fn.needs_input_grad[0]:
             dx = torch.empty((T, K), dtype=_out_dtype(dy.dtype), device=dy2.device)
-            lib.linear_dgrad(g8, bg, w8, None, b_fwd[_W:_W + 1], dx, conv=layer.conv)
-            dx = dx.reshape(fn.x_shape)
         if fn.needs_input_grad[1]:
             dw = torch.empty((N, K), dtype=_out_dtype(layer.weight.dtype), device=dy2.device)
+        if dx is not None and dw is not None:
+            # the two backward matmuls share dY8 and do not depend on each other (Section 2.2): one launch
+            lib.linear_group([(fp8lin.MATMUL_DGRAD, g8, bg, w8, b_fwd[_W:_W + 1], dx),
+                              (fp8lin.MATMUL_WGRAD, g8, bg, x8, b_fwd[_X:_X + 1], dw)], conv=layer.conv)
+        elif dx is not None:
+            lib.linear_dgrad(g8, bg, w8, None, b_fwd[_W:_W + 1], dx, conv=layer.conv)
+        elif dw is not None:
             lib.linear_wgrad(g8, None, bg, x8, None, b_fwd[_X:_X + 1], dw, T, conv=layer.conv)
-            if dw.dtype != layer.weight.dtype:
-                dw = dw.to(layer.weight.dtype)
+        if dx is not None:
+            dx = dx.reshape(fn.x_shape)
+        if dw is not None and dw.dtype != layer.weight.dtype:
+            dw = dw.to(layer.weight.dtype)
         if fn.has_bias and fn.needs_input_grad[2]:
             db = dy2.sum(0, dtype=torch.float32).to(layer.bias.dtype)   # not part of the paper's layer
         return dx, dw, db, None

@@ -146,6 +146,35 @@ def test_ragged_last_columns_survive_a_busy_gpu(ctx, lib):
     assert ctx.device_flags(clear=True) & lib.FLAG_TIMEOUT == 0
 
 
+@pytest.mark.parametrize("dt", [torch.float32, torch.bfloat16])
+def test_group_members_whose_rows_are_not_16_byte_multiples(ctx, lib, dt):
+    """Outputs with N = 300 or 1030 columns cannot leave through TMA stores (rows are not multiples of 16 bytes): such
+    members store from registers, inside the same launch as members that do use TMA stores."""
+    members = []
+    for i, (T, K, N) in enumerate([(256, 272, 300), (400, 1040, 1030), (384, 512, 768)]):
+        x = I.normal_bf16(T, K, 1.0, 600 + i, 1, "cuda")
+        w = I.normal_bf16(N, K, 0.02, 600 + i, 2, "cuda")
+        bias = torch.zeros(2, dtype=torch.int32, device="cuda")
+        amax = torch.zeros(2, dtype=torch.float32, device="cuda")
+        x8, w8 = torch.empty((T, K), dtype=torch.uint8, device="cuda"), torch.empty((N, K), dtype=torch.uint8, device="cuda")
+        ctx.cast_e4(x, None, d_amax_out=amax[0:1], d_bias_out=bias[0:1], y=x8)
+        ctx.cast_e4(w, None, d_amax_out=amax[1:2], d_bias_out=bias[1:2], y=w8)
+        _, bx, rx = O.quantise(bits_of(x), O.E4)
+        _, bw, rw = O.quantise(bits_of(w), O.E4)
+        y = torch.full((T, N), float("nan"), dtype=dt, device="cuda")
+        members.append((x8, w8, bias, y, O.linear_fwd(rx, bx + 1, rw, bw + 1)))
+    n0 = lib.launch_count()
+    ctx.linear_group([(lib.MATMUL_FWD, x8, b[0:1], w8, b[1:2], y) for x8, w8, b, y, _ in members])
+    assert lib.launch_count() - n0 == 1
+    torch.cuda.synchronize()
+    for _, _, _, y, ref in members:
+        if dt == torch.float32:
+            assert_gemm_close(y.cpu().numpy(), ref)
+        else:
+            assert_bf16_within_one_ulp(bits_of(y), ref)
+    assert ctx.device_flags(clear=True) & lib.FLAG_TIMEOUT == 0
+
+
 def test_group_with_a_decode_size_member_runs_the_members_own_calls(ctx, lib):
     big, small = Layer(ctx, 512, 1024, 768, 200), Layer(ctx, 16, 2048, 1280, 201)
     ob, os_ = big.outputs(torch.bfloat16), small.outputs(torch.bfloat16)

@@ -951,7 +951,7 @@ def main():
                          "run, tensor-pipe ceiling, fused MLP, other workloads")
     ap.add_argument("--no-ceiling-leg", action="store_true", help="skip the tensor-pipe ceiling measurement")
     ap.add_argument("--sustain-seconds", type=float, default=3.0)
-    ap.add_argument("--e2e-steps", type=int, default=5)
+    ap.add_argument("--e2e-steps", type=int, default=20)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--leg", default="step", choices=["step", "gemm", "cast", "stack", "mlp", "group"])
     ap.add_argument("--shapes", nargs="*", default=[])

@@ -1039,8 +1039,11 @@ def main():
     weight_bytes = float(sum(l.K * l.N for l in wl.layers))
     sm_count = torch.cuda.get_device_properties(local).multi_processor_count
     if decode:
-        roofline = {"bound": "hbm", "kernel": "decode_kernel (activation quantised in the same launch)" if fused_decode(layers[0])
-                    else "decode_kernel (+ splitk_finalize_kernel)",
+        # fp8_linear_infer_cast quantises an activation of at most 64 KB inside the matmul launch, larger ones by a cast launch
+        in_launch = fused_decode(layers[0]) and all(L.T * L.K * 2 <= (64 << 10) for L in layers)
+        roofline = {"bound": "hbm", "kernel": "decode_kernel (activation quantised in the same launch)" if in_launch
+                    else "decode_kernel (+ splitk_finalize_kernel where the contraction is split through the workspace; the "
+                         "activation's cast is a launch of its own)",
                     "achieved": sampled_steps * weight_bytes / (gemm_ms * 1e-3) / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                     "peak_source": f"{peaks['source']} copy bandwidth", "launches": gemm_launches,
                     "avg_launch_ms": gemm_ms / max(1, gemm_launches),

@@ -58,9 +58,19 @@ class _Fp8LinearFn(torch.autograd.Function):
         T = x2.shape[0]
         dev = x2.device
         x8 = torch.empty((T, K), dtype=torch.uint8, device=dev)
-        w8, w8_is_old = layer._quantised_weight(weight)
         y = torch.empty((T, N), dtype=layer.out_dtype or _out_dtype(x.dtype), device=dev)
         am, bi = layer.amax, layer.bias_words
+        if layer.training and layer.scaling != "constant" and T > 128:
+            # training: W and X are quantised together, all passes of both tensors in two launches (fp8_cast_group)
+            w8 = torch.empty((N, K), dtype=torch.uint8, device=dev)
+            lib.cast_group([(fp8lin.E4, weight.detach(), am[_W:_W + 1], bi[_W:_W + 1], w8),
+                            (fp8lin.E4, x2, am[_X:_X + 1], bi[_X:_X + 1], x8)], conv=layer.conv,
+                           predicted=layer.scaling == "predicted")
+            lib.linear_fwd(x8, bi[_X:_X + 1], w8, bi[_W:_W + 1], y, bias_vec=bias_vec, conv=layer.conv)
+            fn.layer, fn.x_shape, fn.has_bias = layer, x.shape, bias_vec is not None
+            fn.save_for_backward(x8, w8, bi[:2].clone())
+            return y.reshape(*x.shape[:-1], N)
+        w8, w8_is_old = layer._quantised_weight(weight)
         # the inference calls may read the weight's bytes early: only once those were written by an earlier forward pass
         frozen = (not layer.training) and w8_is_old
         if frozen and layer.scaling != "constant" and T <= 128:

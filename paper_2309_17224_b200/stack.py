@@ -225,9 +225,11 @@ class Fp8StackHistory(Fp8Stack):
         # the input of the first layer is the one activation no matmul produces: one pass, predicted bias
         c.cast_e4(x, self.pred[0, 1:2], margin=self.margin, d_amax_out=self.amax[0, 1:2],
                   d_bias_out=self.bias[0, 1:2], y=self.x8[0])
+        # all weights were updated by the step before: one grouped call quantises them (FP8-AMAX, just in time)
+        w16s = [w.to(torch.bfloat16) for w in self.w32]
+        c.cast_group([(fp8lin_E4, w16s[l], self.amax[l, 0:1], self.bias[l, 0:1], self.w8[l]) for l in range(L)])
         for l in range(L):
-            w16 = self.w32[l].to(torch.bfloat16)
-            c.cast_e4(w16, None, d_amax_out=self.amax[l, 0:1], d_bias_out=self.bias[l, 0:1], y=self.w8[l])
+            w16 = w16s[l]
             if l + 1 < L:
                 c.linear_fwd_q(self.x8[l], self.pred[l, 1:2], self.w8[l], self.bias[l, 0:1], self.x8[l + 1],
                                self.pred[l + 1, 1:2], y_pre=self.y[l], d_amax_z=self.amax[l + 1, 1:2], act=ACT_GELU)

@@ -377,7 +377,8 @@ FP8_API fp8_status_t fp8_linear_infer_cast(fp8_ctx *ctx, const void *x, fp8_dtyp
  * With at most 16 items, all of more than 128 output rows, one persistent kernel walks the output tiles of all
  * items in one sequence (shortest contractions first), so the launch pays one ramp and one drain and the last wave
  * of one matmul is filled with the first tiles of the next; any other group runs as its members' own calls, in
- * order.  Argument errors of any member are returned before anything of a one-launch group is enqueued. */
+ * order.  Argument errors of any member of a one-launch group are returned before the launch (the d_amax_out words
+ * of members listed before the faulty one may already have been cleared). */
 typedef enum { FP8_MATMUL_FWD = 0, FP8_MATMUL_DGRAD = 1, FP8_MATMUL_WGRAD = 2 } fp8_matmul_kind_t;
 typedef struct {
     int32_t kind;            /* fp8_matmul_kind_t */

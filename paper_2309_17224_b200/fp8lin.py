@@ -34,6 +34,7 @@ SYMBOLS = (
     "fp8_scaling_bias_host", "fp8_cast_e4", "fp8_cast_e5", "fp8_ptq_weights", "fp8_linear_fwd", "fp8_linear_dgrad",
     "fp8_linear_wgrad", "fp8_amax_noalloc", "fp8_linear_fwd_act", "fp8_cast_predicted", "fp8_prediction_stats",
     "fp8_linear_dgrad_act", "fp8_selftest_wait_expiry", "fp8_range_stats", "fp8_linear_fwd_q", "fp8_linear_dgrad_q", "fp8_amax_history_bias", "fp8_launch_count", "fp8_cast_group", "fp8_selftest_mma_ceiling", "fp8_bias_log_append", "fp8_bias_mode", "fp8_linear_f16acc", "fp8_linear_infer", "fp8_linear_infer_cast", "fp8_linear_group",
+    "fp8h_gelu", "fp8h_gelu_backward", "fp8h_mse_grad", "fp8h_sgd",
 )
 
 if not os.path.exists(LIB_PATH):
@@ -97,6 +98,10 @@ class MatmulItem(ctypes.Structure):
 
 
 _lib.fp8_linear_group.argtypes = [_P, POINTER(MatmulItem), c_int32, c_int, _P]
+_lib.fp8h_gelu.argtypes = [_P, _P, c_int64, _P]
+_lib.fp8h_gelu_backward.argtypes = [_P, _P, _P, c_int64, _P]
+_lib.fp8h_mse_grad.argtypes = [_P, _P, ctypes.c_float, _P, c_int64, _P]
+_lib.fp8h_sgd.argtypes = [_P, _P, ctypes.c_float, _P, c_int64, _P]
 for _name in SYMBOLS:
     if _name != "fp8_status_string":
         getattr(_lib, _name).restype = c_int
@@ -195,6 +200,30 @@ def matmul_items(matmuls):
         it.out, it.out_dt = out.data_ptr(), _DT[out.dtype]
         it.d_amax_out = d_amax_out.data_ptr() if d_amax_out is not None else None
     return arr
+
+
+# -- element-wise kernels of the stress stack (include/fp8_harness.h): harness, not the paper's method -----------------
+def _bf16(t):
+    assert t.dtype == torch.bfloat16 and t.is_contiguous() and t.is_cuda, "contiguous bf16 CUDA tensor expected"
+    return t
+
+
+def harness_gelu(x, y):
+    _check(_lib.fp8h_gelu(_ptr(_bf16(x)), _ptr(_bf16(y)), x.numel(), _stream()), "fp8h_gelu")
+
+
+def harness_gelu_backward(g, pre, out):
+    _check(_lib.fp8h_gelu_backward(_ptr(_bf16(g)), _ptr(_bf16(pre)), _ptr(_bf16(out)), g.numel(), _stream()), "fp8h_gelu_backward")
+
+
+def harness_mse_grad(y, target, scale, g):
+    _check(_lib.fp8h_mse_grad(_ptr(_bf16(y)), _ptr(_bf16(target)), float(scale), _ptr(_bf16(g)), y.numel(), _stream()),
+           "fp8h_mse_grad")
+
+
+def harness_sgd(w32, dw, lr, w16):
+    assert w32.dtype == torch.float32 and w32.is_contiguous()
+    _check(_lib.fp8h_sgd(_ptr(w32), _ptr(_bf16(dw)), float(lr), _ptr(_bf16(w16)), w32.numel(), _stream()), "fp8h_sgd")
 
 
 class Context:

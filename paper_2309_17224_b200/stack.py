@@ -5,10 +5,13 @@ plain SGD on FP32 master weights.  Every step re-quantises every weight,
 activation and gradient tensor with a fresh FP8-AMAX bias, and the input scale
 drifts as 2^(8 sin(step / 20)) so that the biases have to move.
 
-Only the linears belong to the paper's method and run in the library
-(``fp8_cast_e4/e5``, ``fp8_linear_fwd/dgrad/wgrad``); the glue around them
-(GELU and its derivative, the loss gradient, the SGD update) is ordinary FP32
-torch arithmetic rounded to bf16, outside the measured path.
+Only the linears belong to the paper's method (``fp8_cast_e4/e5``,
+``fp8_linear_fwd/dgrad/wgrad``); the glue around them (GELU and its
+derivative, the loss gradient, the SGD update) is FP32 arithmetic rounded to
+bf16, run by the library's harness kernels (``fp8h_*``, include/fp8_harness.h)
+so that a step launches no framework kernels beyond its input and its loss.
+``gelu_bf16`` / ``gelu_grad_f32`` below are the same formulas in torch, kept
+for comparisons.
 """
 from __future__ import annotations
 
@@ -17,6 +20,7 @@ from typing import Dict, List
 
 import torch
 
+from . import fp8lin as _lib
 from . import inputs as I
 
 CONFIG_ID = 5
@@ -70,6 +74,9 @@ class Fp8Stack:
         self.g8t = torch.empty((d, tokens), **u8)
         self.dx = torch.empty((tokens, d), dtype=torch.bfloat16, **dev)
         self.dw = torch.empty((d, d), dtype=torch.bfloat16, **dev)
+        self.w16 = [w.to(torch.bfloat16) for w in self.w32]      # bf16(W32), rewritten by every SGD update
+        self.h = [torch.empty((tokens, d), dtype=torch.bfloat16, **dev) for _ in range(2)]   # GELU outputs, in turn
+        self.g = [torch.empty((tokens, d), dtype=torch.bfloat16, **dev) for _ in range(2)]   # gradients, in turn
         # per layer: amax / bias of W, X, dY
         self.amax = torch.zeros((layers, 3), dtype=torch.float32, **dev)
         self.bias = torch.zeros((layers, 3), dtype=torch.int32, **dev)
@@ -92,7 +99,7 @@ class Fp8Stack:
         c = self.ctx
         have_amax = False   # the previous matmul's epilogue already produced amax(x)
         for l in range(self.L):
-            w16 = self.w32[l].to(torch.bfloat16)
+            w16 = self.w16[l]
             c.cast_e4(w16, None, d_amax_out=self.amax[l, 0:1], d_bias_out=self.bias[l, 0:1], y=self.w8[l], y_t=self.w8t[l])
             if have_amax:
                 c.scaling_bias(self.amax[l, 1:2], fp8lin_E4, CONV_PAPER, 0, self.bias[l, 1:2])
@@ -108,13 +115,14 @@ class Fp8Stack:
                 self._keep(l, x=x, w=w16, x8=self.x8[l], w8=self.w8[l], y=self.y[l])
                 have_amax = False
                 if l + 1 < self.L:
-                    x = gelu_bf16(self.y[l])
+                    x = self.h[l % 2]
+                    _lib.harness_gelu(self.y[l], x)
         return self.y[self.L - 1]
 
     def backward_and_update(self) -> None:
         c = self.ctx
-        out = self.y[self.L - 1].to(torch.float32)
-        g = ((out - self.target.to(torch.float32)) * (2.0 / (self.T * self.d))).to(torch.bfloat16)
+        g = self.g[0]
+        _lib.harness_mse_grad(self.y[self.L - 1], self.target, 2.0 / (self.T * self.d), g)
         have_amax = False   # the previous input-gradient matmul already produced amax(g)
         for l in range(self.L - 1, -1, -1):
             if have_amax:
@@ -131,12 +139,13 @@ class Fp8Stack:
                 self._keep(l, dx=self.dx)
             c.linear_wgrad(None, self.g8t, self.bias[l, 2:3], None, self.x8t[l], self.bias[l, 1:2], self.dw, self.T)
             self._keep(l, g=g, g8=self.g8, dw=self.dw, amax=self.amax[l], bias=self.bias[l])
-            self.w32[l].add_(self.dw.to(torch.float32), alpha=-self.lr)
+            _lib.harness_sgd(self.w32[l], self.dw, self.lr, self.w16[l])
             if l > 0:
                 if self.fused:
                     g, have_amax = self.gact, True
                 else:
-                    g = (self.dx.to(torch.float32) * gelu_grad_f32(self.y[l - 1])).to(torch.bfloat16)
+                    g = self.g[l % 2]
+                    _lib.harness_gelu_backward(self.dx, self.y[l - 1], g)
 
     def step(self, step: int, snap_layers=()) -> Dict[str, object]:
         """One training step.  `snap_layers`: layers whose tensors (every input and output of the library calls of
@@ -226,7 +235,7 @@ class Fp8StackHistory(Fp8Stack):
         c.cast_e4(x, self.pred[0, 1:2], margin=self.margin, d_amax_out=self.amax[0, 1:2],
                   d_bias_out=self.bias[0, 1:2], y=self.x8[0])
         # all weights were updated by the step before: one grouped call quantises them (FP8-AMAX, just in time)
-        w16s = [w.to(torch.bfloat16) for w in self.w32]
+        w16s = self.w16
         c.cast_group([(fp8lin_E4, w16s[l], self.amax[l, 0:1], self.bias[l, 0:1], self.w8[l]) for l in range(L)])
         for l in range(L):
             w16 = w16s[l]
@@ -238,9 +247,9 @@ class Fp8StackHistory(Fp8Stack):
             self._keep(l, w=w16, x8=self.x8[l], w8=self.w8[l], y=self.y[l], bias_x=self.pred[l, 1:2],
                        bias_w=self.bias[l, 0:1], **({"x8_next": self.x8[l + 1], "bias_next": self.pred[l + 1, 1:2],
                                                      "amax_next": self.amax[l + 1, 1:2]} if l + 1 < L else {}))
-        out = self.y[L - 1].to(torch.float32)
-        loss = torch.mean((out - self.target.to(torch.float32)) ** 2)
-        g = ((out - self.target.to(torch.float32)) * (2.0 / (T * self.d))).to(torch.bfloat16)
+        loss = torch.mean((self.y[L - 1].to(torch.float32) - self.target.to(torch.float32)) ** 2)
+        g = self.g[0]
+        _lib.harness_mse_grad(self.y[L - 1], self.target, 2.0 / (T * self.d), g)
         bufs = (self.g8, self.g8b)
         c.cast_e5(g, self.pred[L - 1, 2:3], margin=self.margin, d_amax_out=self.amax[L - 1, 2:3],
                   d_bias_out=self.bias[L - 1, 2:3], y=bufs[(L - 1) % 2])
@@ -252,7 +261,7 @@ class Fp8StackHistory(Fp8Stack):
             c.linear_wgrad(cur, None, self.pred[l, 2:3], self.x8[l], None, self.pred[l, 1:2], self.dw, T)
             self._keep(l, g8=cur, bias_g=self.pred[l, 2:3], dw=self.dw,
                        **({"g8_next": nxt, "bias_g_next": self.pred[l - 1, 2:3], "y_below": self.y[l - 1]} if l > 0 else {}))
-            self.w32[l].add_(self.dw.to(torch.float32), alpha=-self.lr)
+            _lib.harness_sgd(self.w32[l], self.dw, self.lr, self.w16[l])
         used = self.bias.clone()
         used[:, 1:3] = self.pred[:, 1:3]
         rec = {"loss": loss, "bias": used, "amax": self.amax.clone()}

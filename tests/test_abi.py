@@ -22,9 +22,10 @@ def _lib():
 
 def test_library_exports_every_declared_symbol():
     fp8lin = _lib()
-    header = open(os.path.join(ROOT, "include", "fp8lin.h")).read()
+    import glob
+    header = "".join(open(h).read() for h in sorted(glob.glob(os.path.join(ROOT, "include", "*.h"))))
     header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
-    declared = set(re.findall(r"\b(fp8_[a-z0-9_]+)\s*\(", header))
+    declared = set(re.findall(r"\b(fp8h?_[a-z0-9_]+)\s*\(", header))
     assert declared, "no declarations found"
     lib = ctypes.CDLL(fp8lin.LIB_PATH)
     for name in sorted(declared):

@@ -3320,10 +3320,19 @@ fp8_status_t fp8_linear_group(fp8_ctx *ctx, const fp8_matmul_item_t *items, int3
     cfg.stream = (cudaStream_t)stream;
     cfg.attrs = attr;
     cfg.numAttrs = g_no_pdl ? 0 : 1;
-    count_launch();
     const cudaError_t le = wide ? cudaLaunchKernelEx(&cfg, gemm_pair_group_kernel<2>, gg)
                                 : cudaLaunchKernelEx(&cfg, gemm_pair_group_kernel<1>, gg);
-    if (le != cudaSuccess) return FP8_ERR_CUDA;
+    if (le != cudaSuccess) {
+        // the launch was refused (the 11 KB of kernel parameters need a driver that takes more than 4 KB): nothing
+        // has run, the members go out one by one
+        (void)cudaGetLastError();
+        for (int i = 0; i < count; ++i) {
+            const fp8_status_t st = group_item_call(ctx, items[i], conv, stream, nullptr);
+            if (st != FP8_OK) return st;
+        }
+        return FP8_OK;
+    }
+    count_launch();
     return cudaGetLastError() == cudaSuccess ? FP8_OK : FP8_ERR_CUDA;
 }
 
